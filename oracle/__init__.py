@@ -1,0 +1,155 @@
+"""MX+ CPU oracle: ctypes binding of ``mxp_oracle.c``.
+
+TEST INFRASTRUCTURE ONLY.  Importable from ``tests/``, the smoke check and the
+benchmark's CPU-baseline / reference legs.  The product package never imports it
+and it never imports the product package.
+
+The arithmetic lives in the C file (fp64, one block at a time, in the order the
+paper gives it: Sec. 2 Eq. 1, Sec. 4.1-4.2, Sec. 5 Eq. 3 / Eq. 4).  This module only
+marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+MODE_MXFP4 = 0
+MODE_MXFP4_PLUS = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mxp_oracle.c")
+_LIB = os.path.join(_HERE, "libmxp_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, -O2, OpenMP over rows)."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            subprocess.check_call(
+                ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                 "-fno-fast-math", "-ffp-contract=off", _SRC, "-o", tmp, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, p, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        lib.oracle_quantize.argtypes = [p, ci, i64, i64, i64, ci, ci, p, p, p]
+        lib.oracle_quantize.restype = ci
+        lib.oracle_dequantize.argtypes = [p, p, p, i64, i64, ci, ci, p, i64]
+        lib.oracle_dequantize.restype = ci
+        lib.oracle_gemm_fp64.argtypes = [p, i64, p, i64, i64, i64, i64, p, i64]
+        lib.oracle_gemm_fp64.restype = None
+        lib.oracle_e2m1_value.argtypes = [ci]
+        lib.oracle_e2m1_value.restype = ctypes.c_double
+        lib.oracle_bm_split.argtypes = [ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        lib.oracle_bm_split.restype = None
+        lib.oracle_set_threads.argtypes = [ci]
+        lib.oracle_max_threads.restype = ci
+        lib.oracle_get_threads.restype = ci
+        _lib = lib
+    return _lib
+
+
+def set_threads(n: int) -> None:
+    _load().oracle_set_threads(int(n))
+
+
+def get_threads() -> int:
+    return int(_load().oracle_get_threads())
+
+
+def max_threads() -> int:
+    return int(_load().oracle_max_threads())
+
+
+def e2m1_value(code: int) -> float:
+    return float(_load().oracle_e2m1_value(int(code)))
+
+
+def bm_split(m: int):
+    """Eq. 4: E2M1 magnitude codes of (BM_H, BM_L) for the 3-bit BM mantissa m."""
+    h, l = ctypes.c_int(), ctypes.c_int()
+    _load().oracle_bm_split(int(m), ctypes.byref(h), ctypes.byref(l))
+    return h.value, l.value
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def quantize(x: np.ndarray, mode: int, k: int = 32, bf16_bits: bool = False):
+    """Quantize a 2-D array along its rows in blocks of k.
+
+    x: float32, float64, or (bf16_bits=True) uint16 holding bfloat16 bit patterns.
+    Returns (nibbles[rows, cols/2], scales[rows, cols/k], bm_index[rows, cols/k]), uint8.
+    """
+    assert x.ndim == 2
+    x = np.ascontiguousarray(x)
+    if bf16_bits:
+        assert x.dtype == np.uint16
+        kind = 1
+    elif x.dtype == np.float32:
+        kind = 0
+    elif x.dtype == np.float64:
+        kind = 2
+    else:
+        raise TypeError(x.dtype)
+    rows, cols = x.shape
+    if cols % k or k % 2:
+        raise ValueError("cols must be a multiple of the (even) block length")
+    nib = np.zeros((rows, cols // 2), np.uint8)
+    sc = np.zeros((rows, cols // k), np.uint8)
+    idx = np.zeros((rows, cols // k), np.uint8)
+    rc = _load().oracle_quantize(_ptr(x), kind, rows, cols, cols, k, mode,
+                                 _ptr(nib), _ptr(sc), _ptr(idx))
+    if rc != 0:
+        raise ValueError("oracle_quantize rejected its arguments")
+    return nib, sc, idx
+
+
+def dequantize(nib: np.ndarray, sc: np.ndarray, idx, mode: int, k: int = 32) -> np.ndarray:
+    """Eq. 3 decode to float64, shape [rows, cols]."""
+    nib = np.ascontiguousarray(nib, np.uint8)
+    sc = np.ascontiguousarray(sc, np.uint8)
+    rows, half = nib.shape
+    cols = half * 2
+    if idx is None:
+        idx = np.zeros_like(sc)
+    idx = np.ascontiguousarray(idx, np.uint8)
+    assert sc.shape == (rows, cols // k) and idx.shape == sc.shape
+    out = np.empty((rows, cols), np.float64)
+    rc = _load().oracle_dequantize(_ptr(nib), _ptr(sc), _ptr(idx), rows, cols, k, mode,
+                                   _ptr(out), cols)
+    if rc != 0:
+        raise ValueError("oracle_dequantize rejected its arguments")
+    return out
+
+
+def gemm_fp64(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """D = A @ B.T in fp64 by a plain triple loop (A: M x K, B: N x K)."""
+    a = np.ascontiguousarray(a, np.float64)
+    b = np.ascontiguousarray(b, np.float64)
+    m, k = a.shape
+    n, k2 = b.shape
+    assert k == k2
+    d = np.empty((m, n), np.float64)
+    _load().oracle_gemm_fp64(_ptr(a), k, _ptr(b), k, m, n, k, _ptr(d), n)
+    return d
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bfloat16 bit patterns (uint16) to float64."""
+    u = bits.astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)

@@ -1,0 +1,274 @@
+/*
+ * MX+ CPU oracle -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, step-by-step restatement of the MXFP4 / MXFP4+ block format of
+ * "MX+: Pushing the Limits of Microscaling Formats for Efficient LLM Serving"
+ * (Sec. 2 Eq. 1, Sec. 4.1-4.2, Sec. 5 Eq. 3 and Eq. 4).  Only the tests, the smoke
+ * check and the benchmark's CPU-baseline leg may call it.  It shares no code,
+ * table or constant with the CUDA library and must never be reached from the
+ * product path.
+ *
+ * Arithmetic is done on doubles (every bf16 / fp32 input converts exactly).
+ *
+ * Pinned by tests (see tests/test_oracle_*.py): element table, scale, NBM and BM
+ * rounding, flush rule, layout, Eq. 4 split, decode, fp64 GEMM.
+ * Parity unpinned: blocks holding Inf/NaN (the paper does not define them).
+ *
+ * Readings of the paper taken here (each is listed in the design notes):
+ *   - rounding of the element cast: round to nearest, ties to the even code;
+ *   - a BM whose scaled value rounds up to 8 keeps the scale and clamps to 7.5;
+ *   - several equal maxima: the lowest index is the BM;
+ *   - the sign bit of the input is kept even when the magnitude rounds to zero;
+ *   - element 2j sits in the low nibble of byte j; three separate row-major planes;
+ *   - the flush rule and the reserved scale byte 0 apply in plain MXFP4 mode too.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_MODE_MXFP4 0
+#define ORACLE_MODE_MXFP4_PLUS 1
+
+/* Sec. 2: FP4 element = 1 sign, 2 exponent bits (bias 1), 1 mantissa bit,
+ * implicit leading one, IEEE-like subnormals; emax = 3 - 1 = 2. */
+#define EMAX 2
+#define EXP_BIAS 1
+
+static int g_threads = 1;
+
+void oracle_set_threads(int n) { g_threads = n < 1 ? 1 : n; }
+int oracle_get_threads(void) { return g_threads; }
+int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Value of a 3-bit E2M1 magnitude code, from the definition of the type. */
+double oracle_e2m1_value(int code)
+{
+    int e = (code >> 1) & 3;
+    int m = code & 1;
+    if (e == 0) /* subnormal: 2^(1-bias) * 0.m */
+        return ldexp((double)m * 0.5, 1 - EXP_BIAS);
+    return ldexp(1.0 + (double)m * 0.5, e - EXP_BIAS);
+}
+
+/* Nearest E2M1 magnitude to r >= 0.  Ties go to the even code.  Anything beyond
+ * the largest magnitude saturates to it (Sec. 4.3 example: 7.92 -> 6.0). */
+static int e2m1_nearest(double r)
+{
+    int best = 0;
+    double best_d = fabs(r - oracle_e2m1_value(0));
+    for (int c = 1; c < 8; ++c) {
+        double d = fabs(r - oracle_e2m1_value(c));
+        if (d < best_d || (d == best_d && (c & 1) == 0)) {
+            best = c;
+            best_d = d;
+        }
+    }
+    /* 7.0 is midway between 6 and the next binade value 8 (which has an even
+     * mantissa): it rounds to 8 and then saturates, i.e. still code 7. */
+    return best;
+}
+
+/* BM mantissa code in MX+ mode: v in [4, 8), grid 4 + m/2, m = 0..7 (E0M3 stored,
+ * E2M3 effective with the implied exponent emax).  Round to nearest, ties to even
+ * m; a value that would round up to 8 clamps to m = 7. */
+static int bm_code(double v)
+{
+    double t = (v - 4.0) * 2.0; /* in [0, 8) */
+    double fl = floor(t);
+    double frac = t - fl;
+    int m = (int)fl;
+    if (frac > 0.5 || (frac == 0.5 && (m & 1)))
+        m += 1;
+    if (m > 7)
+        m = 7;
+    return m;
+}
+
+/* floor(log2(a)) for finite a > 0, exact. */
+static int floor_log2(double a)
+{
+    int ex;
+    (void)frexp(a, &ex); /* a = f * 2^ex, f in [0.5, 1) */
+    return ex - 1;
+}
+
+/*
+ * One block of k elements (k even, k <= 32; the format uses k = 32).
+ * Outputs: k/2 nibble bytes, one scale byte, one index byte.
+ */
+static void quantize_block(const double *x, int k, int mode, uint8_t *nib,
+                           uint8_t *scale, uint8_t *index)
+{
+    /* Sec. 3.2: BM = the absolute maximum of the block; first one wins. */
+    double amax = 0.0;
+    int bm = 0;
+    int nonfinite = 0;
+    for (int i = 0; i < k; ++i) {
+        double a = fabs(x[i]);
+        if (!(a <= 1.79769313486231570815e+308))
+            nonfinite = 1;
+        if (a > amax) {
+            amax = a;
+            bm = i;
+        }
+    }
+    memset(nib, 0, (size_t)k / 2);
+    if (nonfinite) { /* not defined by the paper: E8M0 NaN byte, data zero */
+        *scale = 0xFF;
+        *index = 0;
+        return;
+    }
+    /* Sec. 4.1 flush rule: floor(log2 BM) <= -127 + emax -> whole block is zero,
+     * signalled by the reserved biased scale 0. */
+    if (amax == 0.0 || floor_log2(amax) <= -127 + EMAX) {
+        *scale = 0;
+        *index = 0;
+        return;
+    }
+    /* Eq. 1: shared_exp = max floor(log2|x|) - emax; E8M0 bias 127. */
+    int se = floor_log2(amax) - EMAX;
+    *scale = (uint8_t)(se + 127);
+    *index = (uint8_t)(mode == ORACLE_MODE_MXFP4_PLUS ? bm : 0);
+    for (int i = 0; i < k; ++i) {
+        double r = ldexp(fabs(x[i]), -se); /* exact */
+        int code;
+        if (mode == ORACLE_MODE_MXFP4_PLUS && i == bm)
+            code = bm_code(r); /* Sec. 4.1: exponent bits reused as mantissa */
+        else
+            code = e2m1_nearest(r);
+        int sign = signbit(x[i]) ? 1 : 0;
+        uint8_t n = (uint8_t)((sign << 3) | code);
+        if (i & 1)
+            nib[i / 2] |= (uint8_t)(n << 4);
+        else
+            nib[i / 2] |= n;
+    }
+}
+
+static double bf16_to_double(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+/*
+ * src_kind: 0 = float32, 1 = bfloat16 bit patterns (uint16), 2 = float64.
+ * Planes: nibbles rows*cols/2, scales rows*cols/k, bm_index rows*cols/k (written
+ * in both modes; all zero in MXFP4 mode).  Returns 0, or -1 on a bad argument.
+ */
+int oracle_quantize(const void *src, int src_kind, int64_t rows, int64_t cols,
+                    int64_t ld_src, int k, int mode, uint8_t *nibbles,
+                    uint8_t *scales, uint8_t *bm_index)
+{
+    if (k < 2 || k > 32 || (k & 1) || cols % k != 0 || rows < 0 || cols < 0)
+        return -1;
+    if (mode != ORACLE_MODE_MXFP4 && mode != ORACLE_MODE_MXFP4_PLUS)
+        return -1;
+    int64_t bpr = cols / k;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+#endif
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < bpr; ++b) {
+            double x[32];
+            for (int i = 0; i < k; ++i) {
+                int64_t off = r * ld_src + b * k + i;
+                if (src_kind == 0)
+                    x[i] = (double)((const float *)src)[off];
+                else if (src_kind == 1)
+                    x[i] = bf16_to_double(((const uint16_t *)src)[off]);
+                else
+                    x[i] = ((const double *)src)[off];
+            }
+            quantize_block(x, k, mode, nibbles + (r * cols + b * k) / 2,
+                           scales + r * bpr + b, bm_index + r * bpr + b);
+        }
+    }
+    return 0;
+}
+
+/* Eq. 3.  Scale byte 0 -> zeros (reserved encoding); 0xFF -> NaN (unpinned). */
+int oracle_dequantize(const uint8_t *nibbles, const uint8_t *scales,
+                      const uint8_t *bm_index, int64_t rows, int64_t cols, int k,
+                      int mode, double *dst, int64_t ld_dst)
+{
+    if (k < 2 || k > 32 || (k & 1) || cols % k != 0)
+        return -1;
+    int64_t bpr = cols / k;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+#endif
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < bpr; ++b) {
+            int sb = scales[r * bpr + b];
+            int bm = (mode == ORACLE_MODE_MXFP4_PLUS) ? (bm_index[r * bpr + b] & 31) : -1;
+            for (int i = 0; i < k; ++i) {
+                uint8_t byte = nibbles[(r * cols + b * k + i) / 2];
+                int n = (i & 1) ? (byte >> 4) : (byte & 15);
+                int s = n >> 3;
+                int code = n & 7;
+                double out;
+                if (sb == 0) {
+                    out = 0.0;
+                } else if (sb == 0xFF) {
+                    out = NAN;
+                } else {
+                    double E;
+                    if (i == bm) /* "MX+ addition": 2^emax * 1.mmm */
+                        E = ldexp(1.0 + (double)code / 8.0, EMAX);
+                    else
+                        E = oracle_e2m1_value(code);
+                    out = ldexp(E, sb - 127);
+                    if (s)
+                        out = -out;
+                }
+                dst[r * ld_dst + b * k + i] = out;
+            }
+        }
+    }
+    return 0;
+}
+
+/* Eq. 4: BM = BM_H + BM_L on the scaled grid, um[3:0] = 1 m2 m1 m0.
+ *   BM_H = 2^emax * um[3:2]     -> 4 or 6      (E2M1 magnitude codes 6, 7)
+ *   BM_L = 2^(emax-2) * um[1:0] -> 0 .. 1.5    (E2M1 magnitude codes 0 .. 3)
+ * Returns the two E2M1 magnitude codes. */
+void oracle_bm_split(int m, int *code_h, int *code_l)
+{
+    int m2 = (m >> 2) & 1, m1 = (m >> 1) & 1, m0 = m & 1;
+    /* um[3:2] read as the fixed-point number 1.m2; um[1:0] as m1.m0 */
+    double h = ldexp(1.0 + (double)m2 * 0.5, EMAX);
+    double l = ldexp((double)m1 + (double)m0 * 0.5, EMAX - 2);
+    *code_h = e2m1_nearest(h);
+    *code_l = e2m1_nearest(l);
+}
+
+/* D[m][n] = sum_k A[m][k] * B[n][k], fp64, k ascending.  A is M x K, B is N x K. */
+void oracle_gemm_fp64(const double *A, int64_t lda, const double *B, int64_t ldb,
+                      int64_t M, int64_t N, int64_t K, double *D, int64_t ldd)
+{
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+#endif
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t kk = 0; kk < K; ++kk)
+                acc += A[m * lda + kk] * B[n * ldb + kk];
+            D[m * ldd + n] = acc;
+        }
+    }
+}
