@@ -1,0 +1,137 @@
+/*
+ * mxp.h -- C ABI of libmxp: MXFP4 / MXFP4+ ("MX+") block quantization, decode and
+ * GEMM on NVIDIA B200 (sm_100a).
+ *
+ * Format (paper Sec. 2 Eq. 1, Sec. 4.1, Sec. 4.2):
+ *   - a block is 32 consecutive elements of a row; every block has one E8M0 scale byte
+ *     (biased by 127) holding shared_exp = floor(log2 BM) - 2, BM = the block's absolute
+ *     maximum (first one if several are equal);
+ *   - elements are 4-bit E2M1 codes (sign, 2 exponent bits with bias 1, 1 mantissa bit),
+ *     element 2j in the low nibble of byte j, rounded to nearest with ties to the even
+ *     code and saturating at 6;
+ *   - in MXFP4+ mode the BM element stores 3 mantissa bits instead (E0M3, value
+ *     4 + m/2 on the scaled grid, exponent implied) and a per-block index byte holds its
+ *     position in bits 4:0 (bits 7:5 are written 0 and ignored on read);
+ *   - a block whose BM has floor(log2 BM) <= -125 is flushed: scale byte 0, all-zero
+ *     nibbles, index 0; scale byte 0 decodes to 32 zeros in both modes;
+ *   - a block holding Inf/NaN gets scale byte 0xFF and zero data (not defined by the
+ *     paper; decodes to NaN).
+ *
+ * Conventions for every entry point:
+ *   - every data pointer is caller-owned DEVICE memory unless stated otherwise; the
+ *     library never allocates, frees or keeps it;
+ *   - matrices are row-major; blocks run along the contiguous dimension (cols = K), so
+ *     the GEMM's B operand is passed as N x K ("weights as [out, in]");
+ *   - `cuda_stream` is a cudaStream_t (NULL = the legacy default stream); work is
+ *     enqueued on it and the call returns without synchronising;
+ *   - errors are return codes; nothing is launched when a call returns
+ *     MXP_ERR_INVALID_ARG / MXP_ERR_UNSUPPORTED / MXP_ERR_WORKSPACE.
+ */
+#ifndef MXP_H_
+#define MXP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MXP_OK = 0,
+    MXP_ERR_INVALID_ARG = 1, /* null / misaligned pointer, bad size, bad enum */
+    MXP_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for */
+    MXP_ERR_WORKSPACE = 3,   /* workspace missing or too small */
+    MXP_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
+    MXP_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see mxp_gemm_status) */
+} mxp_status;
+
+typedef enum { MXP_MODE_MXFP4 = 0, MXP_MODE_MXFP4_PLUS = 1 } mxp_mode;
+typedef enum { MXP_F32 = 0, MXP_BF16 = 1 } mxp_dtype;
+
+/* A packed operand: three row-major device planes. */
+typedef struct {
+    const uint8_t *nibbles;  /* rows * cols / 2 bytes, 16-byte aligned                */
+    const uint8_t *scales;   /* rows * cols / 32 bytes, E8M0                          */
+    const uint8_t *bm_index; /* rows * cols / 32 bytes; may be NULL iff mode == MXFP4 */
+    int64_t rows, cols;      /* cols % 32 == 0                                        */
+    mxp_mode mode;
+} mxp_packed;
+
+/*
+ * Quantize (Eq. 1 shared scale; Sec. 4.1 BM re-encoding and flush rule; Sec. 4.2 layout).
+ *   src      rows x cols elements of `src_dt`, row stride `ld_src` elements
+ *            (ld_src >= cols, ld_src % 8 == 0, 16-byte aligned base)
+ *   nibbles  out, rows * cols / 2 bytes (16-byte aligned)
+ *   scales   out, rows * cols / 32 bytes
+ *   bm_index out, rows * cols / 32 bytes; required for MXFP4+, may be NULL for MXFP4
+ *            (when given in MXFP4 mode it is filled with zeros)
+ * cols must be a multiple of 32.  rows == 0 or cols == 0 is a no-op returning MXP_OK.
+ */
+mxp_status mxp_quantize(const void *src, mxp_dtype src_dt, int64_t rows, int64_t cols,
+                        int64_t ld_src, mxp_mode mode, uint8_t *nibbles, uint8_t *scales,
+                        uint8_t *bm_index, void *cuda_stream);
+
+/*
+ * Decode (Eq. 3): dst[r][c] = (-1)^s * 2^(scale - 127) * E, E = 4 + m/2 for the BM
+ * element of an MXFP4+ block, the E2M1 value otherwise.  Exact in both output types.
+ *   p       host pointer to the operand descriptor (its planes are device memory)
+ *   dst     rows x cols of `dst_dt`, row stride `ld_dst` elements (ld_dst % 8 == 0,
+ *           16-byte aligned base)
+ */
+mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int64_t ld_dst,
+                          void *cuda_stream);
+
+/*
+ * GEMM on MX / MX+ operands (problem statement of Sec. 5; Eq. 3 for the weight-only
+ * form; Eq. 4 / Algorithm 1 for the direct form):
+ *     D[M,N] = dec(A)[M,K] * dec(B)[N,K]^T, fp32 accumulation.
+ * Exactly one of A_dense_bf16 / A_packed is non-NULL:
+ *   - A_dense_bf16 (device, bf16, row stride lda elements): weight-only form, the
+ *     weights B are decoded inside the kernel and multiplied with bf16 activations;
+ *   - A_packed (host pointer to a descriptor): both operands are consumed by the
+ *     block-scaled tensor-core path; any combination of MXFP4 / MXFP4+ modes.
+ *   B_packed   host pointer to the descriptor of the N x K weight operand
+ *   D          M x N of `d_dt` (bf16 rounded to nearest even, or fp32), row stride ldd
+ *   workspace  device scratch of at least mxp_gemm_workspace_bytes(...) bytes, 256-byte
+ *              aligned; may be NULL when that size is 0.  Its first 16 bytes are a status
+ *              block written by the kernels (see mxp_gemm_status).
+ * K % 32 == 0 always; the tensor-core form further needs K % 128 == 0.
+ */
+mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16, int64_t lda,
+                    const mxp_packed *A_packed, const mxp_packed *B_packed, void *D,
+                    mxp_dtype d_dt, int64_t ldd, void *workspace, size_t workspace_bytes,
+                    void *cuda_stream);
+
+/* Bytes of workspace mxp_gemm needs for this problem. a_dense != 0: weight-only form. */
+size_t mxp_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense,
+                                mxp_mode a_mode, mxp_mode b_mode);
+
+/*
+ * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM
+ * left in `workspace`: MXP_OK, or MXP_ERR_TIMEOUT if a bounded wait inside a kernel gave
+ * up (the output is then undefined but the context stays usable).
+ */
+mxp_status mxp_gemm_status(const void *workspace, void *cuda_stream);
+
+/*
+ * Issue-rate probe for the roofline denominator: runs `iters` back-to-back tensor-core
+ * instructions per CTA on operands resident in shared memory (no global traffic) on
+ * every SM and returns the elapsed milliseconds in *ms (synchronises the device).
+ *   kind 0: kind::mxf4 block-scaled E2M1 x E2M1 (128 x 256 x 64 per instruction)
+ *   kind 1: kind::mxf8f6f4 block-scaled E2M3 x E2M3 (128 x 256 x 32 per instruction)
+ * *flops receives the multiply-add work done (2 * M * N * K summed over CTAs).
+ * The paper has no counterpart; it exists so that fractions of peak have a measured
+ * denominator on the device the library runs on.
+ */
+mxp_status mxp_tensor_peak_probe(int kind, int iters, double *ms, double *flops);
+
+const char *mxp_status_string(mxp_status s);
+
+/* Library version string, e.g. "mxp 0.1 sm_100a". */
+const char *mxp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXP_H_ */

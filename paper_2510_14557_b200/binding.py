@@ -1,0 +1,186 @@
+"""ctypes binding of libmxp.so: argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory owned by the caller), passes their
+data pointers and the current CUDA stream through the C ABI declared in ``include/mxp.h``
+and raises ``MxpError`` on a non-zero status.  There is no fallback: if the shared
+library is missing or cannot be loaded, importing a symbol from here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+MXP_OK = 0
+MODE_MXFP4 = 0
+MODE_MXFP4_PLUS = 1
+F32 = 0
+BF16 = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmxp.so")
+
+EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_workspace_bytes",
+           "mxp_gemm_status", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
+
+
+class MxpError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (fn, status_string(status), status))
+
+
+class _Packed(ctypes.Structure):
+    _fields_ = [("nibbles", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("bm_index", ctypes.c_void_p), ("rows", ctypes.c_int64),
+                ("cols", ctypes.c_int64), ("mode", ctypes.c_int)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmxp.so (built in-tree by ``build.py``); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libmxp.so is not built: run `python -m paper_2510_14557_b200.build`")
+        l = ctypes.CDLL(LIB_PATH)
+        i64, vp, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        l.mxp_quantize.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, vp]
+        l.mxp_quantize.restype = ci
+        l.mxp_dequantize.argtypes = [ctypes.POINTER(_Packed), vp, ci, i64, vp]
+        l.mxp_dequantize.restype = ci
+        l.mxp_gemm.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed),
+                               ctypes.POINTER(_Packed), vp, ci, i64, vp, sz, vp]
+        l.mxp_gemm.restype = ci
+        l.mxp_gemm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
+        l.mxp_gemm_workspace_bytes.restype = sz
+        l.mxp_gemm_status.argtypes = [vp, vp]
+        l.mxp_gemm_status.restype = ci
+        l.mxp_tensor_peak_probe.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_double),
+                                            ctypes.POINTER(ctypes.c_double)]
+        l.mxp_tensor_peak_probe.restype = ci
+        l.mxp_status_string.argtypes = [ci]
+        l.mxp_status_string.restype = ctypes.c_char_p
+        l.mxp_version.restype = ctypes.c_char_p
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().mxp_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return lib().mxp_version().decode()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("expected float32 or bfloat16, got %s" % t.dtype)
+
+
+def _check(fn: str, status: int) -> None:
+    if status != MXP_OK:
+        raise MxpError(fn, status)
+
+
+@dataclass
+class Packed:
+    """An MXFP4 / MXFP4+ operand: three uint8 device planes (see include/mxp.h)."""
+    nibbles: torch.Tensor        # [rows, cols/2]
+    scales: torch.Tensor         # [rows, cols/32]
+    bm_index: Optional[torch.Tensor]  # [rows, cols/32] or None (MXFP4)
+    rows: int
+    cols: int
+    mode: int
+
+    def c_struct(self) -> _Packed:
+        return _Packed(self.nibbles.data_ptr(), self.scales.data_ptr(),
+                       self.bm_index.data_ptr() if self.bm_index is not None else None,
+                       self.rows, self.cols, self.mode)
+
+
+def alloc_packed(rows: int, cols: int, mode: int, device="cuda", index_for_mxfp4=False) -> Packed:
+    nib = torch.empty((rows, cols // 2), dtype=torch.uint8, device=device)
+    sc = torch.empty((rows, cols // 32), dtype=torch.uint8, device=device)
+    idx = None
+    if mode == MODE_MXFP4_PLUS or index_for_mxfp4:
+        idx = torch.empty((rows, cols // 32), dtype=torch.uint8, device=device)
+    return Packed(nib, sc, idx, rows, cols, mode)
+
+
+def mxp_quantize(src: torch.Tensor, mode: int, out: Optional[Packed] = None) -> Packed:
+    """Quantizes a 2-D CUDA tensor (float32 / bfloat16, unit inner stride) along its rows."""
+    assert src.is_cuda and src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    if out is None:
+        out = alloc_packed(rows, cols, mode, src.device)
+    st = lib().mxp_quantize(src.data_ptr(), _dt(src), rows, cols, src.stride(0), mode,
+                            out.nibbles.data_ptr(), out.scales.data_ptr(),
+                            out.bm_index.data_ptr() if out.bm_index is not None else None,
+                            _stream())
+    _check("mxp_quantize", st)
+    return out
+
+
+def mxp_dequantize(p: Packed, dtype=torch.float32, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((p.rows, p.cols), dtype=dtype, device=p.nibbles.device)
+    cs = p.c_struct()
+    st = lib().mxp_dequantize(ctypes.byref(cs), out.data_ptr(), _dt(out), out.stride(0), _stream())
+    _check("mxp_dequantize", st)
+    return out
+
+
+def mxp_gemm_workspace_bytes(M: int, N: int, K: int, a_dense: bool, a_mode: int, b_mode: int) -> int:
+    return int(lib().mxp_gemm_workspace_bytes(M, N, K, int(a_dense), a_mode, b_mode))
+
+
+def mxp_gemm(a, b: Packed, out_dtype=torch.bfloat16, out: Optional[torch.Tensor] = None,
+             workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """D = dec(A) @ dec(B).T.  `a` is a bf16 CUDA tensor (weight-only form) or a Packed."""
+    N, K = b.rows, b.cols
+    dense = isinstance(a, torch.Tensor)
+    M = a.shape[0] if dense else a.rows
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=b.nibbles.device)
+    a_mode = MODE_MXFP4 if dense else a.mode
+    need = mxp_gemm_workspace_bytes(M, N, K, dense, a_mode, b.mode)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=b.nibbles.device)
+    ws_ptr = workspace.data_ptr() if workspace is not None else None
+    ws_len = workspace.numel() if workspace is not None else 0
+    bs = b.c_struct()
+    if dense:
+        assert a.dtype == torch.bfloat16 and a.is_cuda and a.stride(1) == 1
+        st = lib().mxp_gemm(M, N, K, a.data_ptr(), a.stride(0), None, ctypes.byref(bs),
+                            out.data_ptr(), _dt(out), out.stride(0), ws_ptr, ws_len, _stream())
+    else:
+        as_ = a.c_struct()
+        st = lib().mxp_gemm(M, N, K, None, 0, ctypes.byref(as_), ctypes.byref(bs),
+                            out.data_ptr(), _dt(out), out.stride(0), ws_ptr, ws_len, _stream())
+    _check("mxp_gemm", st)
+    return out
+
+
+def mxp_gemm_status(workspace: torch.Tensor) -> int:
+    return int(lib().mxp_gemm_status(workspace.data_ptr(), _stream()))
+
+
+def mxp_tensor_peak_probe(kind: int, iters: int):
+    ms, fl = ctypes.c_double(), ctypes.c_double()
+    st = lib().mxp_tensor_peak_probe(kind, iters, ctypes.byref(ms), ctypes.byref(fl))
+    _check("mxp_tensor_peak_probe", st)
+    return ms.value, fl.value

@@ -1,0 +1,139 @@
+// C ABI of libmxp: argument validation and dispatch.  No kernel lives here.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool valid_mode(int m) { return m == MXP_MODE_MXFP4 || m == MXP_MODE_MXFP4_PLUS; }
+bool valid_dtype(int d) { return d == MXP_F32 || d == MXP_BF16; }
+
+// Checks an operand descriptor (host struct, device planes).
+bool valid_packed(const mxp_packed* p)
+{
+    if (p == nullptr) return false;
+    if (!valid_mode(p->mode)) return false;
+    if (p->rows < 0 || p->cols < 0 || p->cols % 32 != 0) return false;
+    if (p->rows == 0 || p->cols == 0) return true;
+    if (p->nibbles == nullptr || p->scales == nullptr) return false;
+    if (!aligned(p->nibbles, 16)) return false;
+    if (p->mode == MXP_MODE_MXFP4_PLUS && p->bm_index == nullptr) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* mxp_status_string(mxp_status s)
+{
+    switch (s) {
+        case MXP_OK: return "ok";
+        case MXP_ERR_INVALID_ARG: return "invalid argument";
+        case MXP_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MXP_ERR_WORKSPACE: return "workspace missing or too small";
+        case MXP_ERR_CUDA: return "CUDA error";
+        case MXP_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* mxp_version(void) { return "mxp 0.1 sm_100a"; }
+
+mxp_status mxp_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t cols,
+                        int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
+                        uint8_t* bm_index, void* cuda_stream)
+{
+    if (!valid_mode(mode) || !valid_dtype(src_dt)) return MXP_ERR_INVALID_ARG;
+    if (rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return MXP_OK;
+    if (src == nullptr || nibbles == nullptr || scales == nullptr) return MXP_ERR_INVALID_ARG;
+    if (mode == MXP_MODE_MXFP4_PLUS && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (ld_src < cols || ld_src % 8 != 0) return MXP_ERR_INVALID_ARG;
+    if (!aligned(src, 16) || !aligned(nibbles, 16)) return MXP_ERR_INVALID_ARG;
+    if (rows * (cols / 32) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    cudaError_t e = mxp::launch_quantize(src, src_dt, rows, cols, ld_src, mode, nibbles, scales,
+                                         bm_index, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+mxp_status mxp_dequantize(const mxp_packed* p, void* dst, mxp_dtype dst_dt, int64_t ld_dst,
+                          void* cuda_stream)
+{
+    if (!valid_packed(p) || !valid_dtype(dst_dt)) return MXP_ERR_INVALID_ARG;
+    if (p->rows == 0 || p->cols == 0) return MXP_OK;
+    if (dst == nullptr || !aligned(dst, 16)) return MXP_ERR_INVALID_ARG;
+    if (ld_dst < p->cols || ld_dst % 8 != 0) return MXP_ERR_INVALID_ARG;
+    if (p->rows * p->cols / 8 / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    cudaError_t e =
+        mxp::launch_dequantize(*p, dst, dst_dt, ld_dst, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+size_t mxp_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense, mxp_mode a_mode,
+                                mxp_mode b_mode)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    if (a_dense) return mxp::skinny_workspace_bytes(M, N, K);
+    return mxp::tc_workspace_bytes(M, N, K, a_mode, b_mode);
+}
+
+mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, int64_t lda,
+                    const mxp_packed* A_packed, const mxp_packed* B_packed, void* D,
+                    mxp_dtype d_dt, int64_t ldd, void* workspace, size_t workspace_bytes,
+                    void* cuda_stream)
+{
+    if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
+    if ((A_dense_bf16 == nullptr) == (A_packed == nullptr)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(B_packed)) return MXP_ERR_INVALID_ARG;
+    if (B_packed->rows != N || B_packed->cols != K) return MXP_ERR_INVALID_ARG;
+    if (A_packed != nullptr) {
+        if (!valid_packed(A_packed)) return MXP_ERR_INVALID_ARG;
+        if (A_packed->rows != M || A_packed->cols != K) return MXP_ERR_INVALID_ARG;
+    } else {
+        if (lda < K || lda % 8 != 0 || !aligned(A_dense_bf16, 16)) return MXP_ERR_INVALID_ARG;
+    }
+    if (M == 0 || N == 0) return MXP_OK;
+    if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (!aligned(D, 16) || ldd % (d_dt == MXP_BF16 ? 8 : 4) != 0) return MXP_ERR_INVALID_ARG;
+    if (K == 0) return MXP_ERR_UNSUPPORTED;  // an empty sum; callers zero D themselves
+    const size_t need = mxp_gemm_workspace_bytes(M, N, K, A_dense_bf16 != nullptr,
+                                                 A_packed ? A_packed->mode : MXP_MODE_MXFP4,
+                                                 B_packed->mode);
+    if (need > 0) {
+        if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
+        if (!aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (A_dense_bf16 != nullptr) {
+        cudaError_t e = mxp::launch_gemm_weight_only(M, N, K, A_dense_bf16, lda, *B_packed, D,
+                                                     d_dt, ldd, workspace, workspace_bytes, stream);
+        if (e == cudaErrorNotSupported) return MXP_ERR_UNSUPPORTED;
+        return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+    }
+    return mxp::launch_gemm_tc(M, N, K, *A_packed, *B_packed, D, d_dt, ldd, workspace,
+                               workspace_bytes, stream);
+}
+
+mxp_status mxp_gemm_status(const void* workspace, void* cuda_stream)
+{
+    if (workspace == nullptr) return MXP_ERR_INVALID_ARG;
+    mxp::StatusBlock sb;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(&sb, workspace, sizeof(sb), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return MXP_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return MXP_ERR_CUDA;
+    return sb.code == 0 ? MXP_OK : static_cast<mxp_status>(sb.code);
+}
+
+mxp_status mxp_tensor_peak_probe(int kind, int iters, double* ms, double* flops)
+{
+    if (ms == nullptr || flops == nullptr || iters <= 0 || kind < 0 || kind > 1)
+        return MXP_ERR_INVALID_ARG;
+    return mxp::tensor_peak_probe(kind, iters, ms, flops);
+}
+
+}  // extern "C"

@@ -1,0 +1,42 @@
+// Shared declarations of the libmxp translation units (device launchers + helpers).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mxp.h"
+
+namespace mxp {
+
+// ---- launchers (each validates nothing: the C ABI layer has done that) -----------------
+cudaError_t launch_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                            int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
+                            uint8_t* bm_index, cudaStream_t stream);
+
+cudaError_t launch_dequantize(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
+                              cudaStream_t stream);
+
+// Weight-only form: D = A(bf16, M x K) * dec(B)^T.
+size_t skinny_workspace_bytes(int64_t M, int64_t N, int64_t K);
+cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                    const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                                    void* workspace, size_t workspace_bytes,
+                                    cudaStream_t stream);
+
+// Block-scaled tensor-core form: both operands packed.
+size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
+mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
+                          const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                          void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+mxp_status tensor_peak_probe(int kind, int iters, double* ms, double* flops);
+
+// First 16 bytes of every GEMM workspace.
+struct StatusBlock {
+    uint32_t code;    // 0 = ok, otherwise an mxp_status
+    uint32_t where;   // which wait gave up (kernel-specific tag)
+    uint32_t pad[2];
+};
+constexpr size_t kStatusBytes = 256;  // keeps what follows 256-byte aligned
+
+}  // namespace mxp

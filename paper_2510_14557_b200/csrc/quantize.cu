@@ -1,0 +1,331 @@
+// MXFP4 / MXFP4+ block quantization and decode kernels (HBM-bound).
+//
+// Quantize (Eq. 1, Sec. 4.1, Sec. 4.2): four lanes own one 32-element block, eight
+// elements (one or two 128-bit loads) each.  A lane group handles four consecutive
+// blocks per pass, so that the scale and index bytes of the group leave as one 32-bit
+// store each.  The block maximum and its first position come out of one integer max over
+// keys (|x| bit pattern, 31 - position), reduced over the four lanes by two shuffles:
+// this is the paper's point that the BM is found for free while computing the scale.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace mxp {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kBlocksPerWarpPass = 32;                      // 8 groups x 4 blocks
+constexpr int kBlocksPerCta = kBlocksPerWarpPass * (kThreads / 32);
+
+// Eight scaled values -> eight E2M1 codes, element 0 in the lowest nibble.
+// cvt.rn.satfinite rounds to nearest-even and saturates at +-6.
+__device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&f)[8])
+{
+    uint32_t r;
+    asm("{ .reg .b8 b0, b1, b2, b3;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n"
+        "  mov.b32 %0, {b0, b1, b2, b3}; }"
+        : "=r"(r)
+        : "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]), "f"(f[6]),
+          "f"(f[7]));
+    return r;
+}
+
+// bf16 path.  Key of one element: 15-bit magnitude pattern in bits 30..16 (monotone in
+// |x|), 31 - position in bits 4..0, so that an unsigned max picks the largest magnitude and,
+// among equal ones, the lowest position.
+__device__ __forceinline__ void load_unit_bf16(const uint4 w4, int pos0, float (&v)[8],
+                                               uint32_t& key)
+{
+    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    uint32_t k = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        v[2 * j] = __uint_as_float(w[j] << 16);
+        v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+        const uint32_t a = w[j] & 0x7FFF7FFFu;
+        const uint32_t klo = (a << 16) | (uint32_t)(31 - (pos0 + 2 * j));
+        const uint32_t khi = (a & 0xFFFF0000u) | (uint32_t)(31 - (pos0 + 2 * j + 1));
+        k = max(k, max(klo, khi));
+    }
+    key = k;
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p)
+{
+    return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+
+// One block's worth of work for this lane (quarter q of block `blk`).
+//   returns the packed nibble word; writes the block's scale / index bytes (same value in
+//   all four lanes of the group).
+template <bool kPlus>
+__device__ __forceinline__ uint32_t encode_quarter(const float (&v)[8], uint32_t amax_bits,
+                                                   int bm, int q, uint32_t& scale_byte,
+                                                   uint32_t& index_byte)
+{
+    // amax_bits: fp32 bit pattern of the block's absolute maximum
+    const uint32_t E = amax_bits >> 23;  // biased exponent (sign already cleared)
+    const bool flush = E <= 2u;          // floor(log2 BM) <= -125, zero and subnormals
+    const bool nonfinite = E == 255u;
+    scale_byte = flush ? 0u : (nonfinite ? 255u : E - 2u);
+    index_byte = (kPlus && !flush && !nonfinite) ? (uint32_t)bm : 0u;
+
+    // 2^-shared_exp = 2^(129 - E): biased exponent 256 - E, in [2, 253] for a kept block
+    const float inv = __uint_as_float((256u - E) << 23);
+    float s[8];
+    uint32_t sign = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        s[i] = v[i] * inv;  // exact (power of two); < 8 in magnitude
+        sign |= (__float_as_uint(v[i]) >> 31) << (4 * i + 3);
+    }
+    // codes from the hardware cast; the sign bit of each nibble is taken from the input so
+    // that values rounding to zero (and -0.0) keep their sign
+    uint32_t word = (cvt_e2m1x8(s) & 0x77777777u) | sign;
+    if (kPlus) {
+        // BM mantissa: top 3 fraction bits of amax, round to nearest even, clamp at 7
+        const uint32_t mant = amax_bits & 0x7FFFFFu;
+        uint32_t m = (mant + 0x7FFFFu + ((mant >> 20) & 1u)) >> 20;
+        m = min(m, 7u);
+        if ((bm >> 3) == q) {
+            const int sh = (bm & 7) * 4;
+            word = (word & ~(7u << sh)) | (m << sh);
+        }
+    }
+    return (flush || nonfinite) ? 0u : word;
+}
+
+// kContig: ld_src == cols, so the source is one flat array of blocks.
+template <typename T, bool kPlus, bool kContig>
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
+                int64_t total_blocks, uint8_t* __restrict__ nibbles,
+                uint8_t* __restrict__ scales, uint8_t* __restrict__ bm_index, int planes_aligned4)
+{
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int g = lane >> 2;  // lane group: blocks 4g .. 4g+3 of the warp's span
+    const int q = lane & 3;   // quarter of the block owned by this lane
+    const int64_t span0 =
+        (int64_t)blockIdx.x * kBlocksPerCta + (int64_t)warp * kBlocksPerWarpPass + 4 * g;
+
+    float v[4][8];
+    uint32_t key[4];
+    uint32_t hi_bits[4];  // fp32 path: the lane's maximum |x| bit pattern
+
+    // ---- issue all loads of the pass first
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int64_t blk = span0 + j;
+        const bool live = blk < total_blocks;
+        int64_t elem;  // offset of the block's first element in src
+        if (kContig) {
+            elem = blk * 32;
+        } else {
+            const int64_t row = blk / cols_blocks;
+            elem = row * ld_src + (blk - row * cols_blocks) * 32;
+        }
+        if (sizeof(T) == 2) {
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (live) w = ldg_stream(reinterpret_cast<const char*>(src) + (elem + q * 8) * 2);
+            load_unit_bf16(w, q * 8, v[j], key[j]);
+            hi_bits[j] = 0;
+        } else {
+            uint4 w0 = make_uint4(0, 0, 0, 0), w1 = w0;
+            if (live) {
+                const char* p = reinterpret_cast<const char*>(src) + (elem + q * 8) * 4;
+                w0 = ldg_stream(p);
+                w1 = ldg_stream(p + 16);
+            }
+            const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+            uint32_t a = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[j][i] = __uint_as_float(w[i]);
+                a = max(a, w[i] & 0x7FFFFFFFu);
+            }
+            hi_bits[j] = a;
+            key[j] = 0;
+            (void)w;
+        }
+    }
+
+    uint32_t words[4], sc_pack = 0, ix_pack = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint32_t amax_bits;
+        int bm;
+        if (sizeof(T) == 2) {
+            uint32_t k = key[j];
+            k = max(k, __shfl_xor_sync(0xFFFFFFFFu, k, 1));
+            k = max(k, __shfl_xor_sync(0xFFFFFFFFu, k, 2));
+            amax_bits = k & 0x7FFF0000u;
+            bm = 31 - (int)(k & 31u);
+        } else {
+            // fp32: 31 magnitude bits do not fit a 32-bit key with the position; reduce the
+            // maximum first, then the first position that holds it.
+            uint32_t a = hi_bits[j];
+            a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, 1));
+            a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, 2));
+            int first = 32;
+#pragma unroll
+            for (int i = 7; i >= 0; --i)
+                if ((__float_as_uint(v[j][i]) & 0x7FFFFFFFu) == a) first = q * 8 + i;
+            first = min(first, __shfl_xor_sync(0xFFFFFFFFu, first, 1));
+            first = min(first, __shfl_xor_sync(0xFFFFFFFFu, first, 2));
+            amax_bits = a;
+            bm = first & 31;
+        }
+        uint32_t sb, ib;
+        words[j] = encode_quarter<kPlus>(v[j], amax_bits, bm, q, sb, ib);
+        sc_pack |= sb << (8 * j);
+        ix_pack |= ib << (8 * j);
+    }
+
+    // ---- stores: 4 bytes of nibbles per lane and block; one word of scales / indices per group
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int64_t blk = span0 + j;
+        if (blk < total_blocks)
+            __stcs(reinterpret_cast<uint32_t*>(nibbles + blk * 16 + q * 4), words[j]);
+    }
+    if (span0 + 3 < total_blocks && planes_aligned4) {
+        if (q == 0) __stcs(reinterpret_cast<uint32_t*>(scales + span0), sc_pack);
+        if (q == 1 && bm_index != nullptr)
+            __stcs(reinterpret_cast<uint32_t*>(bm_index + span0), ix_pack);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (span0 + j < total_blocks) {
+                if (q == 0) scales[span0 + j] = (uint8_t)(sc_pack >> (8 * j));
+                if (q == 1 && bm_index != nullptr)
+                    bm_index[span0 + j] = (uint8_t)(ix_pack >> (8 * j));
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------- decode (Eq. 3)
+// One thread decodes eight elements (one 32-bit word of nibbles).
+__device__ __forceinline__ float e2m1_mag(uint32_t code)
+{
+    // 0, .5, 1, 1.5, 2, 3, 4, 6: subnormal step 0.5 below 1, then 1.m * 2^(e-1)
+    const uint32_t e = code >> 1, m = code & 1u;
+    const float normal = __uint_as_float(((126u + e) << 23) | (m << 22));
+    return e == 0u ? 0.5f * (float)m : normal;
+}
+
+template <typename T, bool kPlus>
+__global__ void __launch_bounds__(kThreads)
+dequantize_kernel(const uint8_t* __restrict__ nibbles, const uint8_t* __restrict__ scales,
+                  const uint8_t* __restrict__ bm_index, int64_t cols, int64_t total_units,
+                  T* __restrict__ dst, int64_t ld_dst)
+{
+    const int64_t u = (int64_t)blockIdx.x * kThreads + threadIdx.x;  // unit of 8 elements
+    if (u >= total_units) return;
+    const int64_t blk = u >> 2;
+    const int q = (int)(u & 3);
+    const uint32_t word = __ldg(reinterpret_cast<const uint32_t*>(nibbles) + u);
+    const uint32_t sb = scales[blk];
+    const int bm = kPlus ? (int)(bm_index[blk] & 31u) : -1;
+    float out[8];
+    // 2^(sb - 127) for sb in 1..254; sb = 0 is the reserved all-zero block; 0xFF decodes NaN
+    const float scale = __uint_as_float(sb << 23);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t n = (word >> (4 * i)) & 15u;
+        const uint32_t code = n & 7u;
+        float mag = e2m1_mag(code);
+        if (kPlus && q * 8 + i == bm) mag = 4.0f + 0.5f * (float)code;  // "MX+ addition"
+        float val = mag * scale;  // exact: <= 4 significant bits times a power of two
+        if (sb == 0u) val = 0.0f;
+        if (sb == 255u) val = __uint_as_float(0x7FC00000u);
+        out[i] = (n & 8u) ? -val : val;
+    }
+    const int64_t e0 = u * 8;
+    const int64_t row = e0 / cols;
+    const int64_t off = row * ld_dst + (e0 - row * cols);
+    if (sizeof(T) == 4) {
+        float4* p = reinterpret_cast<float4*>(reinterpret_cast<float*>(dst) + off);
+        p[0] = make_float4(out[0], out[1], out[2], out[3]);
+        p[1] = make_float4(out[4], out[5], out[6], out[7]);
+    } else {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(out[2 * i], out[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(dst) + off) =
+            make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+template <typename T, bool kPlus>
+cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src,
+                     uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index, cudaStream_t stream)
+{
+    const int64_t total_blocks = rows * (cols / 32);
+    const int64_t grid = (total_blocks + kBlocksPerCta - 1) / kBlocksPerCta;
+    const int aligned4 = ((reinterpret_cast<uintptr_t>(scales) & 3) == 0) &&
+                         ((reinterpret_cast<uintptr_t>(bm_index) & 3) == 0);
+    if (ld_src == cols)
+        quantize_kernel<T, kPlus, true><<<(unsigned)grid, kThreads, 0, stream>>>(
+            static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales,
+            bm_index, aligned4);
+    else
+        quantize_kernel<T, kPlus, false><<<(unsigned)grid, kThreads, 0, stream>>>(
+            static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales,
+            bm_index, aligned4);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                            int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
+                            uint8_t* bm_index, cudaStream_t stream)
+{
+    const bool plus = mode == MXP_MODE_MXFP4_PLUS;
+    if (dt == MXP_BF16)
+        return plus ? launch_q<__nv_bfloat16, true>(src, rows, cols, ld_src, nibbles, scales,
+                                                    bm_index, stream)
+                    : launch_q<__nv_bfloat16, false>(src, rows, cols, ld_src, nibbles, scales,
+                                                     bm_index, stream);
+    return plus ? launch_q<float, true>(src, rows, cols, ld_src, nibbles, scales, bm_index,
+                                        stream)
+                : launch_q<float, false>(src, rows, cols, ld_src, nibbles, scales, bm_index,
+                                         stream);
+}
+
+cudaError_t launch_dequantize(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
+                              cudaStream_t stream)
+{
+    const int64_t units = p.rows * p.cols / 8;
+    const unsigned grid = (unsigned)((units + kThreads - 1) / kThreads);
+    const bool plus = p.mode == MXP_MODE_MXFP4_PLUS;
+    if (dt == MXP_F32) {
+        if (plus)
+            dequantize_kernel<float, true><<<grid, kThreads, 0, stream>>>(
+                p.nibbles, p.scales, p.bm_index, p.cols, units, static_cast<float*>(dst), ld_dst);
+        else
+            dequantize_kernel<float, false><<<grid, kThreads, 0, stream>>>(
+                p.nibbles, p.scales, p.bm_index, p.cols, units, static_cast<float*>(dst), ld_dst);
+    } else {
+        if (plus)
+            dequantize_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, stream>>>(
+                p.nibbles, p.scales, p.bm_index, p.cols, units,
+                static_cast<__nv_bfloat16*>(dst), ld_dst);
+        else
+            dequantize_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, stream>>>(
+                p.nibbles, p.scales, p.bm_index, p.cols, units,
+                static_cast<__nv_bfloat16*>(dst), ld_dst);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace mxp

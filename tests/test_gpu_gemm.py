@@ -1,0 +1,145 @@
+"""GPU parity: mxp_gemm through the C ABI vs the oracle's fp64 product of decoded operands."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_gemm, host_to_packed, to_dev, to_dev_bf16
+from paper_2510_14557_b200 import synth
+
+pytestmark = pytest.mark.gpu
+MX, MXP = 0, 1
+
+
+def mxp():
+    import paper_2510_14557_b200 as m
+    return m
+
+
+def quantized(x_bits_or_f32, mode, bf16=False):
+    q = oracle.quantize(x_bits_or_f32, mode, bf16_bits=bf16)
+    dec = oracle.dequantize(q[0], q[1], q[2], mode)
+    return host_to_packed(q[0], q[1], q[2] if mode == MXP else None, mode), dec
+
+
+# ------------------------------------------------------------------ weight-only form
+@pytest.mark.parametrize("wmode", [MX, MXP])
+@pytest.mark.parametrize("M,N,K", [(1, 64, 128), (8, 48, 256), (16, 100, 4096), (5, 17, 96),
+                                   (16, 33, 32), (40, 64, 512)])
+def test_weight_only_small(M, N, K, wmode):
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K)
+    wp, dw = quantized(w_bits, wmode, bf16=True)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    for dt in (torch.float32, torch.bfloat16):
+        d = mxp().mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=dt)
+        check_gemm(d, da, dw)
+
+
+def test_weight_only_extreme_scales_and_one_hot():
+    # one-hot activations select single decoded weights: exact equality in fp32
+    K, N = 128, 32
+    g = synth.rng(5)
+    w = g.standard_normal((N, K)).astype(np.float32)
+    w *= np.exp2(g.integers(-100, 100, (N, 1))).astype(np.float32)
+    w[3, 32:64] = 0
+    wp, dw = quantized(w, MXP)
+    a = np.zeros((16, K), np.float32)
+    for m in range(16):
+        a[m, (m * 9) % K] = 1.0
+    d = mxp().mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), wp, out_dtype=torch.float32)
+    got = d.cpu().numpy().astype(np.float64)
+    for m in range(16):
+        assert np.array_equal(got[m], dw[:, (m * 9) % K])
+
+
+@pytest.mark.parametrize("M", [1, 8, 16])
+def test_weight_only_config3_sampled(M):
+    a_bits, w_bits = synth.config3(M)
+    wq = oracle.quantize(w_bits, MXP, bf16_bits=True)
+    m = mxp()
+    # encodings of the full weight matrix are bit-exact
+    p = m.mxp_quantize(to_dev_bf16(w_bits), MXP)
+    assert torch.equal(p.nibbles.cpu(), torch.from_numpy(wq[0]))
+    assert torch.equal(p.scales.cpu(), torch.from_numpy(wq[1]))
+    assert torch.equal(p.bm_index.cpu(), torch.from_numpy(wq[2]))
+    d = m.mxp_gemm(to_dev_bf16(a_bits), p, out_dtype=torch.bfloat16)
+    rows = np.unique(np.concatenate([np.arange(0, 11008, 97), [11007, 11006, 5503]]))
+    dw = oracle.dequantize(wq[0][rows], wq[1][rows], wq[2][rows], MXP)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    check_gemm(d[:, torch.from_numpy(rows).cuda()], da, dw)
+
+
+# ------------------------------------------------------------------ tensor-core form
+MODES = [(MX, MX), (MXP, MX), (MX, MXP), (MXP, MXP)]
+
+
+@pytest.mark.parametrize("amode,bmode", MODES)
+def test_tc_config1(amode, bmode):
+    a, b = synth.config1()
+    ap, da = quantized(a, amode)
+    bp, db = quantized(b, bmode)
+    m = mxp()
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32, workspace=ws)
+    assert m.mxp_gemm_status(ws) == 0
+    check_gemm(d, da, db)
+    d16 = m.mxp_gemm(ap, bp, out_dtype=torch.bfloat16, workspace=ws)
+    check_gemm(d16, da, db)
+
+
+@pytest.mark.parametrize("amode,bmode", MODES)
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (128, 256, 256), (100, 72, 384), (300, 520, 1024),
+                                   (1, 8, 128), (257, 129, 2176)])
+def test_tc_shapes(M, N, K, amode, bmode):
+    a = synth.activations_normal(M, K, seed=M + K, outlier_frac=0.02)
+    b = synth.weights(N, K, seed=N + K)
+    ap, da = quantized(a, amode)
+    bp, db = quantized(b, bmode)
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    check_gemm(d, da, db)
+
+
+@pytest.mark.parametrize("amode,bmode", MODES)
+def test_tc_one_hot_b_returns_decoded_a(amode, bmode):
+    # B = identity (1.0 is an exactly representable BM): D must equal dec(A) bit for bit,
+    # which exercises the BM residual passes exactly
+    K = 256
+    a = synth.activations_normal(192, K, seed=77, outlier_frac=0.03)
+    ap, da = quantized(a, amode)
+    bp, db = quantized(np.eye(K, dtype=np.float32), bmode)
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
+
+
+def test_tc_bm_positions_coincide():
+    # both operands MX+ with the BM of every block at the same position: the BM_L x BM_L
+    # term of the expansion is then non-zero everywhere
+    M, N, K = 64, 64, 512
+    g = synth.rng(3)
+    a = (g.standard_normal((M, K)) * 0.3).astype(np.float32)
+    b = (g.standard_normal((N, K)) * 0.3).astype(np.float32)
+    pos = g.integers(0, 32, K // 32)
+    for j, p in enumerate(pos):
+        a[:, 32 * j + p] = g.choice([4.5, 5.5, 6.5, 7.5, -5.0, -7.0], M)
+        b[:, 32 * j + p] = g.choice([4.5, 5.5, 6.5, 7.5, -4.5, -6.5], N)
+    ap, da = quantized(a, MXP)
+    bp, db = quantized(b, MXP)
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    check_gemm(d, da, db)
+    ref = oracle.gemm_fp64(da, db)
+    # values are small dyadic rationals: fp32 accumulation is exact here
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), ref)
+
+
+def test_tc_flushed_and_zero_blocks():
+    M, N, K = 128, 128, 256
+    a = synth.activations_normal(M, K, seed=1)
+    b = synth.weights(N, K, seed=2)
+    a[:, 64:96] = 0
+    b[5, :] = 0
+    b[:, 128:160] *= 1e-42
+    ap, da = quantized(a, MXP)
+    bp, db = quantized(b, MXP)
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    check_gemm(d, da, db)
+    assert float(d[:, 5].abs().max()) == 0.0
