@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the MX+ hot path on B200: activation quantize (bf16 -> MXFP4+) followed by
+the block-scaled GEMM against pre-quantized MXFP4+ weights.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg5|cfg4|small] [--no-parts]
+
+One "step" = mxp_quantize(A) + mxp_gemm(A_q, W_q) on one batch of synthetic activations.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead, on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (M, N, K, label)
+    "cfg5": (8192, 28672, 8192, "prefill 8192x8192x28672 (Llama-70B MLP-like), both operands MX+, quantize->GEMM"),
+    "cfg4": (2048, 4096, 4096, "prefill 2048x4096x4096, both operands MX+, quantize->GEMM"),
+    "small": (256, 512, 512, "small smoke shape, both operands MX+, quantize->GEMM"),
+}
+METRIC = "MX+ quantize->GEMM throughput (prefill, both operands MXFP4+, 2*M*N*K per step)"
+UNIT = "TFLOP/s"
+NOMINAL_FP4_OVER_BF16 = 4.0  # 9 PF dense FP4 vs 2.25 PF dense bf16
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"],
+                "bf16_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "src": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "src": "fallback"}
+
+
+# ------------------------------------------------------------------------- clocks sampling
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_run(M, N, K, rows_a=32, rows_b=2048, seed=4):
+    """One oracle pass on a bounded sample of the workload: quantize rows_a activation rows
+    and rows_b weight rows to MXFP4+, decode them, multiply in fp64.  Returns (seconds, flops)."""
+    import oracle
+    from paper_2510_14557_b200 import synth
+    rows_a, rows_b = min(rows_a, M), min(rows_b, N)
+    a_bits = synth.f32_to_bf16_bits(synth.activations_normal(rows_a, K, seed, 0.01, 30.0))
+    w_bits = synth.f32_to_bf16_bits(synth.weights(rows_b, K, seed + 100))
+    t0 = time.perf_counter()
+    qa = oracle.quantize(a_bits, oracle.MODE_MXFP4_PLUS, bf16_bits=True)
+    qw = oracle.quantize(w_bits, oracle.MODE_MXFP4_PLUS, bf16_bits=True)
+    da = oracle.dequantize(*qa, oracle.MODE_MXFP4_PLUS)
+    dw = oracle.dequantize(*qw, oracle.MODE_MXFP4_PLUS)
+    oracle.gemm_fp64(da, dw)
+    dt = time.perf_counter() - t0
+    return dt, 2.0 * rows_a * rows_b * K
+
+
+def cpu_baseline(M, N, K):
+    import oracle
+    cores = oracle.max_threads()
+    oracle.set_threads(cores)
+    rows_a, rows_b = 32, 2048
+    dt, fl = oracle_sample_run(M, N, K, rows_a, rows_b)
+    # grow the sample once if it was far below the 10 s mark
+    if dt < 5.0 and rows_b * 2 <= N:
+        rows_b = min(N, int(rows_b * min(8.0, 12.0 / max(dt, 0.05))))
+        dt, fl = oracle_sample_run(M, N, K, rows_a, rows_b)
+    return {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d activation rows x %d weight rows x K=%d of the workload "
+                      "(quantize both to MXFP4+, decode, fp64 GEMM), %.1f s" % (min(rows_a, M), min(rows_b, N), K, dt)}
+
+
+def run_reference(args, M, N, K, label):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cores = oracle.max_threads()
+    oracle.set_threads(cores)
+    rows_a, rows_b = 16, 1024
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt, fl = oracle_sample_run(M, N, K, rows_a, rows_b)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = fl / (ms / 1e3) / 1e12
+    sample = "%d activation rows x %d weight rows x K=%d per step" % (min(rows_a, M), min(rows_b, N), K)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": label, "M": M, "N": N, "K": K, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ------------------------------------------------------------------------- multi-rank glue
+def aggregate(ms_local: float, flops_local: float, dist=None):
+    """Max time over ranks and summed work (weak scaling: every rank runs its own batch)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms_local, flops_local
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    f = torch.tensor([flops_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(f.item())
+
+
+# ------------------------------------------------------------------------- GPU legs
+def dev_bf16(bits):
+    import torch
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def time_loop(fn, iters, warmup=3):
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters  # ms
+
+
+def parts(mxp, synth, peaks):
+    """Per-config numbers: quantize (config 2), decode GEMM (config 3), prefill GEMM (config 4),
+    each in MXFP4+ and in plain MXFP4."""
+    import torch
+    out = {}
+    hbm = peaks["hbm_gbs"]
+    fp4_burst = peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16
+    # ---- config 2: quantize 8192 x 8192 bf16 (inputs larger than L2: 134 MB read per launch)
+    x = dev_bf16(synth.config2())
+    n = x.numel()
+    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
+        buf = mxp.alloc_packed(x.shape[0], x.shape[1], mode, index_for_mxfp4=False)
+        ms = time_loop(lambda: mxp.mxp_quantize(x, mode, out=buf), 20)
+        nbytes = n * (2 + 0.5 + 1 / 32 + (1 / 32 if mode == mxp.MODE_MXFP4_PLUS else 0))
+        gbs = nbytes / ms / 1e6
+        out["quantize_cfg2_" + name] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
+    del x
+    # ---- config 3: weight-only decode GEMM; rotate over 8 weight copies (> L2) between launches
+    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
+        a16, w_bits = synth.config3(16)
+        w = dev_bf16(w_bits)
+        copies = []
+        for _ in range(8):
+            copies.append(mxp.mxp_quantize(w, mode))
+        wbytes = 11008 * 4096 * (0.5 + 1 / 32 + (1 / 32 if mode == mxp.MODE_MXFP4_PLUS else 0))
+        for M in (1, 8, 16):
+            a = dev_bf16(a16[:M].copy())
+            d = torch.empty((M, 11008), dtype=torch.bfloat16, device="cuda")
+            state = {"i": 0}
+
+            def run():
+                mxp.mxp_gemm(a, copies[state["i"] % 8], out=d)
+                state["i"] += 1
+            ms = time_loop(run, 40, warmup=8)
+            gbs = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms / 1e6
+            out["decode_cfg3_M%d_%s" % (M, name)] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
+        del copies, w
+    # ---- config 4: prefill GEMM on packed operands, every mode pair
+    a_bits, w_bits = synth.config4()
+    a, w = dev_bf16(a_bits), dev_bf16(w_bits)
+    M, K = a.shape
+    N = w.shape[0]
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    d = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for an, am in (("mxfp4", 0), ("mxfp4+", 1)):
+        for bn, bm in (("mxfp4", 0), ("mxfp4+", 1)):
+            pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
+            tot = 0.0
+            iters = 10
+            for i in range(iters + 3):
+                flush.fill_(i & 255)  # evict L2 between timed launches
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                mxp.mxp_gemm(pa, pw, out=d, workspace=ws)
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    tot += e0.elapsed_time(e1)
+            ms = tot / iters
+            tf = 2.0 * M * N * K / ms / 1e9
+            out["prefill_cfg4_A-%s_W-%s" % (an, bn)] = {
+                "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
+                "frac_fp4_nominal_9PF": tf / 9000.0}
+    return out
+
+
+def run_ours(args, M, N, K, label):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_14557_b200 import build
+    build.build()
+    import paper_2510_14557_b200 as mxp
+    from paper_2510_14557_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    peaks = measured_peaks()
+
+    # synthetic operands (every rank: same weights, its own activation batch)
+    a_bits = synth.f32_to_bf16_bits(synth.activations_normal(M, K, 4 + 1000 * rank, 0.01, 30.0))
+    w_bits = synth.f32_to_bf16_bits(synth.weights(N, K, 104))
+    a_host = torch.from_numpy(a_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    a_dev = a_host.cuda()
+    w_dev = dev_bf16(w_bits)
+    pw = mxp.mxp_quantize(w_dev, mxp.MODE_MXFP4_PLUS)   # weights are quantized once, offline
+    del w_dev, w_bits
+    pa = mxp.alloc_packed(M, K, mxp.MODE_MXFP4_PLUS)
+    d_dev = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    d_host = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    ws = torch.zeros(max(4096, mxp.mxp_gemm_workspace_bytes(M, N, K, False, 1, 1)),
+                     dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        mxp.mxp_quantize(a_dev, mxp.MODE_MXFP4_PLUS, out=pa)
+        if ev is not None:
+            ev[0].record(stream)
+        mxp.mxp_gemm(pa, pw, out=d_dev, workspace=ws)
+        if ev is not None:
+            ev[1].record(stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    if mxp.mxp_gemm_status(ws) != 0:
+        raise RuntimeError("mxp_gemm reported a device-side timeout")
+
+    # ---- device-resident timing
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(kev[i])
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_local = e0.elapsed_time(e1) / args.steps
+    gemm_ms = sum(a.elapsed_time(b) for a, b in kev) / args.steps
+    flops_step = 2.0 * M * N * K
+    ms, flops_all = aggregate(ms_local, flops_step, dist if world > 1 else None)
+
+    # ---- end to end: pinned host activations in, result matrix out, every step
+    for _ in range(2):
+        a_dev.copy_(a_host, non_blocking=True); step(); d_host.copy_(d_dev, non_blocking=True)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(2, min(args.steps, 5))
+    e2.record(stream)
+    for _ in range(e2e_steps):
+        a_dev.copy_(a_host, non_blocking=True)
+        step()
+        d_host.copy_(d_dev, non_blocking=True)
+    e3.record(stream)
+    barrier()
+    e2e_ms, e2e_flops = aggregate(e2.elapsed_time(e3) / e2e_steps, flops_step, dist if world > 1 else None)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
+    achieved = flops_step / gemm_ms / 1e9
+    line = {
+        "metric": METRIC, "value": flops_all / ms / 1e9, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4 (E2M1/E0M3 operands, fp32 accumulate)",
+        "data": "synthetic",
+        "config": {"workload": label, "M": M, "N": N, "K": K, "a_mode": "MXFP4+", "w_mode": "MXFP4+",
+                   "out": "bf16", "l2": "inputs larger than L2 (no flush needed)" if (M * K * 2 + N * K // 2) > (126 << 20)
+                   else "inputs smaller than L2: numbers include L2 hits"},
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": fp4_peak,
+                     "unit": "TFLOP/s", "frac": achieved / fp4_peak, "traffic": None,
+                     "peak_source": "%s bf16 sustained x4 (nominal FP4:bf16 ratio)" % peaks["src"],
+                     "kernel_ms": gemm_ms},
+        "e2e": {"value": e2e_flops / e2e_ms / 1e9, "unit": UNIT, "h2d_bytes_per_step": M * K * 2,
+                "d2h_bytes_per_step": M * N * 2, "ms_per_step": e2e_ms},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+    }
+    if world == 1:
+        if not args.no_parts:
+            del d_dev, d_host, pa, pw, a_dev
+            torch.cuda.empty_cache()
+            try:
+                line["parts"] = parts(mxp, synth, peaks)
+            except Exception as e:  # report, never hide
+                line["parts"] = {"error": repr(e)}
+        line["cpu_baseline"] = cpu_baseline(M, N, K)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-parts", action="store_true")
+    args = ap.parse_args()
+    M, N, K, label = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, M, N, K, label)
+    else:
+        run_ours(args, M, N, K, label)
+
+
+if __name__ == "__main__":
+    main()

@@ -93,6 +93,7 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  *     block-scaled tensor-core path; any combination of MXFP4 / MXFP4+ modes.
  *   B_packed   host pointer to the descriptor of the N x K weight operand
  *   D          M x N of `d_dt` (bf16 rounded to nearest even, or fp32), row stride ldd
+ *              elements (ldd >= N; 16-byte aligned rows let the epilogue use wide stores)
  *   workspace  device scratch of at least mxp_gemm_workspace_bytes(...) bytes, 256-byte
  *              aligned; may be NULL when that size is 0.  Its first 16 bytes are a status
  *              block written by the kernels (see mxp_gemm_status).

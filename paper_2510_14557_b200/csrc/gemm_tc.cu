@@ -56,6 +56,7 @@ struct Params {
     const uint8_t* b_index;
     void* D;
     int64_t ldd;
+    int d_vec_ok;  // D rows are 16-byte aligned: the epilogue may use 128-bit stores
     StatusBlock* status;
 };
 
@@ -362,7 +363,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 ptx::tmem_ld_wait();
                 const int col0 = n0 + 32 * c;
                 if (row < prm.M && col0 < prm.N) {
-                    if (col0 + 32 <= prm.N) {
+                    if (col0 + 32 <= prm.N && prm.d_vec_ok) {
                         if (sizeof(OutT) == 4) {
                             uint4* p = reinterpret_cast<uint4*>(drow + 32 * c);
 #pragma unroll
@@ -507,6 +508,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     prm.b_index = B.bm_index;
     prm.D = D;
     prm.ldd = ldd;
+    prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
+                   ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
     prm.status = static_cast<StatusBlock*>(workspace);
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
         return MXP_ERR_CUDA;
