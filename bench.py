@@ -125,13 +125,16 @@ def cpu_baseline(M, N, K):
     oracle.set_threads(cores)
     rows_a, rows_b = 32, 2048
     dt, fl = oracle_sample_run(M, N, K, rows_a, rows_b)
-    # grow the sample once if it was far below the 10 s mark
-    if dt < 5.0 and rows_b * 2 <= N:
-        rows_b = min(N, int(rows_b * min(8.0, 12.0 / max(dt, 0.05))))
+    # grow the sample (more activation rows) until it is about 10 s of CPU work
+    for _ in range(3):
+        if dt >= 8.0 or rows_a >= M:
+            break
+        rows_a = min(M, max(rows_a + 1, int(rows_a * min(16.0, 12.0 / max(dt, 0.05)))))
         dt, fl = oracle_sample_run(M, N, K, rows_a, rows_b)
     return {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "%d activation rows x %d weight rows x K=%d of the workload "
-                      "(quantize both to MXFP4+, decode, fp64 GEMM), %.1f s" % (min(rows_a, M), min(rows_b, N), K, dt)}
+                      "(quantize both to MXFP4+, decode, fp64 GEMM), %.1f s, %d OpenMP threads"
+                      % (min(rows_a, M), min(rows_b, N), K, dt, cores)}
 
 
 def run_reference(args, M, N, K, label):
@@ -194,23 +197,41 @@ def time_loop(fn, iters, warmup=3):
     return e0.elapsed_time(e1) / iters  # ms
 
 
-def parts(mxp, synth, peaks):
+def parts(mxp, synth, peaks, only=None, iters_scale=1.0):
     """Per-config numbers: quantize (config 2), decode GEMM (config 3), prefill GEMM (config 4),
-    each in MXFP4+ and in plain MXFP4."""
+    each in MXFP4+ and in plain MXFP4.  `only` restricts the run to one of
+    "quantize" / "decode" / "prefill" (used for profiler captures of a single kernel)."""
     import torch
     out = {}
-    hbm = peaks["hbm_gbs"]
-    fp4_burst = peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16
+    if only in (None, "quantize"):
+        out.update(part_quantize(mxp, synth, peaks, max(2, int(20 * iters_scale))))
+    if only in (None, "decode"):
+        out.update(part_decode(mxp, synth, peaks, max(2, int(40 * iters_scale))))
+    if only in (None, "prefill"):
+        out.update(part_prefill(mxp, synth, peaks, max(1, int(10 * iters_scale))))
+    return out
+
+
+def part_quantize(mxp, synth, peaks, iters):
+    import torch
+    out = {}
     # ---- config 2: quantize 8192 x 8192 bf16 (inputs larger than L2: 134 MB read per launch)
+    hbm = peaks["hbm_gbs"]
     x = dev_bf16(synth.config2())
     n = x.numel()
     for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
         buf = mxp.alloc_packed(x.shape[0], x.shape[1], mode, index_for_mxfp4=False)
-        ms = time_loop(lambda: mxp.mxp_quantize(x, mode, out=buf), 20)
+        ms = time_loop(lambda: mxp.mxp_quantize(x, mode, out=buf), iters)
         nbytes = n * (2 + 0.5 + 1 / 32 + (1 / 32 if mode == mxp.MODE_MXFP4_PLUS else 0))
         gbs = nbytes / ms / 1e6
         out["quantize_cfg2_" + name] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
-    del x
+    return out
+
+
+def part_decode(mxp, synth, peaks, iters):
+    import torch
+    out = {}
+    hbm = peaks["hbm_gbs"]
     # ---- config 3: weight-only decode GEMM; rotate over 8 weight copies (> L2) between launches
     for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
         a16, w_bits = synth.config3(16)
@@ -227,10 +248,17 @@ def parts(mxp, synth, peaks):
             def run():
                 mxp.mxp_gemm(a, copies[state["i"] % 8], out=d)
                 state["i"] += 1
-            ms = time_loop(run, 40, warmup=8)
+            ms = time_loop(run, iters, warmup=8)
             gbs = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms / 1e6
             out["decode_cfg3_M%d_%s" % (M, name)] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
         del copies, w
+    return out
+
+
+def part_prefill(mxp, synth, peaks, iters):
+    import torch
+    out = {}
+    fp4_burst = peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16
     # ---- config 4: prefill GEMM on packed operands, every mode pair
     a_bits, w_bits = synth.config4()
     a, w = dev_bf16(a_bits), dev_bf16(w_bits)
@@ -243,7 +271,6 @@ def parts(mxp, synth, peaks):
         for bn, bm in (("mxfp4", 0), ("mxfp4+", 1)):
             pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
             tot = 0.0
-            iters = 10
             for i in range(iters + 3):
                 flush.fill_(i & 255)  # evict L2 between timed launches
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -391,9 +418,17 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
     ap.add_argument("--no-parts", action="store_true")
+    ap.add_argument("--only", default=None, choices=["quantize", "decode", "prefill"],
+                    help="run one per-config part only and print its numbers (profiler captures)")
+    ap.add_argument("--iters-scale", type=float, default=1.0)
     args = ap.parse_args()
     M, N, K, label = WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.only is not None:
+        from paper_2510_14557_b200 import build, synth
+        build.build()
+        import paper_2510_14557_b200 as mxp
+        print(json.dumps({"parts": parts(mxp, synth, measured_peaks(), args.only, args.iters_scale)}))
+    elif args.impl == "reference":
         run_reference(args, M, N, K, label)
     else:
         run_ours(args, M, N, K, label)
