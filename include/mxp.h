@@ -127,6 +127,34 @@ mxp_status mxp_gemm_status(const void *workspace, void *cuda_stream);
  */
 mxp_status mxp_tensor_peak_probe(int kind, int iters, double *ms, double *flops);
 
+/*
+ * The packed-operand form of mxp_gemm for callers that cannot allocate device memory
+ * (the paper has no counterpart; this is a deployment convenience).
+ *
+ * Who needs it: code that runs inside another framework's memory pool and must not call
+ * cudaMalloc behind its back, plugins loaded after the pool has taken the whole device,
+ * and callers with no allocator of their own to ask for the GEMM's small workspace.
+ * Here that workspace (the status block the kernel's bounded waits report into) lives in
+ * a fixed device array inside the library: 4096 bytes that every GPU which loads libmxp
+ * holds until the process exits.  The call allocates and frees nothing, on the host or
+ * the device; A, B and D are still the caller's memory, with the same layout rules as
+ * mxp_gemm.  A problem whose workspace need exceeds those 4096 bytes is rejected with
+ * MXP_ERR_WORKSPACE before anything is launched.
+ *
+ * The first call on a device looks up the array's device address (with that device
+ * current) and remembers it; make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps what the previous call left:
+ * the status block is cleared on `cuda_stream` at the start of every call, but two calls
+ * whose kernels overlap on the GPU (different streams) race on it; serialise them.
+ *
+ *   kernel_status  host pointer or NULL.  When given, the call synchronises `cuda_stream`
+ *                  and stores MXP_OK or MXP_ERR_TIMEOUT (what mxp_gemm_status would
+ *                  report); when NULL the call stays asynchronous.
+ */
+mxp_status mxp_gemm_noalloc(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
+                            const mxp_packed *B_packed, void *D, mxp_dtype d_dt, int64_t ldd,
+                            mxp_status *kernel_status, void *cuda_stream);
+
 const char *mxp_status_string(mxp_status s);
 
 /* Library version string, e.g. "mxp 0.1 sm_100a". */

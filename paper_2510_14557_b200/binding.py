@@ -23,7 +23,7 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes",
            "mxp_gemm_status", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
@@ -57,6 +57,9 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed),
                                ctypes.POINTER(_Packed), vp, ci, i64, vp, sz, vp]
         l.mxp_gemm.restype = ci
+        l.mxp_gemm_noalloc.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
+                                       vp, ci, i64, ctypes.POINTER(ci), vp]
+        l.mxp_gemm_noalloc.restype = ci
         l.mxp_gemm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
         l.mxp_gemm_workspace_bytes.restype = sz
         l.mxp_gemm_status.argtypes = [vp, vp]
@@ -173,6 +176,21 @@ def mxp_gemm(a, b: Packed, out_dtype=torch.bfloat16, out: Optional[torch.Tensor]
                             out.data_ptr(), _dt(out), out.stride(0), ws_ptr, ws_len, _stream())
     _check("mxp_gemm", st)
     return out
+
+
+def mxp_gemm_noalloc(a: Packed, b: Packed, out: torch.Tensor, read_status: bool = False):
+    """Packed-operand GEMM that allocates nothing: for callers that may not call cudaMalloc
+    (code living inside another framework's memory pool, plugins loaded once the pool owns
+    the device).  `out` must be preallocated by the caller; the kernel's scratch sits in a
+    4 KB array inside the library.  Returns the kernel status when `read_status` is set
+    (that synchronises the stream), else None."""
+    ks = ctypes.c_int(0)
+    as_, bs = a.c_struct(), b.c_struct()
+    st = lib().mxp_gemm_noalloc(a.rows, b.rows, b.cols, ctypes.byref(as_), ctypes.byref(bs),
+                                out.data_ptr(), _dt(out), out.stride(0),
+                                ctypes.byref(ks) if read_status else None, _stream())
+    _check("mxp_gemm_noalloc", st)
+    return ks.value if read_status else None
 
 
 def mxp_gemm_status(workspace: torch.Tensor) -> int:
