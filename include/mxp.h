@@ -121,6 +121,10 @@ mxp_status mxp_gemm_status(const void *workspace, void *cuda_stream);
  * every SM and returns the elapsed milliseconds in *ms (synchronises the device).
  *   kind 0: kind::mxf4 block-scaled E2M1 x E2M1 (128 x 256 x 64 per instruction)
  *   kind 1: kind::mxf8f6f4 block-scaled E2M3 x E2M3 (128 x 256 x 32 per instruction)
+ *   kind 2: as kind 0 plus the three scale-factor copies (tcgen05.cp) a 128 x 256 tile needs
+ *           per 128 elements of K, into one TMEM buffer
+ *   kind 3: as kind 2 with the copies alternating between two TMEM buffers
+ * `iters` counts groups of two instructions.
  * *flops receives the multiply-add work done (2 * M * N * K summed over CTAs).
  * The paper has no counterpart; it exists so that fractions of peak have a measured
  * denominator on the device the library runs on.

@@ -131,7 +131,7 @@ mxp_status mxp_gemm_status(const void* workspace, void* cuda_stream)
 
 mxp_status mxp_tensor_peak_probe(int kind, int iters, double* ms, double* flops)
 {
-    if (ms == nullptr || flops == nullptr || iters <= 0 || kind < 0 || kind > 1)
+    if (ms == nullptr || flops == nullptr || iters <= 0 || kind < 0 || kind > 3)
         return MXP_ERR_INVALID_ARG;
     return mxp::tensor_peak_probe(kind, iters, ms, flops);
 }

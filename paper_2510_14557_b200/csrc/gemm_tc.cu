@@ -28,7 +28,16 @@ constexpr int BM = 128;             // rows of A per tile
 constexpr int BK = 256;             // elements of K per stage = 128 bytes of nibbles
 constexpr int kRowBytes = BK / 2;   // 128
 constexpr int kAuxThreads = 128;
-constexpr int kThreads = 64 + kAuxThreads;  // warp 0: TMA, warp 1: MMA, warps 2..5: aux + epilogue
+constexpr int kEpiThreads = 256;
+// warp 0: TMA producer, warp 1: MMA issuer, warps 2..5: aux (scales, BM patches),
+// warps 6..13: epilogue (two warps per TMEM lane quarter, half of the columns each)
+constexpr int kThreads = 64 + kAuxThreads + kEpiThreads;
+// K tiles of scale / index bytes the aux threads fetch ahead: the MX+ variants spend 2-4x as
+// long per K tile (residual passes), so half the distance hides the same latency there
+template <bool AP, bool BP>
+struct Prefetch {
+    static constexpr int value = (AP || BP) ? 2 : 4;
+};
 constexpr long long kWaitLimit = 4000000000ll;  // cycles (~2 s) before a wait gives up
 constexpr uint32_t kTmemCols = 512;
 
@@ -56,6 +65,7 @@ struct Params {
     const uint8_t* b_index;
     void* D;
     int64_t ldd;
+    int num_sms;
     int d_vec_ok;  // D rows are 16-byte aligned: the epilogue may use 128-bit stores
     StatusBlock* status;
 };
@@ -118,6 +128,13 @@ __device__ __forceinline__ void clear_row(uint8_t* lo, uint32_t r, uint2 idx)
     }
 }
 
+// Bytes of scale / index planes one aux thread holds for a group of kPrefetch K tiles.
+template <int H, int kPrefetch>
+struct RowBytes {
+    uint2 sa[kPrefetch], ia[kPrefetch];
+    uint2 sb[H][kPrefetch], ib[H][kPrefetch];
+};
+
 template <int BN, bool AP, bool BP, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -125,7 +142,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 {
     using C = Cfg<BN, AP, BP>;
     constexpr int S = C::kStages;
-    constexpr int kBRowsPerThread = BN / kAuxThreads;  // 1 or 2
+    constexpr int H = BN / kAuxThreads;  // B rows per aux thread: 1 or 2
+    constexpr int kPrefetch = Prefetch<AP, BP>::value;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -137,8 +155,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint64_t* full = bars;            // TMA bytes landed
     uint64_t* ready = bars + S;       // aux threads done (scales staged, BM patched)
     uint64_t* empty = bars + 2 * S;   // MMAs that read the stage have completed
-    uint64_t* acc_full = bars + 3 * S;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 1);
+    uint64_t* acc_full = bars + 3 * S;       // accumulator of the current tile is complete
+    uint64_t* acc_empty = bars + 3 * S + 1;  // epilogue has copied the accumulator out
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 2);
     volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
 
     auto a_hi = [&](int s) { return data0 + s * C::kStageData; };
@@ -155,9 +174,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
     const int nbk = prm.K / 32;
     const int ktiles = (prm.K + BK - 1) / BK;
+    // persistent tile loop: tile ids run M-fastest so that CTAs working at the same time
+    // share B tiles and the (smaller) A operand stays in L2
+    const int tiles_m = (prm.M + BM - 1) / BM;
+    const int tiles_n = (prm.N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -166,6 +189,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ptx::mbar_init(&empty[s], 1);
         }
         ptx::mbar_init(acc_full, 1);
+        ptx::mbar_init(acc_empty, kEpiThreads);
         *abort = 0u;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_a);
@@ -198,197 +222,272 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            for (int kt = 0; kt < ktiles; ++kt) {
-                const int s = kt % S;
-                const uint32_t use = kt / S;
-                if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
-                    give_up(abort, prm.status, 0x100 + s);
-                    break;
+            uint32_t c = 0;  // K tiles issued so far (ring position)
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+                for (int kt = 0; kt < ktiles; ++kt, ++c) {
+                    const int s = c % S;
+                    const uint32_t use = c / S;
+                    if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
+                        give_up(abort, prm.status, 0x100 + s);
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_arrive_expect_tx(&full[s], C::kATile + C::kBTile);
+                    ptx::tma_load_2d(a_hi(s), &tmap_a, &full[s], kt * kRowBytes, m0);
+                    ptx::tma_load_2d(b_hi(s), &tmap_b, &full[s], kt * kRowBytes, n0);
                 }
-                ptx::mbar_arrive_expect_tx(&full[s], C::kATile + C::kBTile);
-                ptx::tma_load_2d(a_hi(s), &tmap_a, &full[s], kt * kRowBytes, m0);
-                ptx::tma_load_2d(b_hi(s), &tmap_b, &full[s], kt * kRowBytes, n0);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            uint32_t accumulate = 0;
+        // The whole warp runs this loop so that stage indices, descriptors and TMEM addresses
+        // stay warp-uniform (tcgen05 takes uniform-register operands; per-thread values would
+        // cost a register-file crossing per operand); one elected lane issues.
+        {
+            uint32_t c = 0, ti = 0;
             bool ok = true;
-            for (int kt = 0; kt < ktiles && ok; ++kt) {
-                const int s = kt % S;
-                const uint32_t ph = (kt / S) & 1;
-                if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit) ||
-                    !ptx::mbar_wait(&ready[s], ph, abort, kWaitLimit)) {
-                    give_up(abort, prm.status, 0x200 + s);
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
+                // the epilogue must have drained the previous tile's accumulator
+                if (ti > 0 && !ptx::mbar_wait(acc_empty, (ti - 1) & 1, abort, kWaitLimit)) {
+                    if (lane == 0) give_up(abort, prm.status, 0x600);
                     ok = false;
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const uint64_t da_hi = ptx::smem_desc_sw128(ptx::smem_u32(a_hi(s)));
-                const uint64_t db_hi = ptx::smem_desc_sw128(ptx::smem_u32(b_hi(s)));
-                const uint64_t da_lo = AP ? ptx::smem_desc_sw128(ptx::smem_u32(a_lo(s))) : 0;
-                const uint64_t db_lo = BP ? ptx::smem_desc_sw128(ptx::smem_u32(b_lo(s))) : 0;
-                const int groups = (prm.K - kt * BK) >= BK ? 2 : 1;  // K % 128 == 0
-                for (int g = 0; g < groups; ++g) {
-                    const uint32_t t_sfa = tmem_sfa + 4 * g;
-                    const uint32_t t_sfb = tmem_sfb + (BN / 32) * g;
-                    ptx::tc_cp_sf(t_sfa, ptx::smem_desc_sf(ptx::smem_u32(sfa(s) + 512 * g)));
-#pragma unroll
-                    for (int h = 0; h < BN / 128; ++h)
-                        ptx::tc_cp_sf(t_sfb + 4 * h,
-                                      ptx::smem_desc_sf(ptx::smem_u32(sfb(s) + 1024 * h + 512 * g)));
-#pragma unroll
-                    for (int kk = 0; kk < 2; ++kk) {
-                        // 64 elements = 32 bytes per MMA: advance the start address field
-                        const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
-                        const uint32_t idesc =
-                            ptx::idesc_block_scaled(1, 1, BM, BN, 2 * kk, 2 * kk);
-                        ptx::mma_mxf4(tmem_acc, da_hi + adv, db_hi + adv, idesc, t_sfa, t_sfb,
-                                      accumulate);
-                        accumulate = 1;
-                        if (AP)
-                            ptx::mma_mxf4(tmem_acc, da_lo + adv, db_hi + adv, idesc, t_sfa, t_sfb, 1);
-                        if (BP)
-                            ptx::mma_mxf4(tmem_acc, da_hi + adv, db_lo + adv, idesc, t_sfa, t_sfb, 1);
-                        if (AP && BP)
-                            ptx::mma_mxf4(tmem_acc, da_lo + adv, db_lo + adv, idesc, t_sfa, t_sfb, 1);
+                uint32_t accumulate = 0;
+                for (int kt = 0; kt < ktiles && ok; ++kt, ++c) {
+                    const int s = c % S;
+                    const uint32_t ph = (c / S) & 1;
+                    if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit) ||
+                        !ptx::mbar_wait(&ready[s], ph, abort, kWaitLimit)) {
+                        if (lane == 0) give_up(abort, prm.status, 0x200 + s);
+                        ok = false;
+                        break;
                     }
+                    const uint64_t da_hi = ptx::smem_desc_sw128(ptx::smem_u32(a_hi(s)));
+                    const uint64_t db_hi = ptx::smem_desc_sw128(ptx::smem_u32(b_hi(s)));
+                    const uint64_t da_lo = AP ? ptx::smem_desc_sw128(ptx::smem_u32(a_lo(s))) : 0;
+                    const uint64_t db_lo = BP ? ptx::smem_desc_sw128(ptx::smem_u32(b_lo(s))) : 0;
+                    const uint64_t d_sfa = ptx::smem_desc_sf(ptx::smem_u32(sfa(s)));
+                    const uint64_t d_sfb = ptx::smem_desc_sf(ptx::smem_u32(sfb(s)));
+                    const int groups = (prm.K - kt * BK) >= BK ? 2 : 1;  // K % 128 == 0
+                    if (ptx::elect_one()) {
+                        for (int g = 0; g < groups; ++g) {
+                            const uint32_t t_sfa = tmem_sfa + 4 * g;
+                            const uint32_t t_sfb = tmem_sfb + (BN / 32) * g;
+                            ptx::tc_cp_sf(t_sfa, d_sfa + (uint64_t)(512 * g >> 4));
+#pragma unroll
+                            for (int h = 0; h < BN / 128; ++h)
+                                ptx::tc_cp_sf(t_sfb + 4 * h,
+                                              d_sfb + (uint64_t)((1024 * h + 512 * g) >> 4));
+#pragma unroll
+                            for (int kk = 0; kk < 2; ++kk) {
+                                // 64 elements = 32 bytes per MMA: advance the start address
+                                const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
+                                const uint32_t idesc =
+                                    ptx::idesc_block_scaled(1, 1, BM, BN, 2 * kk, 2 * kk);
+                                ptx::mma_mxf4(tmem_acc, da_hi + adv, db_hi + adv, idesc, t_sfa,
+                                              t_sfb, accumulate | (uint32_t)(g | kk));
+                                if (AP)
+                                    ptx::mma_mxf4(tmem_acc, da_lo + adv, db_hi + adv, idesc,
+                                                  t_sfa, t_sfb, 1);
+                                if (BP)
+                                    ptx::mma_mxf4(tmem_acc, da_hi + adv, db_lo + adv, idesc,
+                                                  t_sfa, t_sfb, 1);
+                                if (AP && BP)
+                                    ptx::mma_mxf4(tmem_acc, da_lo + adv, db_lo + adv, idesc,
+                                                  t_sfa, t_sfb, 1);
+                            }
+                        }
+                        ptx::tc_commit(&empty[s]);
+                    }
+                    __syncwarp();
+                    accumulate = 1;
                 }
-                ptx::tc_commit(&empty[s]);
+                if (ok) {
+                    if (ptx::elect_one()) ptx::tc_commit(acc_full);
+                    __syncwarp();
+                }
             }
-            if (ok) ptx::tc_commit(acc_full);
+        }
+    } else if (warp < 2 + kAuxThreads / 32) {
+        // ------------------------------------------------------------------ aux threads
+        const int t = threadIdx.x - 64;  // 0..127: A row t, B rows t (+128) of the tile
+        const uint32_t sf_off = (uint32_t)(t & 31) * 16u + (uint32_t)(t >> 5) * 4u;
+        const int kgroups = (ktiles + kPrefetch - 1) / kPrefetch;
+        // scale / index bytes are fetched a whole group of K tiles ahead of their use so that
+        // the global-load latency never sits on the per-tile critical path
+        auto load_group = [&](RowBytes<H, kPrefetch>& rb, int tile, int kg) {
+            const int64_t arow = (int64_t)(tile % tiles_m) * BM + t;
+            const int64_t brow0 = (int64_t)(tile / tiles_m) * BN + t;
+#pragma unroll
+            for (int g = 0; g < kPrefetch; ++g) {
+                const int j0 = (kg * kPrefetch + g) * 8;
+                rb.sa[g] = load_row_bytes(prm.a_scales, arow, prm.M, nbk, j0, 0u);
+                rb.ia[g] = AP ? load_row_bytes(prm.a_index, arow, prm.M, nbk, j0, 0u)
+                              : make_uint2(0, 0);
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    rb.sb[h][g] = load_row_bytes(prm.b_scales, brow0 + 128 * h, prm.N, nbk, j0, 0u);
+                    rb.ib[h][g] = BP ? load_row_bytes(prm.b_index, brow0 + 128 * h, prm.N, nbk, j0, 0u)
+                                     : make_uint2(0, 0);
+                }
+            }
+        };
+        RowBytes<H, kPrefetch> cur, nxt;
+        uint32_t c = 0;
+        bool ok = true;
+        if ((int)blockIdx.x < num_tiles) load_group(cur, blockIdx.x, 0);
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            const int64_t arow = (int64_t)(tile % tiles_m) * BM + t;
+            const int64_t brow0 = (int64_t)(tile / tiles_m) * BN + t;
+            for (int kg = 0; kg < kgroups && ok; ++kg) {
+                // issue the loads of the following group (possibly of the next tile) first
+                if (kg + 1 < kgroups)
+                    load_group(nxt, tile, kg + 1);
+                else if (tile + (int)gridDim.x < num_tiles)
+                    load_group(nxt, tile + gridDim.x, 0);
+#pragma unroll
+                for (int g = 0; g < kPrefetch; ++g) {
+                    const int kt = kg * kPrefetch + g;
+                    if (kt >= ktiles || !ok) continue;
+                    const int s = c % S;
+                    const uint32_t use = c / S;
+                    ++c;
+                    if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
+                        give_up(abort, prm.status, 0x300 + s);
+                        ok = false;
+                        continue;
+                    }
+                    // scale atoms: row r -> 16-byte line r % 32, word r / 32; one per K group
+                    *reinterpret_cast<uint32_t*>(sfa(s) + sf_off) = cur.sa[g].x;
+                    *reinterpret_cast<uint32_t*>(sfa(s) + 512 + sf_off) = cur.sa[g].y;
+#pragma unroll
+                    for (int h = 0; h < H; ++h) {
+                        *reinterpret_cast<uint32_t*>(sfb(s) + 1024 * h + sf_off) = cur.sb[h][g].x;
+                        *reinterpret_cast<uint32_t*>(sfb(s) + 1024 * h + 512 + sf_off) =
+                            cur.sb[h][g].y;
+                    }
+                    if (AP || BP) {
+                        if (use > 0) {  // undo the residual nibbles of the stage's previous use
+                            if (AP)
+                                clear_row(a_lo(s), t,
+                                          *reinterpret_cast<const uint2*>(prev_a(s) + t * 8));
+                            if (BP)
+#pragma unroll
+                                for (int h = 0; h < H; ++h)
+                                    clear_row(b_lo(s), t + 128 * h,
+                                              *reinterpret_cast<const uint2*>(prev_b(s) +
+                                                                              (t + 128 * h) * 8));
+                        }
+                        if (!ptx::mbar_wait(&full[s], use & 1, abort, kWaitLimit)) {
+                            give_up(abort, prm.status, 0x400 + s);
+                            ok = false;
+                            continue;
+                        }
+                        const int nblocks = min(8, nbk - kt * 8);
+                        if (AP) {
+                            if (arow < prm.M)
+                                patch_row(a_hi(s), a_lo(s), t, cur.ia[g], cur.sa[g], nblocks);
+                            *reinterpret_cast<uint2*>(prev_a(s) + t * 8) = cur.ia[g];
+                        }
+                        if (BP) {
+#pragma unroll
+                            for (int h = 0; h < H; ++h) {
+                                if (brow0 + 128 * h < prm.N)
+                                    patch_row(b_hi(s), b_lo(s), t + 128 * h, cur.ib[h][g],
+                                              cur.sb[h][g], nblocks);
+                                *reinterpret_cast<uint2*>(prev_b(s) + (t + 128 * h) * 8) =
+                                    cur.ib[h][g];
+                            }
+                        }
+                    }
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(&ready[s]);
+                }
+                cur = nxt;
+            }
         }
     } else {
-        // ------------------------------------------------------------------ aux threads
-        const int t = threadIdx.x - 64;  // 0..127: A row t, B rows t (+128)
-        const int64_t arow = (int64_t)m0 + t;
+        // ------------------------------------------------------------------ epilogue warps
+        // The accumulator is copied out of TMEM into registers (converted on the way), then
+        // handed back to the MMA warp before the global stores are issued, so that the next
+        // tile's main loop overlaps this tile's output.
+        const int q = warp & 3;             // TMEM lane quarter this warp may read
+        const int half = (warp - 6) >> 2;   // which half of the tile's columns
+        constexpr int kColsPerThread = BN / 2;
+        constexpr int kColsPerPass = (sizeof(OutT) == 2) ? kColsPerThread : 64;
+        constexpr int kPasses = kColsPerThread / kColsPerPass;
+        constexpr int kRegs = kColsPerPass * (int)sizeof(OutT) / 4;
+        uint32_t ti = 0;
         bool ok = true;
-        uint2 sa = load_row_bytes(prm.a_scales, arow, prm.M, nbk, 0, 0u);
-        uint2 ia = AP ? load_row_bytes(prm.a_index, arow, prm.M, nbk, 0, 0u) : make_uint2(0, 0);
-        uint2 sbv[kBRowsPerThread], ibv[kBRowsPerThread];
-#pragma unroll
-        for (int h = 0; h < kBRowsPerThread; ++h) {
-            const int64_t brow = (int64_t)n0 + t + 128 * h;
-            sbv[h] = load_row_bytes(prm.b_scales, brow, prm.N, nbk, 0, 0u);
-            ibv[h] = BP ? load_row_bytes(prm.b_index, brow, prm.N, nbk, 0, 0u) : make_uint2(0, 0);
-        }
-        const uint32_t sf_off = (uint32_t)(t & 31) * 16u + (uint32_t)(t >> 5) * 4u;
-        for (int kt = 0; kt < ktiles && ok; ++kt) {
-            const int s = kt % S;
-            const uint32_t use = kt / S;
-            // prefetch the next tile's bytes while this one is processed
-            const int jn = (kt + 1) * 8;
-            const uint2 sa_n = load_row_bytes(prm.a_scales, arow, prm.M, nbk, jn, 0u);
-            const uint2 ia_n = AP ? load_row_bytes(prm.a_index, arow, prm.M, nbk, jn, 0u)
-                                  : make_uint2(0, 0);
-            uint2 sb_n[kBRowsPerThread], ib_n[kBRowsPerThread];
-#pragma unroll
-            for (int h = 0; h < kBRowsPerThread; ++h) {
-                const int64_t brow = (int64_t)n0 + t + 128 * h;
-                sb_n[h] = load_row_bytes(prm.b_scales, brow, prm.N, nbk, jn, 0u);
-                ib_n[h] = BP ? load_row_bytes(prm.b_index, brow, prm.N, nbk, jn, 0u)
-                             : make_uint2(0, 0);
-            }
-            if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
-                give_up(abort, prm.status, 0x300 + s);
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
+            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+            if (!ptx::mbar_wait(acc_full, ti & 1, abort, kWaitLimit)) {
+                give_up(abort, prm.status, 0x500);
                 ok = false;
                 break;
             }
-            // scale atoms: row r -> 16-byte line r % 32, word r / 32; one atom per K group
-            *reinterpret_cast<uint32_t*>(sfa(s) + sf_off) = sa.x;
-            *reinterpret_cast<uint32_t*>(sfa(s) + 512 + sf_off) = sa.y;
+            ptx::tc_fence_after_sync();
+            const int row = m0 + 32 * q + lane;
+            const int cbase = half * kColsPerThread;
+            OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0 + cbase;
 #pragma unroll
-            for (int h = 0; h < kBRowsPerThread; ++h) {
-                *reinterpret_cast<uint32_t*>(sfb(s) + 1024 * h + sf_off) = sbv[h].x;
-                *reinterpret_cast<uint32_t*>(sfb(s) + 1024 * h + 512 + sf_off) = sbv[h].y;
-            }
-            if (AP || BP) {
-                if (use > 0) {  // undo the residual nibbles of the stage's previous use
-                    if (AP)
-                        clear_row(a_lo(s), t, *reinterpret_cast<const uint2*>(prev_a(s) + t * 8));
-                    if (BP)
+            for (int pass = 0; pass < kPasses; ++pass) {
+                uint32_t out[kRegs];
 #pragma unroll
-                        for (int h = 0; h < kBRowsPerThread; ++h)
-                            clear_row(b_lo(s), t + 128 * h,
-                                      *reinterpret_cast<const uint2*>(prev_b(s) + (t + 128 * h) * 8));
-                }
-                if (!ptx::mbar_wait(&full[s], use & 1, abort, kWaitLimit)) {
-                    give_up(abort, prm.status, 0x400 + s);
-                    ok = false;
-                    break;
-                }
-                const int nblocks = min(8, nbk - kt * 8);
-                if (AP) {
-                    if (arow < prm.M) patch_row(a_hi(s), a_lo(s), t, ia, sa, nblocks);
-                    // rows beyond M and blocks beyond K leave nothing to clear next time:
-                    // remember index bytes only where a patch may have been written
-                    *reinterpret_cast<uint2*>(prev_a(s) + t * 8) = ia;
-                }
-                if (BP) {
+                for (int cb = 0; cb < kColsPerPass / 16; ++cb) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16(tmem_acc + ((uint32_t)(32 * q) << 16) + cbase +
+                                           pass * kColsPerPass + 16 * cb,
+                                       r);
+                    ptx::tmem_ld_wait();
+                    if (sizeof(OutT) == 4) {
 #pragma unroll
-                    for (int h = 0; h < kBRowsPerThread; ++h) {
-                        const int64_t brow = (int64_t)n0 + t + 128 * h;
-                        if (brow < prm.N)
-                            patch_row(b_hi(s), b_lo(s), t + 128 * h, ibv[h], sbv[h], nblocks);
-                        *reinterpret_cast<uint2*>(prev_b(s) + (t + 128 * h) * 8) = ibv[h];
+                        for (int i = 0; i < 16; ++i) out[16 * cb + i] = r[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(
+                                __uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                            out[8 * cb + i] = *reinterpret_cast<const uint32_t*>(&h2);
+                        }
                     }
                 }
-            }
-            ptx::fence_proxy_async_smem();
-            ptx::mbar_arrive(&ready[s]);
-            sa = sa_n;
-            ia = ia_n;
-#pragma unroll
-            for (int h = 0; h < kBRowsPerThread; ++h) {
-                sbv[h] = sb_n[h];
-                ibv[h] = ib_n[h];
-            }
-        }
-
-        // ------------------------------------------------------------------ epilogue
-        if (ok && !ptx::mbar_wait(acc_full, 0, abort, kWaitLimit)) {
-            give_up(abort, prm.status, 0x500);
-            ok = false;
-        }
-        if (ok) {
-            ptx::tc_fence_after_sync();
-            const int q = warp & 3;  // TMEM lane quarter this warp may read
-            const int row = m0 + 32 * q + lane;
-            OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(32 * q) << 16) + 32 * c, r);
-                ptx::tmem_ld_wait();
-                const int col0 = n0 + 32 * c;
+                if (pass == kPasses - 1) {
+                    // every column of the accumulator is in registers: release it
+                    ptx::tc_fence_before_sync();
+                    ptx::mbar_arrive(acc_empty);
+                }
+                const int col0 = n0 + cbase + pass * kColsPerPass;
                 if (row < prm.M && col0 < prm.N) {
-                    if (col0 + 32 <= prm.N && prm.d_vec_ok) {
-                        if (sizeof(OutT) == 4) {
-                            uint4* p = reinterpret_cast<uint4*>(drow + 32 * c);
+                    OutT* dp = drow + pass * kColsPerPass;
+                    if (col0 + kColsPerPass <= prm.N && prm.d_vec_ok) {
+                        uint4* p = reinterpret_cast<uint4*>(dp);
 #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                p[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-                        } else {
-                            uint32_t w[16];
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const __nv_bfloat162 h = __floats2bfloat162_rn(
-                                    __uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
-                                w[i] = *reinterpret_cast<const uint32_t*>(&h);
-                            }
-                            uint4* p = reinterpret_cast<uint4*>(drow + 32 * c);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                p[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-                        }
+                        for (int i = 0; i < kRegs / 4; ++i)
+                            p[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2],
+                                              out[4 * i + 3]);
                     } else {
-                        for (int i = 0; i < 32 && col0 + i < prm.N; ++i) {
-                            if (sizeof(OutT) == 4)
-                                reinterpret_cast<float*>(drow)[32 * c + i] = __uint_as_float(r[i]);
-                            else
-                                reinterpret_cast<__nv_bfloat16*>(drow)[32 * c + i] =
-                                    __float2bfloat16_rn(__uint_as_float(r[i]));
+                        constexpr int kRegsPerChunk = 32 * (int)sizeof(OutT) / 4;
+#pragma unroll
+                        for (int cb = 0; cb < kColsPerPass / 32; ++cb) {
+                            if (col0 + 32 * cb >= prm.N) continue;
+#pragma unroll
+                            for (int i = 0; i < kRegsPerChunk; ++i) {
+                                const uint32_t v = out[cb * kRegsPerChunk + i];
+                                if (sizeof(OutT) == 4) {
+                                    if (col0 + 32 * cb + i < prm.N)
+                                        reinterpret_cast<float*>(dp)[32 * cb + i] = __uint_as_float(v);
+                                } else {
+                                    const int cc = col0 + 32 * cb + 2 * i;
+                                    __nv_bfloat16* d16 = reinterpret_cast<__nv_bfloat16*>(dp) + 32 * cb + 2 * i;
+                                    if (cc < prm.N) d16[0] = __ushort_as_bfloat16((unsigned short)(v & 0xFFFFu));
+                                    if (cc + 1 < prm.N) d16[1] = __ushort_as_bfloat16((unsigned short)(v >> 16));
+                                }
+                            }
                         }
                     }
                 }
@@ -435,6 +534,19 @@ EncodeFn encode_fn()
     return fn;
 }
 
+int sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 // Packed nibbles as a 2-D byte tensor [rows][K/2], boxes of 128 bytes x box_rows, 128B swizzle.
 bool make_tmap(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t K, int box_rows)
 {
@@ -462,7 +574,8 @@ mxp_status launch_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const Params
             return MXP_ERR_CUDA;
         attr_set = true;
     }
-    dim3 grid((unsigned)((prm.M + BM - 1) / BM), (unsigned)((prm.N + BN - 1) / BN));
+    const int64_t tiles = (int64_t)((prm.M + BM - 1) / BM) * ((prm.N + BN - 1) / BN);
+    const unsigned grid = (unsigned)(tiles < prm.num_sms ? tiles : prm.num_sms);
     kern<<<grid, kThreads, C::kSmem, stream>>>(ta, tb, prm);
     return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }
@@ -477,6 +590,104 @@ mxp_status launch_modes(bool ap, bool bp, const CUtensorMap& ta, const CUtensorM
     return launch_cfg<BN, false, false, OutT>(ta, tb, prm, stream);
 }
 
+
+// ------------------------------------------------------------------------------ peak probe
+// Issue-only loop: operands and scale atoms sit in shared memory (contents irrelevant), one
+// thread per CTA issues `iters` groups of two MMAs (K = 128 of FP4, or K = 64 of 8-bit
+// containers) into the same accumulator, optionally with the three scale-factor copies a
+// 128x256 tile needs per group, then commits and waits.
+template <int kKind>
+__global__ void __launch_bounds__(128, 1) peak_probe_kernel(int iters, uint32_t* status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~(uintptr_t)1023);
+    uint8_t* a_tile = smem;                 // 128 rows x 128 B
+    uint8_t* b_tile = smem + 16384;         // 256 rows x 128 B
+    uint8_t* sf = smem + 16384 + 32768;     // 3 atoms of 512 B
+    uint64_t* bar = reinterpret_cast<uint64_t*>(sf + 2048);
+    uint32_t* slot = reinterpret_cast<uint32_t*>(bar + 1);
+    __shared__ uint32_t abort_flag;
+    for (int i = threadIdx.x; i < (16384 + 32768 + 2048) / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(smem)[i] = make_uint4(0x22222222u, 0x22222222u, 0x22222222u, 0x22222222u);
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(bar, 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    ptx::fence_proxy_async_smem();
+    if (threadIdx.x < 32) {
+        ptx::tmem_alloc(slot, 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tm = *slot;
+    if (threadIdx.x == 0) {
+        const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(a_tile));
+        const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(b_tile));
+        const uint32_t t_sfa = tm + 256, t_sfb = tm + 264;
+        constexpr bool kF8 = (kKind == 1);
+        constexpr bool kCopies = (kKind >= 2);
+        for (int it = 0; it < iters; ++it) {
+            const uint32_t buf = (kKind == 3) ? (uint32_t)(it & 1) * 16u : 0u;
+            if (kCopies) {
+                ptx::tc_cp_sf(t_sfa + buf, ptx::smem_desc_sf(ptx::smem_u32(sf)));
+                ptx::tc_cp_sf(t_sfb + buf, ptx::smem_desc_sf(ptx::smem_u32(sf + 512)));
+                ptx::tc_cp_sf(t_sfb + buf + 4, ptx::smem_desc_sf(ptx::smem_u32(sf + 1024)));
+            }
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                if (kF8)
+                    ptx::mma_mxf8f6f4(tm, da + 2 * kk, db + 2 * kk,
+                                      ptx::idesc_block_scaled(3, 3, 128, 256, kk, kk), t_sfa, t_sfb,
+                                      (it | kk) ? 1u : 0u);
+                else
+                    ptx::mma_mxf4(tm, da + 2 * kk, db + 2 * kk,
+                                  ptx::idesc_block_scaled(1, 1, 128, 256, 2 * kk, 2 * kk),
+                                  t_sfa + buf, t_sfb + buf, (it | kk) ? 1u : 0u);
+            }
+        }
+        ptx::tc_commit(bar);
+        if (!ptx::mbar_wait(bar, 0, &abort_flag, kWaitLimit) && status != nullptr)
+            atomicCAS(status, 0u, (uint32_t)MXP_ERR_TIMEOUT);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tm, 512);
+    }
+}
+
+template <int kKind>
+mxp_status run_probe(int iters, double* ms, double* flops)
+{
+    const int sms = sm_count();
+    if (sms <= 0) return MXP_ERR_CUDA;
+    constexpr int kSmem = 16384 + 32768 + 2048 + 64 + 1024;
+    auto kern = peak_probe_kernel<kKind>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+        return MXP_ERR_CUDA;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return MXP_ERR_CUDA;
+    kern<<<sms, 128, kSmem>>>(8, nullptr);  // warm-up
+    cudaEventRecord(e0);
+    kern<<<sms, 128, kSmem>>>(iters, nullptr);
+    cudaEventRecord(e1);
+    cudaError_t e = cudaEventSynchronize(e1);
+    float t = 0.f;
+    cudaEventElapsedTime(&t, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+    *ms = t;
+    const double k_per_group = (kKind == 1) ? 64.0 : 128.0;
+    *flops = 2.0 * 128.0 * 256.0 * k_per_group * (double)iters * (double)sms;
+    return MXP_OK;
+}
+
 }  // namespace
 
 size_t tc_workspace_bytes(int64_t, int64_t, int64_t, mxp_mode, mxp_mode) { return kStatusBytes; }
@@ -487,7 +698,6 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
 {
     if (K % 128 != 0) return MXP_ERR_UNSUPPORTED;
     if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return MXP_ERR_UNSUPPORTED;
-    if ((N + 127) / 128 > 65535) return MXP_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(A.scales) & 3) || (reinterpret_cast<uintptr_t>(B.scales) & 3))
         return MXP_ERR_INVALID_ARG;
     const bool ap = A.mode == MXP_MODE_MXFP4_PLUS, bp = B.mode == MXP_MODE_MXFP4_PLUS;
@@ -511,6 +721,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
                    ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
     prm.status = static_cast<StatusBlock*>(workspace);
+    prm.num_sms = sm_count();
+    if (prm.num_sms <= 0) return MXP_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
         return MXP_ERR_CUDA;
     if (d_dt == MXP_F32)
@@ -520,6 +732,15 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                      : launch_modes<128, __nv_bfloat16>(ap, bp, ta, tb, prm, stream);
 }
 
-mxp_status tensor_peak_probe(int, int, double*, double*) { return MXP_ERR_UNSUPPORTED; }
+mxp_status tensor_peak_probe(int kind, int iters, double* ms, double* flops)
+{
+    switch (kind) {
+        case 0: return run_probe<0>(iters, ms, flops);
+        case 1: return run_probe<1>(iters, ms, flops);
+        case 2: return run_probe<2>(iters, ms, flops);
+        case 3: return run_probe<3>(iters, ms, flops);
+    }
+    return MXP_ERR_INVALID_ARG;
+}
 
 }  // namespace mxp
