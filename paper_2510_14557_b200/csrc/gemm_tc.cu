@@ -27,11 +27,13 @@ namespace {
 constexpr int BM = 128;             // rows of A per tile
 constexpr int BK = 256;             // elements of K per stage = 128 bytes of nibbles
 constexpr int kRowBytes = BK / 2;   // 128
-constexpr int kAuxThreads = 128;
+constexpr int kBoxRows = 64;        // rows per TMA box
+constexpr int kAuxThreads = 384;  // one per operand row of a 128 x 256 tile (A rows, then B rows)
 constexpr int kEpiThreads = 256;
-// warp 0: TMA producer, warp 1: MMA issuer, warps 2..5: aux (scales, BM patches),
-// warps 6..13: epilogue (two warps per TMEM lane quarter, half of the columns each)
+// warp 0: TMA producer, warp 1: MMA issuer, warps 2..13: aux (scales, BM patches),
+// warps 14..21: epilogue (two warps per TMEM lane quarter, half of the columns each)
 constexpr int kThreads = 64 + kAuxThreads + kEpiThreads;
+constexpr int kEpiWarp0 = 2 + kAuxThreads / 32;
 // K tiles of scale / index bytes the aux threads fetch ahead: the MX+ variants spend 2-4x as
 // long per K tile (residual passes), so half the distance hides the same latency there
 template <bool AP, bool BP>
@@ -48,14 +50,28 @@ struct Cfg {
     static constexpr int kStageData = kATile * (AP ? 2 : 1) + kBTile * (BP ? 2 : 1);
     static constexpr int kSfA = 2 * 512;               // two K groups of 128
     static constexpr int kSfB = (BN / 128) * 2 * 512;  // per 128 rows, two K groups
-    static constexpr int kPrev = (AP ? BM * 8 : 0) + (BP ? BN * 8 : 0);  // idx bytes of last use
-    static constexpr int kStageAux = kSfA + kSfB + kPrev;
+    static constexpr int kStageAux = kSfA + kSfB;
     static constexpr int kBudget = 220 * 1024;
     static constexpr int kStagesRaw = (kBudget - 1024) / (kStageData + kStageAux);
     static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
     static constexpr int kSmem = kStages * (kStageData + kStageAux) + 1024 /*barriers*/ + 1024 /*align*/;
     static_assert(kStages >= 2, "not enough shared memory for two stages");
 };
+
+// Optional in-kernel timeline (build with -DMXP_TIMELINE): CTA 0 records clock64() at a few
+// points of its first kTimelineTiles K tiles into the workspace behind the status block.
+#ifdef MXP_TIMELINE
+constexpr int kTimelineTiles = 96;
+#define MXP_TL(slot, cond)                                                     \
+    do {                                                                       \
+        if (prm.tl != nullptr && blockIdx.x == 0 && (cond) && c < (uint32_t)kTimelineTiles) \
+            prm.tl[c * 8 + (slot)] = clock64();                                \
+    } while (0)
+#else
+#define MXP_TL(slot, cond) \
+    do {                   \
+    } while (0)
+#endif
 
 struct Params {
     int M, N, K;
@@ -68,6 +84,7 @@ struct Params {
     int num_sms;
     int d_vec_ok;  // D rows are 16-byte aligned: the epilogue may use 128-bit stores
     StatusBlock* status;
+    long long* tl;  // timeline buffer (MXP_TIMELINE builds), else unused
 };
 
 __device__ __forceinline__ void give_up(volatile uint32_t* abort, StatusBlock* st, uint32_t where)
@@ -93,46 +110,56 @@ __device__ __forceinline__ uint2 load_row_bytes(const uint8_t* plane, int64_t ro
     uint2 v = make_uint2(fill, fill);
     if (plane != nullptr && row < rows) {
         const uint32_t* p = reinterpret_cast<const uint32_t*>(plane + row * (int64_t)nbk + j0);
-        if (j0 < nbk) v.x = __ldg(p);
-        if (j0 + 4 < nbk) v.y = __ldg(p + 1);
+        // volatile asm: the loads must be issued here, a whole group of K tiles before their
+        // first use; the compiler would otherwise sink them next to that use
+        if (j0 < nbk) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.x) : "l"(p));
+        if (j0 + 4 < nbk) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.y) : "l"(p + 1));
     }
     return v;
 }
 
 // ReplaceBM / MakeFragment for one operand row and K tile, in shared memory.
-//   hi: the TMA-written tile; lo: the residual tile (zero outside BM positions).
-__device__ __forceinline__ void patch_row(uint8_t* hi, uint8_t* lo, uint32_t r, uint2 idx,
-                                          uint2 sc, int nblocks)
+//   hi: the TMA-written tile row; lo: the residual tile row (zero outside BM positions).
+// `rowoff` = r * 128, `r7` = r & 7 (the swizzle phase of the row).  All byte loads are issued
+// before the first store so that the eight blocks proceed independently.
+__device__ __forceinline__ void patch_row(uint8_t* hi, uint8_t* lo, uint32_t rowoff, uint32_t r7,
+                                          uint2 idx, uint2 sc, int nblocks)
 {
+    uint32_t off[8], b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t ib = ((j < 4 ? idx.x : idx.y) >> (8 * (j & 3))) & 31u;
+        off[j] = rowoff + ((((uint32_t)j ^ r7) << 4) | (ib >> 1));
+        b[j] = hi[off[j]];
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const uint32_t ib = ((j < 4 ? idx.x : idx.y) >> (8 * (j & 3))) & 31u;
         const uint32_t sb = ((j < 4 ? sc.x : sc.y) >> (8 * (j & 3))) & 255u;
         if (j < nblocks && sb != 0u) {
-            const uint32_t off = swz(r, 16u * j + (ib >> 1));
-            const uint32_t b = hi[off];
-            const uint32_t n = (ib & 1u) ? (b >> 4) : (b & 15u);
+            const uint32_t sh = (ib & 1u) * 4u;
+            const uint32_t n = (b[j] >> sh) & 15u;
             const uint32_t h = (n & 8u) | 6u | ((n >> 2) & 1u);  // BM_H: E2M1 code 11 m2
-            const uint32_t l = (n & 8u) | (n & 3u);              // BM_L: E2M1 code 0 m1 m0
-            hi[off] = (uint8_t)((ib & 1u) ? ((b & 0x0Fu) | (h << 4)) : ((b & 0xF0u) | h));
-            lo[off] = (uint8_t)((ib & 1u) ? (l << 4) : l);
+            const uint32_t l = n & 0xBu;                         // BM_L: E2M1 code 0 m1 m0
+            hi[off[j]] = (uint8_t)((b[j] & ~(15u << sh)) | (h << sh));
+            lo[off[j]] = (uint8_t)(l << sh);
         }
     }
 }
-__device__ __forceinline__ void clear_row(uint8_t* lo, uint32_t r, uint2 idx)
+// Zeroes one 128-byte row of a residual tile (the swizzle only permutes bytes inside the row).
+// Lanes of a warp own consecutive rows (128 bytes apart = the same banks), so each lane walks
+// its row's 16-byte chunks in an order rotated by the row number: no bank conflicts.
+__device__ __forceinline__ void zero_row(uint8_t* lo, uint32_t rowoff, uint32_t r7)
 {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint32_t ib = ((j < 4 ? idx.x : idx.y) >> (8 * (j & 3))) & 31u;
-        lo[swz(r, 16u * j + (ib >> 1))] = 0;
-    }
+    for (uint32_t i = 0; i < 8; ++i)
+        *reinterpret_cast<uint4*>(lo + rowoff + ((i ^ r7) << 4)) = make_uint4(0, 0, 0, 0);
 }
 
 // Bytes of scale / index planes one aux thread holds for a group of kPrefetch K tiles.
-template <int H, int kPrefetch>
+template <int kPrefetch>
 struct RowBytes {
-    uint2 sa[kPrefetch], ia[kPrefetch];
-    uint2 sb[H][kPrefetch], ib[H][kPrefetch];
+    uint2 sc[kPrefetch], ix[kPrefetch];
 };
 
 template <int BN, bool AP, bool BP, typename OutT>
@@ -142,7 +169,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 {
     using C = Cfg<BN, AP, BP>;
     constexpr int S = C::kStages;
-    constexpr int H = BN / kAuxThreads;  // B rows per aux thread: 1 or 2
+    constexpr int kAuxUsed = BM + BN;  // aux threads that own a row of this tile shape
     constexpr int kPrefetch = Prefetch<AP, BP>::value;
 
     extern __shared__ uint8_t smem_raw[];
@@ -168,10 +195,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     };
     auto sfa = [&](int s) { return aux0 + s * C::kStageAux; };
     auto sfb = [&](int s) { return aux0 + s * C::kStageAux + C::kSfA; };
-    auto prev_a = [&](int s) { return aux0 + s * C::kStageAux + C::kSfA + C::kSfB; };
-    auto prev_b = [&](int s) {
-        return aux0 + s * C::kStageAux + C::kSfA + C::kSfB + (AP ? BM * 8 : 0);
-    };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nbk = prm.K / 32;
@@ -185,11 +208,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             ptx::mbar_init(&full[s], 1);
-            ptx::mbar_init(&ready[s], kAuxThreads);
+            ptx::mbar_init(&ready[s], kAuxUsed / 32);  // one arrival per aux warp
             ptx::mbar_init(&empty[s], 1);
         }
         ptx::mbar_init(acc_full, 1);
-        ptx::mbar_init(acc_empty, kEpiThreads);
+        ptx::mbar_init(acc_empty, kEpiThreads / 32);  // one arrival per epilogue warp
         *abort = 0u;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_a);
@@ -234,9 +257,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         ok = false;
                         break;
                     }
+                    MXP_TL(0, true);
                     ptx::mbar_arrive_expect_tx(&full[s], C::kATile + C::kBTile);
-                    ptx::tma_load_2d(a_hi(s), &tmap_a, &full[s], kt * kRowBytes, m0);
-                    ptx::tma_load_2d(b_hi(s), &tmap_b, &full[s], kt * kRowBytes, n0);
+                    // several small boxes per operand: the copy engine walks the rows of one
+                    // box in order, so more boxes in flight shorten the time to the last byte
+#pragma unroll
+                    for (int i = 0; i < BM / kBoxRows; ++i)
+                        ptx::tma_load_2d(a_hi(s) + i * kBoxRows * kRowBytes, &tmap_a, &full[s],
+                                         kt * kRowBytes, m0 + i * kBoxRows);
+#pragma unroll
+                    for (int i = 0; i < BN / kBoxRows; ++i)
+                        ptx::tma_load_2d(b_hi(s) + i * kBoxRows * kRowBytes, &tmap_b, &full[s],
+                                         kt * kRowBytes, n0 + i * kBoxRows);
                 }
             }
         }
@@ -260,12 +292,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 for (int kt = 0; kt < ktiles && ok; ++kt, ++c) {
                     const int s = c % S;
                     const uint32_t ph = (c / S) & 1;
-                    if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit) ||
+                    // with an MX+ operand every aux thread has already waited for the TMA bytes
+                    if ((!(AP || BP) && !ptx::mbar_wait(&full[s], ph, abort, kWaitLimit)) ||
                         !ptx::mbar_wait(&ready[s], ph, abort, kWaitLimit)) {
                         if (lane == 0) give_up(abort, prm.status, 0x200 + s);
                         ok = false;
                         break;
                     }
+                    MXP_TL(1, lane == 0);
                     const uint64_t da_hi = ptx::smem_desc_sw128(ptx::smem_u32(a_hi(s)));
                     const uint64_t db_hi = ptx::smem_desc_sw128(ptx::smem_u32(b_hi(s)));
                     const uint64_t da_lo = AP ? ptx::smem_desc_sw128(ptx::smem_u32(a_lo(s))) : 0;
@@ -303,6 +337,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         }
                         ptx::tc_commit(&empty[s]);
                     }
+                    MXP_TL(2, lane == 0);
                     __syncwarp();
                     accumulate = 1;
                 }
@@ -312,102 +347,94 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
             }
         }
-    } else if (warp < 2 + kAuxThreads / 32) {
+    } else if (warp < kEpiWarp0) {
         // ------------------------------------------------------------------ aux threads
-        const int t = threadIdx.x - 64;  // 0..127: A row t, B rows t (+128) of the tile
-        const uint32_t sf_off = (uint32_t)(t & 31) * 16u + (uint32_t)(t >> 5) * 4u;
-        const int kgroups = (ktiles + kPrefetch - 1) / kPrefetch;
-        // scale / index bytes are fetched a whole group of K tiles ahead of their use so that
-        // the global-load latency never sits on the per-tile critical path
-        auto load_group = [&](RowBytes<H, kPrefetch>& rb, int tile, int kg) {
-            const int64_t arow = (int64_t)(tile % tiles_m) * BM + t;
-            const int64_t brow0 = (int64_t)(tile / tiles_m) * BN + t;
-#pragma unroll
-            for (int g = 0; g < kPrefetch; ++g) {
-                const int j0 = (kg * kPrefetch + g) * 8;
-                rb.sa[g] = load_row_bytes(prm.a_scales, arow, prm.M, nbk, j0, 0u);
-                rb.ia[g] = AP ? load_row_bytes(prm.a_index, arow, prm.M, nbk, j0, 0u)
-                              : make_uint2(0, 0);
-#pragma unroll
-                for (int h = 0; h < H; ++h) {
-                    rb.sb[h][g] = load_row_bytes(prm.b_scales, brow0 + 128 * h, prm.N, nbk, j0, 0u);
-                    rb.ib[h][g] = BP ? load_row_bytes(prm.b_index, brow0 + 128 * h, prm.N, nbk, j0, 0u)
-                                     : make_uint2(0, 0);
-                }
-            }
-        };
-        RowBytes<H, kPrefetch> cur, nxt;
-        uint32_t c = 0;
-        bool ok = true;
-        if ((int)blockIdx.x < num_tiles) load_group(cur, blockIdx.x, 0);
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int64_t arow = (int64_t)(tile % tiles_m) * BM + t;
-            const int64_t brow0 = (int64_t)(tile / tiles_m) * BN + t;
-            for (int kg = 0; kg < kgroups && ok; ++kg) {
-                // issue the loads of the following group (possibly of the next tile) first
-                if (kg + 1 < kgroups)
-                    load_group(nxt, tile, kg + 1);
-                else if (tile + (int)gridDim.x < num_tiles)
-                    load_group(nxt, tile + gridDim.x, 0);
+        // One thread per operand row of the tile: u < 128 owns A row u, otherwise B row u - 128.
+        const int u = threadIdx.x - 64;
+        if (u < kAuxUsed) {
+            const bool is_a = u < BM;
+            const int r = is_a ? u : u - BM;  // row inside the A or B tile
+            const bool plus = is_a ? AP : BP;
+            const uint8_t* sc_plane = is_a ? prm.a_scales : prm.b_scales;
+            const uint8_t* ix_plane = is_a ? prm.a_index : prm.b_index;
+            const int rows_total = is_a ? prm.M : prm.N;
+            // scale atom of 128 rows: row q -> 16-byte line q % 32, word q / 32
+            const uint32_t sf_off = (is_a ? 0u : (uint32_t)C::kSfA + (uint32_t)(r >> 7) * 1024u) +
+                                    (uint32_t)(r & 31) * 16u + (uint32_t)((r & 127) >> 5) * 4u;
+            const uint32_t rowoff = (uint32_t)r * 128u, r7 = (uint32_t)r & 7u;
+            const int kgroups = (ktiles + kPrefetch - 1) / kPrefetch;
+            // scale / index bytes are fetched a whole group of K tiles ahead of their use so
+            // that the global-load latency never sits on the per-tile critical path
+            auto load_group = [&](RowBytes<kPrefetch>& rb, int tile, int kg) {
+                const int64_t row =
+                    is_a ? (int64_t)(tile % tiles_m) * BM + r : (int64_t)(tile / tiles_m) * BN + r;
 #pragma unroll
                 for (int g = 0; g < kPrefetch; ++g) {
-                    const int kt = kg * kPrefetch + g;
-                    if (kt >= ktiles || !ok) continue;
-                    const int s = c % S;
-                    const uint32_t use = c / S;
-                    ++c;
-                    if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
-                        give_up(abort, prm.status, 0x300 + s);
-                        ok = false;
-                        continue;
-                    }
-                    // scale atoms: row r -> 16-byte line r % 32, word r / 32; one per K group
-                    *reinterpret_cast<uint32_t*>(sfa(s) + sf_off) = cur.sa[g].x;
-                    *reinterpret_cast<uint32_t*>(sfa(s) + 512 + sf_off) = cur.sa[g].y;
+                    const int j0 = (kg * kPrefetch + g) * 8;
+                    rb.sc[g] = load_row_bytes(sc_plane, row, rows_total, nbk, j0, 0u);
+                    rb.ix[g] = plus ? load_row_bytes(ix_plane, row, rows_total, nbk, j0, 0u)
+                                    : make_uint2(0, 0);
+                }
+            };
+            RowBytes<kPrefetch> cur, nxt;
+            uint32_t c = 0;
+            bool ok = true;
+            if ((int)blockIdx.x < num_tiles) load_group(cur, blockIdx.x, 0);
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int64_t row =
+                    is_a ? (int64_t)(tile % tiles_m) * BM + r : (int64_t)(tile / tiles_m) * BN + r;
+                for (int kg = 0; kg < kgroups && ok; ++kg) {
+                    // issue the loads of the following group (possibly of the next tile) first
+                    if (kg + 1 < kgroups)
+                        load_group(nxt, tile, kg + 1);
+                    else if (tile + (int)gridDim.x < num_tiles)
+                        load_group(nxt, tile + gridDim.x, 0);
 #pragma unroll
-                    for (int h = 0; h < H; ++h) {
-                        *reinterpret_cast<uint32_t*>(sfb(s) + 1024 * h + sf_off) = cur.sb[h][g].x;
-                        *reinterpret_cast<uint32_t*>(sfb(s) + 1024 * h + 512 + sf_off) =
-                            cur.sb[h][g].y;
-                    }
-                    if (AP || BP) {
-                        if (use > 0) {  // undo the residual nibbles of the stage's previous use
-                            if (AP)
-                                clear_row(a_lo(s), t,
-                                          *reinterpret_cast<const uint2*>(prev_a(s) + t * 8));
-                            if (BP)
-#pragma unroll
-                                for (int h = 0; h < H; ++h)
-                                    clear_row(b_lo(s), t + 128 * h,
-                                              *reinterpret_cast<const uint2*>(prev_b(s) +
-                                                                              (t + 128 * h) * 8));
-                        }
-                        if (!ptx::mbar_wait(&full[s], use & 1, abort, kWaitLimit)) {
-                            give_up(abort, prm.status, 0x400 + s);
+                    for (int g = 0; g < kPrefetch; ++g) {
+                        const int kt = kg * kPrefetch + g;
+                        if (kt >= ktiles || !ok) continue;
+                        const int s = c % S;
+                        const uint32_t use = c / S;
+                        if (use > 0 &&
+                            !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
+                            give_up(abort, prm.status, 0x300 + s);
                             ok = false;
+                            ++c;
                             continue;
                         }
-                        const int nblocks = min(8, nbk - kt * 8);
-                        if (AP) {
-                            if (arow < prm.M)
-                                patch_row(a_hi(s), a_lo(s), t, cur.ia[g], cur.sa[g], nblocks);
-                            *reinterpret_cast<uint2*>(prev_a(s) + t * 8) = cur.ia[g];
-                        }
-                        if (BP) {
-#pragma unroll
-                            for (int h = 0; h < H; ++h) {
-                                if (brow0 + 128 * h < prm.N)
-                                    patch_row(b_hi(s), b_lo(s), t + 128 * h, cur.ib[h][g],
-                                              cur.sb[h][g], nblocks);
-                                *reinterpret_cast<uint2*>(prev_b(s) + (t + 128 * h) * 8) =
-                                    cur.ib[h][g];
+                        MXP_TL(3, u == 0);
+                        uint8_t* sfp = sfa(s) + sf_off;  // A atoms, then B atoms, per stage
+                        *reinterpret_cast<uint32_t*>(sfp) = cur.sc[g].x;
+                        *reinterpret_cast<uint32_t*>(sfp + 512) = cur.sc[g].y;
+                        if (AP || BP) {
+                            uint8_t* hi = is_a ? a_hi(s) : b_hi(s);
+                            uint8_t* lo = is_a ? a_lo(s) : b_lo(s);
+                            if (plus && use > 0)  // wipe the residual nibbles of the last use
+                                zero_row(lo, rowoff, r7);
+                            if (!ptx::mbar_wait(&full[s], use & 1, abort, kWaitLimit)) {
+                                give_up(abort, prm.status, 0x400 + s);
+                                ok = false;
+                                ++c;
+                                continue;
+                            }
+                            MXP_TL(4, u == 0);
+                            if (plus) {
+                                if (row < rows_total)
+                                    patch_row(hi, lo, rowoff, r7, cur.ix[g], cur.sc[g],
+                                              min(8, nbk - kt * 8));
                             }
                         }
+                        // every lane publishes its writes to the async proxy, then one lane
+                        // arrives for the warp (hundreds of arrivals would serialise on the barrier)
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&ready[s]);
+                        MXP_TL(5, u == 0);
+                        MXP_TL(6, u == BM);
+                        ++c;
                     }
-                    ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(&ready[s]);
+                    cur = nxt;
                 }
-                cur = nxt;
             }
         }
     } else {
@@ -415,12 +442,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // The accumulator is copied out of TMEM into registers (converted on the way), then
         // handed back to the MMA warp before the global stores are issued, so that the next
         // tile's main loop overlaps this tile's output.
-        const int q = warp & 3;             // TMEM lane quarter this warp may read
-        const int half = (warp - 6) >> 2;   // which half of the tile's columns
+        const int q = warp & 3;                     // TMEM lane quarter this warp may read
+        const int half = (warp - kEpiWarp0) >> 2;   // which half of the tile's columns
         constexpr int kColsPerThread = BN / 2;
-        constexpr int kColsPerPass = (sizeof(OutT) == 2) ? kColsPerThread : 64;
-        constexpr int kPasses = kColsPerThread / kColsPerPass;
-        constexpr int kRegs = kColsPerPass * (int)sizeof(OutT) / 4;
+        constexpr int kChunk = (sizeof(OutT) == 2) ? 64 : 32;  // columns per register batch
+        constexpr int kChunks = kColsPerThread / kChunk;
+        constexpr int kRegs = kChunk * (int)sizeof(OutT) / 4;   // 32 either way
         uint32_t ti = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++ti) {
@@ -435,58 +462,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int cbase = half * kColsPerThread;
             OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0 + cbase;
 #pragma unroll
-            for (int pass = 0; pass < kPasses; ++pass) {
+            for (int ch = 0; ch < kChunks; ++ch) {
                 uint32_t out[kRegs];
 #pragma unroll
-                for (int cb = 0; cb < kColsPerPass / 16; ++cb) {
-                    uint32_t r[16];
-                    ptx::tmem_ld_32x16(tmem_acc + ((uint32_t)(32 * q) << 16) + cbase +
-                                           pass * kColsPerPass + 16 * cb,
-                                       r);
+                for (int cb = 0; cb < kChunk / 16; ++cb) {
+                    uint32_t rr[16];
+                    ptx::tmem_ld_32x16(
+                        tmem_acc + ((uint32_t)(32 * q) << 16) + cbase + ch * kChunk + 16 * cb, rr);
                     ptx::tmem_ld_wait();
                     if (sizeof(OutT) == 4) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) out[16 * cb + i] = r[i];
+                        for (int i = 0; i < 16; ++i) out[16 * cb + i] = rr[i];
                     } else {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const __nv_bfloat162 h2 = __floats2bfloat162_rn(
-                                __uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                                __uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1]));
                             out[8 * cb + i] = *reinterpret_cast<const uint32_t*>(&h2);
                         }
                     }
                 }
-                if (pass == kPasses - 1) {
-                    // every column of the accumulator is in registers: release it
+                if (ch == kChunks - 1) {
+                    // the last columns are in registers: hand the accumulator back
                     ptx::tc_fence_before_sync();
-                    ptx::mbar_arrive(acc_empty);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(acc_empty);
                 }
-                const int col0 = n0 + cbase + pass * kColsPerPass;
+                const int col0 = n0 + cbase + ch * kChunk;
                 if (row < prm.M && col0 < prm.N) {
-                    OutT* dp = drow + pass * kColsPerPass;
-                    if (col0 + kColsPerPass <= prm.N && prm.d_vec_ok) {
+                    OutT* dp = drow + ch * kChunk;
+                    if (col0 + kChunk <= prm.N && prm.d_vec_ok) {
                         uint4* p = reinterpret_cast<uint4*>(dp);
 #pragma unroll
                         for (int i = 0; i < kRegs / 4; ++i)
                             p[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2],
                                               out[4 * i + 3]);
                     } else {
-                        constexpr int kRegsPerChunk = 32 * (int)sizeof(OutT) / 4;
 #pragma unroll
-                        for (int cb = 0; cb < kColsPerPass / 32; ++cb) {
-                            if (col0 + 32 * cb >= prm.N) continue;
-#pragma unroll
-                            for (int i = 0; i < kRegsPerChunk; ++i) {
-                                const uint32_t v = out[cb * kRegsPerChunk + i];
-                                if (sizeof(OutT) == 4) {
-                                    if (col0 + 32 * cb + i < prm.N)
-                                        reinterpret_cast<float*>(dp)[32 * cb + i] = __uint_as_float(v);
-                                } else {
-                                    const int cc = col0 + 32 * cb + 2 * i;
-                                    __nv_bfloat16* d16 = reinterpret_cast<__nv_bfloat16*>(dp) + 32 * cb + 2 * i;
-                                    if (cc < prm.N) d16[0] = __ushort_as_bfloat16((unsigned short)(v & 0xFFFFu));
-                                    if (cc + 1 < prm.N) d16[1] = __ushort_as_bfloat16((unsigned short)(v >> 16));
-                                }
+                        for (int i = 0; i < kRegs; ++i) {
+                            const uint32_t v = out[i];
+                            if (sizeof(OutT) == 4) {
+                                if (col0 + i < prm.N)
+                                    reinterpret_cast<float*>(dp)[i] = __uint_as_float(v);
+                            } else {
+                                __nv_bfloat16* d16 = reinterpret_cast<__nv_bfloat16*>(dp) + 2 * i;
+                                if (col0 + 2 * i < prm.N)
+                                    d16[0] = __ushort_as_bfloat16((unsigned short)(v & 0xFFFFu));
+                                if (col0 + 2 * i + 1 < prm.N)
+                                    d16[1] = __ushort_as_bfloat16((unsigned short)(v >> 16));
                             }
                         }
                     }
@@ -690,7 +713,14 @@ mxp_status run_probe(int iters, double* ms, double* flops)
 
 }  // namespace
 
-size_t tc_workspace_bytes(int64_t, int64_t, int64_t, mxp_mode, mxp_mode) { return kStatusBytes; }
+size_t tc_workspace_bytes(int64_t, int64_t, int64_t, mxp_mode, mxp_mode)
+{
+#ifdef MXP_TIMELINE
+    return kStatusBytes + (size_t)kTimelineTiles * 8 * sizeof(long long);
+#else
+    return kStatusBytes;
+#endif
+}
 
 mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                           const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
@@ -706,7 +736,7 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
         return MXP_ERR_INVALID_ARG;
     const int bn = (N > 128) ? 256 : 128;
     CUtensorMap ta, tb;
-    if (!make_tmap(&ta, A.nibbles, M, K, BM) || !make_tmap(&tb, B.nibbles, N, K, bn))
+    if (!make_tmap(&ta, A.nibbles, M, K, kBoxRows) || !make_tmap(&tb, B.nibbles, N, K, kBoxRows))
         return MXP_ERR_CUDA;
     Params prm;
     prm.M = (int)M;
@@ -721,6 +751,11 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
                    ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
     prm.status = static_cast<StatusBlock*>(workspace);
+#ifdef MXP_TIMELINE
+    prm.tl = reinterpret_cast<long long*>(static_cast<char*>(workspace) + kStatusBytes);
+#else
+    prm.tl = nullptr;
+#endif
     prm.num_sms = sm_count();
     if (prm.num_sms <= 0) return MXP_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
