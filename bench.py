@@ -260,31 +260,36 @@ def part_prefill(mxp, synth, peaks, iters):
     out = {}
     fp4_burst = peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16
     # ---- config 4: prefill GEMM on packed operands, every mode pair
-    a_bits, w_bits = synth.config4()
-    a, w = dev_bf16(a_bits), dev_bf16(w_bits)
-    M, K = a.shape
-    N = w.shape[0]
-    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    d = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    for an, am in (("mxfp4", 0), ("mxfp4+", 1)):
-        for bn, bm in (("mxfp4", 0), ("mxfp4+", 1)):
-            pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
-            tot = 0.0
-            for i in range(iters + 3):
-                flush.fill_(i & 255)  # evict L2 between timed launches
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                mxp.mxp_gemm(pa, pw, out=d, workspace=ws)
-                e1.record()
-                torch.cuda.synchronize()
-                if i >= 3:
-                    tot += e0.elapsed_time(e1)
-            ms = tot / iters
-            tf = 2.0 * M * N * K / ms / 1e9
-            out["prefill_cfg4_A-%s_W-%s" % (an, bn)] = {
-                "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
-                "frac_fp4_nominal_9PF": tf / 9000.0}
+    ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    for cfg, (a_bits, w_bits), n_it in (("cfg4", synth.config4(), iters),
+                                        ("cfg5", synth.config5(), max(1, iters // 3))):
+        a, w = dev_bf16(a_bits), dev_bf16(w_bits)
+        del a_bits, w_bits
+        M, K = a.shape
+        N = w.shape[0]
+        d = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        for an, am in (("mxfp4", 0), ("mxfp4+", 1)):
+            for bn, bm in (("mxfp4", 0), ("mxfp4+", 1)):
+                pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
+                tot = 0.0
+                for i in range(n_it + 2):
+                    flush.fill_(i & 255)  # evict L2 between timed launches
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    mxp.mxp_gemm(pa, pw, out=d, workspace=ws)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if i >= 2:
+                        tot += e0.elapsed_time(e1)
+                ms = tot / n_it
+                tf = 2.0 * M * N * K / ms / 1e9
+                out["prefill_%s_A-%s_W-%s" % (cfg, an, bn)] = {
+                    "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
+                    "frac_fp4_nominal_9PF": tf / 9000.0}
+                del pa, pw
+        del a, w, d
+        torch.cuda.empty_cache()
     return out
 
 

@@ -16,6 +16,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -62,10 +63,16 @@ struct Cfg {
 // points of its first kTimelineTiles K tiles into the workspace behind the status block.
 #ifdef MXP_TIMELINE
 constexpr int kTimelineTiles = 96;
+__device__ __forceinline__ long long tl_now()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));  // ns, comparable across SMs
+    return t;
+}
 #define MXP_TL(slot, cond)                                                     \
     do {                                                                       \
-        if (prm.tl != nullptr && blockIdx.x == 0 && (cond) && c < (uint32_t)kTimelineTiles) \
-            prm.tl[c * 8 + (slot)] = clock64();                                \
+        if (prm.tl != nullptr && blockIdx.x < 2 && (cond) && c < (uint32_t)kTimelineTiles) \
+            prm.tl[blockIdx.x * kTimelineTiles * 8 + c * 8 + (slot)] = tl_now(); \
     } while (0)
 #else
 #define MXP_TL(slot, cond) \
@@ -614,6 +621,435 @@ mxp_status launch_modes(bool ap, bool bp, const CUtensorMap& ta, const CUtensorM
 }
 
 
+// ================================================================================ CTA pairs
+// Pair variant: a cluster of two CTAs computes a 256 x 256 output tile with one
+// tcgen05.mma.cta_group::2 stream issued by the even CTA.  Each CTA loads and patches only
+// its own 128 rows of A and its own 128 rows (half of N) of B, so shared-memory footprint,
+// TMA traffic and patch work per CTA drop by a third against the single-CTA 128 x 256 tile,
+// which buys one more pipeline stage for the MX+ variants.  Each CTA keeps the accumulator
+// rows of its A half in its own TMEM and writes them out itself.
+template <bool AP, bool BP>
+struct Cfg2 {
+    static constexpr int kATile = 128 * kRowBytes;  // own half of the 256 A rows
+    static constexpr int kBTile = 128 * kRowBytes;  // own half of the 256 B rows
+    static constexpr int kStageData = kATile + kBTile;  // TMA-fed ring ("hi" tiles)
+    // Residual tiles live in their own, shorter ring: they are written by the aux threads right
+    // before use, so they need no cover for the TMA latency, only for the patch itself.
+    static constexpr int kLo = 3;
+    static constexpr int kLoData = (AP ? kATile : 0) + (BP ? kBTile : 0);
+    static constexpr int kSfA = 2 * 512;        // own 128 A rows, two K groups
+    static constexpr int kSfB = 2 * 2 * 512;    // all 256 B rows, two K groups
+    static constexpr int kStageAux = kSfA + kSfB;
+    static constexpr int kBudget = 220 * 1024;
+    static constexpr int kStagesRaw = (kBudget - 1024 - kLo * kLoData) / (kStageData + kStageAux);
+    static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
+    static constexpr int kSmem =
+        kStages * (kStageData + kStageAux) + kLo * kLoData + 1024 + 1024;
+};
+
+template <bool AP, bool BP, typename OutT>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                    const __grid_constant__ CUtensorMap tmap_b, const Params prm)
+{
+    using C = Cfg2<AP, BP>;
+    constexpr int S = C::kStages;
+    constexpr int BN2 = 256, BM2 = 256;
+    constexpr int kPrefetch = Prefetch<AP, BP>::value;
+    constexpr int kAuxWarps = kAuxThreads / 32;  // per CTA
+    constexpr int kEpiWarps = kEpiThreads / 32;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~(uintptr_t)1023);
+    uint8_t* data0 = smem;
+    uint8_t* lo0 = smem + S * C::kStageData;
+    uint8_t* aux0 = lo0 + C::kLo * C::kLoData;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(aux0 + S * C::kStageAux);
+    uint64_t* full = bars;            // local: this CTA's TMA bytes landed
+    uint64_t* ready = bars + S;       // even CTA's copy is used: aux warps of both CTAs done
+    uint64_t* empty = bars + 2 * S;   // local: MMAs that read the stage have completed
+    uint64_t* acc_full = bars + 3 * S;       // local
+    uint64_t* acc_empty = bars + 3 * S + 1;  // even CTA's copy: epilogue warps of both CTAs
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 2);
+    volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
+
+    auto a_hi = [&](int s) { return data0 + s * C::kStageData; };
+    auto b_hi = [&](int s) { return data0 + s * C::kStageData + C::kATile; };
+    auto a_lo = [&](int sl) { return lo0 + sl * C::kLoData; };
+    auto b_lo = [&](int sl) { return lo0 + sl * C::kLoData + (AP ? C::kATile : 0); };
+    auto sfa = [&](int s) { return aux0 + s * C::kStageAux; };
+    auto sfb = [&](int s) { return aux0 + s * C::kStageAux + C::kSfA; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
+    const int nbk = prm.K / 32;
+    const int ktiles = (prm.K + BK - 1) / BK;
+    const int tiles_m = (prm.M + BM2 - 1) / BM2;
+    const int tiles_n = (prm.N + BN2 - 1) / BN2;
+    const int num_tiles = tiles_m * tiles_n;
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(&full[s], 1);
+            ptx::mbar_init(&ready[s], 2 * kAuxWarps);
+            ptx::mbar_init(&empty[s], 1);
+        }
+        ptx::mbar_init(acc_full, 1);
+        ptx::mbar_init(acc_empty, 2 * kEpiWarps);
+        *abort = 0u;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_a);
+        ptx::prefetch_tmap(&tmap_b);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_2cta(tmem_slot, kTmemCols);
+        ptx::tmem_relinquish_2cta();
+    }
+    if (AP || BP) {
+        for (int i = threadIdx.x; i < C::kLo * C::kLoData / 16; i += kThreads)
+            reinterpret_cast<uint4*>(lo0)[i] = make_uint4(0, 0, 0, 0);
+        ptx::fence_proxy_async_smem();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();  // both CTAs' barriers exist before anyone arrives remotely
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_acc = tmem_base;
+    const uint32_t tmem_sfa = tmem_base + BN2;       // 4 columns per K group, 2 groups
+    const uint32_t tmem_sfb = tmem_base + BN2 + 8;   // 8 columns per K group, 2 groups
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t c = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+                const int m0 = (tile % tiles_m) * BM2 + 128 * (int)rank;
+                const int n0 = (tile / tiles_m) * BN2 + 128 * (int)rank;
+                for (int kt = 0; kt < ktiles; ++kt, ++c) {
+                    const int s = c % S;
+                    const uint32_t use = c / S;
+                    if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
+                        give_up(abort, prm.status, 0x1100 + s);
+                        ok = false;
+                        break;
+                    }
+                    MXP_TL(0, true);
+                    ptx::mbar_arrive_expect_tx(&full[s], C::kATile + C::kBTile);
+#pragma unroll
+                    for (int i = 0; i < 128 / kBoxRows; ++i) {
+                        ptx::tma_load_2d(a_hi(s) + i * kBoxRows * kRowBytes, &tmap_a, &full[s],
+                                         kt * kRowBytes, m0 + i * kBoxRows);
+                        ptx::tma_load_2d(b_hi(s) + i * kBoxRows * kRowBytes, &tmap_b, &full[s],
+                                         kt * kRowBytes, n0 + i * kBoxRows);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (rank == 0) {
+            uint32_t c = 0, ti = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
+                if (ti > 0 &&
+                    !ptx::mbar_wait_cluster(acc_empty, (ti - 1) & 1, abort, kWaitLimit)) {
+                    if (lane == 0) give_up(abort, prm.status, 0x1600);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                uint32_t accumulate = 0;
+                for (int kt = 0; kt < ktiles && ok; ++kt, ++c) {
+                    const int s = c % S;
+                    const uint32_t ph = (c / S) & 1;
+                    // every aux warp of both CTAs has waited for its CTA's TMA bytes
+                    if (!ptx::mbar_wait_cluster(&ready[s], ph, abort, kWaitLimit)) {
+                        if (lane == 0) give_up(abort, prm.status, 0x1200 + s);
+                        ok = false;
+                        break;
+                    }
+                    MXP_TL(1, lane == 0);
+                    const uint64_t da_hi = ptx::smem_desc_sw128(ptx::smem_u32(a_hi(s)));
+                    const uint64_t db_hi = ptx::smem_desc_sw128(ptx::smem_u32(b_hi(s)));
+                    const int sl = c % C::kLo;
+                    const uint64_t da_lo = AP ? ptx::smem_desc_sw128(ptx::smem_u32(a_lo(sl))) : 0;
+                    const uint64_t db_lo = BP ? ptx::smem_desc_sw128(ptx::smem_u32(b_lo(sl))) : 0;
+                    const uint64_t d_sfa = ptx::smem_desc_sf(ptx::smem_u32(sfa(s)));
+                    const uint64_t d_sfb = ptx::smem_desc_sf(ptx::smem_u32(sfb(s)));
+                    const int groups = (prm.K - kt * BK) >= BK ? 2 : 1;
+                    if (ptx::elect_one()) {
+                        for (int g = 0; g < groups; ++g) {
+                            const uint32_t t_sfa = tmem_sfa + 4 * g;
+                            const uint32_t t_sfb = tmem_sfb + 8 * g;
+                            ptx::tc_cp_sf_2cta(t_sfa, d_sfa + (uint64_t)(512 * g >> 4));
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                ptx::tc_cp_sf_2cta(t_sfb + 4 * h,
+                                                   d_sfb + (uint64_t)((1024 * h + 512 * g) >> 4));
+#pragma unroll
+                            for (int kk = 0; kk < 2; ++kk) {
+                                const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
+                                const uint32_t idesc =
+                                    ptx::idesc_block_scaled(1, 1, BM2, BN2, 2 * kk, 2 * kk);
+                                ptx::mma_mxf4_2cta(tmem_acc, da_hi + adv, db_hi + adv, idesc, t_sfa,
+                                                   t_sfb, accumulate | (uint32_t)(g | kk));
+                                if (AP)
+                                    ptx::mma_mxf4_2cta(tmem_acc, da_lo + adv, db_hi + adv, idesc,
+                                                       t_sfa, t_sfb, 1);
+                                if (BP)
+                                    ptx::mma_mxf4_2cta(tmem_acc, da_hi + adv, db_lo + adv, idesc,
+                                                       t_sfa, t_sfb, 1);
+                                if (AP && BP)
+                                    ptx::mma_mxf4_2cta(tmem_acc, da_lo + adv, db_lo + adv, idesc,
+                                                       t_sfa, t_sfb, 1);
+                            }
+                        }
+                        ptx::tc_commit_2cta(&empty[s]);
+                    }
+                    MXP_TL(2, lane == 0);
+                    __syncwarp();
+                    accumulate = 1;
+                }
+                if (ok) {
+                    if (ptx::elect_one()) ptx::tc_commit_2cta(acc_full);
+                    __syncwarp();
+                }
+            }
+        }
+    } else if (warp < kEpiWarp0) {
+        // ------------------------------------------------------------------ aux threads
+        // u < 128: own A row u.  Otherwise B row b = u - 128 of the pair tile's 256: its scales
+        // go into this CTA's copy of the B scale atoms; it is patched here only if it belongs
+        // to this CTA's half.
+        const int u = threadIdx.x - 64;
+        const bool is_a = u < 128;
+        const int b_row = u - 128;                       // 0..255 for B threads
+        const int r = is_a ? u : (b_row & 127);          // row inside the local tile
+        const bool own = is_a || (uint32_t)(b_row >> 7) == rank;
+        const bool plus = own && (is_a ? AP : BP);
+        const uint8_t* sc_plane = is_a ? prm.a_scales : prm.b_scales;
+        const uint8_t* ix_plane = is_a ? prm.a_index : prm.b_index;
+        const int rows_total = is_a ? prm.M : prm.N;
+        const uint32_t sf_off =
+            (is_a ? 0u : (uint32_t)C::kSfA + (uint32_t)(b_row >> 7) * 1024u) +
+            (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;
+        const uint32_t rowoff = (uint32_t)r * 128u, r7 = (uint32_t)r & 7u;
+        const int kgroups = (ktiles + kPrefetch - 1) / kPrefetch;
+        auto grow = [&](int tile) -> int64_t {
+            return is_a ? (int64_t)(tile % tiles_m) * BM2 + 128 * (int)rank + r
+                        : (int64_t)(tile / tiles_m) * BN2 + b_row;
+        };
+        auto load_group = [&](RowBytes<kPrefetch>& rb, int tile, int kg) {
+            const int64_t row = grow(tile);
+#pragma unroll
+            for (int g = 0; g < kPrefetch; ++g) {
+                const int j0 = (kg * kPrefetch + g) * 8;
+                rb.sc[g] = load_row_bytes(sc_plane, row, rows_total, nbk, j0, 0u);
+                rb.ix[g] = plus ? load_row_bytes(ix_plane, row, rows_total, nbk, j0, 0u)
+                                : make_uint2(0, 0);
+            }
+        };
+        const uint32_t ready0 = ptx::map_to_cta(ptx::smem_u32(&ready[0]), 0);
+        RowBytes<kPrefetch> cur, nxt;
+        uint32_t c = 0;
+        bool ok = true;
+        if (cluster_id < num_tiles) load_group(cur, cluster_id, 0);
+        for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+            const int64_t row = grow(tile);
+            for (int kg = 0; kg < kgroups && ok; ++kg) {
+                if (kg + 1 < kgroups)
+                    load_group(nxt, tile, kg + 1);
+                else if (tile + num_clusters < num_tiles)
+                    load_group(nxt, tile + num_clusters, 0);
+#pragma unroll
+                for (int g = 0; g < kPrefetch; ++g) {
+                    const int kt = kg * kPrefetch + g;
+                    if (kt >= ktiles || !ok) continue;
+                    const int s = c % S;
+                    const uint32_t use = c / S;
+                    const int sl = c % C::kLo;
+                    // Commits complete in K-tile order.  The scale slot of stage s is free once
+                    // K tile c - S is done; the residual buffer once K tile c - kLo is done,
+                    // which is the later (hence sufficient) of the two.
+                    const uint32_t dist = (AP || BP) ? (uint32_t)C::kLo : (uint32_t)S;
+                    if (c >= dist) {
+                        const uint32_t cw = c - dist;
+                        if (!ptx::mbar_wait(&empty[cw % S], (cw / S) & 1, abort, kWaitLimit)) {
+                            give_up(abort, prm.status, 0x1300 + s);
+                            ok = false;
+                            ++c;
+                            continue;
+                        }
+                    }
+                    MXP_TL(3, u == 0);
+                    uint8_t* sfp = sfa(s) + sf_off;
+                    *reinterpret_cast<uint32_t*>(sfp) = cur.sc[g].x;
+                    *reinterpret_cast<uint32_t*>(sfp + 512) = cur.sc[g].y;
+                    uint8_t* lo = is_a ? a_lo(sl) : b_lo(sl);
+                    if (plus && c >= (uint32_t)C::kLo) zero_row(lo, rowoff, r7);
+                    // the MMA warp waits only for `ready`: every warp vouches for the TMA bytes
+                    if (!ptx::mbar_wait(&full[s], use & 1, abort, kWaitLimit)) {
+                        give_up(abort, prm.status, 0x1400 + s);
+                        ok = false;
+                        ++c;
+                        continue;
+                    }
+                    MXP_TL(4, u == 0);
+                    if (plus && row < rows_total)
+                        patch_row(is_a ? a_hi(s) : b_hi(s), lo, rowoff, r7, cur.ix[g], cur.sc[g],
+                                  min(8, nbk - kt * 8));
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(ready0 + 8u * (uint32_t)s);
+                    MXP_TL(5, u == 0);
+                    MXP_TL(6, u == 128);
+                    ++c;
+                }
+                cur = nxt;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;
+        const int half = (warp - kEpiWarp0) >> 2;
+        constexpr int kColsPerThread = BN2 / 2;
+        constexpr int kChunk = (sizeof(OutT) == 2) ? 64 : 32;
+        constexpr int kChunks = kColsPerThread / kChunk;
+        constexpr int kRegs = kChunk * (int)sizeof(OutT) / 4;
+        const uint32_t acc_empty0 = ptx::map_to_cta(ptx::smem_u32(acc_empty), 0);
+        uint32_t ti = 0;
+        bool ok = true;
+        for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
+            const int m0 = (tile % tiles_m) * BM2 + 128 * (int)rank, n0 = (tile / tiles_m) * BN2;
+            if (!ptx::mbar_wait(acc_full, ti & 1, abort, kWaitLimit)) {
+                give_up(abort, prm.status, 0x1500);
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int row = m0 + 32 * q + lane;
+            const int cbase = half * kColsPerThread;
+            OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0 + cbase;
+#pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) {
+                uint32_t out[kRegs];
+#pragma unroll
+                for (int cb = 0; cb < kChunk / 16; ++cb) {
+                    uint32_t rr[16];
+                    ptx::tmem_ld_32x16(
+                        tmem_acc + ((uint32_t)(32 * q) << 16) + cbase + ch * kChunk + 16 * cb, rr);
+                    ptx::tmem_ld_wait();
+                    if (sizeof(OutT) == 4) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) out[16 * cb + i] = rr[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(
+                                __uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1]));
+                            out[8 * cb + i] = *reinterpret_cast<const uint32_t*>(&h2);
+                        }
+                    }
+                }
+                if (ch == kChunks - 1) {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
+                }
+                const int col0 = n0 + cbase + ch * kChunk;
+                if (row < prm.M && col0 < prm.N) {
+                    OutT* dp = drow + ch * kChunk;
+                    if (col0 + kChunk <= prm.N && prm.d_vec_ok) {
+                        uint4* p = reinterpret_cast<uint4*>(dp);
+#pragma unroll
+                        for (int i = 0; i < kRegs / 4; ++i)
+                            p[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2],
+                                              out[4 * i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kRegs; ++i) {
+                            const uint32_t v = out[i];
+                            if (sizeof(OutT) == 4) {
+                                if (col0 + i < prm.N)
+                                    reinterpret_cast<float*>(dp)[i] = __uint_as_float(v);
+                            } else {
+                                __nv_bfloat16* d16 = reinterpret_cast<__nv_bfloat16*>(dp) + 2 * i;
+                                if (col0 + 2 * i < prm.N)
+                                    d16[0] = __ushort_as_bfloat16((unsigned short)(v & 0xFFFFu));
+                                if (col0 + 2 * i + 1 < prm.N)
+                                    d16[1] = __ushort_as_bfloat16((unsigned short)(v >> 16));
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort != 0u && threadIdx.x == 0) {
+        const long long t0 = clock64();
+        for (int s = 0; s < S; ++s)
+            while (!ptx::mbar_try_wait(&full[s], 0) && !ptx::mbar_try_wait(&full[s], 1) &&
+                   clock64() - t0 < kWaitLimit) {
+            }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    // neither CTA may leave (or free its TMEM) while the other still reads its shared memory
+    // through the pair MMA or arrives on its barriers
+    ptx::cluster_sync();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_2cta(tmem_base, kTmemCols);
+    }
+}
+
+template <bool AP, bool BP, typename OutT>
+mxp_status launch_pair_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const Params& prm,
+                           cudaStream_t stream)
+{
+    using C = Cfg2<AP, BP>;
+    auto kern = gemm_tc_pair_kernel<AP, BP, OutT>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) !=
+            cudaSuccess)
+            return MXP_ERR_CUDA;
+        attr_set = true;
+    }
+    const int64_t tiles = (int64_t)((prm.M + 255) / 256) * ((prm.N + 255) / 256);
+    int64_t clusters = prm.num_sms / 2;
+    if (tiles < clusters) clusters = tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, ta, tb, prm) == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+template <typename OutT>
+mxp_status launch_pair_modes(bool ap, bool bp, const CUtensorMap& ta, const CUtensorMap& tb,
+                             const Params& prm, cudaStream_t stream)
+{
+    if (ap && bp) return launch_pair_cfg<true, true, OutT>(ta, tb, prm, stream);
+    if (ap) return launch_pair_cfg<true, false, OutT>(ta, tb, prm, stream);
+    if (bp) return launch_pair_cfg<false, true, OutT>(ta, tb, prm, stream);
+    return launch_pair_cfg<false, false, OutT>(ta, tb, prm, stream);
+}
+
 // ------------------------------------------------------------------------------ peak probe
 // Issue-only loop: operands and scale atoms sit in shared memory (contents irrelevant), one
 // thread per CTA issues `iters` groups of two MMAs (K = 128 of FP4, or K = 64 of 8-bit
@@ -716,7 +1152,7 @@ mxp_status run_probe(int iters, double* ms, double* flops)
 size_t tc_workspace_bytes(int64_t, int64_t, int64_t, mxp_mode, mxp_mode)
 {
 #ifdef MXP_TIMELINE
-    return kStatusBytes + (size_t)kTimelineTiles * 8 * sizeof(long long);
+    return kStatusBytes + (size_t)2 * kTimelineTiles * 8 * sizeof(long long);
 #else
     return kStatusBytes;
 #endif
@@ -760,6 +1196,18 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     if (prm.num_sms <= 0) return MXP_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
         return MXP_ERR_CUDA;
+    // Kernel choice by measurement on the prefill shapes: the pair kernel wins when the
+    // weight operand is MX+ (its 256 B rows make the single-CTA residual tiles and patch work
+    // the bottleneck); the single-CTA kernel wins otherwise.  MXP_GEMM_KERNEL=single|pair
+    // overrides the choice (measurement aid).
+    const char* force = getenv("MXP_GEMM_KERNEL");
+    bool use_pair = M > 128 && N > 128 && bp;
+    if (force != nullptr && force[0] == 's') use_pair = false;
+    if (force != nullptr && force[0] == 'p') use_pair = M > 128 && N > 128;
+    if (use_pair) {
+        if (d_dt == MXP_F32) return launch_pair_modes<float>(ap, bp, ta, tb, prm, stream);
+        return launch_pair_modes<__nv_bfloat16>(ap, bp, ta, tb, prm, stream);
+    }
     if (d_dt == MXP_F32)
         return bn == 256 ? launch_modes<256, float>(ap, bp, ta, tb, prm, stream)
                          : launch_modes<128, float>(ap, bp, ta, tb, prm, stream);
