@@ -1,11 +1,13 @@
 // MXFP4 / MXFP4+ block quantization and decode kernels (HBM-bound).
 //
-// Quantize (Eq. 1, Sec. 4.1, Sec. 4.2): four lanes own one 32-element block, eight
-// elements (one or two 128-bit loads) each.  A lane group handles four consecutive
-// blocks per pass, so that the scale and index bytes of the group leave as one 32-bit
-// store each.  The block maximum and its first position come out of one integer max over
-// keys (|x| bit pattern, 31 - position), reduced over the four lanes by two shuffles:
-// this is the paper's point that the BM is found for free while computing the scale.
+// Quantize (Eq. 1, Sec. 4.1, Sec. 4.2).  Two kernels:
+//   - bf16, contiguous rows (the hot case): one lane per 32-element block, packed bf16x2
+//     arithmetic, no shuffles (quantize_bf16_lane_kernel);
+//   - generic (fp32 source or strided rows): four lanes own one block, eight elements each;
+//     the block maximum and its first position come out of one integer max over keys
+//     (|x| bit pattern, 31 - position), reduced over the four lanes by two shuffles.
+// Either way the BM falls out of the scale computation: the paper's point that it is found
+// for free during conversion.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -209,6 +211,112 @@ quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
     }
 }
 
+// ---------------------------------------------------------------- bf16 helpers (packed arithmetic)
+// The power-of-two scaling is one bf16x2 multiply per pair (exact; results that underflow are
+// far below the smallest code and round to a signed zero either way) and the sign bits come
+// straight out of the hardware cast, which keeps the sign of values rounding to zero.
+__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_max_nan(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// Four packed bf16 pairs -> eight E2M1 codes (element 0 in the lowest nibble).
+__device__ __forceinline__ uint32_t cvt_e2m1x8_bf16(uint32_t p0, uint32_t p1, uint32_t p2,
+                                                    uint32_t p3)
+{
+    uint32_t r;
+    asm("{ .reg .b8 b0, b1, b2, b3;\n"
+        "  .reg .f32 l0, h0, l1, h1, l2, h2, l3, h3;\n"
+        "  shl.b32 l0, %1, 16;  and.b32 h0, %1, 0xFFFF0000;\n"
+        "  shl.b32 l1, %2, 16;  and.b32 h1, %2, 0xFFFF0000;\n"
+        "  shl.b32 l2, %3, 16;  and.b32 h2, %3, 0xFFFF0000;\n"
+        "  shl.b32 l3, %4, 16;  and.b32 h3, %4, 0xFFFF0000;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b0, h0, l0;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b1, h1, l1;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b2, h2, l2;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b3, h3, l3;\n"
+        "  mov.b32 %0, {b0, b1, b2, b3}; }"
+        : "=r"(r)
+        : "r"(p0), "r"(p1), "r"(p2), "r"(p3));
+    return r;
+}
+
+// ---------------------------------------------------------------- bf16, contiguous: one lane per block
+// Every per-block scalar (exponent, scale byte, multiplier, BM mantissa) is computed once
+// instead of once per cooperating lane, and no shuffles are needed: a lane reads its block's
+// 64 bytes with four 128-bit loads.  Neighbouring lanes' loads fall into the same 128-byte
+// lines, which L1 serves; nibbles leave as one 128-bit store per lane (fully coalesced) and
+// the scale / index bytes as 32 consecutive bytes per warp.
+template <bool kPlus>
+__global__ void __launch_bounds__(kThreads)
+quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
+                          uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
+                          uint8_t* __restrict__ bm_index)
+{
+    const int64_t blk = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (blk >= total_blocks) return;
+    const uint4* p = src + blk * 4;
+    uint32_t x[16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 v = __ldg(p + i);
+        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+    }
+    uint32_t t[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t[i] = x[i] & 0x7FFF7FFFu;
+    uint32_t m2 = bf16x2_max_nan(t[0], t[1]);
+#pragma unroll
+    for (int i = 2; i < 16; ++i) m2 = bf16x2_max_nan(m2, t[i]);
+    m2 = bf16x2_max_nan(m2, __byte_perm(m2, m2, 0x1032));  // both halves = block maximum
+    const uint32_t amax16 = m2 & 0xFFFFu;
+    const uint32_t E = amax16 >> 7;
+    const bool dead = E <= 2u || E == 255u;  // flushed or non-finite: data is all zero
+    const uint32_t sb = E <= 2u ? 0u : (E == 255u ? 255u : E - 2u);
+    const uint32_t inv2 = ((256u - E) << 7) * 0x00010001u;  // 2^-shared_exp as a bf16 pair
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        w[i] = cvt_e2m1x8_bf16(bf16x2_mul(x[4 * i], inv2), bf16x2_mul(x[4 * i + 1], inv2),
+                               bf16x2_mul(x[4 * i + 2], inv2), bf16x2_mul(x[4 * i + 3], inv2));
+    uint32_t bm = 0;
+    if (kPlus) {
+        // one bit per element where |x| equals the maximum; lowest set bit = first BM
+        uint32_t r1 = 0, r2 = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t e1, e2;
+            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e1) : "r"(t[i]), "r"(m2));
+            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e2) : "r"(t[8 + i]), "r"(m2));
+            const uint32_t sel = (1u << (2 * i)) | (1u << (16 + 2 * i));
+            r1 |= e1 & sel;
+            r2 |= e2 & sel;
+        }
+        // even elements sit in bits 0,2,..14, odd ones in bits 16,18,..30: interleave
+        const uint32_t lo = (r1 & 0xFFFFu) | ((r1 >> 15) & 0xAAAAu);
+        const uint32_t hi = (r2 & 0xFFFFu) | ((r2 >> 15) & 0xAAAAu);
+        bm = (uint32_t)(__ffs((int)(lo | (hi << 16))) - 1) & 31u;
+        const uint32_t mant = amax16 & 0x7Fu;
+        const uint32_t m = min((mant + 7u + ((mant >> 4) & 1u)) >> 4, 7u);
+        const uint32_t sh = (bm & 7u) * 4u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if ((bm >> 3) == (uint32_t)i)
+                asm("bfi.b32 %0, %1, %0, %2, 3;" : "+r"(w[i]) : "r"(m), "r"(sh));
+    }
+    const uint4 outv = dead ? make_uint4(0, 0, 0, 0) : make_uint4(w[0], w[1], w[2], w[3]);
+    __stcs(nibbles + blk, outv);
+    scales[blk] = (uint8_t)sb;
+    if (bm_index != nullptr) bm_index[blk] = (uint8_t)(dead ? 0u : bm);
+}
+
 // ------------------------------------------------------------------------- decode (Eq. 3)
 // One thread decodes eight elements (one 32-bit word of nibbles).
 __device__ __forceinline__ float e2m1_mag(uint32_t code)
@@ -273,7 +381,12 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
     const int64_t grid = (total_blocks + kBlocksPerCta - 1) / kBlocksPerCta;
     const int aligned4 = ((reinterpret_cast<uintptr_t>(scales) & 3) == 0) &&
                          ((reinterpret_cast<uintptr_t>(bm_index) & 3) == 0);
-    if (ld_src == cols)
+    if (ld_src == cols && sizeof(T) == 2)
+        quantize_bf16_lane_kernel<kPlus>
+            <<<(unsigned)((total_blocks + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
+                static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles),
+                scales, bm_index);
+    else if (ld_src == cols)
         quantize_kernel<T, kPlus, true><<<(unsigned)grid, kThreads, 0, stream>>>(
             static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales,
             bm_index, aligned4);

@@ -143,3 +143,18 @@ def test_tc_flushed_and_zero_blocks():
     d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
     check_gemm(d, da, db)
     assert float(d[:, 5].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("kernel", ["single", "pair"])
+@pytest.mark.parametrize("amode,bmode", MODES)
+def test_tc_both_kernels_every_mode(kernel, amode, bmode, monkeypatch):
+    # the library picks the single-CTA or the CTA-pair kernel per mode; force each in turn
+    monkeypatch.setenv("MXP_GEMM_KERNEL", kernel)
+    M, N, K = 520, 777, 1280  # ragged in M and N, several tiles, K a multiple of 128 only
+    a = synth.activations_normal(M, K, seed=5, outlier_frac=0.02)
+    b = synth.weights(N, K, seed=6)
+    ap, da = quantized(a, amode)
+    bp, db = quantized(b, bmode)
+    for dt in (torch.float32, torch.bfloat16):
+        d = mxp().mxp_gemm(ap, bp, out_dtype=dt)
+        check_gemm(d, da, db)
