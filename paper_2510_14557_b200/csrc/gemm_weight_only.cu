@@ -18,7 +18,7 @@
 namespace mxp {
 namespace {
 
-constexpr int kWarps = 8;
+constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kRowsPerCta = 16;
 
@@ -47,12 +47,14 @@ __device__ __forceinline__ void decode_block(const uint4 nib, uint32_t sb, uint3
                                              uint32_t (&out)[16])
 {
     const uint32_t w[4] = {nib.x, nib.y, nib.z, nib.w};
+    // Left shifts are written as multiplies so that they issue on the FMA pipe (IMAD) and
+    // leave the integer ALU pipe, which this kernel saturates first, to the mask / merge ops.
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const uint32_t x = w[j];
-        out[4 * j + 0] = ((x << 6) & 0x01C001C0u) | ((x << 12) & 0x80008000u);
-        out[4 * j + 1] = ((x << 2) & 0x01C001C0u) | ((x << 8) & 0x80008000u);
-        out[4 * j + 2] = ((x >> 2) & 0x01C001C0u) | ((x << 4) & 0x80008000u);
+        out[4 * j + 0] = ((x * 64u) & 0x01C001C0u) | ((x * 4096u) & 0x80008000u);
+        out[4 * j + 1] = ((x * 4u) & 0x01C001C0u) | ((x * 256u) & 0x80008000u);
+        out[4 * j + 2] = ((x >> 2) & 0x01C001C0u) | ((x * 16u) & 0x80008000u);
         out[4 * j + 3] = ((x >> 6) & 0x01C001C0u) | (x & 0x80008000u);
     }
     if (kPlus) {
@@ -121,14 +123,23 @@ gemm_wo_kernel(int M, int N, int K, const __nv_bfloat16* __restrict__ A, int64_t
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
     const int chunks = (nb + 3) / 4;
-    for (int c = warp; c < chunks; c += kWarps) {
-        const int b = 4 * c + t;  // this lane's block within the row
-        const bool live = b < nb;
-        uint4 wa = make_uint4(0, 0, 0, 0), wb = wa;
-        uint32_t sa = 0, sbb = 0, ia = 0, ib = 0;
-        if (live) {
-            wa = __ldcs(reinterpret_cast<const uint4*>(nibA + (int64_t)b * 16));
-            wb = __ldcs(reinterpret_cast<const uint4*>(nibB + (int64_t)b * 16));
+    // per-lane byte offsets of this lane's first block (4 * warp + t) in the two weight rows
+    const uint8_t* pA = nibA + (int64_t)(4 * warp + t) * 16;
+    const uint8_t* pB = nibB + (int64_t)(4 * warp + t) * 16;
+    const __nv_bfloat16* aBase = A + (int64_t)(4 * warp + t) * 32;
+
+    // Software pipeline: the weight bytes of the following chunk are requested before the
+    // current one is decoded, so every warp keeps two chunks of W in flight.
+    uint4 wa = make_uint4(0, 0, 0, 0), wb = wa;
+    uint32_t sa = 0, sbb = 0, ia = 0, ib = 0;
+    auto fetch = [&](int c) {
+        const int b = 4 * c + t;
+        wa = wb = make_uint4(0, 0, 0, 0);
+        sa = sbb = ia = ib = 0;
+        if (b < nb) {
+            const int64_t off = (int64_t)(c - warp) * 64;  // 4 blocks x 16 bytes per chunk
+            wa = __ldcs(reinterpret_cast<const uint4*>(pA + off));
+            wb = __ldcs(reinterpret_cast<const uint4*>(pB + off));
             sa = scA[b];
             sbb = scB[b];
             if (kPlus) {
@@ -136,13 +147,22 @@ gemm_wo_kernel(int M, int N, int K, const __nv_bfloat16* __restrict__ A, int64_t
                 ib = ixB[b];
             }
         }
+    };
+    if (warp < chunks) fetch(warp);
+    for (int c = warp; c < chunks; c += kWarps) {
+        const int b = 4 * c + t;  // this lane's block within the row
+        const bool live = b < nb;
+        const uint4 cwa = wa, cwb = wb;
+        const uint32_t csa = sa, csb = sbb, cia = ia, cib = ib;
+        if (c + kWarps < chunks) fetch(c + kWarps);
         // activations of this lane's block for column m = 8*mt + g, pair-permuted to match
         uint32_t q[kMT][16];
 #pragma unroll
         for (int mt = 0; mt < kMT; ++mt) {
             const int m = m0 + 8 * mt + g;
             const bool ok = live && m < M;
-            const uint4* ap = reinterpret_cast<const uint4*>(A + (int64_t)m * lda + (int64_t)b * 32);
+            const uint4* ap =
+                reinterpret_cast<const uint4*>(aBase + (int64_t)m * lda + (int64_t)(c - warp) * 128);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 uint4 x = make_uint4(0, 0, 0, 0);
@@ -154,8 +174,8 @@ gemm_wo_kernel(int M, int N, int K, const __nv_bfloat16* __restrict__ A, int64_t
             }
         }
         uint32_t pa[16], pb[16];
-        decode_block<kPlus>(wa, sa, ia, pa);
-        decode_block<kPlus>(wb, sbb, ib, pb);
+        decode_block<kPlus>(cwa, csa, cia, pa);
+        decode_block<kPlus>(cwb, csb, cib, pb);
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
 #pragma unroll
