@@ -28,18 +28,20 @@ namespace {
 constexpr int BM = 128;             // rows of A per tile
 constexpr int BK = 256;             // elements of K per stage = 128 bytes of nibbles
 constexpr int kRowBytes = BK / 2;   // 128
-constexpr int kBoxRows = 64;        // rows per TMA box
+constexpr int kBoxRows = 128;       // rows per TMA box (measured: best bytes/clk per SM)
 constexpr int kAuxThreads = 384;  // one per operand row of a 128 x 256 tile (A rows, then B rows)
 constexpr int kEpiThreads = 256;
 // warp 0: TMA producer, warp 1: MMA issuer, warps 2..13: aux (scales, BM patches),
 // warps 14..21: epilogue (two warps per TMEM lane quarter, half of the columns each)
 constexpr int kThreads = 64 + kAuxThreads + kEpiThreads;
 constexpr int kEpiWarp0 = 2 + kAuxThreads / 32;
-// K tiles of scale / index bytes the aux threads fetch ahead: the MX+ variants spend 2-4x as
-// long per K tile (residual passes), so half the distance hides the same latency there
+// K tiles of scale / index bytes the aux threads fetch ahead (one group).  The loads of a
+// group are issued a whole group early; a group has to last longer than a global load under
+// full TMA traffic (1-2 us), or every group boundary stalls the pipeline.  The MX+ variants
+// spend 2-4x as long per K tile, so half the distance hides the same latency there.
 template <bool AP, bool BP>
 struct Prefetch {
-    static constexpr int value = (AP || BP) ? 2 : 4;
+    static constexpr int value = (AP || BP) ? 4 : 8;
 };
 constexpr long long kWaitLimit = 4000000000ll;  // cycles (~2 s) before a wait gives up
 constexpr uint32_t kTmemCols = 512;
@@ -110,19 +112,39 @@ __device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t c)
 }
 
 // Loads the 8 scale (or index) bytes of one row for the K tile starting at block j0.
-// K % 128 == 0, so the row holds a multiple of four bytes and words are 4-byte aligned.
-__device__ __forceinline__ uint2 load_row_bytes(const uint8_t* plane, int64_t row, int rows,
-                                                int nbk, int j0, uint32_t fill)
+// `row_ptr` points at the row's first byte (nullptr for rows outside the matrix); K % 128 == 0,
+// so a row holds a multiple of four bytes and words are 4-byte aligned; with K % 256 == 0
+// (`pair_ok`) the two words of a tile can go in one 8-byte load.  The loads are volatile asm:
+// they must be issued where written, a whole group of K tiles before their first use (the
+// compiler would otherwise sink them next to that use), and they are kept to one instruction
+// per tile so that issuing a group does not itself stall the aux warp.
+__device__ __forceinline__ uint2 load_row_bytes(const uint8_t* row_ptr, int nbk, int j0, bool pair_ok)
 {
-    uint2 v = make_uint2(fill, fill);
-    if (plane != nullptr && row < rows) {
-        const uint32_t* p = reinterpret_cast<const uint32_t*>(plane + row * (int64_t)nbk + j0);
-        // volatile asm: the loads must be issued here, a whole group of K tiles before their
-        // first use; the compiler would otherwise sink them next to that use
-        if (j0 < nbk) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.x) : "l"(p));
-        if (j0 + 4 < nbk) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.y) : "l"(p + 1));
+    uint2 v = make_uint2(0u, 0u);
+    if (row_ptr != nullptr && j0 < nbk) {
+        const uint8_t* p = row_ptr + j0;
+        if (pair_ok) {
+            asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+        } else {
+            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.x) : "l"(p));
+            if (j0 + 4 < nbk) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v.y) : "l"(p + 4));
+        }
     }
     return v;
+}
+
+// Two consecutive K tiles (16 bytes) of one row in a single load; needs K % 512 == 0 (the
+// row pitch, and with it every pair start, is then 16-byte aligned).  Each load instruction
+// of a warp touches 32 different lines (one per row), so halving the instruction count halves
+// the L1 wavefronts this prefetch costs.
+__device__ __forceinline__ void load_row_bytes16(const uint8_t* row_ptr, int nbk, int j0, uint2& t0,
+                                                 uint2& t1)
+{
+    t0 = t1 = make_uint2(0u, 0u);
+    if (row_ptr != nullptr && j0 < nbk)
+        asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(t0.x), "=r"(t0.y), "=r"(t1.x), "=r"(t1.y)
+                     : "l"(row_ptr + j0));
 }
 
 // ReplaceBM / MakeFragment for one operand row and K tile, in shared memory.
@@ -372,15 +394,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int kgroups = (ktiles + kPrefetch - 1) / kPrefetch;
             // scale / index bytes are fetched a whole group of K tiles ahead of their use so
             // that the global-load latency never sits on the per-tile critical path
+            const bool pair_ok = (nbk & 7) == 0;
             auto load_group = [&](RowBytes<kPrefetch>& rb, int tile, int kg) {
                 const int64_t row =
                     is_a ? (int64_t)(tile % tiles_m) * BM + r : (int64_t)(tile / tiles_m) * BN + r;
+                const bool in = row < rows_total;
+                const uint8_t* sc_row = in ? sc_plane + row * nbk : nullptr;
+                const uint8_t* ix_row = (in && plus) ? ix_plane + row * nbk : nullptr;
+                if ((nbk & 15) == 0) {
 #pragma unroll
-                for (int g = 0; g < kPrefetch; ++g) {
-                    const int j0 = (kg * kPrefetch + g) * 8;
-                    rb.sc[g] = load_row_bytes(sc_plane, row, rows_total, nbk, j0, 0u);
-                    rb.ix[g] = plus ? load_row_bytes(ix_plane, row, rows_total, nbk, j0, 0u)
-                                    : make_uint2(0, 0);
+                    for (int g = 0; g < kPrefetch; g += 2) {
+                        const int j0 = (kg * kPrefetch + g) * 8;
+                        load_row_bytes16(sc_row, nbk, j0, rb.sc[g], rb.sc[g + 1]);
+                        load_row_bytes16(ix_row, nbk, j0, rb.ix[g], rb.ix[g + 1]);
+                    }
+                } else {
+#pragma unroll
+                    for (int g = 0; g < kPrefetch; ++g) {
+                        const int j0 = (kg * kPrefetch + g) * 8;
+                        rb.sc[g] = load_row_bytes(sc_row, nbk, j0, pair_ok);
+                        rb.ix[g] = load_row_bytes(ix_row, nbk, j0, pair_ok);
+                    }
                 }
             };
             RowBytes<kPrefetch> cur, nxt;
@@ -843,14 +877,26 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             return is_a ? (int64_t)(tile % tiles_m) * BM2 + 128 * (int)rank + r
                         : (int64_t)(tile / tiles_m) * BN2 + b_row;
         };
+        const bool pair_ok = (nbk & 7) == 0;
         auto load_group = [&](RowBytes<kPrefetch>& rb, int tile, int kg) {
             const int64_t row = grow(tile);
+            const bool in = row < rows_total;
+            const uint8_t* sc_row = in ? sc_plane + row * nbk : nullptr;
+            const uint8_t* ix_row = (in && plus) ? ix_plane + row * nbk : nullptr;
+            if ((nbk & 15) == 0) {
 #pragma unroll
-            for (int g = 0; g < kPrefetch; ++g) {
-                const int j0 = (kg * kPrefetch + g) * 8;
-                rb.sc[g] = load_row_bytes(sc_plane, row, rows_total, nbk, j0, 0u);
-                rb.ix[g] = plus ? load_row_bytes(ix_plane, row, rows_total, nbk, j0, 0u)
-                                : make_uint2(0, 0);
+                for (int g = 0; g < kPrefetch; g += 2) {
+                    const int j0 = (kg * kPrefetch + g) * 8;
+                    load_row_bytes16(sc_row, nbk, j0, rb.sc[g], rb.sc[g + 1]);
+                    load_row_bytes16(ix_row, nbk, j0, rb.ix[g], rb.ix[g + 1]);
+                }
+            } else {
+#pragma unroll
+                for (int g = 0; g < kPrefetch; ++g) {
+                    const int j0 = (kg * kPrefetch + g) * 8;
+                    rb.sc[g] = load_row_bytes(sc_row, nbk, j0, pair_ok);
+                    rb.ix[g] = load_row_bytes(ix_row, nbk, j0, pair_ok);
+                }
             }
         };
         const uint32_t ready0 = ptx::map_to_cta(ptx::smem_u32(&ready[0]), 0);
