@@ -701,11 +701,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     uint8_t* aux0 = lo0 + C::kLo * C::kLoData;
     uint64_t* bars = reinterpret_cast<uint64_t*>(aux0 + S * C::kStageAux);
     uint64_t* full = bars;            // local: this CTA's TMA bytes landed
-    uint64_t* ready = bars + S;       // even CTA's copy is used: aux warps of both CTAs done
+    uint64_t* ready = bars + S;       // local: this CTA's aux warps are done with the stage
     uint64_t* empty = bars + 2 * S;   // local: MMAs that read the stage have completed
-    uint64_t* acc_full = bars + 3 * S;       // local
-    uint64_t* acc_empty = bars + 3 * S + 1;  // even CTA's copy: epilogue warps of both CTAs
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * S + 2);
+    uint64_t* peer_ready = bars + 3 * S;     // even CTA's copy: the odd CTA's stage is ready
+    uint64_t* acc_full = bars + 4 * S;       // local
+    uint64_t* acc_empty = bars + 4 * S + 1;  // even CTA's copy: epilogue warps of both CTAs
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * S + 2);
     volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
 
     auto a_hi = [&](int s) { return data0 + s * C::kStageData; };
@@ -727,8 +728,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             ptx::mbar_init(&full[s], 1);
-            ptx::mbar_init(&ready[s], 2 * kAuxWarps);
+            ptx::mbar_init(&ready[s], kAuxWarps);
             ptx::mbar_init(&empty[s], 1);
+            ptx::mbar_init(&peer_ready[s], 1);
         }
         ptx::mbar_init(acc_full, 1);
         ptx::mbar_init(acc_empty, 2 * kEpiWarps);
@@ -800,8 +802,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 for (int kt = 0; kt < ktiles && ok; ++kt, ++c) {
                     const int s = c % S;
                     const uint32_t ph = (c / S) & 1;
-                    // every aux warp of both CTAs has waited for its CTA's TMA bytes
-                    if (!ptx::mbar_wait_cluster(&ready[s], ph, abort, kWaitLimit)) {
+                    // every aux warp has waited for its CTA's TMA bytes; the odd CTA's warps
+                    // report through its forwarder (one cluster-scope arrival per stage)
+                    if (!ptx::mbar_wait(&ready[s], ph, abort, kWaitLimit) ||
+                        !ptx::mbar_wait_cluster(&peer_ready[s], ph, abort, kWaitLimit)) {
                         if (lane == 0) give_up(abort, prm.status, 0x1200 + s);
                         ok = false;
                         break;
@@ -853,6 +857,24 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     __syncwarp();
                 }
             }
+        } else if (lane == 0) {
+            // Forwarder of the odd CTA: its aux warps arrive on a local barrier (cheap, CTA
+            // scope); this thread, which has no memory traffic of its own to drain, passes
+            // each completed stage on to the even CTA with one cluster-scope arrival.
+            const uint32_t peer_ready0 = ptx::map_to_cta(ptx::smem_u32(&peer_ready[0]), 0);
+            uint32_t c = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+                for (int kt = 0; kt < ktiles; ++kt, ++c) {
+                    const int s = c % S;
+                    if (!ptx::mbar_wait(&ready[s], (c / S) & 1, abort, kWaitLimit)) {
+                        give_up(abort, prm.status, 0x1700 + s);
+                        ok = false;
+                        break;
+                    }
+                    ptx::mbar_arrive_cluster(peer_ready0 + 8u * (uint32_t)s);
+                }
+            }
         }
     } else if (warp < kEpiWarp0) {
         // ------------------------------------------------------------------ aux threads
@@ -899,7 +921,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 }
             }
         };
-        const uint32_t ready0 = ptx::map_to_cta(ptx::smem_u32(&ready[0]), 0);
         RowBytes<kPrefetch> cur, nxt;
         uint32_t c = 0;
         bool ok = true;
@@ -950,7 +971,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                   min(8, nbk - kt * 8));
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive_cluster(ready0 + 8u * (uint32_t)s);
+                    if (lane == 0) ptx::mbar_arrive(&ready[s]);
                     MXP_TL(5, u == 0);
                     MXP_TL(6, u == 128);
                     ++c;
@@ -1242,12 +1263,12 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     if (prm.num_sms <= 0) return MXP_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
         return MXP_ERR_CUDA;
-    // Kernel choice by measurement on the prefill shapes: the pair kernel wins when the
-    // weight operand is MX+ (its 256 B rows make the single-CTA residual tiles and patch work
-    // the bottleneck); the single-CTA kernel wins otherwise.  MXP_GEMM_KERNEL=single|pair
+    // Kernel choice by measurement on the prefill shapes: the pair kernel wins whenever an
+    // operand is MX+ (a third less residual-tile memory and patch work per CTA buys pipeline
+    // depth); the single-CTA kernel wins for plain MXFP4.  MXP_GEMM_KERNEL=single|pair
     // overrides the choice (measurement aid).
     const char* force = getenv("MXP_GEMM_KERNEL");
-    bool use_pair = M > 128 && N > 128 && bp;
+    bool use_pair = M > 128 && N > 128 && (ap || bp);
     if (force != nullptr && force[0] == 's') use_pair = false;
     if (force != nullptr && force[0] == 'p') use_pair = M > 128 && N > 128;
     if (use_pair) {
