@@ -857,23 +857,25 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     __syncwarp();
                 }
             }
-        } else if (lane == 0) {
-            // Forwarder of the odd CTA: its aux warps arrive on a local barrier (cheap, CTA
-            // scope); this thread, which has no memory traffic of its own to drain, passes
-            // each completed stage on to the even CTA with one cluster-scope arrival.
-            const uint32_t peer_ready0 = ptx::map_to_cta(ptx::smem_u32(&peer_ready[0]), 0);
-            uint32_t c = 0;
-            bool ok = true;
-            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-                for (int kt = 0; kt < ktiles; ++kt, ++c) {
-                    const int s = c % S;
-                    if (!ptx::mbar_wait(&ready[s], (c / S) & 1, abort, kWaitLimit)) {
-                        give_up(abort, prm.status, 0x1700 + s);
-                        ok = false;
-                        break;
-                    }
-                    ptx::mbar_arrive_cluster(peer_ready0 + 8u * (uint32_t)s);
+        } else if (lane < S) {
+            // Forwarders of the odd CTA: its aux warps arrive on a local barrier (cheap, CTA
+            // scope); these lanes, which have no memory traffic of their own to drain, pass
+            // each completed stage on to the even CTA with one cluster-scope arrival.  A
+            // cluster-scope release takes most of a microsecond, so there is one lane per
+            // pipeline stage: their arrivals overlap, and each barrier's phases are still
+            // consumed in order by a single thread.
+            const uint32_t peer_ready_s =
+                ptx::map_to_cta(ptx::smem_u32(&peer_ready[lane]), 0);
+            int64_t my_tiles = 0;
+            for (int tile = cluster_id; tile < num_tiles; tile += num_clusters) ++my_tiles;
+            const int64_t total = my_tiles * ktiles;
+            uint32_t use = 0;
+            for (int64_t c = lane; c < total; c += S, ++use) {
+                if (!ptx::mbar_wait(&ready[lane], use & 1, abort, kWaitLimit)) {
+                    give_up(abort, prm.status, 0x1700 + lane);
+                    break;
                 }
+                ptx::mbar_arrive_cluster(peer_ready_s);
             }
         }
     } else if (warp < kEpiWarp0) {
