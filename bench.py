@@ -61,7 +61,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -384,6 +384,12 @@ def run_ours(args, M, N, K, label):
 
     fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
     achieved = flops_step / gemm_ms / 1e9
+    # issue-only tcgen05 kind::mxf4 rate on this device (operands resident in shared memory)
+    try:
+        pms, pfl = mxp.mxp_tensor_peak_probe(0, 20000)
+        probe_tflops = pfl / pms / 1e9
+    except Exception:
+        probe_tflops = None
     line = {
         "metric": METRIC, "value": flops_all / ms / 1e9, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms,
@@ -395,7 +401,8 @@ def run_ours(args, M, N, K, label):
         "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": fp4_peak,
                      "unit": "TFLOP/s", "frac": achieved / fp4_peak, "traffic": None,
                      "peak_source": "%s bf16 sustained x4 (nominal FP4:bf16 ratio)" % peaks["src"],
-                     "kernel_ms": gemm_ms},
+                     "kernel_ms": gemm_ms, "mxf4_issue_probe_tflops": probe_tflops,
+                     "frac_of_issue_probe": (achieved / probe_tflops) if probe_tflops else None},
         "e2e": {"value": e2e_flops / e2e_ms / 1e9, "unit": UNIT, "h2d_bytes_per_step": M * K * 2,
                 "d2h_bytes_per_step": M * N * 2, "ms_per_step": e2e_ms},
         "gpu_launches": 2 * args.steps,
