@@ -261,7 +261,6 @@ def part_prefill(mxp, synth, peaks, iters):
     fp4_burst = peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16
     # ---- config 4: prefill GEMM on packed operands, every mode pair
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
     for cfg, (a_bits, w_bits), n_it in (("cfg4", synth.config4(), iters),
                                         ("cfg5", synth.config5(), max(1, iters // 3))):
         a, w = dev_bf16(a_bits), dev_bf16(w_bits)
@@ -269,6 +268,8 @@ def part_prefill(mxp, synth, peaks, iters):
         M, K = a.shape
         N = w.shape[0]
         d = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros(max(4096, mxp.mxp_gemm_workspace_bytes(M, N, K, False, 1, 1)),
+                         dtype=torch.uint8, device="cuda")
         for an, am in (("mxfp4", 0), ("mxfp4+", 1)):
             for bn, bm in (("mxfp4", 0), ("mxfp4+", 1)):
                 pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
@@ -288,7 +289,7 @@ def part_prefill(mxp, synth, peaks, iters):
                     "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
                     "frac_fp4_nominal_9PF": tf / 9000.0}
                 del pa, pw
-        del a, w, d
+        del a, w, d, ws
         torch.cuda.empty_cache()
     return out
 

@@ -94,9 +94,17 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  *   B_packed   host pointer to the descriptor of the N x K weight operand
  *   D          M x N of `d_dt` (bf16 rounded to nearest even, or fp32), row stride ldd
  *              elements (ldd >= N; 16-byte aligned rows let the epilogue use wide stores)
- *   workspace  device scratch of at least mxp_gemm_workspace_bytes(...) bytes, 256-byte
- *              aligned; may be NULL when that size is 0.  Its first 16 bytes are a status
- *              block written by the kernels (see mxp_gemm_status).
+ *   workspace  device scratch, 256-byte aligned, of at least
+ *              mxp_gemm_min_workspace_bytes(...) bytes (MXP_ERR_WORKSPACE otherwise); may be
+ *              NULL when that size is 0.  With mxp_gemm_workspace_bytes(...) bytes the
+ *              tensor-core form first re-tiles the scales and, for MX+ operands, widens the
+ *              4-bit codes to E4M3 bytes (exact for every E2M1 value and for the BM values
+ *              of Eq. 3) inside the workspace and then runs its fastest kernel; with less
+ *              it runs kernels that work on the packed planes in place (Eq. 4 / Algorithm 1:
+ *              BM split and residual MMAs), which are slower.  Same result either way.
+ *              Its first 16 bytes are a status block written by the kernels (see
+ *              mxp_gemm_status).  The workspace holds nothing the caller has to keep
+ *              between calls.
  * K % 32 == 0 always; the tensor-core form further needs K % 128 == 0.
  */
 mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16, int64_t lda,
@@ -104,9 +112,12 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16, i
                     mxp_dtype d_dt, int64_t ldd, void *workspace, size_t workspace_bytes,
                     void *cuda_stream);
 
-/* Bytes of workspace mxp_gemm needs for this problem. a_dense != 0: weight-only form. */
+/* Bytes of workspace with which mxp_gemm runs its fastest kernel for this problem
+ * (a_dense != 0: weight-only form), and the least it accepts. */
 size_t mxp_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense,
                                 mxp_mode a_mode, mxp_mode b_mode);
+size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense,
+                                    mxp_mode a_mode, mxp_mode b_mode);
 
 /*
  * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM

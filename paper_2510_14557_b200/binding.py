@@ -23,7 +23,7 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_status", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_noalloc.restype = ci
         l.mxp_gemm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
         l.mxp_gemm_workspace_bytes.restype = sz
+        l.mxp_gemm_min_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
+        l.mxp_gemm_min_workspace_bytes.restype = sz
         l.mxp_gemm_status.argtypes = [vp, vp]
         l.mxp_gemm_status.restype = ci
         l.mxp_tensor_peak_probe.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_double),
@@ -149,6 +151,10 @@ def mxp_dequantize(p: Packed, dtype=torch.float32, out: Optional[torch.Tensor] =
 
 def mxp_gemm_workspace_bytes(M: int, N: int, K: int, a_dense: bool, a_mode: int, b_mode: int) -> int:
     return int(lib().mxp_gemm_workspace_bytes(M, N, K, int(a_dense), a_mode, b_mode))
+
+
+def mxp_gemm_min_workspace_bytes(M: int, N: int, K: int, a_dense: bool, a_mode: int, b_mode: int) -> int:
+    return int(lib().mxp_gemm_min_workspace_bytes(M, N, K, int(a_dense), a_mode, b_mode))
 
 
 def mxp_gemm(a, b: Packed, out_dtype=torch.bfloat16, out: Optional[torch.Tensor] = None,

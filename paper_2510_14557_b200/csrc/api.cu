@@ -80,6 +80,14 @@ size_t mxp_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense, mx
     return mxp::tc_workspace_bytes(M, N, K, a_mode, b_mode);
 }
 
+size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense, mxp_mode,
+                                    mxp_mode)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    if (a_dense) return mxp::skinny_workspace_bytes(M, N, K);
+    return mxp::tc_compact_workspace_bytes();
+}
+
 mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, int64_t lda,
                     const mxp_packed* A_packed, const mxp_packed* B_packed, void* D,
                     mxp_dtype d_dt, int64_t ldd, void* workspace, size_t workspace_bytes,
@@ -100,9 +108,9 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     if (K == 0) return MXP_ERR_UNSUPPORTED;  // an empty sum; callers zero D themselves
-    const size_t need = mxp_gemm_workspace_bytes(M, N, K, A_dense_bf16 != nullptr,
-                                                 A_packed ? A_packed->mode : MXP_MODE_MXFP4,
-                                                 B_packed->mode);
+    const size_t need = mxp_gemm_min_workspace_bytes(M, N, K, A_dense_bf16 != nullptr,
+                                                     A_packed ? A_packed->mode : MXP_MODE_MXFP4,
+                                                     B_packed->mode);
     if (need > 0) {
         if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
         if (!aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;

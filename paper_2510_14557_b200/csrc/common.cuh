@@ -1,6 +1,7 @@
 // Shared declarations of the libmxp translation units (device launchers + helpers).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -25,9 +26,25 @@ cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void*
 
 // Block-scaled tensor-core form: both operands packed.
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
+size_t tc_compact_workspace_bytes();  // enough for the kernels that work in place
 mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                           const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
                           void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+// Streamed CTA-pair kernel on prepacked operands (scale atoms, E4M3-widened MX+ data): needs
+// M, N > 128 and a workspace of stream_workspace_bytes() (0 = shape not supported).
+size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
+mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
+                                 const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                                 void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no libcuda link).
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                              const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                              const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn tensormap_encode_fn();
+int sm_count();  // of the current device, cached; -1 on error
 
 mxp_status tensor_peak_probe(int kind, int iters, double* ms, double* flops);
 

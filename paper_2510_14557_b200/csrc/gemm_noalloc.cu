@@ -63,7 +63,7 @@ extern "C" mxp_status mxp_gemm_noalloc(int64_t M, int64_t N, int64_t K, const mx
     if (reinterpret_cast<uintptr_t>(D) % (d_dt == MXP_BF16 ? 2 : 4) != 0) return MXP_ERR_INVALID_ARG;
 
     // the scratch this problem needs must fit the array the library carries
-    const size_t need = mxp::tc_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode);
+    const size_t need = mxp::tc_compact_workspace_bytes();
     if (need > kScratchBytes) return MXP_ERR_WORKSPACE;
 
     void* scratch = nullptr;

@@ -578,43 +578,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 }
 
 // ------------------------------------------------------------------------------ host side
-using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                              const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                              const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn()
-{
-    static EncodeFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
-                cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeFn>(p);
-    });
-    return fn;
-}
-
-int sm_count()
-{
-    static int cached[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
-    if (cached[dev] == 0) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
-        cached[dev] = n;
-    }
-    return cached[dev];
-}
-
 // Packed nibbles as a 2-D byte tensor [rows][K/2], boxes of 128 bytes x box_rows, 128B swizzle.
 bool make_tmap(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t K, int box_rows)
 {
-    EncodeFn fn = encode_fn();
+    EncodeFn fn = tensormap_encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
@@ -1218,7 +1185,7 @@ mxp_status run_probe(int iters, double* ms, double* flops)
 
 }  // namespace
 
-size_t tc_workspace_bytes(int64_t, int64_t, int64_t, mxp_mode, mxp_mode)
+size_t tc_compact_workspace_bytes()
 {
 #ifdef MXP_TIMELINE
     return kStatusBytes + (size_t)2 * kTimelineTiles * 8 * sizeof(long long);
@@ -1227,9 +1194,16 @@ size_t tc_workspace_bytes(int64_t, int64_t, int64_t, mxp_mode, mxp_mode)
 #endif
 }
 
+size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
+{
+    const size_t fast = stream_workspace_bytes(M, N, K, a_mode, b_mode);
+    const size_t compact = tc_compact_workspace_bytes();
+    return fast > compact ? fast : compact;
+}
+
 mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                           const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                          void* workspace, size_t, cudaStream_t stream)
+                          void* workspace, size_t workspace_bytes, cudaStream_t stream)
 {
     if (K % 128 != 0) return MXP_ERR_UNSUPPORTED;
     if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return MXP_ERR_UNSUPPORTED;
@@ -1270,6 +1244,13 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     // depth); the single-CTA kernel wins for plain MXFP4.  MXP_GEMM_KERNEL=single|pair
     // overrides the choice (measurement aid).
     const char* force = getenv("MXP_GEMM_KERNEL");
+    // Default: the streamed pair kernel on prepacked operands, when the shape allows it and
+    // the caller's workspace has room for the prepacked copies; otherwise the kernels below,
+    // which work in place and need only the status block.
+    const size_t fast = stream_workspace_bytes(M, N, K, A.mode, B.mode);
+    const bool forced_other = force != nullptr && (force[0] == 's' || force[0] == 'p');
+    if (fast != 0 && workspace_bytes >= fast && !forced_other)
+        return launch_gemm_tc_stream(M, N, K, A, B, D, d_dt, ldd, workspace, workspace_bytes, stream);
     bool use_pair = M > 128 && N > 128 && (ap || bp);
     if (force != nullptr && force[0] == 's') use_pair = false;
     if (force != nullptr && force[0] == 'p') use_pair = M > 128 && N > 128;

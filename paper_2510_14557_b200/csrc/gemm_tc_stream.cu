@@ -1,0 +1,596 @@
+// Streamed CTA-pair GEMM on prepacked operands (sm_100a).
+//
+//   D[M,N] = dec(A)[M,K] * dec(B)[N,K]^T, fp32 accumulation in tensor memory.
+//
+// Everything the tensor core reads arrives in shared memory by TMA, so no thread touches
+// operand data between HBM and the MMA.  That needs two cheap bandwidth passes first:
+//
+//   * scales: the row-major E8M0 plane is re-tiled into the 32-row x 16-byte atoms that
+//     tcgen05.cp copies into tensor memory ([row group of 128][K group of 128][512 bytes]);
+//   * MX+ operands (and their plain partner): every 4-bit code is widened to an E4M3 byte.
+//     E4M3 holds all E2M1 values and the BM values 4 + m/2 of Eq. 3 exactly, so the block's
+//     BM is simply written as 0x48 | m and one kind::mxf8f6f4 pass replaces the main MMA plus
+//     the residual MMAs of Eq. 4 / Algorithm 1.  On this GPU an 8-bit-container MMA costs two
+//     FP4 MMAs, i.e. what one MX+ operand costs with the split and half of what two cost.
+//
+// Plain MXFP4 x MXFP4 needs only the scale pass and runs kind::mxf4 on the nibble planes.
+//
+// Kernel: clusters of two CTAs, one 256 x 256 output tile per cluster and step, persistent.
+// Warp 0 of each CTA issues the TMA loads for its own 128 rows of A, 128 rows of B and the
+// scale atoms; all of them signal one mbarrier in the even CTA, whose warp 1 issues
+// tcgen05.mma.cta_group::2 and commits to both CTAs.  Warps 2-9 drain the accumulator.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <cstdlib>
+#include <mutex>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace mxp {
+
+// ------------------------------------------------------------------------------ host helpers
+EncodeFn tensormap_encode_fn()
+{
+    static EncodeFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
+                cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    });
+    return fn;
+}
+
+int sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+constexpr int kTile = 256;          // output tile of a CTA pair: 256 x 256
+constexpr int kRowBytes = 128;      // bytes of one operand row per stage (one swizzle span)
+constexpr int kHalfTile = 128 * kRowBytes;  // 16 KB: this CTA's 128 rows of A (or of B)
+constexpr int kAtom = 512;          // scale bytes of 128 rows x 4 blocks
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr long long kWaitLimit = 4000000000ll;  // cycles (~2 s) before a wait gives up
+constexpr uint32_t kTmemCols = 512;
+
+// kWide = false: rows are 256 packed E2M1 codes (two scale atoms per stage), kind::mxf4.
+// kWide = true : rows are 128 E4M3 bytes (one scale atom per stage), kind::mxf8f6f4.
+template <bool kWide>
+struct SCfg {
+    static constexpr int kGroups = kWide ? 1 : 2;           // K groups of 128 elements per stage
+    static constexpr int kSfA = kGroups * kAtom;            // own 128 rows of A
+    static constexpr int kSfB = 2 * kGroups * kAtom;        // all 256 rows of B
+    static constexpr int kStage = 2 * kHalfTile + kSfA + kSfB;
+    static constexpr int kStages = 6;
+    static constexpr int kSmem = kStages * kStage + 1024 /*barriers*/ + 1024 /*align*/;
+    static constexpr int kElemsPerStage = kWide ? 128 : 256;
+};
+
+struct SParams {
+    int M, N, K;
+    void* D;
+    int64_t ldd;
+    int d_vec_ok;
+    StatusBlock* status;
+};
+
+__device__ __forceinline__ void give_up(volatile uint32_t* abort, StatusBlock* st, uint32_t where)
+{
+    *abort = 1u;
+    if (st != nullptr) {
+        atomicCAS(&st->code, 0u, (uint32_t)MXP_ERR_TIMEOUT);
+        st->where = where;
+    }
+}
+
+template <bool kWide, typename OutT>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                      const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_sfa,
+                      const __grid_constant__ CUtensorMap tmap_sfb, const SParams prm)
+{
+    using C = SCfg<kWide>;
+    constexpr int S = C::kStages;
+    constexpr int G = C::kGroups;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * C::kStage);
+    uint64_t* full = bars;           // even CTA's copy is used: TMA bytes of both CTAs
+    uint64_t* empty = bars + S;      // local: the MMAs that read the stage have completed
+    uint64_t* acc_full = bars + 2 * S;       // local
+    uint64_t* acc_empty = bars + 2 * S + 1;  // even CTA's copy: epilogue warps of both CTAs
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 2);
+    volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
+
+    auto a_tile = [&](int s) { return smem + s * C::kStage; };
+    auto b_tile = [&](int s) { return smem + s * C::kStage + kHalfTile; };
+    auto sfa = [&](int s) { return smem + s * C::kStage + 2 * kHalfTile; };
+    auto sfb = [&](int s) { return smem + s * C::kStage + 2 * kHalfTile + C::kSfA; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
+    const int kstages = (prm.K + C::kElemsPerStage - 1) / C::kElemsPerStage;
+    const int tiles_m = (prm.M + kTile - 1) / kTile;
+    const int tiles_n = (prm.N + kTile - 1) / kTile;
+    const int num_tiles = tiles_m * tiles_n;
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(&full[s], 1);
+            ptx::mbar_init(&empty[s], 1);
+        }
+        ptx::mbar_init(acc_full, 1);
+        ptx::mbar_init(acc_empty, 2 * kEpiWarps);
+        *abort = 0u;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_a);
+        ptx::prefetch_tmap(&tmap_b);
+        ptx::prefetch_tmap(&tmap_sfa);
+        ptx::prefetch_tmap(&tmap_sfb);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_2cta(tmem_slot, kTmemCols);
+        ptx::tmem_relinquish_2cta();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();  // both CTAs' barriers exist before anything signals them remotely
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_acc = tmem_base;
+    const uint32_t tmem_sfa = tmem_base + kTile;      // 4 columns per K group
+    const uint32_t tmem_sfb = tmem_base + kTile + 8;  // 8 columns per K group
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint32_t full0 = ptx::map_to_cta(ptx::smem_u32(&full[0]), 0);
+            uint32_t c = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+                const int tm = tile % tiles_m, tn = tile / tiles_m;
+                const int m0 = tm * kTile + 128 * (int)rank;
+                const int n0 = tn * kTile + 128 * (int)rank;
+                for (int kt = 0; kt < kstages; ++kt, ++c) {
+                    const int s = c % S;
+                    const uint32_t use = c / S;
+                    if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
+                        give_up(abort, prm.status, 0x2100 + s);
+                        ok = false;
+                        break;
+                    }
+#ifdef MXP_EXP_NOTMA
+                    if (rank == 0) ptx::mbar_arrive(&full[s]);
+                    continue;
+#endif
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * C::kStage);
+                    ptx::tma_load_2d_pair(a_tile(s), &tmap_a, full0 + 8u * (uint32_t)s, kt * kRowBytes, m0);
+                    ptx::tma_load_2d_pair(b_tile(s), &tmap_b, full0 + 8u * (uint32_t)s, kt * kRowBytes, n0);
+                    ptx::tma_load_3d_pair(sfa(s), &tmap_sfa, full0 + 8u * (uint32_t)s, 0, kt * G, 2 * tm + (int)rank);
+                    ptx::tma_load_3d_pair(sfb(s), &tmap_sfb, full0 + 8u * (uint32_t)s, 0, kt * G, 2 * tn);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (rank == 0) {
+            uint32_t c = 0, ti = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
+                if (ti > 0 &&
+                    !ptx::mbar_wait_cluster(acc_empty, (ti - 1) & 1, abort, kWaitLimit)) {
+                    if (lane == 0) give_up(abort, prm.status, 0x2600);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                uint32_t accumulate = 0;
+                for (int kt = 0; kt < kstages && ok; ++kt, ++c) {
+                    const int s = c % S;
+                    const uint32_t ph = (c / S) & 1;
+                    if (!ptx::mbar_wait_cluster(&full[s], ph, abort, kWaitLimit)) {
+                        if (lane == 0) give_up(abort, prm.status, 0x2200 + s);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(a_tile(s)));
+                    const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(b_tile(s)));
+                    const uint64_t d_sfa = ptx::smem_desc_sf(ptx::smem_u32(sfa(s)));
+                    const uint64_t d_sfb = ptx::smem_desc_sf(ptx::smem_u32(sfb(s)));
+                    const int groups =
+                        kWide ? 1 : ((prm.K - kt * C::kElemsPerStage) >= C::kElemsPerStage ? 2 : 1);
+                    if (ptx::elect_one()) {
+#ifdef MXP_EXP_NOMMA
+                        for (int g = 0; g < 0; ++g) {
+#else
+                        for (int g = 0; g < groups; ++g) {
+#endif
+                            const uint32_t t_sfa = tmem_sfa + 4 * g;
+                            const uint32_t t_sfb = tmem_sfb + 8 * g;
+                            ptx::tc_cp_sf_2cta(t_sfa, d_sfa + (uint64_t)(kAtom * g >> 4));
+#pragma unroll
+                            for (int h = 0; h < 2; ++h)
+                                ptx::tc_cp_sf_2cta(t_sfb + 4 * h,
+                                                   d_sfb + (uint64_t)((G * kAtom * h + kAtom * g) >> 4));
+                            if (kWide) {
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const uint32_t idesc =
+                                        ptx::idesc_block_scaled(0, 0, kTile, kTile, kk, kk);
+                                    ptx::mma_mxf8f6f4_2cta(tmem_acc, da + (uint64_t)(2 * kk),
+                                                           db + (uint64_t)(2 * kk), idesc, t_sfa,
+                                                           t_sfb, accumulate | (uint32_t)kk);
+                                }
+                            } else {
+#pragma unroll
+                                for (int kk = 0; kk < 2; ++kk) {
+                                    const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
+                                    const uint32_t idesc =
+                                        ptx::idesc_block_scaled(1, 1, kTile, kTile, 2 * kk, 2 * kk);
+                                    ptx::mma_mxf4_2cta(tmem_acc, da + adv, db + adv, idesc, t_sfa,
+                                                       t_sfb, accumulate | (uint32_t)(g | kk));
+                                }
+                            }
+                        }
+                        ptx::tc_commit_2cta(&empty[s]);
+                    }
+                    __syncwarp();
+                    accumulate = 1;
+                }
+                if (ok) {
+                    if (ptx::elect_one()) ptx::tc_commit_2cta(acc_full);
+                    __syncwarp();
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;  // the TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;
+        constexpr int kColsPerThread = kTile / 2;
+        constexpr int kChunk = (sizeof(OutT) == 2) ? 64 : 32;
+        constexpr int kChunks = kColsPerThread / kChunk;
+        constexpr int kRegs = kChunk * (int)sizeof(OutT) / 4;
+        const uint32_t acc_empty0 = ptx::map_to_cta(ptx::smem_u32(acc_empty), 0);
+        uint32_t ti = 0;
+        bool ok = true;
+        for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
+            const int m0 = (tile % tiles_m) * kTile + 128 * (int)rank, n0 = (tile / tiles_m) * kTile;
+            if (!ptx::mbar_wait(acc_full, ti & 1, abort, kWaitLimit)) {
+                give_up(abort, prm.status, 0x2500);
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int row = m0 + 32 * q + lane;
+            const int cbase = half * kColsPerThread;
+            OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0 + cbase;
+#pragma unroll
+            for (int ch = 0; ch < kChunks; ++ch) {
+                uint32_t out[kRegs];
+#pragma unroll
+                for (int cb = 0; cb < kChunk / 16; ++cb) {
+                    uint32_t rr[16];
+                    ptx::tmem_ld_32x16(
+                        tmem_acc + ((uint32_t)(32 * q) << 16) + cbase + ch * kChunk + 16 * cb, rr);
+                    ptx::tmem_ld_wait();
+                    if (sizeof(OutT) == 4) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) out[16 * cb + i] = rr[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(
+                                __uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1]));
+                            out[8 * cb + i] = *reinterpret_cast<const uint32_t*>(&h2);
+                        }
+                    }
+                }
+                if (ch == kChunks - 1) {
+                    // last read of the accumulator: the next tile's MMAs may overwrite it
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
+                }
+                const int col0 = n0 + cbase + ch * kChunk;
+                if (row < prm.M && col0 < prm.N) {
+                    OutT* dp = drow + ch * kChunk;
+                    if (col0 + kChunk <= prm.N && prm.d_vec_ok) {
+                        uint4* p = reinterpret_cast<uint4*>(dp);
+#pragma unroll
+                        for (int i = 0; i < kRegs / 4; ++i)
+                            p[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2],
+                                              out[4 * i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kRegs; ++i) {
+                            const uint32_t v = out[i];
+                            if (sizeof(OutT) == 4) {
+                                if (col0 + i < prm.N)
+                                    reinterpret_cast<float*>(dp)[i] = __uint_as_float(v);
+                            } else {
+                                __nv_bfloat16* d16 = reinterpret_cast<__nv_bfloat16*>(dp) + 2 * i;
+                                if (col0 + 2 * i < prm.N)
+                                    d16[0] = __ushort_as_bfloat16((unsigned short)(v & 0xFFFFu));
+                                if (col0 + 2 * i + 1 < prm.N)
+                                    d16[1] = __ushort_as_bfloat16((unsigned short)(v >> 16));
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    // After a timeout, copies may still be in flight into this pair's shared memory: give
+    // them (bounded) time to land before the CTAs leave.  `full` of the even CTA counts both.
+    if (*abort != 0u && threadIdx.x == 0 && rank == 0) {
+        const long long t0 = clock64();
+        for (int s = 0; s < S; ++s)
+            while (!ptx::mbar_try_wait(&full[s], 0) && !ptx::mbar_try_wait(&full[s], 1) &&
+                   clock64() - t0 < kWaitLimit) {
+            }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    // neither CTA may leave (or free its TMEM) while the other still reads its shared memory
+    // through the pair MMA or signals its barriers
+    ptx::cluster_sync();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_2cta(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------ prepack
+// Scale plane [rows][nbk] -> atoms [ceil(rows/128)][nbk/4][512]: inside an atom the four
+// scale bytes of row r (r < 128) sit at (r % 32) * 16 + (r / 32) * 4.  Rows past the end are
+// written as zero.  One CTA handles 128 rows x up to 32 K groups through shared memory so
+// that both the reads and the writes are contiguous.
+__global__ void __launch_bounds__(256) prepack_scales_kernel(const uint8_t* __restrict__ scales,
+                                                             int rows, int nbk,
+                                                             uint8_t* __restrict__ out)
+{
+    __shared__ uint32_t tile[32 * 129];  // [kg][atom word], padded against bank conflicts
+    const int kgroups = nbk >> 2;
+    const int rg = blockIdx.y, kg0 = blockIdx.x * 32;
+    const int nkg = min(32, kgroups - kg0);
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(scales);
+    for (int i = threadIdx.x; i < 128 * 32; i += 256) {
+        const int r = i >> 5, kg = i & 31;
+        const int64_t row = (int64_t)rg * 128 + r;
+        uint32_t v = 0;
+        if (kg < nkg && row < rows) v = src[row * kgroups + kg0 + kg];
+        tile[kg * 129 + (r & 31) * 4 + (r >> 5)] = v;
+    }
+    __syncthreads();
+    uint32_t* dst = reinterpret_cast<uint32_t*>(out) + ((int64_t)rg * kgroups + kg0) * 128;
+    for (int i = threadIdx.x; i < nkg * 128; i += 256) dst[i] = tile[(i >> 7) * 129 + (i & 127)];
+}
+
+// Packed codes [rows][K/2] (+ scale and BM index planes) -> E4M3 bytes [rows][K].  One thread
+// per 32-element block.  E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6 are the E4M3 bytes 00 30 38
+// 3C 40 44 48 4C; the BM of an MX+ block (Eq. 3: 4 + m/2, stored as sign + 3 mantissa bits)
+// is 0x48 | m.  A block with scale byte 0 (flushed) becomes zeros.
+template <bool kPlus>
+__global__ void __launch_bounds__(256) widen_e4m3_kernel(const uint8_t* __restrict__ nibbles,
+                                                         const uint8_t* __restrict__ scales,
+                                                         const uint8_t* __restrict__ bm_index,
+                                                         int64_t nblocks, uint8_t* __restrict__ out)
+{
+    const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= nblocks) return;
+    const uint4 w4 = reinterpret_cast<const uint4*>(nibbles)[b];
+    const uint32_t sc = scales[b];
+    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t x = h ? (w[i] >> 16) : w[i];
+            const uint32_t mag = __byte_perm(0x3C383000u, 0x4C484440u, x & 0x7777u);
+            // sign bits 3, 7, 11, 15 -> 7, 15, 23, 31
+            const uint32_t sg = ((x & 0x8u) << 4) | ((x & 0x80u) << 8) | ((x & 0x800u) << 12) |
+                                ((x & 0x8000u) << 16);
+            o[2 * i + h] = sc ? (mag | sg) : 0u;
+        }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(out + b * 32);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    if (kPlus && sc) {
+        const uint32_t idx = bm_index[b] & 31u;
+        const uint32_t nib = (w[idx >> 3] >> ((idx & 7u) * 4u)) & 0xFu;
+        // same thread, later store to the same address: lands after the vector store
+        out[b * 32 + idx] = (uint8_t)(((nib & 8u) << 4) | 0x48u | (nib & 7u));
+    }
+}
+
+// 2-D byte tensor [rows][row_bytes], boxes of 128 bytes x 128 rows, 128B swizzle.
+bool make_tmap_rows(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t row_bytes)
+{
+    EncodeFn fn = tensormap_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)kRowBytes, 128u};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Scale atoms as a 3-D tensor of 32-bit words [row groups][K groups][128], boxes of
+// 128 x kgroups_per_stage x rgs.
+bool make_tmap_atoms(CUtensorMap* m, const uint8_t* base, int64_t rgs_total, int64_t kgroups,
+                     int box_kg, int box_rg)
+{
+    EncodeFn fn = tensormap_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {128u, (cuuint64_t)kgroups, (cuuint64_t)rgs_total};
+    const cuuint64_t strides[2] = {(cuuint64_t)kAtom, (cuuint64_t)kAtom * (cuuint64_t)kgroups};
+    const cuuint32_t box[3] = {128u, (cuuint32_t)box_kg, (cuuint32_t)box_rg};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Layout {
+    size_t sfa, sfb, wa, wb, total;
+};
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+Layout layout(int64_t M, int64_t N, int64_t K, bool wide)
+{
+    Layout l;
+    const size_t kgroups = (size_t)(K / 128);
+    size_t off = kStatusBytes;
+    off = round_up(off, 1024);
+    l.sfa = off;
+    off += (size_t)((M + 127) / 128) * kgroups * kAtom;
+    off = round_up(off, 1024);
+    l.sfb = off;
+    off += (size_t)((N + 127) / 128) * kgroups * kAtom;
+    off = round_up(off, 1024);
+    l.wa = off;
+    if (wide) off += (size_t)M * (size_t)K;
+    off = round_up(off, 1024);
+    l.wb = off;
+    if (wide) off += (size_t)N * (size_t)K;
+    l.total = round_up(off, 1024);
+    return l;
+}
+
+template <bool kWide, typename OutT>
+mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tsa,
+                         const CUtensorMap& tsb, const SParams& prm, int num_sms,
+                         cudaStream_t stream)
+{
+    using C = SCfg<kWide>;
+    auto kern = gemm_tc_stream_kernel<kWide, OutT>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) !=
+            cudaSuccess)
+            return MXP_ERR_CUDA;
+        attr_set = true;
+    }
+    const int64_t tiles = (int64_t)((prm.M + kTile - 1) / kTile) * ((prm.N + kTile - 1) / kTile);
+    int64_t clusters = num_sms / 2;
+    if (tiles < clusters) clusters = tiles;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, ta, tb, tsa, tsb, prm) == cudaSuccess ? MXP_OK
+                                                                               : MXP_ERR_CUDA;
+}
+
+}  // namespace
+
+size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
+{
+    if (M <= 128 || N <= 128 || K % 128 != 0) return 0;
+    const bool wide = a_mode == MXP_MODE_MXFP4_PLUS || b_mode == MXP_MODE_MXFP4_PLUS;
+    return layout(M, N, K, wide).total;
+}
+
+mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
+                                 const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                                 void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    const bool ap = A.mode == MXP_MODE_MXFP4_PLUS, bp = B.mode == MXP_MODE_MXFP4_PLUS;
+    const bool wide = ap || bp;
+    const Layout l = layout(M, N, K, wide);
+    if (workspace == nullptr || workspace_bytes < l.total) return MXP_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return MXP_ERR_INVALID_ARG;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MXP_ERR_CUDA;
+    const int nbk = (int)(K / 32);
+    const int kgroups = nbk / 4;
+    const int rga = (int)((M + 127) / 128), rgb = (int)((N + 127) / 128);
+
+    prepack_scales_kernel<<<dim3((kgroups + 31) / 32, rga), 256, 0, stream>>>(A.scales, (int)M, nbk,
+                                                                             ws + l.sfa);
+    prepack_scales_kernel<<<dim3((kgroups + 31) / 32, rgb), 256, 0, stream>>>(B.scales, (int)N, nbk,
+                                                                             ws + l.sfb);
+    if (wide) {
+        const int64_t nba = M * nbk, nbb = N * nbk;
+        if (ap)
+            widen_e4m3_kernel<true><<<(unsigned)((nba + 255) / 256), 256, 0, stream>>>(
+                A.nibbles, A.scales, A.bm_index, nba, ws + l.wa);
+        else
+            widen_e4m3_kernel<false><<<(unsigned)((nba + 255) / 256), 256, 0, stream>>>(
+                A.nibbles, A.scales, nullptr, nba, ws + l.wa);
+        if (bp)
+            widen_e4m3_kernel<true><<<(unsigned)((nbb + 255) / 256), 256, 0, stream>>>(
+                B.nibbles, B.scales, B.bm_index, nbb, ws + l.wb);
+        else
+            widen_e4m3_kernel<false><<<(unsigned)((nbb + 255) / 256), 256, 0, stream>>>(
+                B.nibbles, B.scales, nullptr, nbb, ws + l.wb);
+    }
+    if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+
+    CUtensorMap ta, tb, tsa, tsb;
+    const int box_kg = wide ? 1 : 2;
+    const bool maps_ok =
+        (wide ? make_tmap_rows(&ta, ws + l.wa, M, K) && make_tmap_rows(&tb, ws + l.wb, N, K)
+              : make_tmap_rows(&ta, A.nibbles, M, K / 2) && make_tmap_rows(&tb, B.nibbles, N, K / 2)) &&
+        make_tmap_atoms(&tsa, ws + l.sfa, rga, kgroups, box_kg, 1) &&
+        make_tmap_atoms(&tsb, ws + l.sfb, rgb, kgroups, box_kg, 2);
+    if (!maps_ok) return MXP_ERR_CUDA;
+
+    SParams prm;
+    prm.M = (int)M;
+    prm.N = (int)N;
+    prm.K = (int)K;
+    prm.D = D;
+    prm.ldd = ldd;
+    prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
+                   ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
+    prm.status = static_cast<StatusBlock*>(workspace);
+    if (wide)
+        return d_dt == MXP_F32
+                   ? launch_stream<true, float>(ta, tb, tsa, tsb, prm, num_sms, stream)
+                   : launch_stream<true, __nv_bfloat16>(ta, tb, tsa, tsb, prm, num_sms, stream);
+    return d_dt == MXP_F32
+               ? launch_stream<false, float>(ta, tb, tsa, tsb, prm, num_sms, stream)
+               : launch_stream<false, __nv_bfloat16>(ta, tb, tsa, tsb, prm, num_sms, stream);
+}
+
+}  // namespace mxp
