@@ -1237,8 +1237,6 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
 #endif
     prm.num_sms = sm_count();
     if (prm.num_sms <= 0) return MXP_ERR_CUDA;
-    if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
-        return MXP_ERR_CUDA;
     // Kernel choice by measurement on the prefill shapes: the pair kernel wins whenever an
     // operand is MX+ (a third less residual-tile memory and patch work per CTA buys pipeline
     // depth); the single-CTA kernel wins for plain MXFP4.  MXP_GEMM_KERNEL=single|pair
@@ -1251,6 +1249,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     const bool forced_other = force != nullptr && (force[0] == 's' || force[0] == 'p');
     if (fast != 0 && workspace_bytes >= fast && !forced_other)
         return launch_gemm_tc_stream(M, N, K, A, B, D, d_dt, ldd, workspace, workspace_bytes, stream);
+    if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
+        return MXP_ERR_CUDA;
     bool use_pair = M > 128 && N > 128 && (ap || bp);
     if (force != nullptr && force[0] == 's') use_pair = false;
     if (force != nullptr && force[0] == 'p') use_pair = M > 128 && N > 128;

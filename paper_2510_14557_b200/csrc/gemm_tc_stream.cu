@@ -100,6 +100,20 @@ __device__ __forceinline__ void give_up(volatile uint32_t* abort, StatusBlock* s
     }
 }
 
+// Tile order: bands of kBand tile rows, walked column by column, so that the tiles in flight
+// at any time (one per CTA pair) cover a compact block of the output and their A and B
+// panels stay resident in L2 instead of being re-streamed from HBM every wave.
+constexpr int kBand = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn)
+{
+    const int per_band = kBand * tiles_n;
+    const int band = tile / per_band;
+    const int r = tile - band * per_band;
+    const int h = min(kBand, tiles_m - band * kBand);  // height of this (maybe last) band
+    tn = r / h;
+    tm = band * kBand + (r - tn * h);
+}
+
 template <bool kWide, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -169,7 +183,8 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             uint32_t c = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-                const int tm = tile % tiles_m, tn = tile / tiles_m;
+                int tm, tn;
+                tile_coords(tile, tiles_m, tiles_n, tm, tn);
                 const int m0 = tm * kTile + 128 * (int)rank;
                 const int n0 = tn * kTile + 128 * (int)rank;
                 for (int kt = 0; kt < kstages; ++kt, ++c) {
@@ -209,7 +224,7 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 for (int kt = 0; kt < kstages && ok; ++kt, ++c) {
                     const int s = c % S;
                     const uint32_t ph = (c / S) & 1;
-                    if (!ptx::mbar_wait_cluster(&full[s], ph, abort, kWaitLimit)) {
+                    if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit)) {
                         if (lane == 0) give_up(abort, prm.status, 0x2200 + s);
                         ok = false;
                         break;
@@ -267,17 +282,19 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
+        // Each warp owns 32 accumulator rows (its TMEM lane quarter) x 128 columns.  All 128
+        // columns go to registers first and the accumulator is released at once, so the
+        // next tile's MMAs overlap the conversion and the global stores.
         const int q = warp & 3;  // the TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;
-        constexpr int kColsPerThread = kTile / 2;
-        constexpr int kChunk = (sizeof(OutT) == 2) ? 64 : 32;
-        constexpr int kChunks = kColsPerThread / kChunk;
-        constexpr int kRegs = kChunk * (int)sizeof(OutT) / 4;
+        constexpr int kCols = kTile / 2;
         const uint32_t acc_empty0 = ptx::map_to_cta(ptx::smem_u32(acc_empty), 0);
         uint32_t ti = 0;
         bool ok = true;
         for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
-            const int m0 = (tile % tiles_m) * kTile + 128 * (int)rank, n0 = (tile / tiles_m) * kTile;
+            int tm, tn;
+            tile_coords(tile, tiles_m, tiles_n, tm, tn);
+            const int m0 = tm * kTile + 128 * (int)rank, n0 = tn * kTile;
             if (!ptx::mbar_wait(acc_full, ti & 1, abort, kWaitLimit)) {
                 give_up(abort, prm.status, 0x2500);
                 ok = false;
@@ -285,59 +302,47 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
             ptx::tc_fence_after_sync();
             const int row = m0 + 32 * q + lane;
-            const int cbase = half * kColsPerThread;
+            const int cbase = half * kCols;
+            uint32_t rr[kCols];
+#pragma unroll
+            for (int cb = 0; cb < kCols / 32; ++cb)
+                ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(32 * q) << 16) + cbase + 32 * cb,
+                                   reinterpret_cast<uint32_t(&)[32]>(rr[32 * cb]));
+            ptx::tmem_ld_wait();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
+            if (row >= prm.M) continue;
             OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0 + cbase;
+            const int col0 = n0 + cbase;
+            if (col0 + kCols <= prm.N && prm.d_vec_ok) {
+                uint4* p = reinterpret_cast<uint4*>(drow);
+                if (sizeof(OutT) == 4) {
 #pragma unroll
-            for (int ch = 0; ch < kChunks; ++ch) {
-                uint32_t out[kRegs];
+                    for (int i = 0; i < kCols / 4; ++i)
+                        p[i] = make_uint4(rr[4 * i], rr[4 * i + 1], rr[4 * i + 2], rr[4 * i + 3]);
+                } else {
 #pragma unroll
-                for (int cb = 0; cb < kChunk / 16; ++cb) {
-                    uint32_t rr[16];
-                    ptx::tmem_ld_32x16(
-                        tmem_acc + ((uint32_t)(32 * q) << 16) + cbase + ch * kChunk + 16 * cb, rr);
-                    ptx::tmem_ld_wait();
-                    if (sizeof(OutT) == 4) {
+                    for (int i = 0; i < kCols / 8; ++i) {
+                        uint32_t o[4];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) out[16 * cb + i] = rr[i];
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
+                        for (int k = 0; k < 4; ++k) {
                             const __nv_bfloat162 h2 = __floats2bfloat162_rn(
-                                __uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1]));
-                            out[8 * cb + i] = *reinterpret_cast<const uint32_t*>(&h2);
+                                __uint_as_float(rr[8 * i + 2 * k]), __uint_as_float(rr[8 * i + 2 * k + 1]));
+                            o[k] = *reinterpret_cast<const uint32_t*>(&h2);
                         }
+                        p[i] = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
-                if (ch == kChunks - 1) {
-                    // last read of the accumulator: the next tile's MMAs may overwrite it
-                    ptx::tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
-                }
-                const int col0 = n0 + cbase + ch * kChunk;
-                if (row < prm.M && col0 < prm.N) {
-                    OutT* dp = drow + ch * kChunk;
-                    if (col0 + kChunk <= prm.N && prm.d_vec_ok) {
-                        uint4* p = reinterpret_cast<uint4*>(dp);
+            } else {
 #pragma unroll
-                        for (int i = 0; i < kRegs / 4; ++i)
-                            p[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2],
-                                              out[4 * i + 3]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < kRegs; ++i) {
-                            const uint32_t v = out[i];
-                            if (sizeof(OutT) == 4) {
-                                if (col0 + i < prm.N)
-                                    reinterpret_cast<float*>(dp)[i] = __uint_as_float(v);
-                            } else {
-                                __nv_bfloat16* d16 = reinterpret_cast<__nv_bfloat16*>(dp) + 2 * i;
-                                if (col0 + 2 * i < prm.N)
-                                    d16[0] = __ushort_as_bfloat16((unsigned short)(v & 0xFFFFu));
-                                if (col0 + 2 * i + 1 < prm.N)
-                                    d16[1] = __ushort_as_bfloat16((unsigned short)(v >> 16));
-                            }
-                        }
+                for (int i = 0; i < kCols; ++i) {
+                    if (col0 + i < prm.N) {
+                        if (sizeof(OutT) == 4)
+                            reinterpret_cast<float*>(drow)[i] = __uint_as_float(rr[i]);
+                        else
+                            reinterpret_cast<__nv_bfloat16*>(drow)[i] =
+                                __float2bfloat16_rn(__uint_as_float(rr[i]));
                     }
                 }
             }
@@ -366,49 +371,58 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
 }
 
 // ------------------------------------------------------------------------------ prepack
-// Scale plane [rows][nbk] -> atoms [ceil(rows/128)][nbk/4][512]: inside an atom the four
-// scale bytes of row r (r < 128) sit at (r % 32) * 16 + (r / 32) * 4.  Rows past the end are
-// written as zero.  One CTA handles 128 rows x up to 32 K groups through shared memory so
-// that both the reads and the writes are contiguous.
-__global__ void __launch_bounds__(256) prepack_scales_kernel(const uint8_t* __restrict__ scales,
-                                                             int rows, int nbk,
-                                                             uint8_t* __restrict__ out)
+// One launch prepares both operands.  Its CTAs are of two kinds, told apart by block index:
+//
+// scale CTAs: scale plane [rows][nbk] -> atoms [ceil(rows/128)][nbk/4][512]; inside an atom
+//   the four scale bytes of row r (r < 128) sit at (r % 32) * 16 + (r / 32) * 4.  Rows past
+//   the end are written as zero.  A CTA handles 128 rows x up to 32 K groups through shared
+//   memory, so reads and writes are both contiguous.
+// widen CTAs (only when an operand is MX+): packed codes [rows][K/2] -> E4M3 bytes [rows][K],
+//   one thread per 16 elements (8 bytes in, 16 bytes out, both contiguous across the warp).
+//   E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6 are the E4M3 bytes 00 30 38 3C 40 44 48 4C; the
+//   BM of an MX+ block (Eq. 3: 4 + m/2, stored as sign + 3 mantissa bits) is 0x48 | m.  A
+//   block with scale byte 0 (flushed) becomes zeros.
+struct PrepackOperand {
+    const uint8_t* nibbles;
+    const uint8_t* scales;
+    const uint8_t* bm_index;  // nullptr: plain MXFP4
+    uint8_t* atoms;
+    uint8_t* wide;            // nullptr: not widened
+    int rows, nbk;
+    unsigned scale_ctas;      // ceil(rows/128) * ceil(nbk/128)
+    unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
+};
+
+__device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigned id, uint32_t* tile)
 {
-    __shared__ uint32_t tile[32 * 129];  // [kg][atom word], padded against bank conflicts
-    const int kgroups = nbk >> 2;
-    const int rg = blockIdx.y, kg0 = blockIdx.x * 32;
+    const int kgroups = op.nbk >> 2;
+    const int kchunks = (kgroups + 31) >> 5;
+    const int rg = (int)(id / (unsigned)kchunks), kg0 = (int)(id % (unsigned)kchunks) * 32;
     const int nkg = min(32, kgroups - kg0);
-    const uint32_t* src = reinterpret_cast<const uint32_t*>(scales);
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(op.scales);
     for (int i = threadIdx.x; i < 128 * 32; i += 256) {
         const int r = i >> 5, kg = i & 31;
         const int64_t row = (int64_t)rg * 128 + r;
         uint32_t v = 0;
-        if (kg < nkg && row < rows) v = src[row * kgroups + kg0 + kg];
-        tile[kg * 129 + (r & 31) * 4 + (r >> 5)] = v;
+        if (kg < nkg && row < op.rows) v = src[row * kgroups + kg0 + kg];
+        tile[kg * 129 + (r & 31) * 4 + (r >> 5)] = v;  // rows of 129 words: no bank conflicts
     }
     __syncthreads();
-    uint32_t* dst = reinterpret_cast<uint32_t*>(out) + ((int64_t)rg * kgroups + kg0) * 128;
+    uint32_t* dst = reinterpret_cast<uint32_t*>(op.atoms) + ((int64_t)rg * kgroups + kg0) * 128;
     for (int i = threadIdx.x; i < nkg * 128; i += 256) dst[i] = tile[(i >> 7) * 129 + (i & 127)];
 }
 
-// Packed codes [rows][K/2] (+ scale and BM index planes) -> E4M3 bytes [rows][K].  One thread
-// per 32-element block.  E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6 are the E4M3 bytes 00 30 38
-// 3C 40 44 48 4C; the BM of an MX+ block (Eq. 3: 4 + m/2, stored as sign + 3 mantissa bits)
-// is 0x48 | m.  A block with scale byte 0 (flushed) becomes zeros.
-template <bool kPlus>
-__global__ void __launch_bounds__(256) widen_e4m3_kernel(const uint8_t* __restrict__ nibbles,
-                                                         const uint8_t* __restrict__ scales,
-                                                         const uint8_t* __restrict__ bm_index,
-                                                         int64_t nblocks, uint8_t* __restrict__ out)
+__device__ __forceinline__ void widen_e4m3(const PrepackOperand& op, unsigned id)
 {
-    const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= nblocks) return;
-    const uint4 w4 = reinterpret_cast<const uint4*>(nibbles)[b];
-    const uint32_t sc = scales[b];
-    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-    uint32_t o[8];
+    const int64_t t = (int64_t)id * 256 + threadIdx.x;  // half block: 16 elements
+    const int64_t b = t >> 1;
+    if (b >= (int64_t)op.rows * op.nbk) return;
+    const uint2 w2 = reinterpret_cast<const uint2*>(op.nibbles)[t];
+    const uint32_t sc = op.scales[b];
+    const uint32_t w[2] = {w2.x, w2.y};
+    uint32_t o[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 2; ++i) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const uint32_t x = h ? (w[i] >> 16) : w[i];
@@ -416,18 +430,41 @@ __global__ void __launch_bounds__(256) widen_e4m3_kernel(const uint8_t* __restri
             // sign bits 3, 7, 11, 15 -> 7, 15, 23, 31
             const uint32_t sg = ((x & 0x8u) << 4) | ((x & 0x80u) << 8) | ((x & 0x800u) << 12) |
                                 ((x & 0x8000u) << 16);
-            o[2 * i + h] = sc ? (mag | sg) : 0u;
+            o[2 * i + h] = mag | sg;
         }
     }
-    uint4* dst = reinterpret_cast<uint4*>(out + b * 32);
-    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-    if (kPlus && sc) {
-        const uint32_t idx = bm_index[b] & 31u;
-        const uint32_t nib = (w[idx >> 3] >> ((idx & 7u) * 4u)) & 0xFu;
-        // same thread, later store to the same address: lands after the vector store
-        out[b * 32 + idx] = (uint8_t)(((nib & 8u) << 4) | 0x48u | (nib & 7u));
+    if (op.bm_index != nullptr) {
+        const uint32_t idx = op.bm_index[b] & 31u;
+        if ((idx >> 4) == (uint32_t)(t & 1)) {
+            const uint32_t e = idx & 15u;
+            const uint32_t nib = (w[e >> 3] >> ((e & 7u) * 4u)) & 0xFu;
+            const uint32_t byte = ((nib & 8u) << 4) | 0x48u | (nib & 7u);
+            const uint32_t sh = (e & 3u) * 8u;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if ((e >> 2) == (uint32_t)k) o[k] = (o[k] & ~(0xFFu << sh)) | (byte << sh);
+        }
     }
+    if (sc == 0u) o[0] = o[1] = o[2] = o[3] = 0u;
+    reinterpret_cast<uint4*>(op.wide)[t] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+__global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, const PrepackOperand b,
+                                                      StatusBlock* status)
+{
+    __shared__ uint32_t tile[32 * 129];
+    unsigned id = blockIdx.x;
+    if (id == 0 && threadIdx.x == 0) {
+        status->code = 0u;  // the GEMM that follows on the stream reports into this block
+        status->where = 0u;
+    }
+    if (id < a.scale_ctas) return prepack_scales(a, id, tile);
+    id -= a.scale_ctas;
+    if (id < b.scale_ctas) return prepack_scales(b, id, tile);
+    id -= b.scale_ctas;
+    if (id < a.widen_ctas) return widen_e4m3(a, id);
+    id -= a.widen_ctas;
+    widen_e4m3(b, id);
 }
 
 // 2-D byte tensor [rows][row_bytes], boxes of 128 bytes x 128 rows, 128B swizzle.
@@ -544,26 +581,26 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     const int nbk = (int)(K / 32);
     const int kgroups = nbk / 4;
     const int rga = (int)((M + 127) / 128), rgb = (int)((N + 127) / 128);
+    if ((reinterpret_cast<uintptr_t>(A.nibbles) | reinterpret_cast<uintptr_t>(B.nibbles)) & 15)
+        return MXP_ERR_INVALID_ARG;
 
-    prepack_scales_kernel<<<dim3((kgroups + 31) / 32, rga), 256, 0, stream>>>(A.scales, (int)M, nbk,
-                                                                             ws + l.sfa);
-    prepack_scales_kernel<<<dim3((kgroups + 31) / 32, rgb), 256, 0, stream>>>(B.scales, (int)N, nbk,
-                                                                             ws + l.sfb);
-    if (wide) {
-        const int64_t nba = M * nbk, nbb = N * nbk;
-        if (ap)
-            widen_e4m3_kernel<true><<<(unsigned)((nba + 255) / 256), 256, 0, stream>>>(
-                A.nibbles, A.scales, A.bm_index, nba, ws + l.wa);
-        else
-            widen_e4m3_kernel<false><<<(unsigned)((nba + 255) / 256), 256, 0, stream>>>(
-                A.nibbles, A.scales, nullptr, nba, ws + l.wa);
-        if (bp)
-            widen_e4m3_kernel<true><<<(unsigned)((nbb + 255) / 256), 256, 0, stream>>>(
-                B.nibbles, B.scales, B.bm_index, nbb, ws + l.wb);
-        else
-            widen_e4m3_kernel<false><<<(unsigned)((nbb + 255) / 256), 256, 0, stream>>>(
-                B.nibbles, B.scales, nullptr, nbb, ws + l.wb);
-    }
+    auto operand = [&](const mxp_packed& P, int64_t rows, size_t atoms_off, size_t wide_off) {
+        PrepackOperand op;
+        op.nibbles = P.nibbles;
+        op.scales = P.scales;
+        op.bm_index = P.mode == MXP_MODE_MXFP4_PLUS ? P.bm_index : nullptr;
+        op.atoms = ws + atoms_off;
+        op.wide = wide ? ws + wide_off : nullptr;
+        op.rows = (int)rows;
+        op.nbk = nbk;
+        op.scale_ctas = (unsigned)(((rows + 127) / 128) * ((kgroups + 31) / 32));
+        op.widen_ctas = wide ? (unsigned)((rows * nbk * 2 + 255) / 256) : 0u;
+        return op;
+    };
+    const PrepackOperand pa = operand(A, M, l.sfa, l.wa), pb = operand(B, N, l.sfb, l.wb);
+    const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
+    if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
+    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, pb, static_cast<StatusBlock*>(workspace));
     if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
 
     CUtensorMap ta, tb, tsa, tsb;
