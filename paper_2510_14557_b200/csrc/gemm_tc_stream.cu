@@ -180,6 +180,9 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             const uint32_t full0 = ptx::map_to_cta(ptx::smem_u32(&full[0]), 0);
+            // the launch may overlap the tail of the prepack kernel: its output is first
+            // touched here
+            ptx::grid_dependency_wait();
             uint32_t c = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
@@ -453,6 +456,7 @@ __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, co
                                                       StatusBlock* status)
 {
     __shared__ uint32_t tile[32 * 129];
+    ptx::grid_launch_dependents();  // the GEMM's prologue may start while this grid drains
     unsigned id = blockIdx.x;
     if (id == 0 && threadIdx.x == 0) {
         status->code = 0u;  // the GEMM that follows on the stream reports into this block
@@ -546,13 +550,15 @@ mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUt
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = C::kSmem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kern, ta, tb, tsa, tsb, prm) == cudaSuccess ? MXP_OK
                                                                                : MXP_ERR_CUDA;
 }
