@@ -24,6 +24,15 @@ cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void*
                                     void* workspace, size_t workspace_bytes,
                                     cudaStream_t stream);
 
+// Streamed variant for decode shapes (N % 16 == 0, K % 256 == 0, activations that fit shared
+// memory).  `status` (may be nullptr) is a StatusBlock the kernel writes only when a wait
+// runs out.
+bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                         const mxp_packed& B);
+cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                  const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                                  void* status, cudaStream_t stream);
+
 // Block-scaled tensor-core form: both operands packed.
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
 size_t tc_compact_workspace_bytes();  // enough for the kernels that work in place

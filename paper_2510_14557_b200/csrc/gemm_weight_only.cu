@@ -13,6 +13,8 @@
 // (= (4 + m/2) * 2^-126), patched in before the multiply: this is Eq. 3's BM branch.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace mxp {
@@ -232,13 +234,26 @@ void launch_mt(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, cons
 
 }  // namespace
 
-size_t skinny_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
+size_t skinny_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }  // a status block is optional
 
 cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                     const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                                    void*, size_t, cudaStream_t stream)
+                                    void* workspace, size_t workspace_bytes, cudaStream_t stream)
 {
     if (M > (1 << 20) || N > (1ll << 30) || K > (1ll << 30)) return cudaErrorNotSupported;
+    // Decode shapes go to the streamed kernel; MXP_WO_KERNEL=old|stream overrides (measurement
+    // and test aid).  A workspace, if given, receives the status of its bounded waits.
+    const char* force = getenv("MXP_WO_KERNEL");
+    const bool want_old = force != nullptr && force[0] == 'o';
+    if (!want_old && M <= 64 && wo_stream_supported(M, N, K, A, lda, B)) {
+        void* status = nullptr;
+        if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {
+            status = workspace;
+            if (cudaMemsetAsync(status, 0, sizeof(StatusBlock), stream) != cudaSuccess)
+                return cudaErrorUnknown;
+        }
+        return launch_gemm_wo_stream(M, N, K, A, lda, B, D, d_dt, ldd, status, stream);
+    }
     if ((M + 15) / 16 > 65535) return cudaErrorNotSupported;
     const bool plus = B.mode == MXP_MODE_MXFP4_PLUS;
     if (d_dt == MXP_F32) {

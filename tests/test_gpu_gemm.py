@@ -69,6 +69,44 @@ def test_weight_only_config3_sampled(M):
     check_gemm(d[:, torch.from_numpy(rows).cuda()], da, dw)
 
 
+@pytest.mark.parametrize("kernel", ["old", "stream"])
+@pytest.mark.parametrize("wmode", [MX, MXP])
+@pytest.mark.parametrize("M,N,K", [(1, 32, 256), (3, 48, 2304), (8, 160, 4352), (9, 64, 512),
+                                   (16, 2384, 4096), (40, 64, 768)])
+def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
+    # shapes the streamed kernel takes (N % 16 == 0, K % 256 == 0): several 2048-element stages,
+    # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles
+    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K)
+    wp, dw = quantized(w_bits, wmode, bf16=True)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    for dt in (torch.float32, torch.bfloat16):
+        d = mxp().mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=dt)
+        check_gemm(d, da, dw)
+
+
+@pytest.mark.parametrize("kernel", ["old", "stream"])
+def test_weight_only_one_hot_and_scale_spread(kernel, monkeypatch):
+    # one-hot activations select single decoded weights (exact in fp32), with weight rows and
+    # activation rows spread over 60 binades each, a flushed block and a zero block
+    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
+    K, N = 512, 48
+    g = synth.rng(11)
+    w = g.standard_normal((N, K)).astype(np.float32)
+    w *= np.exp2(g.integers(-30, 30, (N, 1))).astype(np.float32)
+    w[3, 32:64] = 0
+    w[5, 64:96] = 1e-44
+    wp, dw = quantized(w, MXP)
+    a = np.zeros((16, K), np.float32)
+    for m in range(16):
+        a[m, (m * 37) % K] = 2.0 ** (4 * m - 30)
+    d = mxp().mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), wp, out_dtype=torch.float32)
+    got = d.cpu().numpy().astype(np.float64)
+    for m in range(16):
+        want = (dw[:, (m * 37) % K] * 2.0 ** (4 * m - 30)).astype(np.float32).astype(np.float64)
+        assert np.array_equal(got[m], want)
+
+
 # ------------------------------------------------------------------ tensor-core form
 MODES = [(MX, MX), (MXP, MX), (MX, MXP), (MXP, MXP)]
 
