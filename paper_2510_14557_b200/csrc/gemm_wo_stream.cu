@@ -12,12 +12,12 @@
 //   * patch the block's BM to 4 + m/2 (Eq. 3's BM branch) with masks from a small table,
 //   * run two m16n8k16 f16 MMAs against the activations of the block (fresh accumulator),
 //   * add that partial sum times 2^(shared_exp) of the weight block into the running fp32 sum.
-// Activations are bf16; so that they fit f16 they are normalised once per CTA, row by row,
-// by the power of two that puts the row's largest magnitude in [2^14, 2^15): every element
-// within 2^28 of that maximum stays exact (f16 keeps 11 significant bits), smaller ones are
-// rounded at 2^-39 of the maximum, far inside the GEMM's error bound, which is relative to the
-// row's norm.  The power of two goes back in when the reducers store D.  No scale multiply
-// touches the weights, so the weight side costs one cast per element pair.
+// Activations are bf16; so that they fit f16 each 256-element chunk of an activation row is
+// normalised by the power of two that puts its largest magnitude in [2^14, 2^15): every
+// element within 2^28 of that maximum stays exact (f16 keeps 11 significant bits), smaller
+// ones are rounded at 2^-39 of the maximum, far inside the GEMM's error bound, which is
+// relative to the row's norm.  The power of two goes back in once per chunk.  No scale
+// multiply touches the weights, so the weight side costs one cast per element pair.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -87,7 +87,7 @@ __host__ __device__ inline WoLayout wo_layout(int K, int mp, bool plus, int red_
     l.act = off;
     off += nb * mp * 64;
     l.fa = off;
-    off += 2 * (size_t)mp * 4;  // per column: largest magnitude (setup), then the factor
+    off += (nb / 8 + 1) * (size_t)mp * 4;  // factor per 256-element chunk and column
     l.meta = off;
     l.meta_stride = (int)(kRows * nb * (plus ? 2 : 1));
     off += (size_t)meta_bufs * l.meta_stride;
@@ -270,7 +270,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
             ptx::mbar_init(&red_full[b], kCW);
             ptx::mbar_init(&red_free[b], kRW);
         }
-        for (int i = 0; i < kMp; ++i) reinterpret_cast<uint32_t*>(smem + L.fa)[i] = 0u;  // row maxima
         ptx::mbar_init(setup_bar, kCW);
         *abort = 0u;
         ptx::fence_mbar_init();
@@ -331,65 +330,49 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
             if ((p >> 3) == tt) k[(p & 7u) >> 1] = (p & 1u) ? 0x0000FFFFu : 0xFFFF0000u;
             reinterpret_cast<uint4*>(smem + L.lut)[threadIdx.x] = make_uint4(k[0], k[1], k[2], k[3]);
         }
-        // activations of this CTA's columns -> f16 [block][column][32], each row normalised by
-        // its own power of two: pass 1 finds the rows' largest magnitudes, pass 2 converts
-        uint32_t* rowmax = reinterpret_cast<uint32_t*>(smem + L.fa);
-        float* fa = reinterpret_cast<float*>(smem + L.fa) + kMp;
-        uint32_t sphase = 0;
-        auto setup_sync = [&]() -> bool {
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(setup_bar);
-            const bool r = ptx::mbar_wait(setup_bar, sphase & 1u, abort, kWaitLimit);
-            ++sphase;
-            return r;
-        };
-        // each thread keeps its blocks in registers between the two steps (at most four)
-        constexpr int kMaxItems = 4;
-        uint4 x[kMaxItems][4];
-        for (int base = 0; base < nb * kMp; base += kCT * kMaxItems) {
+        // Activations -> f16 [block][column][32].  Every warp prepares exactly the chunks it
+        // will consume (no cross-warp step): each 256-element chunk of a column is normalised
+        // by its own power of two, kept in fa[chunk][column].
+        float* fa = reinterpret_cast<float*>(smem + L.fa);
+        constexpr int kItems = kChunkBlocks * kMp / 32;  // blocks per lane and chunk
+        for (int sl = 0; sl < slabs; ++sl) {
+            const int chunk = sl * kCW + warp;
+            const int kb0 = chunk * kChunkBlocks;
+            if (kb0 >= nb) break;
+            const int mc = lane % kMp;
+            uint4 x[kItems][4];
+            uint32_t mx = 0;
 #pragma unroll
-            for (int u = 0; u < kMaxItems; ++u) {
-                const int i = base + u * kCT + threadIdx.x;
-                const int kb = i / kMp, mc = i - kb * kMp;
+            for (int u = 0; u < kItems; ++u) {
+                const int kb = kb0 + lane / kMp + u * (32 / kMp);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) x[u][j] = make_uint4(0, 0, 0, 0);
-                if (i < nb * kMp && m0 + mc < prm.M) {
+                for (int q = 0; q < 4; ++q) x[u][q] = make_uint4(0, 0, 0, 0);
+                if (m0 + mc < prm.M) {
                     const uint4* src = reinterpret_cast<const uint4*>(
                         prm.A + (int64_t)(m0 + mc) * prm.lda + kb * 32);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) x[u][j] = __ldg(src + j);
-                    atomicMax(&rowmax[mc], block_max(x[u]));
+                    for (int q = 0; q < 4; ++q) x[u][q] = __ldg(src + q);
                 }
+                mx = max(mx, block_max(x[u]));
             }
-        }
-        const bool one_round = nb * kMp <= kCT * kMaxItems;
-        bool ok = setup_sync();
-        for (int base = 0; base < nb * kMp; base += kCT * kMaxItems) {
 #pragma unroll
-            for (int u = 0; u < kMaxItems; ++u) {
-                const int i = base + u * kCT + threadIdx.x;
-                if (i >= nb * kMp) continue;
-                const int kb = i / kMp, mc = i - kb * kMp;
-                if (!one_round) {  // the registers hold the last round only: load again
+            for (int o = kMp; o < 32; o <<= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+            const int mulfield = row_mulfield(mx);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) x[u][j] = make_uint4(0, 0, 0, 0);
-                    if (m0 + mc < prm.M) {
-                        const uint4* src = reinterpret_cast<const uint4*>(
-                            prm.A + (int64_t)(m0 + mc) * prm.lda + kb * 32);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) x[u][j] = __ldg(src + j);
-                    }
-                }
+            for (int u = 0; u < kItems; ++u) {
+                const int kb = kb0 + lane / kMp + u * (32 / kMp);
                 uint4 y[4];
-                normalise_block(x[u], row_mulfield(rowmax[mc]), y);
-                uint4* dst = reinterpret_cast<uint4*>(smem + L.act + (size_t)i * 64);
+                normalise_block(x[u], mulfield, y);
+                uint4* dst = reinterpret_cast<uint4*>(smem + L.act + ((size_t)kb * kMp + mc) * 64);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) dst[j] = y[j];
+                for (int q = 0; q < 4; ++q) dst[q] = y[q];
             }
+            if (lane < kMp) fa[chunk * kMp + mc] = __uint_as_float((uint32_t)(254 - mulfield) << 23);
         }
-        if (threadIdx.x < kMp)
-            fa[threadIdx.x] = __uint_as_float((uint32_t)(254 - row_mulfield(rowmax[threadIdx.x])) << 23);
-        ok = ok && setup_sync();
+        // the BM mask table was written by the first four warps: one barrier before its use
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(setup_bar);
+        bool ok = ptx::mbar_wait(setup_bar, 0, abort, kWaitLimit);
         if (!ok && lane == 0) report(prm.status, abort, 0x3500);
         if (threadIdx.x == 0) WO_TL(1);
 
@@ -423,6 +406,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                 if (threadIdx.x == 0) WO_TL(32 + (int)it * slabs + sl);
                 const int kb0 = sl * (kSlab / 32) + warp * kChunkBlocks;
                 if (kb0 < nb) {
+                    float cacc[kMT][4];
+#pragma unroll
+                    for (int i = 0; i < kMT; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) cacc[i][j] = 0.f;
                     const uint2 scA = lds64(sc + kb0), scB = lds64(sc + 8 * nb + kb0);
                     uint2 ixA = make_uint2(0, 0), ixB = ixA;
                     if (kPlus) {
@@ -452,11 +440,21 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                             float c[4];
                             mma_f16_16816_first(c, hA[0], hB[0], hA[1], hB[1], b.x, b.y);
                             mma_f16_16816(c, hA[2], hB[2], hA[3], hB[3], b.z, b.w);
-                            acc[mt][0] = fmaf(c[0], sA, acc[mt][0]);
-                            acc[mt][1] = fmaf(c[1], sA, acc[mt][1]);
-                            acc[mt][2] = fmaf(c[2], sB, acc[mt][2]);
-                            acc[mt][3] = fmaf(c[3], sB, acc[mt][3]);
+                            cacc[mt][0] = fmaf(c[0], sA, cacc[mt][0]);
+                            cacc[mt][1] = fmaf(c[1], sA, cacc[mt][1]);
+                            cacc[mt][2] = fmaf(c[2], sB, cacc[mt][2]);
+                            cacc[mt][3] = fmaf(c[3], sB, cacc[mt][3]);
                         }
+                    }
+                    // the power of two taken out of this chunk of the activation columns
+#pragma unroll
+                    for (int mt = 0; mt < kMT; ++mt) {
+                        const float2 f2 = *reinterpret_cast<const float2*>(
+                            fa + (kb0 / kChunkBlocks) * kMp + 8 * mt + 2 * t);
+                        acc[mt][0] = fmaf(cacc[mt][0], f2.x, acc[mt][0]);
+                        acc[mt][1] = fmaf(cacc[mt][1], f2.y, acc[mt][1]);
+                        acc[mt][2] = fmaf(cacc[mt][2], f2.x, acc[mt][2]);
+                        acc[mt][3] = fmaf(cacc[mt][3], f2.y, acc[mt][3]);
                     }
                 }
                 __syncwarp();
@@ -494,7 +492,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
         // ------------------------------------------------------------------ reducer warps
         const int tid = threadIdx.x - 32 * (kCW + 1);
         const float* red = reinterpret_cast<const float*>(smem + L.red);
-        const float* fa = reinterpret_cast<const float*>(smem + L.fa) + kMp;
         uint32_t it = 0;
         for (int rg = blockIdx.x; rg < rgs; rg += gridDim.x, ++it) {
             const int64_t n0 = (int64_t)rg * kRows;
@@ -510,7 +507,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                 float sum = 0.f;
 #pragma unroll
                 for (int w = 0; w < kCW; ++w) sum += rb[((size_t)w * kRows + r) * (kMp + 1) + mcol];
-                sum *= fa[mcol];  // the power of two taken out of activation row m
                 const int m = m0 + mcol;
                 if (m < prm.M) {
                     if (sizeof(OutT) == 4)
