@@ -415,41 +415,43 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
     for (int i = threadIdx.x; i < nkg * 128; i += 256) dst[i] = tile[(i >> 7) * 129 + (i & 127)];
 }
 
+// Four E2M1 codes (low 16 bits of x) -> four E4M3 bytes.  Magnitude: byte table lookup with
+// the codes' low three bits as selector.  Sign: a second lookup with the raw codes as selector
+// uses prmt's sign-replicate mode (selector bit 3): it returns 0xFF for a negative code and a
+// table byte whose bit 0 is clear for a positive one, so bit 0 of each byte is the sign.
+__device__ __forceinline__ uint32_t e2m1x4_to_e4m3x4(uint32_t x)
+{
+    const uint32_t mag = __byte_perm(0x3C383000u, 0x4C484440u, x & 0x7777u);
+    uint32_t neg;  // PTX prmt (not the intrinsic, which defines only three selector bits)
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(neg) : "r"(0x80808080u), "r"(x));
+    return mag | ((neg << 7) & 0x80808080u);
+}
+
 __device__ __forceinline__ void widen_e4m3(const PrepackOperand& op, unsigned id)
 {
-    const int64_t t = (int64_t)id * 256 + threadIdx.x;  // half block: 16 elements
-    const int64_t b = t >> 1;
-    if (b >= (int64_t)op.rows * op.nbk) return;
-    const uint2 w2 = reinterpret_cast<const uint2*>(op.nibbles)[t];
+    const uint32_t t = id * 256u + threadIdx.x;  // half block: 16 elements
+    const uint32_t b = t >> 1;
+    if (b >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
+    const uint2 w = reinterpret_cast<const uint2*>(op.nibbles)[t];
     const uint32_t sc = op.scales[b];
-    const uint32_t w[2] = {w2.x, w2.y};
-    uint32_t o[4];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t x = h ? (w[i] >> 16) : w[i];
-            const uint32_t mag = __byte_perm(0x3C383000u, 0x4C484440u, x & 0x7777u);
-            // sign bits 3, 7, 11, 15 -> 7, 15, 23, 31
-            const uint32_t sg = ((x & 0x8u) << 4) | ((x & 0x80u) << 8) | ((x & 0x800u) << 12) |
-                                ((x & 0x8000u) << 16);
-            o[2 * i + h] = mag | sg;
-        }
-    }
+    uint4 o;
+    o.x = e2m1x4_to_e4m3x4(w.x);
+    o.y = e2m1x4_to_e4m3x4(w.x >> 16);
+    o.z = e2m1x4_to_e4m3x4(w.y);
+    o.w = e2m1x4_to_e4m3x4(w.y >> 16);
+    if (sc == 0u) o = make_uint4(0u, 0u, 0u, 0u);
+    uint8_t* dst = op.wide + (size_t)t * 16u;
+    *reinterpret_cast<uint4*>(dst) = o;
     if (op.bm_index != nullptr) {
-        const uint32_t idx = op.bm_index[b] & 31u;
-        if ((idx >> 4) == (uint32_t)(t & 1)) {
-            const uint32_t e = idx & 15u;
-            const uint32_t nib = (w[e >> 3] >> ((e & 7u) * 4u)) & 0xFu;
-            const uint32_t byte = ((nib & 8u) << 4) | 0x48u | (nib & 7u);
-            const uint32_t sh = (e & 3u) * 8u;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if ((e >> 2) == (uint32_t)k) o[k] = (o[k] & ~(0xFFu << sh)) | (byte << sh);
-        }
+        // Eq. 3, BM branch.  Same thread, later store to the same bytes: lands after the
+        // vector store above.
+        const uint32_t p = op.bm_index[b] & 31u;
+        const uint32_t e = p & 15u;
+        const uint32_t word = (e & 8u) ? w.y : w.x;
+        const uint32_t nib = (word >> ((e & 7u) * 4u)) & 15u;
+        if ((p >> 4) == (t & 1u) && sc != 0u)
+            dst[e] = (uint8_t)(((nib & 8u) << 4) | 0x48u | (nib & 7u));
     }
-    if (sc == 0u) o[0] = o[1] = o[2] = o[3] = 0u;
-    reinterpret_cast<uint4*>(op.wide)[t] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, const PrepackOperand b,
@@ -568,6 +570,9 @@ mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUt
 size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
 {
     if (M <= 128 || N <= 128 || K % 128 != 0) return 0;
+    // the prepack kernel indexes half blocks (16 elements) of an operand with 32 bits
+    if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
+        return 0;
     const bool wide = a_mode == MXP_MODE_MXFP4_PLUS || b_mode == MXP_MODE_MXFP4_PLUS;
     return layout(M, N, K, wide).total;
 }
@@ -605,7 +610,9 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     };
     const PrepackOperand pa = operand(A, M, l.sfa, l.wa), pb = operand(B, N, l.sfb, l.wb);
     const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
-    if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
+    // the widening threads index their operand with 32 bits
+    if (ctas > 0x7FFFFFFFull || (uint64_t)M * nbk * 2 >= (1ull << 32) || (uint64_t)N * nbk * 2 >= (1ull << 32))
+        return MXP_ERR_UNSUPPORTED;
     prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, pb, static_cast<StatusBlock*>(workspace));
     if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
 
