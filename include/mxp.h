@@ -120,6 +120,37 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
                                     mxp_mode a_mode, mxp_mode b_mode);
 
 /*
+ * Weights prepared once.  mxp_gemm with the full workspace re-tiles the scales of both
+ * operands and, when either is MXFP4+, widens both to E4M3 bytes on every call (see
+ * `workspace` above).  For an operand that does not change between calls (the N x K
+ * weights) that work can be done once:
+ *   mxp_gemm_prepack_bytes  bytes of the prepacked form of a rows x K operand; `wide` != 0
+ *                           if the GEMMs it will be used in have an MXFP4+ operand on
+ *                           either side (then it holds one E4M3 byte per element, exact
+ *                           for every E2M1 value and for the BM values of Eq. 3), 0 for
+ *                           MXFP4 x MXFP4 (scale atoms only).  0: shape not supported
+ *                           (K % 128 != 0).
+ *   mxp_gemm_prepack        writes that form of `P` into `out` (device, 256-byte aligned,
+ *                           `out_bytes` >= the size above).  Asynchronous on `cuda_stream`.
+ *   mxp_gemm_prepacked      mxp_gemm's packed-operand form with B's prepacked copy:
+ *                           `B_prepacked` must come from mxp_gemm_prepack(B_packed, wide)
+ *                           with wide == (A is MXFP4+ or B is MXFP4+); B_packed still
+ *                           describes the operand (planes, shape, mode).  Needs M > 128 and
+ *                           N > 128 and mxp_gemm_workspace_bytes(...) of workspace
+ *                           (MXP_ERR_UNSUPPORTED / MXP_ERR_WORKSPACE otherwise; fall back
+ *                           to mxp_gemm).  Same result as mxp_gemm.
+ * The paper describes the format and its decode (Sec. 4, Eq. 3), not this staging: it is
+ * an implementation device of this library.
+ */
+size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide);
+mxp_status mxp_gemm_prepack(const mxp_packed *P, int wide, void *out, size_t out_bytes,
+                            void *cuda_stream);
+mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
+                              const mxp_packed *B_packed, const void *B_prepacked, void *D,
+                              mxp_dtype d_dt, int64_t ldd, void *workspace,
+                              size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM
  * left in `workspace`: MXP_OK, or MXP_ERR_TIMEOUT if a bounded wait inside a kernel gave
  * up (the output is then undefined but the context stays usable).

@@ -24,6 +24,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
 EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
+           "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_gemm_status", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
@@ -64,6 +65,13 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_workspace_bytes.restype = sz
         l.mxp_gemm_min_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
         l.mxp_gemm_min_workspace_bytes.restype = sz
+        l.mxp_gemm_prepack_bytes.argtypes = [i64, i64, ci]
+        l.mxp_gemm_prepack_bytes.restype = sz
+        l.mxp_gemm_prepack.argtypes = [ctypes.POINTER(_Packed), ci, vp, sz, vp]
+        l.mxp_gemm_prepack.restype = ci
+        l.mxp_gemm_prepacked.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
+                                         vp, vp, ci, i64, vp, sz, vp]
+        l.mxp_gemm_prepacked.restype = ci
         l.mxp_gemm_status.argtypes = [vp, vp]
         l.mxp_gemm_status.restype = ci
         l.mxp_tensor_peak_probe.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_double),
@@ -181,6 +189,38 @@ def mxp_gemm(a, b: Packed, out_dtype=torch.bfloat16, out: Optional[torch.Tensor]
         st = lib().mxp_gemm(M, N, K, None, 0, ctypes.byref(as_), ctypes.byref(bs),
                             out.data_ptr(), _dt(out), out.stride(0), ws_ptr, ws_len, _stream())
     _check("mxp_gemm", st)
+    return out
+
+
+def mxp_gemm_prepack(p: Packed, wide: bool, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Prepacked copy of an operand (normally the weights) for mxp_gemm_prepacked.  `wide` must
+    be True when either operand of the later GEMMs is MXFP4+."""
+    need = int(lib().mxp_gemm_prepack_bytes(p.rows, p.cols, int(wide)))
+    if need == 0:
+        raise MxpError("mxp_gemm_prepack_bytes", 2)
+    if out is None:
+        out = torch.empty(need, dtype=torch.uint8, device=p.nibbles.device)
+    cs = p.c_struct()
+    st = lib().mxp_gemm_prepack(ctypes.byref(cs), int(wide), out.data_ptr(), out.numel(), _stream())
+    _check("mxp_gemm_prepack", st)
+    return out
+
+
+def mxp_gemm_prepacked(a: Packed, b: Packed, b_prepacked: torch.Tensor, out_dtype=torch.bfloat16,
+                       out: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """D = dec(A) @ dec(B).T with B's prepacked copy from mxp_gemm_prepack."""
+    M, N, K = a.rows, b.rows, b.cols
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=b.nibbles.device)
+    if workspace is None:
+        workspace = torch.empty(mxp_gemm_workspace_bytes(M, N, K, False, a.mode, b.mode),
+                                dtype=torch.uint8, device=b.nibbles.device)
+    as_, bs = a.c_struct(), b.c_struct()
+    st = lib().mxp_gemm_prepacked(M, N, K, ctypes.byref(as_), ctypes.byref(bs), b_prepacked.data_ptr(),
+                                  out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
+                                  workspace.numel(), _stream())
+    _check("mxp_gemm_prepacked", st)
     return out
 
 

@@ -126,6 +126,42 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
                                workspace_bytes, stream);
 }
 
+size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide)
+{
+    return mxp::stream_prepack_bytes(rows, K, wide != 0);
+}
+
+mxp_status mxp_gemm_prepack(const mxp_packed* P, int wide, void* out, size_t out_bytes,
+                            void* cuda_stream)
+{
+    if (!valid_packed(P)) return MXP_ERR_INVALID_ARG;
+    if (P->rows == 0 || P->cols == 0) return MXP_OK;
+    if (P->mode == MXP_MODE_MXFP4_PLUS && !wide) return MXP_ERR_INVALID_ARG;
+    return mxp::stream_prepack(*P, wide != 0, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed* A_packed,
+                              const mxp_packed* B_packed, const void* B_prepacked, void* D,
+                              mxp_dtype d_dt, int64_t ldd, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream)
+{
+    if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(A_packed) || !valid_packed(B_packed)) return MXP_ERR_INVALID_ARG;
+    if (A_packed->rows != M || A_packed->cols != K || B_packed->rows != N || B_packed->cols != K)
+        return MXP_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return MXP_OK;
+    if (K == 0) return MXP_ERR_UNSUPPORTED;
+    if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
+    if (!aligned(A_packed->scales, 4) || !aligned(B_packed->scales, 4)) return MXP_ERR_INVALID_ARG;
+    if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)
+        return MXP_ERR_UNSUPPORTED;
+    return mxp::launch_gemm_tc_stream(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
+                                      workspace, workspace_bytes,
+                                      static_cast<cudaStream_t>(cuda_stream));
+}
+
 mxp_status mxp_gemm_status(const void* workspace, void* cuda_stream)
 {
     if (workspace == nullptr) return MXP_ERR_INVALID_ARG;

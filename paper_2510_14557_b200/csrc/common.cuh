@@ -44,8 +44,14 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
 // M, N > 128 and a workspace of stream_workspace_bytes() (0 = shape not supported).
 size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
-                                 const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                                 void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                                 const mxp_packed& B, const void* b_prepacked, void* D,
+                                 mxp_dtype d_dt, int64_t ldd, void* workspace,
+                                 size_t workspace_bytes, cudaStream_t stream);
+// One operand in the form that kernel reads (scale atoms; E4M3 bytes when `wide`), written
+// once, e.g. for weights.  stream_prepack_bytes() == 0: shape not supported.
+size_t stream_prepack_bytes(int64_t rows, int64_t K, bool wide);
+mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_bytes,
+                          cudaStream_t stream);
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no libcuda link).
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,

@@ -1248,7 +1248,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     const size_t fast = stream_workspace_bytes(M, N, K, A.mode, B.mode);
     const bool forced_other = force != nullptr && (force[0] == 's' || force[0] == 'p');
     if (fast != 0 && workspace_bytes >= fast && !forced_other)
-        return launch_gemm_tc_stream(M, N, K, A, B, D, d_dt, ldd, workspace, workspace_bytes, stream);
+        return launch_gemm_tc_stream(M, N, K, A, B, nullptr, D, d_dt, ldd, workspace, workspace_bytes,
+                                     stream);
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
         return MXP_ERR_CUDA;
     bool use_pair = M > 128 && N > 128 && (ap || bp);

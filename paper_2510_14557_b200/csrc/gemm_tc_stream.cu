@@ -460,7 +460,7 @@ __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, co
     __shared__ uint32_t tile[32 * 129];
     ptx::grid_launch_dependents();  // the GEMM's prologue may start while this grid drains
     unsigned id = blockIdx.x;
-    if (id == 0 && threadIdx.x == 0) {
+    if (id == 0 && threadIdx.x == 0 && status != nullptr) {
         status->code = 0u;  // the GEMM that follows on the stream reports into this block
         status->where = 0u;
     }
@@ -577,15 +577,83 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
     return layout(M, N, K, wide).total;
 }
 
+namespace {
+// Prepacked form of one operand in a caller-owned buffer: scale atoms, then (wide) E4M3 bytes.
+struct PackedLayout {
+    size_t atoms, wide, total;
+};
+PackedLayout packed_layout(int64_t rows, int64_t K, bool wide)
+{
+    PackedLayout l;
+    l.atoms = 0;
+    l.wide = round_up((size_t)((rows + 127) / 128) * (size_t)(K / 128) * kAtom, 1024);
+    l.total = l.wide + (wide ? round_up((size_t)rows * (size_t)K, 1024) : 0);
+    return l;
+}
+
+PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, bool wide, uint8_t* atoms,
+                               uint8_t* wide_bytes)
+{
+    const int nbk = (int)(K / 32);
+    const int kgroups = nbk / 4;
+    PrepackOperand op;
+    op.nibbles = P.nibbles;
+    op.scales = P.scales;
+    op.bm_index = P.mode == MXP_MODE_MXFP4_PLUS ? P.bm_index : nullptr;
+    op.atoms = atoms;
+    op.wide = wide ? wide_bytes : nullptr;
+    op.rows = (int)rows;
+    op.nbk = nbk;
+    op.scale_ctas = (unsigned)(((rows + 127) / 128) * ((kgroups + 31) / 32));
+    op.widen_ctas = wide ? (unsigned)((rows * nbk * 2 + 255) / 256) : 0u;
+    return op;
+}
+PrepackOperand no_operand()
+{
+    PrepackOperand op = {};
+    return op;
+}
+}  // namespace
+
+size_t stream_prepack_bytes(int64_t rows, int64_t K, bool wide)
+{
+    if (rows <= 0 || K <= 0 || K % 128 != 0) return 0;
+    if ((uint64_t)rows * (uint64_t)K / 16 >= (1ull << 32)) return 0;
+    return packed_layout(rows, K, wide).total;
+}
+
+mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_bytes,
+                          cudaStream_t stream)
+{
+    const size_t need = stream_prepack_bytes(P.rows, P.cols, wide);
+    if (need == 0) return MXP_ERR_UNSUPPORTED;
+    if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
+        (reinterpret_cast<uintptr_t>(P.scales) & 3))
+        return MXP_ERR_INVALID_ARG;
+    const PackedLayout l = packed_layout(P.rows, P.cols, wide);
+    uint8_t* o = static_cast<uint8_t*>(out);
+    const PrepackOperand pa = prepack_operand(P, P.rows, P.cols, wide, o + l.atoms, o + l.wide);
+    const uint64_t ctas = (uint64_t)pa.scale_ctas + pa.widen_ctas;
+    if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
+    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, no_operand(), nullptr);
+    return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+// `b_prepacked` (may be nullptr): B already in the form stream_prepack() writes for the same
+// `wide`; then only A is prepared here and the workspace needs no room for B.
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
-                                 const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                                 void* workspace, size_t workspace_bytes, cudaStream_t stream)
+                                 const mxp_packed& B, const void* b_prepacked, void* D,
+                                 mxp_dtype d_dt, int64_t ldd, void* workspace,
+                                 size_t workspace_bytes, cudaStream_t stream)
 {
     const bool ap = A.mode == MXP_MODE_MXFP4_PLUS, bp = B.mode == MXP_MODE_MXFP4_PLUS;
     const bool wide = ap || bp;
-    const Layout l = layout(M, N, K, wide);
+    const Layout l = layout(M, b_prepacked ? 0 : N, K, wide);
     if (workspace == nullptr || workspace_bytes < l.total) return MXP_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return MXP_ERR_INVALID_ARG;
+    if (b_prepacked != nullptr && (reinterpret_cast<uintptr_t>(b_prepacked) & 255))
+        return MXP_ERR_INVALID_ARG;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const int num_sms = sm_count();
     if (num_sms <= 0) return MXP_ERR_CUDA;
@@ -594,35 +662,28 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     const int rga = (int)((M + 127) / 128), rgb = (int)((N + 127) / 128);
     if ((reinterpret_cast<uintptr_t>(A.nibbles) | reinterpret_cast<uintptr_t>(B.nibbles)) & 15)
         return MXP_ERR_INVALID_ARG;
-
-    auto operand = [&](const mxp_packed& P, int64_t rows, size_t atoms_off, size_t wide_off) {
-        PrepackOperand op;
-        op.nibbles = P.nibbles;
-        op.scales = P.scales;
-        op.bm_index = P.mode == MXP_MODE_MXFP4_PLUS ? P.bm_index : nullptr;
-        op.atoms = ws + atoms_off;
-        op.wide = wide ? ws + wide_off : nullptr;
-        op.rows = (int)rows;
-        op.nbk = nbk;
-        op.scale_ctas = (unsigned)(((rows + 127) / 128) * ((kgroups + 31) / 32));
-        op.widen_ctas = wide ? (unsigned)((rows * nbk * 2 + 255) / 256) : 0u;
-        return op;
-    };
-    const PrepackOperand pa = operand(A, M, l.sfa, l.wa), pb = operand(B, N, l.sfb, l.wb);
-    const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
     // the widening threads index their operand with 32 bits
-    if (ctas > 0x7FFFFFFFull || (uint64_t)M * nbk * 2 >= (1ull << 32) || (uint64_t)N * nbk * 2 >= (1ull << 32))
+    if ((uint64_t)M * nbk * 2 >= (1ull << 32) || (uint64_t)N * nbk * 2 >= (1ull << 32))
         return MXP_ERR_UNSUPPORTED;
+
+    const PackedLayout lb = packed_layout(N, K, wide);
+    const uint8_t* b_atoms = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms : ws + l.sfb;
+    const uint8_t* b_wide = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.wide : ws + l.wb;
+    const PrepackOperand pa = prepack_operand(A, M, K, wide, ws + l.sfa, ws + l.wa);
+    const PrepackOperand pb =
+        b_prepacked ? no_operand() : prepack_operand(B, N, K, wide, ws + l.sfb, ws + l.wb);
+    const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
+    if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
     prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, pb, static_cast<StatusBlock*>(workspace));
     if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
 
     CUtensorMap ta, tb, tsa, tsb;
     const int box_kg = wide ? 1 : 2;
     const bool maps_ok =
-        (wide ? make_tmap_rows(&ta, ws + l.wa, M, K) && make_tmap_rows(&tb, ws + l.wb, N, K)
+        (wide ? make_tmap_rows(&ta, ws + l.wa, M, K) && make_tmap_rows(&tb, b_wide, N, K)
               : make_tmap_rows(&ta, A.nibbles, M, K / 2) && make_tmap_rows(&tb, B.nibbles, N, K / 2)) &&
         make_tmap_atoms(&tsa, ws + l.sfa, rga, kgroups, box_kg, 1) &&
-        make_tmap_atoms(&tsb, ws + l.sfb, rgb, kgroups, box_kg, 2);
+        make_tmap_atoms(&tsb, b_atoms, rgb, kgroups, box_kg, 2);
     if (!maps_ok) return MXP_ERR_CUDA;
 
     SParams prm;

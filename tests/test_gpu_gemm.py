@@ -196,3 +196,79 @@ def test_tc_both_kernels_every_mode(kernel, amode, bmode, monkeypatch):
     for dt in (torch.float32, torch.bfloat16):
         d = mxp().mxp_gemm(ap, bp, out_dtype=dt)
         check_gemm(d, da, db)
+
+
+# ------------------------------------------------------------------ streamed kernel, prepack
+def _raw_operand(rows, K, mode, seed, scale_lo=120, scale_hi=134):
+    """Packed planes filled directly: every code, BM position and mantissa occurs."""
+    g = synth.rng(seed)
+    nib = g.integers(0, 256, (rows, K // 2), dtype=np.uint8)
+    sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
+    idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8) if mode == MXP else None
+    dec = oracle.dequantize(nib, sc, idx, mode)
+    return host_to_packed(nib, sc, idx, mode), dec
+
+
+@pytest.mark.parametrize("amode,bmode", MODES)
+def test_tc_stream_every_code_position_and_mantissa(amode, bmode):
+    # B = identity (exactly representable): D must equal the oracle's decode of A bit for bit
+    # for random raw planes, i.e. for every E2M1 code, BM position and BM mantissa; shapes go
+    # to the streamed kernel (M, N > 128)
+    M, K = 384, 256
+    ap, da = _raw_operand(M, K, amode, seed=21)
+    eye = np.eye(K, dtype=np.float32)
+    bp, db = quantized(eye, bmode)
+    assert np.array_equal(db, eye.astype(np.float64))
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
+
+
+@pytest.mark.parametrize("amode,bmode", MODES)
+@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 129, 2176), (512, 512, 128)])
+def test_tc_prepacked_weights_match_mxp_gemm(M, N, K, amode, bmode):
+    ap, da = _raw_operand(M, K, amode, seed=M + 1)
+    bp, db = _raw_operand(N, K, bmode, seed=N + 2)
+    m = mxp()
+    wide = amode == MXP or bmode == MXP
+    pre = m.mxp_gemm_prepack(bp, wide)
+    for dt in (torch.float32, torch.bfloat16):
+        d0 = m.mxp_gemm(ap, bp, out_dtype=dt)
+        d1 = m.mxp_gemm_prepacked(ap, bp, pre, out_dtype=dt)
+        check_gemm(d1, da, db)
+        assert torch.equal(d0, d1)
+
+
+def test_tc_prepack_rejects_bad_arguments():
+    from paper_2510_14557_b200 import MxpError
+    m = mxp()
+    bp, _ = _raw_operand(256, 256, MXP, seed=5)
+    with pytest.raises(MxpError):  # an MXFP4+ operand has no narrow prepacked form
+        m.mxp_gemm_prepack(bp, False)
+    pre = m.mxp_gemm_prepack(bp, True)
+    small, _ = _raw_operand(64, 256, MXP, seed=6)
+    with pytest.raises(MxpError):  # M <= 128: no streamed kernel, the caller uses mxp_gemm
+        m.mxp_gemm_prepacked(small, bp, pre)
+    with pytest.raises(MxpError):
+        m.mxp_gemm_prepack(bp, True, out=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+
+
+def test_tc_stream_flushed_blocks_and_bm_coincidence():
+    # streamed-kernel shapes: BMs of both operands at the same position in every block,
+    # plus flushed (scale byte 0) and all-zero blocks
+    M, N, K = 192, 320, 512
+    g = synth.rng(9)
+    a = (g.standard_normal((M, K)) * 0.3).astype(np.float32)
+    b = (g.standard_normal((N, K)) * 0.3).astype(np.float32)
+    pos = g.integers(0, 32, K // 32)
+    for j, p in enumerate(pos):
+        a[:, 32 * j + p] = g.choice([4.5, 5.5, 6.5, 7.5, -5.0, -7.0], M)
+        b[:, 32 * j + p] = g.choice([4.5, 5.5, 6.5, 7.5, -4.5, -6.5], N)
+    a[5, 64:96] = 0
+    a[6, 96:128] = 1e-44
+    b[7, 0:32] = 0
+    b[8, 32:64] = -1e-44
+    ap, da = quantized(a, MXP)
+    bp, db = quantized(b, MXP)
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    ref = oracle.gemm_fp64(da, db)
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), ref)
