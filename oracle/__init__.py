@@ -19,6 +19,7 @@ import numpy as np
 
 MODE_MXFP4 = 0
 MODE_MXFP4_PLUS = 1
+MODE_MXFP4_PP = 2  # MX++ (Sec. 4.3)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "mxp_oracle.c")

@@ -20,7 +20,11 @@
  *   - several equal maxima: the lowest index is the BM;
  *   - the sign bit of the input is kept even when the magnitude rounds to zero;
  *   - element 2j sits in the low nibble of byte j; three separate row-major planes;
- *   - the flush rule and the reserved scale byte 0 apply in plain MXFP4 mode too.
+ *   - the flush rule and the reserved scale byte 0 apply in plain MXFP4 mode too;
+ *   - MX++ (Sec. 4.3): the scale byte keeps the BM's shared exponent, the three reserved
+ *     bits of the index byte hold delta = shared_exp - shared_exp_new; "second-largest
+ *     exponent" is the largest exponent among the non-zero NBM elements (the block
+ *     without its BM); a block whose NBMs are all zero takes the lower clip (delta = 7).
  */
 #include <math.h>
 #include <stdint.h>
@@ -32,6 +36,7 @@
 
 #define ORACLE_MODE_MXFP4 0
 #define ORACLE_MODE_MXFP4_PLUS 1
+#define ORACLE_MODE_MXFP4_PP 2 /* MX++ (Sec. 4.3): NBMs get their own, smaller shared exponent */
 
 /* Sec. 2: FP4 element = 1 sign, 2 exponent bits (bias 1), 1 mantissa bit,
  * implicit leading one, IEEE-like subnormals; emax = 3 - 1 = 2. */
@@ -139,14 +144,34 @@ static void quantize_block(const double *x, int k, int mode, uint8_t *nib,
     /* Eq. 1: shared_exp = max floor(log2|x|) - emax; E8M0 bias 127. */
     int se = floor_log2(amax) - EMAX;
     *scale = (uint8_t)(se + 127);
-    *index = (uint8_t)(mode == ORACLE_MODE_MXFP4_PLUS ? bm : 0);
+    int plus = (mode == ORACLE_MODE_MXFP4_PLUS || mode == ORACLE_MODE_MXFP4_PP);
+    int se_nbm = se;
+    if (mode == ORACLE_MODE_MXFP4_PP) {
+        /* Sec. 4.3: e = max2(floor(log2|x|)) - emax + 1 over the block without its BM,
+         * shared_exp_new = CLIP(e, {shared_exp - 7, shared_exp}). */
+        int have = 0, max2 = 0;
+        for (int i = 0; i < k; ++i) {
+            if (i == bm || x[i] == 0.0)
+                continue;
+            int ex = floor_log2(fabs(x[i]));
+            if (!have || ex > max2) {
+                max2 = ex;
+                have = 1;
+            }
+        }
+        se_nbm = se - 7; /* nothing but zeros beside the BM: the lower clip */
+        if (have) {
+            int e = max2 - EMAX + 1;
+            se_nbm = e < se - 7 ? se - 7 : (e > se ? se : e);
+        }
+    }
+    *index = (uint8_t)(plus ? (bm | ((se - se_nbm) << 5)) : 0);
     for (int i = 0; i < k; ++i) {
-        double r = ldexp(fabs(x[i]), -se); /* exact */
         int code;
-        if (mode == ORACLE_MODE_MXFP4_PLUS && i == bm)
-            code = bm_code(r); /* Sec. 4.1: exponent bits reused as mantissa */
+        if (plus && i == bm)
+            code = bm_code(ldexp(fabs(x[i]), -se)); /* Sec. 4.1: exponent bits reused as mantissa */
         else
-            code = e2m1_nearest(r);
+            code = e2m1_nearest(ldexp(fabs(x[i]), -se_nbm)); /* exact scaling */
         int sign = signbit(x[i]) ? 1 : 0;
         uint8_t n = (uint8_t)((sign << 3) | code);
         if (i & 1)
@@ -175,7 +200,7 @@ int oracle_quantize(const void *src, int src_kind, int64_t rows, int64_t cols,
 {
     if (k < 2 || k > 32 || (k & 1) || cols % k != 0 || rows < 0 || cols < 0)
         return -1;
-    if (mode != ORACLE_MODE_MXFP4 && mode != ORACLE_MODE_MXFP4_PLUS)
+    if (mode != ORACLE_MODE_MXFP4 && mode != ORACLE_MODE_MXFP4_PLUS && mode != ORACLE_MODE_MXFP4_PP)
         return -1;
     int64_t bpr = cols / k;
 #ifdef _OPENMP
@@ -214,7 +239,10 @@ int oracle_dequantize(const uint8_t *nibbles, const uint8_t *scales,
     for (int64_t r = 0; r < rows; ++r) {
         for (int64_t b = 0; b < bpr; ++b) {
             int sb = scales[r * bpr + b];
-            int bm = (mode == ORACLE_MODE_MXFP4_PLUS) ? (bm_index[r * bpr + b] & 31) : -1;
+            int plus = (mode == ORACLE_MODE_MXFP4_PLUS || mode == ORACLE_MODE_MXFP4_PP);
+            int bm = plus ? (bm_index[r * bpr + b] & 31) : -1;
+            /* MX++: the NBMs' shared exponent lies delta below the BM's */
+            int delta = (mode == ORACLE_MODE_MXFP4_PP) ? (bm_index[r * bpr + b] >> 5) : 0;
             for (int i = 0; i < k; ++i) {
                 uint8_t byte = nibbles[(r * cols + b * k + i) / 2];
                 int n = (i & 1) ? (byte >> 4) : (byte & 15);
@@ -226,12 +254,10 @@ int oracle_dequantize(const uint8_t *nibbles, const uint8_t *scales,
                 } else if (sb == 0xFF) {
                     out = NAN;
                 } else {
-                    double E;
                     if (i == bm) /* "MX+ addition": 2^emax * 1.mmm */
-                        E = ldexp(1.0 + (double)code / 8.0, EMAX);
+                        out = ldexp(ldexp(1.0 + (double)code / 8.0, EMAX), sb - 127);
                     else
-                        E = oracle_e2m1_value(code);
-                    out = ldexp(E, sb - 127);
+                        out = ldexp(oracle_e2m1_value(code), sb - 127 - delta);
                     if (s)
                         out = -out;
                 }
