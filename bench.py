@@ -223,10 +223,11 @@ def part_quantize(mxp, synth, peaks, iters):
     hbm = peaks["hbm_gbs"]
     x = dev_bf16(synth.config2())
     n = x.numel()
-    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
+    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4),
+                       ("mxfp4++", mxp.MODE_MXFP4_PP)):
         buf = mxp.alloc_packed(x.shape[0], x.shape[1], mode, index_for_mxfp4=False)
         ms = time_loop(lambda: mxp.mxp_quantize(x, mode, out=buf), iters)
-        nbytes = n * (2 + 0.5 + 1 / 32 + (1 / 32 if mode == mxp.MODE_MXFP4_PLUS else 0))
+        nbytes = n * (2 + 0.5 + 1 / 32 + (1 / 32 if mode != mxp.MODE_MXFP4 else 0))
         gbs = nbytes / ms / 1e6
         out["quantize_cfg2_" + name] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
     return out

@@ -12,6 +12,11 @@
  *   - in MXFP4+ mode the BM element stores 3 mantissa bits instead (E0M3, value
  *     4 + m/2 on the scaled grid, exponent implied) and a per-block index byte holds its
  *     position in bits 4:0 (bits 7:5 are written 0 and ignored on read);
+ *   - in MX++ mode (Sec. 4.3) the scale byte and the BM are those of MXFP4+, and the
+ *     other elements (NBMs) use shared_exp_new = CLIP(max2 - 2 + 1, {shared_exp - 7,
+ *     shared_exp}), max2 = the largest floor(log2|x|) among the non-zero NBMs (lower clip
+ *     if there are none); delta = shared_exp - shared_exp_new sits in bits 7:5 of the
+ *     index byte; an NBM decodes to 2^(shared_exp - delta) times its E2M1 value;
  *   - a block whose BM has floor(log2 BM) <= -125 is flushed: scale byte 0, all-zero
  *     nibbles, index 0; scale byte 0 decodes to 32 zeros in both modes;
  *   - a block holding Inf/NaN gets scale byte 0xFF and zero data (not defined by the
@@ -46,7 +51,11 @@ typedef enum {
     MXP_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see mxp_gemm_status) */
 } mxp_status;
 
-typedef enum { MXP_MODE_MXFP4 = 0, MXP_MODE_MXFP4_PLUS = 1 } mxp_mode;
+typedef enum {
+    MXP_MODE_MXFP4 = 0,
+    MXP_MODE_MXFP4_PLUS = 1, /* MX+  (Sec. 4.1): BM with 3 mantissa bits, index byte */
+    MXP_MODE_MXFP4_PP = 2    /* MX++ (Sec. 4.3): MX+ and a finer shared exponent for the NBMs */
+} mxp_mode;
 typedef enum { MXP_F32 = 0, MXP_BF16 = 1 } mxp_dtype;
 
 /* A packed operand: three row-major device planes. */

@@ -17,6 +17,7 @@ import torch
 MXP_OK = 0
 MODE_MXFP4 = 0
 MODE_MXFP4_PLUS = 1
+MODE_MXFP4_PP = 2
 F32 = 0
 BF16 = 1
 
@@ -129,7 +130,7 @@ def alloc_packed(rows: int, cols: int, mode: int, device="cuda", index_for_mxfp4
     nib = torch.empty((rows, cols // 2), dtype=torch.uint8, device=device)
     sc = torch.empty((rows, cols // 32), dtype=torch.uint8, device=device)
     idx = None
-    if mode == MODE_MXFP4_PLUS or index_for_mxfp4:
+    if mode != MODE_MXFP4 or index_for_mxfp4:
         idx = torch.empty((rows, cols // 32), dtype=torch.uint8, device=device)
     return Packed(nib, sc, idx, rows, cols, mode)
 

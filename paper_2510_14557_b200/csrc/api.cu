@@ -7,7 +7,10 @@ namespace {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-bool valid_mode(int m) { return m == MXP_MODE_MXFP4 || m == MXP_MODE_MXFP4_PLUS; }
+bool valid_mode(int m)
+{
+    return m == MXP_MODE_MXFP4 || m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP;
+}
 bool valid_dtype(int d) { return d == MXP_F32 || d == MXP_BF16; }
 
 // Checks an operand descriptor (host struct, device planes).
@@ -19,7 +22,7 @@ bool valid_packed(const mxp_packed* p)
     if (p->rows == 0 || p->cols == 0) return true;
     if (p->nibbles == nullptr || p->scales == nullptr) return false;
     if (!aligned(p->nibbles, 16)) return false;
-    if (p->mode == MXP_MODE_MXFP4_PLUS && p->bm_index == nullptr) return false;
+    if (p->mode != MXP_MODE_MXFP4 && p->bm_index == nullptr) return false;
     return true;
 }
 
@@ -50,7 +53,7 @@ mxp_status mxp_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t
     if (rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return MXP_OK;
     if (src == nullptr || nibbles == nullptr || scales == nullptr) return MXP_ERR_INVALID_ARG;
-    if (mode == MXP_MODE_MXFP4_PLUS && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (mode != MXP_MODE_MXFP4 && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
     if (ld_src < cols || ld_src % 8 != 0) return MXP_ERR_INVALID_ARG;
     if (!aligned(src, 16) || !aligned(nibbles, 16)) return MXP_ERR_INVALID_ARG;
     if (rows * (cols / 32) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
@@ -108,6 +111,10 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     if (K == 0) return MXP_ERR_UNSUPPORTED;  // an empty sum; callers zero D themselves
+    // MX++ operands: quantize and decode only so far
+    if (B_packed->mode == MXP_MODE_MXFP4_PP ||
+        (A_packed != nullptr && A_packed->mode == MXP_MODE_MXFP4_PP))
+        return MXP_ERR_UNSUPPORTED;
     const size_t need = mxp_gemm_min_workspace_bytes(M, N, K, A_dense_bf16 != nullptr,
                                                      A_packed ? A_packed->mode : MXP_MODE_MXFP4,
                                                      B_packed->mode);
@@ -136,6 +143,7 @@ mxp_status mxp_gemm_prepack(const mxp_packed* P, int wide, void* out, size_t out
 {
     if (!valid_packed(P)) return MXP_ERR_INVALID_ARG;
     if (P->rows == 0 || P->cols == 0) return MXP_OK;
+    if (P->mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
     if (P->mode == MXP_MODE_MXFP4_PLUS && !wide) return MXP_ERR_INVALID_ARG;
     return mxp::stream_prepack(*P, wide != 0, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -153,6 +161,8 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
     if (M == 0 || N == 0) return MXP_OK;
     if (K == 0) return MXP_ERR_UNSUPPORTED;
     if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (A_packed->mode == MXP_MODE_MXFP4_PP || B_packed->mode == MXP_MODE_MXFP4_PP)
+        return MXP_ERR_UNSUPPORTED;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     if (!aligned(A_packed->scales, 4) || !aligned(B_packed->scales, 4)) return MXP_ERR_INVALID_ARG;
     if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)

@@ -8,6 +8,11 @@
 //     (|x| bit pattern, 31 - position), reduced over the four lanes by two shuffles.
 // Either way the BM falls out of the scale computation: the paper's point that it is found
 // for free during conversion.
+//
+// Mode 2 is MX++ (Sec. 4.3): the NBMs are scaled with their own shared exponent
+// shared_exp_new = CLIP(max2 - emax + 1, {shared_exp - 7, shared_exp}), max2 the largest
+// exponent among the non-zero NBMs; delta = shared_exp - shared_exp_new goes into the three
+// reserved bits of the index byte.  The scale byte and the BM nibble are those of MX+.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -64,25 +69,48 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p)
 // One block's worth of work for this lane (quarter q of block `blk`).
 //   returns the packed nibble word; writes the block's scale / index bytes (same value in
 //   all four lanes of the group).
-template <bool kPlus>
-__device__ __forceinline__ uint32_t encode_quarter(const float (&v)[8], uint32_t amax_bits,
-                                                   int bm, int q, uint32_t& scale_byte,
-                                                   uint32_t& index_byte)
+// Biased floor(log2) of a non-zero fp32 magnitude pattern (127 = 2^0), subnormals included.
+__device__ __forceinline__ int biased_floor_log2(uint32_t a)
 {
+    const int e = (int)(a >> 23);
+    return e != 0 ? e : 9 - __clz((int)a);
+}
+// MX++: delta = shared_exp - shared_exp_new from the biased exponents of the BM (E) and of
+// the largest NBM magnitude pattern (a2, fp32 bits; 0: every NBM is zero).
+__device__ __forceinline__ uint32_t mxpp_delta(uint32_t E, uint32_t a2)
+{
+    const int se_b = (int)E - 2;
+    int nb = se_b - 7;
+    if (a2 != 0u) nb = min(max(biased_floor_log2(a2) - 1, se_b - 7), se_b);
+    return (uint32_t)(se_b - nb);
+}
+
+// kMode: 0 MXFP4, 1 MXFP4+, 2 MX++.  a2_bits (MX++ only): largest NBM magnitude of the block.
+template <int kMode>
+__device__ __forceinline__ uint32_t encode_quarter(const float (&v)[8], uint32_t amax_bits,
+                                                   uint32_t a2_bits, int bm, int q,
+                                                   uint32_t& scale_byte, uint32_t& index_byte)
+{
+    constexpr bool kPlus = kMode >= 1;
     // amax_bits: fp32 bit pattern of the block's absolute maximum
     const uint32_t E = amax_bits >> 23;  // biased exponent (sign already cleared)
     const bool flush = E <= 2u;          // floor(log2 BM) <= -125, zero and subnormals
     const bool nonfinite = E == 255u;
     scale_byte = flush ? 0u : (nonfinite ? 255u : E - 2u);
-    index_byte = (kPlus && !flush && !nonfinite) ? (uint32_t)bm : 0u;
+    const uint32_t delta = (kMode == 2 && !flush && !nonfinite) ? mxpp_delta(E, a2_bits) : 0u;
+    index_byte = (kPlus && !flush && !nonfinite) ? ((uint32_t)bm | (delta << 5)) : 0u;
 
-    // 2^-shared_exp = 2^(129 - E): biased exponent 256 - E, in [2, 253] for a kept block
-    const float inv = __uint_as_float((256u - E) << 23);
+    // 2^-shared_exp(_new) = 2^(129 - E + delta): biased exponent 256 - E + delta, in [2, 253]
+    // without delta; with it the factor is applied in two exact steps
+    const uint32_t kexp = 256u - E + delta;
+    const float inv = __uint_as_float(min(kexp, 254u) << 23);
+    const float inv_hi = __uint_as_float((127u + kexp - min(kexp, 254u)) << 23);
     float s[8];
     uint32_t sign = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         s[i] = v[i] * inv;  // exact (power of two); < 8 in magnitude
+        if (kMode == 2) s[i] *= inv_hi;
         sign |= (__float_as_uint(v[i]) >> 31) << (4 * i + 3);
     }
     // codes from the hardware cast; the sign bit of each nibble is taken from the input so
@@ -102,7 +130,7 @@ __device__ __forceinline__ uint32_t encode_quarter(const float (&v)[8], uint32_t
 }
 
 // kContig: ld_src == cols, so the source is one flat array of blocks.
-template <typename T, bool kPlus, bool kContig>
+template <typename T, int kMode, bool kContig>
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
                 int64_t total_blocks, uint8_t* __restrict__ nibbles,
@@ -182,8 +210,19 @@ quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
             amax_bits = a;
             bm = first & 31;
         }
+        uint32_t a2 = 0;
+        if (kMode == 2) {
+            // largest magnitude among the block's other elements (fp32 bit patterns)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t a = __float_as_uint(v[j][i]) & 0x7FFFFFFFu;
+                if (q * 8 + i != bm) a2 = max(a2, a);
+            }
+            a2 = max(a2, __shfl_xor_sync(0xFFFFFFFFu, a2, 1));
+            a2 = max(a2, __shfl_xor_sync(0xFFFFFFFFu, a2, 2));
+        }
         uint32_t sb, ib;
-        words[j] = encode_quarter<kPlus>(v[j], amax_bits, bm, q, sb, ib);
+        words[j] = encode_quarter<kMode>(v[j], amax_bits, a2, bm, q, sb, ib);
         sc_pack |= sb << (8 * j);
         ix_pack |= ib << (8 * j);
     }
@@ -254,7 +293,7 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8_bf16(uint32_t p0, uint32_t p1, ui
 // 64 bytes with four 128-bit loads.  Neighbouring lanes' loads fall into the same 128-byte
 // lines, which L1 serves; nibbles leave as one 128-bit store per lane (fully coalesced) and
 // the scale / index bytes as 32 consecutive bytes per warp.
-template <bool kPlus>
+template <int kMode>
 __global__ void __launch_bounds__(kThreads)
 quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
                           uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
@@ -280,31 +319,54 @@ quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
     const uint32_t E = amax16 >> 7;
     const bool dead = E <= 2u || E == 255u;  // flushed or non-finite: data is all zero
     const uint32_t sb = E <= 2u ? 0u : (E == 255u ? 255u : E - 2u);
-    const uint32_t inv2 = ((256u - E) << 7) * 0x00010001u;  // 2^-shared_exp as a bf16 pair
+    constexpr bool kPlus = kMode >= 1;
+    uint32_t bm = 0, m = 0, delta = 0;
+    if (kPlus) {
+        // one bit per element where |x| equals the maximum; lowest set bit = first BM
+        uint32_t r1 = 0, r2 = 0;
+        uint32_t eq[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(eq[i]) : "r"(t[i]), "r"(m2));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t sel = (1u << (2 * i)) | (1u << (16 + 2 * i));
+            r1 |= eq[i] & sel;
+            r2 |= eq[8 + i] & sel;
+        }
+        // even elements sit in bits 0,2,..14, odd ones in bits 16,18,..30: interleave
+        const uint32_t lo = (r1 & 0xFFFFu) | ((r1 >> 15) & 0xAAAAu);
+        const uint32_t hi = (r2 & 0xFFFFu) | ((r2 >> 15) & 0xAAAAu);
+        const uint32_t map = lo | (hi << 16);
+        bm = (uint32_t)(__ffs((int)map) - 1) & 31u;
+        const uint32_t mant = amax16 & 0x7Fu;
+        m = min((mant + 7u + ((mant >> 4) & 1u)) >> 4, 7u);
+        if (kMode == 2) {
+            // MX++: largest magnitude among the NBMs.  Clearing every element equal to the
+            // maximum leaves the smaller ones; if the maximum occurs twice it is an NBM too.
+            uint32_t n2 = t[0] & ~eq[0];
+#pragma unroll
+            for (int i = 1; i < 16; ++i) n2 = bf16x2_max_nan(n2, t[i] & ~eq[i]);
+            n2 = bf16x2_max_nan(n2, __byte_perm(n2, n2, 0x1032));
+            const uint32_t a2 = (__popc(map) >= 2 ? amax16 : (n2 & 0xFFFFu)) << 16;
+            delta = dead ? 0u : mxpp_delta(E, a2);
+        }
+    }
+    // 2^-shared_exp(_new) as a bf16 pair: exponent field 256 - E + delta; beyond 254 (only
+    // blocks near the bottom of the bf16 range) the factor is applied in two exact steps
+    const uint32_t kexp = 256u - E + delta;
+    const uint32_t inv2 = (min(kexp, 254u) << 7) * 0x00010001u;
+    if (kMode == 2 && kexp > 254u) {
+        const uint32_t up = ((127u + kexp - 254u) << 7) * 0x00010001u;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = bf16x2_mul(x[i], up);
+    }
     uint32_t w[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
         w[i] = cvt_e2m1x8_bf16(bf16x2_mul(x[4 * i], inv2), bf16x2_mul(x[4 * i + 1], inv2),
                                bf16x2_mul(x[4 * i + 2], inv2), bf16x2_mul(x[4 * i + 3], inv2));
-    uint32_t bm = 0;
     if (kPlus) {
-        // one bit per element where |x| equals the maximum; lowest set bit = first BM
-        uint32_t r1 = 0, r2 = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            uint32_t e1, e2;
-            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e1) : "r"(t[i]), "r"(m2));
-            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e2) : "r"(t[8 + i]), "r"(m2));
-            const uint32_t sel = (1u << (2 * i)) | (1u << (16 + 2 * i));
-            r1 |= e1 & sel;
-            r2 |= e2 & sel;
-        }
-        // even elements sit in bits 0,2,..14, odd ones in bits 16,18,..30: interleave
-        const uint32_t lo = (r1 & 0xFFFFu) | ((r1 >> 15) & 0xAAAAu);
-        const uint32_t hi = (r2 & 0xFFFFu) | ((r2 >> 15) & 0xAAAAu);
-        bm = (uint32_t)(__ffs((int)(lo | (hi << 16))) - 1) & 31u;
-        const uint32_t mant = amax16 & 0x7Fu;
-        const uint32_t m = min((mant + 7u + ((mant >> 4) & 1u)) >> 4, 7u);
         const uint32_t sh = (bm & 7u) * 4u;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
@@ -314,7 +376,7 @@ quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
     const uint4 outv = dead ? make_uint4(0, 0, 0, 0) : make_uint4(w[0], w[1], w[2], w[3]);
     __stcs(nibbles + blk, outv);
     scales[blk] = (uint8_t)sb;
-    if (bm_index != nullptr) bm_index[blk] = (uint8_t)(dead ? 0u : bm);
+    if (bm_index != nullptr) bm_index[blk] = (uint8_t)(dead ? 0u : (bm | (delta << 5)));
 }
 
 // ------------------------------------------------------------------------- decode (Eq. 3)
@@ -327,7 +389,7 @@ __device__ __forceinline__ float e2m1_mag(uint32_t code)
     return e == 0u ? 0.5f * (float)m : normal;
 }
 
-template <typename T, bool kPlus>
+template <typename T, int kMode>
 __global__ void __launch_bounds__(kThreads)
 dequantize_kernel(const uint8_t* __restrict__ nibbles, const uint8_t* __restrict__ scales,
                   const uint8_t* __restrict__ bm_index, int64_t cols, int64_t total_units,
@@ -339,17 +401,21 @@ dequantize_kernel(const uint8_t* __restrict__ nibbles, const uint8_t* __restrict
     const int q = (int)(u & 3);
     const uint32_t word = __ldg(reinterpret_cast<const uint32_t*>(nibbles) + u);
     const uint32_t sb = scales[blk];
-    const int bm = kPlus ? (int)(bm_index[blk] & 31u) : -1;
+    constexpr bool kPlus = kMode >= 1;
+    const uint32_t ib = kPlus ? bm_index[blk] : 0u;
+    const int bm = kPlus ? (int)(ib & 31u) : -1;
     float out[8];
     // 2^(sb - 127) for sb in 1..254; sb = 0 is the reserved all-zero block; 0xFF decodes NaN
     const float scale = __uint_as_float(sb << 23);
+    // MX++: the NBMs' shared exponent lies delta below (the product may be subnormal: exact)
+    const float scale_nbm = kMode == 2 ? scale * __uint_as_float((127u - (ib >> 5)) << 23) : scale;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const uint32_t n = (word >> (4 * i)) & 15u;
         const uint32_t code = n & 7u;
-        float mag = e2m1_mag(code);
-        if (kPlus && q * 8 + i == bm) mag = 4.0f + 0.5f * (float)code;  // "MX+ addition"
-        float val = mag * scale;  // exact: <= 4 significant bits times a power of two
+        const bool is_bm = kPlus && q * 8 + i == bm;
+        const float mag = is_bm ? 4.0f + 0.5f * (float)code : e2m1_mag(code);  // "MX+ addition"
+        float val = mag * (is_bm ? scale : scale_nbm);  // exact: <= 4 significant bits times 2^k
         if (sb == 0u) val = 0.0f;
         if (sb == 255u) val = __uint_as_float(0x7FC00000u);
         out[i] = (n & 8u) ? -val : val;
@@ -373,7 +439,7 @@ dequantize_kernel(const uint8_t* __restrict__ nibbles, const uint8_t* __restrict
     }
 }
 
-template <typename T, bool kPlus>
+template <typename T, int kMode>
 cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src,
                      uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index, cudaStream_t stream)
 {
@@ -382,16 +448,16 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
     const int aligned4 = ((reinterpret_cast<uintptr_t>(scales) & 3) == 0) &&
                          ((reinterpret_cast<uintptr_t>(bm_index) & 3) == 0);
     if (ld_src == cols && sizeof(T) == 2)
-        quantize_bf16_lane_kernel<kPlus>
+        quantize_bf16_lane_kernel<kMode>
             <<<(unsigned)((total_blocks + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
                 static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles),
                 scales, bm_index);
     else if (ld_src == cols)
-        quantize_kernel<T, kPlus, true><<<(unsigned)grid, kThreads, 0, stream>>>(
+        quantize_kernel<T, kMode, true><<<(unsigned)grid, kThreads, 0, stream>>>(
             static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales,
             bm_index, aligned4);
     else
-        quantize_kernel<T, kPlus, false><<<(unsigned)grid, kThreads, 0, stream>>>(
+        quantize_kernel<T, kMode, false><<<(unsigned)grid, kThreads, 0, stream>>>(
             static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales,
             bm_index, aligned4);
     return cudaGetLastError();
@@ -403,42 +469,52 @@ cudaError_t launch_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t
                             int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
                             uint8_t* bm_index, cudaStream_t stream)
 {
-    const bool plus = mode == MXP_MODE_MXFP4_PLUS;
-    if (dt == MXP_BF16)
-        return plus ? launch_q<__nv_bfloat16, true>(src, rows, cols, ld_src, nibbles, scales,
-                                                    bm_index, stream)
-                    : launch_q<__nv_bfloat16, false>(src, rows, cols, ld_src, nibbles, scales,
-                                                     bm_index, stream);
-    return plus ? launch_q<float, true>(src, rows, cols, ld_src, nibbles, scales, bm_index,
-                                        stream)
-                : launch_q<float, false>(src, rows, cols, ld_src, nibbles, scales, bm_index,
-                                         stream);
+    if (dt == MXP_BF16) {
+        switch (mode) {
+            case MXP_MODE_MXFP4_PP:
+                return launch_q<__nv_bfloat16, 2>(src, rows, cols, ld_src, nibbles, scales, bm_index, stream);
+            case MXP_MODE_MXFP4_PLUS:
+                return launch_q<__nv_bfloat16, 1>(src, rows, cols, ld_src, nibbles, scales, bm_index, stream);
+            default:
+                return launch_q<__nv_bfloat16, 0>(src, rows, cols, ld_src, nibbles, scales, bm_index, stream);
+        }
+    }
+    switch (mode) {
+        case MXP_MODE_MXFP4_PP:
+            return launch_q<float, 2>(src, rows, cols, ld_src, nibbles, scales, bm_index, stream);
+        case MXP_MODE_MXFP4_PLUS:
+            return launch_q<float, 1>(src, rows, cols, ld_src, nibbles, scales, bm_index, stream);
+        default:
+            return launch_q<float, 0>(src, rows, cols, ld_src, nibbles, scales, bm_index, stream);
+    }
+}
+
+template <typename T>
+static cudaError_t launch_dq(const mxp_packed& p, T* dst, int64_t ld_dst, cudaStream_t stream)
+{
+    const int64_t units = p.rows * p.cols / 8;
+    const unsigned grid = (unsigned)((units + kThreads - 1) / kThreads);
+    switch (p.mode) {
+        case MXP_MODE_MXFP4_PP:
+            dequantize_kernel<T, 2><<<grid, kThreads, 0, stream>>>(p.nibbles, p.scales, p.bm_index,
+                                                                   p.cols, units, dst, ld_dst);
+            break;
+        case MXP_MODE_MXFP4_PLUS:
+            dequantize_kernel<T, 1><<<grid, kThreads, 0, stream>>>(p.nibbles, p.scales, p.bm_index,
+                                                                   p.cols, units, dst, ld_dst);
+            break;
+        default:
+            dequantize_kernel<T, 0><<<grid, kThreads, 0, stream>>>(p.nibbles, p.scales, p.bm_index,
+                                                                   p.cols, units, dst, ld_dst);
+    }
+    return cudaGetLastError();
 }
 
 cudaError_t launch_dequantize(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
                               cudaStream_t stream)
 {
-    const int64_t units = p.rows * p.cols / 8;
-    const unsigned grid = (unsigned)((units + kThreads - 1) / kThreads);
-    const bool plus = p.mode == MXP_MODE_MXFP4_PLUS;
-    if (dt == MXP_F32) {
-        if (plus)
-            dequantize_kernel<float, true><<<grid, kThreads, 0, stream>>>(
-                p.nibbles, p.scales, p.bm_index, p.cols, units, static_cast<float*>(dst), ld_dst);
-        else
-            dequantize_kernel<float, false><<<grid, kThreads, 0, stream>>>(
-                p.nibbles, p.scales, p.bm_index, p.cols, units, static_cast<float*>(dst), ld_dst);
-    } else {
-        if (plus)
-            dequantize_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, stream>>>(
-                p.nibbles, p.scales, p.bm_index, p.cols, units,
-                static_cast<__nv_bfloat16*>(dst), ld_dst);
-        else
-            dequantize_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, stream>>>(
-                p.nibbles, p.scales, p.bm_index, p.cols, units,
-                static_cast<__nv_bfloat16*>(dst), ld_dst);
-    }
-    return cudaGetLastError();
+    if (dt == MXP_F32) return launch_dq(p, static_cast<float*>(dst), ld_dst, stream);
+    return launch_dq(p, static_cast<__nv_bfloat16*>(dst), ld_dst, stream);
 }
 
 }  // namespace mxp

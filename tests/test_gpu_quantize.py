@@ -4,11 +4,11 @@ import pytest
 import torch
 
 import oracle
-from helpers import packed_to_host, host_to_packed, to_dev, to_dev_bf16
+from helpers import bf16_round, packed_to_host, host_to_packed, to_dev, to_dev_bf16
 from paper_2510_14557_b200 import synth
 
 pytestmark = pytest.mark.gpu
-MX, MXP = 0, 1
+MX, MXP, MXPP = 0, 1, 2   # MXPP: MX++ (Sec. 4.3)
 
 
 def mxp():
@@ -21,7 +21,7 @@ def assert_planes_equal(p, ref, mode, what=""):
     rn, rs, ri = ref
     assert np.array_equal(sc, rs), "scales differ " + what
     assert np.array_equal(nib, rn), "nibbles differ %s (%d bytes)" % (what, int((nib != rn).sum()))
-    if mode == MXP:
+    if mode != MX:
         assert np.array_equal(idx, ri), "indices differ " + what
 
 
@@ -56,7 +56,7 @@ def adversarial_f32():
     return x.reshape(-1, 128)  # four blocks per row
 
 
-@pytest.mark.parametrize("mode", [MX, MXP])
+@pytest.mark.parametrize("mode", [MX, MXP, MXPP])
 def test_config1_fp32_bit_exact(mode):
     a, b = synth.config1()
     for x in (a, b):
@@ -64,7 +64,7 @@ def test_config1_fp32_bit_exact(mode):
         assert_planes_equal(p, oracle.quantize(x, mode), mode)
 
 
-@pytest.mark.parametrize("mode", [MX, MXP])
+@pytest.mark.parametrize("mode", [MX, MXP, MXPP])
 def test_adversarial_blocks_fp32_and_bf16(mode):
     x = adversarial_f32()
     p = mxp().mxp_quantize(to_dev(x), mode)
@@ -74,7 +74,7 @@ def test_adversarial_blocks_fp32_and_bf16(mode):
     assert_planes_equal(p, oracle.quantize(bits, mode, bf16_bits=True), mode, "bf16")
 
 
-@pytest.mark.parametrize("mode", [MX, MXP])
+@pytest.mark.parametrize("mode", [MX, MXP, MXPP])
 def test_every_bf16_pattern_as_block_max(mode):
     # all 65536 bf16 bit patterns, each once as the first element of a block
     bits = np.zeros((2048, 32 * 32), np.uint16)
@@ -87,7 +87,7 @@ def test_every_bf16_pattern_as_block_max(mode):
 
 
 @pytest.mark.parametrize("shape", [(1, 32), (3, 96), (5, 8192), (257, 2080), (1000, 32), (64, 4096)])
-@pytest.mark.parametrize("mode", [MX, MXP])
+@pytest.mark.parametrize("mode", [MX, MXP, MXPP])
 def test_ragged_sizes_bf16(shape, mode):
     bits = synth.config2(shape[0], shape[1], seed=shape[0] + shape[1])
     p = mxp().mxp_quantize(to_dev_bf16(bits), mode)
@@ -125,7 +125,7 @@ def test_empty_input_is_a_no_op():
     assert p.nibbles.numel() == 0
 
 
-@pytest.mark.parametrize("mode", [MX, MXP])
+@pytest.mark.parametrize("mode", [MX, MXP, MXPP])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_dequantize_bit_exact(mode, dtype):
     m = mxp()
@@ -133,9 +133,12 @@ def test_dequantize_bit_exact(mode, dtype):
     x = np.nan_to_num(x, nan=0.0, posinf=3e38, neginf=-3e38)
     nib, sc, idx = oracle.quantize(x, mode)
     ref = oracle.dequantize(nib, sc, idx, mode)
-    got = m.mxp_dequantize(host_to_packed(nib, sc, idx if mode == MXP else None, mode), dtype)
+    got = m.mxp_dequantize(host_to_packed(nib, sc, idx if mode != MX else None, mode), dtype)
     g = got.float().cpu().numpy().astype(np.float64)
-    # decode is exact in both output types, signed zeros included
+    # decode is exact in both output types, signed zeros included (MX++ NBMs of blocks at the
+    # very bottom of the range fall below bf16's subnormal grid: nearest-even there)
+    if mode == MXPP and dtype == torch.bfloat16:
+        ref = bf16_round(ref)
     assert np.array_equal(g, ref)
     assert np.array_equal(np.signbit(g), np.signbit(ref))
 
@@ -155,7 +158,40 @@ def test_dequantize_all_codes_every_position():
         nib[r, pos // 2] = (byte & 0x0F) | (nibv << 4) if pos & 1 else (byte & 0xF0) | nibv
         idx[r, 0] = pos | 0xE0  # reserved bits set: must be ignored
         sc[r, 0] = [1, 126, 127, 130, 252, 0][r % 6]  # 252: largest byte the quantizer emits
-    for mode in (MX, MXP):
+    for mode in (MX, MXP, MXPP):   # in MX++ mode the top index bits are delta = 7
         ref = oracle.dequantize(nib, sc, idx, mode)
         got = m.mxp_dequantize(host_to_packed(nib, sc, idx, mode), torch.float32)
         assert np.array_equal(got.cpu().numpy().astype(np.float64), ref)
+
+
+def test_mxpp_second_maximum_cases():
+    # MX++ (Sec. 4.3): blocks that exercise the NBM exponent: maximum occurring twice,
+    # NBMs all zero, NBM maximum in every binade below the BM, subnormal NBMs, tiny blocks
+    rows = []
+    for sh in (0, 40, -40, -110, -118, 100):
+        for gap in range(0, 12):
+            b = np.zeros(32, np.float32)
+            b[7] = -1.75
+            b[20] = 1.3 * 2.0 ** -gap
+            b[21] = -0.9 * 2.0 ** -gap
+            b[3] = 0.11 * 2.0 ** -gap
+            rows.append(b * np.float32(2.0 ** sh))
+    b = np.zeros(32, np.float32); b[9] = 5.0; rows.append(b.copy())                 # NBMs all zero
+    b[30] = 5.0; rows.append(b.copy())                                              # maximum twice
+    b = np.zeros(32, np.float32); b[0] = 2.0 ** -100; b[1] = 1e-41; rows.append(b.copy())  # subnormal NBM
+    b = np.zeros(32, np.float32); b[0] = 2.0 ** -121; b[1] = 2.0 ** -127; rows.append(b.copy())
+    x = np.stack(rows)
+    x = np.concatenate([x, np.zeros(((-x.shape[0]) % 4, 32), np.float32)]).reshape(-1, 128)
+    p = mxp().mxp_quantize(to_dev(x), MXPP)
+    ref = oracle.quantize(x, MXPP)
+    assert_planes_equal(p, ref, MXPP, "fp32")
+    assert int((ref[2] >> 5).max()) == 7 and int((ref[2] >> 5).min()) == 0
+    bits = synth.f32_to_bf16_bits(x)
+    p = mxp().mxp_quantize(to_dev_bf16(bits), MXPP)
+    assert_planes_equal(p, oracle.quantize(bits, MXPP, bf16_bits=True), MXPP, "bf16")
+    wide = torch.zeros((x.shape[0], 256), dtype=torch.bfloat16, device="cuda")      # strided bf16
+    wide[:, :128] = to_dev_bf16(bits)
+    p = mxp().mxp_quantize(wide[:, :128], MXPP)
+    assert_planes_equal(p, oracle.quantize(bits, MXPP, bf16_bits=True), MXPP, "bf16 strided")
+    got = mxp().mxp_dequantize(p, torch.float32).cpu().numpy().astype(np.float64)
+    assert np.array_equal(got, oracle.dequantize(*oracle.quantize(bits, MXPP, bf16_bits=True), MXPP))
