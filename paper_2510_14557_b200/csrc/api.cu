@@ -111,10 +111,8 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     if (K == 0) return MXP_ERR_UNSUPPORTED;  // an empty sum; callers zero D themselves
-    // MX++ operands: quantize and decode only so far
-    if (B_packed->mode == MXP_MODE_MXFP4_PP ||
-        (A_packed != nullptr && A_packed->mode == MXP_MODE_MXFP4_PP))
-        return MXP_ERR_UNSUPPORTED;
+    // MX++ weights with bf16 activations: not built yet
+    if (A_packed == nullptr && B_packed->mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
     const size_t need = mxp_gemm_min_workspace_bytes(M, N, K, A_dense_bf16 != nullptr,
                                                      A_packed ? A_packed->mode : MXP_MODE_MXFP4,
                                                      B_packed->mode);
@@ -143,8 +141,7 @@ mxp_status mxp_gemm_prepack(const mxp_packed* P, int wide, void* out, size_t out
 {
     if (!valid_packed(P)) return MXP_ERR_INVALID_ARG;
     if (P->rows == 0 || P->cols == 0) return MXP_OK;
-    if (P->mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
-    if (P->mode == MXP_MODE_MXFP4_PLUS && !wide) return MXP_ERR_INVALID_ARG;
+    if (P->mode != MXP_MODE_MXFP4 && !wide) return MXP_ERR_INVALID_ARG;
     return mxp::stream_prepack(*P, wide != 0, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -161,8 +158,6 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
     if (M == 0 || N == 0) return MXP_OK;
     if (K == 0) return MXP_ERR_UNSUPPORTED;
     if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
-    if (A_packed->mode == MXP_MODE_MXFP4_PP || B_packed->mode == MXP_MODE_MXFP4_PP)
-        return MXP_ERR_UNSUPPORTED;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     if (!aligned(A_packed->scales, 4) || !aligned(B_packed->scales, 4)) return MXP_ERR_INVALID_ARG;
     if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)

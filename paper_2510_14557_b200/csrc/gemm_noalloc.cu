@@ -50,6 +50,7 @@ extern "C" mxp_status mxp_gemm_noalloc(int64_t M, int64_t N, int64_t K, const mx
     if (d_dt != MXP_F32 && d_dt != MXP_BF16) return MXP_ERR_INVALID_ARG;
     if (A_packed == nullptr || B_packed == nullptr) return MXP_ERR_INVALID_ARG;
     for (const mxp_packed* p : {A_packed, B_packed}) {
+        if (p->mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;  // needs the prepacked path
         if (p->mode != MXP_MODE_MXFP4 && p->mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_INVALID_ARG;
         if (p->cols != K || p->nibbles == nullptr || p->scales == nullptr) return MXP_ERR_INVALID_ARG;
         if (reinterpret_cast<uintptr_t>(p->nibbles) % 16 != 0) return MXP_ERR_INVALID_ARG;

@@ -1250,6 +1250,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     if (fast != 0 && workspace_bytes >= fast && !forced_other)
         return launch_gemm_tc_stream(M, N, K, A, B, nullptr, D, d_dt, ldd, workspace, workspace_bytes,
                                      stream);
+    // the in-place kernels implement Eq. 4 for MXFP4+ only: an MX++ operand needs the prepacked path
+    if (A.mode == MXP_MODE_MXFP4_PP || B.mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
     if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
         return MXP_ERR_CUDA;
     bool use_pair = M > 128 && N > 128 && (ap || bp);

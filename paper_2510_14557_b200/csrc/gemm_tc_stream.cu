@@ -392,9 +392,20 @@ struct PrepackOperand {
     uint8_t* atoms;
     uint8_t* wide;            // nullptr: not widened
     int rows, nbk;
+    int pp;                   // MX++ operand: index bits 7:5 hold delta (Sec. 4.3)
     unsigned scale_ctas;      // ceil(rows/128) * ceil(nbk/128)
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
 };
+
+// MX++ (Sec. 4.3): the tensor core gets one scale per block, the NBMs' shared exponent lies
+// delta below the BM's.  The block is handed over with scale 2^(shared_exp - t),
+// t = min(delta, 5, scale byte - 1): the BM becomes (4 + m/2) * 2^t (at most 240, an E4M3
+// value), the NBMs E2M1 * 2^-(delta - t) (E4M3 values down to 2^-8): everything stays exact.
+__device__ __forceinline__ uint32_t mxpp_shift(uint32_t scale_byte, uint32_t delta)
+{
+    if (scale_byte == 0u || scale_byte == 255u) return 0u;
+    return min(min(delta, 5u), scale_byte - 1u);
+}
 
 __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigned id, uint32_t* tile)
 {
@@ -407,7 +418,19 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
         const int r = i >> 5, kg = i & 31;
         const int64_t row = (int64_t)rg * 128 + r;
         uint32_t v = 0;
-        if (kg < nkg && row < op.rows) v = src[row * kgroups + kg0 + kg];
+        if (kg < nkg && row < op.rows) {
+            v = src[row * kgroups + kg0 + kg];
+            if (op.pp) {
+                const uint32_t ix = reinterpret_cast<const uint32_t*>(op.bm_index)[row * kgroups + kg0 + kg];
+                uint32_t o = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const uint32_t sb = (v >> (8 * b)) & 255u;
+                    o |= (sb - mxpp_shift(sb, (ix >> (8 * b + 5)) & 7u)) << (8 * b);
+                }
+                v = o;
+            }
+        }
         tile[kg * 129 + (r & 31) * 4 + (r >> 5)] = v;  // rows of 129 words: no bank conflicts
     }
     __syncthreads();
@@ -419,9 +442,35 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
 // the codes' low three bits as selector.  Sign: a second lookup with the raw codes as selector
 // uses prmt's sign-replicate mode (selector bit 3): it returns 0xFF for a negative code and a
 // table byte whose bit 0 is clear for a positive one, so bit 0 of each byte is the sign.
-__device__ __forceinline__ uint32_t e2m1x4_to_e4m3x4(uint32_t x)
+// E4M3 byte of an E2M1 magnitude code (0, .5, 1, 1.5, 2, 3, 4, 6) times 2^-j, j = 0..7:
+// normal while the value is at least 2^-6, a multiple of 2^-9 below.
+constexpr uint32_t e4m3_of_code_shifted(int code, int j)
 {
-    const uint32_t mag = __byte_perm(0x3C383000u, 0x4C484440u, x & 0x7777u);
+    const int e = code >> 1, m = code & 1;
+    if (code == 0) return 0u;
+    // value = (e ? (2 + m) << (e - 1) : m) / 2 halves -> in units of 2^-9: times 2^(8 - j)
+    const int num = (e ? (2 + m) << (e - 1) : m);  // value * 2
+    const int units = j <= 8 ? num << (8 - j) : 0; // value * 2^-j in units of 2^-9
+    if (units < 8) return (uint32_t)units;          // subnormal
+    int ex = 0, u = units;
+    while (u >= 16) { u >>= 1; ++ex; }              // u in [8, 16): 1.mmm
+    return (uint32_t)(((ex + 1) << 3) | (u & 7));
+}
+constexpr uint32_t e4m3_lut_word(int j, int hi)
+{
+    return e4m3_of_code_shifted(4 * hi + 0, j) | (e4m3_of_code_shifted(4 * hi + 1, j) << 8) |
+           (e4m3_of_code_shifted(4 * hi + 2, j) << 16) | (e4m3_of_code_shifted(4 * hi + 3, j) << 24);
+}
+static_assert(e4m3_lut_word(0, 0) == 0x3C383000u && e4m3_lut_word(0, 1) == 0x4C484440u, "E4M3 table");
+__constant__ uint2 kE4m3Lut[8] = {
+    {e4m3_lut_word(0, 0), e4m3_lut_word(0, 1)}, {e4m3_lut_word(1, 0), e4m3_lut_word(1, 1)},
+    {e4m3_lut_word(2, 0), e4m3_lut_word(2, 1)}, {e4m3_lut_word(3, 0), e4m3_lut_word(3, 1)},
+    {e4m3_lut_word(4, 0), e4m3_lut_word(4, 1)}, {e4m3_lut_word(5, 0), e4m3_lut_word(5, 1)},
+    {e4m3_lut_word(6, 0), e4m3_lut_word(6, 1)}, {e4m3_lut_word(7, 0), e4m3_lut_word(7, 1)}};
+
+__device__ __forceinline__ uint32_t e2m1x4_to_e4m3x4(uint32_t x, uint2 lut = make_uint2(0x3C383000u, 0x4C484440u))
+{
+    const uint32_t mag = __byte_perm(lut.x, lut.y, x & 0x7777u);
     uint32_t neg;  // PTX prmt (not the intrinsic, which defines only three selector bits)
     asm("prmt.b32 %0, %1, %1, %2;" : "=r"(neg) : "r"(0x80808080u), "r"(x));
     return mag | ((neg << 7) & 0x80808080u);
@@ -434,23 +483,28 @@ __device__ __forceinline__ void widen_e4m3(const PrepackOperand& op, unsigned id
     if (b >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
     const uint2 w = reinterpret_cast<const uint2*>(op.nibbles)[t];
     const uint32_t sc = op.scales[b];
+    const uint32_t ib = op.bm_index != nullptr ? op.bm_index[b] : 0u;
+    // MX++: BM scaled up by 2^shift, NBMs down by 2^-(delta - shift) (see mxpp_shift)
+    const uint32_t delta = op.pp ? ib >> 5 : 0u;
+    const uint32_t shift = op.pp ? mxpp_shift(sc, delta) : 0u;
+    const uint2 lut = op.pp ? kE4m3Lut[delta - shift] : make_uint2(0x3C383000u, 0x4C484440u);
     uint4 o;
-    o.x = e2m1x4_to_e4m3x4(w.x);
-    o.y = e2m1x4_to_e4m3x4(w.x >> 16);
-    o.z = e2m1x4_to_e4m3x4(w.y);
-    o.w = e2m1x4_to_e4m3x4(w.y >> 16);
+    o.x = e2m1x4_to_e4m3x4(w.x, lut);
+    o.y = e2m1x4_to_e4m3x4(w.x >> 16, lut);
+    o.z = e2m1x4_to_e4m3x4(w.y, lut);
+    o.w = e2m1x4_to_e4m3x4(w.y >> 16, lut);
     if (sc == 0u) o = make_uint4(0u, 0u, 0u, 0u);
     uint8_t* dst = op.wide + (size_t)t * 16u;
     *reinterpret_cast<uint4*>(dst) = o;
     if (op.bm_index != nullptr) {
         // Eq. 3, BM branch.  Same thread, later store to the same bytes: lands after the
         // vector store above.
-        const uint32_t p = op.bm_index[b] & 31u;
+        const uint32_t p = ib & 31u;
         const uint32_t e = p & 15u;
         const uint32_t word = (e & 8u) ? w.y : w.x;
         const uint32_t nib = (word >> ((e & 7u) * 4u)) & 15u;
         if ((p >> 4) == (t & 1u) && sc != 0u)
-            dst[e] = (uint8_t)(((nib & 8u) << 4) | 0x48u | (nib & 7u));
+            dst[e] = (uint8_t)(((nib & 8u) << 4) | (0x48u + (shift << 3)) | (nib & 7u));
     }
 }
 
@@ -573,7 +627,7 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
     // the prepack kernel indexes half blocks (16 elements) of an operand with 32 bits
     if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
         return 0;
-    const bool wide = a_mode == MXP_MODE_MXFP4_PLUS || b_mode == MXP_MODE_MXFP4_PLUS;
+    const bool wide = a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4;
     return layout(M, N, K, wide).total;
 }
 
@@ -599,7 +653,8 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     PrepackOperand op;
     op.nibbles = P.nibbles;
     op.scales = P.scales;
-    op.bm_index = P.mode == MXP_MODE_MXFP4_PLUS ? P.bm_index : nullptr;
+    op.bm_index = P.mode != MXP_MODE_MXFP4 ? P.bm_index : nullptr;
+    op.pp = P.mode == MXP_MODE_MXFP4_PP;
     op.atoms = atoms;
     op.wide = wide ? wide_bytes : nullptr;
     op.rows = (int)rows;
@@ -629,7 +684,8 @@ mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_
     if (need == 0) return MXP_ERR_UNSUPPORTED;
     if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
-        (reinterpret_cast<uintptr_t>(P.scales) & 3))
+        (reinterpret_cast<uintptr_t>(P.scales) & 3) ||
+        (P.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(P.bm_index) & 3)))
         return MXP_ERR_INVALID_ARG;
     const PackedLayout l = packed_layout(P.rows, P.cols, wide);
     uint8_t* o = static_cast<uint8_t*>(out);
@@ -647,7 +703,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
                                  mxp_dtype d_dt, int64_t ldd, void* workspace,
                                  size_t workspace_bytes, cudaStream_t stream)
 {
-    const bool ap = A.mode == MXP_MODE_MXFP4_PLUS, bp = B.mode == MXP_MODE_MXFP4_PLUS;
+    const bool ap = A.mode != MXP_MODE_MXFP4, bp = B.mode != MXP_MODE_MXFP4;
     const bool wide = ap || bp;
     const Layout l = layout(M, b_prepacked ? 0 : N, K, wide);
     if (workspace == nullptr || workspace_bytes < l.total) return MXP_ERR_WORKSPACE;
@@ -665,6 +721,10 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     // the widening threads index their operand with 32 bits
     if ((uint64_t)M * nbk * 2 >= (1ull << 32) || (uint64_t)N * nbk * 2 >= (1ull << 32))
         return MXP_ERR_UNSUPPORTED;
+    // MX++: the scale re-tiling reads the index plane a word at a time
+    if ((A.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(A.bm_index) & 3)) ||
+        (B.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(B.bm_index) & 3)))
+        return MXP_ERR_INVALID_ARG;
 
     const PackedLayout lb = packed_layout(N, K, wide);
     const uint8_t* b_atoms = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms : ws + l.sfb;

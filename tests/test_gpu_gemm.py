@@ -19,7 +19,7 @@ def mxp():
 def quantized(x_bits_or_f32, mode, bf16=False):
     q = oracle.quantize(x_bits_or_f32, mode, bf16_bits=bf16)
     dec = oracle.dequantize(q[0], q[1], q[2], mode)
-    return host_to_packed(q[0], q[1], q[2] if mode == MXP else None, mode), dec
+    return host_to_packed(q[0], q[1], q[2] if mode != MX else None, mode), dec
 
 
 # ------------------------------------------------------------------ weight-only form
@@ -199,12 +199,19 @@ def test_tc_both_kernels_every_mode(kernel, amode, bmode, monkeypatch):
 
 
 # ------------------------------------------------------------------ streamed kernel, prepack
+MXPP = 2   # MX++ (Sec. 4.3): delta in the index byte's top three bits
+
+
 def _raw_operand(rows, K, mode, seed, scale_lo=120, scale_hi=134):
-    """Packed planes filled directly: every code, BM position and mantissa occurs."""
+    """Packed planes filled directly: every code, BM position, mantissa (and delta) occurs."""
     g = synth.rng(seed)
     nib = g.integers(0, 256, (rows, K // 2), dtype=np.uint8)
     sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
-    idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8) if mode == MXP else None
+    idx = None
+    if mode == MXP:
+        idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8)
+    if mode == MXPP:
+        idx = g.integers(0, 256, (rows, K // 32), dtype=np.uint8)
     dec = oracle.dequantize(nib, sc, idx, mode)
     return host_to_packed(nib, sc, idx, mode), dec
 
@@ -272,3 +279,66 @@ def test_tc_stream_flushed_blocks_and_bm_coincidence():
     d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
     ref = oracle.gemm_fp64(da, db)
     assert np.array_equal(d.cpu().numpy().astype(np.float64), ref)
+
+
+# ------------------------------------------------------------------ MX++ operands (Sec. 4.3)
+PP_MODES = [(MXPP, MX), (MX, MXPP), (MXPP, MXP), (MXP, MXPP), (MXPP, MXPP)]
+
+
+@pytest.mark.parametrize("amode,bmode", PP_MODES)
+def test_tc_mxpp_every_code_position_mantissa_and_delta(amode, bmode):
+    # identity on one side: D must equal the oracle's decode of the other operand bit for bit,
+    # for random raw planes (every code, BM position, BM mantissa and delta 0..7)
+    K = 256
+    eye = np.eye(K, dtype=np.float32)
+    if amode == MXPP:
+        ap, da = _raw_operand(384, K, amode, seed=31)
+        bp, db = quantized(eye, bmode)
+        d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+        assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
+    if bmode == MXPP:
+        ap, da = quantized(eye, amode)
+        bp, db = _raw_operand(384, K, bmode, seed=32)
+        d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+        assert np.array_equal(d.cpu().numpy().astype(np.float64), db.T)
+
+
+def test_tc_mxpp_tiny_scale_bytes():
+    # scale bytes 1..8 with every delta: the shift handed to the tensor core is limited by the
+    # scale byte, the NBMs go down to E4M3 subnormals
+    K = 256
+    ap, da = _raw_operand(256, K, MXPP, seed=41, scale_lo=1, scale_hi=9)
+    bp, db = quantized(np.eye(K, dtype=np.float32) * np.float32(2.0 ** 100), MXP)
+    d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+    want = (da * 2.0 ** 100).astype(np.float32).astype(np.float64)
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("amode,bmode", PP_MODES)
+def test_tc_mxpp_quantized_operands_and_prepack(amode, bmode):
+    M, N, K = 300, 520, 1024
+    a = synth.activations_normal(M, K, seed=3, outlier_frac=0.02)
+    b = synth.weights(N, K, seed=4).astype(np.float32)
+    ap, da = quantized(a, amode)
+    bp, db = quantized(b, bmode)
+    m = mxp()
+    pre = m.mxp_gemm_prepack(bp, True)
+    for dt in (torch.float32, torch.bfloat16):
+        d0 = m.mxp_gemm(ap, bp, out_dtype=dt)
+        check_gemm(d0, da, db)
+        assert torch.equal(d0, m.mxp_gemm_prepacked(ap, bp, pre, out_dtype=dt))
+
+
+def test_mxpp_without_the_prepacked_path_is_reported():
+    from paper_2510_14557_b200 import MxpError
+    m = mxp()
+    ap, _ = _raw_operand(64, 256, MXPP, seed=1)      # M <= 128: only in-place kernels apply
+    bp, _ = _raw_operand(256, 256, MXP, seed=2)
+    with pytest.raises(MxpError) as e:
+        m.mxp_gemm(ap, bp)
+    assert e.value.status == 2                        # MXP_ERR_UNSUPPORTED
+    a = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
+    wp, _ = _raw_operand(256, 256, MXPP, seed=3)
+    with pytest.raises(MxpError) as e:
+        m.mxp_gemm(a, wp)                              # weight-only form: not built for MX++
+    assert e.value.status == 2
