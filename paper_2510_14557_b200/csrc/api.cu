@@ -111,8 +111,6 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     if (K == 0) return MXP_ERR_UNSUPPORTED;  // an empty sum; callers zero D themselves
-    // MX++ weights with bf16 activations: not built yet
-    if (A_packed == nullptr && B_packed->mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
     const size_t need = mxp_gemm_min_workspace_bytes(M, N, K, A_dense_bf16 != nullptr,
                                                      A_packed ? A_packed->mode : MXP_MODE_MXFP4,
                                                      B_packed->mode);

@@ -44,10 +44,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 // Decode one block (four words of nibbles) into 16 bf16x2 registers.  Register 4w + i holds
 // elements (8w + i, 8w + i + 4): the two nibbles sit 16 bits apart, so one shift and mask
 // places both codes.
-template <bool kPlus>
+// kMode: 0 MXFP4, 1 MXFP4+, 2 MX++ (Sec. 4.3: bits 7:5 of the index byte `bm` hold delta; the
+// NBMs' shared exponent lies delta below the block's, so the BM is entered 2^delta larger).
+template <int kMode>
 __device__ __forceinline__ void decode_block(const uint4 nib, uint32_t sb, uint32_t bm,
                                              uint32_t (&out)[16])
 {
+    constexpr bool kPlus = kMode >= 1;
+    const uint32_t delta = kMode == 2 ? (bm >> 5) : 0u;
     const uint32_t w[4] = {nib.x, nib.y, nib.z, nib.w};
     // Left shifts are written as multiplies so that they issue on the FMA pipe (IMAD) and
     // leave the integer ALU pipe, which this kernel saturates first, to the mask / merge ops.
@@ -64,7 +68,8 @@ __device__ __forceinline__ void decode_block(const uint4 nib, uint32_t sb, uint3
         const uint32_t p = bm & 31u;
         const uint32_t word = (p & 16u) ? ((p & 8u) ? w[3] : w[2]) : ((p & 8u) ? w[1] : w[0]);
         const uint32_t n = (word >> ((p & 7u) * 4u)) & 15u;
-        const uint32_t pat = 0x180u | ((n & 7u) << 4) | ((n & 8u) << 12);  // (4 + m/2) * 2^-126
+        const uint32_t pat =
+            (0x180u + (delta << 7)) | ((n & 7u) << 4) | ((n & 8u) << 12);  // (4 + m/2) * 2^(delta - 126)
         const uint32_t reg = ((p >> 3) << 2) | (p & 3u);
         const bool upper = (p & 4u) != 0u;
         const uint32_t keep = upper ? 0x0000FFFFu : 0xFFFF0000u;
@@ -75,14 +80,16 @@ __device__ __forceinline__ void decode_block(const uint4 nib, uint32_t sb, uint3
     }
     // multiplier 2^(126 + shared_exp) = 2^(sb - 1): bf16 exponent field 126 + sb.  It tops
     // out at 254; the remainder goes into a second multiply (only for blocks with |x| >= 16).
-    const uint32_t e1 = min(126u + sb, 254u);
+    // (MX++: 126 + sb - delta; below 1 only for blocks at the very bottom of the range)
+    const int total = 126 + (int)sb - (int)delta;
+    const uint32_t e1 = (uint32_t)min(max(total, 1), 254);
     uint32_t m1 = (e1 << 7) * 0x00010001u;
     if (sb == 0u) m1 = 0u;                 // reserved scale: the whole block is zero
     if (sb == 255u) m1 = 0x7FC07FC0u;      // non-finite marker decodes to NaN
 #pragma unroll
     for (int r = 0; r < 16; ++r) out[r] = hmul2_bf16(out[r], m1);
-    if (__any_sync(0xFFFFFFFFu, sb >= 129u && sb != 255u)) {
-        const uint32_t e2 = 127u + (126u + sb - e1);
+    if (__any_sync(0xFFFFFFFFu, total != (int)e1 && sb != 255u && sb != 0u)) {
+        const uint32_t e2 = (uint32_t)(127 + total - (int)e1);
         const uint32_t m2 = (sb == 255u ? 0x3F80u : (e2 << 7)) * 0x00010001u;
 #pragma unroll
         for (int r = 0; r < 16; ++r) out[r] = hmul2_bf16(out[r], m2);
@@ -97,12 +104,13 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 }
 
 // kMT: number of 8-column activation tiles (M <= 8 * kMT handled per CTA pass).
-template <int kMT, bool kPlus, typename OutT>
+template <int kMT, int kMode, typename OutT>
 __global__ void __launch_bounds__(kThreads)
 gemm_wo_kernel(int M, int N, int K, const __nv_bfloat16* __restrict__ A, int64_t lda,
                const uint8_t* __restrict__ nibbles, const uint8_t* __restrict__ scales,
                const uint8_t* __restrict__ bm_index, OutT* __restrict__ D, int64_t ldd)
 {
+    constexpr bool kPlus = kMode >= 1;
     __shared__ float red[kWarps][kRowsPerCta][8 * kMT + 1];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -176,8 +184,8 @@ gemm_wo_kernel(int M, int N, int K, const __nv_bfloat16* __restrict__ A, int64_t
             }
         }
         uint32_t pa[16], pb[16];
-        decode_block<kPlus>(cwa, csa, cia, pa);
-        decode_block<kPlus>(cwb, csb, cib, pb);
+        decode_block<kMode>(cwa, csa, cia, pa);
+        decode_block<kMode>(cwb, csb, cib, pb);
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
 #pragma unroll
@@ -211,25 +219,25 @@ gemm_wo_kernel(int M, int N, int K, const __nv_bfloat16* __restrict__ A, int64_t
     }
 }
 
-template <int kMT, bool kPlus, typename OutT>
+template <int kMT, int kMode, typename OutT>
 void launch(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const mxp_packed& B,
             void* D, int64_t ldd, cudaStream_t stream)
 {
     dim3 grid((unsigned)((N + kRowsPerCta - 1) / kRowsPerCta),
               (unsigned)((M + 8 * kMT - 1) / (8 * kMT)));
-    gemm_wo_kernel<kMT, kPlus, OutT><<<grid, kThreads, 0, stream>>>(
+    gemm_wo_kernel<kMT, kMode, OutT><<<grid, kThreads, 0, stream>>>(
         (int)M, (int)N, (int)K, static_cast<const __nv_bfloat16*>(A), lda, B.nibbles, B.scales,
         B.bm_index, static_cast<OutT*>(D), ldd);
 }
 
-template <bool kPlus, typename OutT>
+template <int kMode, typename OutT>
 void launch_mt(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const mxp_packed& B,
                void* D, int64_t ldd, cudaStream_t stream)
 {
     if (M <= 8)
-        launch<1, kPlus, OutT>(M, N, K, A, lda, B, D, ldd, stream);
+        launch<1, kMode, OutT>(M, N, K, A, lda, B, D, ldd, stream);
     else
-        launch<2, kPlus, OutT>(M, N, K, A, lda, B, D, ldd, stream);
+        launch<2, kMode, OutT>(M, N, K, A, lda, B, D, ldd, stream);
 }
 
 }  // namespace
@@ -255,13 +263,14 @@ cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void*
         return launch_gemm_wo_stream(M, N, K, A, lda, B, D, d_dt, ldd, status, stream);
     }
     if ((M + 15) / 16 > 65535) return cudaErrorNotSupported;
-    const bool plus = B.mode == MXP_MODE_MXFP4_PLUS;
     if (d_dt == MXP_F32) {
-        if (plus) launch_mt<true, float>(M, N, K, A, lda, B, D, ldd, stream);
-        else launch_mt<false, float>(M, N, K, A, lda, B, D, ldd, stream);
+        if (B.mode == MXP_MODE_MXFP4_PP) launch_mt<2, float>(M, N, K, A, lda, B, D, ldd, stream);
+        else if (B.mode == MXP_MODE_MXFP4_PLUS) launch_mt<1, float>(M, N, K, A, lda, B, D, ldd, stream);
+        else launch_mt<0, float>(M, N, K, A, lda, B, D, ldd, stream);
     } else {
-        if (plus) launch_mt<true, __nv_bfloat16>(M, N, K, A, lda, B, D, ldd, stream);
-        else launch_mt<false, __nv_bfloat16>(M, N, K, A, lda, B, D, ldd, stream);
+        if (B.mode == MXP_MODE_MXFP4_PP) launch_mt<2, __nv_bfloat16>(M, N, K, A, lda, B, D, ldd, stream);
+        else if (B.mode == MXP_MODE_MXFP4_PLUS) launch_mt<1, __nv_bfloat16>(M, N, K, A, lda, B, D, ldd, stream);
+        else launch_mt<0, __nv_bfloat16>(M, N, K, A, lda, B, D, ldd, stream);
     }
     return cudaGetLastError();
 }

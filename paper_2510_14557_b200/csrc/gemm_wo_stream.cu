@@ -149,11 +149,17 @@ __device__ __forceinline__ void cvt_e2m1x8(uint32_t w, uint32_t (&h)[4])
 // lane's four f16x2 registers, which bits to keep (all of them unless the lane's word holds
 // element p).  The f16 pattern of the BM is built from the lane's own word; where the lane
 // does not hold the BM the pattern is garbage and fully masked.
-__device__ __forceinline__ void patch_bm(uint32_t w, uint32_t p, uint32_t lut_t, uint32_t (&h)[4])
+// `ib` is the block's index byte: position in bits 4:0; in MX++ mode (kPP) bits 7:5 hold
+// delta, and the BM, which keeps the block's own shared exponent, is entered 2^delta larger
+// than the NBMs it sits among (at most 7.5 * 128, an f16 value).
+template <bool kPP>
+__device__ __forceinline__ void patch_bm(uint32_t w, uint32_t ib, uint32_t lut_t, uint32_t (&h)[4])
 {
+    const uint32_t p = ib & 31u;
     const uint4 keep = lds128(lut_t + p * 64u);
     const uint32_t x = w >> ((p & 7u) * 4u);
     uint32_t pat = ((x << 7) & 0x0380u) | 0x4400u;  // 4 + m/2
+    if (kPP) pat += (ib >> 5) << 10;                 // times 2^delta
     pat |= (x << 12) & 0x8000u;                      // sign
     pat *= 0x00010001u;                              // both halves; the mask picks one
     h[0] = (h[0] & keep.x) | (pat & ~keep.x);
@@ -229,9 +235,11 @@ __device__ __forceinline__ void normalise_block(const uint4 (&x)[4], int mulfiel
     } while (0)
 #endif
 
-template <int kMT, bool kPlus, typename OutT>
+template <int kMT, int kMode, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoParams prm)
 {
+    constexpr bool kPlus = kMode >= 1;  // 1: MXFP4+, 2: MX++ (Sec. 4.3)
+    constexpr bool kPP = kMode == 2;
     constexpr int kMp = 8 * kMT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) &
@@ -427,13 +435,20 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                         cvt_e2m1x8(wA, hA);
                         cvt_e2m1x8(wB, hB);
                         const int sh = 8 * (j & 3);
+                        const uint32_t ibA = ((j < 4 ? ixA.x : ixA.y) >> sh) & 255u;
+                        const uint32_t ibB = ((j < 4 ? ixB.x : ixB.y) >> sh) & 255u;
                         if (kPlus) {
-                            patch_bm(wA, ((j < 4 ? ixA.x : ixA.y) >> sh) & 31u, lut_t, hA);
-                            patch_bm(wB, ((j < 4 ? ixB.x : ixB.y) >> sh) & 31u, lut_t, hB);
+                            patch_bm<kPP>(wA, ibA, lut_t, hA);
+                            patch_bm<kPP>(wB, ibB, lut_t, hB);
                         }
-                        // 2^(scale byte - 127) as a float: a zero byte (flushed block) gives 0
-                        const float sA = __uint_as_float((((j < 4 ? scA.x : scA.y) >> sh) & 255u) << 23);
-                        const float sB = __uint_as_float((((j < 4 ? scB.x : scB.y) >> sh) & 255u) << 23);
+                        // 2^(scale byte - 127) as a float: a zero byte (flushed block) gives 0;
+                        // MX++: the NBMs' exponent lies delta below (exact, subnormals included)
+                        float sA = __uint_as_float((((j < 4 ? scA.x : scA.y) >> sh) & 255u) << 23);
+                        float sB = __uint_as_float((((j < 4 ? scB.x : scB.y) >> sh) & 255u) << 23);
+                        if (kPP) {
+                            sA *= __uint_as_float((127u - (ibA >> 5)) << 23);
+                            sB *= __uint_as_float((127u - (ibB >> 5)) << 23);
+                        }
 #pragma unroll
                         for (int mt = 0; mt < kMT; ++mt) {
                             const uint4 b = lds128(ap + (uint32_t)((j * kMp + 8 * mt) * 64));
@@ -552,14 +567,15 @@ inline bool wo_plan(int K, int mp, bool plus, int* stages, int* red_buffers, int
     return false;
 }
 
-template <int kMT, bool kPlus, typename OutT>
+template <int kMT, int kMode, typename OutT>
 cudaError_t launch(WoParams prm, int num_sms, cudaStream_t stream)
 {
+    constexpr bool kPlus = kMode >= 1;
     if (!wo_plan(prm.K, 8 * kMT, kPlus, &prm.stages, &prm.red_buffers, &prm.meta_bufs))
         return cudaErrorNotSupported;
     const size_t smem = wo_layout(prm.K, 8 * kMT, kPlus, prm.red_buffers, prm.meta_bufs).fixed +
                         (size_t)prm.stages * kStageBytes;
-    auto kern = gemm_wo_stream_kernel<kMT, kPlus, OutT>;
+    auto kern = gemm_wo_stream_kernel<kMT, kMode, OutT>;
     static size_t attr_smem = 0;  // raised as needed, once per size: the call is not free
     if (smem > attr_smem) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -588,7 +604,7 @@ bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t
          reinterpret_cast<uintptr_t>(B.scales)) & 15)
         return false;
     if (lda % 8 != 0) return false;
-    const bool plus = B.mode == MXP_MODE_MXFP4_PLUS;
+    const bool plus = B.mode != MXP_MODE_MXFP4;
     if (plus && (reinterpret_cast<uintptr_t>(B.bm_index) & 15)) return false;
     int st, rb, mb;
     return wo_plan((int)K, M <= 8 ? 8 : 16, plus, &st, &rb, &mb);
@@ -613,15 +629,25 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
     prm.stages = prm.red_buffers = prm.meta_bufs = 0;
     const int sms = sm_count();
     if (sms <= 0) return cudaErrorUnknown;
-    const bool plus = B.mode == MXP_MODE_MXFP4_PLUS;
     const bool f32 = d_dt == MXP_F32;
-    if (M <= 8) {
-        if (plus) return f32 ? launch<1, true, float>(prm, sms, stream) : launch<1, true, __nv_bfloat16>(prm, sms, stream);
-        return f32 ? launch<1, false, float>(prm, sms, stream) : launch<1, false, __nv_bfloat16>(prm, sms, stream);
+    const int mode = (int)B.mode;
+#define MXP_WO_LAUNCH(MT)                                                                  \
+    switch (mode) {                                                                        \
+        case 2:                                                                            \
+            return f32 ? launch<MT, 2, float>(prm, sms, stream)                            \
+                       : launch<MT, 2, __nv_bfloat16>(prm, sms, stream);                   \
+        case 1:                                                                            \
+            return f32 ? launch<MT, 1, float>(prm, sms, stream)                            \
+                       : launch<MT, 1, __nv_bfloat16>(prm, sms, stream);                   \
+        default:                                                                           \
+            return f32 ? launch<MT, 0, float>(prm, sms, stream)                            \
+                       : launch<MT, 0, __nv_bfloat16>(prm, sms, stream);                   \
     }
-    if (plus) return f32 ? launch<2, true, float>(prm, sms, stream) : launch<2, true, __nv_bfloat16>(prm, sms, stream);
-    return f32 ? launch<2, false, float>(prm, sms, stream) : launch<2, false, __nv_bfloat16>(prm, sms, stream);
+    if (M <= 8) {
+        MXP_WO_LAUNCH(1)
+    }
+    MXP_WO_LAUNCH(2)
+#undef MXP_WO_LAUNCH
 }
-
 
 }  // namespace mxp

@@ -70,7 +70,7 @@ def test_weight_only_config3_sampled(M):
 
 
 @pytest.mark.parametrize("kernel", ["old", "stream"])
-@pytest.mark.parametrize("wmode", [MX, MXP])
+@pytest.mark.parametrize("wmode", [MX, MXP, 2])
 @pytest.mark.parametrize("M,N,K", [(1, 32, 256), (3, 48, 2304), (8, 160, 4352), (9, 64, 512),
                                    (16, 2384, 4096), (40, 64, 768)])
 def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
@@ -337,8 +337,21 @@ def test_mxpp_without_the_prepacked_path_is_reported():
     with pytest.raises(MxpError) as e:
         m.mxp_gemm(ap, bp)
     assert e.value.status == 2                        # MXP_ERR_UNSUPPORTED
-    a = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
-    wp, _ = _raw_operand(256, 256, MXPP, seed=3)
-    with pytest.raises(MxpError) as e:
-        m.mxp_gemm(a, wp)                              # weight-only form: not built for MX++
-    assert e.value.status == 2
+
+
+@pytest.mark.parametrize("kernel", ["old", "stream"])
+def test_weight_only_mxpp_raw_planes_one_hot(kernel, monkeypatch):
+    # one-hot activations return single decoded weights exactly (fp32 output): random raw MX++
+    # planes, i.e. every code, BM position, BM mantissa and delta
+    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
+    K, N = 512, 64
+    wp, dw = _raw_operand(N, K, MXPP, seed=51, scale_lo=100, scale_hi=150)
+    a = np.zeros((16, K), np.float32)
+    cols = [(m * 37 + 5) % K for m in range(16)]
+    for m, c in enumerate(cols):
+        a[m, c] = 2.0 ** (m - 8)
+    d = mxp().mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), wp, out_dtype=torch.float32)
+    got = d.cpu().numpy().astype(np.float64)
+    for m, c in enumerate(cols):
+        want = (dw[:, c] * 2.0 ** (m - 8)).astype(np.float32).astype(np.float64)
+        assert np.array_equal(got[m], want)
