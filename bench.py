@@ -238,14 +238,15 @@ def part_decode(mxp, synth, peaks, iters):
     out = {}
     hbm = peaks["hbm_gbs"]
     # ---- config 3: weight-only decode GEMM; rotate over 8 weight copies (> L2) between launches
-    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
+    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4),
+                       ("mxfp4++", mxp.MODE_MXFP4_PP)):
         a16, w_bits = synth.config3(16)
         w = dev_bf16(w_bits)
         copies = []
         for _ in range(8):
             copies.append(mxp.mxp_quantize(w, mode))
-        wbytes = 11008 * 4096 * (0.5 + 1 / 32 + (1 / 32 if mode == mxp.MODE_MXFP4_PLUS else 0))
-        for M in (1, 8, 16):
+        wbytes = 11008 * 4096 * (0.5 + 1 / 32 + (1 / 32 if mode != mxp.MODE_MXFP4 else 0))
+        for M in ((1, 8, 16) if mode != mxp.MODE_MXFP4_PP else (1,)):
             a = dev_bf16(a16[:M].copy())
             d = torch.empty((M, 11008), dtype=torch.bfloat16, device="cuda")
             state = {"i": 0}
@@ -294,6 +295,24 @@ def part_prefill(mxp, synth, peaks, iters):
                     "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
                     "frac_fp4_nominal_9PF": tf / 9000.0}
                 del pa, pw
+        if cfg == "cfg5":   # MX++ on both sides: same kernel, delta handled by the prepack
+            pa, pw = mxp.mxp_quantize(a, mxp.MODE_MXFP4_PP), mxp.mxp_quantize(w, mxp.MODE_MXFP4_PP)
+            tot = 0.0
+            for i in range(n_it + 2):
+                flush.fill_(i & 255)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                mxp.mxp_gemm(pa, pw, out=d, workspace=ws)
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 2:
+                    tot += e0.elapsed_time(e1)
+            ms = tot / n_it
+            tf = 2.0 * M * N * K / ms / 1e9
+            out["prefill_cfg5_A-mxfp4++_W-mxfp4++"] = {
+                "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
+                "frac_fp4_nominal_9PF": tf / 9000.0}
+            del pa, pw
         del a, w, d, ws
         torch.cuda.empty_cache()
     return out
