@@ -78,7 +78,10 @@ struct SCfg {
     static constexpr int kSfA = kGroups * kAtom;            // own 128 rows of A
     static constexpr int kSfB = 2 * kGroups * kAtom;        // all 256 rows of B
     static constexpr int kStage = 2 * kHalfTile + kSfA + kSfB;
-    static constexpr int kStages = 6;
+#ifndef MXP_S_STAGES
+#define MXP_S_STAGES 6
+#endif
+    static constexpr int kStages = MXP_S_STAGES;
     static constexpr int kSmem = kStages * kStage + 1024 /*barriers*/ + 1024 /*align*/;
     static constexpr int kElemsPerStage = kWide ? 128 : 256;
 };
@@ -102,8 +105,12 @@ __device__ __forceinline__ void give_up(volatile uint32_t* abort, StatusBlock* s
 
 // Tile order: bands of kBand tile rows, walked column by column, so that the tiles in flight
 // at any time (one per CTA pair) cover a compact block of the output and their A and B
-// panels stay resident in L2 instead of being re-streamed from HBM every wave.
-constexpr int kBand = 8;
+// panels stay resident in L2 instead of being re-streamed from HBM every wave.  (16 measured
+// best on the 8192 x 28672 x 8192 prefill shape; 8 and 4 are within 3 %.)
+#ifndef MXP_S_BAND
+#define MXP_S_BAND 16
+#endif
+constexpr int kBand = MXP_S_BAND;
 __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn)
 {
     const int per_band = kBand * tiles_n;
@@ -527,6 +534,9 @@ __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, co
     widen_e4m3(b, id);
 }
 
+#ifndef MXP_S_L2PROMO
+#define MXP_S_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
 // 2-D byte tensor [rows][row_bytes], boxes of 128 bytes x 128 rows, 128B swizzle.
 bool make_tmap_rows(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t row_bytes)
 {
@@ -538,7 +548,7 @@ bool make_tmap_rows(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t r
     const cuuint32_t estr[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              MXP_S_L2PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Scale atoms as a 3-D tensor of 32-bit words [row groups][K groups][128], boxes of
