@@ -257,6 +257,23 @@ def part_decode(mxp, synth, peaks, iters):
             ms = time_loop(run, iters, warmup=8)
             gbs = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms / 1e6
             out["decode_cfg3_M%d_%s" % (M, name)] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
+            if True:
+                # the same eight launches replayed from a CUDA graph: what a decode loop that
+                # captures its layers sees (less launch gap between the kernels)
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    for _ in range(8):
+                        run()
+                torch.cuda.current_stream().wait_stream(side)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    for _ in range(8):
+                        run()
+                ms_g = time_loop(graph.replay, max(1, iters // 8), warmup=2) / 8
+                out["decode_cfg3_M%d_%s" % (M, name)]["us_cuda_graph"] = ms_g * 1e3
+                out["decode_cfg3_M%d_%s" % (M, name)]["frac_hbm_cuda_graph"] = \
+                    (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_g / 1e6 / hbm
         del copies, w
     return out
 
