@@ -27,6 +27,7 @@
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
+#include "e4m3_widen.cuh"
 
 namespace mxp {
 
@@ -404,16 +405,6 @@ struct PrepackOperand {
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
 };
 
-// MX++ (Sec. 4.3): the tensor core gets one scale per block, the NBMs' shared exponent lies
-// delta below the BM's.  The block is handed over with scale 2^(shared_exp - t),
-// t = min(delta, 5, scale byte - 1): the BM becomes (4 + m/2) * 2^t (at most 240, an E4M3
-// value), the NBMs E2M1 * 2^-(delta - t) (E4M3 values down to 2^-8): everything stays exact.
-__device__ __forceinline__ uint32_t mxpp_shift(uint32_t scale_byte, uint32_t delta)
-{
-    if (scale_byte == 0u || scale_byte == 255u) return 0u;
-    return min(min(delta, 5u), scale_byte - 1u);
-}
-
 __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigned id, uint32_t* tile)
 {
     const int kgroups = op.nbk >> 2;
@@ -443,44 +434,6 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
     __syncthreads();
     uint32_t* dst = reinterpret_cast<uint32_t*>(op.atoms) + ((int64_t)rg * kgroups + kg0) * 128;
     for (int i = threadIdx.x; i < nkg * 128; i += 256) dst[i] = tile[(i >> 7) * 129 + (i & 127)];
-}
-
-// Four E2M1 codes (low 16 bits of x) -> four E4M3 bytes.  Magnitude: byte table lookup with
-// the codes' low three bits as selector.  Sign: a second lookup with the raw codes as selector
-// uses prmt's sign-replicate mode (selector bit 3): it returns 0xFF for a negative code and a
-// table byte whose bit 0 is clear for a positive one, so bit 0 of each byte is the sign.
-// E4M3 byte of an E2M1 magnitude code (0, .5, 1, 1.5, 2, 3, 4, 6) times 2^-j, j = 0..7:
-// normal while the value is at least 2^-6, a multiple of 2^-9 below.
-constexpr uint32_t e4m3_of_code_shifted(int code, int j)
-{
-    const int e = code >> 1, m = code & 1;
-    if (code == 0) return 0u;
-    // value = (e ? (2 + m) << (e - 1) : m) / 2 halves -> in units of 2^-9: times 2^(8 - j)
-    const int num = (e ? (2 + m) << (e - 1) : m);  // value * 2
-    const int units = j <= 8 ? num << (8 - j) : 0; // value * 2^-j in units of 2^-9
-    if (units < 8) return (uint32_t)units;          // subnormal
-    int ex = 0, u = units;
-    while (u >= 16) { u >>= 1; ++ex; }              // u in [8, 16): 1.mmm
-    return (uint32_t)(((ex + 1) << 3) | (u & 7));
-}
-constexpr uint32_t e4m3_lut_word(int j, int hi)
-{
-    return e4m3_of_code_shifted(4 * hi + 0, j) | (e4m3_of_code_shifted(4 * hi + 1, j) << 8) |
-           (e4m3_of_code_shifted(4 * hi + 2, j) << 16) | (e4m3_of_code_shifted(4 * hi + 3, j) << 24);
-}
-static_assert(e4m3_lut_word(0, 0) == 0x3C383000u && e4m3_lut_word(0, 1) == 0x4C484440u, "E4M3 table");
-__constant__ uint2 kE4m3Lut[8] = {
-    {e4m3_lut_word(0, 0), e4m3_lut_word(0, 1)}, {e4m3_lut_word(1, 0), e4m3_lut_word(1, 1)},
-    {e4m3_lut_word(2, 0), e4m3_lut_word(2, 1)}, {e4m3_lut_word(3, 0), e4m3_lut_word(3, 1)},
-    {e4m3_lut_word(4, 0), e4m3_lut_word(4, 1)}, {e4m3_lut_word(5, 0), e4m3_lut_word(5, 1)},
-    {e4m3_lut_word(6, 0), e4m3_lut_word(6, 1)}, {e4m3_lut_word(7, 0), e4m3_lut_word(7, 1)}};
-
-__device__ __forceinline__ uint32_t e2m1x4_to_e4m3x4(uint32_t x, uint2 lut = make_uint2(0x3C383000u, 0x4C484440u))
-{
-    const uint32_t mag = __byte_perm(lut.x, lut.y, x & 0x7777u);
-    uint32_t neg;  // PTX prmt (not the intrinsic, which defines only three selector bits)
-    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(neg) : "r"(0x80808080u), "r"(x));
-    return mag | ((neg << 7) & 0x80808080u);
 }
 
 __device__ __forceinline__ void widen_e4m3(const PrepackOperand& op, unsigned id)
