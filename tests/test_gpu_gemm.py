@@ -72,7 +72,8 @@ def test_weight_only_config3_sampled(M):
 @pytest.mark.parametrize("kernel", ["old", "stream"])
 @pytest.mark.parametrize("wmode", [MX, MXP, 2])
 @pytest.mark.parametrize("M,N,K", [(1, 32, 256), (3, 48, 2304), (8, 160, 4352), (9, 64, 512),
-                                   (16, 2384, 4096), (40, 64, 768)])
+                                   (16, 2384, 4096), (40, 64, 768), (5, 77, 1024), (16, 300, 512),
+                                   (1, 19000, 512)])
 def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
     # shapes the streamed kernel takes (N % 16 == 0, K % 256 == 0): several 2048-element stages,
     # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles
