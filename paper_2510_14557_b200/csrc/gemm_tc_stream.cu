@@ -586,7 +586,11 @@ mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUt
 
 size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
 {
-    if (M <= 128 || N <= 128 || K % 128 != 0) return 0;
+    // Small M or N is better served by the in-place single-CTA kernel, except for MX++
+    // operands, which only this path handles (rows past the end are zero-filled by TMA).
+    const bool pp = a_mode == MXP_MODE_MXFP4_PP || b_mode == MXP_MODE_MXFP4_PP;
+    if (M < 1 || N < 1 || K % 128 != 0) return 0;
+    if (!pp && (M <= 128 || N <= 128)) return 0;
     // the prepack kernel indexes half blocks (16 elements) of an operand with 32 bits
     if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
         return 0;

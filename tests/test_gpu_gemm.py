@@ -333,11 +333,21 @@ def test_tc_mxpp_quantized_operands_and_prepack(amode, bmode):
 def test_mxpp_without_the_prepacked_path_is_reported():
     from paper_2510_14557_b200 import MxpError
     m = mxp()
-    ap, _ = _raw_operand(64, 256, MXPP, seed=1)      # M <= 128: only in-place kernels apply
+    ap, _ = _raw_operand(64, 256, MXPP, seed=1)
     bp, _ = _raw_operand(256, 256, MXP, seed=2)
-    with pytest.raises(MxpError) as e:
-        m.mxp_gemm(ap, bp)
+    small = torch.zeros(4096, dtype=torch.uint8, device="cuda")   # minimum workspace only:
+    with pytest.raises(MxpError) as e:                            # the in-place kernels
+        m.mxp_gemm(ap, bp, workspace=small)
     assert e.value.status == 2                        # MXP_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 128), (64, 256, 256), (129, 7, 384), (100, 72, 1024)])
+def test_tc_mxpp_small_shapes(M, N, K):
+    # MX++ with M or N <= 128 goes through the streamed kernel too (TMA zero-fills the rest)
+    ap, da = _raw_operand(M, K, MXPP, seed=M + 7)
+    bp, db = _raw_operand(N, K, MXPP, seed=N + 9)
+    for dt in (torch.float32, torch.bfloat16):
+        check_gemm(mxp().mxp_gemm(ap, bp, out_dtype=dt), da, db)
 
 
 @pytest.mark.parametrize("kernel", ["old", "stream"])
