@@ -167,6 +167,16 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed 
 mxp_status mxp_gemm_status(const void *workspace, void *cuda_stream);
 
 /*
+ * Self-test of the bounded device-side waits (the paper has no counterpart: it is how this
+ * library's kernels report a wait that runs out instead of hanging).  Launches one warp
+ * that waits, for at most `limit_cycles` SM clock cycles (1 .. 2e9), on a barrier nothing
+ * signals.  Afterwards mxp_gemm_status(workspace, stream) must return MXP_ERR_TIMEOUT, and
+ * the device must be usable as before.  `workspace`: device, 16-byte aligned, >= 16 bytes.
+ */
+mxp_status mxp_wait_selftest(void *workspace, size_t workspace_bytes, int64_t limit_cycles,
+                             void *cuda_stream);
+
+/*
  * Issue-rate probe for the roofline denominator: runs `iters` back-to-back tensor-core
  * instructions per CTA on operands resident in shared memory (no global traffic) on
  * every SM and returns the elapsed milliseconds in *ms (synchronises the device).

@@ -26,7 +26,7 @@ LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
 EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
-           "mxp_gemm_status", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
+           "mxp_gemm_status", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
 class MxpError(RuntimeError):
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_prepacked.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
                                          vp, vp, ci, i64, vp, sz, vp]
         l.mxp_gemm_prepacked.restype = ci
+        l.mxp_wait_selftest.argtypes = [vp, sz, i64, vp]
+        l.mxp_wait_selftest.restype = ci
         l.mxp_gemm_status.argtypes = [vp, vp]
         l.mxp_gemm_status.restype = ci
         l.mxp_tensor_peak_probe.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_double),
@@ -238,6 +240,12 @@ def mxp_gemm_noalloc(a: Packed, b: Packed, out: torch.Tensor, read_status: bool 
                                 ctypes.byref(ks) if read_status else None, _stream())
     _check("mxp_gemm_noalloc", st)
     return ks.value if read_status else None
+
+
+def mxp_wait_selftest(workspace: torch.Tensor, limit_cycles: int) -> None:
+    """Launches the bounded-wait self-test; read the outcome with mxp_gemm_status(workspace)."""
+    _check("mxp_wait_selftest", lib().mxp_wait_selftest(workspace.data_ptr(), workspace.numel(),
+                                                        int(limit_cycles), _stream()))
 
 
 def mxp_gemm_status(workspace: torch.Tensor) -> int:

@@ -165,6 +165,15 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
                                       static_cast<cudaStream_t>(cuda_stream));
 }
 
+mxp_status mxp_wait_selftest(void* workspace, size_t workspace_bytes, int64_t limit_cycles,
+                             void* cuda_stream)
+{
+    if (workspace == nullptr || workspace_bytes < sizeof(mxp::StatusBlock) || !aligned(workspace, 16))
+        return MXP_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > 2000000000ll) return MXP_ERR_INVALID_ARG;  // <= ~1 s
+    return mxp::launch_wait_selftest(workspace, limit_cycles, static_cast<cudaStream_t>(cuda_stream));
+}
+
 mxp_status mxp_gemm_status(const void* workspace, void* cuda_stream)
 {
     if (workspace == nullptr) return MXP_ERR_INVALID_ARG;

@@ -61,6 +61,27 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
 EncodeFn tensormap_encode_fn();
 int sm_count();  // of the current device, cached; -1 on error
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to
+// the device's context, and the call is not free).  `done` is the caller's per-kernel record.
+struct SmemAttrOnce {
+    bool done[64] = {};
+};
+template <typename Kernel>
+cudaError_t ensure_dynamic_smem(Kernel kern, int bytes, SmemAttrOnce& once)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && once.done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) once.done[dev] = true;
+    return e;
+}
+
+// Launches the bounded-wait self-test (see selftest.cu); the result is read with the status
+// block like a GEMM's.
+mxp_status launch_wait_selftest(void* workspace, int64_t limit_cycles, cudaStream_t stream);
+
 mxp_status tensor_peak_probe(int kind, int iters, double* ms, double* flops);
 
 // First 16 bytes of every GEMM workspace.

@@ -598,13 +598,8 @@ mxp_status launch_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const Params
 {
     using C = Cfg<BN, AP, BP>;
     auto kern = gemm_tc_kernel<BN, AP, BP, OutT>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) !=
-            cudaSuccess)
-            return MXP_ERR_CUDA;
-        attr_set = true;
-    }
+    static SmemAttrOnce once;
+    if (ensure_dynamic_smem(kern, C::kSmem, once) != cudaSuccess) return MXP_ERR_CUDA;
     const int64_t tiles = (int64_t)((prm.M + BM - 1) / BM) * ((prm.N + BN - 1) / BN);
     const unsigned grid = (unsigned)(tiles < prm.num_sms ? tiles : prm.num_sms);
     kern<<<grid, kThreads, C::kSmem, stream>>>(ta, tb, prm);
@@ -1051,13 +1046,8 @@ mxp_status launch_pair_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const P
 {
     using C = Cfg2<AP, BP>;
     auto kern = gemm_tc_pair_kernel<AP, BP, OutT>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) !=
-            cudaSuccess)
-            return MXP_ERR_CUDA;
-        attr_set = true;
-    }
+    static SmemAttrOnce once;
+    if (ensure_dynamic_smem(kern, C::kSmem, once) != cudaSuccess) return MXP_ERR_CUDA;
     const int64_t tiles = (int64_t)((prm.M + 255) / 256) * ((prm.N + 255) / 256);
     int64_t clusters = prm.num_sms / 2;
     if (tiles < clusters) clusters = tiles;

@@ -554,13 +554,8 @@ mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUt
 {
     using C = SCfg<kWide>;
     auto kern = gemm_tc_stream_kernel<kWide, OutT>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmem) !=
-            cudaSuccess)
-            return MXP_ERR_CUDA;
-        attr_set = true;
-    }
+    static SmemAttrOnce once;
+    if (ensure_dynamic_smem(kern, C::kSmem, once) != cudaSuccess) return MXP_ERR_CUDA;
     const int64_t tiles = (int64_t)((prm.M + kTile - 1) / kTile) * ((prm.N + kTile - 1) / kTile);
     int64_t clusters = num_sms / 2;
     if (tiles < clusters) clusters = tiles;

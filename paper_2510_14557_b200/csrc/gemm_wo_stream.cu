@@ -576,13 +576,9 @@ cudaError_t launch(WoParams prm, int num_sms, cudaStream_t stream)
     const size_t smem = wo_layout(prm.K, 8 * kMT, kPlus, prm.red_buffers, prm.meta_bufs).fixed +
                         (size_t)prm.stages * kStageBytes;
     auto kern = gemm_wo_stream_kernel<kMT, kMode, OutT>;
-    static size_t attr_smem = 0;  // raised as needed, once per size: the call is not free
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kSmemMax);
-        if (e != cudaSuccess) return e;
-        attr_smem = kSmemMax;
-    }
+    static SmemAttrOnce once;
+    const cudaError_t ea = ensure_dynamic_smem(kern, (int)kSmemMax, once);
+    if (ea != cudaSuccess) return ea;
     const int rgs = prm.N / kRows;
     const int mtiles = (prm.M + 8 * kMT - 1) / (8 * kMT);
     int gx = num_sms / mtiles;

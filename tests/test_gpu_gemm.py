@@ -366,3 +366,24 @@ def test_weight_only_mxpp_raw_planes_one_hot(kernel, monkeypatch):
     for m, c in enumerate(cols):
         want = (dw[:, c] * 2.0 ** (m - 8)).astype(np.float32).astype(np.float64)
         assert np.array_equal(got[m], want)
+
+
+# ------------------------------------------------------------------ bounded waits
+def test_bounded_wait_reports_timeout_and_leaves_the_device_usable():
+    # a wait that nothing satisfies comes back after its cycle limit, the kernel reports
+    # MXP_ERR_TIMEOUT through the status block and exits normally (no trap, no hang)
+    m = mxp()
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    m.mxp_wait_selftest(ws, 2_000_000)            # about a millisecond
+    assert m.mxp_gemm_status(ws) == 5             # MXP_ERR_TIMEOUT
+    torch.cuda.synchronize()
+    # the context is intact: a GEMM right after gives a correct result and a clean status
+    ap, da = _raw_operand(192, 256, MXP, seed=61)
+    bp, db = _raw_operand(320, 256, MXP, seed=62)
+    need = m.mxp_gemm_workspace_bytes(192, 320, 256, False, 1, 1)
+    ws2 = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32, workspace=ws2)
+    check_gemm(d, da, db)
+    assert m.mxp_gemm_status(ws2) == 0
+    with pytest.raises(Exception):
+        m.mxp_wait_selftest(ws, 0)                # limit out of range: rejected, nothing launched
