@@ -311,6 +311,15 @@ def part_prefill(mxp, synth, peaks, iters):
                 out["prefill_%s_A-%s_W-%s" % (cfg, an, bn)] = {
                     "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
                     "frac_fp4_nominal_9PF": tf / 9000.0}
+                try:  # the GEMM kernel's own cycle / nanosecond stamps (last launch)
+                    cyc, ns = mxp.mxp_gemm_clock_stamp(ws)
+                    macs = 8192 if (am or bm) else 16384  # per SM per clock: 8-bit containers, FP4
+                    sms = torch.cuda.get_device_properties(0).multi_processor_count
+                    out["prefill_%s_A-%s_W-%s" % (cfg, an, bn)].update({
+                        "kernel_us": ns / 1e3, "sm_mhz_in_kernel": cyc / ns * 1e3,
+                        "tensor_pipe_util_at_that_clock": 2.0 * M * N * K / (cyc * sms * 2 * macs)})
+                except mxp.MxpError:
+                    pass
                 del pa, pw
         if cfg == "cfg5":   # MX++ on both sides: same kernel, delta handled by the prepack
             pa, pw = mxp.mxp_quantize(a, mxp.MODE_MXFP4_PP), mxp.mxp_quantize(w, mxp.MODE_MXFP4_PP)
@@ -401,6 +410,8 @@ def run_ours(args, M, N, K, label):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms_local = e0.elapsed_time(e1) / args.steps
+    # SM cycles and nanoseconds the last step's GEMM kernel ran for, stamped by the kernel itself
+    stamp_cycles, stamp_ns = mxp.mxp_gemm_clock_stamp(ws)
     gemm_ms = sum(a.elapsed_time(b) for a, b in kev) / args.steps
     flops_step = 2.0 * M * N * K
     ms, flops_all = aggregate(ms_local, flops_step, dist if world > 1 else None)
@@ -469,6 +480,13 @@ def run_ours(args, M, N, K, label):
             probes[name] = pfl / pms / 1e9
         except Exception:
             probes[name] = None
+    # The board's power limit, not the tensor pipe, sets the SM clock of a dense GEMM: the kernel's
+    # own cycle and nanosecond stamps give the clock it really ran at, and the share of the tensor
+    # pipe's rate AT THAT CLOCK (nominal 8192 8-bit-container MACs per SM per clock) it used.
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
+    in_kernel_mhz = stamp_cycles / stamp_ns * 1e3
+    kernel_only_tflops = flops_step / stamp_ns / 1e3
+    pipe_tflops_at_clock = sms * 2 * 8192 * in_kernel_mhz * 1e6 / 1e12
     line = {
         "metric": METRIC, "value": flops_all / ms / 1e9, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms,
@@ -484,7 +502,11 @@ def run_ours(args, M, N, K, label):
                      "unit": "TFLOP/s", "frac": achieved / fp8_peak, "traffic": NCU_DRAM_TRAFFIC.get(args.workload),
                      "peak_source": "%s bf16 sustained x2 (nominal 8-bit-container : bf16 ratio)" % peaks["src"],
                      "kernel_ms": gemm_ms, "frac_of_fp4_peak_x4_bf16": achieved / fp4_peak,
-                     "issue_probe_tflops": probes},
+                     "issue_probe_tflops": probes,
+                     "in_kernel": {"sm_mhz": in_kernel_mhz, "kernel_us": stamp_ns / 1e3,
+                                   "tflops": kernel_only_tflops,
+                                   "tensor_pipe_tflops_at_that_clock": pipe_tflops_at_clock,
+                                   "tensor_pipe_util": kernel_only_tflops / pipe_tflops_at_clock}},
         "e2e": {"value": e2e_flops / e2e_ms / 1e9, "unit": UNIT, "h2d_bytes_per_step": M * K * 2,
                 "d2h_bytes_per_step": M * N * 2, "ms_per_step": e2e_ms},
         "gpu_launches": 3 * args.steps,  # quantize, prepack, GEMM

@@ -167,6 +167,19 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed 
 mxp_status mxp_gemm_status(const void *workspace, void *cuda_stream);
 
 /*
+ * How fast the SMs were clocked during the last GEMM that ran the streamed tensor-core kernel
+ * with this `workspace` (the path taken when the workspace has mxp_gemm_workspace_bytes(...)
+ * bytes; measurement aid, no counterpart in the paper).  The kernel's first CTA reads the SM
+ * cycle counter and the GPU's nanosecond timer when it starts and after its last tile;
+ * *sm_cycles / *nanoseconds is the SM clock in GHz the kernel really ran at, which a dense
+ * tensor-core kernel at the board's power limit holds well below the nominal maximum.
+ * Synchronises `cuda_stream`.  `workspace`: device, >= 256 bytes; the outputs are host
+ * pointers.  MXP_ERR_UNSUPPORTED when the workspace holds no stamp (another kernel ran).
+ */
+mxp_status mxp_gemm_clock_stamp(const void *workspace, void *cuda_stream, uint64_t *sm_cycles,
+                                uint64_t *nanoseconds);
+
+/*
  * Self-test of the bounded device-side waits (the paper has no counterpart: it is how this
  * library's kernels report a wait that runs out instead of hanging).  Launches one warp
  * that waits, for at most `limit_cycles` SM clock cycles (1 .. 2e9), on a barrier nothing

@@ -26,7 +26,7 @@ LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
 EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
-           "mxp_gemm_status", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
+           "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
 class MxpError(RuntimeError):
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         l.mxp_wait_selftest.restype = ci
         l.mxp_gemm_status.argtypes = [vp, vp]
         l.mxp_gemm_status.restype = ci
+        l.mxp_gemm_clock_stamp.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]
+        l.mxp_gemm_clock_stamp.restype = ci
         l.mxp_tensor_peak_probe.argtypes = [ci, ci, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_double)]
         l.mxp_tensor_peak_probe.restype = ci
@@ -250,6 +252,14 @@ def mxp_wait_selftest(workspace: torch.Tensor, limit_cycles: int) -> None:
 
 def mxp_gemm_status(workspace: torch.Tensor) -> int:
     return int(lib().mxp_gemm_status(workspace.data_ptr(), _stream()))
+
+
+def mxp_gemm_clock_stamp(workspace: torch.Tensor):
+    """(sm_cycles, nanoseconds) of the last streamed tensor-core GEMM that used `workspace`."""
+    clk, ns = ctypes.c_uint64(), ctypes.c_uint64()
+    st = lib().mxp_gemm_clock_stamp(workspace.data_ptr(), _stream(), ctypes.byref(clk), ctypes.byref(ns))
+    _check("mxp_gemm_clock_stamp", st)
+    return clk.value, ns.value
 
 
 def mxp_tensor_peak_probe(kind: int, iters: int):

@@ -185,6 +185,23 @@ mxp_status mxp_gemm_status(const void* workspace, void* cuda_stream)
     return sb.code == 0 ? MXP_OK : static_cast<mxp_status>(sb.code);
 }
 
+mxp_status mxp_gemm_clock_stamp(const void* workspace, void* cuda_stream, uint64_t* sm_cycles,
+                                uint64_t* nanoseconds)
+{
+    if (workspace == nullptr || sm_cycles == nullptr || nanoseconds == nullptr)
+        return MXP_ERR_INVALID_ARG;
+    mxp::ClockStamp cs;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(&cs, static_cast<const uint8_t*>(workspace) + mxp::kClockStampOffset,
+                        sizeof(cs), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return MXP_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return MXP_ERR_CUDA;
+    if (cs.ns_end <= cs.ns_begin || cs.clk_end <= cs.clk_begin) return MXP_ERR_UNSUPPORTED;
+    *sm_cycles = cs.clk_end - cs.clk_begin;
+    *nanoseconds = cs.ns_end - cs.ns_begin;
+    return MXP_OK;
+}
+
 mxp_status mxp_tensor_peak_probe(int kind, int iters, double* ms, double* flops)
 {
     if (ms == nullptr || flops == nullptr || iters <= 0 || kind < 0 || kind > 3)

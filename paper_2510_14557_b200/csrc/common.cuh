@@ -92,4 +92,12 @@ struct StatusBlock {
 };
 constexpr size_t kStatusBytes = 256;  // keeps what follows 256-byte aligned
 
+// Bytes 64..95 of a workspace of the streamed tensor-core GEMM: SM cycle counter and global
+// nanosecond timer, read by its first CTA when it starts and when it has stored its last tile.
+// cycles / nanoseconds is the SM clock the kernel actually ran at (the power cap lowers it).
+struct ClockStamp {
+    unsigned long long clk_begin, ns_begin, clk_end, ns_end;
+};
+constexpr size_t kClockStampOffset = 64;
+
 }  // namespace mxp

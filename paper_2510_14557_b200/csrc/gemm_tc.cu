@@ -1242,8 +1242,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                                      stream);
     // the in-place kernels implement Eq. 4 for MXFP4+ only: an MX++ operand needs the prepacked path
     if (A.mode == MXP_MODE_MXFP4_PP || B.mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
-    if (cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), stream) != cudaSuccess)
-        return MXP_ERR_CUDA;
+    // status block and clock stamp (these kernels leave no stamp)
+    if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return MXP_ERR_CUDA;
     bool use_pair = M > 128 && N > 128 && (ap || bp);
     if (force != nullptr && force[0] == 's') use_pair = false;
     if (force != nullptr && force[0] == 'p') use_pair = M > 128 && N > 128;

@@ -15,13 +15,17 @@
 //
 // Plain MXFP4 x MXFP4 needs only the scale pass and runs kind::mxf4 on the nibble planes.
 //
-// Kernel: clusters of two CTAs, one 256 x 256 output tile per cluster and step, persistent.
-// Warp 0 of each CTA issues the TMA loads for its own 128 rows of A, 128 rows of B and the
-// scale atoms; all of them signal one mbarrier in the even CTA, whose warp 1 issues
-// tcgen05.mma.cta_group::2 and commits to both CTAs.  Warps 2-9 drain the accumulator.
+// Kernel: clusters of two CTAs, persistent, one 256 x 480 (kind::mxf4: 256 x 448) output tile
+// per cluster and step, held in two accumulators that share the A tile: per flop that is 23 %
+// fewer bytes through TMA than a 256 x 256 tile, and the copies into shared memory, not the
+// tensor pipe, were what bounded the 256 x 256 kernel.  Warp 0 of each CTA issues the TMA loads
+// for its own 128 rows of A, its share of both halves of B and the scale atoms; all of them
+// signal one mbarrier in the even CTA, whose warp 1 issues tcgen05.mma.cta_group::2 and commits
+// to both CTAs.  Warps 2-9 drain the accumulators.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <cstdlib>
 #include <mutex>
 
@@ -62,9 +66,13 @@ int sm_count()
 
 namespace {
 
-constexpr int kTile = 256;          // output tile of a CTA pair: 256 x 256
+// Output tile of a CTA pair: 256 rows x `halves` accumulators of sub_n() columns.  With two,
+// they are 240 (kind::mxf4: 224) rather than 256 columns wide so that the scale factors (20
+// tensor memory columns per K group in flight) fit beside them in the 512 columns.
+constexpr int kTileM = 256;
+constexpr int sub_n(bool wide, int halves) { return halves == 1 ? 256 : wide ? 240 : 224; }
 constexpr int kRowBytes = 128;      // bytes of one operand row per stage (one swizzle span)
-constexpr int kHalfTile = 128 * kRowBytes;  // 16 KB: this CTA's 128 rows of A (or of B)
+constexpr int kHalfTile = 128 * kRowBytes;  // 16 KB: this CTA's 128 rows of A
 constexpr int kAtom = 512;          // scale bytes of 128 rows x 4 blocks
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
@@ -73,16 +81,20 @@ constexpr uint32_t kTmemCols = 512;
 
 // kWide = false: rows are 256 packed E2M1 codes (two scale atoms per stage), kind::mxf4.
 // kWide = true : rows are 128 E4M3 bytes (one scale atom per stage), kind::mxf8f6f4.
-template <bool kWide>
+// kHalves = 2: the tile has two halves (accumulators); 1: a single 256 x 256 accumulator, for
+// shapes whose larger tiles would not fill the GPU evenly.
+template <bool kWide, int kHalves>
 struct SCfg {
     static constexpr int kGroups = kWide ? 1 : 2;           // K groups of 128 elements per stage
     static constexpr int kSfA = kGroups * kAtom;            // own 128 rows of A
-    static constexpr int kSfB = 2 * kGroups * kAtom;        // all 256 rows of B
-    static constexpr int kStage = 2 * kHalfTile + kSfA + kSfB;
-#ifndef MXP_S_STAGES
-#define MXP_S_STAGES 6
-#endif
-    static constexpr int kStages = MXP_S_STAGES;
+    static constexpr int kSubN = sub_n(kWide, kHalves);     // columns of one accumulator
+    static constexpr int kTileN = kHalves * kSubN;
+    static constexpr int kBRows = kSubN / 2;                // rows of a B half each CTA supplies
+    static constexpr int kBTile = kBRows * kRowBytes;       // 15 (14) KB
+    static constexpr int kSfB = 2 * kHalves * kGroups * kAtom;  // all rows of the B halves
+    static constexpr int kStageRaw = kHalfTile + kHalves * kBTile + kSfA + kSfB;
+    static constexpr int kStage = (kStageRaw + 1023) / 1024 * 1024;  // swizzled tiles: 1024-aligned
+    static constexpr int kStages = kHalves == 2 ? 4 : 6;
     static constexpr int kSmem = kStages * kStage + 1024 /*barriers*/ + 1024 /*align*/;
     static constexpr int kElemsPerStage = kWide ? 128 : 256;
 };
@@ -122,14 +134,14 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
     tm = band * kBand + (r - tn * h);
 }
 
-template <bool kWide, typename OutT>
+template <bool kWide, int kHalves, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                       const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_sfa,
                       const __grid_constant__ CUtensorMap tmap_sfb, const SParams prm)
 {
-    using C = SCfg<kWide>;
+    using C = SCfg<kWide, kHalves>;
     constexpr int S = C::kStages;
     constexpr int G = C::kGroups;
 
@@ -145,15 +157,15 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
     volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
 
     auto a_tile = [&](int s) { return smem + s * C::kStage; };
-    auto b_tile = [&](int s) { return smem + s * C::kStage + kHalfTile; };
-    auto sfa = [&](int s) { return smem + s * C::kStage + 2 * kHalfTile; };
-    auto sfb = [&](int s) { return smem + s * C::kStage + 2 * kHalfTile + C::kSfA; };
+    auto b_tile = [&](int s, int j) { return smem + s * C::kStage + kHalfTile + j * C::kBTile; };
+    auto sfa = [&](int s) { return smem + s * C::kStage + kHalfTile + kHalves * C::kBTile; };
+    auto sfb = [&](int s) { return smem + s * C::kStage + kHalfTile + kHalves * C::kBTile + C::kSfA; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
     const int kstages = (prm.K + C::kElemsPerStage - 1) / C::kElemsPerStage;
-    const int tiles_m = (prm.M + kTile - 1) / kTile;
-    const int tiles_n = (prm.N + kTile - 1) / kTile;
+    const int tiles_m = (prm.M + kTileM - 1) / kTileM;
+    const int tiles_n = (prm.N + C::kTileN - 1) / C::kTileN;
     const int num_tiles = tiles_m * tiles_n;
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
 
@@ -180,9 +192,25 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
     ptx::cluster_sync();  // both CTAs' barriers exist before anything signals them remotely
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_acc = tmem_base;
-    const uint32_t tmem_sfa = tmem_base + kTile;      // 4 columns per K group
-    const uint32_t tmem_sfb = tmem_base + kTile + 8;  // 8 columns per K group
+    ClockStamp* stamp = reinterpret_cast<ClockStamp*>(reinterpret_cast<uint8_t*>(prm.status) +
+                                                      kClockStampOffset);
+    if (blockIdx.x == 0 && threadIdx.x == 64) {  // an epilogue warp: the last to finish
+        stamp->clk_begin = (unsigned long long)clock64();
+        stamp->ns_begin = ptx::globaltimer_ns();
+    }
+    // Accumulators at columns 0 and 256; scale factors in the gaps behind them.  Per K group:
+    // 4 columns for A's 128 rows, 8 for each half of B.  Two halves: kind::mxf8f6f4 has one
+    // group in flight (A at 240, B halves at 248 and 496); kind::mxf4 two (group g at
+    // 224 + 256 g: A, then the B halves 8 and 16 columns on).  One half: A at 256 + 4 g, B at
+    // 264 + 8 g.
+    auto tmem_sfa = [&](int g) {
+        return tmem_base + (kHalves == 1 ? 256u + 4u * g : kWide ? 240u : 224u + 256u * g);
+    };
+    auto tmem_sfb = [&](int g, int j) {
+        return tmem_base + (kHalves == 1 ? 264u + 8u * g
+                            : kWide      ? (j == 0 ? 248u : 496u)
+                                         : 232u + 256u * g + 8u * j);
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -196,8 +224,8 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
                 int tm, tn;
                 tile_coords(tile, tiles_m, tiles_n, tm, tn);
-                const int m0 = tm * kTile + 128 * (int)rank;
-                const int n0 = tn * kTile + 128 * (int)rank;
+                const int m0 = tm * kTileM + 128 * (int)rank;
+                const int n0 = tn * C::kTileN + C::kBRows * (int)rank;
                 for (int kt = 0; kt < kstages; ++kt, ++c) {
                     const int s = c % S;
                     const uint32_t use = c / S;
@@ -210,11 +238,15 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     if (rank == 0) ptx::mbar_arrive(&full[s]);
                     continue;
 #endif
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * C::kStage);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * C::kStageRaw);
                     ptx::tma_load_2d_pair(a_tile(s), &tmap_a, full0 + 8u * (uint32_t)s, kt * kRowBytes, m0);
-                    ptx::tma_load_2d_pair(b_tile(s), &tmap_b, full0 + 8u * (uint32_t)s, kt * kRowBytes, n0);
+#pragma unroll
+                    for (int j = 0; j < kHalves; ++j)
+                        ptx::tma_load_2d_pair(b_tile(s, j), &tmap_b, full0 + 8u * (uint32_t)s,
+                                              kt * kRowBytes, n0 + j * C::kSubN);
                     ptx::tma_load_3d_pair(sfa(s), &tmap_sfa, full0 + 8u * (uint32_t)s, 0, kt * G, 2 * tm + (int)rank);
-                    ptx::tma_load_3d_pair(sfb(s), &tmap_sfb, full0 + 8u * (uint32_t)s, 0, kt * G, 2 * tn);
+                    ptx::tma_load_3d_pair(sfb(s), &tmap_sfb, full0 + 8u * (uint32_t)s, 0, kt * G,
+                                          2 * kHalves * tn);
                 }
             }
         }
@@ -224,6 +256,10 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             uint32_t c = 0, ti = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
+                int tm, tn;
+                tile_coords(tile, tiles_m, tiles_n, tm, tn);
+                // a right half that lies wholly past column N gets no MMAs
+                const int halves = (kHalves == 2 && tn * C::kTileN + C::kSubN < prm.N) ? 2 : 1;
                 if (ti > 0 &&
                     !ptx::mbar_wait_cluster(acc_empty, (ti - 1) & 1, abort, kWaitLimit)) {
                     if (lane == 0) give_up(abort, prm.status, 0x2600);
@@ -242,7 +278,6 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     }
                     ptx::tc_fence_after_sync();
                     const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(a_tile(s)));
-                    const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(b_tile(s)));
                     const uint64_t d_sfa = ptx::smem_desc_sf(ptx::smem_u32(sfa(s)));
                     const uint64_t d_sfb = ptx::smem_desc_sf(ptx::smem_u32(sfb(s)));
                     const int groups =
@@ -253,30 +288,35 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #else
                         for (int g = 0; g < groups; ++g) {
 #endif
-                            const uint32_t t_sfa = tmem_sfa + 4 * g;
-                            const uint32_t t_sfb = tmem_sfb + 8 * g;
-                            ptx::tc_cp_sf_2cta(t_sfa, d_sfa + (uint64_t)(kAtom * g >> 4));
+                            ptx::tc_cp_sf_2cta(tmem_sfa(g), d_sfa + (uint64_t)(kAtom * g >> 4));
+                            // B's atoms in shared memory: [half j][128-row part h][K group g]
 #pragma unroll
-                            for (int h = 0; h < 2; ++h)
-                                ptx::tc_cp_sf_2cta(t_sfb + 4 * h,
-                                                   d_sfb + (uint64_t)((G * kAtom * h + kAtom * g) >> 4));
-                            if (kWide) {
+                            for (int jh = 0; jh < 2 * kHalves; ++jh)
+                                ptx::tc_cp_sf_2cta(tmem_sfb(g, jh >> 1) + 4 * (jh & 1),
+                                                   d_sfb + (uint64_t)((G * kAtom * jh + kAtom * g) >> 4));
+                            for (int j = 0; j < halves; ++j) {
+                                const uint32_t tmem_acc = tmem_base + 256u * j;
+                                const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(b_tile(s, j)));
+                                if (kWide) {
 #pragma unroll
-                                for (int kk = 0; kk < 4; ++kk) {
-                                    const uint32_t idesc =
-                                        ptx::idesc_block_scaled(0, 0, kTile, kTile, kk, kk);
-                                    ptx::mma_mxf8f6f4_2cta(tmem_acc, da + (uint64_t)(2 * kk),
-                                                           db + (uint64_t)(2 * kk), idesc, t_sfa,
-                                                           t_sfb, accumulate | (uint32_t)kk);
-                                }
-                            } else {
+                                    for (int kk = 0; kk < 4; ++kk) {
+                                        const uint32_t idesc =
+                                            ptx::idesc_block_scaled(0, 0, kTileM, C::kSubN, kk, kk);
+                                        ptx::mma_mxf8f6f4_2cta(tmem_acc, da + (uint64_t)(2 * kk),
+                                                               db + (uint64_t)(2 * kk), idesc,
+                                                               tmem_sfa(g), tmem_sfb(g, j),
+                                                               accumulate | (uint32_t)kk);
+                                    }
+                                } else {
 #pragma unroll
-                                for (int kk = 0; kk < 2; ++kk) {
-                                    const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
-                                    const uint32_t idesc =
-                                        ptx::idesc_block_scaled(1, 1, kTile, kTile, 2 * kk, 2 * kk);
-                                    ptx::mma_mxf4_2cta(tmem_acc, da + adv, db + adv, idesc, t_sfa,
-                                                       t_sfb, accumulate | (uint32_t)(g | kk));
+                                    for (int kk = 0; kk < 2; ++kk) {
+                                        const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
+                                        const uint32_t idesc = ptx::idesc_block_scaled(
+                                            1, 1, kTileM, C::kSubN, 2 * kk, 2 * kk);
+                                        ptx::mma_mxf4_2cta(tmem_acc, da + adv, db + adv, idesc,
+                                                           tmem_sfa(g), tmem_sfb(g, j),
+                                                           accumulate | (uint32_t)(g | kk));
+                                    }
                                 }
                             }
                         }
@@ -293,19 +333,23 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        // Each warp owns 32 accumulator rows (its TMEM lane quarter) x 128 columns.  All 128
-        // columns go to registers first and the accumulator is released at once, so the
-        // next tile's MMAs overlap the conversion and the global stores.
+        // Each warp owns 32 rows (its TMEM lane quarter) and moves chunks of half an accumulator
+        // (120, 112 or 128 columns) through registers.  Two halves: warps 2-5 drain the left
+        // accumulator, 6-9 the right one, two chunks each.  One half: warps 2-5 take its left
+        // chunk, 6-9 its right chunk.
+        // A warp releases the accumulators as soon as it has read its last chunk.
         const int q = warp & 3;  // the TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;
-        constexpr int kCols = kTile / 2;
+        const int wsel = (warp - 2) >> 2;
+        const int j = kHalves == 2 ? wsel : 0;
+        const int ch0 = kHalves == 2 ? 0 : wsel, ch1 = kHalves == 2 ? 2 : wsel + 1;
+        constexpr int kCols = C::kSubN / 2;
         const uint32_t acc_empty0 = ptx::map_to_cta(ptx::smem_u32(acc_empty), 0);
         uint32_t ti = 0;
         bool ok = true;
         for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++ti) {
             int tm, tn;
             tile_coords(tile, tiles_m, tiles_n, tm, tn);
-            const int m0 = tm * kTile + 128 * (int)rank, n0 = tn * kTile;
+            const int m0 = tm * kTileM + 128 * (int)rank, n0 = tn * C::kTileN + j * C::kSubN;
             if (!ptx::mbar_wait(acc_full, ti & 1, abort, kWaitLimit)) {
                 give_up(abort, prm.status, 0x2500);
                 ok = false;
@@ -313,53 +357,65 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
             ptx::tc_fence_after_sync();
             const int row = m0 + 32 * q + lane;
-            const int cbase = half * kCols;
-            uint32_t rr[kCols];
+            const uint32_t taddr = tmem_base + 256u * j + ((uint32_t)(32 * q) << 16);
+            for (int ch = ch0; ch < ch1; ++ch) {
+                uint32_t rr[kCols];
+                const uint32_t ta = taddr + ch * kCols;
+                constexpr int k32 = kCols / 32, k16 = (kCols % 32) / 16, k8 = (kCols % 16) / 8;
 #pragma unroll
-            for (int cb = 0; cb < kCols / 32; ++cb)
-                ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(32 * q) << 16) + cbase + 32 * cb,
-                                   reinterpret_cast<uint32_t(&)[32]>(rr[32 * cb]));
-            ptx::tmem_ld_wait();
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
-            if (row >= prm.M) continue;
-            OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + n0 + cbase;
-            const int col0 = n0 + cbase;
-            if (col0 + kCols <= prm.N && prm.d_vec_ok) {
-                uint4* p = reinterpret_cast<uint4*>(drow);
-                if (sizeof(OutT) == 4) {
+                for (int cb = 0; cb < k32; ++cb)
+                    ptx::tmem_ld_32x32(ta + 32 * cb, reinterpret_cast<uint32_t(&)[32]>(rr[32 * cb]));
+                if (k16) ptx::tmem_ld_32x16(ta + 32 * k32, reinterpret_cast<uint32_t(&)[16]>(rr[kCols - 16 - 8 * k8]));
+                if (k8) ptx::tmem_ld_32x8(ta + kCols - 8, reinterpret_cast<uint32_t(&)[8]>(rr[kCols - 8]));
+                ptx::tmem_ld_wait();
+                if (ch == ch1 - 1) {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(acc_empty0);
+                }
+                const int col0 = n0 + ch * kCols;
+                if (row >= prm.M || col0 >= prm.N) continue;
+                OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + col0;
+                if (col0 + kCols <= prm.N && prm.d_vec_ok) {
+                    uint4* p = reinterpret_cast<uint4*>(drow);
+                    if (sizeof(OutT) == 4) {
 #pragma unroll
-                    for (int i = 0; i < kCols / 4; ++i)
-                        p[i] = make_uint4(rr[4 * i], rr[4 * i + 1], rr[4 * i + 2], rr[4 * i + 3]);
+                        for (int i = 0; i < kCols / 4; ++i)
+                            p[i] = make_uint4(rr[4 * i], rr[4 * i + 1], rr[4 * i + 2], rr[4 * i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kCols / 8; ++i) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const __nv_bfloat162 h2 =
+                                    __floats2bfloat162_rn(__uint_as_float(rr[8 * i + 2 * k]),
+                                                          __uint_as_float(rr[8 * i + 2 * k + 1]));
+                                o[k] = *reinterpret_cast<const uint32_t*>(&h2);
+                            }
+                            p[i] = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < kCols / 8; ++i) {
-                        uint32_t o[4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(
-                                __uint_as_float(rr[8 * i + 2 * k]), __uint_as_float(rr[8 * i + 2 * k + 1]));
-                            o[k] = *reinterpret_cast<const uint32_t*>(&h2);
+                    for (int i = 0; i < kCols; ++i) {
+                        if (col0 + i < prm.N) {
+                            if (sizeof(OutT) == 4)
+                                reinterpret_cast<float*>(drow)[i] = __uint_as_float(rr[i]);
+                            else
+                                reinterpret_cast<__nv_bfloat16*>(drow)[i] =
+                                    __float2bfloat16_rn(__uint_as_float(rr[i]));
                         }
-                        p[i] = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < kCols; ++i) {
-                    if (col0 + i < prm.N) {
-                        if (sizeof(OutT) == 4)
-                            reinterpret_cast<float*>(drow)[i] = __uint_as_float(rr[i]);
-                        else
-                            reinterpret_cast<__nv_bfloat16*>(drow)[i] =
-                                __float2bfloat16_rn(__uint_as_float(rr[i]));
                     }
                 }
             }
         }
     }
 
+    if (blockIdx.x == 0 && threadIdx.x == 64) {
+        stamp->clk_end = (unsigned long long)clock64();
+        stamp->ns_end = ptx::globaltimer_ns();
+    }
     // ---------------------------------------------------------------------- teardown
     // After a timeout, copies may still be in flight into this pair's shared memory: give
     // them (bounded) time to land before the CTAs leave.  `full` of the even CTA counts both.
@@ -384,10 +440,12 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
 // ------------------------------------------------------------------------------ prepack
 // One launch prepares both operands.  Its CTAs are of two kinds, told apart by block index:
 //
-// scale CTAs: scale plane [rows][nbk] -> atoms [ceil(rows/128)][nbk/4][512]; inside an atom
-//   the four scale bytes of row r (r < 128) sit at (r % 32) * 16 + (r / 32) * 4.  Rows past
-//   the end are written as zero.  A CTA handles 128 rows x up to 32 K groups through shared
-//   memory, so reads and writes are both contiguous.
+// scale CTAs: scale plane [rows][nbk] -> atoms [row groups][nbk/4][512]; inside an atom the
+//   four scale bytes of row r (r < 128) sit at (r % 32) * 16 + (r / 32) * 4.  Row groups follow
+//   the GEMM's accumulators: two per `tile_rows` rows (256 for A; 240 or 224, one half tile,
+//   for B), the second starting 128 rows in, so for B it holds 112 or 96 rows.  Rows past the
+//   end of the half tile or of the operand are written as zero.  A CTA handles one row group x up to 32 K groups
+//   through shared memory, so reads and writes are both contiguous.
 // widen CTAs (only when an operand is MX+): packed codes [rows][K/2] -> E4M3 bytes [rows][K],
 //   one thread per 16 elements (8 bytes in, 16 bytes out, both contiguous across the warp).
 //   E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6 are the E4M3 bytes 00 30 38 3C 40 44 48 4C; the
@@ -400,8 +458,9 @@ struct PrepackOperand {
     uint8_t* atoms;
     uint8_t* wide;            // nullptr: not widened
     int rows, nbk;
+    int tile_rows;            // rows per accumulator: kTileM for A, sub_n() for B
     int pp;                   // MX++ operand: index bits 7:5 hold delta (Sec. 4.3)
-    unsigned scale_ctas;      // ceil(rows/128) * ceil(nbk/128)
+    unsigned scale_ctas;      // row groups * ceil(nbk/128)
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
 };
 
@@ -414,9 +473,10 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
     const uint32_t* src = reinterpret_cast<const uint32_t*>(op.scales);
     for (int i = threadIdx.x; i < 128 * 32; i += 256) {
         const int r = i >> 5, kg = i & 31;
-        const int64_t row = (int64_t)rg * 128 + r;
+        const int in_tile = (rg & 1) * 128 + r;
+        const int64_t row = (int64_t)(rg >> 1) * op.tile_rows + in_tile;
         uint32_t v = 0;
-        if (kg < nkg && row < op.rows) {
+        if (kg < nkg && in_tile < op.tile_rows && row < op.rows) {
             v = src[row * kgroups + kg0 + kg];
             if (op.pp) {
                 const uint32_t ix = reinterpret_cast<const uint32_t*>(op.bm_index)[row * kgroups + kg0 + kg];
@@ -490,14 +550,14 @@ __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, co
 #ifndef MXP_S_L2PROMO
 #define MXP_S_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
 #endif
-// 2-D byte tensor [rows][row_bytes], boxes of 128 bytes x 128 rows, 128B swizzle.
-bool make_tmap_rows(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t row_bytes)
+// 2-D byte tensor [rows][row_bytes], boxes of 128 bytes x box_rows rows, 128B swizzle.
+bool make_tmap_rows(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t row_bytes, int box_rows)
 {
     EncodeFn fn = tensormap_encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-    const cuuint32_t box[2] = {(cuuint32_t)kRowBytes, 128u};
+    const cuuint32_t box[2] = {(cuuint32_t)kRowBytes, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -525,7 +585,10 @@ struct Layout {
 };
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// scale row groups (atoms of 128 rows) of an operand whose output tiles take `tile_rows` rows
+inline int64_t row_groups(int64_t rows, int tile_rows) { return 2 * ((rows + tile_rows - 1) / tile_rows); }
 
+// Sized for either tiling of B's scales (the tile shape is chosen per call).
 Layout layout(int64_t M, int64_t N, int64_t K, bool wide)
 {
     Layout l;
@@ -533,10 +596,10 @@ Layout layout(int64_t M, int64_t N, int64_t K, bool wide)
     size_t off = kStatusBytes;
     off = round_up(off, 1024);
     l.sfa = off;
-    off += (size_t)((M + 127) / 128) * kgroups * kAtom;
+    off += (size_t)row_groups(M, kTileM) * kgroups * kAtom;
     off = round_up(off, 1024);
     l.sfb = off;
-    off += (size_t)((N + 127) / 128) * kgroups * kAtom;
+    off += (size_t)std::max(row_groups(N, sub_n(wide, 1)), row_groups(N, sub_n(wide, 2))) * kgroups * kAtom;
     off = round_up(off, 1024);
     l.wa = off;
     if (wide) off += (size_t)M * (size_t)K;
@@ -547,16 +610,32 @@ Layout layout(int64_t M, int64_t N, int64_t K, bool wide)
     return l;
 }
 
-template <bool kWide, typename OutT>
+// Two halves per tile unless that leaves the last wave of tiles much emptier than single
+// halves would: compare the columns each CTA pair walks through either way.
+int choose_halves(int64_t M, int64_t N, bool wide, int num_sms)
+{
+    const char* env = std::getenv("MXP_S_HALVES");  // "1" / "2": tests and experiments
+    if (env != nullptr && (env[0] == '1' || env[0] == '2')) return env[0] - '0';
+    const int64_t clusters = num_sms / 2, tiles_m = (M + kTileM - 1) / kTileM;
+    auto cost = [&](int h) {  // columns a CTA pair walks through
+        const int64_t tile_n = (int64_t)h * sub_n(wide, h);
+        const int64_t tiles = tiles_m * ((N + tile_n - 1) / tile_n);
+        return (tiles + clusters - 1) / clusters * tile_n;
+    };
+    return cost(1) < cost(2) ? 1 : 2;
+}
+
+template <bool kWide, int kHalves, typename OutT>
 mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tsa,
                          const CUtensorMap& tsb, const SParams& prm, int num_sms,
                          cudaStream_t stream)
 {
-    using C = SCfg<kWide>;
-    auto kern = gemm_tc_stream_kernel<kWide, OutT>;
+    using C = SCfg<kWide, kHalves>;
+    auto kern = gemm_tc_stream_kernel<kWide, kHalves, OutT>;
     static SmemAttrOnce once;
     if (ensure_dynamic_smem(kern, C::kSmem, once) != cudaSuccess) return MXP_ERR_CUDA;
-    const int64_t tiles = (int64_t)((prm.M + kTile - 1) / kTile) * ((prm.N + kTile - 1) / kTile);
+    const int64_t tiles =
+        (int64_t)((prm.M + kTileM - 1) / kTileM) * ((prm.N + C::kTileN - 1) / C::kTileN);
     int64_t clusters = num_sms / 2;
     if (tiles < clusters) clusters = tiles;
     cudaLaunchConfig_t cfg = {};
@@ -594,21 +673,24 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
 }
 
 namespace {
-// Prepacked form of one operand in a caller-owned buffer: scale atoms, then (wide) E4M3 bytes.
+// Prepacked form of the B operand in a caller-owned buffer: scale atoms, then (wide) E4M3 bytes.
 struct PackedLayout {
-    size_t atoms, wide, total;
+    size_t atoms[2];  // scale atoms tiled for one-half tiles, for two-half tiles
+    size_t wide, total;
 };
 PackedLayout packed_layout(int64_t rows, int64_t K, bool wide)
 {
     PackedLayout l;
-    l.atoms = 0;
-    l.wide = round_up((size_t)((rows + 127) / 128) * (size_t)(K / 128) * kAtom, 1024);
+    l.atoms[0] = 0;
+    l.atoms[1] = round_up((size_t)row_groups(rows, sub_n(wide, 1)) * (size_t)(K / 128) * kAtom, 1024);
+    l.wide = l.atoms[1] +
+             round_up((size_t)row_groups(rows, sub_n(wide, 2)) * (size_t)(K / 128) * kAtom, 1024);
     l.total = l.wide + (wide ? round_up((size_t)rows * (size_t)K, 1024) : 0);
     return l;
 }
 
-PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, bool wide, uint8_t* atoms,
-                               uint8_t* wide_bytes)
+PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, bool wide, int tile_rows,
+                               uint8_t* atoms, uint8_t* wide_bytes)
 {
     const int nbk = (int)(K / 32);
     const int kgroups = nbk / 4;
@@ -621,7 +703,8 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     op.wide = wide ? wide_bytes : nullptr;
     op.rows = (int)rows;
     op.nbk = nbk;
-    op.scale_ctas = (unsigned)(((rows + 127) / 128) * ((kgroups + 31) / 32));
+    op.tile_rows = tile_rows;
+    op.scale_ctas = (unsigned)(row_groups(rows, tile_rows) * ((kgroups + 31) / 32));
     op.widen_ctas = wide ? (unsigned)((rows * nbk * 2 + 255) / 256) : 0u;
     return op;
 }
@@ -651,10 +734,15 @@ mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_
         return MXP_ERR_INVALID_ARG;
     const PackedLayout l = packed_layout(P.rows, P.cols, wide);
     uint8_t* o = static_cast<uint8_t*>(out);
-    const PrepackOperand pa = prepack_operand(P, P.rows, P.cols, wide, o + l.atoms, o + l.wide);
-    const uint64_t ctas = (uint64_t)pa.scale_ctas + pa.widen_ctas;
+    // both tilings of the scales (the GEMM picks its tile shape per call); widened bytes once
+    const PrepackOperand p1 =
+        prepack_operand(P, P.rows, P.cols, wide, sub_n(wide, 1), o + l.atoms[0], o + l.wide);
+    PrepackOperand p2 =
+        prepack_operand(P, P.rows, P.cols, wide, sub_n(wide, 2), o + l.atoms[1], o + l.wide);
+    p2.widen_ctas = 0;
+    const uint64_t ctas = (uint64_t)p1.scale_ctas + p2.scale_ctas + p1.widen_ctas;
     if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
-    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, no_operand(), nullptr);
+    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(p1, p2, nullptr);
     return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }
 
@@ -677,7 +765,9 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     if (num_sms <= 0) return MXP_ERR_CUDA;
     const int nbk = (int)(K / 32);
     const int kgroups = nbk / 4;
-    const int rga = (int)((M + 127) / 128), rgb = (int)((N + 127) / 128);
+    const int halves = choose_halves(M, N, wide, num_sms);
+    const int sub = sub_n(wide, halves);
+    const int rga = (int)row_groups(M, kTileM), rgb = (int)row_groups(N, sub);
     if ((reinterpret_cast<uintptr_t>(A.nibbles) | reinterpret_cast<uintptr_t>(B.nibbles)) & 15)
         return MXP_ERR_INVALID_ARG;
     // the widening threads index their operand with 32 bits
@@ -689,11 +779,12 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
         return MXP_ERR_INVALID_ARG;
 
     const PackedLayout lb = packed_layout(N, K, wide);
-    const uint8_t* b_atoms = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms : ws + l.sfb;
+    const uint8_t* b_atoms =
+        b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms[halves - 1] : ws + l.sfb;
     const uint8_t* b_wide = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.wide : ws + l.wb;
-    const PrepackOperand pa = prepack_operand(A, M, K, wide, ws + l.sfa, ws + l.wa);
+    const PrepackOperand pa = prepack_operand(A, M, K, wide, kTileM, ws + l.sfa, ws + l.wa);
     const PrepackOperand pb =
-        b_prepacked ? no_operand() : prepack_operand(B, N, K, wide, ws + l.sfb, ws + l.wb);
+        b_prepacked ? no_operand() : prepack_operand(B, N, K, wide, sub, ws + l.sfb, ws + l.wb);
     const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
     if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
     prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, pb, static_cast<StatusBlock*>(workspace));
@@ -702,10 +793,11 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     CUtensorMap ta, tb, tsa, tsb;
     const int box_kg = wide ? 1 : 2;
     const bool maps_ok =
-        (wide ? make_tmap_rows(&ta, ws + l.wa, M, K) && make_tmap_rows(&tb, b_wide, N, K)
-              : make_tmap_rows(&ta, A.nibbles, M, K / 2) && make_tmap_rows(&tb, B.nibbles, N, K / 2)) &&
+        (wide ? make_tmap_rows(&ta, ws + l.wa, M, K, 128) && make_tmap_rows(&tb, b_wide, N, K, sub / 2)
+              : make_tmap_rows(&ta, A.nibbles, M, K / 2, 128) &&
+                    make_tmap_rows(&tb, B.nibbles, N, K / 2, sub / 2)) &&
         make_tmap_atoms(&tsa, ws + l.sfa, rga, kgroups, box_kg, 1) &&
-        make_tmap_atoms(&tsb, b_atoms, rgb, kgroups, box_kg, 2);
+        make_tmap_atoms(&tsb, b_atoms, rgb, kgroups, box_kg, 2 * halves);
     if (!maps_ok) return MXP_ERR_CUDA;
 
     SParams prm;
@@ -717,13 +809,13 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
                    ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
     prm.status = static_cast<StatusBlock*>(workspace);
-    if (wide)
-        return d_dt == MXP_F32
-                   ? launch_stream<true, float>(ta, tb, tsa, tsb, prm, num_sms, stream)
-                   : launch_stream<true, __nv_bfloat16>(ta, tb, tsa, tsb, prm, num_sms, stream);
-    return d_dt == MXP_F32
-               ? launch_stream<false, float>(ta, tb, tsa, tsb, prm, num_sms, stream)
-               : launch_stream<false, __nv_bfloat16>(ta, tb, tsa, tsb, prm, num_sms, stream);
+    const bool f32 = d_dt == MXP_F32;
+#define MXP_S_LAUNCH(W, H)                                                                    \
+    (f32 ? launch_stream<W, H, float>(ta, tb, tsa, tsb, prm, num_sms, stream)                 \
+         : launch_stream<W, H, __nv_bfloat16>(ta, tb, tsa, tsb, prm, num_sms, stream))
+    if (wide) return halves == 2 ? MXP_S_LAUNCH(true, 2) : MXP_S_LAUNCH(true, 1);
+    return halves == 2 ? MXP_S_LAUNCH(false, 2) : MXP_S_LAUNCH(false, 1);
+#undef MXP_S_LAUNCH
 }
 
 }  // namespace mxp

@@ -246,6 +246,44 @@ def test_tc_prepacked_weights_match_mxp_gemm(M, N, K, amode, bmode):
         assert torch.equal(d0, d1)
 
 
+@pytest.mark.parametrize("halves", ["1", "2"])
+@pytest.mark.parametrize("amode,bmode", [(MX, MX), (MXP, MXP), (MX, 2)])
+@pytest.mark.parametrize("M,N,K", [(300, 250, 256), (257, 481, 384), (300, 959, 256), (513, 1000, 128),
+                                   (256, 448, 512), (384, 960, 128)])
+def test_tc_stream_tile_halves_and_ragged_edges(M, N, K, amode, bmode, halves, monkeypatch):
+    # the streamed kernel's output tile has one or two halves of 240 (plain MXFP4: 224) columns;
+    # N values just past a half, just past a tile, exact multiples, and ragged on both sides,
+    # with either tile shape forced
+    monkeypatch.setenv("MXP_S_HALVES", halves)
+    ap, da = _raw_operand(M, K, amode, seed=M + N)
+    bp, db = _raw_operand(N, K, bmode, seed=N + K)
+    m = mxp()
+    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode), dtype=torch.uint8, device="cuda")
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm(ap, bp, out_dtype=dt, workspace=ws)
+        assert m.mxp_gemm_status(ws) == 0
+        check_gemm(d, da, db)
+
+
+def test_tc_stream_clock_stamp():
+    # the streamed kernel leaves the SM cycles and nanoseconds its first CTA ran for; the in-place
+    # kernels clear the stamp
+    from paper_2510_14557_b200 import MxpError
+    M, N, K = 512, 1024, 1024
+    ap, _ = _raw_operand(M, K, MXP, seed=1)
+    bp, _ = _raw_operand(N, K, MXP, seed=2)
+    m = mxp()
+    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, MXP, MXP), dtype=torch.uint8, device="cuda")
+    m.mxp_gemm(ap, bp, workspace=ws)
+    cycles, ns = m.mxp_gemm_clock_stamp(ws)
+    assert 500 < ns < 10_000_000
+    assert 0.1 < cycles / ns < 2.5          # GHz
+    small = ws[:4096]
+    m.mxp_gemm(ap, bp, workspace=small)      # too small for the streamed path: in-place kernels
+    with pytest.raises(MxpError):
+        m.mxp_gemm_clock_stamp(small)
+
+
 def test_tc_prepack_rejects_bad_arguments():
     from paper_2510_14557_b200 import MxpError
     m = mxp()
