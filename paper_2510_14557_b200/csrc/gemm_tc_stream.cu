@@ -78,6 +78,7 @@ constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr long long kWaitLimit = 4000000000ll;  // cycles (~2 s) before a wait gives up
 constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kFmtE4M3 = 0, kFmtE2M3 = 3;  // instruction-descriptor codes, kind::mxf8f6f4
 
 // kWide = false: rows are 256 packed E2M1 codes (two scale atoms per stage), kind::mxf4.
 // kWide = true : rows are 128 E4M3 bytes (one scale atom per stage), kind::mxf8f6f4.
@@ -101,6 +102,7 @@ struct SCfg {
 
 struct SParams {
     int M, N, K;
+    uint32_t a_fmt, b_fmt;  // kind::mxf8f6f4 operand formats (kFmtE2M3 / kFmtE4M3); wide only
     void* D;
     int64_t ldd;
     int d_vec_ok;
@@ -300,8 +302,8 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                 if (kWide) {
 #pragma unroll
                                     for (int kk = 0; kk < 4; ++kk) {
-                                        const uint32_t idesc =
-                                            ptx::idesc_block_scaled(0, 0, kTileM, C::kSubN, kk, kk);
+                                        const uint32_t idesc = ptx::idesc_block_scaled(
+                                            prm.a_fmt, prm.b_fmt, kTileM, C::kSubN, kk, kk);
                                         ptx::mma_mxf8f6f4_2cta(tmem_acc, da + (uint64_t)(2 * kk),
                                                                db + (uint64_t)(2 * kk), idesc,
                                                                tmem_sfa(g), tmem_sfb(g, j),
@@ -496,7 +498,25 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
     for (int i = threadIdx.x; i < nkg * 128; i += 256) dst[i] = tile[(i >> 7) * 129 + (i & 127)];
 }
 
-__device__ __forceinline__ void widen_e4m3(const PrepackOperand& op, unsigned id)
+// Eight E2M1 codes (nibble i of x) -> eight E2M3 codes, 6 bits each, code i at bits 6i..6i+5.
+// Both formats have exponent bias 1, so the E2M3 code of an E2M1 value is its code with two
+// zero mantissa bits appended: s e e m -> s e e m 0 0.  The nibbles are spread from a pitch of
+// 4 bits to a pitch of 6 in three steps (by 8, 4 and 2 bits for bits 2, 1 and 0 of i).
+__device__ __forceinline__ uint64_t e2m1x8_to_e2m3x8(uint32_t x)
+{
+    uint64_t y = x;
+    y = (y & 0x000000000000FFFFull) | ((y & 0x00000000FFFF0000ull) << 8);
+    y = (y & 0x00000000FF0000FFull) | ((y & 0x000000FF0000FF00ull) << 4);
+    y = (y & 0x000000F00F00F00Full) | ((y & 0x00000F00F00F00F0ull) << 2);
+    return y << 2;
+}
+
+// One thread per 16 elements (half a block): 8 bytes of codes in, 16 bytes out.
+//  * E2M3 (MXFP4 and MXFP4+ operands): the 16 six-bit codes packed into 12 bytes, then 4 bytes
+//    of padding, which is how kind::mxf8f6f4 reads 6-bit operands from shared memory.  The BM of
+//    an MX+ block, 4 + m/2 (Eq. 3), is the E2M3 code s 11 mmm.
+//  * E4M3 (MX++ operands, whose rescaled values need the exponent range): one byte per code.
+__device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned id)
 {
     const uint32_t t = id * 256u + threadIdx.x;  // half block: 16 elements
     const uint32_t b = t >> 1;
@@ -504,28 +524,41 @@ __device__ __forceinline__ void widen_e4m3(const PrepackOperand& op, unsigned id
     const uint2 w = reinterpret_cast<const uint2*>(op.nibbles)[t];
     const uint32_t sc = op.scales[b];
     const uint32_t ib = op.bm_index != nullptr ? op.bm_index[b] : 0u;
+    // the BM, if this half block holds it: element e, code nib
+    const uint32_t p = ib & 31u;
+    const uint32_t e = p & 15u;
+    const uint32_t nib = (((e & 8u) ? w.y : w.x) >> ((e & 7u) * 4u)) & 15u;
+    const bool has_bm = op.bm_index != nullptr && (p >> 4) == (t & 1u);
+    uint8_t* dst = op.wide + (size_t)t * 16u;
+    if (!op.pp) {
+        uint64_t lo = e2m1x8_to_e2m3x8(w.x), hi = e2m1x8_to_e2m3x8(w.y);
+        if (has_bm) {  // Eq. 3, BM branch
+            const uint32_t sh = 6u * (e & 7u);
+            const uint64_t code = ((nib & 8u) << 2) | 0x18u | (nib & 7u);
+            uint64_t& half = (e & 8u) ? hi : lo;
+            half = (half & ~(0x3Full << sh)) | (code << sh);
+        }
+        uint4 o = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32) | ((uint32_t)hi << 16),
+                             (uint32_t)(hi >> 16), 0u);
+        if (sc == 0u) o = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(dst) = o;
+        return;
+    }
     // MX++: BM scaled up by 2^shift, NBMs down by 2^-(delta - shift) (see mxpp_shift)
-    const uint32_t delta = op.pp ? ib >> 5 : 0u;
-    const uint32_t shift = op.pp ? mxpp_shift(sc, delta) : 0u;
-    const uint2 lut = op.pp ? kE4m3Lut[delta - shift] : make_uint2(0x3C383000u, 0x4C484440u);
+    const uint32_t delta = ib >> 5;
+    const uint32_t shift = mxpp_shift(sc, delta);
+    const uint2 lut = kE4m3Lut[delta - shift];
     uint4 o;
     o.x = e2m1x4_to_e4m3x4(w.x, lut);
     o.y = e2m1x4_to_e4m3x4(w.x >> 16, lut);
     o.z = e2m1x4_to_e4m3x4(w.y, lut);
     o.w = e2m1x4_to_e4m3x4(w.y >> 16, lut);
     if (sc == 0u) o = make_uint4(0u, 0u, 0u, 0u);
-    uint8_t* dst = op.wide + (size_t)t * 16u;
     *reinterpret_cast<uint4*>(dst) = o;
-    if (op.bm_index != nullptr) {
-        // Eq. 3, BM branch.  Same thread, later store to the same bytes: lands after the
-        // vector store above.
-        const uint32_t p = ib & 31u;
-        const uint32_t e = p & 15u;
-        const uint32_t word = (e & 8u) ? w.y : w.x;
-        const uint32_t nib = (word >> ((e & 7u) * 4u)) & 15u;
-        if ((p >> 4) == (t & 1u) && sc != 0u)
-            dst[e] = (uint8_t)(((nib & 8u) << 4) | (0x48u + (shift << 3)) | (nib & 7u));
-    }
+    // Eq. 3, BM branch.  Same thread, later store to the same bytes: lands after the vector
+    // store above.
+    if (has_bm && sc != 0u)
+        dst[e] = (uint8_t)(((nib & 8u) << 4) | (0x48u + (shift << 3)) | (nib & 7u));
 }
 
 __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, const PrepackOperand b,
@@ -542,9 +575,9 @@ __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, co
     id -= a.scale_ctas;
     if (id < b.scale_ctas) return prepack_scales(b, id, tile);
     id -= b.scale_ctas;
-    if (id < a.widen_ctas) return widen_e4m3(a, id);
+    if (id < a.widen_ctas) return widen_codes(a, id);
     id -= a.widen_ctas;
-    widen_e4m3(b, id);
+    widen_codes(b, id);
 }
 
 #ifndef MXP_S_L2PROMO
@@ -804,6 +837,8 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     prm.M = (int)M;
     prm.N = (int)N;
     prm.K = (int)K;
+    prm.a_fmt = A.mode == MXP_MODE_MXFP4_PP ? kFmtE4M3 : kFmtE2M3;
+    prm.b_fmt = B.mode == MXP_MODE_MXFP4_PP ? kFmtE4M3 : kFmtE2M3;
     prm.D = D;
     prm.ldd = ldd;
     prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
