@@ -33,6 +33,14 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
                                   const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
                                   void* status, cudaStream_t stream);
 
+// Tensor-core variant for decode shapes whose weights no thread touches (TMA unpacks the 4-bit
+// codes into the layout kind::mxf8f6f4 reads; MXFP4 and MXFP4+ weights, K % 512 == 0, M <= 64).
+bool wo_tma_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                      const mxp_packed& B);
+cudaError_t launch_gemm_wo_tma(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                               const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                               void* status, cudaStream_t stream);
+
 // Block-scaled tensor-core form: both operands packed.
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
 size_t tc_compact_workspace_bytes();  // enough for the kernels that work in place

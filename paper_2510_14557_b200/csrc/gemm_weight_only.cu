@@ -253,6 +253,16 @@ cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void*
     // and test aid).  A workspace, if given, receives the status of its bounded waits.
     const char* force = getenv("MXP_WO_KERNEL");
     const bool want_old = force != nullptr && force[0] == 'o';
+    const bool want_tma = force != nullptr && force[0] == 't';
+    if (want_tma && wo_tma_supported(M, N, K, A, lda, B)) {
+        void* status = nullptr;
+        if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {
+            status = workspace;
+            if (cudaMemsetAsync(status, 0, sizeof(StatusBlock), stream) != cudaSuccess)
+                return cudaErrorUnknown;
+        }
+        return launch_gemm_wo_tma(M, N, K, A, lda, B, D, d_dt, ldd, status, stream);
+    }
     if (!want_old && M <= 64 && wo_stream_supported(M, N, K, A, lda, B)) {
         void* status = nullptr;
         if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {

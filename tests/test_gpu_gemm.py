@@ -69,14 +69,16 @@ def test_weight_only_config3_sampled(M):
     check_gemm(d[:, torch.from_numpy(rows).cuda()], da, dw)
 
 
-@pytest.mark.parametrize("kernel", ["old", "stream"])
+@pytest.mark.parametrize("kernel", ["old", "stream", "tma"])
 @pytest.mark.parametrize("wmode", [MX, MXP, 2])
 @pytest.mark.parametrize("M,N,K", [(1, 32, 256), (3, 48, 2304), (8, 160, 4352), (9, 64, 512),
                                    (16, 2384, 4096), (40, 64, 768), (5, 77, 1024), (16, 300, 512),
-                                   (1, 19000, 512)])
+                                   (1, 19000, 512), (1, 11008, 4096), (7, 20000, 1536)])
 def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
     # shapes the streamed kernel takes (N % 16 == 0, K % 256 == 0): several 2048-element stages,
-    # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles
+    # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles; the
+    # TMA kernel takes those with K % 512 == 0 (MXFP4 / MXFP4+ weights): fewer rows than SMs,
+    # ragged last CTA, several activation tiles, more than 128 rows per CTA
     monkeypatch.setenv("MXP_WO_KERNEL", kernel)
     a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K)
     wp, dw = quantized(w_bits, wmode, bf16=True)
@@ -86,7 +88,7 @@ def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
         check_gemm(d, da, dw)
 
 
-@pytest.mark.parametrize("kernel", ["old", "stream"])
+@pytest.mark.parametrize("kernel", ["old", "stream", "tma"])
 def test_weight_only_one_hot_and_scale_spread(kernel, monkeypatch):
     # one-hot activations select single decoded weights (exact in fp32), with weight rows and
     # activation rows spread over 60 binades each, a flushed block and a zero block
