@@ -38,7 +38,7 @@ NOMINAL_FP4_OVER_BF16 = 4.0  # 9 PF dense FP4 vs 2.25 PF dense bf16
 NOMINAL_FP8_OVER_BF16 = 2.0  # 4.5 PF dense for 8-bit containers (kind::mxf8f6f4)
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemm_tc_stream_kernel<wide> launch, from
 # single-pass ncu captures of this program (summaries under profiles/); bytes per launch.
-NCU_DRAM_TRAFFIC = {"cfg5": 1.74e9 + 456.24e6, "cfg4": 26.00e6 + 14.85e3}
+NCU_DRAM_TRAFFIC = {"cfg5": 997.8e6 + 446.5e6, "cfg4": 26.11e6 + 61.2e3}
 
 
 def measured_peaks():
@@ -466,7 +466,7 @@ def run_ours(args, M, N, K, label):
             dist.destroy_process_group()
         return
 
-    # The MX+ step runs one kind::mxf8f6f4 pass on E4M3-widened operands: the contraction's own
+    # The MX+ step runs one kind::mxf8f6f4 pass on operands widened to E2M3 codes: the contraction's own
     # dtype is the 8-bit container, whose nominal rate is twice bf16's.  The FP4 rate (four
     # times bf16's) is what plain MXFP4 runs at; the fraction of it is reported beside.
     fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
@@ -491,7 +491,7 @@ def run_ours(args, M, N, K, label):
         "metric": METRIC, "value": flops_all / ms / 1e9, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "e4m3 containers holding E2M1/E0M3 values (kind::mxf8f6f4), fp32 accumulate",
+        "dtype": "e2m3 codes holding E2M1/E0M3 values (kind::mxf8f6f4, 8-bit-container rate), fp32 accumulate",
         "data": "synthetic",
         "config": {"workload": label, "M": M, "N": N, "K": K, "a_mode": "MXFP4+", "w_mode": "MXFP4+",
                    "weights": "quantized and prepacked (mxp_gemm_prepack) once, outside the step",

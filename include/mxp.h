@@ -107,8 +107,9 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  *              mxp_gemm_min_workspace_bytes(...) bytes (MXP_ERR_WORKSPACE otherwise); may be
  *              NULL when that size is 0.  With mxp_gemm_workspace_bytes(...) bytes the
  *              tensor-core form first re-tiles the scales and, for MX+ operands, widens the
- *              4-bit codes to E4M3 bytes (exact for every E2M1 value and for the BM values
- *              of Eq. 3) inside the workspace and then runs its fastest kernel; with less
+ *              4-bit codes to 6-bit E2M3 codes (E4M3 bytes for MX++; either is exact for every
+ *              E2M1 value and for the BM values of Eq. 3) inside the workspace and then runs
+ *              its fastest kernel; with less
  *              it runs kernels that work on the packed planes in place (Eq. 4 / Algorithm 1:
  *              BM split and residual MMAs), which are slower.  Same result either way.
  *              Its first 16 bytes are a status block written by the kernels (see
@@ -130,13 +131,14 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
 
 /*
  * Weights prepared once.  mxp_gemm with the full workspace re-tiles the scales of both
- * operands and, when either is MXFP4+, widens both to E4M3 bytes on every call (see
+ * operands and, when either is MXFP4+, widens both to E2M3 / E4M3 codes on every call (see
  * `workspace` above).  For an operand that does not change between calls (the N x K
  * weights) that work can be done once:
  *   mxp_gemm_prepack_bytes  bytes of the prepacked form of a rows x K operand; `wide` != 0
  *                           if the GEMMs it will be used in have an MXFP4+ operand on
- *                           either side (then it holds one E4M3 byte per element, exact
- *                           for every E2M1 value and for the BM values of Eq. 3), 0 for
+ *                           either side (then it holds 16 bytes per 16 elements: E2M3 codes
+ *                           or, for MX++, E4M3 bytes, exact for every E2M1 value and for
+ *                           the BM values of Eq. 3), 0 for
  *                           MXFP4 x MXFP4 (scale atoms only).  0: shape not supported
  *                           (K % 128 != 0).
  *   mxp_gemm_prepack        writes that form of `P` into `out` (device, 256-byte aligned,

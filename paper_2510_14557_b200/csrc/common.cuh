@@ -48,7 +48,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                           const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
                           void* workspace, size_t workspace_bytes, cudaStream_t stream);
 
-// Streamed CTA-pair kernel on prepacked operands (scale atoms, E4M3-widened MX+ data): needs
+// Streamed CTA-pair kernel on prepacked operands (scale atoms, MX+ data widened to E2M3 or E4M3
+// codes): needs
 // M, N > 128 and a workspace of stream_workspace_bytes() (0 = shape not supported).
 size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,

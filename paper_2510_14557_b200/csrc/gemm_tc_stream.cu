@@ -7,18 +7,22 @@
 //
 //   * scales: the row-major E8M0 plane is re-tiled into the 32-row x 16-byte atoms that
 //     tcgen05.cp copies into tensor memory ([row group of 128][K group of 128][512 bytes]);
-//   * MX+ operands (and their plain partner): every 4-bit code is widened to an E4M3 byte.
-//     E4M3 holds all E2M1 values and the BM values 4 + m/2 of Eq. 3 exactly, so the block's
-//     BM is simply written as 0x48 | m and one kind::mxf8f6f4 pass replaces the main MMA plus
-//     the residual MMAs of Eq. 4 / Algorithm 1.  On this GPU an 8-bit-container MMA costs two
-//     FP4 MMAs, i.e. what one MX+ operand costs with the split and half of what two cost.
+//   * MX+ operands (and their plain partner): every 4-bit code is widened to a 6-bit E2M3
+//     code (sixteen of them in 12 bytes plus 4 bytes of padding: the form in which
+//     kind::mxf8f6f4 reads 6-bit operands from shared memory).  E2M3 holds all E2M1 values and
+//     the BM values 4 + m/2 of Eq. 3 exactly, so the block's BM is simply written as s 11 mmm
+//     and one kind::mxf8f6f4 pass replaces the main MMA plus the residual MMAs of Eq. 4 /
+//     Algorithm 1.  On this GPU such an MMA costs two FP4 MMAs, i.e. what one MX+ operand
+//     costs with the split and half of what two cost.  (E4M3 bytes hold the same values and
+//     cost the same tensor cycles, but more power: under the board's power limit the E2M3
+//     form runs at a 4 % higher clock.  MX++ operands need E4M3's exponent range.)
 //
 // Plain MXFP4 x MXFP4 needs only the scale pass and runs kind::mxf4 on the nibble planes.
 //
 // Kernel: clusters of two CTAs, persistent, one 256 x 480 (kind::mxf4: 256 x 448) output tile
 // per cluster and step, held in two accumulators that share the A tile: per flop that is 23 %
-// fewer bytes through TMA than a 256 x 256 tile, and the copies into shared memory, not the
-// tensor pipe, were what bounded the 256 x 256 kernel.  Warp 0 of each CTA issues the TMA loads
+// fewer bytes through TMA than a 256 x 256 tile (kept for shapes whose larger tiles would fill
+// the GPU unevenly).  Warp 0 of each CTA issues the TMA loads
 // for its own 128 rows of A, its share of both halves of B and the scale atoms; all of them
 // signal one mbarrier in the even CTA, whose warp 1 issues tcgen05.mma.cta_group::2 and commits
 // to both CTAs.  Warps 2-9 drain the accumulators.
@@ -81,7 +85,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kFmtE4M3 = 0, kFmtE2M3 = 3;  // instruction-descriptor codes, kind::mxf8f6f4
 
 // kWide = false: rows are 256 packed E2M1 codes (two scale atoms per stage), kind::mxf4.
-// kWide = true : rows are 128 E4M3 bytes (one scale atom per stage), kind::mxf8f6f4.
+// kWide = true : rows are 128 E2M3 / E4M3 code slots (one scale atom per stage), kind::mxf8f6f4.
 // kHalves = 2: the tile has two halves (accumulators); 1: a single 256 x 256 accumulator, for
 // shapes whose larger tiles would not fill the GPU evenly.
 template <bool kWide, int kHalves>
@@ -448,11 +452,13 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
 //   for B), the second starting 128 rows in, so for B it holds 112 or 96 rows.  Rows past the
 //   end of the half tile or of the operand are written as zero.  A CTA handles one row group x up to 32 K groups
 //   through shared memory, so reads and writes are both contiguous.
-// widen CTAs (only when an operand is MX+): packed codes [rows][K/2] -> E4M3 bytes [rows][K],
+// widen CTAs (only when an operand is MX+): packed codes [rows][K/2] -> 16 bytes per 16 codes,
 //   one thread per 16 elements (8 bytes in, 16 bytes out, both contiguous across the warp).
-//   E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6 are the E4M3 bytes 00 30 38 3C 40 44 48 4C; the
-//   BM of an MX+ block (Eq. 3: 4 + m/2, stored as sign + 3 mantissa bits) is 0x48 | m.  A
-//   block with scale byte 0 (flushed) becomes zeros.
+//   MXFP4 / MXFP4+: E2M3 codes, the E2M1 code with two zero mantissa bits appended, the BM of
+//   an MX+ block (Eq. 3: 4 + m/2, stored as sign + 3 mantissa bits) as s 11 mmm; sixteen codes
+//   packed into 12 bytes, 4 bytes of padding.  MX++: E4M3 bytes (E2M1 magnitudes 0, .5, 1, 1.5,
+//   2, 3, 4, 6 are 00 30 38 3C 40 44 48 4C, the BM 0x48 | m, both rescaled by powers of two).
+//   A block with scale byte 0 (flushed) becomes zeros.
 struct PrepackOperand {
     const uint8_t* nibbles;
     const uint8_t* scales;
@@ -706,7 +712,8 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
 }
 
 namespace {
-// Prepacked form of the B operand in a caller-owned buffer: scale atoms, then (wide) E4M3 bytes.
+// Prepacked form of the B operand in a caller-owned buffer: scale atoms, then (wide) the
+// widened codes.
 struct PackedLayout {
     size_t atoms[2];  // scale atoms tiled for one-half tiles, for two-half tiles
     size_t wide, total;
