@@ -204,6 +204,9 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
         stamp->clk_begin = (unsigned long long)clock64();
         stamp->ns_begin = ptx::globaltimer_ns();
     }
+#ifdef MXP_S_GRIDSTAMP  // measurement builds: earliest begin, latest and earliest end over all CTAs
+    if (threadIdx.x == 64) atomicMin(reinterpret_cast<unsigned long long*>(stamp) + 4, ptx::globaltimer_ns());
+#endif
     // Accumulators at columns 0 and 256; scale factors in the gaps behind them.  Per K group:
     // 4 columns for A's 128 rows, 8 for each half of B.  Two halves: kind::mxf8f6f4 has one
     // group in flight (A at 240, B halves at 248 and 496); kind::mxf4 two (group g at
@@ -422,6 +425,12 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
         stamp->clk_end = (unsigned long long)clock64();
         stamp->ns_end = ptx::globaltimer_ns();
     }
+#ifdef MXP_S_GRIDSTAMP
+    if (threadIdx.x == 64) {
+        atomicMax(reinterpret_cast<unsigned long long*>(stamp) + 5, ptx::globaltimer_ns());
+        atomicMin(reinterpret_cast<unsigned long long*>(stamp) + 6, ptx::globaltimer_ns());
+    }
+#endif
     // ---------------------------------------------------------------------- teardown
     // After a timeout, copies may still be in flight into this pair's shared memory: give
     // them (bounded) time to land before the CTAs leave.  `full` of the even CTA counts both.
