@@ -20,6 +20,8 @@ import numpy as np
 MODE_MXFP4 = 0
 MODE_MXFP4_PLUS = 1
 MODE_MXFP4_PP = 2  # MX++ (Sec. 4.3)
+FMT_E2M3 = 6       # MXFP6 / MXFP6+ elements (Table "Concrete MX-compliant formats")
+FMT_E4M3 = 8       # MXFP8 / MXFP8+ elements
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "mxp_oracle.c")
@@ -56,6 +58,14 @@ def _load():
         lib.oracle_e2m1_value.restype = ctypes.c_double
         lib.oracle_bm_split.argtypes = [ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         lib.oracle_bm_split.restype = None
+        lib.oracle_elem_value.argtypes = [ci, ci]
+        lib.oracle_elem_value.restype = ctypes.c_double
+        lib.oracle_quantize_wide.argtypes = [p, ci, i64, i64, i64, ci, ci, ci, p, p, p]
+        lib.oracle_quantize_wide.restype = ci
+        lib.oracle_dequantize_wide.argtypes = [p, p, p, i64, i64, ci, ci, ci, p, i64]
+        lib.oracle_dequantize_wide.restype = ci
+        lib.oracle_pack6.argtypes = [p, i64, p]
+        lib.oracle_pack6.restype = None
         lib.oracle_set_threads.argtypes = [ci]
         lib.oracle_max_threads.restype = ci
         lib.oracle_get_threads.restype = ci
@@ -135,6 +145,62 @@ def dequantize(nib: np.ndarray, sc: np.ndarray, idx, mode: int, k: int = 32) -> 
                                    _ptr(out), cols)
     if rc != 0:
         raise ValueError("oracle_dequantize rejected its arguments")
+    return out
+
+
+def elem_value(fmt: int, code: int) -> float:
+    """Value of a magnitude code of the E2M3 (fmt 6) or E4M3 (fmt 8) element type."""
+    return float(_load().oracle_elem_value(int(fmt), int(code)))
+
+
+def quantize_wide(x: np.ndarray, fmt: int, plus: bool, k: int = 32, bf16_bits: bool = False):
+    """MXFP6(+) / MXFP8(+): returns (codes[rows, cols] one per byte, scales, bm_index)."""
+    assert x.ndim == 2
+    x = np.ascontiguousarray(x)
+    if bf16_bits:
+        assert x.dtype == np.uint16
+        kind = 1
+    elif x.dtype == np.float32:
+        kind = 0
+    elif x.dtype == np.float64:
+        kind = 2
+    else:
+        raise TypeError(x.dtype)
+    rows, cols = x.shape
+    if cols % k:
+        raise ValueError("cols must be a multiple of the block length")
+    codes = np.zeros((rows, cols), np.uint8)
+    sc = np.zeros((rows, cols // k), np.uint8)
+    idx = np.zeros((rows, cols // k), np.uint8)
+    rc = _load().oracle_quantize_wide(_ptr(x), kind, rows, cols, cols, k, fmt, int(plus),
+                                      _ptr(codes), _ptr(sc), _ptr(idx))
+    if rc != 0:
+        raise ValueError("oracle_quantize_wide rejected its arguments")
+    return codes, sc, idx
+
+
+def dequantize_wide(codes: np.ndarray, sc: np.ndarray, idx, fmt: int, plus: bool, k: int = 32) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, np.uint8)
+    sc = np.ascontiguousarray(sc, np.uint8)
+    rows, cols = codes.shape
+    if idx is None:
+        idx = np.zeros_like(sc)
+    idx = np.ascontiguousarray(idx, np.uint8)
+    out = np.empty((rows, cols), np.float64)
+    rc = _load().oracle_dequantize_wide(_ptr(codes), _ptr(sc), _ptr(idx), rows, cols, k, fmt,
+                                        int(plus), _ptr(out), cols)
+    if rc != 0:
+        raise ValueError("oracle_dequantize_wide rejected its arguments")
+    return out
+
+
+def pack6(codes: np.ndarray) -> np.ndarray:
+    """6-bit storage of a [rows, cols] code array (cols % 4 == 0): [rows, 3 cols / 4] bytes."""
+    codes = np.ascontiguousarray(codes, np.uint8)
+    rows, cols = codes.shape
+    assert cols % 4 == 0
+    out = np.zeros((rows, cols // 4 * 3), np.uint8)
+    _load().oracle_pack6(_ptr(codes), rows * cols, _ptr(out))
     return out
 
 

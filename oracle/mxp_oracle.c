@@ -11,7 +11,9 @@
  * Arithmetic is done on doubles (every bf16 / fp32 input converts exactly).
  *
  * Pinned by tests (see tests/test_oracle_*.py): element table, scale, NBM and BM
- * rounding, flush rule, layout, Eq. 4 split, decode, fp64 GEMM.
+ * rounding, flush rule, layout, Eq. 4 split, decode, fp64 GEMM; the MXFP6(+) / MXFP8(+)
+ * functions at the end of the file likewise (element tables, casts against a library cast
+ * and a closed form, BM grid, flush thresholds, 6-bit packing, round trips).
  * Parity unpinned: blocks holding Inf/NaN (the paper does not define them).
  *
  * Readings of the paper taken here (each is listed in the design notes):
@@ -280,6 +282,205 @@ void oracle_bm_split(int m, int *code_h, int *code_l)
     double l = ldexp((double)m1 + (double)m0 * 0.5, EMAX - 2);
     *code_h = e2m1_nearest(h);
     *code_l = e2m1_nearest(l);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * MXFP6 / MXFP6+ (E2M3 elements) and MXFP8 / MXFP8+ (E4M3 elements): Sec. 2 Table "Concrete
+ * MX-compliant formats", Sec. 4.1 (BM re-encoding), Sec. 4.2 (layout).  Same scheme as MXFP4+:
+ * shared_exp = floor(log2 BM) - emax with emax = 2 (E2M3) or 8 (E4M3); the BM keeps its sign
+ * bit and spends every other bit on mantissa (E0M5: 4 + m/8, m = 0..31; E0M7: 256 + 2 m,
+ * m = 0..127), its exponent being emax by construction.
+ *
+ * Readings taken here (the paper gives no worked example at these widths):
+ *   - element casts round to nearest, ties to the even code, and saturate at the largest
+ *     finite magnitude (7.5; 448: the E4M3 code S.1111.111 is NaN and never produced);
+ *   - a BM whose scaled value rounds up to 2^(emax+1) clamps to the largest m;
+ *   - flush rule with the format's own emax: floor(log2 BM) <= -127 + emax;
+ *   - codes are produced one per byte here (sign in bit 5 resp. 7); oracle_pack6 gives the
+ *     6-bit storage order: code i of a row in bits 6 i .. 6 i + 5 of the little-endian bit
+ *     stream, so four codes fill three bytes.
+ * ------------------------------------------------------------------------------------------ */
+#define ORACLE_FMT_E2M3 6
+#define ORACLE_FMT_E4M3 8
+
+static int fmt_ebits(int fmt) { return fmt == ORACLE_FMT_E2M3 ? 2 : 4; }
+static int fmt_mbits(int fmt) { return 3; (void)fmt; }
+static int fmt_bias(int fmt) { return fmt == ORACLE_FMT_E2M3 ? 1 : 7; }
+static int fmt_emax(int fmt) { return fmt == ORACLE_FMT_E2M3 ? 2 : 8; }
+/* number of finite magnitude codes: all 32 for E2M3; E4M3 loses 1111.111 (NaN) */
+static int fmt_ncodes(int fmt) { return fmt == ORACLE_FMT_E2M3 ? 32 : 127; }
+
+/* Value of a magnitude code (exponent and mantissa bits, no sign), from the definition of
+ * the type: subnormals 2^(1-bias) * 0.mmm, normals 2^(e-bias) * 1.mmm. */
+double oracle_elem_value(int fmt, int code)
+{
+    int mb = fmt_mbits(fmt);
+    int e = code >> mb;
+    int m = code & ((1 << mb) - 1);
+    (void)fmt_ebits;
+    if (e == 0)
+        return ldexp((double)m / (double)(1 << mb), 1 - fmt_bias(fmt));
+    return ldexp(1.0 + (double)m / (double)(1 << mb), e - fmt_bias(fmt));
+}
+
+/* Nearest magnitude code to r >= 0 by exhaustive search; ties go to the even code; beyond
+ * the largest finite magnitude the search returns that magnitude (saturation). */
+static int elem_nearest(int fmt, double r)
+{
+    int n = fmt_ncodes(fmt);
+    int best = 0;
+    double best_d = fabs(r - oracle_elem_value(fmt, 0));
+    for (int c = 1; c < n; ++c) {
+        double d = fabs(r - oracle_elem_value(fmt, c));
+        if (d < best_d || (d == best_d && (c & 1) == 0)) {
+            best = c;
+            best_d = d;
+        }
+    }
+    return best;
+}
+
+/* BM mantissa: v in [2^emax, 2^(emax+1)), grid 2^emax * (1 + m / 2^mb) with mb = 5 or 7. */
+static int bm_code_wide(int fmt, double v)
+{
+    int mb = fmt - 1; /* every bit but the sign */
+    double t = (ldexp(v, -fmt_emax(fmt)) - 1.0) * (double)(1 << mb); /* in [0, 2^mb) */
+    double fl = floor(t);
+    double frac = t - fl;
+    int m = (int)fl;
+    if (frac > 0.5 || (frac == 0.5 && (m & 1)))
+        m += 1;
+    if (m > (1 << mb) - 1)
+        m = (1 << mb) - 1;
+    return m;
+}
+
+/* One block of k elements -> k code bytes (sign above the magnitude code), scale, index. */
+static void quantize_block_wide(const double *x, int k, int fmt, int plus, uint8_t *codes,
+                                uint8_t *scale, uint8_t *index)
+{
+    double amax = 0.0;
+    int bm = 0, nonfinite = 0;
+    int emax = fmt_emax(fmt);
+    for (int i = 0; i < k; ++i) {
+        double a = fabs(x[i]);
+        if (!(a <= 1.79769313486231570815e+308))
+            nonfinite = 1;
+        if (a > amax) { /* Sec. 3.2: the absolute maximum, first one wins */
+            amax = a;
+            bm = i;
+        }
+    }
+    if (k < 1 || k > 32)
+        return;
+    memset(codes, 0, (size_t)k);
+    *index = 0;
+    if (nonfinite) { /* not defined by the paper */
+        *scale = 0xFF;
+        return;
+    }
+    if (amax == 0.0 || floor_log2(amax) <= -127 + emax) { /* Sec. 4.1 flush rule */
+        *scale = 0;
+        return;
+    }
+    int se = floor_log2(amax) - emax; /* Eq. 1 */
+    *scale = (uint8_t)(se + 127);
+    if (plus)
+        *index = (uint8_t)bm;
+    for (int i = 0; i < k; ++i) {
+        int code;
+        if (plus && i == bm)
+            code = bm_code_wide(fmt, ldexp(fabs(x[i]), -se));
+        else
+            code = elem_nearest(fmt, ldexp(fabs(x[i]), -se));
+        int sign = signbit(x[i]) ? 1 : 0;
+        codes[i] = (uint8_t)((sign << (fmt - 1)) | code);
+    }
+}
+
+/* src_kind as in oracle_quantize; fmt 6 (E2M3) or 8 (E4M3); codes: rows*cols bytes. */
+int oracle_quantize_wide(const void *src, int src_kind, int64_t rows, int64_t cols,
+                         int64_t ld_src, int k, int fmt, int plus, uint8_t *codes,
+                         uint8_t *scales, uint8_t *bm_index)
+{
+    if (k < 1 || k > 32 || cols % k != 0 || rows < 0 || cols < 0)
+        return -1;
+    if (fmt != ORACLE_FMT_E2M3 && fmt != ORACLE_FMT_E4M3)
+        return -1;
+    int64_t bpr = cols / k;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+#endif
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < bpr; ++b) {
+            double x[32];
+            for (int i = 0; i < k; ++i) {
+                int64_t off = r * ld_src + b * k + i;
+                if (src_kind == 0)
+                    x[i] = (double)((const float *)src)[off];
+                else if (src_kind == 1)
+                    x[i] = bf16_to_double(((const uint16_t *)src)[off]);
+                else
+                    x[i] = ((const double *)src)[off];
+            }
+            quantize_block_wide(x, k, fmt, plus, codes + r * cols + b * k, scales + r * bpr + b,
+                                bm_index + r * bpr + b);
+        }
+    }
+    return 0;
+}
+
+/* Eq. 3 at the wider formats.  Scale byte 0 -> zeros; 0xFF -> NaN (unpinned). */
+int oracle_dequantize_wide(const uint8_t *codes, const uint8_t *scales, const uint8_t *bm_index,
+                           int64_t rows, int64_t cols, int k, int fmt, int plus, double *dst,
+                           int64_t ld_dst)
+{
+    if (k < 1 || k > 32 || cols % k != 0)
+        return -1;
+    if (fmt != ORACLE_FMT_E2M3 && fmt != ORACLE_FMT_E4M3)
+        return -1;
+    int64_t bpr = cols / k;
+    int mb = fmt - 1;
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < bpr; ++b) {
+            int sb = scales[r * bpr + b];
+            int bm = plus ? (bm_index[r * bpr + b] & 31) : -1;
+            for (int i = 0; i < k; ++i) {
+                int c = codes[r * cols + b * k + i];
+                int s = (c >> mb) & 1;
+                int mag = c & ((1 << mb) - 1);
+                double out;
+                if (sb == 0)
+                    out = 0.0;
+                else if (sb == 0xFF)
+                    out = NAN;
+                else {
+                    if (i == bm) /* 2^emax * 1.m with every non-sign bit as mantissa */
+                        out = ldexp(ldexp(1.0 + (double)mag / (double)(1 << mb), fmt_emax(fmt)), sb - 127);
+                    else
+                        out = ldexp(oracle_elem_value(fmt, mag), sb - 127);
+                    if (s)
+                        out = -out;
+                }
+                dst[r * ld_dst + b * k + i] = out;
+            }
+        }
+    }
+    return 0;
+}
+
+/* 6-bit storage order: code i in bits 6 i .. 6 i + 5 of the little-endian bit stream.
+ * n codes (n % 4 == 0) -> 3 n / 4 bytes. */
+void oracle_pack6(const uint8_t *codes, int64_t n, uint8_t *out)
+{
+    memset(out, 0, (size_t)(n / 4 * 3));
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t bit = 6 * i;
+        unsigned v = (unsigned)(codes[i] & 63) << (bit & 7);
+        out[bit >> 3] |= (uint8_t)(v & 0xFF);
+        if ((bit & 7) > 2)
+            out[(bit >> 3) + 1] |= (uint8_t)(v >> 8);
+    }
 }
 
 /* D[m][n] = sum_k A[m][k] * B[n][k], fp64, k ascending.  A is M x K, B is N x K. */
