@@ -224,10 +224,13 @@ def part_quantize(mxp, synth, peaks, iters):
     x = dev_bf16(synth.config2())
     n = x.numel()
     for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4),
-                       ("mxfp4++", mxp.MODE_MXFP4_PP)):
+                       ("mxfp4++", mxp.MODE_MXFP4_PP), ("mxfp6+", mxp.MODE_MXFP6_PLUS),
+                       ("mxfp6", mxp.MODE_MXFP6), ("mxfp8+", mxp.MODE_MXFP8_PLUS),
+                       ("mxfp8", mxp.MODE_MXFP8)):
         buf = mxp.alloc_packed(x.shape[0], x.shape[1], mode, index_for_mxfp4=False)
         ms = time_loop(lambda: mxp.mxp_quantize(x, mode, out=buf), iters)
-        nbytes = n * (2 + 0.5 + 1 / 32 + (1 / 32 if mode != mxp.MODE_MXFP4 else 0))
+        # bf16 in; element codes, one scale byte (and one index byte) per block of 32 out
+        nbytes = n * (2 + mxp.binding.element_bits(mode) / 8 + 1 / 32 + (1 / 32 if buf.bm_index is not None else 0))
         gbs = nbytes / ms / 1e6
         out["quantize_cfg2_" + name] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
     return out

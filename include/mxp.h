@@ -54,11 +54,19 @@ typedef enum {
 typedef enum {
     MXP_MODE_MXFP4 = 0,
     MXP_MODE_MXFP4_PLUS = 1, /* MX+  (Sec. 4.1): BM with 3 mantissa bits, index byte */
-    MXP_MODE_MXFP4_PP = 2    /* MX++ (Sec. 4.3): MX+ and a finer shared exponent for the NBMs */
+    MXP_MODE_MXFP4_PP = 2,   /* MX++ (Sec. 4.3): MX+ and a finer shared exponent for the NBMs */
+    /* The same scheme at the other element widths (Table of MX formats, Sec. 4.1-4.2);
+     * mxp_quantize and mxp_dequantize only, the GEMMs return MXP_ERR_UNSUPPORTED for them. */
+    MXP_MODE_MXFP6 = 3,      /* E2M3 elements, emax 2 */
+    MXP_MODE_MXFP6_PLUS = 4, /* ... with the BM as sign + 5 mantissa bits: 4 + m/8, index byte */
+    MXP_MODE_MXFP8 = 5,      /* E4M3 elements, emax 8 */
+    MXP_MODE_MXFP8_PLUS = 6  /* ... with the BM as sign + 7 mantissa bits: 256 + 2 m, index byte */
 } mxp_mode;
 typedef enum { MXP_F32 = 0, MXP_BF16 = 1 } mxp_dtype;
 
-/* A packed operand: three row-major device planes. */
+/* A packed operand: three row-major device planes.  MXFP6 modes: `nibbles` holds rows * cols
+ * 6-bit codes, code i of a row in bits 6i..6i+5 of the little-endian bit stream (3/4 byte per
+ * element); MXFP8 modes: one byte per element. */
 typedef struct {
     const uint8_t *nibbles;  /* rows * cols / 2 bytes, 16-byte aligned                */
     const uint8_t *scales;   /* rows * cols / 32 bytes, E8M0                          */
@@ -76,6 +84,10 @@ typedef struct {
  *   bm_index out, rows * cols / 32 bytes; required for MXFP4+, may be NULL for MXFP4
  *            (when given in MXFP4 mode it is filled with zeros)
  * cols must be a multiple of 32.  rows == 0 or cols == 0 is a no-op returning MXP_OK.
+ * MXFP6 / MXFP8 modes: the same with emax 2 / 8 in Eq. 1 and the flush rule, E2M3 / E4M3
+ * element casts (round to nearest even, saturating at 7.5 / 448) and `nibbles` sized
+ * rows * cols * 3 / 4 resp. rows * cols bytes; in the + modes the BM is stored as its sign and
+ * 5 resp. 7 mantissa bits (scaled value 4 + m/8 resp. 256 + 2 m).
  */
 mxp_status mxp_quantize(const void *src, mxp_dtype src_dt, int64_t rows, int64_t cols,
                         int64_t ld_src, mxp_mode mode, uint8_t *nibbles, uint8_t *scales,

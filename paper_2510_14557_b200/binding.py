@@ -18,6 +18,7 @@ MXP_OK = 0
 MODE_MXFP4 = 0
 MODE_MXFP4_PLUS = 1
 MODE_MXFP4_PP = 2
+MODE_MXFP6, MODE_MXFP6_PLUS, MODE_MXFP8, MODE_MXFP8_PLUS = 3, 4, 5, 6  # quantize / dequantize only
 F32 = 0
 BF16 = 1
 
@@ -130,11 +131,15 @@ class Packed:
                        self.rows, self.cols, self.mode)
 
 
+def element_bits(mode: int) -> int:
+    return 6 if mode in (MODE_MXFP6, MODE_MXFP6_PLUS) else 8 if mode in (MODE_MXFP8, MODE_MXFP8_PLUS) else 4
+
+
 def alloc_packed(rows: int, cols: int, mode: int, device="cuda", index_for_mxfp4=False) -> Packed:
-    nib = torch.empty((rows, cols // 2), dtype=torch.uint8, device=device)
+    nib = torch.empty((rows, cols * element_bits(mode) // 8), dtype=torch.uint8, device=device)
     sc = torch.empty((rows, cols // 32), dtype=torch.uint8, device=device)
     idx = None
-    if mode != MODE_MXFP4 or index_for_mxfp4:
+    if mode not in (MODE_MXFP4, MODE_MXFP6, MODE_MXFP8) or index_for_mxfp4:
         idx = torch.empty((rows, cols // 32), dtype=torch.uint8, device=device)
     return Packed(nib, sc, idx, rows, cols, mode)
 

@@ -7,9 +7,17 @@ namespace {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// modes every entry point takes: the 4-bit ones
 bool valid_mode(int m)
 {
     return m == MXP_MODE_MXFP4 || m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP;
+}
+// 6- and 8-bit element modes: quantize and decode only
+bool wide_mode(int m) { return m >= MXP_MODE_MXFP6 && m <= MXP_MODE_MXFP8_PLUS; }
+bool plus_mode(int m)
+{
+    return m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP || m == MXP_MODE_MXFP6_PLUS ||
+           m == MXP_MODE_MXFP8_PLUS;
 }
 bool valid_dtype(int d) { return d == MXP_F32 || d == MXP_BF16; }
 
@@ -49,14 +57,19 @@ mxp_status mxp_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t
                         int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
                         uint8_t* bm_index, void* cuda_stream)
 {
-    if (!valid_mode(mode) || !valid_dtype(src_dt)) return MXP_ERR_INVALID_ARG;
+    if ((!valid_mode(mode) && !wide_mode(mode)) || !valid_dtype(src_dt)) return MXP_ERR_INVALID_ARG;
     if (rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return MXP_OK;
     if (src == nullptr || nibbles == nullptr || scales == nullptr) return MXP_ERR_INVALID_ARG;
-    if (mode != MXP_MODE_MXFP4 && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (plus_mode(mode) && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
     if (ld_src < cols || ld_src % 8 != 0) return MXP_ERR_INVALID_ARG;
     if (!aligned(src, 16) || !aligned(nibbles, 16)) return MXP_ERR_INVALID_ARG;
     if (rows * (cols / 32) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    if (wide_mode(mode))
+        return mxp::launch_quantize_wide(src, src_dt, rows, cols, ld_src, mode, nibbles, scales,
+                                         bm_index, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+                   ? MXP_OK
+                   : MXP_ERR_CUDA;
     cudaError_t e = mxp::launch_quantize(src, src_dt, rows, cols, ld_src, mode, nibbles, scales,
                                          bm_index, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
@@ -65,6 +78,17 @@ mxp_status mxp_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t
 mxp_status mxp_dequantize(const mxp_packed* p, void* dst, mxp_dtype dst_dt, int64_t ld_dst,
                           void* cuda_stream)
 {
+    if (p != nullptr && wide_mode(p->mode)) {
+        if (p->rows < 0 || p->cols < 0 || p->cols % 32 != 0 || !valid_dtype(dst_dt)) return MXP_ERR_INVALID_ARG;
+        if (p->rows == 0 || p->cols == 0) return MXP_OK;
+        if (p->nibbles == nullptr || p->scales == nullptr || !aligned(p->nibbles, 16)) return MXP_ERR_INVALID_ARG;
+        if (plus_mode(p->mode) && p->bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+        if (dst == nullptr || !aligned(dst, 16) || ld_dst < p->cols || ld_dst % 8 != 0) return MXP_ERR_INVALID_ARG;
+        if (p->rows * (p->cols / 32) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+        return mxp::launch_dequantize_wide(*p, dst, dst_dt, ld_dst, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+                   ? MXP_OK
+                   : MXP_ERR_CUDA;
+    }
     if (!valid_packed(p) || !valid_dtype(dst_dt)) return MXP_ERR_INVALID_ARG;
     if (p->rows == 0 || p->cols == 0) return MXP_OK;
     if (dst == nullptr || !aligned(dst, 16)) return MXP_ERR_INVALID_ARG;

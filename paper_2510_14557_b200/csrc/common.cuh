@@ -33,6 +33,13 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
                                   const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
                                   void* status, cudaStream_t stream);
 
+// MXFP6(+) / MXFP8(+): quantize and decode only (quantize_wide.cu).
+cudaError_t launch_quantize_wide(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                                 int64_t ld_src, mxp_mode mode, uint8_t* codes, uint8_t* scales,
+                                 uint8_t* bm_index, cudaStream_t stream);
+cudaError_t launch_dequantize_wide(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
+                                   cudaStream_t stream);
+
 // Tensor-core variant for decode shapes whose weights no thread touches (TMA unpacks the 4-bit
 // codes into the layout kind::mxf8f6f4 reads; MXFP4 and MXFP4+ weights, K % 512 == 0, M <= 64).
 bool wo_tma_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,

@@ -45,7 +45,8 @@ def test_argument_validation_without_launch(lib):
     assert q(fake, 1, 4, 48, 48, 1, fake, fake, fake, null) == 1      # cols % 32
     assert q(fake, 1, 4, 64, 64, 1, fake, fake, null, null) == 1      # MX+ needs an index plane
     assert q(fake, 7, 4, 64, 64, 1, fake, fake, fake, null) == 1      # bad dtype
-    assert q(fake, 1, 4, 64, 64, 5, fake, fake, fake, null) == 1      # bad mode
+    assert q(fake, 1, 4, 64, 64, 9, fake, fake, fake, null) == 1      # bad mode
+    assert q(fake, 1, 4, 64, 64, 6, fake, fake, null, null) == 1      # MXFP8+ needs an index plane
     assert q(fake, 1, 4, 64, 60, 1, fake, fake, fake, null) == 1      # ld < cols
     assert q(ctypes.c_void_p(4100), 1, 4, 64, 64, 1, fake, fake, fake, null) == 1  # misaligned
     assert q(null, 1, 0, 64, 64, 1, null, null, null, null) == 0      # empty is a no-op
