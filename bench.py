@@ -342,6 +342,29 @@ def part_prefill(mxp, synth, peaks, iters):
                 "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
                 "frac_fp4_nominal_9PF": tf / 9000.0}
             del pa, pw
+            # MXFP6 / MXFP6+ operands (E2M3 elements; an MXFP6+ operand costs a second pass)
+            for an, am, bn, bm in (("mxfp6", mxp.MODE_MXFP6, "mxfp6", mxp.MODE_MXFP6),
+                                   ("mxfp6+", mxp.MODE_MXFP6_PLUS, "mxfp6", mxp.MODE_MXFP6),
+                                   ("mxfp6+", mxp.MODE_MXFP6_PLUS, "mxfp4", mxp.MODE_MXFP4)):
+                ws6 = torch.zeros(mxp.mxp_gemm_workspace_bytes(M, N, K, False, am, bm),
+                                  dtype=torch.uint8, device="cuda")
+                pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
+                tot = 0.0
+                for i in range(n_it + 2):
+                    flush.fill_(i & 255)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    mxp.mxp_gemm(pa, pw, out=d, workspace=ws6)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if i >= 2:
+                        tot += e0.elapsed_time(e1)
+                ms = tot / n_it
+                tf = 2.0 * M * N * K / ms / 1e9
+                out["prefill_cfg5_A-%s_W-%s" % (an, bn)] = {
+                    "us": ms * 1e3, "TFLOP/s": tf, "frac_fp4_peak_4x_bf16_burst": tf / fp4_burst,
+                    "frac_fp4_nominal_9PF": tf / 9000.0}
+                del pa, pw, ws6
         del a, w, d, ws
         torch.cuda.empty_cache()
     return out

@@ -21,16 +21,18 @@ bool plus_mode(int m)
 }
 bool valid_dtype(int d) { return d == MXP_F32 || d == MXP_BF16; }
 
-// Checks an operand descriptor (host struct, device planes).
-bool valid_packed(const mxp_packed* p)
+// Checks an operand descriptor (host struct, device planes).  `six_ok`: the caller also takes
+// MXFP6 / MXFP6+ operands (the packed x packed GEMM does).
+bool valid_packed(const mxp_packed* p, bool six_ok = false)
 {
     if (p == nullptr) return false;
-    if (!valid_mode(p->mode)) return false;
+    const bool six = p->mode == MXP_MODE_MXFP6 || p->mode == MXP_MODE_MXFP6_PLUS;
+    if (!valid_mode(p->mode) && !(six_ok && six)) return false;
     if (p->rows < 0 || p->cols < 0 || p->cols % 32 != 0) return false;
     if (p->rows == 0 || p->cols == 0) return true;
     if (p->nibbles == nullptr || p->scales == nullptr) return false;
     if (!aligned(p->nibbles, 16)) return false;
-    if (p->mode != MXP_MODE_MXFP4 && p->bm_index == nullptr) return false;
+    if (plus_mode(p->mode) && p->bm_index == nullptr) return false;
     return true;
 }
 
@@ -123,10 +125,10 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
     if ((A_dense_bf16 == nullptr) == (A_packed == nullptr)) return MXP_ERR_INVALID_ARG;
-    if (!valid_packed(B_packed)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(B_packed, A_packed != nullptr)) return MXP_ERR_INVALID_ARG;
     if (B_packed->rows != N || B_packed->cols != K) return MXP_ERR_INVALID_ARG;
     if (A_packed != nullptr) {
-        if (!valid_packed(A_packed)) return MXP_ERR_INVALID_ARG;
+        if (!valid_packed(A_packed, true)) return MXP_ERR_INVALID_ARG;
         if (A_packed->rows != M || A_packed->cols != K) return MXP_ERR_INVALID_ARG;
     } else {
         if (lda < K || lda % 8 != 0 || !aligned(A_dense_bf16, 16)) return MXP_ERR_INVALID_ARG;

@@ -1241,7 +1241,7 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
         return launch_gemm_tc_stream(M, N, K, A, B, nullptr, D, d_dt, ldd, workspace, workspace_bytes,
                                      stream);
     // the in-place kernels implement Eq. 4 for MXFP4+ only: an MX++ operand needs the prepacked path
-    if (A.mode == MXP_MODE_MXFP4_PP || B.mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;
+    if (A.mode > MXP_MODE_MXFP4_PLUS || B.mode > MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
     // status block and clock stamp (these kernels leave no stamp)
     if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return MXP_ERR_CUDA;
     bool use_pair = M > 128 && N > 128 && (ap || bp);

@@ -107,6 +107,10 @@ struct SCfg {
 struct SParams {
     int M, N, K;
     uint32_t a_fmt, b_fmt;  // kind::mxf8f6f4 operand formats (kFmtE2M3 / kFmtE4M3); wide only
+    // An MXFP6+ operand is the sum of two E2M3 planes (its BM does not fit one E2M3 code):
+    // plane p of A starts at row p * M of its widened copy (B: p * N), and the K loop runs once
+    // per pair of planes: D = sum over (pa, pb) of A_pa * B_pb^T, same scales in every pass.
+    int parts_a, parts_b;
     void* D;
     int64_t ldd;
     int d_vec_ok;
@@ -169,7 +173,8 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
-    const int kstages = (prm.K + C::kElemsPerStage - 1) / C::kElemsPerStage;
+    const int kbase = (prm.K + C::kElemsPerStage - 1) / C::kElemsPerStage;  // stages of one pass
+    const int kstages = kbase * prm.parts_a * prm.parts_b;
     const int tiles_m = (prm.M + kTileM - 1) / kTileM;
     const int tiles_n = (prm.N + C::kTileN - 1) / C::kTileN;
     const int num_tiles = tiles_m * tiles_n;
@@ -235,9 +240,18 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 tile_coords(tile, tiles_m, tiles_n, tm, tn);
                 const int m0 = tm * kTileM + 128 * (int)rank;
                 const int n0 = tn * C::kTileN + C::kBRows * (int)rank;
+                int kk = 0, pa = 0, pb = 0;  // stage within the pass, plane of A, plane of B
                 for (int kt = 0; kt < kstages; ++kt, ++c) {
                     const int s = c % S;
                     const uint32_t use = c / S;
+                    const int ka = kk, ya = pa * prm.M, yb = pb * prm.N;
+                    if (++kk == kbase) {
+                        kk = 0;
+                        if (++pb == prm.parts_b) {
+                            pb = 0;
+                            ++pa;
+                        }
+                    }
                     if (use > 0 && !ptx::mbar_wait(&empty[s], (use - 1) & 1, abort, kWaitLimit)) {
                         give_up(abort, prm.status, 0x2100 + s);
                         ok = false;
@@ -248,13 +262,13 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     continue;
 #endif
                     if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * C::kStageRaw);
-                    ptx::tma_load_2d_pair(a_tile(s), &tmap_a, full0 + 8u * (uint32_t)s, kt * kRowBytes, m0);
+                    ptx::tma_load_2d_pair(a_tile(s), &tmap_a, full0 + 8u * (uint32_t)s, ka * kRowBytes, ya + m0);
 #pragma unroll
                     for (int j = 0; j < kHalves; ++j)
                         ptx::tma_load_2d_pair(b_tile(s, j), &tmap_b, full0 + 8u * (uint32_t)s,
-                                              kt * kRowBytes, n0 + j * C::kSubN);
-                    ptx::tma_load_3d_pair(sfa(s), &tmap_sfa, full0 + 8u * (uint32_t)s, 0, kt * G, 2 * tm + (int)rank);
-                    ptx::tma_load_3d_pair(sfb(s), &tmap_sfb, full0 + 8u * (uint32_t)s, 0, kt * G,
+                                              ka * kRowBytes, yb + n0 + j * C::kSubN);
+                    ptx::tma_load_3d_pair(sfa(s), &tmap_sfa, full0 + 8u * (uint32_t)s, 0, ka * G, 2 * tm + (int)rank);
+                    ptx::tma_load_3d_pair(sfb(s), &tmap_sfb, full0 + 8u * (uint32_t)s, 0, ka * G,
                                           2 * kHalves * tn);
                 }
             }
@@ -290,7 +304,7 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     const uint64_t d_sfa = ptx::smem_desc_sf(ptx::smem_u32(sfa(s)));
                     const uint64_t d_sfb = ptx::smem_desc_sf(ptx::smem_u32(sfb(s)));
                     const int groups =
-                        kWide ? 1 : ((prm.K - kt * C::kElemsPerStage) >= C::kElemsPerStage ? 2 : 1);
+                        kWide ? 1 : ((prm.K - (kt % kbase) * C::kElemsPerStage) >= C::kElemsPerStage ? 2 : 1);
                     if (ptx::elect_one()) {
 #ifdef MXP_EXP_NOMMA
                         for (int g = 0; g < 0; ++g) {
@@ -477,6 +491,8 @@ struct PrepackOperand {
     int rows, nbk;
     int tile_rows;            // rows per accumulator: kTileM for A, sub_n() for B
     int pp;                   // MX++ operand: index bits 7:5 hold delta (Sec. 4.3)
+    int six;                  // source codes are packed 6-bit E2M3 (MXFP6 / MXFP6+), not nibbles
+    size_t plane_bytes;       // MXFP6+: distance to the second plane of the widened copy, else 0
     unsigned scale_ctas;      // row groups * ceil(nbk/128)
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
 };
@@ -526,6 +542,54 @@ __device__ __forceinline__ uint64_t e2m1x8_to_e2m3x8(uint32_t x)
     return y << 2;
 }
 
+// Replaces the 6-bit field at bit position `bit` (< 96) of a 16-byte chunk.
+__device__ __forceinline__ void set_code6(uint4& v, uint32_t bit, uint32_t code)
+{
+    const uint32_t wi = bit >> 5, sh = bit & 31u;
+    const unsigned long long mask = 63ull << sh, val = (unsigned long long)code << sh;
+    uint32_t x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        if (wi == (uint32_t)i) {
+            x[i] = (x[i] & ~(uint32_t)mask) | (uint32_t)val;
+            x[i + 1] = (x[i + 1] & ~(uint32_t)(mask >> 32)) | (uint32_t)(val >> 32);
+        }
+    }
+    v = make_uint4(x[0], x[1], x[2], x[3]);
+}
+
+// MXFP6 / MXFP6+ operand: its sixteen 6-bit codes per half block already are E2M3 codes in the
+// bit order the tensor core reads, so they are copied into the 16-byte slot.  The BM of an
+// MXFP6+ block, 4 + m/8 with five mantissa bits, is no E2M3 value: it is entered as the sum
+// of two that are, 4 + (m >> 2)/2 in the first plane (code s 11 hhh) and (m & 3)/8 in a second
+// plane that is zero everywhere else (subnormal code s 00 0ll); the GEMM adds the products of
+// both planes (Eq. 4's split at this width, with dense residual passes).
+__device__ __forceinline__ void widen_six(const PrepackOperand& op, uint32_t t, uint32_t b)
+{
+    const uint32_t* in = reinterpret_cast<const uint32_t*>(op.nibbles) + (size_t)t * 3u;
+    uint4 o = make_uint4(in[0], in[1], in[2], 0u), lo = make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t sc = op.scales[b];
+    if (op.bm_index != nullptr) {
+        const uint32_t p = op.bm_index[b] & 31u;
+        if ((p >> 4) == (t & 1u)) {
+            const uint32_t bit = 6u * (p & 15u);
+            const uint32_t x[4] = {o.x, o.y, o.z, o.w};
+            const uint32_t wi = bit >> 5;
+            const unsigned long long win =
+                (unsigned long long)(wi == 0 ? x[0] : wi == 1 ? x[1] : x[2]) |
+                ((unsigned long long)(wi == 0 ? x[1] : wi == 1 ? x[2] : x[3]) << 32);
+            const uint32_t code = (uint32_t)(win >> (bit & 31u)) & 63u;
+            const uint32_t sign = code & 32u, m = code & 31u;
+            set_code6(o, bit, sign | 0x18u | (m >> 2));
+            set_code6(lo, bit, sign | (m & 3u));
+        }
+    }
+    if (sc == 0u) o = lo = make_uint4(0u, 0u, 0u, 0u);
+    uint8_t* dst = op.wide + (size_t)t * 16u;
+    *reinterpret_cast<uint4*>(dst) = o;
+    if (op.plane_bytes != 0) *reinterpret_cast<uint4*>(dst + op.plane_bytes) = lo;
+}
+
 // One thread per 16 elements (half a block): 8 bytes of codes in, 16 bytes out.
 //  * E2M3 (MXFP4 and MXFP4+ operands): the 16 six-bit codes packed into 12 bytes, then 4 bytes
 //    of padding, which is how kind::mxf8f6f4 reads 6-bit operands from shared memory.  The BM of
@@ -536,6 +600,7 @@ __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned i
     const uint32_t t = id * 256u + threadIdx.x;  // half block: 16 elements
     const uint32_t b = t >> 1;
     if (b >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
+    if (op.six) return widen_six(op, t, b);
     const uint2 w = reinterpret_cast<const uint2*>(op.nibbles)[t];
     const uint32_t sc = op.scales[b];
     const uint32_t ib = op.bm_index != nullptr ? op.bm_index[b] : 0u;
@@ -636,8 +701,16 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // scale row groups (atoms of 128 rows) of an operand whose output tiles take `tile_rows` rows
 inline int64_t row_groups(int64_t rows, int tile_rows) { return 2 * ((rows + tile_rows - 1) / tile_rows); }
 
+// E2M3 planes an operand is widened into: two for MXFP6+ (see widen_six), else one.
+inline int mode_parts(mxp_mode m) { return m == MXP_MODE_MXFP6_PLUS ? 2 : 1; }
+inline bool mode_six(mxp_mode m) { return m == MXP_MODE_MXFP6 || m == MXP_MODE_MXFP6_PLUS; }
+inline bool mode_plus(mxp_mode m)
+{
+    return m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP || m == MXP_MODE_MXFP6_PLUS;
+}
+
 // Sized for either tiling of B's scales (the tile shape is chosen per call).
-Layout layout(int64_t M, int64_t N, int64_t K, bool wide)
+Layout layout(int64_t M, int64_t N, int64_t K, bool wide, int parts_a = 1, int parts_b = 1)
 {
     Layout l;
     const size_t kgroups = (size_t)(K / 128);
@@ -650,10 +723,10 @@ Layout layout(int64_t M, int64_t N, int64_t K, bool wide)
     off += (size_t)std::max(row_groups(N, sub_n(wide, 1)), row_groups(N, sub_n(wide, 2))) * kgroups * kAtom;
     off = round_up(off, 1024);
     l.wa = off;
-    if (wide) off += (size_t)M * (size_t)K;
+    if (wide) off += (size_t)M * (size_t)K * (size_t)parts_a;
     off = round_up(off, 1024);
     l.wb = off;
-    if (wide) off += (size_t)N * (size_t)K;
+    if (wide) off += (size_t)N * (size_t)K * (size_t)parts_b;
     l.total = round_up(off, 1024);
     return l;
 }
@@ -710,14 +783,17 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
 {
     // Small M or N is better served by the in-place single-CTA kernel, except for MX++
     // operands, which only this path handles (rows past the end are zero-filled by TMA).
-    const bool pp = a_mode == MXP_MODE_MXFP4_PP || b_mode == MXP_MODE_MXFP4_PP;
+    // (and MXFP6 operands, likewise)
+    const bool pp = a_mode == MXP_MODE_MXFP4_PP || b_mode == MXP_MODE_MXFP4_PP ||
+                    mode_six(a_mode) || mode_six(b_mode);
     if (M < 1 || N < 1 || K % 128 != 0) return 0;
     if (!pp && (M <= 128 || N <= 128)) return 0;
     // the prepack kernel indexes half blocks (16 elements) of an operand with 32 bits
     if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
         return 0;
     const bool wide = a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4;
-    return layout(M, N, K, wide).total;
+    if (a_mode > MXP_MODE_MXFP6_PLUS || b_mode > MXP_MODE_MXFP6_PLUS) return 0;  // no MXFP8 GEMM
+    return layout(M, N, K, wide, mode_parts(a_mode), mode_parts(b_mode)).total;
 }
 
 namespace {
@@ -746,8 +822,10 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     PrepackOperand op;
     op.nibbles = P.nibbles;
     op.scales = P.scales;
-    op.bm_index = P.mode != MXP_MODE_MXFP4 ? P.bm_index : nullptr;
+    op.bm_index = mode_plus(P.mode) ? P.bm_index : nullptr;
     op.pp = P.mode == MXP_MODE_MXFP4_PP;
+    op.six = mode_six(P.mode);
+    op.plane_bytes = P.mode == MXP_MODE_MXFP6_PLUS ? (size_t)rows * (size_t)K : 0;
     op.atoms = atoms;
     op.wide = wide ? wide_bytes : nullptr;
     op.rows = (int)rows;
@@ -776,6 +854,8 @@ mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_
 {
     const size_t need = stream_prepack_bytes(P.rows, P.cols, wide);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
+    // an MXFP6+ operand needs two planes, which this form has no room for: mxp_gemm takes it
+    if (P.mode > MXP_MODE_MXFP6 || (mode_six(P.mode) && !wide)) return MXP_ERR_UNSUPPORTED;
     if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
         (reinterpret_cast<uintptr_t>(P.scales) & 3) ||
@@ -804,7 +884,10 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
 {
     const bool ap = A.mode != MXP_MODE_MXFP4, bp = B.mode != MXP_MODE_MXFP4;
     const bool wide = ap || bp;
-    const Layout l = layout(M, b_prepacked ? 0 : N, K, wide);
+    if (A.mode > MXP_MODE_MXFP6_PLUS || B.mode > MXP_MODE_MXFP6_PLUS) return MXP_ERR_UNSUPPORTED;
+    const int parts_a = mode_parts(A.mode), parts_b = mode_parts(B.mode);
+    if (b_prepacked != nullptr && parts_b != 1) return MXP_ERR_UNSUPPORTED;
+    const Layout l = layout(M, b_prepacked ? 0 : N, K, wide, parts_a, parts_b);
     if (workspace == nullptr || workspace_bytes < l.total) return MXP_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return MXP_ERR_INVALID_ARG;
     if (b_prepacked != nullptr && (reinterpret_cast<uintptr_t>(b_prepacked) & 255))
@@ -842,7 +925,8 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     CUtensorMap ta, tb, tsa, tsb;
     const int box_kg = wide ? 1 : 2;
     const bool maps_ok =
-        (wide ? make_tmap_rows(&ta, ws + l.wa, M, K, 128) && make_tmap_rows(&tb, b_wide, N, K, sub / 2)
+        (wide ? make_tmap_rows(&ta, ws + l.wa, M * parts_a, K, 128) &&
+                    make_tmap_rows(&tb, b_wide, N * parts_b, K, sub / 2)
               : make_tmap_rows(&ta, A.nibbles, M, K / 2, 128) &&
                     make_tmap_rows(&tb, B.nibbles, N, K / 2, sub / 2)) &&
         make_tmap_atoms(&tsa, ws + l.sfa, rga, kgroups, box_kg, 1) &&
@@ -855,6 +939,8 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     prm.K = (int)K;
     prm.a_fmt = A.mode == MXP_MODE_MXFP4_PP ? kFmtE4M3 : kFmtE2M3;
     prm.b_fmt = B.mode == MXP_MODE_MXFP4_PP ? kFmtE4M3 : kFmtE2M3;
+    prm.parts_a = parts_a;
+    prm.parts_b = parts_b;
     prm.D = D;
     prm.ldd = ldd;
     prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&

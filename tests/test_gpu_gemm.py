@@ -427,3 +427,83 @@ def test_bounded_wait_reports_timeout_and_leaves_the_device_usable():
     assert m.mxp_gemm_status(ws2) == 0
     with pytest.raises(Exception):
         m.mxp_wait_selftest(ws, 0)                # limit out of range: rejected, nothing launched
+
+
+# ------------------------------------------------------------------ MXFP6 / MXFP6+ operands
+MX6, MX6P = 3, 4
+
+
+def _raw_operand6(rows, K, plus, seed, scale_lo=118, scale_hi=136):
+    """MXFP6(+) planes filled directly: every E2M3 code, BM position and five-bit BM mantissa."""
+    g = synth.rng(seed)
+    codes = g.integers(0, 64, (rows, K), dtype=np.uint8)
+    sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
+    idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8) if plus else None
+    dec = oracle.dequantize_wide(codes, sc, idx, oracle.FMT_E2M3, plus)
+    from paper_2510_14557_b200 import Packed
+    p = Packed(to_dev(oracle.pack6(codes)), to_dev(sc), to_dev(idx) if plus else None, rows, K,
+               MX6P if plus else MX6)
+    return p, dec
+
+
+def _any_operand(rows, K, mode, seed):
+    if mode in (MX6, MX6P):
+        return _raw_operand6(rows, K, mode == MX6P, seed)
+    return _raw_operand(rows, K, mode, seed)
+
+
+@pytest.mark.parametrize("amode,bmode", [(MX6, MX6), (MX6P, MX6), (MX6, MX6P), (MX6P, MX6P),
+                                         (MX6P, MX), (MX6P, MXP), (MXP, MX6P), (MX6P, MXPP), (MX, MX6)])
+@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 129, 384), (64, 100, 256), (513, 1000, 128)])
+def test_tc_mxfp6_operands(M, N, K, amode, bmode):
+    # E2M3 elements go to the tensor core as they are; the BM of an MXFP6+ block enters as the
+    # sum of two E2M3 values in two planes, and the K loop runs once per pair of planes
+    ap, da = _any_operand(M, K, amode, seed=M + 3)
+    bp, db = _any_operand(N, K, bmode, seed=N + 4)
+    m = mxp()
+    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode), dtype=torch.uint8, device="cuda")
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm(ap, bp, out_dtype=dt, workspace=ws)
+        assert m.mxp_gemm_status(ws) == 0
+        check_gemm(d, da, db)
+
+
+@pytest.mark.parametrize("amode", [MX6, MX6P])
+def test_tc_mxfp6_identity_partner_returns_the_decode(amode):
+    # B = identity: D must equal the oracle's decode of A bit for bit, for every E2M3 code, BM
+    # position and BM mantissa (the two planes of a BM add up exactly)
+    M, K = 384, 256
+    ap, da = _raw_operand6(M, K, amode == MX6P, seed=23)
+    eye = np.eye(K, dtype=np.float32)
+    for bmode in (MX, MX6P):
+        if bmode == MX:
+            bp, db = quantized(eye, MX)
+        else:
+            codes, sc, idx = oracle.quantize_wide(eye, oracle.FMT_E2M3, True)
+            db = oracle.dequantize_wide(codes, sc, idx, oracle.FMT_E2M3, True)
+            from paper_2510_14557_b200 import Packed
+            bp = Packed(to_dev(oracle.pack6(codes)), to_dev(sc), to_dev(idx), K, K, MX6P)
+        assert np.array_equal(db, eye.astype(np.float64))
+        d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
+        assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
+
+
+def test_tc_mxfp6_quantized_end_to_end_and_rejections():
+    from paper_2510_14557_b200 import MxpError
+    m = mxp()
+    a = synth.activations_normal(320, 512, seed=31, outlier_frac=0.02)
+    w = synth.weights(384, 512, seed=32)
+    pa = m.mxp_quantize(to_dev(a), MX6P)
+    pw = m.mxp_quantize(to_dev(w), MX6)
+    ca, sa, ia = oracle.quantize_wide(a, oracle.FMT_E2M3, True)
+    cw, sw, iw = oracle.quantize_wide(w, oracle.FMT_E2M3, False)
+    da = oracle.dequantize_wide(ca, sa, ia, oracle.FMT_E2M3, True)
+    dw = oracle.dequantize_wide(cw, sw, None, oracle.FMT_E2M3, False)
+    check_gemm(m.mxp_gemm(pa, pw, out_dtype=torch.float32), da, dw)
+    with pytest.raises(MxpError):   # the in-place kernels (minimum workspace) are 4-bit only
+        m.mxp_gemm(pa, pw, workspace=torch.zeros(4096, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(MxpError):   # no weight-only form for 6-bit weights
+        m.mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), pw)
+    p8 = m.mxp_quantize(to_dev(a), 6)
+    with pytest.raises(MxpError):   # MXFP8 operands: quantize and decode only
+        m.mxp_gemm(p8, p8)

@@ -141,14 +141,15 @@ def test_dequantize_bit_exact(mode, dtype):
     assert np.array_equal(np.signbit(got), np.signbit(ref))
 
 
-def test_wide_modes_are_rejected_by_the_gemms():
+def test_unsupported_uses_of_the_wide_modes_are_rejected():
     from paper_2510_14557_b200 import MxpError
     m = mxp()
     a = torch.randn(256, 256, device="cuda", dtype=torch.bfloat16)
     p6 = m.mxp_quantize(a, 4)
-    with pytest.raises(MxpError):
+    p8 = m.mxp_quantize(a, 6)
+    with pytest.raises(MxpError):  # weight-only form: 4-bit weights only
         m.mxp_gemm(a, p6)
-    with pytest.raises(MxpError):
-        m.mxp_gemm(p6, p6)
+    with pytest.raises(MxpError):  # MXFP8 operands: quantize and decode only
+        m.mxp_gemm(p8, p8)
     with pytest.raises(MxpError):  # the + modes need the index plane
-        m.mxp_quantize(a, 6, out=m.Packed(p6.nibbles, p6.scales, None, 256, 256, 6))
+        m.mxp_quantize(a, 6, out=m.Packed(p8.nibbles, p8.scales, None, 256, 256, 6))
