@@ -176,6 +176,31 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed 
                               size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Quantization fused with the preparation of the GEMM operand (Sec. 5, software integration:
+ * the activations are quantized right before the matrix multiply that consumes them).
+ *   mxp_quantize_gemm_ready  mxp_quantize of an M x K bf16 matrix with contiguous rows
+ *                            (ld_src == K; MXFP4 or MXFP4+; anything else MXP_ERR_UNSUPPORTED)
+ *                            that also writes, into `workspace`, the operand in the form the
+ *                            streamed tensor-core kernel reads (what mxp_gemm_prepacked would
+ *                            otherwise derive from the packed planes in a launch of its own)
+ *                            and clears the workspace's status block.  `workspace`: device,
+ *                            256-byte aligned, at least mxp_gemm_workspace_bytes(M, N, K, 0,
+ *                            mode, b_mode) bytes for the GEMM it will serve; M > 128,
+ *                            K % 128 == 0.
+ *   mxp_gemm_ready           mxp_gemm_prepacked for an A prepared that way in the same
+ *                            `workspace` (nothing may have written to it in between) and a B
+ *                            prepacked with wide != 0: one launch.  Same result as mxp_gemm.
+ */
+mxp_status mxp_quantize_gemm_ready(const void *src, mxp_dtype src_dt, int64_t M, int64_t K,
+                                   int64_t ld_src, mxp_mode mode, uint8_t *nibbles,
+                                   uint8_t *scales, uint8_t *bm_index, void *workspace,
+                                   size_t workspace_bytes, void *cuda_stream);
+mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
+                          const mxp_packed *B_packed, const void *B_prepacked, void *D,
+                          mxp_dtype d_dt, int64_t ldd, void *workspace, size_t workspace_bytes,
+                          void *cuda_stream);
+
+/*
  * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM
  * left in `workspace`: MXP_OK, or MXP_ERR_TIMEOUT if a bounded wait inside a kernel gave
  * up (the output is then undefined but the context stays usable).

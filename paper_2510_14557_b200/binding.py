@@ -27,6 +27,7 @@ LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
 EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
+           "mxp_quantize_gemm_ready", "mxp_gemm_ready",
            "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_prepacked.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
                                          vp, vp, ci, i64, vp, sz, vp]
         l.mxp_gemm_prepacked.restype = ci
+        l.mxp_gemm_ready.argtypes = l.mxp_gemm_prepacked.argtypes
+        l.mxp_gemm_ready.restype = ci
+        l.mxp_quantize_gemm_ready.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, vp, sz, vp]
+        l.mxp_quantize_gemm_ready.restype = ci
         l.mxp_wait_selftest.argtypes = [vp, sz, i64, vp]
         l.mxp_wait_selftest.restype = ci
         l.mxp_gemm_status.argtypes = [vp, vp]
@@ -231,6 +236,35 @@ def mxp_gemm_prepacked(a: Packed, b: Packed, b_prepacked: torch.Tensor, out_dtyp
                                   out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
                                   workspace.numel(), _stream())
     _check("mxp_gemm_prepacked", st)
+    return out
+
+
+def mxp_quantize_gemm_ready(src: torch.Tensor, mode: int, workspace: torch.Tensor,
+                            out: Optional[Packed] = None) -> Packed:
+    """mxp_quantize that also writes A's GEMM-ready form into `workspace` (see include/mxp.h)."""
+    assert src.is_cuda and src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    if out is None:
+        out = alloc_packed(rows, cols, mode, src.device)
+    st = lib().mxp_quantize_gemm_ready(src.data_ptr(), _dt(src), rows, cols, src.stride(0), mode,
+                                       out.nibbles.data_ptr(), out.scales.data_ptr(),
+                                       out.bm_index.data_ptr() if out.bm_index is not None else None,
+                                       workspace.data_ptr(), workspace.numel(), _stream())
+    _check("mxp_quantize_gemm_ready", st)
+    return out
+
+
+def mxp_gemm_ready(a: Packed, b: Packed, b_prepacked: torch.Tensor, workspace: torch.Tensor,
+                   out_dtype=torch.bfloat16, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """D = dec(A) @ dec(B).T, A prepared in `workspace` by mxp_quantize_gemm_ready."""
+    M, N, K = a.rows, b.rows, b.cols
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=b.nibbles.device)
+    as_, bs = a.c_struct(), b.c_struct()
+    st = lib().mxp_gemm_ready(M, N, K, ctypes.byref(as_), ctypes.byref(bs), b_prepacked.data_ptr(),
+                              out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
+                              workspace.numel(), _stream())
+    _check("mxp_gemm_ready", st)
     return out
 
 

@@ -191,6 +191,53 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
                                       static_cast<cudaStream_t>(cuda_stream));
 }
 
+mxp_status mxp_quantize_gemm_ready(const void* src, mxp_dtype src_dt, int64_t M, int64_t K,
+                                   int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
+                                   uint8_t* bm_index, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream)
+{
+    if (mode != MXP_MODE_MXFP4 && mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
+    if (!valid_dtype(src_dt) || M <= 0 || K <= 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (src == nullptr || nibbles == nullptr || scales == nullptr) return MXP_ERR_INVALID_ARG;
+    if (mode != MXP_MODE_MXFP4 && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (!aligned(src, 16) || !aligned(nibbles, 16)) return MXP_ERR_INVALID_ARG;
+    if (src_dt != MXP_BF16 || ld_src != K) return MXP_ERR_UNSUPPORTED;  // the fused kernel's case
+    size_t atoms = 0, slots = 0, total = 0;
+    if (!mxp::stream_a_ready_layout(M, K, &atoms, &slots, &total)) return MXP_ERR_UNSUPPORTED;
+    if (workspace == nullptr || workspace_bytes < total) return MXP_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaError_t e = mxp::launch_quantize_ready(src, M, K, mode, nibbles, scales, bm_index, ws + atoms,
+                                               ws + slots, workspace,
+                                               static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed* A_packed,
+                          const mxp_packed* B_packed, const void* B_prepacked, void* D,
+                          mxp_dtype d_dt, int64_t ldd, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream)
+{
+    if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(A_packed) || !valid_packed(B_packed)) return MXP_ERR_INVALID_ARG;
+    if (A_packed->rows != M || A_packed->cols != K || B_packed->rows != N || B_packed->cols != K)
+        return MXP_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return MXP_OK;
+    if (K == 0) return MXP_ERR_UNSUPPORTED;
+    if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
+    if (!aligned(B_packed->scales, 4)) return MXP_ERR_INVALID_ARG;
+    size_t atoms = 0, slots = 0, total = 0;
+    if (!mxp::stream_a_ready_layout(M, K, &atoms, &slots, &total) || N <= 128)
+        return MXP_ERR_UNSUPPORTED;
+    if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)
+        return MXP_ERR_UNSUPPORTED;
+    return mxp::launch_gemm_tc_stream(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
+                                      workspace, workspace_bytes,
+                                      static_cast<cudaStream_t>(cuda_stream), true);
+}
+
 mxp_status mxp_wait_selftest(void* workspace, size_t workspace_bytes, int64_t limit_cycles,
                              void* cuda_stream)
 {

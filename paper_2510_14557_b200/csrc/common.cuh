@@ -62,7 +62,14 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                                  const mxp_packed& B, const void* b_prepacked, void* D,
                                  mxp_dtype d_dt, int64_t ldd, void* workspace,
-                                 size_t workspace_bytes, cudaStream_t stream);
+                                 size_t workspace_bytes, cudaStream_t stream, bool a_ready = false);
+// Quantizer that also writes A in the form that kernel reads (with a prepacked B no prepack
+// launch is left): offsets inside the GEMM's workspace, and the launch (bf16, contiguous rows,
+// MXFP4 / MXFP4+).
+bool stream_a_ready_layout(int64_t M, int64_t K, size_t* atoms, size_t* slots, size_t* total);
+cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, mxp_mode mode,
+                                  uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
+                                  uint8_t* atoms, uint8_t* slots, void* status, cudaStream_t stream);
 // One operand in the form that kernel reads (scale atoms; E4M3 bytes when `wide`), written
 // once, e.g. for weights.  stream_prepack_bytes() == 0: shape not supported.
 size_t stream_prepack_bytes(int64_t rows, int64_t K, bool wide);

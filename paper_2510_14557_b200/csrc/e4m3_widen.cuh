@@ -1,6 +1,6 @@
-// E2M1 / MX+ / MX++ codes as E4M3 bytes: what the kernels that run kind::mxf8f6f4 on widened
-// operands share.  E4M3 holds every E2M1 value, the BM values 4 + m/2 of Eq. 3 and their
-// power-of-two multiples used for MX++ exactly.
+// E2M1 / MX+ / MX++ codes as E2M3 codes or E4M3 bytes: what the kernels that run
+// kind::mxf8f6f4 on widened operands share.  Both types hold every E2M1 value and the BM values
+// 4 + m/2 of Eq. 3 exactly; E4M3 also their power-of-two multiples used for MX++.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -55,6 +55,38 @@ __device__ __forceinline__ uint32_t e2m1x4_to_e4m3x4(uint32_t x, uint2 lut = mak
     uint32_t neg;  // PTX prmt (not the intrinsic, which defines only three selector bits)
     asm("prmt.b32 %0, %1, %1, %2;" : "=r"(neg) : "r"(0x80808080u), "r"(x));
     return mag | ((neg << 7) & 0x80808080u);
+}
+
+// Eight E2M1 codes (nibble i of x) -> eight E2M3 codes, 6 bits each, code i at bits 6i..6i+5.
+// Both formats have exponent bias 1, so the E2M3 code of an E2M1 value is its code with two
+// zero mantissa bits appended: s e e m -> s e e m 0 0.  The nibbles are spread from a pitch of
+// 4 bits to a pitch of 6 in three steps (by 8, 4 and 2 bits for bits 2, 1 and 0 of i).
+__device__ __forceinline__ uint64_t e2m1x8_to_e2m3x8(uint32_t x)
+{
+    uint64_t y = x;
+    y = (y & 0x000000000000FFFFull) | ((y & 0x00000000FFFF0000ull) << 8);
+    y = (y & 0x00000000FF0000FFull) | ((y & 0x000000FF0000FF00ull) << 4);
+    y = (y & 0x000000F00F00F00Full) | ((y & 0x00000F00F00F00F0ull) << 2);
+    return y << 2;
+}
+
+// Sixteen E2M1 codes of an MXFP4 / MXFP4+ half block (w0: codes 0-7, w1: codes 8-15) as the
+// 16-byte slot kind::mxf8f6f4 reads: sixteen E2M3 codes in 12 bytes, 4 bytes of padding.  bm_pos
+// (0..15, or >= 16 for none): that code is the BM of an MX+ block, stored as s m2 m1 m0 and
+// meaning 4 + m/2 (Eq. 3): E2M3 code s 11 mmm.
+__device__ __forceinline__ uint4 e2m1x16_to_e2m3_slot(uint32_t w0, uint32_t w1, uint32_t bm_pos)
+{
+    unsigned long long lo = e2m1x8_to_e2m3x8(w0), hi = e2m1x8_to_e2m3x8(w1);
+    if (bm_pos < 16u) {
+        const uint32_t nib = (((bm_pos & 8u) ? w1 : w0) >> ((bm_pos & 7u) * 4u)) & 15u;
+        const uint32_t sh = 6u * (bm_pos & 7u);
+        const unsigned long long code = ((nib & 8u) << 2) | 0x18u | (nib & 7u);
+        if (bm_pos & 8u)
+            hi = (hi & ~(0x3Full << sh)) | (code << sh);
+        else
+            lo = (lo & ~(0x3Full << sh)) | (code << sh);
+    }
+    return make_uint4((uint32_t)lo, (uint32_t)(lo >> 32) | ((uint32_t)hi << 16), (uint32_t)(hi >> 16), 0u);
 }
 
 }  // namespace mxp

@@ -529,19 +529,6 @@ __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigne
     for (int i = threadIdx.x; i < nkg * 128; i += 256) dst[i] = tile[(i >> 7) * 129 + (i & 127)];
 }
 
-// Eight E2M1 codes (nibble i of x) -> eight E2M3 codes, 6 bits each, code i at bits 6i..6i+5.
-// Both formats have exponent bias 1, so the E2M3 code of an E2M1 value is its code with two
-// zero mantissa bits appended: s e e m -> s e e m 0 0.  The nibbles are spread from a pitch of
-// 4 bits to a pitch of 6 in three steps (by 8, 4 and 2 bits for bits 2, 1 and 0 of i).
-__device__ __forceinline__ uint64_t e2m1x8_to_e2m3x8(uint32_t x)
-{
-    uint64_t y = x;
-    y = (y & 0x000000000000FFFFull) | ((y & 0x00000000FFFF0000ull) << 8);
-    y = (y & 0x00000000FF0000FFull) | ((y & 0x000000FF0000FF00ull) << 4);
-    y = (y & 0x000000F00F00F00Full) | ((y & 0x00000F00F00F00F0ull) << 2);
-    return y << 2;
-}
-
 // Replaces the 6-bit field at bit position `bit` (< 96) of a 16-byte chunk.
 __device__ __forceinline__ void set_code6(uint4& v, uint32_t bit, uint32_t code)
 {
@@ -611,15 +598,7 @@ __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned i
     const bool has_bm = op.bm_index != nullptr && (p >> 4) == (t & 1u);
     uint8_t* dst = op.wide + (size_t)t * 16u;
     if (!op.pp) {
-        uint64_t lo = e2m1x8_to_e2m3x8(w.x), hi = e2m1x8_to_e2m3x8(w.y);
-        if (has_bm) {  // Eq. 3, BM branch
-            const uint32_t sh = 6u * (e & 7u);
-            const uint64_t code = ((nib & 8u) << 2) | 0x18u | (nib & 7u);
-            uint64_t& half = (e & 8u) ? hi : lo;
-            half = (half & ~(0x3Full << sh)) | (code << sh);
-        }
-        uint4 o = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32) | ((uint32_t)hi << 16),
-                             (uint32_t)(hi >> 16), 0u);
+        uint4 o = e2m1x16_to_e2m3_slot(w.x, w.y, has_bm ? e : 16u);  // Eq. 3, BM branch included
         if (sc == 0u) o = make_uint4(0u, 0u, 0u, 0u);
         *reinterpret_cast<uint4*>(dst) = o;
         return;
@@ -875,15 +854,30 @@ mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_
     return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }
 
+// Where a quantizer that prepares A for the GEMM itself has to write inside the workspace of a
+// call with a prepacked B (mxp_quantize_gemm_ready): scale atoms and 16-byte code slots.
+bool stream_a_ready_layout(int64_t M, int64_t K, size_t* atoms, size_t* slots, size_t* total)
+{
+    if (M <= 128 || K <= 0 || K % 128 != 0 || (uint64_t)M * (uint64_t)K / 16 >= (1ull << 32)) return false;
+    const Layout l = layout(M, 0, K, true);
+    *atoms = l.sfa;
+    *slots = l.wa;
+    *total = l.total;
+    return true;
+}
+
 // `b_prepacked` (may be nullptr): B already in the form stream_prepack() writes for the same
 // `wide`; then only A is prepared here and the workspace needs no room for B.
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                                  const mxp_packed& B, const void* b_prepacked, void* D,
                                  mxp_dtype d_dt, int64_t ldd, void* workspace,
-                                 size_t workspace_bytes, cudaStream_t stream)
+                                 size_t workspace_bytes, cudaStream_t stream, bool a_ready)
 {
     const bool ap = A.mode != MXP_MODE_MXFP4, bp = B.mode != MXP_MODE_MXFP4;
-    const bool wide = ap || bp;
+    const bool wide = ap || bp || a_ready;
+    // `a_ready`: A's atoms and code slots are in the workspace already (and the status block is
+    // cleared); needs a prepacked B, so that nothing is left to prepare
+    if (a_ready && (b_prepacked == nullptr || A.mode > MXP_MODE_MXFP4_PLUS)) return MXP_ERR_UNSUPPORTED;
     if (A.mode > MXP_MODE_MXFP6_PLUS || B.mode > MXP_MODE_MXFP6_PLUS) return MXP_ERR_UNSUPPORTED;
     const int parts_a = mode_parts(A.mode), parts_b = mode_parts(B.mode);
     if (b_prepacked != nullptr && parts_b != 1) return MXP_ERR_UNSUPPORTED;
@@ -914,13 +908,16 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     const uint8_t* b_atoms =
         b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms[halves - 1] : ws + l.sfb;
     const uint8_t* b_wide = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.wide : ws + l.wb;
-    const PrepackOperand pa = prepack_operand(A, M, K, wide, kTileM, ws + l.sfa, ws + l.wa);
+    const PrepackOperand pa =
+        a_ready ? no_operand() : prepack_operand(A, M, K, wide, kTileM, ws + l.sfa, ws + l.wa);
     const PrepackOperand pb =
         b_prepacked ? no_operand() : prepack_operand(B, N, K, wide, sub, ws + l.sfb, ws + l.wb);
     const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
     if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
-    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, pb, static_cast<StatusBlock*>(workspace));
-    if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+    if (ctas != 0) {
+        prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(pa, pb, static_cast<StatusBlock*>(workspace));
+        if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+    }
 
     CUtensorMap ta, tb, tsa, tsb;
     const int box_kg = wide ? 1 : 2;

@@ -16,6 +16,7 @@
 #include <cuda_bf16.h>
 
 #include "common.cuh"
+#include "e4m3_widen.cuh"
 
 namespace mxp {
 namespace {
@@ -293,13 +294,28 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8_bf16(uint32_t p0, uint32_t p1, ui
 // 64 bytes with four 128-bit loads.  Neighbouring lanes' loads fall into the same 128-byte
 // lines, which L1 serves; nibbles leave as one 128-bit store per lane (fully coalesced) and
 // the scale / index bytes as 32 consecutive bytes per warp.
-template <int kMode>
+// What the kReady variant also writes: the operand in the form the streamed tensor-core GEMM
+// reads (Sec. 5: quantization fused with the preparation of the matrix-multiply operand), i.e.
+// what prepack_kernel would make of the packed planes: the scale byte inside its 32-row x
+// 16-byte atom and the block's 32 codes as two 16-byte slots of E2M3 codes, BM included.
+struct GemmReady {
+    uint8_t* atoms;      // [ceil(rows/128)][nbk/4][512]
+    uint4* slots;        // [rows][nbk][2]
+    int nbk;             // blocks per row
+    StatusBlock* status; // zeroed here for the GEMM that follows
+};
+
+template <int kMode, bool kReady>
 __global__ void __launch_bounds__(kThreads)
 quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
                           uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
-                          uint8_t* __restrict__ bm_index)
+                          uint8_t* __restrict__ bm_index, const GemmReady ready)
 {
     const int64_t blk = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (kReady && blk == 0 && ready.status != nullptr) {
+        ready.status->code = 0u;
+        ready.status->where = 0u;
+    }
     if (blk >= total_blocks) return;
     const uint4* p = src + blk * 4;
     uint32_t x[16];
@@ -377,6 +393,19 @@ quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
     __stcs(nibbles + blk, outv);
     scales[blk] = (uint8_t)sb;
     if (bm_index != nullptr) bm_index[blk] = (uint8_t)(dead ? 0u : (bm | (delta << 5)));
+    if (kReady) {
+        static_assert(!kReady || kMode <= 1, "GEMM-ready output: MXFP4 and MXFP4+ only");
+        const uint32_t p = (kPlus && !dead) ? bm : 32u;  // BM position, none in a dead block
+        uint4 s0 = e2m1x16_to_e2m3_slot(outv.x, outv.y, p < 16u ? p : 16u);
+        uint4 s1 = e2m1x16_to_e2m3_slot(outv.z, outv.w, (p >= 16u && p < 32u) ? p - 16u : 16u);
+        __stcs(ready.slots + 2 * blk, s0);
+        __stcs(ready.slots + 2 * blk + 1, s1);
+        const int64_t row = blk / ready.nbk;
+        const int kb = (int)(blk - row * ready.nbk);
+        const int r = (int)(row & 127);
+        ready.atoms[((row >> 7) * (ready.nbk >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)] =
+            (uint8_t)sb;
+    }
 }
 
 // ------------------------------------------------------------------------- decode (Eq. 3)
@@ -448,10 +477,10 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
     const int aligned4 = ((reinterpret_cast<uintptr_t>(scales) & 3) == 0) &&
                          ((reinterpret_cast<uintptr_t>(bm_index) & 3) == 0);
     if (ld_src == cols && sizeof(T) == 2)
-        quantize_bf16_lane_kernel<kMode>
+        quantize_bf16_lane_kernel<kMode, false>
             <<<(unsigned)((total_blocks + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
                 static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles),
-                scales, bm_index);
+                scales, bm_index, GemmReady{});
     else if (ld_src == cols)
         quantize_kernel<T, kMode, true><<<(unsigned)grid, kThreads, 0, stream>>>(
             static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales,
@@ -464,6 +493,29 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
 }
 
 }  // namespace
+
+// bf16, contiguous rows, MXFP4 / MXFP4+: quantize and write the GEMM-ready form as well.
+cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, mxp_mode mode,
+                                  uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
+                                  uint8_t* atoms, uint8_t* slots, void* status, cudaStream_t stream)
+{
+    const int64_t total_blocks = rows * (cols / 32);
+    GemmReady ready;
+    ready.atoms = atoms;
+    ready.slots = reinterpret_cast<uint4*>(slots);
+    ready.nbk = (int)(cols / 32);
+    ready.status = static_cast<StatusBlock*>(status);
+    const unsigned grid = (unsigned)((total_blocks + kThreads - 1) / kThreads);
+    if (mode == MXP_MODE_MXFP4_PLUS)
+        quantize_bf16_lane_kernel<1, true><<<grid, kThreads, 0, stream>>>(
+            static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles), scales,
+            bm_index, ready);
+    else
+        quantize_bf16_lane_kernel<0, true><<<grid, kThreads, 0, stream>>>(
+            static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles), scales,
+            bm_index, ready);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
                             int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,

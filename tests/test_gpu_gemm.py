@@ -507,3 +507,45 @@ def test_tc_mxfp6_quantized_end_to_end_and_rejections():
     p8 = m.mxp_quantize(to_dev(a), 6)
     with pytest.raises(MxpError):   # MXFP8 operands: quantize and decode only
         m.mxp_gemm(p8, p8)
+
+
+# ------------------------------------------------------------------ fused quantize -> GEMM
+@pytest.mark.parametrize("amode,bmode", [(MXP, MXP), (MXP, MX), (MX, MXP)])
+@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 1000, 384), (512, 512, 128)])
+def test_quantize_gemm_ready_matches_the_two_step_path(M, N, K, amode, bmode):
+    # the quantizer writes the packed planes (bit-exact, as mxp_quantize) and A's GEMM-ready
+    # form; the GEMM then needs no prepack launch and returns what mxp_gemm returns
+    m = mxp()
+    a_bits = synth.f32_to_bf16_bits(synth.activations_normal(M, K, seed=M + K, outlier_frac=0.02))
+    a_bits[3, 32:64] = 0                       # a zero block
+    a_bits[5, 64:96] = 0x0001                  # a flushed block
+    bp, db = _raw_operand(N, K, bmode, seed=N)
+    pre = m.mxp_gemm_prepack(bp, True)
+    ws = torch.full((m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode),), 0xA5, dtype=torch.uint8, device="cuda")
+    pa = m.mxp_quantize_gemm_ready(to_dev_bf16(a_bits), amode, ws)
+    ref = oracle.quantize(a_bits, amode, bf16_bits=True)
+    assert np.array_equal(pa.nibbles.cpu().numpy(), ref[0])
+    assert np.array_equal(pa.scales.cpu().numpy(), ref[1])
+    if amode != MX:
+        assert np.array_equal(pa.bm_index.cpu().numpy(), ref[2])
+    da = oracle.dequantize(*ref, amode)
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm_ready(pa, bp, pre, ws, out_dtype=dt)
+        assert m.mxp_gemm_status(ws) == 0
+        check_gemm(d, da, db)
+        assert torch.equal(d, m.mxp_gemm(pa, bp, out_dtype=dt))
+
+
+def test_quantize_gemm_ready_rejections():
+    from paper_2510_14557_b200 import MxpError
+    m = mxp()
+    ws = torch.zeros(1 << 22, dtype=torch.uint8, device="cuda")
+    x = torch.randn(256, 256, device="cuda")
+    with pytest.raises(MxpError):   # fp32 source: not the fused kernel's case
+        m.mxp_quantize_gemm_ready(x, MXP, ws)
+    with pytest.raises(MxpError):   # MX++ keeps its own prepack
+        m.mxp_quantize_gemm_ready(x.bfloat16(), MXPP, ws)
+    with pytest.raises(MxpError):   # M <= 128: no streamed kernel
+        m.mxp_quantize_gemm_ready(x.bfloat16()[:64].contiguous(), MXP, ws)
+    with pytest.raises(MxpError):   # workspace too small
+        m.mxp_quantize_gemm_ready(x.bfloat16(), MXP, ws[:4096])
