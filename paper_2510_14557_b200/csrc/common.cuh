@@ -48,6 +48,14 @@ cudaError_t launch_gemm_wo_tma(int64_t M, int64_t N, int64_t K, const void* A, i
                                const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
                                void* status, cudaStream_t stream);
 
+// Tensor-core variant on the FP4 path (kind::mxf4 on the nibble plane as stored; activations as
+// base-4 digit planes; MXFP4 and MXFP4+ weights, K % 512 == 0, M <= 4).
+bool wo_fp4_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                      const mxp_packed& B);
+cudaError_t launch_gemm_wo_fp4(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                               const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
+                               void* status, cudaStream_t stream);
+
 // Block-scaled tensor-core form: both operands packed.
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
 size_t tc_compact_workspace_bytes();  // enough for the kernels that work in place

@@ -254,6 +254,16 @@ cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void*
     const char* force = getenv("MXP_WO_KERNEL");
     const bool want_old = force != nullptr && force[0] == 'o';
     const bool want_tma = force != nullptr && force[0] == 't';
+    const bool want_fp4 = force != nullptr && force[0] == 'f';
+    if (want_fp4 && wo_fp4_supported(M, N, K, A, lda, B)) {
+        void* status = nullptr;
+        if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {
+            status = workspace;
+            if (cudaMemsetAsync(status, 0, sizeof(StatusBlock), stream) != cudaSuccess)
+                return cudaErrorUnknown;
+        }
+        return launch_gemm_wo_fp4(M, N, K, A, lda, B, D, d_dt, ldd, status, stream);
+    }
     if (want_tma && wo_tma_supported(M, N, K, A, lda, B)) {
         void* status = nullptr;
         if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {

@@ -364,7 +364,11 @@ gemm_wo_tma_kernel(const __grid_constant__ CUtensorMap tmap_w,
                 break;
             }
             ptx::tc_fence_after_sync();
-            for (int st = iss; st < nst; st += kIssuers) {
+            // Stages are dealt out by their running number and the number of slots is a multiple
+            // of kIssuers: slot and issuer stay paired, an issuer sees every fill of its slots in
+            // turn, and the parity of the fill it waits for is never ambiguous.
+            const int first = (iss - (int)(c % kIssuers) + kIssuers) % kIssuers;
+            for (int st = first; st < nst; st += kIssuers) {
                 const uint32_t cc = c + (uint32_t)st;
                 const int s = cc % S;
                 const uint32_t ph = (cc / S) & 1;
@@ -389,7 +393,7 @@ gemm_wo_tma_kernel(const __grid_constant__ CUtensorMap tmap_w,
                         ptx::mma_mxf8f6f4(tmem_acc + (uint32_t)((2 * iss + (kk & 1)) * kNrows),
                                           da + (uint64_t)(2 * kk), db + (uint64_t)(2 * kk),
                                           ptx::idesc_block_scaled(kFmtE2M1, kFmtE4M3, 128, kNrows, kk, kk),
-                                          tmem_sfa, tmem_sfb, (st == iss && kk < 2) ? 0u : 1u);
+                                          tmem_sfa, tmem_sfb, (st == first && kk < 2) ? 0u : 1u);
                     ptx::tc_commit(&empty[s]);
                 }
                 __syncwarp();
@@ -447,8 +451,9 @@ gemm_wo_tma_kernel(const __grid_constant__ CUtensorMap tmap_w,
             float acc[kNrows];
 #pragma unroll
             for (int j = 0; j < kNrows; ++j) acc[j] = 0.f;
-            const int used = nst >= kIssuers ? kAcc : 2 * nst;  // issuers that had a stage
-            for (int a = 0; a < used; ++a) {
+            for (int a = 0; a < kAcc; ++a) {
+                // issuer a / 2 wrote its accumulators only if it had a stage of this tile
+                if (((a >> 1) - (int)((ti * (uint32_t)nst) % kIssuers) + kIssuers) % kIssuers >= nst) continue;
                 uint32_t r2[kNrows];
                 ptx::tmem_ld_32x16(tmem_acc + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * kNrows), r2);
                 ptx::tmem_ld_wait();
@@ -637,7 +642,8 @@ bool tma_plan(int64_t M, int64_t N, int64_t K, bool plus, int num_sms, TmaPlan* 
     const size_t per_stage = (size_t)((p->rows_per_tile + 7) / 8 * 8) * 128;
     if (fixed + 4 * per_stage + 128 * 128 > kSmemMax) return false;
     int stages = (int)((kSmemMax - fixed - 128 * 128) / per_stage);
-    p->stages = stages > kMaxStages ? kMaxStages : stages;
+    stages = stages > kMaxStages ? kMaxStages : stages;
+    p->stages = stages / kIssuers * kIssuers;  // every slot belongs to one issuer
     p->smem = tma_layout((int)K, (int)M, p->rows_per_tile, p->stages, plus).total;
     return p->smem <= kSmemMax;
 }

@@ -87,6 +87,22 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
+// The same with a pause between polls, for waits that last microseconds (an accumulator that a
+// whole tile has to fill): a warp polling without pause competes for issue slots with the
+// warps doing the work it waits for.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
+                                                  long long limit_cycles, unsigned pause_ns)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        __nanosleep(pause_ns);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort != 0u) return false;
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+}
+
 // ---------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem()
 {

@@ -69,16 +69,18 @@ def test_weight_only_config3_sampled(M):
     check_gemm(d[:, torch.from_numpy(rows).cuda()], da, dw)
 
 
-@pytest.mark.parametrize("kernel", ["old", "stream", "tma"])
+@pytest.mark.parametrize("kernel", ["old", "stream", "tma", "fp4"])
 @pytest.mark.parametrize("wmode", [MX, MXP, 2])
 @pytest.mark.parametrize("M,N,K", [(1, 32, 256), (3, 48, 2304), (8, 160, 4352), (9, 64, 512),
                                    (16, 2384, 4096), (40, 64, 768), (5, 77, 1024), (16, 300, 512),
-                                   (1, 19000, 512), (1, 11008, 4096), (7, 20000, 1536)])
+                                   (1, 19000, 512), (1, 11008, 4096), (7, 20000, 1536),
+                                   (2, 300, 512), (3, 2384, 4096), (4, 40000, 1024), (1, 64, 8192)])
 def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
     # shapes the streamed kernel takes (N % 16 == 0, K % 256 == 0): several 2048-element stages,
     # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles; the
     # TMA kernel takes those with K % 512 == 0 (MXFP4 / MXFP4+ weights): fewer rows than SMs,
-    # ragged last CTA, several activation tiles, more than 128 rows per CTA
+    # ragged last CTA, several activation tiles, more than 128 rows per CTA; the FP4-path kernel
+    # those of them with M <= 4 (every other combination falls through to the streamed kernel)
     monkeypatch.setenv("MXP_WO_KERNEL", kernel)
     a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K)
     wp, dw = quantized(w_bits, wmode, bf16=True)
@@ -88,7 +90,7 @@ def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
         check_gemm(d, da, dw)
 
 
-@pytest.mark.parametrize("kernel", ["old", "stream", "tma"])
+@pytest.mark.parametrize("kernel", ["old", "stream", "tma", "fp4"])
 def test_weight_only_one_hot_and_scale_spread(kernel, monkeypatch):
     # one-hot activations select single decoded weights (exact in fp32), with weight rows and
     # activation rows spread over 60 binades each, a flushed block and a zero block
@@ -549,3 +551,26 @@ def test_quantize_gemm_ready_rejections():
         m.mxp_quantize_gemm_ready(x.bfloat16()[:64].contiguous(), MXP, ws)
     with pytest.raises(MxpError):   # workspace too small
         m.mxp_quantize_gemm_ready(x.bfloat16(), MXP, ws[:4096])
+
+
+@pytest.mark.parametrize("kernel", ["fp4", "tma"])
+@pytest.mark.parametrize("wmode", [MX, MXP])
+def test_weight_only_tensor_paths_one_hot_rows(kernel, wmode, monkeypatch):
+    # the tensor-core decode kernels take M <= 4 (fp4) / M <= 64 (tma): one-hot activations
+    # select single decoded weights, BM or not, exactly (the BM arrives as the E2M1 misreading
+    # from the tensor core plus the correction from the CUDA cores: the sum is exact in fp32)
+    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
+    K, N = 1024, 200
+    wp, dw = _raw_operand(N, K, wmode, seed=71, scale_lo=100, scale_hi=150)
+    a = np.zeros((4, K), np.float32)
+    cols = [5, 300, 777, 1023]
+    for m, c in enumerate(cols):
+        a[m, c] = 2.0 ** (3 * m - 4)
+    m_ = mxp()
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    d = m_.mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), wp, out_dtype=torch.float32, workspace=ws)
+    assert m_.mxp_gemm_status(ws) == 0
+    got = d.cpu().numpy().astype(np.float64)
+    for m, c in enumerate(cols):
+        want = (dw[:, c] * 2.0 ** (3 * m - 4)).astype(np.float32).astype(np.float64)
+        assert np.array_equal(got[m], want)
