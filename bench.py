@@ -249,17 +249,26 @@ def part_decode(mxp, synth, peaks, iters):
         for _ in range(8):
             copies.append(mxp.mxp_quantize(w, mode))
         wbytes = 11008 * 4096 * (0.5 + 1 / 32 + (1 / 32 if mode != mxp.MODE_MXFP4 else 0))
-        for M in ((1, 8, 16) if mode != mxp.MODE_MXFP4_PP else (1,)):
+        # (M, kernel): the default kernel choice, and at M = 1 the opt-in FP4-tensor-path kernel
+        cases = [(1, None), (8, None), (16, None)] if mode != mxp.MODE_MXFP4_PP else [(1, None)]
+        if mode != mxp.MODE_MXFP4_PP:
+            cases.append((1, "fp4"))
+        for M, kern in cases:
             a = dev_bf16(a16[:M].copy())
             d = torch.empty((M, 11008), dtype=torch.bfloat16, device="cuda")
             state = {"i": 0}
+            if kern is None:
+                os.environ.pop("MXP_WO_KERNEL", None)
+            else:
+                os.environ["MXP_WO_KERNEL"] = kern   # read by the library on every call
+            key = "decode_cfg3_M%d_%s" % (M, name) + ("" if kern is None else "_kernel-" + kern)
 
             def run():
                 mxp.mxp_gemm(a, copies[state["i"] % 8], out=d)
                 state["i"] += 1
             ms = time_loop(run, iters, warmup=8)
             gbs = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms / 1e6
-            out["decode_cfg3_M%d_%s" % (M, name)] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
+            out[key] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
             if True:
                 # the same eight launches replayed from a CUDA graph: what a decode loop that
                 # captures its layers sees (less launch gap between the kernels)
@@ -274,9 +283,9 @@ def part_decode(mxp, synth, peaks, iters):
                     for _ in range(8):
                         run()
                 ms_g = time_loop(graph.replay, max(1, iters // 8), warmup=2) / 8
-                out["decode_cfg3_M%d_%s" % (M, name)]["us_cuda_graph"] = ms_g * 1e3
-                out["decode_cfg3_M%d_%s" % (M, name)]["frac_hbm_cuda_graph"] = \
-                    (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_g / 1e6 / hbm
+                out[key]["us_cuda_graph"] = ms_g * 1e3
+                out[key]["frac_hbm_cuda_graph"] = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_g / 1e6 / hbm
+        os.environ.pop("MXP_WO_KERNEL", None)
         del copies, w
     return out
 

@@ -52,7 +52,15 @@ constexpr uint32_t kTmemCols = 512;
 constexpr int kAtom = 512;
 constexpr int kMaxStages = 16;
 constexpr int kMaxGroups = 32;       // groups of two stages (16 blocks) per tile: K <= 16384
-constexpr int kMetaBufs = 4;         // such groups of scale / index bytes in flight
+// (the scale / index bytes of all groups of a tile are kept: the TMA thread never has to wait
+// for a reader of theirs, in particular not for the activation set-up to finish)
+// Activation rows per CTA: 1, 2 or 4.  The MMA's N is 16 (32 for 4): with one activation row its
+// seven digit planes fill rows 0-6 and the tile pitch is 8 rows, so the MMA's rows 8-15 are the
+// next stage's rows 0-7: finite E2M1 codes with finite scales whose accumulator columns nobody
+// reads.  The scale atoms of the activations are kept at a pitch of their kN used rows.
+__host__ __device__ constexpr int fp4_n(int ntok) { return ntok == 4 ? 32 : 16; }
+__host__ __device__ constexpr int fp4_act_pitch(int ntok) { return ntok == 1 ? 1024 : fp4_n(ntok) * 128; }
+__host__ __device__ constexpr int fp4_sfb_pitch(int ntok) { return fp4_n(ntok) * 16; }
 constexpr long long kWaitLimit = 4000000000ll;
 constexpr size_t kSmemMax = 227 * 1024;
 
@@ -73,9 +81,8 @@ struct Fp4Params {
 struct Fp4Layout {
     size_t ring, ring_stride, sfa, meta, meta_stride, act, sfb, abf, corr, bars, total;
 };
-// ntok: activation rows per CTA (2 or 4); nrows: MMA N (16 or 32)
 __host__ __device__ inline Fp4Layout fp4_layout(int K, int mrows, int rows_per_tile, int stages,
-                                                bool plus, int ntok, int nrows)
+                                                bool plus, int ntok)
 {
     Fp4Layout l;
     const size_t nst = (size_t)K / kStageK;
@@ -87,20 +94,20 @@ __host__ __device__ inline Fp4Layout fp4_layout(int K, int mrows, int rows_per_t
     l.sfa = off;  // two atoms per stage of the tile: written once per tile
     off += nst * 2 * kAtom;
     l.meta = off;
-    l.meta_stride = rows8 * 16 * 2;  // scale tile, then index tile
-    off += kMetaBufs * l.meta_stride;
+    l.meta_stride = rows8 * 16 * (plus ? 2 : 1);  // scale tile, then (MX+) index tile
+    off += (nst / 2) * l.meta_stride;
     off = (off + 1023) / 1024 * 1024;
-    l.act = off;  // [stage][nrows][128 bytes]
-    off += nst * (size_t)nrows * 128;
-    l.sfb = off;  // [stage][2 atoms]
-    off += nst * 2 * kAtom;
+    l.act = off;  // [stage][rows][128 bytes]; the last stage's MMA reads kN rows
+    off += nst * (size_t)fp4_act_pitch(ntok) + (size_t)fp4_n(ntok) * 128;
+    l.sfb = off;  // [stage][2 atoms]; the last copy reads a whole atom
+    off += nst * 2 * (size_t)fp4_sfb_pitch(ntok) + kAtom;
     l.abf = off;
     if (plus) off += (size_t)mrows * (size_t)K * 2;
     off = (off + 15) / 16 * 16;
     l.corr = off;  // partial corrections [kTpr][ntok][128 rows], fp32
     if (plus) off += kTpr * (size_t)ntok * 128 * 4;
     l.bars = off;
-    off += 1024;
+    off += 1280;
     // the last slot's 128-row read must stay inside the allocation
     const size_t ring_read_end = l.ring + (size_t)(stages > 0 ? stages - 1 : 0) * l.ring_stride + 128 * 128;
     if (off < ring_read_end) off = ring_read_end;
@@ -134,28 +141,29 @@ __device__ __forceinline__ uint32_t swz_chunk(uint32_t r, uint32_t c)
     } while (0)
 #endif
 
-// kTok: activation rows per CTA (2 or 4; grid.y walks M); kPlus: the weights are MXFP4+.
+// kTok: activation rows per CTA (1, 2 or 4; grid.y walks M); kPlus: the weights are MXFP4+.
 template <int kTok, bool kPlus, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
                    const __grid_constant__ CUtensorMap tmap_sc,
                    const __grid_constant__ CUtensorMap tmap_ix, const Fp4Params prm)
 {
-    constexpr int kN = kTok == 2 ? 16 : 32;  // MMA N: kSlices * kTok digit rows, padded
-    static_assert(kSlices * kTok <= kN, "digit rows must fit the MMA's N");
+    constexpr int kN = fp4_n(kTok);  // MMA N: kSlices * kTok digit rows, padded
+    constexpr int kActPitch = fp4_act_pitch(kTok), kSfbPitch = fp4_sfb_pitch(kTok);
+    static_assert(kSlices * kTok <= kN && kSlices * kTok <= kActPitch / 128, "digit rows must fit");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~(uintptr_t)1023);
     const int S = prm.stages;
     const int m0 = blockIdx.y * kTok;
     const int mrows = min(kTok, prm.M - m0);
-    const Fp4Layout L = fp4_layout(prm.K, min(prm.M, kTok), prm.rows_per_tile, S, kPlus, kTok, kN);
+    const Fp4Layout L = fp4_layout(prm.K, min(prm.M, kTok), prm.rows_per_tile, S, kPlus, kTok);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // TMA: weight tile landed
     uint64_t* empty = full + kMaxStages;       // MMAs (and BM reads) of the slot are done
     uint64_t* sfa_ready = empty + kMaxStages;  // [kMaxGroups] row warps wrote the group's scale atoms
     uint64_t* meta_full = sfa_ready + kMaxGroups;
-    uint64_t* meta_empty = meta_full + kMetaBufs;
-    uint64_t* acc_full = meta_empty + kMetaBufs;
+    uint64_t* meta_empty = meta_full + kMaxGroups;
+    uint64_t* acc_full = meta_empty + kMaxGroups;
     uint64_t* acc_empty = acc_full + 1;
     uint64_t* corr_full = acc_empty + 1;       // correction warps wrote their partial sums
     uint64_t* corr_empty = corr_full + 1;      // row warps have read them
@@ -166,6 +174,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nb = prm.K / 32;
     const int nst = prm.K / kStageK;
+    const int meta_bufs = nst / 2;  // one per group of two stages: all of a tile's
     const int rows8 = (prm.rows_per_tile + 7) / 8 * 8;
 
     auto ring = [&](int s) { return smem + L.ring + (size_t)s * L.ring_stride; };
@@ -192,7 +201,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
             ptx::mbar_init(&empty[s], kPlus ? 1 + kCorrWarps : 1);
         }
         for (int g = 0; g < kMaxGroups; ++g) ptx::mbar_init(&sfa_ready[g], 4);
-        for (int g = 0; g < kMetaBufs; ++g) {
+        for (int g = 0; g < kMaxGroups; ++g) {
             ptx::mbar_init(&meta_full[g], 1);
             ptx::mbar_init(&meta_empty[g], kPlus ? 4 + kCorrWarps : 4);
         }
@@ -231,8 +240,8 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
                 if (n0 >= prm.N) break;
                 for (int st = 0; st < nst; ++st, ++c) {
                     if ((st & 1) == 0) {
-                        const int g = gc % kMetaBufs;
-                        const uint32_t ug = gc / kMetaBufs;
+                        const int g = gc % meta_bufs;
+                        const uint32_t ug = gc / meta_bufs;
                         if (ug > 0 && !ptx::mbar_wait(&meta_empty[g], (ug - 1) & 1, abort, kWaitLimit)) {
                             report(prm.status, abort, 0x6000 + g);
                             ok = false;
@@ -264,12 +273,14 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
         // correction.
         const int tid = threadIdx.x - 32;
         constexpr int kPrep = kThreads - 32;
-        for (int i = tid; i < nst * kN * 8; i += kPrep)   // absent rows: zero codes ...
+        for (int i = tid; i < (nst * kActPitch + kN * 128) / 16; i += kPrep)   // absent rows: zero codes ...
             reinterpret_cast<uint4*>(smem + L.act)[i] = make_uint4(0u, 0u, 0u, 0u);
-        for (int i = tid; i < nst * 2 * 32; i += kPrep)   // ... with any finite scale
+        for (int i = tid; i < (nst * 2 * kSfbPitch + kAtom) / 16; i += kPrep)  // ... with any finite scale
             reinterpret_cast<uint4*>(smem + L.sfb)[i] =
                 make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+        if (tid == 0) TL(70);
         asm volatile("bar.sync 1, %0;" ::"r"(kPrep) : "memory");  // the writes below land on top
+        if (tid == 0) TL(71);
         // four threads per block of 32 activations, eight elements each
         for (int i0 = 0; i0 < ntask; i0 += kPrep) {
             const int i = i0 + tid;
@@ -293,6 +304,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
             }
             eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 1));
             eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 2));
+            if (tid == 0) TL(72);
             if (!on) continue;
             const bool nonfinite = eb == 255u;
             // 14-bit magnitude of an element relative to the block: |a| / 2^(E - 13)
@@ -307,7 +319,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
                 const uint32_t mag = sh >= 0 ? m8 << sh : (sh > -9 ? (m8 + (1u << (-sh - 1))) >> (-sh) : 0u);
                 qv[e] = mag | ((h >> 15) << 31);
             }
-            uint8_t* tile = smem + L.act + (size_t)(kb >> 3) * (kN * 128);
+            uint8_t* tile = smem + L.act + (size_t)(kb >> 3) * kActPitch;
             uint32_t sgn = 0u;  // the eight sign bits, each on top of its nibble
 #pragma unroll
             for (int e = 0; e < 8; ++e) sgn |= (qv[e] >> 31) << (4 * e + 3);
@@ -331,7 +343,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
                 const int row = j * kTok + mc;
                 *reinterpret_cast<uint32_t*>(tile + swz_chunk((uint32_t)row, (uint32_t)(kb & 7)) + 4 * qd) = w;
                 if (qd == 0)
-                    smem[L.sfb + (size_t)(kb >> 2) * kAtom + (row & 31) * 16 + (row >> 5) * 4 + (kb & 3)] =
+                    smem[L.sfb + (size_t)(kb >> 2) * kSfbPitch + row * 16 + (kb & 3)] =
                         (uint8_t)(nonfinite ? 255 : max(sbyte, 0));
             }
         }
@@ -375,7 +387,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
                 ptx::tc_fence_after_sync();
                 if (lane == 0) TL(8 + st);
                 const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(ring(s)));
-                const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(smem + L.act + (size_t)st * (kN * 128)));
+                const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(smem + L.act + (size_t)st * kActPitch));
                 if (ptx::elect_one()) {
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {  // 128 elements: one scale atom per operand
@@ -383,7 +395,7 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
                         const uint32_t t_sfb = t_sfa + 4u;
                         ptx::tc_cp_sf(t_sfa, ptx::smem_desc_sf(ptx::smem_u32(sfa(2 * st + g))));
                         ptx::tc_cp_sf(t_sfb, ptx::smem_desc_sf(ptx::smem_u32(
-                                                 smem + L.sfb + (size_t)(2 * st + g) * kAtom)));
+                                                 smem + L.sfb + (size_t)(2 * st + g) * kSfbPitch)));
 #pragma unroll
                         for (int kk = 0; kk < 2; ++kk) {  // 64 elements = 32 bytes per MMA
                             const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
@@ -418,8 +430,8 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
             const bool live = row < rows_here;
             // (the MMAs of the tile before have completed: this warp drained its accumulators)
             for (int st0 = 0; st0 < nst && ok; st0 += 2, ++gc) {
-                const int g = gc % kMetaBufs;
-                if (!ptx::mbar_wait(&meta_full[g], (gc / kMetaBufs) & 1, abort, kWaitLimit)) {
+                const int g = gc % meta_bufs;
+                if (!ptx::mbar_wait(&meta_full[g], (gc / meta_bufs) & 1, abort, kWaitLimit)) {
                     if (lane == 0) report(prm.status, abort, 0x6600 + g);
                     ok = false;
                     break;
@@ -519,9 +531,9 @@ gemm_wo_fp4_kernel(const __grid_constant__ CUtensorMap tmap_w,
 #pragma unroll
             for (int m = 0; m < kTok; ++m) corr[m] = 0.f;
             for (int st0 = 0; st0 < nst && ok; st0 += 2, ++gc, c += 2) {
-                const int g = gc % kMetaBufs;
+                const int g = gc % meta_bufs;
                 const int s0 = c % S, s1 = (c + 1) % S;
-                if (!ptx::mbar_wait(&meta_full[g], (gc / kMetaBufs) & 1, abort, kWaitLimit) ||
+                if (!ptx::mbar_wait(&meta_full[g], (gc / meta_bufs) & 1, abort, kWaitLimit) ||
                     !ptx::mbar_wait(&full[s0], (c / S) & 1, abort, kWaitLimit) ||
                     !ptx::mbar_wait(&full[s1], ((c + 1) / S) & 1, abort, kWaitLimit)) {
                     if (lane == 0) report(prm.status, abort, 0x6800 + g);
@@ -619,8 +631,7 @@ struct Fp4Plan {
 // Rows per CTA so that every SM gets work, at most 128 per tile; as many ring slots as fit.
 bool fp4_plan(int64_t M, int64_t N, int64_t K, bool plus, int num_sms, Fp4Plan* p)
 {
-    p->ntok = M <= 2 ? 2 : 4;
-    const int nrows = p->ntok == 2 ? 16 : 32;
+    p->ntok = M <= 1 ? 1 : M <= 2 ? 2 : 4;
     p->mtiles = (int)((M + p->ntok - 1) / p->ntok);
     p->gx = num_sms / p->mtiles;
     if (p->gx < 1) p->gx = 1;
@@ -629,13 +640,13 @@ bool fp4_plan(int64_t M, int64_t N, int64_t K, bool plus, int num_sms, Fp4Plan* 
     p->tiles_per_cta = (int)((rows_per_cta + max_rows - 1) / max_rows);
     p->rows_per_tile = (int)((N + (int64_t)p->gx * p->tiles_per_cta - 1) / ((int64_t)p->gx * p->tiles_per_cta));
     const int mrows = (int)(M < p->ntok ? M : p->ntok);
-    const size_t fixed = fp4_layout((int)K, mrows, p->rows_per_tile, 0, plus, p->ntok, nrows).total;
+    const size_t fixed = fp4_layout((int)K, mrows, p->rows_per_tile, 0, plus, p->ntok).total;
     const size_t per_stage = (size_t)((p->rows_per_tile + 7) / 8 * 8) * 128;
     if (fixed + 4 * per_stage + 128 * 128 > kSmemMax) return false;
     int stages = (int)((kSmemMax - fixed - 128 * 128) / per_stage);
     stages = stages > kMaxStages ? kMaxStages : stages;
     p->stages = stages / kIssuers * kIssuers;  // every slot belongs to one issuer
-    p->smem = fp4_layout((int)K, mrows, p->rows_per_tile, p->stages, plus, p->ntok, nrows).total;
+    p->smem = fp4_layout((int)K, mrows, p->rows_per_tile, p->stages, plus, p->ntok).total;
     return p->smem <= kSmemMax;
 }
 
@@ -720,6 +731,7 @@ cudaError_t launch_gemm_wo_fp4(int64_t M, int64_t N, int64_t K, const void* A, i
 #define MXP_FP4_LAUNCH(T, P)                                                  \
     (f32 ? launch<T, P, float>(tw, ts, ti, prm, plan, stream)                 \
          : launch<T, P, __nv_bfloat16>(tw, ts, ti, prm, plan, stream))
+    if (plan.ntok == 1) return plus ? MXP_FP4_LAUNCH(1, true) : MXP_FP4_LAUNCH(1, false);
     if (plan.ntok == 2) return plus ? MXP_FP4_LAUNCH(2, true) : MXP_FP4_LAUNCH(2, false);
     return plus ? MXP_FP4_LAUNCH(4, true) : MXP_FP4_LAUNCH(4, false);
 #undef MXP_FP4_LAUNCH
