@@ -285,6 +285,26 @@ def part_decode(mxp, synth, peaks, iters):
                 ms_g = time_loop(graph.replay, max(1, iters // 8), warmup=2) / 8
                 out[key]["us_cuda_graph"] = ms_g * 1e3
                 out[key]["frac_hbm_cuda_graph"] = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_g / 1e6 / hbm
+            if kern is None:
+                # the eight launches as a chain of programmatic dependents (each grid's weight
+                # stream starts while the previous grid drains; activations and output stay
+                # ordered): what a captured decode loop over constant weights can use
+                def run_chained():
+                    mxp.mxp_gemm_decode_chained(a, copies[state["i"] % 8], d)
+                    state["i"] += 1
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    for _ in range(8):
+                        run_chained()
+                torch.cuda.current_stream().wait_stream(side)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    for _ in range(8):
+                        run_chained()
+                ms_c = time_loop(graph.replay, max(1, iters // 8), warmup=2) / 8
+                out[key]["us_cuda_graph_chained"] = ms_c * 1e3
+                out[key]["frac_hbm_cuda_graph_chained"] = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_c / 1e6 / hbm
         os.environ.pop("MXP_WO_KERNEL", None)
         del copies, w
     return out

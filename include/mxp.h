@@ -201,6 +201,34 @@ mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed *A_p
                           void *cuda_stream);
 
 /*
+ * The weight-only form of mxp_gemm for a chain of decode GEMMs on one stream (Sec. 7.1:
+ * "conversion before computation", the memory-bound token-generation phase, where one such
+ * GEMM follows another and each streams its own weights once).  Same operation and result
+ * as mxp_gemm(A_dense_bf16, B_packed); the difference is when the grid may start: it is
+ * launched as a programmatic dependent of the preceding kernel on `cuda_stream`, so its
+ * CTAs are scheduled while that kernel drains and begin streaming B's planes at once.
+ * Ordering that still holds: A is read and D is written only after the preceding kernel has
+ * completed and its writes are visible.  Ordering the caller gives up: B's three planes
+ * (nibbles, scales, bm_index) must not be written by the kernel that precedes this call on
+ * the stream (weights quantised once, ahead of the decode loop, satisfy this; quantising B
+ * immediately before this call does not: use mxp_gemm there).  Every streamed weight-only
+ * kernel of this library releases its own dependents when it starts, so a chain of these
+ * calls overlaps launch to launch; after any other kernel the call behaves like mxp_gemm.
+ * May be captured into a CUDA graph (the launches become programmatic dependency edges).
+ *
+ *   M <= 64, N % 16 == 0, K % 256 == 0, pointers 16-byte aligned, lda % 8 == 0; otherwise
+ *   MXP_ERR_UNSUPPORTED and nothing is launched (use mxp_gemm).
+ *   status_block   device pointer (16 bytes, 16-byte aligned) or NULL.  NOT cleared by the
+ *                  call (a clear between the kernels would break the chain): zero it once,
+ *                  the first bounded wait that runs out in any call of the chain leaves
+ *                  MXP_ERR_TIMEOUT there; read it with mxp_gemm_status.
+ */
+mxp_status mxp_gemm_decode_chained(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16,
+                                   int64_t lda, const mxp_packed *B_packed, void *D,
+                                   mxp_dtype d_dt, int64_t ldd, void *status_block,
+                                   void *cuda_stream);
+
+/*
  * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM
  * left in `workspace`: MXP_OK, or MXP_ERR_TIMEOUT if a bounded wait inside a kernel gave
  * up (the output is then undefined but the context stays usable).

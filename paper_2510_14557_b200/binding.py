@@ -25,7 +25,7 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
            "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
@@ -64,6 +64,9 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_noalloc.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
                                        vp, ci, i64, ctypes.POINTER(ci), vp]
         l.mxp_gemm_noalloc.restype = ci
+        l.mxp_gemm_decode_chained.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, ci,
+                                              i64, vp, vp]
+        l.mxp_gemm_decode_chained.restype = ci
         l.mxp_gemm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
         l.mxp_gemm_workspace_bytes.restype = sz
         l.mxp_gemm_min_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
@@ -281,6 +284,21 @@ def mxp_gemm_noalloc(a: Packed, b: Packed, out: torch.Tensor, read_status: bool 
                                 ctypes.byref(ks) if read_status else None, _stream())
     _check("mxp_gemm_noalloc", st)
     return ks.value if read_status else None
+
+
+def mxp_gemm_decode_chained(a: torch.Tensor, b: Packed, out: torch.Tensor,
+                            status_block: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Weight-only GEMM launched as a programmatic dependent of the preceding kernel on the
+    stream (a chain of decode GEMMs).  `b` must not be written by that preceding kernel; `a`
+    and `out` are ordered as usual.  `status_block`: 16 zeroed bytes on the device, or None."""
+    assert a.dtype == torch.bfloat16 and a.is_cuda and a.stride(1) == 1
+    bs = b.c_struct()
+    st = lib().mxp_gemm_decode_chained(a.shape[0], b.rows, b.cols, a.data_ptr(), a.stride(0),
+                                       ctypes.byref(bs), out.data_ptr(), _dt(out), out.stride(0),
+                                       status_block.data_ptr() if status_block is not None else None,
+                                       _stream())
+    _check("mxp_gemm_decode_chained", st)
+    return out
 
 
 def mxp_wait_selftest(workspace: torch.Tensor, limit_cycles: int) -> None:

@@ -155,6 +155,29 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
                                workspace_bytes, stream);
 }
 
+mxp_status mxp_gemm_decode_chained(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16,
+                                   int64_t lda, const mxp_packed* B_packed, void* D,
+                                   mxp_dtype d_dt, int64_t ldd, void* status_block,
+                                   void* cuda_stream)
+{
+    if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!valid_dtype(d_dt) || A_dense_bf16 == nullptr) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(B_packed, false)) return MXP_ERR_INVALID_ARG;
+    if (B_packed->rows != N || B_packed->cols != K) return MXP_ERR_INVALID_ARG;
+    if (lda < K || lda % 8 != 0 || !aligned(A_dense_bf16, 16)) return MXP_ERR_INVALID_ARG;
+    if (status_block != nullptr && !aligned(status_block, 16)) return MXP_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return MXP_OK;
+    if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
+    if (K == 0 || M > 64) return MXP_ERR_UNSUPPORTED;
+    if (!mxp::wo_stream_supported(M, N, K, A_dense_bf16, lda, *B_packed)) return MXP_ERR_UNSUPPORTED;
+    const cudaError_t e = mxp::launch_gemm_wo_stream(M, N, K, A_dense_bf16, lda, *B_packed, D, d_dt,
+                                                     ldd, status_block,
+                                                     static_cast<cudaStream_t>(cuda_stream), true);
+    if (e == cudaErrorNotSupported) return MXP_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
 size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide)
 {
     return mxp::stream_prepack_bytes(rows, K, wide != 0);

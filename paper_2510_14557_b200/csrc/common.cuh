@@ -31,7 +31,7 @@ bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t
                          const mxp_packed& B);
 cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                   const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                                  void* status, cudaStream_t stream);
+                                  void* status, cudaStream_t stream, bool chained = false);
 
 // MXFP6(+) / MXFP8(+): quantize and decode only (quantize_wide.cu).
 cudaError_t launch_quantize_wide(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,

@@ -264,6 +264,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
     const int m0 = blockIdx.y * kMp;
     const bool two_red = prm.red_buffers == 2;
 
+    // Chained launches (Sec. 7.1's decode loop runs one such GEMM after another): let the next
+    // grid on the stream be scheduled as soon as SMs free up.  What this grid must not touch
+    // before the previous one has finished is fenced below (activations in, D out); the weight
+    // planes are read at once.
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) {
         WO_TL(0);
         for (int s = 0; s < kMaxStages; ++s) {
@@ -343,6 +348,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
         // by its own power of two, kept in fa[chunk][column].
         float* fa = reinterpret_cast<float*>(smem + L.fa);
         constexpr int kItems = kChunkBlocks * kMp / 32;  // blocks per lane and chunk
+        ptx::grid_dependency_wait();  // A may be the previous grid's output
         for (int sl = 0; sl < slabs; ++sl) {
             const int chunk = sl * kCW + warp;
             const int kb0 = chunk * kChunkBlocks;
@@ -508,6 +514,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
         const int tid = threadIdx.x - 32 * (kCW + 1);
         const float* red = reinterpret_cast<const float*>(smem + L.red);
         uint32_t it = 0;
+        ptx::grid_dependency_wait();  // D may still be read by the previous grid
         for (int rg = blockIdx.x; rg < rgs; rg += gridDim.x, ++it) {
             const int64_t n0 = (int64_t)rg * kRows;
             const uint32_t rbuf = two_red ? (it & 1u) : 0u;
@@ -568,7 +575,7 @@ inline bool wo_plan(int K, int mp, bool plus, int* stages, int* red_buffers, int
 }
 
 template <int kMT, int kMode, typename OutT>
-cudaError_t launch(WoParams prm, int num_sms, cudaStream_t stream)
+cudaError_t launch(WoParams prm, int num_sms, bool chained, cudaStream_t stream)
 {
     constexpr bool kPlus = kMode >= 1;
     if (!wo_plan(prm.K, 8 * kMT, kPlus, &prm.stages, &prm.red_buffers, &prm.meta_bufs))
@@ -584,8 +591,23 @@ cudaError_t launch(WoParams prm, int num_sms, cudaStream_t stream)
     int gx = num_sms / mtiles;
     if (gx < 1) gx = 1;
     if (gx > rgs) gx = rgs;
-    kern<<<dim3((unsigned)gx, (unsigned)mtiles), kThreads, smem, stream>>>(prm);
-    return cudaGetLastError();
+    if (!chained) {
+        kern<<<dim3((unsigned)gx, (unsigned)mtiles), kThreads, smem, stream>>>(prm);
+        return cudaGetLastError();
+    }
+    // programmatic dependent launch: this grid may start while the previous one on the stream
+    // is draining; only its weight stream runs ahead of the in-kernel dependency wait
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)gx, (unsigned)mtiles);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, prm);
 }
 
 
@@ -608,7 +630,7 @@ bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t
 
 cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                   const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                                  void* status, cudaStream_t stream)
+                                  void* status, cudaStream_t stream, bool chained)
 {
     WoParams prm;
     prm.status = static_cast<StatusBlock*>(status);
@@ -630,14 +652,14 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
 #define MXP_WO_LAUNCH(MT)                                                                  \
     switch (mode) {                                                                        \
         case 2:                                                                            \
-            return f32 ? launch<MT, 2, float>(prm, sms, stream)                            \
-                       : launch<MT, 2, __nv_bfloat16>(prm, sms, stream);                   \
+            return f32 ? launch<MT, 2, float>(prm, sms, chained, stream)                            \
+                       : launch<MT, 2, __nv_bfloat16>(prm, sms, chained, stream);                   \
         case 1:                                                                            \
-            return f32 ? launch<MT, 1, float>(prm, sms, stream)                            \
-                       : launch<MT, 1, __nv_bfloat16>(prm, sms, stream);                   \
+            return f32 ? launch<MT, 1, float>(prm, sms, chained, stream)                            \
+                       : launch<MT, 1, __nv_bfloat16>(prm, sms, chained, stream);                   \
         default:                                                                           \
-            return f32 ? launch<MT, 0, float>(prm, sms, stream)                            \
-                       : launch<MT, 0, __nv_bfloat16>(prm, sms, stream);                   \
+            return f32 ? launch<MT, 0, float>(prm, sms, chained, stream)                            \
+                       : launch<MT, 0, __nv_bfloat16>(prm, sms, chained, stream);                   \
     }
     if (M <= 8) {
         MXP_WO_LAUNCH(1)

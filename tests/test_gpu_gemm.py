@@ -112,6 +112,76 @@ def test_weight_only_one_hot_and_scale_spread(kernel, monkeypatch):
         assert np.array_equal(got[m], want)
 
 
+@pytest.mark.parametrize("wmode", [MX, MXP, 2])
+@pytest.mark.parametrize("M,NK,layers", [(1, 1024, 6), (8, 4096, 4), (16, 2048, 5)])
+def test_weight_only_chained_layers(M, NK, layers, wmode):
+    # A chain of decode GEMMs launched as programmatic dependents: layer i's output is layer
+    # i+1's activation, so a grid that read its input (or wrote its output) before the previous
+    # one had finished would show.  First layer against the oracle; the whole chain bit for bit
+    # against the same chain of ordinary launches, eagerly and replayed from a CUDA graph.
+    m = mxp()
+    a_bits, _ = synth.config3(M, 16, NK, seed=NK + M)
+    ws, decs = [], []
+    for i in range(layers):
+        _, w_bits = synth.config3(1, NK, NK, seed=100 + i)
+        wp, dw = quantized(w_bits, wmode, bf16=True)
+        ws.append(wp)
+        decs.append(dw)
+    a0 = to_dev_bf16(a_bits)
+    status = torch.zeros(16, dtype=torch.uint8, device="cuda")
+
+    def chain(fn):
+        bufs = [torch.zeros((M, NK), dtype=torch.bfloat16, device="cuda") for _ in range(layers)]
+        x = a0
+        for i in range(layers):
+            fn(x, ws[i], bufs[i])
+            x = bufs[i]
+        return bufs
+
+    plain = chain(lambda x, w, o: m.mxp_gemm(x, w, out=o))
+    chained = chain(lambda x, w, o: m.mxp_gemm_decode_chained(x, w, o, status))
+    torch.cuda.synchronize()
+    assert m.mxp_gemm_status(status) == 0
+    check_gemm(chained[0], oracle.bf16_bits_to_f64(a_bits), decs[0])
+    for p_, c_ in zip(plain, chained):
+        assert torch.equal(p_.view(torch.int16), c_.view(torch.int16))
+
+    # the same chain captured: the launches become programmatic dependency edges
+    bufs = [torch.zeros((M, NK), dtype=torch.bfloat16, device="cuda") for _ in range(layers)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        x = a0
+        for i in range(layers):
+            m.mxp_gemm_decode_chained(x, ws[i], bufs[i], status)
+            x = bufs[i]
+    torch.cuda.current_stream().wait_stream(side)
+    for b_ in bufs:
+        b_.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        x = a0
+        for i in range(layers):
+            m.mxp_gemm_decode_chained(x, ws[i], bufs[i], status)
+            x = bufs[i]
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert m.mxp_gemm_status(status) == 0
+    for p_, c_ in zip(plain, bufs):
+        assert torch.equal(p_.view(torch.int16), c_.view(torch.int16))
+
+
+def test_weight_only_chained_rejects_what_it_cannot_run():
+    m = mxp()
+    a_bits, w_bits = synth.config3(4, 24, 256, seed=3)  # N % 16 != 0
+    wp, _ = quantized(w_bits, MXP, bf16=True)
+    out = torch.zeros((4, 24), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(m.MxpError) as e:
+        m.mxp_gemm_decode_chained(to_dev_bf16(a_bits), wp, out)
+    assert e.value.status == 2
+
+
 # ------------------------------------------------------------------ tensor-core form
 MODES = [(MX, MX), (MXP, MX), (MX, MXP), (MXP, MXP)]
 
