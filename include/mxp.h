@@ -96,6 +96,35 @@ mxp_status mxp_quantize(const void *src, mxp_dtype src_dt, int64_t rows, int64_t
                         uint8_t *bm_index, void *cuda_stream);
 
 /*
+ * mxp_quantize with channel reordering fused in (Sec. 8, "Scattering outliers with channel
+ * reordering": outlier channels are spread over the blocks so that more of them become a
+ * block's BM; the reordering costs nothing extra because it happens where the quantizer
+ * touches the data anyway).  Position c of every quantized row holds source channel
+ * order[c]:  out = quantize(src[:, order]).  Both operands of a GEMM must use the same
+ * ordering along K for the product to be unchanged.
+ *   order   device, `cols` entries of int32, 16-byte aligned, read for every row.  Meant to
+ *           be a permutation of 0..cols-1; the library does not check that: entries are
+ *           clamped to cols-1 and applied as a gather.
+ *   src     as for mxp_quantize, but only element-aligned (rows are read channel by channel)
+ *   modes   MXFP4, MXFP4+, MXFP4++; the 6- and 8-bit modes return MXP_ERR_UNSUPPORTED.
+ * Everything else (planes, sizes, errors) as mxp_quantize.
+ *
+ * mxp_channel_order builds such an ordering on the HOST from per-channel outlier counts, by
+ * the rule of the same passage: channels sorted by count, most first (equal counts keep
+ * channel order); the cols/32 highest go one to each block, at its first position, in that
+ * order; the remaining channels fill the other positions front to back, first the half with
+ * the fewer outliers and then the half with the more, each half from its highest count down
+ * (an odd remainder gives the extra channel to the first-placed half).  How outliers are
+ * counted (threshold, calibration samples) is the caller's business.
+ *   outlier_count, order   host arrays of `cols` entries; cols % 32 == 0.
+ */
+mxp_status mxp_quantize_reordered(const void *src, mxp_dtype src_dt, int64_t rows, int64_t cols,
+                                  int64_t ld_src, const int32_t *order, mxp_mode mode,
+                                  uint8_t *nibbles, uint8_t *scales, uint8_t *bm_index,
+                                  void *cuda_stream);
+mxp_status mxp_channel_order(const int64_t *outlier_count, int64_t cols, int32_t *order);
+
+/*
  * Decode (Eq. 3): dst[r][c] = (-1)^s * 2^(scale - 127) * E, E = 4 + m/2 for the BM
  * element of an MXFP4+ block, the E2M1 value otherwise.  Exact in both output types.
  *   p       host pointer to the operand descriptor (its planes are device memory)

@@ -220,3 +220,37 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     """Exact widening of bfloat16 bit patterns (uint16) to float64."""
     u = bits.astype(np.uint32) << np.uint32(16)
     return u.view(np.float32).astype(np.float64)
+
+
+def channel_order(outlier_count) -> np.ndarray:
+    """Channel ordering that scatters outlier channels over the blocks (Sec. 8, "Scattering
+    outliers with channel reordering"), as int32 [cols]: position p takes channel order[p].
+
+    Channels are ranked by outlier count, most first (equal counts: lower channel first).
+    The cols/32 highest-ranked channels go one to each block, at the block's first position.
+    The other channels are cut into the half with more outliers and the half with fewer
+    (the odd one out joins the latter); the positions still free are filled front to back,
+    first with the half that has fewer outliers, then with the half that has more, each in
+    ranked order.  (The passage leaves the direction of "remaining places" and the handling
+    of ties and odd counts open; this is the reading the library documents.)"""
+    cnt = [int(c) for c in np.asarray(outlier_count).reshape(-1)]
+    cols = len(cnt)
+    assert cols > 0 and cols % 32 == 0
+    nblk = cols // 32
+    ranked = sorted(range(cols), key=lambda c: (-cnt[c], c))
+    order = [-1] * cols
+    for j in range(nblk):
+        order[32 * j] = ranked[j]
+    rest = ranked[nblk:]
+    more, fewer = rest[:len(rest) // 2], rest[len(rest) // 2:]
+    free = [p for p in range(cols) if p % 32 != 0]
+    for p, c in zip(free, fewer + more):
+        order[p] = c
+    return np.asarray(order, np.int32)
+
+
+def quantize_reordered(x: np.ndarray, order: np.ndarray, mode: int, bf16_bits: bool = False):
+    """Quantization of the rows with their channels taken in `order` (same passage): the
+    definition is quantize(x[:, order])."""
+    return quantize(np.ascontiguousarray(np.asarray(x)[:, np.asarray(order, np.int64)]), mode,
+                    bf16_bits=bf16_bits)

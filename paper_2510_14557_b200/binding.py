@@ -25,7 +25,7 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
            "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
@@ -64,6 +64,10 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_noalloc.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
                                        vp, ci, i64, ctypes.POINTER(ci), vp]
         l.mxp_gemm_noalloc.restype = ci
+        l.mxp_quantize_reordered.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp, vp, vp, vp]
+        l.mxp_quantize_reordered.restype = ci
+        l.mxp_channel_order.argtypes = [vp, i64, vp]
+        l.mxp_channel_order.restype = ci
         l.mxp_gemm_decode_chained.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, ci,
                                               i64, vp, vp]
         l.mxp_gemm_decode_chained.restype = ci
@@ -164,6 +168,35 @@ def mxp_quantize(src: torch.Tensor, mode: int, out: Optional[Packed] = None) -> 
                             _stream())
     _check("mxp_quantize", st)
     return out
+
+
+def mxp_quantize_reordered(src: torch.Tensor, order: torch.Tensor, mode: int,
+                           out: Optional[Packed] = None) -> Packed:
+    """quantize(src[:, order]) in one pass: `order` is an int32 CUDA tensor of src.shape[1]
+    entries (position c of the quantized rows takes source channel order[c])."""
+    assert src.is_cuda and src.dim() == 2 and src.stride(1) == 1
+    assert order.is_cuda and order.dtype == torch.int32 and order.is_contiguous()
+    rows, cols = src.shape
+    assert order.numel() == cols
+    if out is None:
+        out = alloc_packed(rows, cols, mode, src.device)
+    st = lib().mxp_quantize_reordered(src.data_ptr(), _dt(src), rows, cols, src.stride(0),
+                                      order.data_ptr(), mode, out.nibbles.data_ptr(),
+                                      out.scales.data_ptr(),
+                                      out.bm_index.data_ptr() if out.bm_index is not None else None,
+                                      _stream())
+    _check("mxp_quantize_reordered", st)
+    return out
+
+
+def mxp_channel_order(outlier_count) -> torch.Tensor:
+    """Channel ordering (int32 CPU tensor) from per-channel outlier counts, by the paper's
+    rule; see the header for the exact placement."""
+    cnt = torch.as_tensor(outlier_count, dtype=torch.int64).contiguous().cpu()
+    order = torch.empty(cnt.numel(), dtype=torch.int32)
+    st = lib().mxp_channel_order(cnt.data_ptr(), cnt.numel(), order.data_ptr())
+    _check("mxp_channel_order", st)
+    return order
 
 
 def mxp_dequantize(p: Packed, dtype=torch.float32, out: Optional[torch.Tensor] = None) -> torch.Tensor:

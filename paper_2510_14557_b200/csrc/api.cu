@@ -1,5 +1,7 @@
 // C ABI of libmxp: argument validation and dispatch.  No kernel lives here.
+#include <algorithm>
 #include <cstring>
+#include <vector>
 
 #include "common.cuh"
 
@@ -75,6 +77,56 @@ mxp_status mxp_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t
     cudaError_t e = mxp::launch_quantize(src, src_dt, rows, cols, ld_src, mode, nibbles, scales,
                                          bm_index, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+mxp_status mxp_quantize_reordered(const void* src, mxp_dtype src_dt, int64_t rows, int64_t cols,
+                                  int64_t ld_src, const int32_t* order, mxp_mode mode,
+                                  uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
+                                  void* cuda_stream)
+{
+    if ((!valid_mode(mode) && !wide_mode(mode)) || !valid_dtype(src_dt)) return MXP_ERR_INVALID_ARG;
+    if (rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return MXP_OK;
+    if (src == nullptr || nibbles == nullptr || scales == nullptr || order == nullptr)
+        return MXP_ERR_INVALID_ARG;
+    if (plus_mode(mode) && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (ld_src < cols) return MXP_ERR_INVALID_ARG;
+    if (!aligned(src, src_dt == MXP_BF16 ? 2 : 4) || !aligned(nibbles, 16) || !aligned(order, 16))
+        return MXP_ERR_INVALID_ARG;
+    if (wide_mode(mode) || cols > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    if (rows * (cols / 32) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    cudaError_t e = mxp::launch_quantize_reordered(src, src_dt, rows, cols, ld_src, order, mode,
+                                                   nibbles, scales, bm_index,
+                                                   static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+mxp_status mxp_channel_order(const int64_t* outlier_count, int64_t cols, int32_t* order)
+{
+    if (outlier_count == nullptr || order == nullptr) return MXP_ERR_INVALID_ARG;
+    if (cols <= 0 || cols % 32 != 0 || cols > 0x7FFFFFFFll) return MXP_ERR_INVALID_ARG;
+    // channels by outlier count, most first; equal counts keep channel order
+    std::vector<int32_t> by_count((size_t)cols);
+    for (int64_t c = 0; c < cols; ++c) by_count[(size_t)c] = (int32_t)c;
+    std::stable_sort(by_count.begin(), by_count.end(), [&](int32_t a, int32_t b) {
+        return outlier_count[a] > outlier_count[b];
+    });
+    const int64_t nblk = cols / 32;
+    // the nblk channels with the most outliers: one per block, at the block's first position
+    for (int64_t j = 0; j < nblk; ++j) order[32 * j] = by_count[(size_t)j];
+    // the rest fills the other positions front to back: first the half with fewer outliers,
+    // then the half with more, each from its most-outlier channel down
+    const int64_t rest = cols - nblk, upper = rest / 2;
+    int64_t pos = 0;
+    auto place = [&](int64_t from, int64_t to) {
+        for (int64_t i = from; i < to; ++i) {
+            if (pos % 32 == 0) ++pos;
+            order[pos++] = by_count[(size_t)(nblk + i)];
+        }
+    };
+    place(upper, rest);
+    place(0, upper);
+    return MXP_OK;
 }
 
 mxp_status mxp_dequantize(const mxp_packed* p, void* dst, mxp_dtype dst_dt, int64_t ld_dst,

@@ -14,6 +14,11 @@ cudaError_t launch_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t
                             int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
                             uint8_t* bm_index, cudaStream_t stream);
 
+cudaError_t launch_quantize_reordered(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                                      int64_t ld_src, const int32_t* order, mxp_mode mode,
+                                      uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
+                                      cudaStream_t stream);
+
 cudaError_t launch_dequantize(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
                               cudaStream_t stream);
 

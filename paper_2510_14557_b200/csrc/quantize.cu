@@ -130,61 +130,16 @@ __device__ __forceinline__ uint32_t encode_quarter(const float (&v)[8], uint32_t
     return (flush || nonfinite) ? 0u : word;
 }
 
-// kContig: ld_src == cols, so the source is one flat array of blocks.
-template <typename T, int kMode, bool kContig>
-__global__ void __launch_bounds__(kThreads)
-quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
-                int64_t total_blocks, uint8_t* __restrict__ nibbles,
-                uint8_t* __restrict__ scales, uint8_t* __restrict__ bm_index, int planes_aligned4)
+// Second half of a pass: the four lanes of a group hold the four quarters of blocks
+// span0 .. span0+3 (v: values, key / hi_bits: the lane's maximum); blocks at or past `limit`
+// are not stored.
+template <typename T, int kMode>
+__device__ __forceinline__ void finish_pass(const float (&v)[4][8], const uint32_t (&key)[4],
+                                            const uint32_t (&hi_bits)[4], int64_t span0, int q,
+                                            int64_t total_blocks, uint8_t* __restrict__ nibbles,
+                                            uint8_t* __restrict__ scales,
+                                            uint8_t* __restrict__ bm_index, int planes_aligned4)
 {
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const int g = lane >> 2;  // lane group: blocks 4g .. 4g+3 of the warp's span
-    const int q = lane & 3;   // quarter of the block owned by this lane
-    const int64_t span0 =
-        (int64_t)blockIdx.x * kBlocksPerCta + (int64_t)warp * kBlocksPerWarpPass + 4 * g;
-
-    float v[4][8];
-    uint32_t key[4];
-    uint32_t hi_bits[4];  // fp32 path: the lane's maximum |x| bit pattern
-
-    // ---- issue all loads of the pass first
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int64_t blk = span0 + j;
-        const bool live = blk < total_blocks;
-        int64_t elem;  // offset of the block's first element in src
-        if (kContig) {
-            elem = blk * 32;
-        } else {
-            const int64_t row = blk / cols_blocks;
-            elem = row * ld_src + (blk - row * cols_blocks) * 32;
-        }
-        if (sizeof(T) == 2) {
-            uint4 w = make_uint4(0, 0, 0, 0);
-            if (live) w = ldg_stream(reinterpret_cast<const char*>(src) + (elem + q * 8) * 2);
-            load_unit_bf16(w, q * 8, v[j], key[j]);
-            hi_bits[j] = 0;
-        } else {
-            uint4 w0 = make_uint4(0, 0, 0, 0), w1 = w0;
-            if (live) {
-                const char* p = reinterpret_cast<const char*>(src) + (elem + q * 8) * 4;
-                w0 = ldg_stream(p);
-                w1 = ldg_stream(p + 16);
-            }
-            const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-            uint32_t a = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                v[j][i] = __uint_as_float(w[i]);
-                a = max(a, w[i] & 0x7FFFFFFFu);
-            }
-            hi_bits[j] = a;
-            key[j] = 0;
-            (void)w;
-        }
-    }
-
     uint32_t words[4], sc_pack = 0, ix_pack = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -251,6 +206,171 @@ quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
     }
 }
 
+// kContig: ld_src == cols, so the source is one flat array of blocks.
+// kGather: channel reordering fused into the quantizer (Sec. 8, "Scattering outliers with
+// channel reordering"): position c of the quantized row takes source channel order[c], so a
+// block is 32 channels that the caller's ordering placed together; nothing else changes.
+template <typename T, int kMode, bool kContig, bool kGather = false>
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t cols_blocks,
+                int64_t total_blocks, uint8_t* __restrict__ nibbles,
+                uint8_t* __restrict__ scales, uint8_t* __restrict__ bm_index, int planes_aligned4,
+                const int32_t* __restrict__ order = nullptr)
+{
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int g = lane >> 2;  // lane group: blocks 4g .. 4g+3 of the warp's span
+    const int q = lane & 3;   // quarter of the block owned by this lane
+    const int64_t span0 =
+        (int64_t)blockIdx.x * kBlocksPerCta + (int64_t)warp * kBlocksPerWarpPass + 4 * g;
+
+    float v[4][8];
+    uint32_t key[4];
+    uint32_t hi_bits[4];  // fp32 path: the lane's maximum |x| bit pattern
+
+    // ---- issue all loads of the pass first
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int64_t blk = span0 + j;
+        const bool live = blk < total_blocks;
+        int64_t elem;  // offset of the block's first element in src
+        if (kContig) {
+            elem = blk * 32;
+        } else {
+            const int64_t row = blk / cols_blocks;
+            elem = row * ld_src + (blk - row * cols_blocks) * 32;
+        }
+        uint32_t ch[8];  // kGather: the lane's eight source channels, clamped into the row
+        if (kGather) {
+            const int64_t row = blk / cols_blocks;
+            const int64_t c0 = (blk - row * cols_blocks) * 32 + q * 8;
+            elem = row * ld_src;
+            uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
+            if (live) {
+                o0 = __ldg(reinterpret_cast<const uint4*>(order + c0));
+                o1 = __ldg(reinterpret_cast<const uint4*>(order + c0) + 1);
+            }
+            const uint32_t o[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+            const uint32_t last = (uint32_t)(cols_blocks * 32 - 1);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ch[i] = min(o[i], last);
+        }
+        if (sizeof(T) == 2) {
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (kGather) {
+                if (live) {
+                    const unsigned short* s16 = reinterpret_cast<const unsigned short*>(src) + elem;
+                    w.x = (uint32_t)__ldg(s16 + ch[0]) | ((uint32_t)__ldg(s16 + ch[1]) << 16);
+                    w.y = (uint32_t)__ldg(s16 + ch[2]) | ((uint32_t)__ldg(s16 + ch[3]) << 16);
+                    w.z = (uint32_t)__ldg(s16 + ch[4]) | ((uint32_t)__ldg(s16 + ch[5]) << 16);
+                    w.w = (uint32_t)__ldg(s16 + ch[6]) | ((uint32_t)__ldg(s16 + ch[7]) << 16);
+                }
+            } else if (live) {
+                w = ldg_stream(reinterpret_cast<const char*>(src) + (elem + q * 8) * 2);
+            }
+            load_unit_bf16(w, q * 8, v[j], key[j]);
+            hi_bits[j] = 0;
+        } else {
+            uint4 w0 = make_uint4(0, 0, 0, 0), w1 = w0;
+            if (kGather) {
+                if (live) {
+                    const uint32_t* s32 = reinterpret_cast<const uint32_t*>(src) + elem;
+                    w0 = make_uint4(__ldg(s32 + ch[0]), __ldg(s32 + ch[1]), __ldg(s32 + ch[2]),
+                                    __ldg(s32 + ch[3]));
+                    w1 = make_uint4(__ldg(s32 + ch[4]), __ldg(s32 + ch[5]), __ldg(s32 + ch[6]),
+                                    __ldg(s32 + ch[7]));
+                }
+            } else if (live) {
+                const char* p = reinterpret_cast<const char*>(src) + (elem + q * 8) * 4;
+                w0 = ldg_stream(p);
+                w1 = ldg_stream(p + 16);
+            }
+            const uint32_t w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+            uint32_t a = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[j][i] = __uint_as_float(w[i]);
+                a = max(a, w[i] & 0x7FFFFFFFu);
+            }
+            hi_bits[j] = a;
+            key[j] = 0;
+            (void)w;
+        }
+    }
+
+    finish_pass<T, kMode>(v, key, hi_bits, span0, q, total_blocks, nibbles, scales, bm_index,
+                          planes_aligned4);
+}
+
+// Channel reordering with the row staged in shared memory: a CTA copies one source row with
+// coalesced 16-byte loads, then its lanes pick their channels out of shared memory, where an
+// arbitrary ordering costs bank conflicts instead of one 128-byte line per element.  Rows are
+// dealt to the CTAs round robin; several CTAs per SM overlap one's copy with another's casts.
+template <typename T, int kMode>
+__global__ void __launch_bounds__(kThreads)
+quantize_reordered_staged_kernel(const T* __restrict__ src, int64_t ld_src, int64_t rows,
+                                 int cols_blocks, const int32_t* __restrict__ order,
+                                 uint8_t* __restrict__ nibbles, uint8_t* __restrict__ scales,
+                                 uint8_t* __restrict__ bm_index, int planes_aligned4)
+{
+    extern __shared__ uint4 row_smem[];
+    const T* row_s = reinterpret_cast<const T*>(row_smem);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, q = lane & 3;
+    const int cols = cols_blocks * 32;
+    const int vecs = cols * (int)sizeof(T) / 16;
+    const uint32_t last = (uint32_t)(cols - 1);
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const uint4* src_row = reinterpret_cast<const uint4*>(src + row * ld_src);
+        __syncthreads();  // the previous row has been read
+        for (int i = threadIdx.x; i < vecs; i += kThreads) row_smem[i] = ldg_stream(src_row + i);
+        __syncthreads();
+        const int64_t row_blk0 = row * cols_blocks;
+        // (warp-uniform trip count: finish_pass shuffles within the whole warp)
+        for (int base = warp * kBlocksPerWarpPass; base < cols_blocks; base += kBlocksPerCta) {
+            const int b0 = base + 4 * g;
+            float v[4][8];
+            uint32_t key[4], hi_bits[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool live = b0 + j < cols_blocks;
+                uint4 o0 = make_uint4(0, 0, 0, 0), o1 = o0;
+                if (live) {
+                    const uint4* op = reinterpret_cast<const uint4*>(order + (b0 + j) * 32 + q * 8);
+                    o0 = __ldg(op);
+                    o1 = __ldg(op + 1);
+                }
+                const uint32_t o[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+                if (sizeof(T) == 2) {
+                    const unsigned short* s16 = reinterpret_cast<const unsigned short*>(row_s);
+                    uint32_t w[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        w[i] = live ? (uint32_t)s16[min(o[2 * i], last)] |
+                                          ((uint32_t)s16[min(o[2 * i + 1], last)] << 16)
+                                    : 0u;
+                    load_unit_bf16(make_uint4(w[0], w[1], w[2], w[3]), q * 8, v[j], key[j]);
+                    hi_bits[j] = 0;
+                } else {
+                    const uint32_t* s32 = reinterpret_cast<const uint32_t*>(row_s);
+                    uint32_t a = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t w = live ? s32[min(o[i], last)] : 0u;
+                        v[j][i] = __uint_as_float(w);
+                        a = max(a, w & 0x7FFFFFFFu);
+                    }
+                    hi_bits[j] = a;
+                    key[j] = 0;
+                }
+            }
+            // blocks past the end of this row are not stored
+            finish_pass<T, kMode>(v, key, hi_bits, row_blk0 + b0, q, row_blk0 + cols_blocks, nibbles,
+                                  scales, bm_index, planes_aligned4);
+        }
+    }
+}
+
 // ---------------------------------------------------------------- bf16 helpers (packed arithmetic)
 // The power-of-two scaling is one bf16x2 multiply per pair (exact; results that underflow are
 // far below the smallest code and round to a signed zero either way) and the sign bits come
@@ -305,25 +425,15 @@ struct GemmReady {
     StatusBlock* status; // zeroed here for the GEMM that follows
 };
 
+// One block of 32 bf16 values (x: sixteen pairs, element 0 in the low half of x[0]) -> its
+// codes, scale byte and index byte, stored as block number `blk`.
 template <int kMode, bool kReady>
-__global__ void __launch_bounds__(kThreads)
-quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
-                          uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
-                          uint8_t* __restrict__ bm_index, const GemmReady ready)
+__device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t blk,
+                                                    uint4* __restrict__ nibbles,
+                                                    uint8_t* __restrict__ scales,
+                                                    uint8_t* __restrict__ bm_index,
+                                                    const GemmReady& ready)
 {
-    const int64_t blk = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (kReady && blk == 0 && ready.status != nullptr) {
-        ready.status->code = 0u;
-        ready.status->where = 0u;
-    }
-    if (blk >= total_blocks) return;
-    const uint4* p = src + blk * 4;
-    uint32_t x[16];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint4 v = __ldg(p + i);
-        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
-    }
     uint32_t t[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) t[i] = x[i] & 0x7FFF7FFFu;
@@ -405,6 +515,79 @@ quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
         const int r = (int)(row & 127);
         ready.atoms[((row >> 7) * (ready.nbk >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)] =
             (uint8_t)sb;
+    }
+}
+
+template <int kMode, bool kReady>
+__global__ void __launch_bounds__(kThreads)
+quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
+                          uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
+                          uint8_t* __restrict__ bm_index, const GemmReady ready)
+{
+    const int64_t blk = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (kReady && blk == 0 && ready.status != nullptr) {
+        ready.status->code = 0u;
+        ready.status->where = 0u;
+    }
+    if (blk >= total_blocks) return;
+    const uint4* p = src + blk * 4;
+    uint32_t x[16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 v = __ldg(p + i);
+        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+    }
+    quantize_block_bf16<kMode, kReady>(x, blk, nibbles, scales, bm_index, ready);
+}
+
+// Channel reordering fused into the bf16 quantizer (Sec. 8, "Scattering outliers with channel
+// reordering"), one lane per block as above.  A CTA keeps the ordering in shared memory for
+// its whole life (clamped into the row once, and laid out so that the lanes of a warp read
+// neighbouring 16-byte vectors) and copies one source row at a time with coalesced 16-byte
+// loads; a lane then picks its block's 32 channels out of shared memory, where an arbitrary
+// ordering costs bank conflicts instead of a 128-byte line per element.  Rows are dealt to
+// the CTAs round robin; several CTAs per SM overlap one's row copy with another's casts.
+// Shared memory: cols ushort (the row) + cols ushort (the ordering; cols <= 65536).
+template <int kMode>
+__global__ void __launch_bounds__(kThreads)
+quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld_src, int64_t rows,
+                               int cols_blocks, const int32_t* __restrict__ order,
+                               uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
+                               uint8_t* __restrict__ bm_index)
+{
+    extern __shared__ uint4 dyn_smem[];
+    const int cols = cols_blocks * 32;
+    unsigned short* row_s = reinterpret_cast<unsigned short*>(dyn_smem);
+    unsigned short* ord_s = row_s + cols;
+    constexpr int kPerVec = 8;  // ordering entries per 16-byte vector
+    constexpr int kVecs = 4;    // vectors per block
+    // ordering entry e of block b sits in vector (e / kPerVec) * cols_blocks + b
+    const uint32_t last = (uint32_t)(cols - 1);
+    for (int c = threadIdx.x; c < cols; c += kThreads) {
+        const int b = c >> 5, e = c & 31;
+        ord_s[((e / kPerVec) * cols_blocks + b) * kPerVec + e % kPerVec] =
+            (unsigned short)min((uint32_t)__ldg(order + c), last);
+    }
+    const int vecs = cols / 8;
+    const GemmReady none{};
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const uint4* src_row = reinterpret_cast<const uint4*>(src + row * ld_src);
+        __syncthreads();  // the previous row has been read (first pass: the ordering is written)
+        for (int i = threadIdx.x; i < vecs; i += kThreads) dyn_smem[i] = ldg_stream(src_row + i);
+        __syncthreads();
+        for (int b = threadIdx.x; b < cols_blocks; b += kThreads) {
+            uint32_t x[16];
+#pragma unroll
+            for (int k = 0; k < kVecs; ++k) {
+                const uint4 o = reinterpret_cast<const uint4*>(ord_s)[k * cols_blocks + b];
+                const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    x[4 * k + i] = (uint32_t)row_s[ow[i] & 0xFFFFu] |
+                                   ((uint32_t)row_s[ow[i] >> 16] << 16);
+            }
+            quantize_block_bf16<kMode, false>(x, row * cols_blocks + b, nibbles, scales, bm_index, none);
+        }
     }
 }
 
@@ -492,7 +675,76 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
     return cudaGetLastError();
 }
 
+template <typename T, int kMode>
+cudaError_t launch_q_reordered(const void* src, int64_t rows, int64_t cols, int64_t ld_src,
+                               const int32_t* order, uint8_t* nibbles, uint8_t* scales,
+                               uint8_t* bm_index, cudaStream_t stream)
+{
+    const int64_t total_blocks = rows * (cols / 32);
+    const int64_t grid = (total_blocks + kBlocksPerCta - 1) / kBlocksPerCta;
+    const int aligned4 = ((reinterpret_cast<uintptr_t>(scales) & 3) == 0) &&
+                         ((reinterpret_cast<uintptr_t>(bm_index) & 3) == 0);
+    const size_t row_bytes = (size_t)cols * sizeof(T);
+    const bool vec_rows = (reinterpret_cast<uintptr_t>(src) & 15) == 0 &&
+                          (ld_src * sizeof(T)) % 16 == 0;
+    const int sms = sm_count();
+    if (sizeof(T) == 2 && vec_rows && sms > 0 && (reinterpret_cast<uintptr_t>(nibbles) & 15) == 0) {
+        // row and ordering as 16-bit entries: cols <= 51200 fits, wider rows take the path below
+        const size_t smem = (size_t)cols * 4;
+        if (smem <= 200 * 1024) {
+            int per_sm = (int)((200 * 1024) / smem);
+            if (per_sm > 6) per_sm = 6;
+            int64_t ctas = (int64_t)sms * per_sm;
+            if (ctas > rows) ctas = rows;
+            auto kern = quantize_bf16_reordered_kernel<kMode>;
+            static SmemAttrOnce once;
+            const cudaError_t ea = ensure_dynamic_smem(kern, 200 * 1024, once);
+            if (ea != cudaSuccess) return ea;
+            kern<<<(unsigned)ctas, kThreads, smem, stream>>>(
+                static_cast<const __nv_bfloat16*>(src), ld_src, rows, (int)(cols / 32), order,
+                reinterpret_cast<uint4*>(nibbles), scales, bm_index);
+            return cudaGetLastError();
+        }
+    }
+    if (vec_rows && row_bytes <= 200 * 1024 && sms > 0) {
+        auto kern = quantize_reordered_staged_kernel<T, kMode>;
+        static SmemAttrOnce once;
+        const cudaError_t ea = ensure_dynamic_smem(kern, 200 * 1024, once);
+        if (ea != cudaSuccess) return ea;
+        int per_sm = (int)((200 * 1024) / row_bytes);
+        if (per_sm > 6) per_sm = 6;
+        int64_t ctas = (int64_t)sms * per_sm;
+        if (ctas > rows) ctas = rows;
+        kern<<<(unsigned)ctas, kThreads, row_bytes, stream>>>(
+            static_cast<const T*>(src), ld_src, rows, (int)(cols / 32), order, nibbles, scales,
+            bm_index, aligned4 && (cols / 32) % 4 == 0);
+        return cudaGetLastError();
+    }
+    quantize_kernel<T, kMode, false, true><<<(unsigned)grid, kThreads, 0, stream>>>(
+        static_cast<const T*>(src), ld_src, cols / 32, total_blocks, nibbles, scales, bm_index,
+        aligned4, order);
+    return cudaGetLastError();
+}
+
 }  // namespace
+
+cudaError_t launch_quantize_reordered(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                                      int64_t ld_src, const int32_t* order, mxp_mode mode,
+                                      uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
+                                      cudaStream_t stream)
+{
+#define MXP_QR(T, MODE) \
+    launch_q_reordered<T, MODE>(src, rows, cols, ld_src, order, nibbles, scales, bm_index, stream)
+    if (dt == MXP_BF16) {
+        if (mode == MXP_MODE_MXFP4_PP) return MXP_QR(__nv_bfloat16, 2);
+        if (mode == MXP_MODE_MXFP4_PLUS) return MXP_QR(__nv_bfloat16, 1);
+        return MXP_QR(__nv_bfloat16, 0);
+    }
+    if (mode == MXP_MODE_MXFP4_PP) return MXP_QR(float, 2);
+    if (mode == MXP_MODE_MXFP4_PLUS) return MXP_QR(float, 1);
+    return MXP_QR(float, 0);
+#undef MXP_QR
+}
 
 // bf16, contiguous rows, MXFP4 / MXFP4+: quantize and write the GEMM-ready form as well.
 cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, mxp_mode mode,
