@@ -547,7 +547,7 @@ quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
 // loads; a lane then picks its block's 32 channels out of shared memory, where an arbitrary
 // ordering costs bank conflicts instead of a 128-byte line per element.  Rows are dealt to
 // the CTAs round robin; several CTAs per SM overlap one's row copy with another's casts.
-// Shared memory: cols ushort (the row) + cols ushort (the ordering; cols <= 65536).
+// Shared memory: two rows of cols ushort + cols ushort for the ordering (cols <= 65536).
 template <int kMode>
 __global__ void __launch_bounds__(kThreads)
 quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld_src, int64_t rows,
@@ -557,8 +557,9 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
 {
     extern __shared__ uint4 dyn_smem[];
     const int cols = cols_blocks * 32;
-    unsigned short* row_s = reinterpret_cast<unsigned short*>(dyn_smem);
-    unsigned short* ord_s = row_s + cols;
+    unsigned short* row_buf[2] = {reinterpret_cast<unsigned short*>(dyn_smem),
+                                  reinterpret_cast<unsigned short*>(dyn_smem) + cols};
+    unsigned short* ord_s = row_buf[1] + cols;
     constexpr int kPerVec = 8;  // ordering entries per 16-byte vector
     constexpr int kVecs = 4;    // vectors per block
     // ordering entry e of block b sits in vector (e / kPerVec) * cols_blocks + b
@@ -570,11 +571,26 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
     }
     const int vecs = cols / 8;
     const GemmReady none{};
-    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
-        const uint4* src_row = reinterpret_cast<const uint4*>(src + row * ld_src);
-        __syncthreads();  // the previous row has been read (first pass: the ordering is written)
-        for (int i = threadIdx.x; i < vecs; i += kThreads) dyn_smem[i] = ldg_stream(src_row + i);
-        __syncthreads();
+    // two row buffers filled with asynchronous 16-byte copies: the next row is on its way
+    // while this one is cast
+    auto fetch = [&](int64_t row, int buf) {
+        if (row < rows) {
+            const uint4* src_row = reinterpret_cast<const uint4*>(src + row * ld_src);
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(row_buf[buf]);
+            for (int i = threadIdx.x; i < vecs; i += kThreads)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i),
+                             "l"(src_row + i)
+                             : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    fetch(blockIdx.x, 0);
+    int it = 0;
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x, ++it) {
+        fetch(row + gridDim.x, (it + 1) & 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        __syncthreads();  // this row has landed for every thread (first pass: the ordering too)
+        const unsigned short* row_s = row_buf[it & 1];
         for (int b = threadIdx.x; b < cols_blocks; b += kThreads) {
             uint32_t x[16];
 #pragma unroll
@@ -588,7 +604,9 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
             }
             quantize_block_bf16<kMode, false>(x, row * cols_blocks + b, nibbles, scales, bm_index, none);
         }
+        __syncthreads();  // all reads of this buffer are done before the next pass refills it
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------- decode (Eq. 3)
@@ -689,8 +707,9 @@ cudaError_t launch_q_reordered(const void* src, int64_t rows, int64_t cols, int6
                           (ld_src * sizeof(T)) % 16 == 0;
     const int sms = sm_count();
     if (sizeof(T) == 2 && vec_rows && sms > 0 && (reinterpret_cast<uintptr_t>(nibbles) & 15) == 0) {
-        // row and ordering as 16-bit entries: cols <= 51200 fits, wider rows take the path below
-        const size_t smem = (size_t)cols * 4;
+        // two rows and the ordering as 16-bit entries: cols <= 34112 fits, wider rows take the
+        // path below
+        const size_t smem = (size_t)cols * 6;
         if (smem <= 200 * 1024) {
             int per_sm = (int)((200 * 1024) / smem);
             if (per_sm > 6) per_sm = 6;
