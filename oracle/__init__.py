@@ -64,6 +64,12 @@ def _load():
         lib.oracle_quantize_wide.restype = ci
         lib.oracle_dequantize_wide.argtypes = [p, p, p, i64, i64, ci, ci, ci, p, i64]
         lib.oracle_dequantize_wide.restype = ci
+        lib.oracle_nvfp4_quantize.argtypes = [p, ci, i64, i64, ctypes.c_float, ci, p, p, p]
+        lib.oracle_nvfp4_quantize.restype = ci
+        lib.oracle_nvfp4_dequantize.argtypes = [p, p, p, i64, i64, ctypes.c_float, ci, p]
+        lib.oracle_nvfp4_dequantize.restype = ci
+        lib.oracle_e4m3_round.argtypes = [ctypes.c_float]
+        lib.oracle_e4m3_round.restype = ci
         lib.oracle_pack6.argtypes = [p, i64, p]
         lib.oracle_pack6.restype = None
         lib.oracle_set_threads.argtypes = [ci]
@@ -254,3 +260,47 @@ def quantize_reordered(x: np.ndarray, order: np.ndarray, mode: int, bf16_bits: b
     definition is quantize(x[:, order])."""
     return quantize(np.ascontiguousarray(np.asarray(x)[:, np.asarray(order, np.int64)]), mode,
                     bf16_bits=bf16_bits)
+
+
+def e4m3_round(q: float) -> int:
+    """E4M3 byte (sign 0) nearest to q >= 0: ties to even, saturating at 448."""
+    return int(_load().oracle_e4m3_round(float(q)))
+
+
+def nvfp4_quantize(x: np.ndarray, tensor_scale: float, plus: bool, bf16_bits: bool = False):
+    """NVFP4 / NVFP4+ (Sec. 8, "Applicability of MX+ to NVFP4"): blocks of 16, E4M3 block
+    scale over the fp32 `tensor_scale`.  Returns (nibbles[rows, cols/2], scales[rows, cols/16],
+    bm_index[rows, cols/32]: two 4-bit indices per byte, zero for plain NVFP4)."""
+    assert x.ndim == 2
+    x = np.ascontiguousarray(x)
+    if bf16_bits:
+        assert x.dtype == np.uint16
+        kind = 1
+    else:
+        assert x.dtype == np.float32
+        kind = 0
+    rows, cols = x.shape
+    if cols % 32:
+        raise ValueError("cols must be a multiple of 32")
+    nib = np.zeros((rows, cols // 2), np.uint8)
+    sc = np.zeros((rows, cols // 16), np.uint8)
+    idx = np.zeros((rows, cols // 32), np.uint8)
+    rc = _load().oracle_nvfp4_quantize(_ptr(x), kind, rows, cols, float(tensor_scale), int(plus),
+                                       _ptr(nib), _ptr(sc), _ptr(idx))
+    if rc != 0:
+        raise ValueError("oracle_nvfp4_quantize rejected its arguments")
+    return nib, sc, idx
+
+
+def nvfp4_dequantize(nib: np.ndarray, sc: np.ndarray, idx, tensor_scale: float, plus: bool) -> np.ndarray:
+    """Decoded values as float32 (the definition rounds once to binary32)."""
+    nib = np.ascontiguousarray(nib, np.uint8)
+    sc = np.ascontiguousarray(sc, np.uint8)
+    rows, cols = nib.shape[0], nib.shape[1] * 2
+    idx = np.zeros((rows, cols // 32), np.uint8) if idx is None else np.ascontiguousarray(idx, np.uint8)
+    out = np.zeros((rows, cols), np.float32)
+    rc = _load().oracle_nvfp4_dequantize(_ptr(nib), _ptr(sc), _ptr(idx), rows, cols,
+                                         float(tensor_scale), int(plus), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_nvfp4_dequantize rejected its arguments")
+    return out

@@ -483,6 +483,129 @@ void oracle_pack6(const uint8_t *codes, int64_t n, uint8_t *out)
     }
 }
 
+/* ------------------------------------------------------------------------------------------
+ * NVFP4 / NVFP4+ (Sec. 8, "Applicability of MX+ to NVFP4"): E2M1 elements in blocks of 16
+ * with an E4M3 block scale on top of one fp32 scale for the whole tensor.  The scale maps the
+ * block's largest magnitude (the BM) onto the largest E2M1 magnitude, 6, so the BM's exponent
+ * field is at its maximum and, as in MX+, can be spent on mantissa: NVFP4+ stores the BM as
+ * sign + three mantissa bits, value 4 + m/2, and adds a 4-bit BM index per block.  Blocks whose
+ * scale byte is 00000010b or smaller keep the plain NVFP4 form (their scale is too coarse for
+ * the BM to land in [4, 8) reliably); their index nibble is 0.
+ *
+ * The passage fixes neither the arithmetic nor the layout.  Readings taken here:
+ *   - all scale arithmetic is IEEE binary32, one rounding per step, in this order:
+ *       q = amax / (6 * ts)          (the product 6 * ts rounded first, then the division)
+ *       scale byte = E4M3(q), round to nearest, ties to even, saturating at 448
+ *       d = value(scale byte) * ts ; r = 1 / d ; scaled_i = x_i * r
+ *   - scaled_i -> E2M1, round to nearest, ties to even code, saturating at 6; the sign bit of
+ *     the input is kept even when the magnitude rounds to zero;
+ *   - scale byte 0 (amax too small for the tensor scale): all codes 0, index 0;
+ *   - BM = first element with the largest magnitude; m = round-to-nearest-even((v - 4) * 2)
+ *     with v = amax * r, clamped to 0..7 (v can leave [4, 8) only when the scale saturated);
+ *   - element 2j in the low nibble of byte j; one scale byte per block; index nibbles two per
+ *     byte, block 2j of a row in the low nibble (cols % 32 == 0 keeps rows byte aligned);
+ *   - decode: x_i = +-E_i * d with d as above and one binary32 rounding of the product.
+ * Parity unpinned: Inf / NaN inputs, ts <= 0.
+ * ------------------------------------------------------------------------------------------ */
+static float f32_mul(float a, float b) { volatile float r = a * b; return r; }
+static float f32_div(float a, float b) { volatile float r = a / b; return r; }
+
+/* E4M3 byte (sign 0) nearest to q >= 0, saturating: the search over the type's 127 finite
+ * magnitudes used for MXFP8 elements above. */
+int oracle_e4m3_round(float q) { return elem_nearest(ORACLE_FMT_E4M3, (double)q); }
+
+static void nvfp4_block(const float *x, float ts, int plus, uint8_t *nib, uint8_t *scale,
+                        int *index)
+{
+    float amax = 0.0f;
+    int bm = 0;
+    for (int i = 0; i < 16; ++i) {
+        float a = fabsf(x[i]);
+        if (a > amax) {
+            amax = a;
+            bm = i;
+        }
+    }
+    float q = f32_div(amax, f32_mul(6.0f, ts));
+    int sb = oracle_e4m3_round(q);
+    *scale = (uint8_t)sb;
+    *index = 0;
+    memset(nib, 0, 8);
+    if (sb == 0)
+        return;
+    float d = f32_mul((float)oracle_elem_value(ORACLE_FMT_E4M3, sb), ts);
+    float r = f32_div(1.0f, d);
+    int extend = plus && sb > 2;
+    for (int i = 0; i < 16; ++i) {
+        float sc = f32_mul(x[i], r);
+        int code;
+        if (extend && i == bm)
+            code = bm_code(fmin(fmax((double)fabsf(sc), 4.0), 8.0));
+        else
+            code = e2m1_nearest((double)fabsf(sc));
+        if (signbit(x[i]))
+            code |= 8;
+        nib[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
+    }
+    if (extend)
+        *index = bm;
+}
+
+/* src_kind as in oracle_quantize (0 float32, 1 bfloat16 bits).  Planes: nibbles rows*cols/2,
+ * scales rows*cols/16, bm_index rows*cols/32 (written in both modes; zero for NVFP4). */
+int oracle_nvfp4_quantize(const void *src, int src_kind, int64_t rows, int64_t cols, float ts,
+                          int plus, uint8_t *nibbles, uint8_t *scales, uint8_t *bm_index)
+{
+    if (rows < 0 || cols < 0 || cols % 32 != 0 || (src_kind != 0 && src_kind != 1))
+        return -1;
+    int64_t nb = cols / 16;
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < nb; ++b) {
+            float x[16];
+            for (int i = 0; i < 16; ++i) {
+                int64_t e = r * cols + b * 16 + i;
+                x[i] = src_kind == 0 ? ((const float *)src)[e]
+                                     : (float)bf16_to_double(((const uint16_t *)src)[e]);
+            }
+            int idx;
+            nvfp4_block(x, ts, plus, nibbles + (r * nb + b) * 8, scales + r * nb + b, &idx);
+            uint8_t *ib = bm_index + (r * nb + b) / 2;
+            if (b & 1)
+                *ib = (uint8_t)((*ib & 0x0F) | (idx << 4));
+            else
+                *ib = (uint8_t)idx;
+        }
+    }
+    return 0;
+}
+
+int oracle_nvfp4_dequantize(const uint8_t *nibbles, const uint8_t *scales,
+                            const uint8_t *bm_index, int64_t rows, int64_t cols, float ts,
+                            int plus, float *out)
+{
+    if (rows < 0 || cols < 0 || cols % 32 != 0)
+        return -1;
+    int64_t nb = cols / 16;
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < nb; ++b) {
+            int sb = scales[r * nb + b];
+            float d = f32_mul((float)oracle_elem_value(ORACLE_FMT_E4M3, sb & 127), ts);
+            int extend = plus && sb > 2;
+            int bm = (bm_index[(r * nb + b) / 2] >> (4 * (b & 1))) & 15;
+            for (int i = 0; i < 16; ++i) {
+                int code = (nibbles[(r * nb + b) * 8 + i / 2] >> (4 * (i & 1))) & 15;
+                double mag = (extend && i == bm) ? 4.0 + 0.5 * (code & 7)
+                                                 : oracle_e2m1_value(code & 7);
+                float v = f32_mul((float)mag, d);
+                out[r * cols + b * 16 + i] = (code & 8) ? -v : v;
+            }
+        }
+    }
+    return 0;
+}
+
 /* D[m][n] = sum_k A[m][k] * B[n][k], fp64, k ascending.  A is M x K, B is N x K. */
 void oracle_gemm_fp64(const double *A, int64_t lda, const double *B, int64_t ldb,
                       int64_t M, int64_t N, int64_t K, double *D, int64_t ldd)

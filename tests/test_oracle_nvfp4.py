@@ -1,0 +1,141 @@
+"""Pins for the NVFP4 / NVFP4+ oracle (Sec. 8, "Applicability of MX+ to NVFP4"); no GPU."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2510_14557_b200 import synth
+
+E4M3 = oracle.FMT_E4M3
+E2M1 = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+
+
+def nib_codes(nib):
+    return np.stack([nib & 15, nib >> 4], axis=-1).reshape(nib.shape[0], -1)
+
+
+def idx_nibbles(idx):
+    return np.stack([idx & 15, idx >> 4], axis=-1).reshape(idx.shape[0], -1)
+
+
+def test_e4m3_scale_cast_against_a_library_cast():
+    # torch's float8_e4m3fn cast is an independent implementation of the same rounding
+    g = synth.rng(1)
+    q = np.concatenate([np.exp2(g.uniform(-12, 8.8, 4000)), np.arange(0, 448, 0.37),
+                        [0.0, 2.0 ** -10, 2.0 ** -9, 3 * 2.0 ** -10, 448.0, 447.9, 15.5, 17.0, 18.0]]).astype(np.float32)
+    q = q[q <= 448.0]
+    want = torch.from_numpy(q).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = np.array([oracle.e4m3_round(v) for v in q], np.uint8)
+    assert np.array_equal(got, want)
+    # beyond the largest finite value: saturates (0x7E = 448), never the NaN pattern
+    assert oracle.e4m3_round(500.0) == 0x7E and oracle.e4m3_round(1e9) == 0x7E
+    # decode of every byte against the same library
+    vals = torch.arange(0, 127, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy()
+    assert all(oracle.elem_value(E4M3, c) == float(vals[c]) for c in range(127))
+
+
+def test_hand_example():
+    # tensor scale 1, largest magnitude 6: q = 1, scale byte 0x38 (1.0), values are their own codes
+    x = np.zeros((1, 32), np.float32)
+    x[0, :6] = [3.0, -1.5, 0.5, 6.0, -0.2, 0.8]
+    x[0, 16:20] = [0.75, -12.0, 5.0, 11.0]   # second block: amax 12 -> q = 2, scale 2.0 (0x40)
+    for plus in (False, True):
+        nib, sc, idx = oracle.nvfp4_quantize(x, 1.0, plus)
+        assert sc.tolist() == [[0x38, 0x40]]
+        c = nib_codes(nib)[0]
+        #      3.0  -1.5   0.5  6.0(BM)              -0.2 -> -0 ; 0.8 -> 1.0 (nearer than 0.5)
+        assert c[:6].tolist() == [5, 0x8 | 3, 1, 4 if plus else 7, 0x8, 2]
+        # second block, scaled by 1/2: 0.375 -> 0.5 ; -6 (BM) ; 2.5 -> tie -> 2.0 ; 5.5 -> 6
+        assert c[16:20].tolist() == [1, 0x8 | (4 if plus else 7), 4, 7]
+        assert idx.tolist() == [[3 | (1 << 4)]] if plus else idx.tolist() == [[0]]
+        d = oracle.nvfp4_dequantize(nib, sc, idx, 1.0, plus)
+        assert d[0, 3] == 6.0 and d[0, 17] == -12.0 and d[0, 19] == 12.0 and d[0, 18] == 4.0
+
+
+def test_bm_gains_mantissa_and_nothing_else_changes():
+    g = synth.rng(7)
+    x = (g.standard_normal((64, 256)) * np.exp2(g.integers(-6, 6, (64, 1)))).astype(np.float32)
+    ts = float(np.abs(x).max() / (6 * 448))
+    n0, s0, i0 = oracle.nvfp4_quantize(x, ts, False)
+    n1, s1, i1 = oracle.nvfp4_quantize(x, ts, True)
+    assert np.array_equal(s0, s1) and not i0.any()
+    c0, c1 = nib_codes(n0), nib_codes(n1)
+    bm = idx_nibbles(i1)
+    blocks = np.arange(256) // 16
+    is_bm = (np.arange(256)[None, :] % 16) == bm[:, blocks]
+    ext = (s1 > 2)[:, blocks]
+    assert np.array_equal(c0[~(is_bm & ext)], c1[~(is_bm & ext)])          # NBMs identical
+    # the BM of an extended block is the first largest magnitude of its block
+    xa = np.abs(x).reshape(64, 16, 16)
+    assert np.array_equal(bm[s1 > 2], xa.argmax(axis=2)[s1 > 2])
+    # and it is represented at least as well as before; the scaled BM sits near 6
+    d0 = oracle.nvfp4_dequantize(n0, s0, i0, ts, False).astype(np.float64)
+    d1 = oracle.nvfp4_dequantize(n1, s1, i1, ts, True).astype(np.float64)
+    e0, e1 = np.abs(d0 - x), np.abs(d1 - x)
+    assert np.all(e1[is_bm & ext] <= e0[is_bm & ext] + 1e-12)
+    # (the gain is modest by construction: the scale already puts the BM within 6.25 % of 6,
+    # so the finer grid 5.5 / 6 / 6.5 only helps the BMs that land more than 0.25 away from 6)
+    assert e1[is_bm & ext].mean() < e0[is_bm & ext].mean()
+    assert (e1[is_bm & ext] < e0[is_bm & ext]).mean() > 0.05
+    scale = np.array([oracle.elem_value(E4M3, int(b)) for b in s1.reshape(-1)]).reshape(s1.shape) * ts
+    v = xa.max(axis=2) / scale
+    normal = s1 >= 8
+    assert v[normal].min() > 6 / 1.0626 and v[normal].max() < 6 / 0.9374
+
+
+def test_coarse_scales_fall_back_to_plain_nvfp4():
+    # blocks whose scale byte is 0, 1 or 2 keep the plain form and index 0
+    x = np.zeros((1, 128), np.float32)
+    x[0, 0::16] = [1.0, 2.0 ** -9 * 6, 2.0 ** -9 * 12, 2.0 ** -9 * 18, 2.0 ** -9 * 24, 2.0 ** -20, 0.0, 3.0]
+    x[0, 1::16] = x[0, 0::16] * 0.5
+    n0, s0, i0 = oracle.nvfp4_quantize(x, 1.0, False)
+    n1, s1, i1 = oracle.nvfp4_quantize(x, 1.0, True)
+    assert s1[0].tolist() == [oracle.e4m3_round(1 / 6), 1, 2, 3, 4, 0, 0, 0x30]
+    c0, c1 = nib_codes(n0)[0], nib_codes(n1)[0]
+    for b, sb in enumerate(s1[0]):
+        same = np.array_equal(c0[16 * b:16 * b + 16], c1[16 * b:16 * b + 16])
+        assert same == (sb <= 2)
+    assert not nib_codes(n1)[0][80:112].any()        # scale byte 0: everything flushed
+    assert idx_nibbles(i1)[0].tolist() == [0] * 8    # every BM here is element 0 anyway
+    x[0, 5] = 2.0 ** -9 * 12.5                       # block 0.. move a BM: block 2 stays plain
+    x2 = np.roll(x, 3, axis=1)
+    _, s2, i2 = oracle.nvfp4_quantize(x2, 1.0, True)
+    assert idx_nibbles(i2)[0][0] == 3 and idx_nibbles(i2)[0][1] == 0 and s2[0, 1] <= 2
+
+
+def test_element_rounding_against_a_nearest_search():
+    # scale byte 0x38 (1.0) and tensor scale 1: scaled values are the inputs; every multiple
+    # of 1/16 up to 6 next to a 6.0 that pins the scale
+    vals = np.arange(0, 97) / 16.0
+    for v in vals:
+        x = np.zeros((1, 32), np.float32)
+        x[0, 0], x[0, 1], x[0, 2] = 6.0, v, -v
+        nib, sc, _ = oracle.nvfp4_quantize(x, 1.0, False)
+        assert sc[0, 0] == 0x38
+        d = [abs(v - t) for t in E2M1]
+        best = min(range(8), key=lambda c: (d[c], c & 1))   # nearest, ties to the even code
+        c = nib_codes(nib)[0]
+        assert c[1] == best and c[2] == (8 | best)
+
+
+def test_round_trip_of_representable_blocks():
+    # values already on the grid of their block come back exactly: the BM is 6 times a power of
+    # two (scale exactly representable, BM code 7 resp. m = 4), every other element a smaller
+    # E2M1 value times the same scale; all binary32 products are exact here
+    g = synth.rng(3)
+    ts = 2.0 ** -3
+    grid = np.array(E2M1[:7] + [-t for t in E2M1[:7]], np.float32)     # magnitudes up to 4
+    for plus in (False, True):
+        x = grid[g.integers(0, 14, (32, 64))]
+        pos = g.integers(0, 16, (32, 4))
+        for r in range(32):
+            for b in range(4):
+                x[r, 16 * b + pos[r, b]] = 6.0 if (r + b) & 1 else -6.0
+        s = np.exp2(g.integers(-4, 5, (32, 4))).astype(np.float32)
+        x = x * np.repeat(s, 16, axis=1) * np.float32(ts)
+        q = oracle.nvfp4_quantize(x, ts, plus)
+        assert np.array_equal(oracle.nvfp4_dequantize(q[0], q[1], q[2], ts, plus), x)
+        if plus:
+            assert np.array_equal(idx_nibbles(q[2]), pos.astype(np.uint8))
+            c = nib_codes(q[0]).reshape(32, 4, 16)
+            bmc = np.take_along_axis(c, pos[..., None], axis=2)[..., 0]
+            assert set((bmc & 7).reshape(-1).tolist()) == {4}
