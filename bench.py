@@ -233,6 +233,12 @@ def part_quantize(mxp, synth, peaks, iters):
         nbytes = n * (2 + mxp.binding.element_bits(mode) / 8 + 1 / 32 + (1 / 32 if buf.bm_index is not None else 0))
         gbs = nbytes / ms / 1e6
         out["quantize_cfg2_" + name] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
+    # ---- NVFP4 / NVFP4+ (blocks of 16, E4M3 scale): 2 B in, 4 bits + 1/16 B (+ 1/32 B) out
+    for name, plus in (("nvfp4+", True), ("nvfp4", False)):
+        ms = time_loop(lambda: mxp.mxp_nvfp4_quantize(x, 2.0 ** -8, plus), iters)
+        nbytes = n * (2 + 0.5 + 1 / 16 + (1 / 32 if plus else 0))
+        gbs = nbytes / ms / 1e6
+        out["quantize_cfg2_" + name] = {"us": ms * 1e3, "GB/s": gbs, "frac_hbm": gbs / hbm}
     # ---- the same with channel reordering fused in: ordering built by the library's rule from
     # per-channel outlier counts (|x| > 3 sigma) of a 512-row sample of the input
     sample = x[:512].float()

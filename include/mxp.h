@@ -125,6 +125,42 @@ mxp_status mxp_quantize_reordered(const void *src, mxp_dtype src_dt, int64_t row
 mxp_status mxp_channel_order(const int64_t *outlier_count, int64_t cols, int32_t *order);
 
 /*
+ * NVFP4 and NVFP4+ (Sec. 8, "Applicability of MX+ to NVFP4").  NVFP4: E2M1 elements in blocks
+ * of 16 along the row, one E4M3 scale byte per block, one fp32 scale for the tensor.  NVFP4+
+ * gives the block's largest-magnitude element (BM) three mantissa bits in place of its
+ * exponent and mantissa bits (value 4 + m/2 times the block's scale, as in MXFP4+) and stores
+ * a 4-bit BM index per block; blocks whose scale byte is 00000010b or less keep the plain
+ * NVFP4 form and index 0.
+ *
+ *   tensor_scale  the per-tensor fp32 scale, chosen by the caller, > 0 and finite (the usual
+ *                 choice: largest magnitude of the tensor / (6 * 448), so that block scales
+ *                 use the E4M3 range; a larger value pushes more blocks into the fallback)
+ *   plus          0: NVFP4, != 0: NVFP4+
+ *   nibbles       rows*cols/2 bytes, element 2j of a row in the low nibble of byte j
+ *   scales        rows*cols/16 bytes, E4M3 (sign bit 0), row-major; 2-byte aligned
+ *   bm_index      rows*cols/32 bytes: two 4-bit indices per byte, the even block of a row in
+ *                 the low nibble; NULL allowed iff plus == 0 (then not written / not read)
+ *   cols % 32 == 0; src / dst rows 16-byte aligned (ld % 8 == 0), nibbles 16-byte aligned.
+ *
+ * What is computed, each step one IEEE binary32 operation (the paper fixes none; the CPU
+ * oracle of the test suite follows the same steps, so the codes are bit-exact):
+ *   q = amax / (6 * tensor_scale);  scale byte = E4M3(q), round to nearest even, saturating
+ *   at 448;  d = value(scale byte) * tensor_scale;  r = 1 / d;  element codes = E2M1(x * r),
+ *   round to nearest even, saturating at 6, sign of x kept;  scale byte 0: all codes 0;
+ *   BM (first of equal maxima), NVFP4+ only: m = nearest-even((clamp(amax * r, 4, 8) - 4) * 2),
+ *   at most 7.  Decode: x = +-E * d, E the E2M1 value or 4 + m/2, one rounding to binary32
+ *   (then to bf16, nearest even, for a bf16 destination).
+ * Inf / NaN inputs are outside the contract.
+ */
+mxp_status mxp_nvfp4_quantize(const void *src, mxp_dtype src_dt, int64_t rows, int64_t cols,
+                              int64_t ld_src, float tensor_scale, int plus, uint8_t *nibbles,
+                              uint8_t *scales, uint8_t *bm_index, void *cuda_stream);
+mxp_status mxp_nvfp4_dequantize(const uint8_t *nibbles, const uint8_t *scales,
+                                const uint8_t *bm_index, int64_t rows, int64_t cols,
+                                float tensor_scale, int plus, void *dst, mxp_dtype dst_dt,
+                                int64_t ld_dst, void *cuda_stream);
+
+/*
  * Decode (Eq. 3): dst[r][c] = (-1)^s * 2^(scale - 127) * E, E = 4 + m/2 for the BM
  * element of an MXFP4+ block, the E2M1 value otherwise.  Exact in both output types.
  *   p       host pointer to the operand descriptor (its planes are device memory)

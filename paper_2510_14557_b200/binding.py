@@ -25,7 +25,7 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
            "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_noalloc.restype = ci
         l.mxp_quantize_reordered.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp, vp, vp, vp]
         l.mxp_quantize_reordered.restype = ci
+        l.mxp_nvfp4_quantize.argtypes = [vp, ci, i64, i64, i64, ctypes.c_float, ci, vp, vp, vp, vp]
+        l.mxp_nvfp4_quantize.restype = ci
+        l.mxp_nvfp4_dequantize.argtypes = [vp, vp, vp, i64, i64, ctypes.c_float, ci, vp, ci, i64, vp]
+        l.mxp_nvfp4_dequantize.restype = ci
         l.mxp_channel_order.argtypes = [vp, i64, vp]
         l.mxp_channel_order.restype = ci
         l.mxp_gemm_decode_chained.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, ci,
@@ -186,6 +190,33 @@ def mxp_quantize_reordered(src: torch.Tensor, order: torch.Tensor, mode: int,
                                       out.bm_index.data_ptr() if out.bm_index is not None else None,
                                       _stream())
     _check("mxp_quantize_reordered", st)
+    return out
+
+
+def mxp_nvfp4_quantize(src: torch.Tensor, tensor_scale: float, plus: bool):
+    """NVFP4 / NVFP4+ of a 2-D CUDA tensor: returns (nibbles, scales, bm_index or None) as uint8
+    tensors [rows, cols/2], [rows, cols/16], [rows, cols/32]."""
+    assert src.is_cuda and src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    nib = torch.empty((rows, cols // 2), dtype=torch.uint8, device=src.device)
+    sc = torch.empty((rows, cols // 16), dtype=torch.uint8, device=src.device)
+    idx = torch.empty((rows, cols // 32), dtype=torch.uint8, device=src.device) if plus else None
+    st = lib().mxp_nvfp4_quantize(src.data_ptr(), _dt(src), rows, cols, src.stride(0),
+                                  float(tensor_scale), int(plus), nib.data_ptr(), sc.data_ptr(),
+                                  idx.data_ptr() if plus else None, _stream())
+    _check("mxp_nvfp4_quantize", st)
+    return nib, sc, idx
+
+
+def mxp_nvfp4_dequantize(nib: torch.Tensor, sc: torch.Tensor, idx: Optional[torch.Tensor],
+                         tensor_scale: float, plus: bool, dtype=torch.float32) -> torch.Tensor:
+    rows, cols = nib.shape[0], nib.shape[1] * 2
+    out = torch.empty((rows, cols), dtype=dtype, device=nib.device)
+    st = lib().mxp_nvfp4_dequantize(nib.data_ptr(), sc.data_ptr(),
+                                    idx.data_ptr() if idx is not None else None, rows, cols,
+                                    float(tensor_scale), int(plus), out.data_ptr(), _dt(out),
+                                    out.stride(0), _stream())
+    _check("mxp_nvfp4_dequantize", st)
     return out
 
 

@@ -101,6 +101,43 @@ mxp_status mxp_quantize_reordered(const void* src, mxp_dtype src_dt, int64_t row
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }
 
+mxp_status mxp_nvfp4_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t cols,
+                              int64_t ld_src, float tensor_scale, int plus, uint8_t* nibbles,
+                              uint8_t* scales, uint8_t* bm_index, void* cuda_stream)
+{
+    if (!valid_dtype(src_dt) || rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!(tensor_scale > 0.f) || !(tensor_scale < 3.0e38f)) return MXP_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return MXP_OK;
+    if (src == nullptr || nibbles == nullptr || scales == nullptr) return MXP_ERR_INVALID_ARG;
+    if (plus && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (ld_src < cols || ld_src % 8 != 0) return MXP_ERR_INVALID_ARG;
+    if (!aligned(src, 16) || !aligned(nibbles, 16) || !aligned(scales, 2)) return MXP_ERR_INVALID_ARG;
+    if (rows * (cols / 32) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    cudaError_t e = mxp::launch_nvfp4_quantize(src, src_dt, rows, cols, ld_src, tensor_scale,
+                                               plus != 0, nibbles, scales, bm_index,
+                                               static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+mxp_status mxp_nvfp4_dequantize(const uint8_t* nibbles, const uint8_t* scales,
+                                const uint8_t* bm_index, int64_t rows, int64_t cols,
+                                float tensor_scale, int plus, void* dst, mxp_dtype dst_dt,
+                                int64_t ld_dst, void* cuda_stream)
+{
+    if (!valid_dtype(dst_dt) || rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!(tensor_scale > 0.f) || !(tensor_scale < 3.0e38f)) return MXP_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return MXP_OK;
+    if (nibbles == nullptr || scales == nullptr || dst == nullptr) return MXP_ERR_INVALID_ARG;
+    if (plus && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+    if (!aligned(nibbles, 4) || !aligned(dst, 16) || ld_dst < cols || ld_dst % 8 != 0)
+        return MXP_ERR_INVALID_ARG;
+    if (rows * (cols / 8) / 256 + 1 > 0x7FFFFFFFll) return MXP_ERR_UNSUPPORTED;
+    cudaError_t e = mxp::launch_nvfp4_dequantize(nibbles, scales, bm_index, rows, cols, tensor_scale,
+                                                 plus != 0, dst, dst_dt, ld_dst,
+                                                 static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
 mxp_status mxp_channel_order(const int64_t* outlier_count, int64_t cols, int32_t* order)
 {
     if (outlier_count == nullptr || order == nullptr) return MXP_ERR_INVALID_ARG;

@@ -19,6 +19,14 @@ cudaError_t launch_quantize_reordered(const void* src, mxp_dtype dt, int64_t row
                                       uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
                                       cudaStream_t stream);
 
+cudaError_t launch_nvfp4_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                                  int64_t ld_src, float ts, bool plus, uint8_t* nibbles,
+                                  uint8_t* scales, uint8_t* bm_index, cudaStream_t stream);
+cudaError_t launch_nvfp4_dequantize(const uint8_t* nibbles, const uint8_t* scales,
+                                    const uint8_t* bm_index, int64_t rows, int64_t cols, float ts,
+                                    bool plus, void* dst, mxp_dtype dt, int64_t ld_dst,
+                                    cudaStream_t stream);
+
 cudaError_t launch_dequantize(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
                               cudaStream_t stream);
 

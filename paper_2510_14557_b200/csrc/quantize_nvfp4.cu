@@ -1,0 +1,224 @@
+// NVFP4 / NVFP4+ quantize and decode (Sec. 8, "Applicability of MX+ to NVFP4").
+//
+// NVFP4: E2M1 elements in blocks of 16, an E4M3 scale per block, one fp32 scale `ts` for the
+// tensor.  The block scale is amax / (6 ts) rounded to E4M3, which puts the block's largest
+// magnitude (the BM) next to 6, the top of the E2M1 range: its exponent field is at its
+// maximum, so, as in MX+, NVFP4+ spends the BM's exponent bits on mantissa (value 4 + m/2,
+// m = 0..7) and stores a 4-bit BM index per block.  Blocks whose scale byte is 2 or less keep
+// the plain form (index nibble 0).
+//
+// Arithmetic (the passage fixes none; every step is one IEEE binary32 operation, so that the
+// codes are reproducible):  q = amax / (6 ts);  byte = E4M3(q), nearest-even, saturating;
+// d = value(byte) * ts;  r = 1 / d;  scaled = x * r;  code = E2M1(scaled), nearest-even,
+// saturating, sign of the input kept;  BM: m = nearest-even((clamp(amax * r, 4, 8) - 4) * 2),
+// at most 7.  Decode: +-E * d with one rounding.
+//
+// HBM-bound: one lane owns 32 consecutive elements (two blocks): 64 or 128 bytes in, 16 bytes
+// of codes, two scale bytes and one index byte out, all as full-width coalesced accesses.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace mxp {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint32_t f32_to_e4m3_byte(float q)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.f), "f"(q));
+    return (uint32_t)r & 0xFFu;
+}
+__device__ __forceinline__ float e4m3_byte_to_f32(uint32_t b)
+{
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)b));
+    return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
+__device__ __forceinline__ uint32_t cvt_e2m1x8(const float* f)
+{
+    uint32_t r;
+    asm("{ .reg .b8 b0, b1, b2, b3;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n"
+        "  mov.b32 %0, {b0, b1, b2, b3}; }"
+        : "=r"(r)
+        : "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "f"(f[4]), "f"(f[5]), "f"(f[6]), "f"(f[7]));
+    return r;
+}
+
+// One block of 16: two words of codes, the scale byte and the BM index (0 when not extended).
+template <bool kPlus>
+__device__ __forceinline__ void nvfp4_block(const float* x, float ts, float six_ts, uint32_t& w0,
+                                            uint32_t& w1, uint32_t& scale_byte, uint32_t& index)
+{
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(x[i]));
+    int bm = 0;
+#pragma unroll
+    for (int i = 15; i >= 0; --i)
+        if (fabsf(x[i]) == amax) bm = i;  // the first of equal maxima
+    const uint32_t sb = f32_to_e4m3_byte(__fdiv_rn(amax, six_ts));
+    const float d = __fmul_rn(e4m3_byte_to_f32(sb), ts);
+    const float r = __frcp_rn(d);
+    float s[16];
+    uint32_t sign = 0, sign1 = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        sign |= (__float_as_uint(x[i]) >> 31) << (4 * i + 3);
+        sign1 |= (__float_as_uint(x[8 + i]) >> 31) << (4 * i + 3);
+    }
+    w0 = (cvt_e2m1x8(s) & 0x77777777u) | sign;
+    w1 = (cvt_e2m1x8(s + 8) & 0x77777777u) | sign1;
+    index = 0;
+    if (kPlus && sb > 2u) {
+        const float v = fminf(fmaxf(__fmul_rn(amax, r), 4.f), 8.f);
+        const uint32_t m = (uint32_t)min(__float2int_rn((v - 4.f) * 2.f), 7);
+        const uint32_t sh = (uint32_t)(bm & 7) * 4u;
+        if (bm < 8) w0 = (w0 & ~(7u << sh)) | (m << sh);
+        else w1 = (w1 & ~(7u << sh)) | (m << sh);
+        index = (uint32_t)bm;
+    }
+    if (sb == 0u) w0 = w1 = 0u;
+    scale_byte = sb;
+}
+
+template <typename T, bool kPlus>
+__global__ void __launch_bounds__(kThreads)
+nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_per_row,
+                      int64_t total_units, float ts, uint4* __restrict__ nibbles,
+                      uint16_t* __restrict__ scales, uint8_t* __restrict__ bm_index)
+{
+    const int64_t u = (int64_t)blockIdx.x * kThreads + threadIdx.x;  // unit of 32 elements
+    if (u >= total_units) return;
+    const int64_t row = u / units_per_row;
+    const T* p = src + row * ld_src + (u - row * units_per_row) * 32;
+    float x[32];
+    if (sizeof(T) == 2) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p) + i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                x[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+                x[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p) + i);
+            x[4 * i] = __uint_as_float(v.x);
+            x[4 * i + 1] = __uint_as_float(v.y);
+            x[4 * i + 2] = __uint_as_float(v.z);
+            x[4 * i + 3] = __uint_as_float(v.w);
+        }
+    }
+    const float six_ts = __fmul_rn(6.f, ts);
+    uint32_t w[4], sb0, sb1, i0, i1;
+    nvfp4_block<kPlus>(x, ts, six_ts, w[0], w[1], sb0, i0);
+    nvfp4_block<kPlus>(x + 16, ts, six_ts, w[2], w[3], sb1, i1);
+    __stcs(nibbles + u, make_uint4(w[0], w[1], w[2], w[3]));
+    scales[u] = (uint16_t)(sb0 | (sb1 << 8));
+    if (kPlus) bm_index[u] = (uint8_t)(i0 | (i1 << 4));
+}
+
+// One thread decodes eight elements (one word of codes, half a block).
+template <typename T, bool kPlus>
+__global__ void __launch_bounds__(kThreads)
+nvfp4_dequantize_kernel(const uint32_t* __restrict__ nibbles, const uint8_t* __restrict__ scales,
+                        const uint8_t* __restrict__ bm_index, int64_t cols, int64_t total_words,
+                        float ts, T* __restrict__ dst, int64_t ld_dst)
+{
+    const int64_t u = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (u >= total_words) return;
+    const int64_t blk = u >> 1;
+    const uint32_t word = __ldg(nibbles + u);
+    const uint32_t sb = scales[blk];
+    const float d = __fmul_rn(e4m3_byte_to_f32(sb & 127u), ts);
+    int bm = -1;
+    if (kPlus && sb > 2u) {
+        bm = (int)((bm_index[blk >> 1] >> (4 * (blk & 1))) & 15u) - 8 * (int)(u & 1);  // within this word
+    }
+    float out[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t c = (word >> (4 * i)) & 15u;
+        const uint32_t e = (c >> 1) & 3u, m = c & 1u;
+        float mag = e == 0u ? 0.5f * (float)m : __uint_as_float(((126u + e) << 23) | (m << 22));
+        if (kPlus && i == bm) mag = 4.f + 0.5f * (float)(c & 7u);
+        const float v = __fmul_rn(mag, d);
+        out[i] = (c & 8u) ? -v : v;
+    }
+    const int64_t e0 = u * 8, row = e0 / cols;
+    T* q = dst + row * ld_dst + (e0 - row * cols);
+    if (sizeof(T) == 4) {
+        reinterpret_cast<uint4*>(q)[0] = make_uint4(__float_as_uint(out[0]), __float_as_uint(out[1]),
+                                                    __float_as_uint(out[2]), __float_as_uint(out[3]));
+        reinterpret_cast<uint4*>(q)[1] = make_uint4(__float_as_uint(out[4]), __float_as_uint(out[5]),
+                                                    __float_as_uint(out[6]), __float_as_uint(out[7]));
+    } else {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(out[2 * i], out[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(q) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_nvfp4_quantize(const void* src, mxp_dtype dt, int64_t rows, int64_t cols,
+                                  int64_t ld_src, float ts, bool plus, uint8_t* nibbles,
+                                  uint8_t* scales, uint8_t* bm_index, cudaStream_t stream)
+{
+    const int64_t units = rows * (cols / 32);
+    const unsigned grid = (unsigned)((units + kThreads - 1) / kThreads);
+#define MXP_NVQ(T, P)                                                                         \
+    nvfp4_quantize_kernel<T, P><<<grid, kThreads, 0, stream>>>(                               \
+        static_cast<const T*>(src), ld_src, cols / 32, units, ts, reinterpret_cast<uint4*>(nibbles), \
+        reinterpret_cast<uint16_t*>(scales), bm_index)
+    if (dt == MXP_BF16) {
+        if (plus) MXP_NVQ(__nv_bfloat16, true);
+        else MXP_NVQ(__nv_bfloat16, false);
+    } else {
+        if (plus) MXP_NVQ(float, true);
+        else MXP_NVQ(float, false);
+    }
+#undef MXP_NVQ
+    return cudaGetLastError();
+}
+
+cudaError_t launch_nvfp4_dequantize(const uint8_t* nibbles, const uint8_t* scales,
+                                    const uint8_t* bm_index, int64_t rows, int64_t cols, float ts,
+                                    bool plus, void* dst, mxp_dtype dt, int64_t ld_dst,
+                                    cudaStream_t stream)
+{
+    const int64_t words = rows * (cols / 8);
+    const unsigned grid = (unsigned)((words + kThreads - 1) / kThreads);
+#define MXP_NVD(T, P)                                                                          \
+    nvfp4_dequantize_kernel<T, P><<<grid, kThreads, 0, stream>>>(                              \
+        reinterpret_cast<const uint32_t*>(nibbles), scales, bm_index, cols, words, ts,         \
+        static_cast<T*>(dst), ld_dst)
+    if (dt == MXP_BF16) {
+        if (plus) MXP_NVD(__nv_bfloat16, true);
+        else MXP_NVD(__nv_bfloat16, false);
+    } else {
+        if (plus) MXP_NVD(float, true);
+        else MXP_NVD(float, false);
+    }
+#undef MXP_NVD
+    return cudaGetLastError();
+}
+
+}  // namespace mxp
