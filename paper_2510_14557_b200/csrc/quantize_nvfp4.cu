@@ -52,37 +52,47 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float* f)
 }
 
 // One block of 16: two words of codes, the scale byte and the BM index (0 when not extended).
-template <bool kPlus>
+// kKey: the values came from bf16, so their low 16 bits are zero and (magnitude bits | 15 -
+// position) is a key whose unsigned maximum gives the largest magnitude and, among equal
+// ones, the first position in one pass.
+template <bool kPlus, bool kKey>
 __device__ __forceinline__ void nvfp4_block(const float* x, float ts, float six_ts, uint32_t& w0,
                                             uint32_t& w1, uint32_t& scale_byte, uint32_t& index)
 {
     float amax = 0.f;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(x[i]));
     int bm = 0;
+    if (kPlus && kKey) {
+        uint32_t key = 0;
 #pragma unroll
-    for (int i = 15; i >= 0; --i)
-        if (fabsf(x[i]) == amax) bm = i;  // the first of equal maxima
+        for (int i = 0; i < 16; ++i)
+            key = max(key, (__float_as_uint(x[i]) & 0x7FFFFFFFu) | (uint32_t)(15 - i));
+        amax = __uint_as_float(key & 0x7FFF0000u);
+        bm = 15 - (int)(key & 15u);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(x[i]));
+        if (kPlus) {
+#pragma unroll
+            for (int i = 15; i >= 0; --i)
+                if (fabsf(x[i]) == amax) bm = i;  // the first of equal maxima
+        }
+    }
     const uint32_t sb = f32_to_e4m3_byte(__fdiv_rn(amax, six_ts));
     const float d = __fmul_rn(e4m3_byte_to_f32(sb), ts);
     const float r = __frcp_rn(d);
+    // r > 0, so x * r has the sign of x even where it underflows, and the hardware cast keeps
+    // the sign of a value that rounds to zero: the codes' sign bits are the inputs'
     float s[16];
-    uint32_t sign = 0, sign1 = 0;
 #pragma unroll
     for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        sign |= (__float_as_uint(x[i]) >> 31) << (4 * i + 3);
-        sign1 |= (__float_as_uint(x[8 + i]) >> 31) << (4 * i + 3);
-    }
-    w0 = (cvt_e2m1x8(s) & 0x77777777u) | sign;
-    w1 = (cvt_e2m1x8(s + 8) & 0x77777777u) | sign1;
+    w0 = cvt_e2m1x8(s);
+    w1 = cvt_e2m1x8(s + 8);
     index = 0;
     if (kPlus && sb > 2u) {
         const float v = fminf(fmaxf(__fmul_rn(amax, r), 4.f), 8.f);
         const uint32_t m = (uint32_t)min(__float2int_rn((v - 4.f) * 2.f), 7);
         const uint32_t sh = (uint32_t)(bm & 7) * 4u;
-        if (bm < 8) w0 = (w0 & ~(7u << sh)) | (m << sh);
+        if (bm < 8) w0 = (w0 & ~(7u << sh)) | (m << sh);  // the sign bit stays
         else w1 = (w1 & ~(7u << sh)) | (m << sh);
         index = (uint32_t)bm;
     }
@@ -124,8 +134,8 @@ nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_p
     }
     const float six_ts = __fmul_rn(6.f, ts);
     uint32_t w[4], sb0, sb1, i0, i1;
-    nvfp4_block<kPlus>(x, ts, six_ts, w[0], w[1], sb0, i0);
-    nvfp4_block<kPlus>(x + 16, ts, six_ts, w[2], w[3], sb1, i1);
+    nvfp4_block<kPlus, sizeof(T) == 2>(x, ts, six_ts, w[0], w[1], sb0, i0);
+    nvfp4_block<kPlus, sizeof(T) == 2>(x + 16, ts, six_ts, w[2], w[3], sb1, i1);
     __stcs(nibbles + u, make_uint4(w[0], w[1], w[2], w[3]));
     scales[u] = (uint16_t)(sb0 | (sb1 << 8));
     if (kPlus) bm_index[u] = (uint8_t)(i0 | (i1 << 4));
