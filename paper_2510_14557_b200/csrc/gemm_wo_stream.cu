@@ -5,13 +5,18 @@
 //   * a producer warp moves 16 weight rows x 2048 elements per stage into shared memory with
 //     bulk copies (mbarrier ring), plus the 16 rows' scale and BM-index bytes per row group;
 //   * sixteen consumer warps each take one 128-element chunk of every stage;
-//   * two reducer warps add the consumers' partial sums in a fixed order and store D, so the
-//     consumers go straight on to the next row group.
+//   * two reducer warps add the partial sums in a fixed order and store D, so the consumers
+//     go straight on to the next row group;
+//   * MX+ modes: two correction warps handle the BM (below).
 // Per 32-element block the four lanes of a quad hold the block's four words for two rows and
 //   * turn the E2M1 codes into f16 pairs with the hardware cast (cvt.rn.f16x2.e2m1x2),
-//   * patch the block's BM to 4 + m/2 (Eq. 3's BM branch) with masks from a small table,
 //   * run two m16n8k16 f16 MMAs against the activations of the block (fresh accumulator),
 //   * add that partial sum times 2^(shared_exp) of the weight block into the running fp32 sum.
+// The BM (Eq. 3's BM branch: 4 + m/2 instead of the E2M1 value of the same bits) never enters
+// that loop: a quad would spend as many instructions on locating and patching one element as
+// on the other 31 together, in all four lanes.  The consumers multiply the BM's code as E2M1
+// and one thread per weight row and eighth of the blocks adds
+// (4 + m/2 - E2M1(m)) * 2^shared_exp * a[k_BM] per block: a dozen scalar instructions.
 // Activations are bf16; so that they fit f16 each 256-element chunk of an activation row is
 // normalised by the power of two that puts its largest magnitude in [2^14, 2^15): every
 // element within 2^28 of that maximum stays exact (f16 keeps 11 significant bits), smaller
@@ -31,8 +36,12 @@ namespace {
 
 constexpr int kCW = 16;                      // consumer warps
 constexpr int kRW = 2;                       // reducer warps
+constexpr int kXW = 4;                       // BM correction warps (MX+ modes)
+constexpr int kXSub = 32 * kXW / 16;         // correction threads per weight row: 8
 constexpr int kProducerWarp = kCW;
-constexpr int kThreads = 32 * (kCW + 1 + kRW);
+constexpr int kThreadsBase = 32 * (kCW + 1 + kRW);
+constexpr int kThreadsCorr = kThreadsBase + 32 * kXW;  // with the correction warps
+constexpr int kLutBytes = 32 * 4 * 16;       // [BM position][lane of the quad] -> 4 keep masks
 constexpr int kRows = 16;                    // weight rows per step
 constexpr int kSlab = 4096;                  // elements of K per stage
 constexpr int kChunkBlocks = kSlab / 32 / kCW;  // 8 blocks of 32 per warp and stage
@@ -40,7 +49,6 @@ constexpr int kMaxStages = 6;
 constexpr int kMaxMetaBufs = 4;              // row groups whose scale / index bytes may be in flight
 constexpr int kRowStride = kSlab / 2 + 16;   // bytes; the pad spreads the rows over the banks
 constexpr int kStageBytes = kRows * kRowStride;
-constexpr int kLutBytes = 32 * 4 * 16;       // [BM position][lane of the quad] -> 4 keep masks
 constexpr long long kWaitLimit = 4000000000ll;
 constexpr size_t kSmemMax = 227 * 1024;
 
@@ -76,7 +84,7 @@ struct WoLayout {
     int meta_stride;  // bytes of one metadata buffer (scales + index of 16 rows)
     int red_stride;   // bytes of one partial-sum buffer
 };
-__host__ __device__ inline WoLayout wo_layout(int K, int mp, bool plus, int red_buffers,
+__host__ __device__ inline WoLayout wo_layout(int K, int mp, bool plus, bool corr, int red_buffers,
                                               int meta_bufs)
 {
     WoLayout l;
@@ -92,7 +100,7 @@ __host__ __device__ inline WoLayout wo_layout(int K, int mp, bool plus, int red_
     l.meta_stride = (int)(kRows * nb * (plus ? 2 : 1));
     off += (size_t)meta_bufs * l.meta_stride;
     l.red = off = align16(off);
-    l.red_stride = kCW * kRows * (mp + 1) * 4;
+    l.red_stride = (kCW + (corr ? 1 : 0)) * kRows * (mp + 1) * 4;
     off += (size_t)red_buffers * l.red_stride;
     l.ring = off = align16(off);
     l.fixed = off + 128;  // + slack for aligning the base; the ring follows
@@ -114,6 +122,18 @@ __device__ __forceinline__ uint32_t lds32(uint32_t a)
 {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds8(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
 __device__ __forceinline__ uint2 lds64(uint32_t a)
@@ -235,16 +255,22 @@ __device__ __forceinline__ void normalise_block(const uint4 (&x)[4], int mulfiel
     } while (0)
 #endif
 
-template <int kMT, int kMode, typename OutT>
-__global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoParams prm)
+// kCorr (MX+ modes, one activation row): the BM is handled by the correction warps; otherwise
+// the consumers patch it into their f16 fragments, which costs the same for any number of
+// activation columns, while the correction threads' work grows with each column.
+template <int kMT, int kMode, bool kCorr, typename OutT>
+__global__ void __launch_bounds__(kCorr ? kThreadsCorr : kThreadsBase, 1)
+gemm_wo_stream_kernel(const WoParams prm)
 {
     constexpr bool kPlus = kMode >= 1;  // 1: MXFP4+, 2: MX++ (Sec. 4.3)
     constexpr bool kPP = kMode == 2;
+    constexpr bool kPatch = kPlus && !kCorr;
+    static_assert(!kCorr || kPlus, "correction warps are for the MX+ modes");
     constexpr int kMp = 8 * kMT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) &
                                                ~(uintptr_t)127);
-    const WoLayout L = wo_layout(prm.K, kMp, kPlus, prm.red_buffers, prm.meta_bufs);
+    const WoLayout L = wo_layout(prm.K, kMp, kPlus, kCorr, prm.red_buffers, prm.meta_bufs);
     const uint32_t kMetaBufs = (uint32_t)prm.meta_bufs;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);
     uint64_t* empty = full + kMaxStages;
@@ -273,14 +299,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
         WO_TL(0);
         for (int s = 0; s < kMaxStages; ++s) {
             ptx::mbar_init(&full[s], 1);
-            ptx::mbar_init(&empty[s], kCW);
+            ptx::mbar_init(&empty[s], kCW + (kCorr ? kXW : 0));
         }
         for (int b = 0; b < kMaxMetaBufs; ++b) {
             ptx::mbar_init(&meta_full[b], 1);
-            ptx::mbar_init(&meta_empty[b], kCW);
+            ptx::mbar_init(&meta_empty[b], kCW + (kCorr ? kXW : 0));
         }
         for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(&red_full[b], kCW);
+            ptx::mbar_init(&red_full[b], kCW + (kCorr ? kXW : 0));
             ptx::mbar_init(&red_free[b], kRW);
         }
         ptx::mbar_init(setup_bar, kCW);
@@ -337,7 +363,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
         const int g = lane >> 2, t = lane & 3;
         constexpr int kCT = 32 * kCW;  // consumer threads
         // BM mask table: entry [p][t] keeps everything unless word t holds element p
-        if (threadIdx.x < 128) {
+        if (kPatch && threadIdx.x < 128) {
             const uint32_t p = threadIdx.x >> 2, tt = threadIdx.x & 3;
             uint32_t k[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
             if ((p >> 3) == tt) k[(p & 7u) >> 1] = (p & 1u) ? 0x0000FFFFu : 0xFFFF0000u;
@@ -383,7 +409,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
             }
             if (lane < kMp) fa[chunk * kMp + mc] = __uint_as_float((uint32_t)(254 - mulfield) << 23);
         }
-        // the BM mask table was written by the first four warps: one barrier before its use
+        // every warp's share of the activations (and the mask table) is in place before use
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(setup_bar);
         bool ok = ptx::mbar_wait(setup_bar, 0, abort, kWaitLimit);
@@ -427,7 +453,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                         for (int j = 0; j < 4; ++j) cacc[i][j] = 0.f;
                     const uint2 scA = lds64(sc + kb0), scB = lds64(sc + 8 * nb + kb0);
                     uint2 ixA = make_uint2(0, 0), ixB = ixA;
-                    if (kPlus) {
+                    if (kPP || kPatch) {  // MX++: delta; patching: the BM's position
                         ixA = lds64(ix + kb0);
                         ixB = lds64(ix + 8 * nb + kb0);
                     }
@@ -443,7 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                         const int sh = 8 * (j & 3);
                         const uint32_t ibA = ((j < 4 ? ixA.x : ixA.y) >> sh) & 255u;
                         const uint32_t ibB = ((j < 4 ? ixB.x : ixB.y) >> sh) & 255u;
-                        if (kPlus) {
+                        if (kPatch) {
                             patch_bm<kPP>(wA, ibA, lut_t, hA);
                             patch_bm<kPP>(wB, ibB, lut_t, hB);
                         }
@@ -509,6 +535,128 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&red_full[rbuf]);
         }
+    } else if (kCorr && warp >= kCW + 1 + kRW) {
+        // ------------------------------------------------------------------ BM correction warps
+        // The consumers multiply every code as E2M1, the BM's `s m2 m1 m0` included (as the
+        // value of its low three bits, at the NBMs' scale).  Eq. 3's BM branch says 4 + m/2 at
+        // the block's own scale; per block and weight row these warps add the difference times
+        // the activation at the BM's position.  One thread per weight row and eighth of the
+        // blocks; a row's eight threads add up their sums, which go to the reducers as one
+        // more partial sum per row.
+        {
+            const int tid = threadIdx.x - 32 * (kCW + 1 + kRW);
+            const int row = tid / kXSub, sub = tid % kXSub;  // a row's threads are neighbouring lanes
+            const int mcols = min(kMp, prm.M - m0);
+            // per code `s m2 m1 m0` (entry = lane & 15): Eq. 3's BM value 4 + m/2 and the E2M1
+            // value of the same bits, both signed
+            const uint32_t lm = (uint32_t)lane & 7u;
+            const float sgn = (lane & 8) ? -1.f : 1.f;
+            const float bm_true = sgn * (4.f + 0.5f * (float)lm);
+            const float bm_e2m1 =
+                sgn * (lm < 2u ? 0.5f * (float)lm : __uint_as_float(((126u + (lm >> 1)) << 23) | ((lm & 1u) << 22)));
+            const float* fa = reinterpret_cast<const float*>(smem + L.fa);
+            float* red = reinterpret_cast<float*>(smem + L.red);
+            bool ok = ptx::mbar_wait(setup_bar, 0, abort, kWaitLimit);  // activations are in place
+            if (!ok && lane == 0) report(prm.status, abort, 0x3700);
+            uint32_t it = 0, round = 0;
+            int s = 0;
+            for (int rg = blockIdx.x; rg < rgs && ok; rg += gridDim.x, ++it) {
+                const uint32_t mb = it % kMetaBufs;
+                if (!ptx::mbar_wait(&meta_full[mb], (it / kMetaBufs) & 1, abort, kWaitLimit)) {
+                    if (lane == 0) report(prm.status, abort, 0x3800);
+                    break;
+                }
+                const uint32_t sc = sbase + (uint32_t)L.meta + mb * (uint32_t)L.meta_stride + (uint32_t)(row * nb);
+                const uint32_t ix = sc + (uint32_t)(kRows * nb);
+                float acc[kMp];
+#pragma unroll
+                for (int c = 0; c < kMp; ++c) acc[c] = 0.f;
+                for (int sl = 0; sl < slabs && ok; ++sl) {
+                    if (!ptx::mbar_wait(&full[s], round & 1, abort, kWaitLimit)) {
+                        if (lane == 0) report(prm.status, abort, 0x3900 + s);
+                        ok = false;
+                        break;
+                    }
+                    const int nblk = min(kSlab, prm.K - sl * kSlab) / 32;
+                    const uint32_t wrow = sbase + (uint32_t)L.ring + (uint32_t)(s * kStageBytes + row * kRowStride);
+                    // eight blocks at a time (one 8-byte word of index and of scale bytes), the
+                    // groups dealt round robin to the row's eight threads; the loads of a group
+                    // are issued together so that their latencies overlap
+                    // (warp-uniform trip count: the table lookups are full-warp shuffles; a
+                    // thread past the last group works on group 0 and adds nothing)
+                    for (int g0 = 0; g0 < nblk / 8; g0 += kXSub) {
+                        const bool on = g0 + sub < nblk / 8;
+                        const int g8 = on ? g0 + sub : 0;
+                        const int kb0 = sl * (kSlab / 32) + 8 * g8;
+                        const uint2 ib8 = lds64(ix + kb0), sc8 = lds64(sc + kb0);
+                        uint32_t pos[8], byte[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            pos[u] = __byte_perm(u < 4 ? ib8.x : ib8.y, 0u, 0x4440u + (u & 3));
+                            byte[u] = lds8(wrow + (8 * g8 + u) * 16 + ((pos[u] & 31u) >> 1));
+                        }
+                        float cf[8];
+                        uint32_t ap[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const uint32_t p = pos[u] & 31u;
+                            // (bit 4 may hold the neighbouring code's low bit: the tables repeat
+                            // every 16 lanes and a shuffle takes its source lane modulo 32)
+                            const uint32_t nib = byte[u] >> ((p << 2) & 4u);
+                            // 2^(scale byte - 127); a zero byte (flushed block) gives 0
+                            const float scale =
+                                __uint_as_float(__byte_perm(u < 4 ? sc8.x : sc8.y, 0u, 0x4440u + (u & 3)) << 23);
+                            // the tables sit one entry per lane: a shuffle is the lookup
+                            if (kPP) {  // the consumers entered E2M1(m) at the NBMs' scale, delta binades down
+                                const float tv = __shfl_sync(0xFFFFFFFFu, bm_true, (int)nib);
+                                const float ev = __shfl_sync(0xFFFFFFFFu, bm_e2m1, (int)nib);
+                                cf[u] = fmaf(-ev, __uint_as_float((127u - (pos[u] >> 5)) << 23), tv) * scale;
+                            } else {
+                                cf[u] = __shfl_sync(0xFFFFFFFFu, bm_true - bm_e2m1, (int)nib) * scale;
+                            }
+                            ap[u] = sbase + (uint32_t)L.act + (uint32_t)((kb0 + u) * kMp) * 64u + p * 2u;
+                        }
+                        const float* fk = fa + (kb0 / kChunkBlocks) * kMp;  // one chunk = these 8 blocks
+#pragma unroll
+                        for (int c = 0; c < kMp; ++c) {
+                            if (c < mcols) {
+                                float part = 0.f;
+#pragma unroll
+                                for (int u = 0; u < 8; ++u)
+                                    part = fmaf(cf[u], __half2float(__ushort_as_half(
+                                                           (unsigned short)lds16(ap[u] + c * 64))), part);
+                                acc[c] = fmaf(part, on ? fk[c] : 0.f, acc[c]);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&empty[s]);
+                    if (++s == S) {
+                        s = 0;
+                        ++round;
+                    }
+                }
+                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&meta_empty[mb]);
+                const uint32_t rbuf = two_red ? (it & 1u) : 0u;
+                const uint32_t ruse = two_red ? (it >> 1) : it;
+                if (ruse > 0 && !ptx::mbar_wait(&red_free[rbuf], (ruse - 1) & 1, abort, kWaitLimit)) {
+                    if (lane == 0) report(prm.status, abort, 0x3A00);
+                    break;
+                }
+                float* r0 = red + (size_t)rbuf * (L.red_stride / 4) + ((size_t)kCW * kRows + row) * (kMp + 1);
+#pragma unroll
+                for (int c = 0; c < kMp; ++c) {
+                    float v = acc[c];
+#pragma unroll
+                    for (int o = 1; o < kXSub; o <<= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+                    if (sub == 0) r0[c] = v;
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&red_full[rbuf]);
+            }
+        }
     } else {
         // ------------------------------------------------------------------ reducer warps
         const int tid = threadIdx.x - 32 * (kCW + 1);
@@ -528,7 +676,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
                 const int r = e % kRows, mcol = e / kRows;
                 float sum = 0.f;
 #pragma unroll
-                for (int w = 0; w < kCW; ++w) sum += rb[((size_t)w * kRows + r) * (kMp + 1) + mcol];
+                for (int w = 0; w < kCW + (kCorr ? 1 : 0); ++w)
+                    sum += rb[((size_t)w * kRows + r) * (kMp + 1) + mcol];
                 const int m = m0 + mcol;
                 if (m < prm.M) {
                     if (sizeof(OutT) == 4)
@@ -557,11 +706,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_wo_stream_kernel(const WoPar
 
 // Ring depth and numbers of partial-sum and metadata buffers that fit; the roomier choices
 // are tried first.  False if not even two stages fit.
-inline bool wo_plan(int K, int mp, bool plus, int* stages, int* red_buffers, int* meta_bufs)
+inline bool wo_plan(int K, int mp, bool plus, bool corr, int* stages, int* red_buffers, int* meta_bufs)
 {
     const int rbs[3] = {2, 1, 1}, mbs[3] = {4, 4, 2};
     for (int c = 0; c < 3; ++c) {
-        const size_t fixed = wo_layout(K, mp, plus, rbs[c], mbs[c]).fixed;
+        const size_t fixed = wo_layout(K, mp, plus, corr, rbs[c], mbs[c]).fixed;
         if (fixed >= kSmemMax) continue;
         const int st = (int)((kSmemMax - fixed) / kStageBytes);
         if (st >= 3 || (c == 2 && st >= 2)) {
@@ -574,15 +723,16 @@ inline bool wo_plan(int K, int mp, bool plus, int* stages, int* red_buffers, int
     return false;
 }
 
-template <int kMT, int kMode, typename OutT>
+template <int kMT, int kMode, bool kCorr, typename OutT>
 cudaError_t launch(WoParams prm, int num_sms, bool chained, cudaStream_t stream)
 {
     constexpr bool kPlus = kMode >= 1;
-    if (!wo_plan(prm.K, 8 * kMT, kPlus, &prm.stages, &prm.red_buffers, &prm.meta_bufs))
+    constexpr int kThreads = kCorr ? kThreadsCorr : kThreadsBase;
+    if (!wo_plan(prm.K, 8 * kMT, kPlus, kCorr, &prm.stages, &prm.red_buffers, &prm.meta_bufs))
         return cudaErrorNotSupported;
-    const size_t smem = wo_layout(prm.K, 8 * kMT, kPlus, prm.red_buffers, prm.meta_bufs).fixed +
+    const size_t smem = wo_layout(prm.K, 8 * kMT, kPlus, kCorr, prm.red_buffers, prm.meta_bufs).fixed +
                         (size_t)prm.stages * kStageBytes;
-    auto kern = gemm_wo_stream_kernel<kMT, kMode, OutT>;
+    auto kern = gemm_wo_stream_kernel<kMT, kMode, kCorr, OutT>;
     static SmemAttrOnce once;
     const cudaError_t ea = ensure_dynamic_smem(kern, (int)kSmemMax, once);
     if (ea != cudaSuccess) return ea;
@@ -625,7 +775,7 @@ bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t
     const bool plus = B.mode != MXP_MODE_MXFP4;
     if (plus && (reinterpret_cast<uintptr_t>(B.bm_index) & 15)) return false;
     int st, rb, mb;
-    return wo_plan((int)K, M <= 8 ? 8 : 16, plus, &st, &rb, &mb);
+    return wo_plan((int)K, M <= 8 ? 8 : 16, plus, plus && M == 1, &st, &rb, &mb);
 }
 
 cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
@@ -649,22 +799,26 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
     if (sms <= 0) return cudaErrorUnknown;
     const bool f32 = d_dt == MXP_F32;
     const int mode = (int)B.mode;
-#define MXP_WO_LAUNCH(MT)                                                                  \
+#define MXP_WO_LAUNCH(MT, CORR)                                                            \
     switch (mode) {                                                                        \
         case 2:                                                                            \
-            return f32 ? launch<MT, 2, float>(prm, sms, chained, stream)                            \
-                       : launch<MT, 2, __nv_bfloat16>(prm, sms, chained, stream);                   \
+            return f32 ? launch<MT, 2, CORR, float>(prm, sms, chained, stream)             \
+                       : launch<MT, 2, CORR, __nv_bfloat16>(prm, sms, chained, stream);    \
         case 1:                                                                            \
-            return f32 ? launch<MT, 1, float>(prm, sms, chained, stream)                            \
-                       : launch<MT, 1, __nv_bfloat16>(prm, sms, chained, stream);                   \
+            return f32 ? launch<MT, 1, CORR, float>(prm, sms, chained, stream)             \
+                       : launch<MT, 1, CORR, __nv_bfloat16>(prm, sms, chained, stream);    \
         default:                                                                           \
-            return f32 ? launch<MT, 0, float>(prm, sms, chained, stream)                            \
-                       : launch<MT, 0, __nv_bfloat16>(prm, sms, chained, stream);                   \
+            return f32 ? launch<MT, 0, false, float>(prm, sms, chained, stream)            \
+                       : launch<MT, 0, false, __nv_bfloat16>(prm, sms, chained, stream);   \
+    }
+    // one activation row: the BM goes to the correction warps (see the kernel)
+    if (M == 1) {
+        MXP_WO_LAUNCH(1, true)
     }
     if (M <= 8) {
-        MXP_WO_LAUNCH(1)
+        MXP_WO_LAUNCH(1, false)
     }
-    MXP_WO_LAUNCH(2)
+    MXP_WO_LAUNCH(2, false)
 #undef MXP_WO_LAUNCH
 }
 
