@@ -28,7 +28,8 @@ bool valid_dtype(int d) { return d == MXP_F32 || d == MXP_BF16; }
 bool valid_packed(const mxp_packed* p, bool six_ok = false)
 {
     if (p == nullptr) return false;
-    const bool six = p->mode == MXP_MODE_MXFP6 || p->mode == MXP_MODE_MXFP6_PLUS;
+    const bool six = p->mode == MXP_MODE_MXFP6 || p->mode == MXP_MODE_MXFP6_PLUS ||
+                     p->mode == MXP_MODE_MXFP8;  // (and plain MXFP8: E4M3 codes go in as they are)
     if (!valid_mode(p->mode) && !(six_ok && six)) return false;
     if (p->rows < 0 || p->cols < 0 || p->cols % 32 != 0) return false;
     if (p->rows == 0 || p->cols == 0) return true;
@@ -275,7 +276,7 @@ size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide)
 mxp_status mxp_gemm_prepack(const mxp_packed* P, int wide, void* out, size_t out_bytes,
                             void* cuda_stream)
 {
-    if (!valid_packed(P)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(P, true)) return MXP_ERR_INVALID_ARG;
     if (P->rows == 0 || P->cols == 0) return MXP_OK;
     if (P->mode != MXP_MODE_MXFP4 && !wide) return MXP_ERR_INVALID_ARG;
     return mxp::stream_prepack(*P, wide != 0, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
@@ -288,7 +289,7 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
 {
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
-    if (!valid_packed(A_packed) || !valid_packed(B_packed)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(A_packed, true) || !valid_packed(B_packed, true)) return MXP_ERR_INVALID_ARG;
     if (A_packed->rows != M || A_packed->cols != K || B_packed->rows != N || B_packed->cols != K)
         return MXP_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return MXP_OK;

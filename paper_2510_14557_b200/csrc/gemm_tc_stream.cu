@@ -492,6 +492,7 @@ struct PrepackOperand {
     int tile_rows;            // rows per accumulator: kTileM for A, sub_n() for B
     int pp;                   // MX++ operand: index bits 7:5 hold delta (Sec. 4.3)
     int six;                  // source codes are packed 6-bit E2M3 (MXFP6 / MXFP6+), not nibbles
+    int eight;                // source codes are E4M3 bytes (MXFP8): the MMA reads them as they are
     size_t plane_bytes;       // MXFP6+: distance to the second plane of the widened copy, else 0
     unsigned scale_ctas;      // row groups * ceil(nbk/128)
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
@@ -588,6 +589,11 @@ __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned i
     const uint32_t b = t >> 1;
     if (b >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
     if (op.six) return widen_six(op, t, b);
+    if (op.eight) {
+        // MXFP8: one byte per element already; a flushed block's codes are zero by construction
+        reinterpret_cast<uint4*>(op.wide)[t] = reinterpret_cast<const uint4*>(op.nibbles)[t];
+        return;
+    }
     const uint2 w = reinterpret_cast<const uint2*>(op.nibbles)[t];
     const uint32_t sc = op.scales[b];
     const uint32_t ib = op.bm_index != nullptr ? op.bm_index[b] : 0u;
@@ -683,6 +689,7 @@ inline int64_t row_groups(int64_t rows, int tile_rows) { return 2 * ((rows + til
 // E2M3 planes an operand is widened into: two for MXFP6+ (see widen_six), else one.
 inline int mode_parts(mxp_mode m) { return m == MXP_MODE_MXFP6_PLUS ? 2 : 1; }
 inline bool mode_six(mxp_mode m) { return m == MXP_MODE_MXFP6 || m == MXP_MODE_MXFP6_PLUS; }
+inline bool mode_eight(mxp_mode m) { return m == MXP_MODE_MXFP8; }
 inline bool mode_plus(mxp_mode m)
 {
     return m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP || m == MXP_MODE_MXFP6_PLUS;
@@ -764,14 +771,14 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
     // operands, which only this path handles (rows past the end are zero-filled by TMA).
     // (and MXFP6 operands, likewise)
     const bool pp = a_mode == MXP_MODE_MXFP4_PP || b_mode == MXP_MODE_MXFP4_PP ||
-                    mode_six(a_mode) || mode_six(b_mode);
+                    mode_six(a_mode) || mode_six(b_mode) || mode_eight(a_mode) || mode_eight(b_mode);
     if (M < 1 || N < 1 || K % 128 != 0) return 0;
     if (!pp && (M <= 128 || N <= 128)) return 0;
     // the prepack kernel indexes half blocks (16 elements) of an operand with 32 bits
     if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
         return 0;
     const bool wide = a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4;
-    if (a_mode > MXP_MODE_MXFP6_PLUS || b_mode > MXP_MODE_MXFP6_PLUS) return 0;  // no MXFP8 GEMM
+    if (a_mode > MXP_MODE_MXFP8 || b_mode > MXP_MODE_MXFP8) return 0;  // no MXFP8+ GEMM
     return layout(M, N, K, wide, mode_parts(a_mode), mode_parts(b_mode)).total;
 }
 
@@ -804,6 +811,7 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     op.bm_index = mode_plus(P.mode) ? P.bm_index : nullptr;
     op.pp = P.mode == MXP_MODE_MXFP4_PP;
     op.six = mode_six(P.mode);
+    op.eight = mode_eight(P.mode);
     op.plane_bytes = P.mode == MXP_MODE_MXFP6_PLUS ? (size_t)rows * (size_t)K : 0;
     op.atoms = atoms;
     op.wide = wide ? wide_bytes : nullptr;
@@ -834,7 +842,9 @@ mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_
     const size_t need = stream_prepack_bytes(P.rows, P.cols, wide);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
     // an MXFP6+ operand needs two planes, which this form has no room for: mxp_gemm takes it
-    if (P.mode > MXP_MODE_MXFP6 || (mode_six(P.mode) && !wide)) return MXP_ERR_UNSUPPORTED;
+    if ((P.mode > MXP_MODE_MXFP6 && !mode_eight(P.mode)) ||
+        ((mode_six(P.mode) || mode_eight(P.mode)) && !wide))
+        return MXP_ERR_UNSUPPORTED;
     if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
         (reinterpret_cast<uintptr_t>(P.scales) & 3) ||
@@ -878,7 +888,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     // `a_ready`: A's atoms and code slots are in the workspace already (and the status block is
     // cleared); needs a prepacked B, so that nothing is left to prepare
     if (a_ready && (b_prepacked == nullptr || A.mode > MXP_MODE_MXFP4_PLUS)) return MXP_ERR_UNSUPPORTED;
-    if (A.mode > MXP_MODE_MXFP6_PLUS || B.mode > MXP_MODE_MXFP6_PLUS) return MXP_ERR_UNSUPPORTED;
+    if (A.mode > MXP_MODE_MXFP8 || B.mode > MXP_MODE_MXFP8) return MXP_ERR_UNSUPPORTED;
     const int parts_a = mode_parts(A.mode), parts_b = mode_parts(B.mode);
     if (b_prepacked != nullptr && parts_b != 1) return MXP_ERR_UNSUPPORTED;
     const Layout l = layout(M, b_prepacked ? 0 : N, K, wide, parts_a, parts_b);
@@ -934,8 +944,8 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     prm.M = (int)M;
     prm.N = (int)N;
     prm.K = (int)K;
-    prm.a_fmt = A.mode == MXP_MODE_MXFP4_PP ? kFmtE4M3 : kFmtE2M3;
-    prm.b_fmt = B.mode == MXP_MODE_MXFP4_PP ? kFmtE4M3 : kFmtE2M3;
+    prm.a_fmt = (A.mode == MXP_MODE_MXFP4_PP || mode_eight(A.mode)) ? kFmtE4M3 : kFmtE2M3;
+    prm.b_fmt = (B.mode == MXP_MODE_MXFP4_PP || mode_eight(B.mode)) ? kFmtE4M3 : kFmtE2M3;
     prm.parts_a = parts_a;
     prm.parts_b = parts_b;
     prm.D = D;

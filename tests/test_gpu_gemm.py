@@ -577,8 +577,64 @@ def test_tc_mxfp6_quantized_end_to_end_and_rejections():
     with pytest.raises(MxpError):   # no weight-only form for 6-bit weights
         m.mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), pw)
     p8 = m.mxp_quantize(to_dev(a), 6)
-    with pytest.raises(MxpError):   # MXFP8 operands: quantize and decode only
+    with pytest.raises(MxpError):   # MXFP8+ operands: quantize and decode only
         m.mxp_gemm(p8, p8)
+
+
+# ------------------------------------------------------------------ MXFP8 operands
+MX8 = 5
+
+
+def _raw_operand8(rows, K, seed, scale_lo=112, scale_hi=130):
+    """MXFP8 planes filled directly: every E4M3 code except the NaN pattern."""
+    g = synth.rng(seed)
+    codes = g.integers(0, 256, (rows, K), dtype=np.uint8)
+    codes[(codes & 0x7F) == 0x7F] = 0x7E
+    sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
+    sc[g.random((rows, K // 32)) < 0.02] = 0          # flushed blocks hold zero codes
+    codes[np.repeat(sc == 0, 32, axis=1)] = 0
+    dec = oracle.dequantize_wide(codes, sc, None, oracle.FMT_E4M3, False)
+    from paper_2510_14557_b200 import Packed
+    return Packed(to_dev(codes), to_dev(sc), None, rows, K, MX8), dec
+
+
+@pytest.mark.parametrize("amode,bmode", [(MX8, MX8), (MX8, MXP), (MX, MX8), (MX6P, MX8), (MX8, MXPP)])
+@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 129, 384), (64, 100, 256), (513, 1000, 128)])
+def test_tc_mxfp8_operands(M, N, K, amode, bmode):
+    # E4M3 elements are an operand format of the same instruction: the codes go in as stored,
+    # next to 4- and 6-bit partners on the other side
+    ap, da = _raw_operand8(M, K, seed=M + 5) if amode == MX8 else _any_operand(M, K, amode, seed=M + 5)
+    bp, db = _raw_operand8(N, K, seed=N + 6) if bmode == MX8 else _any_operand(N, K, bmode, seed=N + 6)
+    m = mxp()
+    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode), dtype=torch.uint8, device="cuda")
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm(ap, bp, out_dtype=dt, workspace=ws)
+        assert m.mxp_gemm_status(ws) == 0
+        check_gemm(d, da, db)
+
+
+def test_tc_mxfp8_identity_and_quantized_end_to_end():
+    m = mxp()
+    # B = identity: D is the decode of A bit for bit, for every E4M3 code
+    M, K = 384, 256
+    ap, da = _raw_operand8(M, K, seed=41)
+    bp, db = quantized(np.eye(K, dtype=np.float32), MX)
+    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32)
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
+    # quantized by the library, against the oracle's encode + decode + fp64 product
+    a = synth.activations_normal(320, 512, seed=43, outlier_frac=0.02)
+    w = synth.weights(384, 512, seed=44)
+    pa, pw = m.mxp_quantize(to_dev(a), MX8), m.mxp_quantize(to_dev(w), MX8)
+    ca, sa, _ = oracle.quantize_wide(a, oracle.FMT_E4M3, False)
+    cw, sw, _ = oracle.quantize_wide(w, oracle.FMT_E4M3, False)
+    check_gemm(m.mxp_gemm(pa, pw, out_dtype=torch.float32),
+               oracle.dequantize_wide(ca, sa, None, oracle.FMT_E4M3, False),
+               oracle.dequantize_wide(cw, sw, None, oracle.FMT_E4M3, False))
+    # prepacked weights
+    pre = m.mxp_gemm_prepack(pw, True)
+    check_gemm(m.mxp_gemm_prepacked(pa, pw, pre, out_dtype=torch.float32),
+               oracle.dequantize_wide(ca, sa, None, oracle.FMT_E4M3, False),
+               oracle.dequantize_wide(cw, sw, None, oracle.FMT_E4M3, False))
 
 
 # ------------------------------------------------------------------ fused quantize -> GEMM
