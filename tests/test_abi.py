@@ -64,3 +64,46 @@ def test_argument_validation_without_launch(lib):
     assert g(4, 8, 128, null, 0, ctypes.byref(a), ctypes.byref(b), fake, 1, 8, null, 0, null) == 3    # workspace
     assert lib.mxp_gemm_workspace_bytes(4, 8, 128, 0, 1, 1) >= 16
     assert lib.mxp_tensor_peak_probe(9, 1, None, None) == 1
+
+
+def test_argument_validation_of_the_later_entry_points(lib):
+    # rejected before anything touches a device, like the calls above
+    import numpy as np
+    from paper_2510_14557_b200.binding import _Packed
+    null = None
+    fake = ctypes.c_void_p(4096)
+    odd = ctypes.c_void_p(4100)
+    qr = lib.mxp_quantize_reordered
+    assert qr(fake, 1, 4, 64, 64, null, 1, fake, fake, fake, null) == 1     # no ordering
+    assert qr(fake, 1, 4, 64, 64, odd, 1, fake, fake, fake, null) == 1      # ordering not 16-byte aligned
+    assert qr(fake, 1, 4, 48, 48, fake, 1, fake, fake, fake, null) == 1     # cols % 32
+    assert qr(fake, 1, 4, 64, 64, fake, 1, fake, fake, null, null) == 1     # MX+ needs an index plane
+    assert qr(fake, 1, 4, 64, 64, fake, 4, fake, fake, fake, null) == 2     # 6-bit modes: unsupported
+    assert qr(fake, 1, 0, 64, 64, null, 1, null, null, null, null) == 0     # empty is a no-op
+    nq = lib.mxp_nvfp4_quantize
+    assert nq(fake, 1, 4, 64, 64, 0.0, 1, fake, fake, fake, null) == 1      # tensor scale must be > 0
+    assert nq(fake, 1, 4, 64, 64, float("nan"), 1, fake, fake, fake, null) == 1
+    assert nq(fake, 1, 4, 48, 48, 1.0, 1, fake, fake, fake, null) == 1      # cols % 32
+    assert nq(fake, 1, 4, 64, 64, 1.0, 1, fake, fake, null, null) == 1      # NVFP4+ needs an index plane
+    assert nq(fake, 1, 4, 64, 64, 1.0, 0, fake, ctypes.c_void_p(4097), null, null) == 1  # scales 2-byte aligned
+    nd = lib.mxp_nvfp4_dequantize
+    assert nd(fake, fake, null, 4, 64, 1.0, 1, fake, 0, 64, null) == 1      # NVFP4+ without indices
+    assert nd(fake, fake, null, 4, 64, 1.0, 0, fake, 0, 60, null) == 1      # ld < cols
+    assert nd(fake, fake, null, 0, 64, 1.0, 0, null, 0, 64, null) == 0      # empty
+    b = _Packed(4096, 4096, 4096, 32, 256, 1)
+    ch = lib.mxp_gemm_decode_chained
+    assert ch(1, 32, 256, null, 256, ctypes.byref(b), fake, 1, 32, null, null) == 1   # no activations
+    assert ch(1, 32, 256, fake, 250, ctypes.byref(b), fake, 1, 32, null, null) == 1   # lda < K
+    assert ch(1, 33, 256, fake, 256, ctypes.byref(b), fake, 1, 33, null, null) == 1   # N mismatch
+    assert ch(1, 32, 256, fake, 256, ctypes.byref(b), fake, 1, 32, ctypes.c_void_p(4104), null) == 1  # status block alignment
+    assert ch(100, 32, 256, fake, 256, ctypes.byref(b), fake, 1, 32, null, null) == 2  # M > 64
+    b6 = _Packed(4096, 4096, None, 32, 256, 3)
+    assert ch(1, 32, 256, fake, 256, ctypes.byref(b6), fake, 1, 32, null, null) == 1  # 6-bit weights
+    # the ordering rule runs on the host
+    cnt = np.arange(64, dtype=np.int64)
+    out = np.zeros(64, np.int32)
+    co = lib.mxp_channel_order
+    assert co(cnt.ctypes.data, 64, out.ctypes.data) == 0
+    assert sorted(out.tolist()) == list(range(64)) and out[0] == 63 and out[32] == 62
+    assert co(cnt.ctypes.data, 48, out.ctypes.data) == 1
+    assert co(null, 64, out.ctypes.data) == 1
