@@ -389,12 +389,13 @@ def part_prefill(mxp, synth, peaks, iters):
                 "frac_fp4_nominal_9PF": tf / 9000.0}
             del pa, pw
             # MXFP6 / MXFP6+ operands (E2M3 elements; an MXFP6+ operand costs a second pass) and
-            # MXFP8 operands (E4M3 elements, read as stored)
+            # MXFP8 operands (E4M3 elements, read as stored; an MXFP8+ operand costs three passes)
             for an, am, bn, bm in (("mxfp6", mxp.MODE_MXFP6, "mxfp6", mxp.MODE_MXFP6),
                                    ("mxfp6+", mxp.MODE_MXFP6_PLUS, "mxfp6", mxp.MODE_MXFP6),
                                    ("mxfp6+", mxp.MODE_MXFP6_PLUS, "mxfp4", mxp.MODE_MXFP4),
                                    ("mxfp8", mxp.MODE_MXFP8, "mxfp8", mxp.MODE_MXFP8),
-                                   ("mxfp8", mxp.MODE_MXFP8, "mxfp4+", mxp.MODE_MXFP4_PLUS)):
+                                   ("mxfp8", mxp.MODE_MXFP8, "mxfp4+", mxp.MODE_MXFP4_PLUS),
+                                   ("mxfp8+", mxp.MODE_MXFP8_PLUS, "mxfp8", mxp.MODE_MXFP8)):
                 ws6 = torch.zeros(mxp.mxp_gemm_workspace_bytes(M, N, K, False, am, bm),
                                   dtype=torch.uint8, device="cuda")
                 pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)

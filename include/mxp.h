@@ -56,11 +56,11 @@ typedef enum {
     MXP_MODE_MXFP4_PLUS = 1, /* MX+  (Sec. 4.1): BM with 3 mantissa bits, index byte */
     MXP_MODE_MXFP4_PP = 2,   /* MX++ (Sec. 4.3): MX+ and a finer shared exponent for the NBMs */
     /* The same scheme at the other element widths (Table of MX formats, Sec. 4.1-4.2):
-     * mxp_quantize and mxp_dequantize; the MXFP6 modes and plain MXFP8 also as operands of the
-     * packed x packed mxp_gemm with its full workspace (an MXFP6+ operand costs one more pass
-     * over K, its BM being entered as the sum of two E2M3 values; MXFP8 codes are read as
-     * stored), and MXFP6 / MXFP8 of mxp_gemm_prepack / mxp_gemm_prepacked; the other GEMM
-     * forms reject them, and MXFP8+ has no GEMM. */
+     * mxp_quantize and mxp_dequantize, and operands of the packed x packed mxp_gemm with its
+     * full workspace (MXFP8 codes are read as stored; an MXFP6+ operand costs one more pass
+     * over K, its BM being entered as the sum of two E2M3 values, an MXFP8+ operand two more,
+     * its BM being the sum of three E4M3 values); plain MXFP6 / MXFP8 also of mxp_gemm_prepack /
+     * mxp_gemm_prepacked; the other GEMM forms reject them. */
     MXP_MODE_MXFP6 = 3,      /* E2M3 elements, emax 2 */
     MXP_MODE_MXFP6_PLUS = 4, /* ... with the BM as sign + 5 mantissa bits: 4 + m/8, index byte */
     MXP_MODE_MXFP8 = 5,      /* E4M3 elements, emax 8 */

@@ -29,7 +29,7 @@ bool valid_packed(const mxp_packed* p, bool six_ok = false)
 {
     if (p == nullptr) return false;
     const bool six = p->mode == MXP_MODE_MXFP6 || p->mode == MXP_MODE_MXFP6_PLUS ||
-                     p->mode == MXP_MODE_MXFP8;  // (and plain MXFP8: E4M3 codes go in as they are)
+                     p->mode == MXP_MODE_MXFP8 || p->mode == MXP_MODE_MXFP8_PLUS;  // (and the 8-bit modes)
     if (!valid_mode(p->mode) && !(six_ok && six)) return false;
     if (p->rows < 0 || p->cols < 0 || p->cols % 32 != 0) return false;
     if (p->rows == 0 || p->cols == 0) return true;

@@ -493,6 +493,7 @@ struct PrepackOperand {
     int pp;                   // MX++ operand: index bits 7:5 hold delta (Sec. 4.3)
     int six;                  // source codes are packed 6-bit E2M3 (MXFP6 / MXFP6+), not nibbles
     int eight;                // source codes are E4M3 bytes (MXFP8): the MMA reads them as they are
+    int eight_plus;           // MXFP8+: E4M3 bytes whose BM is an E0M7 code, entered as three planes
     size_t plane_bytes;       // MXFP6+: distance to the second plane of the widened copy, else 0
     unsigned scale_ctas;      // row groups * ceil(nbk/128)
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
@@ -583,12 +584,56 @@ __device__ __forceinline__ void widen_six(const PrepackOperand& op, uint32_t t, 
 //    of padding, which is how kind::mxf8f6f4 reads 6-bit operands from shared memory.  The BM of
 //    an MX+ block, 4 + m/2 (Eq. 3), is the E2M3 code s 11 mmm.
 //  * E4M3 (MX++ operands, whose rescaled values need the exponent range): one byte per code.
+// E4M3 code (sign 0) of a positive integer with at most four significant bits.
+__device__ __forceinline__ uint32_t e4m3_of_small_int(uint32_t x)
+{
+    const int msb = 31 - __clz((int)x);
+    const uint32_t mant = (msb >= 3 ? x >> (msb - 3) : x << (3 - msb)) & 7u;
+    return ((uint32_t)(msb + 7) << 3) | mant;
+}
+
+// MXFP8+ (Sec. 4.1 at this width): the BM is stored as sign + seven mantissa bits and means
+// 256 + 2 m, which no single E4M3 value holds.  It is entered as the sum of three that do (Eq.
+// 4's split, carried one step further): the multiple of 32 below it (at most 448, the largest
+// E4M3 value), then the top four significant bits of the rest (at most 62, even) and what is
+// left of that (0 or 2).  Plane 0 is the stored plane with the BM replaced, planes 1 and 2 are
+// zero except at BM positions; the GEMM's K loop runs once per plane.
+__device__ __forceinline__ void widen_eight_plus(const PrepackOperand& op, uint32_t t, uint32_t b)
+{
+    uint4 o = reinterpret_cast<const uint4*>(op.nibbles)[t];
+    uint4 mid = make_uint4(0u, 0u, 0u, 0u), lo = mid;
+    const uint32_t sc = op.scales[b];
+    const uint32_t p = op.bm_index[b] & 31u;
+    if ((p >> 4) == (t & 1u)) {
+        const uint32_t e = p & 15u, sh = 8u * (e & 3u);
+        uint32_t* ow = e < 4u ? &o.x : e < 8u ? &o.y : e < 12u ? &o.z : &o.w;
+        uint32_t* mw = e < 4u ? &mid.x : e < 8u ? &mid.y : e < 12u ? &mid.z : &mid.w;
+        uint32_t* lw = e < 4u ? &lo.x : e < 8u ? &lo.y : e < 12u ? &lo.z : &lo.w;
+        const uint32_t byte = (*ow >> sh) & 255u;
+        const uint32_t sign = byte & 0x80u, v = 256u + 2u * (byte & 0x7Fu);
+        const uint32_t hi = min(v & ~31u, 448u), rem = v - hi;
+        *ow = (*ow & ~(255u << sh)) | ((sign | 0x78u | ((hi - 256u) >> 5)) << sh);
+        if (rem != 0u) {
+            const int msb = 31 - __clz((int)rem);
+            const uint32_t keep = msb > 3 ? (rem >> (msb - 3)) << (msb - 3) : rem;
+            *mw = (sign | e4m3_of_small_int(keep)) << sh;
+            if (rem != keep) *lw = (sign | e4m3_of_small_int(rem - keep)) << sh;
+        }
+    }
+    if (sc == 0u) o = mid = lo = make_uint4(0u, 0u, 0u, 0u);
+    uint8_t* dst = op.wide + (size_t)t * 16u;
+    *reinterpret_cast<uint4*>(dst) = o;
+    *reinterpret_cast<uint4*>(dst + op.plane_bytes) = mid;
+    *reinterpret_cast<uint4*>(dst + 2 * op.plane_bytes) = lo;
+}
+
 __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned id)
 {
     const uint32_t t = id * 256u + threadIdx.x;  // half block: 16 elements
     const uint32_t b = t >> 1;
     if (b >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
     if (op.six) return widen_six(op, t, b);
+    if (op.eight_plus) return widen_eight_plus(op, t, b);
     if (op.eight) {
         // MXFP8: one byte per element already; a flushed block's codes are zero by construction
         reinterpret_cast<uint4*>(op.wide)[t] = reinterpret_cast<const uint4*>(op.nibbles)[t];
@@ -687,12 +732,16 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int64_t row_groups(int64_t rows, int tile_rows) { return 2 * ((rows + tile_rows - 1) / tile_rows); }
 
 // E2M3 planes an operand is widened into: two for MXFP6+ (see widen_six), else one.
-inline int mode_parts(mxp_mode m) { return m == MXP_MODE_MXFP6_PLUS ? 2 : 1; }
+inline int mode_parts(mxp_mode m)
+{
+    return m == MXP_MODE_MXFP6_PLUS ? 2 : m == MXP_MODE_MXFP8_PLUS ? 3 : 1;
+}
 inline bool mode_six(mxp_mode m) { return m == MXP_MODE_MXFP6 || m == MXP_MODE_MXFP6_PLUS; }
-inline bool mode_eight(mxp_mode m) { return m == MXP_MODE_MXFP8; }
+inline bool mode_eight(mxp_mode m) { return m == MXP_MODE_MXFP8 || m == MXP_MODE_MXFP8_PLUS; }
 inline bool mode_plus(mxp_mode m)
 {
-    return m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP || m == MXP_MODE_MXFP6_PLUS;
+    return m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP || m == MXP_MODE_MXFP6_PLUS ||
+           m == MXP_MODE_MXFP8_PLUS;
 }
 
 // Sized for either tiling of B's scales (the tile shape is chosen per call).
@@ -778,7 +827,7 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
     if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
         return 0;
     const bool wide = a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4;
-    if (a_mode > MXP_MODE_MXFP8 || b_mode > MXP_MODE_MXFP8) return 0;  // no MXFP8+ GEMM
+    if (a_mode > MXP_MODE_MXFP8_PLUS || b_mode > MXP_MODE_MXFP8_PLUS) return 0;
     return layout(M, N, K, wide, mode_parts(a_mode), mode_parts(b_mode)).total;
 }
 
@@ -811,8 +860,9 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     op.bm_index = mode_plus(P.mode) ? P.bm_index : nullptr;
     op.pp = P.mode == MXP_MODE_MXFP4_PP;
     op.six = mode_six(P.mode);
-    op.eight = mode_eight(P.mode);
-    op.plane_bytes = P.mode == MXP_MODE_MXFP6_PLUS ? (size_t)rows * (size_t)K : 0;
+    op.eight = P.mode == MXP_MODE_MXFP8;
+    op.eight_plus = P.mode == MXP_MODE_MXFP8_PLUS;
+    op.plane_bytes = mode_parts(P.mode) > 1 ? (size_t)rows * (size_t)K : 0;
     op.atoms = atoms;
     op.wide = wide ? wide_bytes : nullptr;
     op.rows = (int)rows;
@@ -842,7 +892,7 @@ mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_
     const size_t need = stream_prepack_bytes(P.rows, P.cols, wide);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
     // an MXFP6+ operand needs two planes, which this form has no room for: mxp_gemm takes it
-    if ((P.mode > MXP_MODE_MXFP6 && !mode_eight(P.mode)) ||
+    if ((P.mode > MXP_MODE_MXFP6 && P.mode != MXP_MODE_MXFP8) ||
         ((mode_six(P.mode) || mode_eight(P.mode)) && !wide))
         return MXP_ERR_UNSUPPORTED;
     if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
@@ -888,7 +938,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     // `a_ready`: A's atoms and code slots are in the workspace already (and the status block is
     // cleared); needs a prepacked B, so that nothing is left to prepare
     if (a_ready && (b_prepacked == nullptr || A.mode > MXP_MODE_MXFP4_PLUS)) return MXP_ERR_UNSUPPORTED;
-    if (A.mode > MXP_MODE_MXFP8 || B.mode > MXP_MODE_MXFP8) return MXP_ERR_UNSUPPORTED;
+    if (A.mode > MXP_MODE_MXFP8_PLUS || B.mode > MXP_MODE_MXFP8_PLUS) return MXP_ERR_UNSUPPORTED;
     const int parts_a = mode_parts(A.mode), parts_b = mode_parts(B.mode);
     if (b_prepacked != nullptr && parts_b != 1) return MXP_ERR_UNSUPPORTED;
     const Layout l = layout(M, b_prepacked ? 0 : N, K, wide, parts_a, parts_b);

@@ -577,34 +577,53 @@ def test_tc_mxfp6_quantized_end_to_end_and_rejections():
     with pytest.raises(MxpError):   # no weight-only form for 6-bit weights
         m.mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), pw)
     p8 = m.mxp_quantize(to_dev(a), 6)
-    with pytest.raises(MxpError):   # MXFP8+ operands: quantize and decode only
-        m.mxp_gemm(p8, p8)
+    with pytest.raises(MxpError):   # an MXFP8+ operand has three planes: no prepacked form
+        m.mxp_gemm_prepack(p8, True)
 
 
 # ------------------------------------------------------------------ MXFP8 operands
 MX8 = 5
 
 
-def _raw_operand8(rows, K, seed, scale_lo=112, scale_hi=130):
-    """MXFP8 planes filled directly: every E4M3 code except the NaN pattern."""
+MX8P = 6
+
+
+def _raw_operand8(rows, K, seed, scale_lo=112, scale_hi=130, plus=False):
+    """MXFP8(+) planes filled directly: every E4M3 code except the NaN pattern and, for MXFP8+,
+    every BM position and seven-bit BM mantissa."""
     g = synth.rng(seed)
     codes = g.integers(0, 256, (rows, K), dtype=np.uint8)
     codes[(codes & 0x7F) == 0x7F] = 0x7E
     sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
     sc[g.random((rows, K // 32)) < 0.02] = 0          # flushed blocks hold zero codes
+    idx = None
+    if plus:
+        idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8)
+        bm_code = g.integers(0, 256, (rows, K // 32), dtype=np.uint8)       # sign + E0M7, 0x7F included
+        cols = (np.arange(K // 32) * 32)[None, :] + idx
+        np.put_along_axis(codes, cols, bm_code, axis=1)
     codes[np.repeat(sc == 0, 32, axis=1)] = 0
-    dec = oracle.dequantize_wide(codes, sc, None, oracle.FMT_E4M3, False)
+    dec = oracle.dequantize_wide(codes, sc, idx, oracle.FMT_E4M3, plus)
     from paper_2510_14557_b200 import Packed
-    return Packed(to_dev(codes), to_dev(sc), None, rows, K, MX8), dec
+    return Packed(to_dev(codes), to_dev(sc), to_dev(idx) if plus else None, rows, K,
+                  MX8P if plus else MX8), dec
 
 
-@pytest.mark.parametrize("amode,bmode", [(MX8, MX8), (MX8, MXP), (MX, MX8), (MX6P, MX8), (MX8, MXPP)])
+def _operand_of(rows, K, mode, seed):
+    if mode in (MX8, MX8P):
+        return _raw_operand8(rows, K, seed, plus=mode == MX8P)
+    return _any_operand(rows, K, mode, seed)
+
+
+@pytest.mark.parametrize("amode,bmode", [(MX8, MX8), (MX8, MXP), (MX, MX8), (MX6P, MX8), (MX8, MXPP),
+                                         (MX8P, MX8), (MX8, MX8P), (MX8P, MX8P), (MX8P, MXP), (MX6P, MX8P)])
 @pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 129, 384), (64, 100, 256), (513, 1000, 128)])
 def test_tc_mxfp8_operands(M, N, K, amode, bmode):
     # E4M3 elements are an operand format of the same instruction: the codes go in as stored,
     # next to 4- and 6-bit partners on the other side
-    ap, da = _raw_operand8(M, K, seed=M + 5) if amode == MX8 else _any_operand(M, K, amode, seed=M + 5)
-    bp, db = _raw_operand8(N, K, seed=N + 6) if bmode == MX8 else _any_operand(N, K, bmode, seed=N + 6)
+    # (an MXFP8+ operand: three planes, the BM being the sum of three E4M3 values)
+    ap, da = _operand_of(M, K, amode, seed=M + 5)
+    bp, db = _operand_of(N, K, bmode, seed=N + 6)
     m = mxp()
     ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode), dtype=torch.uint8, device="cuda")
     for dt in (torch.float32, torch.bfloat16):
@@ -619,6 +638,10 @@ def test_tc_mxfp8_identity_and_quantized_end_to_end():
     M, K = 384, 256
     ap, da = _raw_operand8(M, K, seed=41)
     bp, db = quantized(np.eye(K, dtype=np.float32), MX)
+    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32)
+    assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
+    # ... and for every BM position and seven-bit BM mantissa of MXFP8+ (three planes add up exactly)
+    ap, da = _raw_operand8(M, K, seed=42, plus=True)
     d = m.mxp_gemm(ap, bp, out_dtype=torch.float32)
     assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
     # quantized by the library, against the oracle's encode + decode + fp64 product
