@@ -149,7 +149,9 @@ def test_unsupported_uses_of_the_wide_modes_are_rejected():
     p8 = m.mxp_quantize(a, 6)
     with pytest.raises(MxpError):  # weight-only form: 4-bit weights only
         m.mxp_gemm(a, p6)
-    with pytest.raises(MxpError):  # MXFP8 operands: quantize and decode only
-        m.mxp_gemm(p8, p8)
+    with pytest.raises(MxpError):  # weight-only form: 4-bit weights only
+        m.mxp_gemm(a, p8)
+    with pytest.raises(MxpError):  # an MXFP8+ operand has three planes: no prepacked form
+        m.mxp_gemm_prepack(p8, True)
     with pytest.raises(MxpError):  # the + modes need the index plane
         m.mxp_quantize(a, 6, out=m.Packed(p8.nibbles, p8.scales, None, 256, 256, 6))
