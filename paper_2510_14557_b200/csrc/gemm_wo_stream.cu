@@ -255,7 +255,7 @@ __device__ __forceinline__ void normalise_block(const uint4 (&x)[4], int mulfiel
     } while (0)
 #endif
 
-// kCorr (MX+ modes, one activation row): the BM is handled by the correction warps; otherwise
+// kCorr (MX+ modes, one or two activation rows): the BM is handled by the correction warps; otherwise
 // the consumers patch it into their f16 fragments, which costs the same for any number of
 // activation columns, while the correction threads' work grows with each column.
 template <int kMT, int kMode, bool kCorr, typename OutT>
@@ -761,6 +761,18 @@ cudaError_t launch(WoParams prm, int num_sms, bool chained, cudaStream_t stream)
 }
 
 
+// Largest M for which the correction warps beat patching (measured on config 3, CUDA graph:
+// 14.1 vs 15.2 us at M = 1, 14.8 vs 15.5 at M = 2, 15.7 vs 15.6 at M = 3, 21.3 vs 17.4 at
+// M = 8).  MXP_WO_CORR_MAXM=<0..8> moves the switch-over for measurements.
+int corr_max_m()
+{
+    if (const char* e = getenv("MXP_WO_CORR_MAXM")) {
+        const int v = atoi(e);
+        return v < 0 ? 0 : (v > 8 ? 8 : v);
+    }
+    return 2;
+}
+
 }  // namespace
 
 bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
@@ -775,7 +787,7 @@ bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t
     const bool plus = B.mode != MXP_MODE_MXFP4;
     if (plus && (reinterpret_cast<uintptr_t>(B.bm_index) & 15)) return false;
     int st, rb, mb;
-    return wo_plan((int)K, M <= 8 ? 8 : 16, plus, plus && M == 1, &st, &rb, &mb);
+    return wo_plan((int)K, M <= 8 ? 8 : 16, plus, plus && M <= corr_max_m(), &st, &rb, &mb);
 }
 
 cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
@@ -811,8 +823,8 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
             return f32 ? launch<MT, 0, false, float>(prm, sms, chained, stream)            \
                        : launch<MT, 0, false, __nv_bfloat16>(prm, sms, chained, stream);   \
     }
-    // one activation row: the BM goes to the correction warps (see the kernel)
-    if (M == 1) {
+    // one or two activation rows: the BM goes to the correction warps (see the kernel)
+    if (M <= corr_max_m()) {
         MXP_WO_LAUNCH(1, true)
     }
     if (M <= 8) {

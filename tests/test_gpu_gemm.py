@@ -90,6 +90,22 @@ def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
         check_gemm(d, da, dw)
 
 
+@pytest.mark.parametrize("corr_max_m", ["0", "8"])
+@pytest.mark.parametrize("wmode", [MXP, 2])
+@pytest.mark.parametrize("M,N,K", [(1, 48, 2304), (2, 160, 4352), (3, 2384, 4096), (8, 64, 512),
+                                   (5, 20000, 1536), (1, 64, 8192)])
+def test_weight_only_bm_by_correction_warps_or_by_patch(M, N, K, wmode, corr_max_m, monkeypatch):
+    # the streamed kernel's two ways of handling the BM (correction warps: default for M <= 2;
+    # patched fragments: above), each forced over the whole range of its activation tile
+    monkeypatch.setenv("MXP_WO_KERNEL", "stream")
+    monkeypatch.setenv("MXP_WO_CORR_MAXM", corr_max_m)
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K + 1)
+    wp, dw = quantized(w_bits, wmode, bf16=True)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    for dt in (torch.float32, torch.bfloat16):
+        check_gemm(mxp().mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=dt), da, dw)
+
+
 @pytest.mark.parametrize("kernel", ["old", "stream", "tma", "fp4"])
 def test_weight_only_one_hot_and_scale_spread(kernel, monkeypatch):
     # one-hot activations select single decoded weights (exact in fp32), with weight rows and
