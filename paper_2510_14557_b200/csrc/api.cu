@@ -1,5 +1,6 @@
 // C ABI of libmxp: argument validation and dispatch.  No kernel lives here.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -195,7 +196,15 @@ size_t mxp_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense, mx
                                 mxp_mode b_mode)
 {
     if (M <= 0 || N <= 0 || K <= 0) return 0;
-    if (a_dense) return mxp::skinny_workspace_bytes(M, N, K);
+    if (a_dense) {
+        // more than 64 activation rows: the tensor-core kernel, which needs room for both
+        // operands' prepared forms; decode shapes need none
+        if (M > 64 && N >= 128) {
+            const size_t fast = mxp::stream_dense_workspace_bytes(M, N, K, b_mode);
+            if (fast != 0) return fast;
+        }
+        return mxp::skinny_workspace_bytes(M, N, K);
+    }
     return mxp::tc_workspace_bytes(M, N, K, a_mode, b_mode);
 }
 
@@ -236,6 +245,18 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (A_dense_bf16 != nullptr) {
+        if (M > 64 && N >= 128 && workspace != nullptr && aligned(workspace, 256) &&
+            aligned(B_packed->scales, 4) && getenv("MXP_WO_KERNEL") == nullptr &&
+            (B_packed->mode != MXP_MODE_MXFP4_PP || aligned(B_packed->bm_index, 4))) {
+            const size_t fast = mxp::stream_dense_workspace_bytes(M, N, K, B_packed->mode);
+            if (fast != 0 && workspace_bytes >= fast) {
+                mxp_packed none = {};
+                none.mode = MXP_MODE_MXFP4;
+                return mxp::launch_gemm_tc_stream(M, N, K, none, *B_packed, nullptr, D, d_dt, ldd,
+                                                  workspace, workspace_bytes, stream, false,
+                                                  A_dense_bf16, lda);
+            }
+        }
         cudaError_t e = mxp::launch_gemm_weight_only(M, N, K, A_dense_bf16, lda, *B_packed, D,
                                                      d_dt, ldd, workspace, workspace_bytes, stream);
         if (e == cudaErrorNotSupported) return MXP_ERR_UNSUPPORTED;

@@ -83,7 +83,11 @@ size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, 
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                                  const mxp_packed& B, const void* b_prepacked, void* D,
                                  mxp_dtype d_dt, int64_t ldd, void* workspace,
-                                 size_t workspace_bytes, cudaStream_t stream, bool a_ready = false);
+                                 size_t workspace_bytes, cudaStream_t stream, bool a_ready = false,
+                                 const void* a_dense = nullptr, int64_t lda = 0);
+// Weight-only form on the same kernel (bf16 activations as two E4M3 planes): workspace it
+// needs, 0 = not supported (K % 128, weights other than the 4-bit modes).
+size_t stream_dense_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode b_mode);
 // Quantizer that also writes A in the form that kernel reads (with a prepacked B no prepack
 // launch is left): offsets inside the GEMM's workspace, and the launch (bf16, contiguous rows,
 // MXFP4 / MXFP4+).

@@ -812,7 +812,83 @@ mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUt
                                                                                : MXP_ERR_CUDA;
 }
 
+// Weight-only form at prefill sizes (Sec. 7.1, "conversion before computation"; the paper's
+// matmul table runs M up to 4096): dense bf16 activations become an operand of the same
+// tensor-core kernel.  A bf16 value has eight significant bits, an E4M3 value four, so x = hi +
+// lo with hi = x cut to four significant bits and lo the rest, both scaled by the block's power
+// of two 2^(floor(log2 amax) - 7) (largest scaled magnitude below 256, inside E4M3's 448).  hi
+// is always exact; lo is exact for elements within 2^9 of the block's maximum and otherwise
+// rounded at 2^-10 in scaled units, i.e. below 2^-17 of the block maximum.  Two planes with
+// one E8M0 scale per block of 32: the K loop runs once per plane, like an MXFP6+ operand.
+// One thread per block of 32; rows past M (up to the next multiple of 128) get scale byte 0.
+__global__ void __launch_bounds__(256)
+prepack_dense_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int rows_pad, int nbk,
+                     uint8_t* __restrict__ atoms, uint4* __restrict__ slots, size_t plane_slots,
+                     StatusBlock* status)
+{
+    const int64_t blk = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (blk == 0 && status != nullptr) {
+        status->code = 0u;
+        status->where = 0u;
+    }
+    const int64_t row = blk / nbk;
+    const int kb = (int)(blk - row * nbk);
+    if (row >= rows_pad) return;
+    uint32_t sb = 0;
+    if (row < M) {
+        const uint4* src = reinterpret_cast<const uint4*>(A + row * lda + (int64_t)kb * 32);
+        uint32_t x[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 v = __ldg(src + i);
+            x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+        }
+        uint32_t mx = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) mx = max(mx, max(x[i] & 0x7FFFu, (x[i] >> 16) & 0x7FFFu));
+        const uint32_t E = mx >> 7;  // exponent field of the block's largest magnitude
+        sb = E > 7u ? E - 7u : 0u;
+        const float inv = __uint_as_float((254u - sb) << 23);  // 2^(127 - sb)
+        uint32_t hi[8], lo[8];  // four E4M3 codes per word
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t h = 0, l = 0;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const uint32_t w = x[2 * i + j];
+                const float x0 = __uint_as_float(w << 16), x1 = __uint_as_float(w & 0xFFFF0000u);
+                const float h0 = __uint_as_float((w << 16) & 0xFFF00000u);
+                const float h1 = __uint_as_float(w & 0xFFF00000u);
+                uint16_t hc, lc;
+                asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hc) : "f"(h1 * inv), "f"(h0 * inv));
+                asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;"
+                    : "=h"(lc)
+                    : "f"((x1 - h1) * inv), "f"((x0 - h0) * inv));
+                h |= (uint32_t)hc << (16 * j);
+                l |= (uint32_t)lc << (16 * j);
+            }
+            hi[i] = h;
+            lo[i] = l;
+        }
+        uint4* dst = slots + (row * nbk + kb) * 2;
+        dst[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        dst[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        dst[plane_slots] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        dst[plane_slots + 1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+    }
+    const int r = (int)(row & 127);
+    atoms[((row >> 7) * (nbk >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)] = (uint8_t)sb;
+}
+
 }  // namespace
+
+size_t stream_dense_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode b_mode)
+{
+    if (M < 1 || N < 1 || K % 128 != 0 || b_mode > MXP_MODE_MXFP4_PP) return 0;
+    if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 31) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
+        return 0;
+    return layout(M, N, K, true, 2, 1).total;
+}
 
 size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
 {
@@ -931,15 +1007,19 @@ bool stream_a_ready_layout(int64_t M, int64_t K, size_t* atoms, size_t* slots, s
 mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
                                  const mxp_packed& B, const void* b_prepacked, void* D,
                                  mxp_dtype d_dt, int64_t ldd, void* workspace,
-                                 size_t workspace_bytes, cudaStream_t stream, bool a_ready)
+                                 size_t workspace_bytes, cudaStream_t stream, bool a_ready,
+                                 const void* a_dense, int64_t lda)
 {
+    // `a_dense`: bf16 activations (weight-only form); `A` is then a placeholder of mode MXFP4
+    const bool dense = a_dense != nullptr;
+    if (dense && (a_ready || B.mode > MXP_MODE_MXFP4_PP)) return MXP_ERR_UNSUPPORTED;
     const bool ap = A.mode != MXP_MODE_MXFP4, bp = B.mode != MXP_MODE_MXFP4;
-    const bool wide = ap || bp || a_ready;
+    const bool wide = ap || bp || a_ready || dense;
     // `a_ready`: A's atoms and code slots are in the workspace already (and the status block is
     // cleared); needs a prepacked B, so that nothing is left to prepare
     if (a_ready && (b_prepacked == nullptr || A.mode > MXP_MODE_MXFP4_PLUS)) return MXP_ERR_UNSUPPORTED;
     if (A.mode > MXP_MODE_MXFP8_PLUS || B.mode > MXP_MODE_MXFP8_PLUS) return MXP_ERR_UNSUPPORTED;
-    const int parts_a = mode_parts(A.mode), parts_b = mode_parts(B.mode);
+    const int parts_a = dense ? 2 : mode_parts(A.mode), parts_b = mode_parts(B.mode);
     if (b_prepacked != nullptr && parts_b != 1) return MXP_ERR_UNSUPPORTED;
     const Layout l = layout(M, b_prepacked ? 0 : N, K, wide, parts_a, parts_b);
     if (workspace == nullptr || workspace_bytes < l.total) return MXP_ERR_WORKSPACE;
@@ -954,8 +1034,10 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     const int halves = choose_halves(M, N, wide, num_sms);
     const int sub = sub_n(wide, halves);
     const int rga = (int)row_groups(M, kTileM), rgb = (int)row_groups(N, sub);
-    if ((reinterpret_cast<uintptr_t>(A.nibbles) | reinterpret_cast<uintptr_t>(B.nibbles)) & 15)
+    if (((dense ? reinterpret_cast<uintptr_t>(a_dense) : reinterpret_cast<uintptr_t>(A.nibbles)) |
+         reinterpret_cast<uintptr_t>(B.nibbles)) & 15)
         return MXP_ERR_INVALID_ARG;
+    if (dense && (lda < K || lda % 8 != 0)) return MXP_ERR_INVALID_ARG;
     // the widening threads index their operand with 32 bits
     if ((uint64_t)M * nbk * 2 >= (1ull << 32) || (uint64_t)N * nbk * 2 >= (1ull << 32))
         return MXP_ERR_UNSUPPORTED;
@@ -968,8 +1050,18 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     const uint8_t* b_atoms =
         b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms[halves - 1] : ws + l.sfb;
     const uint8_t* b_wide = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.wide : ws + l.wb;
-    const PrepackOperand pa =
-        a_ready ? no_operand() : prepack_operand(A, M, K, wide, kTileM, ws + l.sfa, ws + l.wa);
+    if (dense) {
+        const int rows_pad = rga * 128;
+        const int64_t blocks = (int64_t)rows_pad * nbk;
+        prepack_dense_kernel<<<(unsigned)((blocks + 255) / 256), 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(a_dense), lda, (int)M, rows_pad, nbk, ws + l.sfa,
+            reinterpret_cast<uint4*>(ws + l.wa), (size_t)M * (size_t)K / 16,
+            static_cast<StatusBlock*>(workspace));
+        if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+    }
+    const PrepackOperand pa = (a_ready || dense)
+                                  ? no_operand()
+                                  : prepack_operand(A, M, K, wide, kTileM, ws + l.sfa, ws + l.wa);
     const PrepackOperand pb =
         b_prepacked ? no_operand() : prepack_operand(B, N, K, wide, sub, ws + l.sfb, ws + l.wb);
     const uint64_t ctas = (uint64_t)pa.scale_ctas + pb.scale_ctas + pa.widen_ctas + pb.widen_ctas;
@@ -994,7 +1086,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     prm.M = (int)M;
     prm.N = (int)N;
     prm.K = (int)K;
-    prm.a_fmt = (A.mode == MXP_MODE_MXFP4_PP || mode_eight(A.mode)) ? kFmtE4M3 : kFmtE2M3;
+    prm.a_fmt = (dense || A.mode == MXP_MODE_MXFP4_PP || mode_eight(A.mode)) ? kFmtE4M3 : kFmtE2M3;
     prm.b_fmt = (B.mode == MXP_MODE_MXFP4_PP || mode_eight(B.mode)) ? kFmtE4M3 : kFmtE2M3;
     prm.parts_a = parts_a;
     prm.parts_b = parts_b;

@@ -198,6 +198,51 @@ def test_weight_only_chained_rejects_what_it_cannot_run():
     assert e.value.status == 2
 
 
+# ------------------------------------------------------------------ weight-only form, prefill sizes
+@pytest.mark.parametrize("wmode", [MX, MXP, 2])
+@pytest.mark.parametrize("M,N,K", [(65, 128, 128), (128, 520, 1024), (300, 1000, 384), (513, 129, 2048)])
+def test_weight_only_many_rows_on_the_tensor_cores(M, N, K, wmode):
+    # more than 64 activation rows: bf16 activations enter the block-scaled tensor-core kernel as
+    # two E4M3 planes (hi + lo) with a power-of-two scale per block of 32
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K)
+    wp, dw = quantized(w_bits, wmode, bf16=True)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    m = mxp()
+    need = m.mxp_gemm_workspace_bytes(M, N, K, True, 0, wmode)
+    assert need > 4096                                  # the tensor-core path is on offer
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=dt, workspace=ws)
+        assert m.mxp_gemm_status(ws) == 0
+        check_gemm(d, da, dw)
+    # without the workspace the general kernel answers, same result within the same bound
+    d = m.mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=torch.float32,
+                   workspace=torch.zeros(4096, dtype=torch.uint8, device="cuda"))
+    check_gemm(d, da, dw)
+
+
+def test_weight_only_many_rows_one_hot_and_magnitude_spread():
+    # one-hot activation rows return single decoded weights exactly (hi carries the value, lo is
+    # zero); rows whose blocks mix magnitudes 2^20 apart stay inside the bound (the small
+    # elements lose bits of their lo part only)
+    M, N, K = 128, 256, 512
+    g = synth.rng(17)
+    w = g.standard_normal((N, K)).astype(np.float32) * np.exp2(g.integers(-20, 20, (N, 1))).astype(np.float32)
+    wp, dw = quantized(w, MXP)
+    a = np.zeros((M, K), np.float32)
+    for r in range(64):
+        a[r, (r * 37) % K] = 2.0 ** (r - 30) * (1.0 + (r % 8) / 8.0)
+    a[64:] = g.standard_normal((64, K)) * np.exp2(g.integers(-20, 1, (64, K)))
+    a_bits = synth.f32_to_bf16_bits(a)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    d = mxp().mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=torch.float32)
+    got = d.cpu().numpy().astype(np.float64)
+    for r in range(64):
+        want = (dw[:, (r * 37) % K] * da[r, (r * 37) % K]).astype(np.float32).astype(np.float64)
+        assert np.array_equal(got[r], want)
+    check_gemm(d, da, dw)
+
+
 # ------------------------------------------------------------------ tensor-core form
 MODES = [(MX, MX), (MXP, MX), (MX, MXP), (MXP, MXP)]
 
