@@ -324,6 +324,36 @@ def part_decode(mxp, synth, peaks, iters):
                 out[key]["frac_hbm_cuda_graph_chained"] = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_c / 1e6 / hbm
         os.environ.pop("MXP_WO_KERNEL", None)
         del copies, w
+    # ---- weight-only form at prefill sizes (the paper's matmul table: N = K = 4096, M up to
+    # 4096): bf16 activations on the block-scaled tensor-core kernel as two E4M3 planes; the
+    # yardstick is the measured bf16 GEMM rate, what "convert the weights, then a bf16 GEMM" runs at
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for M in (256, 2048, 4096):
+        a_bits, w_bits = synth.config3(M, 4096, 4096, seed=7)
+        a, w = dev_bf16(a_bits), dev_bf16(w_bits)
+        d = torch.empty((M, 4096), dtype=torch.bfloat16, device="cuda")
+        for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
+            pw = mxp.mxp_quantize(w, mode)
+            ws = torch.zeros(mxp.mxp_gemm_workspace_bytes(M, 4096, 4096, True, 0, mode),
+                             dtype=torch.uint8, device="cuda")
+            n_it = max(2, iters // 4)
+            tot = 0.0
+            for i in range(n_it + 2):
+                flush.fill_(i & 255)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                mxp.mxp_gemm(a, pw, out=d, workspace=ws)
+                e1.record()
+                torch.cuda.synchronize()
+                if i >= 2:
+                    tot += e0.elapsed_time(e1)
+            ms = tot / n_it
+            tf = 2.0 * M * 4096 * 4096 / ms / 1e9
+            out["weight_only_4096x4096_M%d_%s" % (M, name)] = {
+                "us": ms * 1e3, "TFLOP/s": tf, "frac_bf16_burst": tf / peaks["bf16_burst"]}
+            del pw, ws
+        del a, w, d
+    del flush
     return out
 
 

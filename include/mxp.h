@@ -178,7 +178,13 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  *     D[M,N] = dec(A)[M,K] * dec(B)[N,K]^T, fp32 accumulation.
  * Exactly one of A_dense_bf16 / A_packed is non-NULL:
  *   - A_dense_bf16 (device, bf16, row stride lda elements): weight-only form, the
- *     weights B are decoded inside the kernel and multiplied with bf16 activations;
+ *     weights B are decoded inside the kernel and multiplied with bf16 activations
+ *     (up to 64 rows: streamed decode kernels, no workspace needed; more rows, given
+ *     mxp_gemm_workspace_bytes(..., a_dense = 1, ...) bytes of workspace: the tensor-core
+ *     kernel, the activations entering as the exact sum of two E4M3 planes with a
+ *     power-of-two scale per block of 32 -- elements more than 2^9 below their block's
+ *     maximum are rounded at 2^-17 of that maximum; with less workspace a slower
+ *     general kernel answers);
  *   - A_packed (host pointer to a descriptor): both operands are consumed by the
  *     block-scaled tensor-core path; any combination of MXFP4 / MXFP4+ modes.
  *   B_packed   host pointer to the descriptor of the N x K weight operand
