@@ -239,6 +239,14 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
  *                           to mxp_gemm).  Same result as mxp_gemm.
  * The paper describes the format and its decode (Sec. 4, Eq. 3), not this staging: it is
  * an implementation device of this library.
+ *   mxp_gemm_dense_prepacked  the weight-only form (bf16 activations, more than one tile's
+ *                           worth of rows is where it pays: see mxp_gemm) with B's prepacked
+ *                           copy, which must have been made with wide != 0.  Workspace
+ *                           (device, 256-byte aligned): at least
+ *                           mxp_gemm_dense_prepacked_workspace_bytes(M, K) bytes (0: shape
+ *                           not supported), which hold the activations' two planes and
+ *                           scales.  Any M >= 1; 4-bit weight modes; K % 128 == 0.  Same
+ *                           result as mxp_gemm's tensor-core weight-only path.
  */
 size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide);
 mxp_status mxp_gemm_prepack(const mxp_packed *P, int wide, void *out, size_t out_bytes,
@@ -247,6 +255,12 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed 
                               const mxp_packed *B_packed, const void *B_prepacked, void *D,
                               mxp_dtype d_dt, int64_t ldd, void *workspace,
                               size_t workspace_bytes, void *cuda_stream);
+size_t mxp_gemm_dense_prepacked_workspace_bytes(int64_t M, int64_t K);
+mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16,
+                                    int64_t lda, const mxp_packed *B_packed,
+                                    const void *B_prepacked, void *D, mxp_dtype d_dt,
+                                    int64_t ldd, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream);
 
 /*
  * Quantization fused with the preparation of the GEMM operand (Sec. 5, software integration:

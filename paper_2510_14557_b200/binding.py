@@ -27,6 +27,7 @@ LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
 EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
+           "mxp_gemm_dense_prepacked", "mxp_gemm_dense_prepacked_workspace_bytes",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
            "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
@@ -64,6 +65,11 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_noalloc.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
                                        vp, ci, i64, ctypes.POINTER(ci), vp]
         l.mxp_gemm_noalloc.restype = ci
+        l.mxp_gemm_dense_prepacked_workspace_bytes.argtypes = [i64, i64]
+        l.mxp_gemm_dense_prepacked_workspace_bytes.restype = sz
+        l.mxp_gemm_dense_prepacked.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, vp, ci,
+                                               i64, vp, sz, vp]
+        l.mxp_gemm_dense_prepacked.restype = ci
         l.mxp_quantize_reordered.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp, vp, vp, vp]
         l.mxp_quantize_reordered.restype = ci
         l.mxp_nvfp4_quantize.argtypes = [vp, ci, i64, i64, i64, ctypes.c_float, ci, vp, vp, vp, vp]
@@ -362,6 +368,27 @@ def mxp_gemm_decode_chained(a: torch.Tensor, b: Packed, out: torch.Tensor,
                                        status_block.data_ptr() if status_block is not None else None,
                                        _stream())
     _check("mxp_gemm_decode_chained", st)
+    return out
+
+
+def mxp_gemm_dense_prepacked(a: torch.Tensor, b: Packed, b_prepacked: torch.Tensor,
+                             out_dtype=torch.bfloat16, out: Optional[torch.Tensor] = None,
+                             workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Weight-only GEMM on the tensor-core kernel with B's prepacked copy
+    (mxp_gemm_prepack(b, True)); `a` is a bf16 CUDA tensor with any number of rows."""
+    assert a.dtype == torch.bfloat16 and a.is_cuda and a.stride(1) == 1
+    M, N, K = a.shape[0], b.rows, b.cols
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=a.device)
+    need = int(lib().mxp_gemm_dense_prepacked_workspace_bytes(M, K))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=a.device)
+    bs = b.c_struct()
+    st = lib().mxp_gemm_dense_prepacked(M, N, K, a.data_ptr(), a.stride(0), ctypes.byref(bs),
+                                        b_prepacked.data_ptr(), out.data_ptr(), _dt(out),
+                                        out.stride(0), workspace.data_ptr(), workspace.numel(),
+                                        _stream())
+    _check("mxp_gemm_dense_prepacked", st)
     return out
 
 

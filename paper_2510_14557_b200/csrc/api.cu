@@ -325,6 +325,34 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
                                       static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t mxp_gemm_dense_prepacked_workspace_bytes(int64_t M, int64_t K)
+{
+    return mxp::stream_dense_prepacked_workspace_bytes(M, K);
+}
+
+mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16,
+                                    int64_t lda, const mxp_packed* B_packed,
+                                    const void* B_prepacked, void* D, mxp_dtype d_dt, int64_t ldd,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!valid_dtype(d_dt) || A_dense_bf16 == nullptr) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(B_packed, false)) return MXP_ERR_INVALID_ARG;
+    if (B_packed->rows != N || B_packed->cols != K) return MXP_ERR_INVALID_ARG;
+    if (lda < K || lda % 8 != 0 || !aligned(A_dense_bf16, 16)) return MXP_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return MXP_OK;
+    if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
+    const size_t need = mxp::stream_dense_prepacked_workspace_bytes(M, K);
+    if (need == 0 || mxp::stream_prepack_bytes(N, K, true) == 0) return MXP_ERR_UNSUPPORTED;
+    if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
+    mxp_packed none = {};
+    none.mode = MXP_MODE_MXFP4;
+    return mxp::launch_gemm_tc_stream(M, N, K, none, *B_packed, B_prepacked, D, d_dt, ldd, workspace,
+                                      workspace_bytes, static_cast<cudaStream_t>(cuda_stream),
+                                      false, A_dense_bf16, lda);
+}
+
 mxp_status mxp_quantize_gemm_ready(const void* src, mxp_dtype src_dt, int64_t M, int64_t K,
                                    int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
                                    uint8_t* bm_index, void* workspace, size_t workspace_bytes,

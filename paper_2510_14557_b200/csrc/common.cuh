@@ -88,6 +88,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
 // Weight-only form on the same kernel (bf16 activations as two E4M3 planes): workspace it
 // needs, 0 = not supported (K % 128, weights other than the 4-bit modes).
 size_t stream_dense_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode b_mode);
+size_t stream_dense_prepacked_workspace_bytes(int64_t M, int64_t K);  // with B prepacked
 // Quantizer that also writes A in the form that kernel reads (with a prepacked B no prepack
 // launch is left): offsets inside the GEMM's workspace, and the launch (bf16, contiguous rows,
 // MXFP4 / MXFP4+).

@@ -890,6 +890,12 @@ size_t stream_dense_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode b_
     return layout(M, N, K, true, 2, 1).total;
 }
 
+size_t stream_dense_prepacked_workspace_bytes(int64_t M, int64_t K)
+{
+    if (M < 1 || K < 128 || K % 128 != 0 || (uint64_t)M * (uint64_t)K / 16 >= (1ull << 31)) return 0;
+    return layout(M, 0, K, true, 2, 1).total;
+}
+
 size_t stream_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
 {
     // Small M or N is better served by the in-place single-CTA kernel, except for MX++

@@ -99,6 +99,13 @@ def test_argument_validation_of_the_later_entry_points(lib):
     assert ch(100, 32, 256, fake, 256, ctypes.byref(b), fake, 1, 32, null, null) == 2  # M > 64
     b6 = _Packed(4096, 4096, None, 32, 256, 3)
     assert ch(1, 32, 256, fake, 256, ctypes.byref(b6), fake, 1, 32, null, null) == 1  # 6-bit weights
+    dp = lib.mxp_gemm_dense_prepacked
+    assert dp(70, 32, 256, null, 256, ctypes.byref(b), fake, fake, 1, 32, fake, 1 << 20, null) == 1  # no activations
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), null, fake, 1, 32, fake, 1 << 20, null) == 1  # no prepacked copy
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b6), fake, fake, 1, 32, fake, 1 << 20, null) == 1  # 6-bit weights
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), fake, fake, 1, 32, fake, 16, null) == 3       # workspace
+    assert lib.mxp_gemm_dense_prepacked_workspace_bytes(70, 256) > 70 * 256 * 2
+    assert lib.mxp_gemm_dense_prepacked_workspace_bytes(70, 96) == 0
     # the ordering rule runs on the host
     cnt = np.arange(64, dtype=np.int64)
     out = np.zeros(64, np.int32)

@@ -221,6 +221,28 @@ def test_weight_only_many_rows_on_the_tensor_cores(M, N, K, wmode):
     check_gemm(d, da, dw)
 
 
+@pytest.mark.parametrize("wmode", [MX, MXP, 2])
+@pytest.mark.parametrize("M,N,K", [(1, 256, 512), (16, 1000, 384), (65, 520, 1024), (300, 129, 2048)])
+def test_weight_only_with_prepacked_weights(M, N, K, wmode):
+    # the same tensor-core path with the weights prepared once; any number of activation rows
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K + 2)
+    wp, dw = quantized(w_bits, wmode, bf16=True)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    m = mxp()
+    pre = m.mxp_gemm_prepack(wp, True)
+    a = to_dev_bf16(a_bits)
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm_dense_prepacked(a, wp, pre, out_dtype=dt)
+        check_gemm(d, da, dw)
+    if M > 64:   # what mxp_gemm's own tensor-core path returns, bit for bit
+        d0 = m.mxp_gemm(a, wp, out_dtype=torch.float32)
+        d1 = m.mxp_gemm_dense_prepacked(a, wp, pre, out_dtype=torch.float32)
+        assert torch.equal(d0.view(torch.int32), d1.view(torch.int32))
+    from paper_2510_14557_b200 import MxpError
+    with pytest.raises(MxpError):   # workspace too small
+        m.mxp_gemm_dense_prepacked(a, wp, pre, workspace=torch.zeros(256, dtype=torch.uint8, device="cuda"))
+
+
 def test_weight_only_many_rows_one_hot_and_magnitude_spread():
     # one-hot activation rows return single decoded weights exactly (hi carries the value, lo is
     # zero); rows whose blocks mix magnitudes 2^20 apart stay inside the bound (the small
