@@ -826,6 +826,7 @@ prepack_dense_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, in
                      uint8_t* __restrict__ atoms, uint4* __restrict__ slots, size_t plane_slots,
                      StatusBlock* status)
 {
+    ptx::grid_launch_dependents();  // the GEMM's prologue may start while this grid drains
     const int64_t blk = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (blk == 0 && status != nullptr) {
         status->code = 0u;
