@@ -1,0 +1,87 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times,
+on sampled outputs the oracle computes one by one (configs 2, 4 and 5; config 3 is covered in
+test_gpu_gemm.py)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_gemm, to_dev_bf16
+from paper_2510_14557_b200 import synth
+
+pytestmark = pytest.mark.gpu
+MX, MXP, MXPP = 0, 1, 2
+
+
+def mxp():
+    import paper_2510_14557_b200 as m
+    return m
+
+
+def sample(n, step, extra):
+    return np.unique(np.concatenate([np.arange(0, n, step), np.asarray(extra)]))
+
+
+@pytest.mark.parametrize("mode", [MX, MXP, MXPP])
+def test_quantize_config2_sampled_rows_bit_exact(mode):
+    # 8192 x 8192 bf16 through the one-lane-per-block kernel; every plane of the sampled rows
+    bits = synth.config2()
+    p = mxp().mxp_quantize(to_dev_bf16(bits), mode)
+    rows = sample(8192, 331, [8191, 8190, 4095, 4096])
+    ref = oracle.quantize(bits[rows], mode, bf16_bits=True)
+    sel = torch.from_numpy(rows).cuda()
+    assert np.array_equal(p.nibbles[sel].cpu().numpy(), ref[0])
+    assert np.array_equal(p.scales[sel].cpu().numpy(), ref[1])
+    if mode != MX:
+        assert np.array_equal(p.bm_index[sel].cpu().numpy(), ref[2])
+    # decode of the full matrix, sampled rows, exact
+    d = mxp().mxp_dequantize(p, torch.float32)
+    want = oracle.dequantize(ref[0], ref[1], ref[2], mode)
+    assert np.array_equal(d[sel].cpu().numpy().astype(np.float64), want)
+
+
+def _bench_step_parity(a_bits, w_bits, row_step, col_step):
+    """The benchmark's step: weights quantized and prepacked once; activations through the fused
+    quantizer (packed planes + GEMM-ready planes), then the GEMM on the prepared operands."""
+    m = mxp()
+    M, K = a_bits.shape
+    N = w_bits.shape[0]
+    w = to_dev_bf16(w_bits)
+    pw = m.mxp_quantize(w, MXP)
+    pre = m.mxp_gemm_prepack(pw, True)
+    del w
+    ws = torch.zeros(max(4096, m.mxp_gemm_workspace_bytes(M, N, K, False, MXP, MXP)),
+                     dtype=torch.uint8, device="cuda")
+    a = to_dev_bf16(a_bits)
+    pa = m.mxp_quantize_gemm_ready(a, MXP, ws)
+    d = m.mxp_gemm_ready(pa, pw, pre, ws, out_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    assert m.mxp_gemm_status(ws) == 0
+    rows = sample(M, row_step, [M - 1, M - 2, 255, 256, 257])
+    cols = sample(N, col_step, [N - 1, N - 2, 239, 240, 479, 480, 481])
+    qa = oracle.quantize(a_bits[rows], MXP, bf16_bits=True)
+    qw = oracle.quantize(w_bits[cols], MXP, bf16_bits=True)
+    # the encodings the GEMM consumed are the oracle's, bit for bit
+    rsel, csel = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    assert np.array_equal(pa.nibbles[rsel].cpu().numpy(), qa[0])
+    assert np.array_equal(pa.scales[rsel].cpu().numpy(), qa[1])
+    assert np.array_equal(pa.bm_index[rsel].cpu().numpy(), qa[2])
+    assert np.array_equal(pw.nibbles[csel].cpu().numpy(), qw[0])
+    assert np.array_equal(pw.bm_index[csel].cpu().numpy(), qw[2])
+    da = oracle.dequantize(qa[0], qa[1], qa[2], MXP)
+    dw = oracle.dequantize(qw[0], qw[1], qw[2], MXP)
+    check_gemm(d[rsel][:, csel], da, dw)
+    # the same operands through plain mxp_gemm (prepack inside the call): identical output
+    d2 = m.mxp_gemm(pa, pw, out_dtype=torch.bfloat16, workspace=ws)
+    assert torch.equal(d2[rsel][:, csel], d[rsel][:, csel])
+
+
+def test_prefill_config4_bench_step_sampled():
+    a_bits, w_bits = synth.config4()
+    _bench_step_parity(a_bits, w_bits, row_step=97, col_step=61)
+
+
+def test_prefill_config5_bench_step_sampled():
+    # the headline workload: 8192 x 8192 activations, 28672 x 8192 weights
+    a_bits, w_bits = synth.config5()
+    _bench_step_parity(a_bits, w_bits, row_step=409, col_step=449)
