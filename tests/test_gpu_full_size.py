@@ -85,3 +85,25 @@ def test_prefill_config5_bench_step_sampled():
     # the headline workload: 8192 x 8192 activations, 28672 x 8192 weights
     a_bits, w_bits = synth.config5()
     _bench_step_parity(a_bits, w_bits, row_step=409, col_step=449)
+
+
+def test_weight_only_4096_cubed_sampled():
+    # the largest shape of the paper's matmul table (M = N = K = 4096), weight-only form: the
+    # tensor-core path as mxp_gemm takes it and with the weights prepacked once
+    m = mxp()
+    M = N = K = 4096
+    a_bits, w_bits = synth.config3(M, N, K, seed=7)
+    pw = m.mxp_quantize(to_dev_bf16(w_bits), MXP)
+    a = to_dev_bf16(a_bits)
+    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, True, 0, MXP), dtype=torch.uint8, device="cuda")
+    d = m.mxp_gemm(a, pw, out_dtype=torch.bfloat16, workspace=ws)
+    assert m.mxp_gemm_status(ws) == 0
+    d2 = m.mxp_gemm_dense_prepacked(a, pw, m.mxp_gemm_prepack(pw, True), out_dtype=torch.bfloat16)
+    rows = sample(M, 211, [M - 1, 255, 256])
+    cols = sample(N, 173, [N - 1, 239, 240, 479, 480])
+    qw = oracle.quantize(w_bits[cols], MXP, bf16_bits=True)
+    dw = oracle.dequantize(qw[0], qw[1], qw[2], MXP)
+    da = oracle.bf16_bits_to_f64(a_bits[rows])
+    rsel, csel = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    check_gemm(d[rsel][:, csel], da, dw)
+    assert torch.equal(d, d2)
