@@ -134,7 +134,8 @@ mxp_status mxp_channel_order(const int64_t *outlier_count, int64_t cols, int32_t
  * a 4-bit BM index per block; blocks whose scale byte is 00000010b or less keep the plain
  * NVFP4 form and index 0.
  *
- *   tensor_scale  the per-tensor fp32 scale, chosen by the caller, > 0 and finite (the usual
+ *   tensor_scale  the per-tensor fp32 scale, chosen by the caller, 2^-100 <= ts <= 2^100,
+ *                 MXP_ERR_INVALID_ARG otherwise (the usual
  *                 choice: largest magnitude of the tensor / (6 * 448), so that block scales
  *                 use the E4M3 range; a larger value pushes more blocks into the fallback)
  *   plus          0: NVFP4, != 0: NVFP4+
@@ -144,14 +145,14 @@ mxp_status mxp_channel_order(const int64_t *outlier_count, int64_t cols, int32_t
  *                 the low nibble; NULL allowed iff plus == 0 (then not written / not read)
  *   cols % 32 == 0; src / dst rows 16-byte aligned (ld % 8 == 0), nibbles 16-byte aligned.
  *
- * What is computed, each step one IEEE binary32 operation (the paper fixes none; the CPU
- * oracle of the test suite follows the same steps, so the codes are bit-exact):
- *   q = amax / (6 * tensor_scale);  scale byte = E4M3(q), round to nearest even, saturating
- *   at 448;  d = value(scale byte) * tensor_scale;  r = 1 / d;  element codes = E2M1(x * r),
- *   round to nearest even, saturating at 6, sign of x kept;  scale byte 0: all codes 0;
- *   BM (first of equal maxima), NVFP4+ only: m = nearest-even((clamp(amax * r, 4, 8) - 4) * 2),
- *   at most 7.  Decode: x = +-E * d, E the E2M1 value or 4 + m/2, one rounding to binary32
- *   (then to bf16, nearest even, for a bf16 destination).
+ * What is computed is the definition in real numbers, not a floating-point recipe (the codes
+ * are those of exact arithmetic; the CPU oracle of the test suite states the same in binary64):
+ *   q = amax / (6 * tensor_scale);  scale byte = the E4M3 value nearest to q, ties to the even
+ *   byte, saturating at 448;  d = value(scale byte) * tensor_scale;  element codes = the E2M1
+ *   value nearest to |x| / d, ties to the even code, saturating at 6, sign of x kept;  scale
+ *   byte 0: all codes 0;  BM (first of equal maxima), NVFP4+ only: m = the integer nearest to
+ *   (clamp(amax / d, 4, 8) - 4) * 2, ties to even, at most 7.  Decode: x = +-E * d, E the E2M1
+ *   value or 4 + m/2, rounded once (nearest even) to the destination type, fp32 or bf16.
  * Inf / NaN inputs are outside the contract.
  */
 mxp_status mxp_nvfp4_quantize(const void *src, mxp_dtype src_dt, int64_t rows, int64_t cols,

@@ -46,7 +46,9 @@ def build(force: bool = False) -> str:
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
+        # MXP_ORACLE_LIB: an already built alternative (the mutation test loads deliberately
+        # broken copies of mxp_oracle.c through it to show that the pins notice)
+        lib = ctypes.CDLL(os.environ.get("MXP_ORACLE_LIB") or build())
         i64, p, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
         lib.oracle_quantize.argtypes = [p, ci, i64, i64, i64, ci, ci, p, p, p]
         lib.oracle_quantize.restype = ci
@@ -68,7 +70,7 @@ def _load():
         lib.oracle_nvfp4_quantize.restype = ci
         lib.oracle_nvfp4_dequantize.argtypes = [p, p, p, i64, i64, ctypes.c_float, ci, p]
         lib.oracle_nvfp4_dequantize.restype = ci
-        lib.oracle_e4m3_round.argtypes = [ctypes.c_float]
+        lib.oracle_e4m3_round.argtypes = [ctypes.c_double]
         lib.oracle_e4m3_round.restype = ci
         lib.oracle_pack6.argtypes = [p, i64, p]
         lib.oracle_pack6.restype = None
@@ -293,12 +295,13 @@ def nvfp4_quantize(x: np.ndarray, tensor_scale: float, plus: bool, bf16_bits: bo
 
 
 def nvfp4_dequantize(nib: np.ndarray, sc: np.ndarray, idx, tensor_scale: float, plus: bool) -> np.ndarray:
-    """Decoded values as float32 (the definition rounds once to binary32)."""
+    """Decoded values as float64, exact (E * value(scale byte) * tensor_scale has at most 32
+    significant bits); a consumer rounds once to its own output type."""
     nib = np.ascontiguousarray(nib, np.uint8)
     sc = np.ascontiguousarray(sc, np.uint8)
     rows, cols = nib.shape[0], nib.shape[1] * 2
     idx = np.zeros((rows, cols // 32), np.uint8) if idx is None else np.ascontiguousarray(idx, np.uint8)
-    out = np.zeros((rows, cols), np.float32)
+    out = np.zeros((rows, cols), np.float64)
     rc = _load().oracle_nvfp4_dequantize(_ptr(nib), _ptr(sc), _ptr(idx), rows, cols,
                                          float(tensor_scale), int(plus), _ptr(out))
     if rc != 0:

@@ -492,57 +492,61 @@ void oracle_pack6(const uint8_t *codes, int64_t n, uint8_t *out)
  * scale byte is 00000010b or smaller keep the plain NVFP4 form (their scale is too coarse for
  * the BM to land in [4, 8) reliably); their index nibble is 0.
  *
- * The passage fixes neither the arithmetic nor the layout.  Readings taken here:
- *   - all scale arithmetic is IEEE binary32, one rounding per step, in this order:
- *       q = amax / (6 * ts)          (the product 6 * ts rounded first, then the division)
- *       scale byte = E4M3(q), round to nearest, ties to even, saturating at 448
- *       d = value(scale byte) * ts ; r = 1 / d ; scaled_i = x_i * r
- *   - scaled_i -> E2M1, round to nearest, ties to even code, saturating at 6; the sign bit of
- *     the input is kept even when the magnitude rounds to zero;
+ * The passage says that the scale maps the BM as closely as possible onto the largest E2M1
+ * magnitude and that elements are the inputs divided by the scale; it fixes neither the
+ * rounding nor the layout.  Readings taken here (the definition, in real numbers):
+ *       q = amax / (6 * ts);  scale byte = the E4M3 value nearest to q, ties to the even
+ *       byte, saturating at 448;  d = value(scale byte) * ts  (exact);
+ *       code_i = the E2M1 value nearest to abs(x_i) / d, ties to the even code, saturating at 6;
+ *       the sign bit of the input is kept even when the magnitude rounds to zero;
  *   - scale byte 0 (amax too small for the tensor scale): all codes 0, index 0;
- *   - BM = first element with the largest magnitude; m = round-to-nearest-even((v - 4) * 2)
- *     with v = amax * r, clamped to 0..7 (v can leave [4, 8) only when the scale saturated);
+ *   - BM = first element with the largest magnitude; m = nearest integer to (v - 4) * 2, ties to
+ *     the even m, with v = amax / d clamped to [4, 8] and m to 0..7 (v leaves [4, 8) only when
+ *     the scale saturated);
  *   - element 2j in the low nibble of byte j; one scale byte per block; index nibbles two per
  *     byte, block 2j of a row in the low nibble (cols % 32 == 0 keeps rows byte aligned);
- *   - decode: x_i = +-E_i * d with d as above and one binary32 rounding of the product.
+ *   - decode: x_i = +-E_i * d, E_i the E2M1 value or 4 + m/2 for the BM (exact; a consumer
+ *     rounds it once to its output type).
+ * Arithmetic: doubles.  6 * ts (26 bits), value(byte) * ts (28 bits) and every decoded value
+ * (at most 32 bits) are exact.  The two quotients are rounded at 2^-53; that cannot move a
+ * value across a rounding boundary or onto one: a quotient of a 24-bit by a 28-bit number (or
+ * its boundary t, at most 5 bits, cross-multiplied: x vs t * d, at most 33 bits) is either
+ * exactly the boundary -- then the division is exact -- or differs from it by more than
+ * 2^-34 of its size.
  * Parity unpinned: Inf / NaN inputs, ts <= 0.
  * ------------------------------------------------------------------------------------------ */
-static float f32_mul(float a, float b) { volatile float r = a * b; return r; }
-static float f32_div(float a, float b) { volatile float r = a / b; return r; }
 
 /* E4M3 byte (sign 0) nearest to q >= 0, saturating: the search over the type's 127 finite
  * magnitudes used for MXFP8 elements above. */
-int oracle_e4m3_round(float q) { return elem_nearest(ORACLE_FMT_E4M3, (double)q); }
+int oracle_e4m3_round(double q) { return elem_nearest(ORACLE_FMT_E4M3, q); }
 
-static void nvfp4_block(const float *x, float ts, int plus, uint8_t *nib, uint8_t *scale,
+static void nvfp4_block(const double *x, double ts, int plus, uint8_t *nib, uint8_t *scale,
                         int *index)
 {
-    float amax = 0.0f;
+    double amax = 0.0;
     int bm = 0;
     for (int i = 0; i < 16; ++i) {
-        float a = fabsf(x[i]);
+        double a = fabs(x[i]);
         if (a > amax) {
             amax = a;
             bm = i;
         }
     }
-    float q = f32_div(amax, f32_mul(6.0f, ts));
-    int sb = oracle_e4m3_round(q);
+    int sb = oracle_e4m3_round(amax / (6.0 * ts));
     *scale = (uint8_t)sb;
     *index = 0;
     memset(nib, 0, 8);
     if (sb == 0)
         return;
-    float d = f32_mul((float)oracle_elem_value(ORACLE_FMT_E4M3, sb), ts);
-    float r = f32_div(1.0f, d);
+    double d = oracle_elem_value(ORACLE_FMT_E4M3, sb) * ts;
     int extend = plus && sb > 2;
     for (int i = 0; i < 16; ++i) {
-        float sc = f32_mul(x[i], r);
+        double v = fabs(x[i]) / d;
         int code;
         if (extend && i == bm)
-            code = bm_code(fmin(fmax((double)fabsf(sc), 4.0), 8.0));
+            code = bm_code(fmin(fmax(v, 4.0), 8.0));
         else
-            code = e2m1_nearest((double)fabsf(sc));
+            code = e2m1_nearest(v);
         if (signbit(x[i]))
             code |= 8;
         nib[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
@@ -559,17 +563,20 @@ int oracle_nvfp4_quantize(const void *src, int src_kind, int64_t rows, int64_t c
     if (rows < 0 || cols < 0 || cols % 32 != 0 || (src_kind != 0 && src_kind != 1))
         return -1;
     int64_t nb = cols / 16;
+#ifdef _OPENMP
 #pragma omp parallel for num_threads(g_threads) schedule(static)
+#endif
     for (int64_t r = 0; r < rows; ++r) {
         for (int64_t b = 0; b < nb; ++b) {
-            float x[16];
+            double x[16];
             for (int i = 0; i < 16; ++i) {
                 int64_t e = r * cols + b * 16 + i;
-                x[i] = src_kind == 0 ? ((const float *)src)[e]
-                                     : (float)bf16_to_double(((const uint16_t *)src)[e]);
+                x[i] = src_kind == 0 ? (double)((const float *)src)[e]
+                                     : bf16_to_double(((const uint16_t *)src)[e]);
             }
             int idx;
-            nvfp4_block(x, ts, plus, nibbles + (r * nb + b) * 8, scales + r * nb + b, &idx);
+            nvfp4_block(x, (double)ts, plus, nibbles + (r * nb + b) * 8, scales + r * nb + b,
+                        &idx);
             uint8_t *ib = bm_index + (r * nb + b) / 2;
             if (b & 1)
                 *ib = (uint8_t)((*ib & 0x0F) | (idx << 4));
@@ -580,25 +587,28 @@ int oracle_nvfp4_quantize(const void *src, int src_kind, int64_t rows, int64_t c
     return 0;
 }
 
+/* Decoded values as doubles (exact). */
 int oracle_nvfp4_dequantize(const uint8_t *nibbles, const uint8_t *scales,
                             const uint8_t *bm_index, int64_t rows, int64_t cols, float ts,
-                            int plus, float *out)
+                            int plus, double *out)
 {
     if (rows < 0 || cols < 0 || cols % 32 != 0)
         return -1;
     int64_t nb = cols / 16;
+#ifdef _OPENMP
 #pragma omp parallel for num_threads(g_threads) schedule(static)
+#endif
     for (int64_t r = 0; r < rows; ++r) {
         for (int64_t b = 0; b < nb; ++b) {
             int sb = scales[r * nb + b];
-            float d = f32_mul((float)oracle_elem_value(ORACLE_FMT_E4M3, sb & 127), ts);
+            double d = oracle_elem_value(ORACLE_FMT_E4M3, sb & 127) * (double)ts;
             int extend = plus && sb > 2;
             int bm = (bm_index[(r * nb + b) / 2] >> (4 * (b & 1))) & 15;
             for (int i = 0; i < 16; ++i) {
                 int code = (nibbles[(r * nb + b) * 8 + i / 2] >> (4 * (i & 1))) & 15;
                 double mag = (extend && i == bm) ? 4.0 + 0.5 * (code & 7)
                                                  : oracle_e2m1_value(code & 7);
-                float v = f32_mul((float)mag, d);
+                double v = mag * d;
                 out[r * cols + b * 16 + i] = (code & 8) ? -v : v;
             }
         }

@@ -108,7 +108,9 @@ mxp_status mxp_nvfp4_quantize(const void* src, mxp_dtype src_dt, int64_t rows, i
                               uint8_t* scales, uint8_t* bm_index, void* cuda_stream)
 {
     if (!valid_dtype(src_dt) || rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
-    if (!(tensor_scale > 0.f) || !(tensor_scale < 3.0e38f)) return MXP_ERR_INVALID_ARG;
+    // 2^-100 .. 2^100: keeps value(byte) * ts and its reciprocal normal binary32 numbers
+    if (!(tensor_scale >= 7.8886090522101181e-31f) || !(tensor_scale <= 1.2676506002282294e30f))
+        return MXP_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return MXP_OK;
     if (src == nullptr || nibbles == nullptr || scales == nullptr) return MXP_ERR_INVALID_ARG;
     if (plus && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
@@ -127,7 +129,9 @@ mxp_status mxp_nvfp4_dequantize(const uint8_t* nibbles, const uint8_t* scales,
                                 int64_t ld_dst, void* cuda_stream)
 {
     if (!valid_dtype(dst_dt) || rows < 0 || cols < 0 || cols % 32 != 0) return MXP_ERR_INVALID_ARG;
-    if (!(tensor_scale > 0.f) || !(tensor_scale < 3.0e38f)) return MXP_ERR_INVALID_ARG;
+    // 2^-100 .. 2^100: keeps value(byte) * ts and its reciprocal normal binary32 numbers
+    if (!(tensor_scale >= 7.8886090522101181e-31f) || !(tensor_scale <= 1.2676506002282294e30f))
+        return MXP_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return MXP_OK;
     if (nibbles == nullptr || scales == nullptr || dst == nullptr) return MXP_ERR_INVALID_ARG;
     if (plus && bm_index == nullptr) return MXP_ERR_INVALID_ARG;

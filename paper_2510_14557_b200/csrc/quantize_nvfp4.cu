@@ -7,14 +7,18 @@
 // m = 0..7) and stores a 4-bit BM index per block.  Blocks whose scale byte is 2 or less keep
 // the plain form (index nibble 0).
 //
-// Arithmetic (the passage fixes none; every step is one IEEE binary32 operation, so that the
-// codes are reproducible):  q = amax / (6 ts);  byte = E4M3(q), nearest-even, saturating;
-// d = value(byte) * ts;  r = 1 / d;  scaled = x * r;  code = E2M1(scaled), nearest-even,
-// saturating, sign of the input kept;  BM: m = nearest-even((clamp(amax * r, 4, 8) - 4) * 2),
-// at most 7.  Decode: +-E * d with one rounding.
+// What is computed is the definition in real numbers:  q = amax / (6 ts);  byte = the E4M3
+// value nearest to q (ties to the even byte, saturating at 448);  d = value(byte) * ts;
+// code = the E2M1 value nearest to |x| / d (ties to the even code, saturating at 6, sign of the
+// input kept);  BM: m = nearest integer to (clamp(amax / d, 4, 8) - 4) * 2, ties to even, at
+// most 7.  Decode: +-E * d rounded once to the output type.
+// How: every quotient is first taken in binary32 through a reciprocal, twice -- scaled down and
+// up by 2^-20, which brackets the exact quotient (the binary32 steps err by < 2^-22) -- and
+// both go through the hardware cast.  Where the two casts agree no rounding boundary lies in
+// between and the code is the definition's.  Where they differ, exactly one boundary t lies in
+// between, and the side is decided by comparing |x| with t * d (resp. amax with 6 t ts) in
+// binary64, where those products (at most 33 significant bits) are exact; equality is the tie.
 //
-// HBM-bound: one lane owns 32 consecutive elements (two blocks): 64 or 128 bytes in, 16 bytes
-// of codes, two scale bytes and one index byte out, all as full-width coalesced accesses.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -51,14 +55,27 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float* f)
     return r;
 }
 
+constexpr float kDown = 1.f - 9.5367431640625e-07f;  // 1 - 2^-20
+constexpr float kUp = 1.f + 9.5367431640625e-07f;    // 1 + 2^-20
+
+// Value of an E2M1 magnitude code (0..7) times four: 0 2 4 6 8 12 16 24, five bits each.
+__device__ __forceinline__ uint32_t e2m1_times4(uint32_t c)
+{
+    return (uint32_t)((0xC418831040ull >> (5u * c)) & 31ull);
+}
+
 // One block of 16: two words of codes, the scale byte and the BM index (0 when not extended).
+// `src` points at the block's 16 source elements (read again only for the rare element whose
+// two bracketing casts differ).
 // kKey: the values came from bf16, so their low 16 bits are zero and (magnitude bits | 15 -
 // position) is a key whose unsigned maximum gives the largest magnitude and, among equal
 // ones, the first position in one pass.
-template <bool kPlus, bool kKey>
-__device__ __forceinline__ void nvfp4_block(const float* x, float ts, float six_ts, uint32_t& w0,
-                                            uint32_t& w1, uint32_t& scale_byte, uint32_t& index)
+template <typename T, bool kPlus>
+__device__ __forceinline__ void nvfp4_block(const float* x, const T* __restrict__ src, float ts,
+                                            float six_ts, uint32_t& w0, uint32_t& w1,
+                                            uint32_t& scale_byte, uint32_t& index)
 {
+    constexpr bool kKey = sizeof(T) == 2;
     float amax = 0.f;
     int bm = 0;
     if (kPlus && kKey) {
@@ -77,20 +94,61 @@ __device__ __forceinline__ void nvfp4_block(const float* x, float ts, float six_
                 if (fabsf(x[i]) == amax) bm = i;  // the first of equal maxima
         }
     }
-    const uint32_t sb = f32_to_e4m3_byte(__fdiv_rn(amax, six_ts));
-    const float d = __fmul_rn(e4m3_byte_to_f32(sb), ts);
-    const float r = __frcp_rn(d);
+    // scale byte: E4M3 nearest to amax / (6 ts)
+    const float q = __fdiv_rn(amax, six_ts);
+    uint32_t sb = f32_to_e4m3_byte(__fmul_rn(q, kDown));
+    const uint32_t sb_up = f32_to_e4m3_byte(__fmul_rn(q, kUp));
+    if (sb != sb_up) {  // a boundary between the bytes sb and sb + 1 (never at saturation)
+        const float t = 0.5f * (e4m3_byte_to_f32(sb) + e4m3_byte_to_f32(sb_up));  // exact
+        const double bound = (double)t * 6.0 * (double)ts;                        // exact
+        const double a = (double)amax;
+        if (a > bound || (a == bound && (sb & 1u))) sb = sb_up;
+    }
+    const float e = e4m3_byte_to_f32(sb);
+    const float r = __frcp_rn(__fmul_rn(e, ts));
+    const float r_dn = __fmul_rn(r, kDown), r_up = __fmul_rn(r, kUp);
     // r > 0, so x * r has the sign of x even where it underflows, and the hardware cast keeps
     // the sign of a value that rounds to zero: the codes' sign bits are the inputs'
     float s[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r);
+    for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r_dn);
     w0 = cvt_e2m1x8(s);
     w1 = cvt_e2m1x8(s + 8);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r_up);
+    const uint32_t d0 = w0 ^ cvt_e2m1x8(s), d1 = w1 ^ cvt_e2m1x8(s + 8);
+    if (d0 | d1) {
+        // the upper cast is the next code of the lower one; the boundary between the two is
+        // the mean of their values
+        const double d = (double)e * (double)ts;  // exact
+        uint64_t diff = ((uint64_t)d1 << 32) | d0;
+        uint64_t w = ((uint64_t)w1 << 32) | w0;
+        while (diff) {
+            const int i = (__ffsll((long long)diff) - 1) >> 2;
+            diff &= ~(0xFull << (4 * i));
+            const uint32_t c = (uint32_t)(w >> (4 * i)) & 7u;  // lower code, c < 7
+            const double bound = (double)(e2m1_times4(c) + e2m1_times4(c + 1u)) * 0.125 * d;
+            double a;
+            if (kKey) a = (double)__bfloat162float(reinterpret_cast<const __nv_bfloat16*>(src)[i]);
+            else a = (double)reinterpret_cast<const float*>(src)[i];
+            a = fabs(a);
+            if (a > bound || (a == bound && (c & 1u))) w += 1ull << (4 * i);
+        }
+        w0 = (uint32_t)w;
+        w1 = (uint32_t)(w >> 32);
+    }
     index = 0;
     if (kPlus && sb > 2u) {
-        const float v = fminf(fmaxf(__fmul_rn(amax, r), 4.f), 8.f);
-        const uint32_t m = (uint32_t)min(__float2int_rn((v - 4.f) * 2.f), 7);
+        const float v_dn = fminf(fmaxf(__fmul_rn(amax, r_dn), 4.f), 8.f);
+        const float v_up = fminf(fmaxf(__fmul_rn(amax, r_up), 4.f), 8.f);
+        uint32_t m = (uint32_t)__float2int_rn((v_dn - 4.f) * 2.f);  // 0..8
+        const uint32_t m_up = (uint32_t)__float2int_rn((v_up - 4.f) * 2.f);
+        if (m != m_up) {  // boundary 4.25 + m / 2 between m and m + 1
+            const double bound = (double)(17u + 2u * m) * 0.25 * ((double)e * (double)ts);
+            const double a = (double)amax;
+            if (a > bound || (a == bound && (m & 1u))) m = m_up;
+        }
+        m = min(m, 7u);
         const uint32_t sh = (uint32_t)(bm & 7) * 4u;
         if (bm < 8) w0 = (w0 & ~(7u << sh)) | (m << sh);  // the sign bit stays
         else w1 = (w1 & ~(7u << sh)) | (m << sh);
@@ -134,8 +192,8 @@ nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_p
     }
     const float six_ts = __fmul_rn(6.f, ts);
     uint32_t w[4], sb0, sb1, i0, i1;
-    nvfp4_block<kPlus, sizeof(T) == 2>(x, ts, six_ts, w[0], w[1], sb0, i0);
-    nvfp4_block<kPlus, sizeof(T) == 2>(x + 16, ts, six_ts, w[2], w[3], sb1, i1);
+    nvfp4_block<T, kPlus>(x, p, ts, six_ts, w[0], w[1], sb0, i0);
+    nvfp4_block<T, kPlus>(x + 16, p + 16, ts, six_ts, w[2], w[3], sb1, i1);
     __stcs(nibbles + u, make_uint4(w[0], w[1], w[2], w[3]));
     scales[u] = (uint16_t)(sb0 | (sb1 << 8));
     if (kPlus) bm_index[u] = (uint8_t)(i0 | (i1 << 4));
@@ -153,19 +211,30 @@ nvfp4_dequantize_kernel(const uint32_t* __restrict__ nibbles, const uint8_t* __r
     const int64_t blk = u >> 1;
     const uint32_t word = __ldg(nibbles + u);
     const uint32_t sb = scales[blk];
-    const float d = __fmul_rn(e4m3_byte_to_f32(sb & 127u), ts);
+    const float e = e4m3_byte_to_f32(sb & 127u);
     int bm = -1;
     if (kPlus && sb > 2u) {
         bm = (int)((bm_index[blk >> 1] >> (4 * (blk & 1))) & 15u) - 8 * (int)(u & 1);  // within this word
     }
+    // E * value(byte) is exact in binary32 (at most 8 significant bits), so one multiply by ts
+    // rounds the exact product once.  For a bf16 destination that multiply rounds to odd
+    // (truncate, then set the last bit if anything was cut off), which makes the second
+    // rounding, to bf16, the single correct one.
     float out[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const uint32_t c = (word >> (4 * i)) & 15u;
-        const uint32_t e = (c >> 1) & 3u, m = c & 1u;
-        float mag = e == 0u ? 0.5f * (float)m : __uint_as_float(((126u + e) << 23) | (m << 22));
+        const uint32_t ex = (c >> 1) & 3u, m = c & 1u;
+        float mag = ex == 0u ? 0.5f * (float)m : __uint_as_float(((126u + ex) << 23) | (m << 22));
         if (kPlus && i == bm) mag = 4.f + 0.5f * (float)(c & 7u);
-        const float v = __fmul_rn(mag, d);
+        const float me = __fmul_rn(mag, e);
+        float v;
+        if (sizeof(T) == 4) {
+            v = __fmul_rn(me, ts);
+        } else {
+            v = __fmul_rz(me, ts);
+            if (__fmaf_rn(me, ts, -v) != 0.f) v = __uint_as_float(__float_as_uint(v) | 1u);
+        }
         out[i] = (c & 8u) ? -v : v;
     }
     const int64_t e0 = u * 8, row = e0 / cols;

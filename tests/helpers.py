@@ -50,3 +50,46 @@ def check_gemm(d_gpu: torch.Tensor, da: np.ndarray, db: np.ndarray, ref: np.ndar
     assert not bad.any(), "max err/tol = %g at %s" % (
         np.max(err / (tol + 1e-300)), np.unravel_index(np.argmax(err / (tol + 1e-300)), err.shape))
     return float(np.max(err / (tol + 1e-300)))
+
+
+def f64_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bfloat16 bit patterns, ONE rounding (ties to even), subnormals kept."""
+    x = np.asarray(x, np.float64)
+    mag = np.abs(x)
+    _, ex = np.frexp(mag)                                  # mag = f * 2^ex, f in [0.5, 1)
+    q = np.maximum(ex - 8, -133).astype(np.int64)          # quantum: 8 significant bits; 2^-133 below 2^-126
+    r = np.ldexp(np.rint(np.ldexp(mag, -q)), q)            # rint: ties to even; both ldexp exact
+    bits = r.astype(np.float32).view(np.uint32) >> 16      # exact: r is a bfloat16 value
+    return (bits | (np.signbit(x).astype(np.uint32) << 15)).astype(np.uint16)
+
+
+def nvfp4_boundary_blocks(ts, seed):
+    """Blocks of 16 whose elements sit exactly on, one binary32 step above and one step below
+    a rounding boundary of the element cast, the BM cast or the scale cast, for scales of every
+    mantissa -- the inputs on which a reciprocal-and-multiply recipe and the definition part."""
+    g = synth.rng(seed)
+    ts32 = np.float32(ts)
+    rows = []
+    for _ in range(160):
+        sb = int(g.integers(3, 0x7E))
+        d = np.float64(oracle.elem_value(oracle.FMT_E4M3, sb)) * np.float64(ts32)
+        blk = np.empty(16, np.float64)
+        blk[0] = d * g.choice([5.5, 5.75, 6.0, 6.25, 5.25, 6.75, 5.9])          # the BM
+        ties = g.choice([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], 15)
+        blk[1:] = ties * d * g.choice([-1.0, 1.0], 15)
+        b32 = blk.astype(np.float32)
+        step = g.integers(-1, 2, 16).astype(np.int32)                          # -1, 0, +1 ulp
+        b32 = (b32.view(np.int32) + step).view(np.float32)
+        rows.append(np.roll(b32, int(g.integers(0, 16))))
+    # scale-cast boundaries: amax = 6 ts * (midpoint of two neighbouring oracle.FMT_E4M3 values) +- 1 ulp
+    for sb in list(range(0, 0x7D, 3)):
+        mid = 0.5 * (oracle.elem_value(oracle.FMT_E4M3, sb) + oracle.elem_value(oracle.FMT_E4M3, sb + 1))
+        for step in (-1, 0, 1):
+            a = np.float32(np.float64(6.0) * mid * np.float64(ts32))
+            a = (a.view(np.int32) + np.int32(step)).view(np.float32)
+            blk = np.full(16, a * np.float32(0.3), np.float32)
+            blk[int(g.integers(0, 16))] = -a
+            rows.append(blk)
+    x = np.stack(rows)
+    x = np.concatenate([x, np.zeros(((-x.shape[0]) % 2, 16), np.float32)])
+    return x.reshape(-1, 32)

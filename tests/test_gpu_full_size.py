@@ -1,6 +1,6 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration bench.py times,
-on sampled outputs the oracle computes one by one (configs 2, 4 and 5; config 3 is covered in
-test_gpu_gemm.py)."""
+whole-matrix encodings bit for bit and sampled GEMM outputs the oracle computes one by one
+(configs 2, 4 and 5; config 3 is covered in test_gpu_gemm.py)."""
 import numpy as np
 import pytest
 import torch
@@ -22,22 +22,34 @@ def sample(n, step, extra):
     return np.unique(np.concatenate([np.arange(0, n, step), np.asarray(extra)]))
 
 
+def planes_equal(p, ref, with_index):
+    """Whole planes, bit for bit (compared on the host in one piece)."""
+    assert np.array_equal(p.nibbles.cpu().numpy(), ref[0]), "codes differ"
+    assert np.array_equal(p.scales.cpu().numpy(), ref[1]), "scales differ"
+    if with_index:
+        assert np.array_equal(p.bm_index.cpu().numpy(), ref[2]), "BM indices differ"
+
+
+@pytest.fixture
+def oracle_all_cores():
+    oracle.set_threads(oracle.max_threads())
+    yield
+    oracle.set_threads(1)
+
+
 @pytest.mark.parametrize("mode", [MX, MXP, MXPP])
-def test_quantize_config2_sampled_rows_bit_exact(mode):
-    # 8192 x 8192 bf16 through the one-lane-per-block kernel; every plane of the sampled rows
+def test_quantize_config2_whole_matrix_bit_exact(mode, oracle_all_cores):
+    # 8192 x 8192 bf16 through the one-lane-per-block kernel: every byte of every plane, and
+    # the decode of the whole matrix (exact in fp32), 1024 rows at a time
     bits = synth.config2()
     p = mxp().mxp_quantize(to_dev_bf16(bits), mode)
-    rows = sample(8192, 331, [8191, 8190, 4095, 4096])
-    ref = oracle.quantize(bits[rows], mode, bf16_bits=True)
-    sel = torch.from_numpy(rows).cuda()
-    assert np.array_equal(p.nibbles[sel].cpu().numpy(), ref[0])
-    assert np.array_equal(p.scales[sel].cpu().numpy(), ref[1])
-    if mode != MX:
-        assert np.array_equal(p.bm_index[sel].cpu().numpy(), ref[2])
-    # decode of the full matrix, sampled rows, exact
+    ref = oracle.quantize(bits, mode, bf16_bits=True)
+    planes_equal(p, ref, mode != MX)
     d = mxp().mxp_dequantize(p, torch.float32)
-    want = oracle.dequantize(ref[0], ref[1], ref[2], mode)
-    assert np.array_equal(d[sel].cpu().numpy().astype(np.float64), want)
+    for r0 in range(0, 8192, 1024):
+        r1 = r0 + 1024
+        want = oracle.dequantize(ref[0][r0:r1], ref[1][r0:r1], ref[2][r0:r1], mode)
+        assert np.array_equal(d[r0:r1].cpu().numpy().astype(np.float64), want)
 
 
 def _bench_step_parity(a_bits, w_bits, row_step, col_step):
@@ -57,17 +69,19 @@ def _bench_step_parity(a_bits, w_bits, row_step, col_step):
     d = m.mxp_gemm_ready(pa, pw, pre, ws, out_dtype=torch.bfloat16)
     torch.cuda.synchronize()
     assert m.mxp_gemm_status(ws) == 0
+    # the encodings the GEMM consumed are the oracle's, bit for bit, over the whole of A and W
+    oracle.set_threads(oracle.max_threads())
+    try:
+        planes_equal(pa, oracle.quantize(a_bits, MXP, bf16_bits=True), True)
+        planes_equal(pw, oracle.quantize(w_bits, MXP, bf16_bits=True), True)
+    finally:
+        oracle.set_threads(1)
+    # the output on sampled rows and columns (the fp64 product is O(M N K))
     rows = sample(M, row_step, [M - 1, M - 2, 255, 256, 257])
     cols = sample(N, col_step, [N - 1, N - 2, 239, 240, 479, 480, 481])
     qa = oracle.quantize(a_bits[rows], MXP, bf16_bits=True)
     qw = oracle.quantize(w_bits[cols], MXP, bf16_bits=True)
-    # the encodings the GEMM consumed are the oracle's, bit for bit
     rsel, csel = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
-    assert np.array_equal(pa.nibbles[rsel].cpu().numpy(), qa[0])
-    assert np.array_equal(pa.scales[rsel].cpu().numpy(), qa[1])
-    assert np.array_equal(pa.bm_index[rsel].cpu().numpy(), qa[2])
-    assert np.array_equal(pw.nibbles[csel].cpu().numpy(), qw[0])
-    assert np.array_equal(pw.bm_index[csel].cpu().numpy(), qw[2])
     da = oracle.dequantize(qa[0], qa[1], qa[2], MXP)
     dw = oracle.dequantize(qw[0], qw[1], qw[2], MXP)
     check_gemm(d[rsel][:, csel], da, dw)

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import to_dev, to_dev_bf16
+from helpers import f64_to_bf16_bits, nvfp4_boundary_blocks, to_dev, to_dev_bf16
 from paper_2510_14557_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -101,31 +101,57 @@ def test_decode_bit_exact(plus, dtype):
     nib, sc, idx = oracle.nvfp4_quantize(x, ts, plus)
     want = oracle.nvfp4_dequantize(nib, sc, idx, ts, plus)
     got = mxp().mxp_nvfp4_dequantize(to_dev(nib), to_dev(sc), to_dev(idx) if plus else None, ts, plus, dtype)
+    # the oracle's decode is exact (float64); the library rounds it once to the output type
     if dtype == torch.float32:
-        assert np.array_equal(got.cpu().numpy().view(np.uint32), want.view(np.uint32))
+        assert np.array_equal(got.cpu().numpy().view(np.uint32), want.astype(np.float32).view(np.uint32))
     else:
-        wb = torch.from_numpy(want).to(torch.bfloat16)       # round to nearest even
-        assert torch.equal(got.cpu().view(torch.int16), wb.view(torch.int16))
+        assert np.array_equal(got.cpu().view(torch.int16).numpy().view(np.uint16), f64_to_bf16_bits(want))
     # every possible (code, scale byte) pair, BM in every position
     codes = np.arange(256, dtype=np.uint8).reshape(1, 256).repeat(128, axis=0)     # all byte values
     scb = (np.arange(128) % 127).astype(np.uint8).reshape(128, 1).repeat(32, axis=1)   # 0x7F is the NaN pattern
     rng_idx = g.integers(0, 256, (128, 16)).astype(np.uint8)
-    want = oracle.nvfp4_dequantize(codes, scb, rng_idx, 0.5, plus)
-    got = mxp().mxp_nvfp4_dequantize(to_dev(codes), to_dev(scb), to_dev(rng_idx) if plus else None, 0.5, plus)
-    assert np.array_equal(got.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    # a tensor scale with 24 significant bits: products need the single rounding
+    for ts in (0.5, 0.7330000996589661, 1.0 / 3.0):
+        want = oracle.nvfp4_dequantize(codes, scb, rng_idx, ts, plus)
+        got = mxp().mxp_nvfp4_dequantize(to_dev(codes), to_dev(scb), to_dev(rng_idx) if plus else None, ts, plus, dtype)
+        if dtype == torch.float32:
+            assert np.array_equal(got.cpu().numpy().view(np.uint32), want.astype(np.float32).view(np.uint32))
+        else:
+            assert np.array_equal(got.cpu().view(torch.int16).numpy().view(np.uint16), f64_to_bf16_bits(want))
 
 
-def test_config2_sampled_rows_and_argument_checks():
+@pytest.mark.parametrize("plus", [False, True])
+def test_rounding_boundaries_bit_exact(plus):
+    # elements, BMs and block maxima exactly on, one binary32 step above and one step below a
+    # rounding boundary of the element, BM and scale casts: the codes must be those of exact
+    # arithmetic, whatever a reciprocal in binary32 would make of them
+    for ts, seed in ((1.0, 1), (0.37, 2), (2.0 ** -8, 3), (1.0 / 3.0, 4), (0.6458333134651184, 5)):
+        x = nvfp4_boundary_blocks(ts, seed)
+        ref = oracle.nvfp4_quantize(x, ts, plus)
+        got = mxp().mxp_nvfp4_quantize(to_dev(x), ts, plus)
+        check_planes(got, ref, plus)
+    # bf16 sources: boundaries t * d that bf16 holds (power-of-two tensor scale)
+    x = nvfp4_boundary_blocks(2.0 ** -3, 9)
+    bits = synth.f32_to_bf16_bits(x)
+    ref = oracle.nvfp4_quantize(bits, 2.0 ** -3, plus, bf16_bits=True)
+    got = mxp().mxp_nvfp4_quantize(to_dev_bf16(bits), 2.0 ** -3, plus)
+    check_planes(got, ref, plus)
+
+
+def test_config2_whole_matrix_and_argument_checks():
     m = mxp()
     bits = synth.config2()
-    ts = 2.0 ** -8
-    got = m.mxp_nvfp4_quantize(to_dev_bf16(bits), ts, True)
-    rows = np.unique(np.concatenate([np.arange(0, 8192, 257), [8191, 4095]]))
-    ref = oracle.nvfp4_quantize(bits[rows], ts, True, bf16_bits=True)
-    sel = torch.from_numpy(rows).cuda()
-    check_planes((got[0][sel], got[1][sel], got[2][sel]), ref, True)
+    oracle.set_threads(oracle.max_threads())
+    try:
+        # a power-of-two tensor scale (exact ties are frequent) and the usual amax / (6 * 448)
+        for ts in (2.0 ** -8, float(np.float32(np.abs(oracle.bf16_bits_to_f64(bits)).max() / (6 * 448)))):
+            got = m.mxp_nvfp4_quantize(to_dev_bf16(bits), ts, True)
+            ref = oracle.nvfp4_quantize(bits, ts, True, bf16_bits=True)
+            check_planes(got, ref, True)
+    finally:
+        oracle.set_threads(1)
     x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
-    for bad in (0.0, -1.0, float("inf"), float("nan")):
+    for bad in (0.0, -1.0, float("inf"), float("nan"), 2.0 ** -101, 2.0 ** 101):
         with pytest.raises(m.MxpError) as e:
             m.mxp_nvfp4_quantize(x, bad, True)
         assert e.value.status == 1
