@@ -266,18 +266,11 @@ def part_decode(mxp, synth, peaks, iters):
         for _ in range(8):
             copies.append(mxp.mxp_quantize(w, mode))
         wbytes = 11008 * 4096 * (0.5 + 1 / 32 + (1 / 32 if mode != mxp.MODE_MXFP4 else 0))
-        # (M, kernel): the default kernel choice, and at M = 1 the opt-in FP4-tensor-path kernel
         cases = [(1, None), (8, None), (16, None)] if mode != mxp.MODE_MXFP4_PP else [(1, None)]
-        if mode != mxp.MODE_MXFP4_PP:
-            cases.append((1, "fp4"))
         for M, kern in cases:
             a = dev_bf16(a16[:M].copy())
             d = torch.empty((M, 11008), dtype=torch.bfloat16, device="cuda")
             state = {"i": 0}
-            if kern is None:
-                os.environ.pop("MXP_WO_KERNEL", None)
-            else:
-                os.environ["MXP_WO_KERNEL"] = kern   # read by the library on every call
             key = "decode_cfg3_M%d_%s" % (M, name) + ("" if kern is None else "_kernel-" + kern)
 
             def run():
@@ -322,7 +315,6 @@ def part_decode(mxp, synth, peaks, iters):
                 ms_c = time_loop(graph.replay, max(1, iters // 8), warmup=2) / 8
                 out[key]["us_cuda_graph_chained"] = ms_c * 1e3
                 out[key]["frac_hbm_cuda_graph_chained"] = (wbytes + M * 4096 * 2 + M * 11008 * 2) / ms_c / 1e6 / hbm
-        os.environ.pop("MXP_WO_KERNEL", None)
         del copies, w
     # ---- weight-only form at prefill sizes (the paper's matmul table: N = K = 4096, M up to
     # 4096): bf16 activations on the block-scaled tensor-core kernel as two E4M3 planes; the

@@ -317,6 +317,49 @@ mxp_status mxp_gemm_decode_chained(int64_t M, int64_t N, int64_t K, const void *
                                    void *cuda_stream);
 
 /*
+ * The weight-only form for decode shapes (1 <= M <= 16) with the weights re-tiled once (Sec. 7.1:
+ * the memory-bound token-generation phase; Eq. 3 decode, BM split per Eq. 4).  The GEMM streams
+ * every weight byte exactly once, straight into the FP4 tensor cores:
+ *   mxp_gemm_decode_prepack_bytes  bytes of the re-tiled form of an N x K weight operand in
+ *                            mode MXFP4 or MXFP4+ on the CURRENT device (the tiling depends on
+ *                            its SM count); 0: not supported (K % 256 != 0, other modes).
+ *   mxp_gemm_decode_prepack  writes that form into `out` (device, 256-byte aligned, out_bytes >=
+ *                            the size above).  A re-ordering of the stored 4-bit codes, scales
+ *                            and BM indices; for MXFP4+ the BM's code is replaced by its upper
+ *                            part BM_H (an E2M1 value) and the lower part BM_L is kept in a
+ *                            record byte per block.  Blocks with scale byte 0 become zeros.
+ *   mxp_gemm_decode_workspace_bytes  device scratch one call needs (0: M or K not supported):
+ *                            a status block and the activations' operand images.
+ *   mxp_gemm_decode_prepacked  D[M,N] = A(bf16)[M,K] * dec(B)[N,K]^T.  `b_mode`, N, K must be
+ *                            those B_prepacked was made with, and B_prepacked_bytes the size
+ *                            mxp_gemm_decode_prepack_bytes gives for them (checked before any
+ *                            launch: MXP_ERR_INVALID_ARG).  Two launches: a small kernel turns
+ *                            the activations into five FP4 digit planes per row (balanced base
+ *                            8, a block scale per plane: an element within 2^5 of the largest
+ *                            magnitude of its block of 32 is exact, a smaller one is rounded at
+ *                            2^-13 of that magnitude's binade -- far inside the GEMM's error
+ *                            bound, which is relative to the row norm); the GEMM is launched as
+ *                            its programmatic dependent and starts streaming weights at once.
+ *                            chained != 0: the first kernel is itself launched as a
+ *                            programmatic dependent of whatever precedes it on the stream, with
+ *                            the promise and the status-block rule of mxp_gemm_decode_chained
+ *                            (B_prepacked not written by the preceding kernel; status block
+ *                            not cleared).  M > 16 or unsupported shapes: MXP_ERR_UNSUPPORTED
+ *                            (use mxp_gemm).  Same result as mxp_gemm within its bound; one-hot
+ *                            activation rows return decoded weights bit for bit.
+ * The paper describes the format and its decode, not this staging.
+ */
+size_t mxp_gemm_decode_prepack_bytes(int64_t N, int64_t K, mxp_mode b_mode);
+size_t mxp_gemm_decode_workspace_bytes(int64_t M, int64_t K);
+mxp_status mxp_gemm_decode_prepack(const mxp_packed *B_packed, void *out, size_t out_bytes,
+                                   void *cuda_stream);
+mxp_status mxp_gemm_decode_prepacked(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16,
+                                     int64_t lda, mxp_mode b_mode, const void *B_prepacked,
+                                     size_t B_prepacked_bytes, void *D, mxp_dtype d_dt,
+                                     int64_t ldd, void *workspace, size_t workspace_bytes,
+                                     int chained, void *cuda_stream);
+
+/*
  * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM
  * left in `workspace`: MXP_OK, or MXP_ERR_TIMEOUT if a bounded wait inside a kernel gave
  * up (the output is then undefined but the context stays usable).
@@ -389,6 +432,28 @@ mxp_status mxp_tensor_peak_probe(int kind, int iters, double *ms, double *flops)
 mxp_status mxp_gemm_noalloc(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
                             const mxp_packed *B_packed, void *D, mxp_dtype d_dt, int64_t ldd,
                             mxp_status *kernel_status, void *cuda_stream);
+
+/*
+ * Test and measurement aid (no counterpart in the paper): forces a kernel choice that the
+ * dispatch of mxp_gemm would otherwise make by shape, so that every kernel can be reached with
+ * any operands.  Process-wide and not synchronised with calls in flight; value 0 gives the
+ * choice back to the library.  Not meant for production use.
+ *   MXP_KNOB_INPLACE_KERNEL      packed x packed mxp_gemm: 1 = the in-place single-CTA kernel,
+ *                                2 = the in-place CTA-pair kernel (either also keeps the call
+ *                                away from the streamed kernel on prepacked operands)
+ *   MXP_KNOB_STREAM_HALVES       streamed kernel: 1 / 2 = output tile of one / two halves
+ *   MXP_KNOB_WEIGHT_ONLY_KERNEL  weight-only mxp_gemm: 1 = the general kernel, 2 = the streamed
+ *                                decode kernel where it applies (either keeps M > 64 calls
+ *                                away from the tensor-core path)
+ * Returns MXP_ERR_INVALID_ARG for an unknown knob or a value outside 0..2.
+ */
+typedef enum {
+    MXP_KNOB_INPLACE_KERNEL = 0,
+    MXP_KNOB_STREAM_HALVES = 1,
+    MXP_KNOB_WEIGHT_ONLY_KERNEL = 2,
+    MXP_KNOB_COUNT_ = 3
+} mxp_knob;
+mxp_status mxp_debug_override(int knob, int value);
 
 const char *mxp_status_string(mxp_status s);
 

@@ -25,11 +25,11 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_decode_prepack_bytes", "mxp_gemm_decode_workspace_bytes", "mxp_gemm_decode_prepack", "mxp_gemm_decode_prepacked", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_gemm_dense_prepacked", "mxp_gemm_dense_prepacked_workspace_bytes",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
-           "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
+           "mxp_debug_override", "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
 
 
 class MxpError(RuntimeError):
@@ -81,6 +81,14 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_decode_chained.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, ci,
                                               i64, vp, vp]
         l.mxp_gemm_decode_chained.restype = ci
+        l.mxp_gemm_decode_prepack_bytes.argtypes = [i64, i64, ci]
+        l.mxp_gemm_decode_prepack_bytes.restype = sz
+        l.mxp_gemm_decode_workspace_bytes.argtypes = [i64, i64]
+        l.mxp_gemm_decode_workspace_bytes.restype = sz
+        l.mxp_gemm_decode_prepack.argtypes = [ctypes.POINTER(_Packed), vp, sz, vp]
+        l.mxp_gemm_decode_prepack.restype = ci
+        l.mxp_gemm_decode_prepacked.argtypes = [i64, i64, i64, vp, i64, ci, vp, sz, vp, ci, i64, vp, sz, ci, vp]
+        l.mxp_gemm_decode_prepacked.restype = ci
         l.mxp_gemm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
         l.mxp_gemm_workspace_bytes.restype = sz
         l.mxp_gemm_min_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
@@ -96,6 +104,8 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_ready.restype = ci
         l.mxp_quantize_gemm_ready.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, vp, sz, vp]
         l.mxp_quantize_gemm_ready.restype = ci
+        l.mxp_debug_override.argtypes = [ci, ci]
+        l.mxp_debug_override.restype = ci
         l.mxp_wait_selftest.argtypes = [vp, sz, i64, vp]
         l.mxp_wait_selftest.restype = ci
         l.mxp_gemm_status.argtypes = [vp, vp]
@@ -371,6 +381,47 @@ def mxp_gemm_decode_chained(a: torch.Tensor, b: Packed, out: torch.Tensor,
     return out
 
 
+class DecodeWeights:
+    """Weights re-tiled once for mxp_gemm_decode_prepacked: the device buffer plus the shape and
+    mode it was made from (what the C call wants to see again)."""
+
+    def __init__(self, buf: torch.Tensor, rows: int, cols: int, mode: int):
+        self.buf, self.rows, self.cols, self.mode = buf, rows, cols, mode
+
+
+def mxp_gemm_decode_prepack(b: Packed) -> DecodeWeights:
+    """Re-tiles MXFP4 / MXFP4+ weights for the decode GEMM (once per weight matrix and device)."""
+    need = int(lib().mxp_gemm_decode_prepack_bytes(b.rows, b.cols, b.mode))
+    if need == 0:
+        raise MxpError("mxp_gemm_decode_prepack_bytes", 2)
+    out = torch.empty(need, dtype=torch.uint8, device=b.nibbles.device)
+    bs = b.c_struct()
+    _check("mxp_gemm_decode_prepack", lib().mxp_gemm_decode_prepack(ctypes.byref(bs), out.data_ptr(), out.numel(), _stream()))
+    return DecodeWeights(out, b.rows, b.cols, b.mode)
+
+
+def mxp_gemm_decode_workspace_bytes(M: int, K: int) -> int:
+    return int(lib().mxp_gemm_decode_workspace_bytes(M, K))
+
+
+def mxp_gemm_decode_prepacked(a: torch.Tensor, w: DecodeWeights, out_dtype=torch.bfloat16,
+                              out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                              chained: bool = False) -> torch.Tensor:
+    """D = a @ dec(W).T for 1..16 activation rows on the FP4 tensor path, weights re-tiled by
+    mxp_gemm_decode_prepack.  `chained`: see include/mxp.h."""
+    assert a.dtype == torch.bfloat16 and a.is_cuda and a.stride(1) == 1
+    M, N, K = a.shape[0], w.rows, w.cols
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=a.device)
+    if workspace is None:
+        workspace = torch.zeros(max(256, mxp_gemm_decode_workspace_bytes(M, K)), dtype=torch.uint8, device=a.device)
+    st = lib().mxp_gemm_decode_prepacked(M, N, K, a.data_ptr(), a.stride(0), w.mode, w.buf.data_ptr(),
+                                         w.buf.numel(), out.data_ptr(), _dt(out), out.stride(0),
+                                         workspace.data_ptr(), workspace.numel(), int(chained), _stream())
+    _check("mxp_gemm_decode_prepacked", st)
+    return out
+
+
 def mxp_gemm_dense_prepacked(a: torch.Tensor, b: Packed, b_prepacked: torch.Tensor,
                              out_dtype=torch.bfloat16, out: Optional[torch.Tensor] = None,
                              workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
@@ -390,6 +441,14 @@ def mxp_gemm_dense_prepacked(a: torch.Tensor, b: Packed, b_prepacked: torch.Tens
                                         _stream())
     _check("mxp_gemm_dense_prepacked", st)
     return out
+
+
+KNOB_INPLACE_KERNEL, KNOB_STREAM_HALVES, KNOB_WEIGHT_ONLY_KERNEL = 0, 1, 2
+
+
+def mxp_debug_override(knob: int, value: int) -> None:
+    """Forces a kernel choice (tests and measurements; see include/mxp.h).  0 = automatic."""
+    _check("mxp_debug_override", lib().mxp_debug_override(knob, value))
 
 
 def mxp_wait_selftest(workspace: torch.Tensor, limit_cycles: int) -> None:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmxp.so")
-SOURCES = ["api.cu", "quantize.cu", "quantize_wide.cu", "quantize_nvfp4.cu", "gemm_weight_only.cu", "gemm_wo_stream.cu", "gemm_wo_tma.cu", "gemm_wo_fp4.cu", "gemm_tc.cu", "gemm_tc_stream.cu", "gemm_noalloc.cu", "selftest.cu"]
+SOURCES = ["api.cu", "quantize.cu", "quantize_wide.cu", "quantize_nvfp4.cu", "gemm_weight_only.cu", "gemm_wo_stream.cu", "gemm_decode_tc.cu", "gemm_tc.cu", "gemm_tc_stream.cu", "gemm_noalloc.cu", "selftest.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC",

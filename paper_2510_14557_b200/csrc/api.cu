@@ -4,7 +4,16 @@
 #include <cstring>
 #include <vector>
 
+#include <atomic>
+
 #include "common.cuh"
+
+namespace mxp {
+namespace {
+std::atomic<int> g_override[MXP_KNOB_COUNT_];
+}
+int override_get(int knob) { return knob >= 0 && knob < MXP_KNOB_COUNT_ ? g_override[knob].load(std::memory_order_relaxed) : 0; }
+}  // namespace mxp
 
 namespace {
 
@@ -57,7 +66,14 @@ const char* mxp_status_string(mxp_status s)
     return "unknown status";
 }
 
-const char* mxp_version(void) { return "mxp 0.1 sm_100a"; }
+const char* mxp_version(void) { return "mxp 0.2 sm_100a"; }
+
+mxp_status mxp_debug_override(int knob, int value)
+{
+    if (knob < 0 || knob >= MXP_KNOB_COUNT_ || value < 0 || value > 2) return MXP_ERR_INVALID_ARG;
+    mxp::g_override[knob].store(value, std::memory_order_relaxed);
+    return MXP_OK;
+}
 
 mxp_status mxp_quantize(const void* src, mxp_dtype src_dt, int64_t rows, int64_t cols,
                         int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
@@ -250,7 +266,7 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (A_dense_bf16 != nullptr) {
         if (M > 64 && N >= 128 && workspace != nullptr && aligned(workspace, 256) &&
-            aligned(B_packed->scales, 4) && getenv("MXP_WO_KERNEL") == nullptr &&
+            aligned(B_packed->scales, 4) && mxp::override_get(MXP_KNOB_WEIGHT_ONLY_KERNEL) == 0 &&
             (B_packed->mode != MXP_MODE_MXFP4_PP || aligned(B_packed->bm_index, 4))) {
             const size_t fast = mxp::stream_dense_workspace_bytes(M, N, K, B_packed->mode);
             if (fast != 0 && workspace_bytes >= fast) {
@@ -291,6 +307,44 @@ mxp_status mxp_gemm_decode_chained(int64_t M, int64_t N, int64_t K, const void* 
                                                      static_cast<cudaStream_t>(cuda_stream), true);
     if (e == cudaErrorNotSupported) return MXP_ERR_UNSUPPORTED;
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+size_t mxp_gemm_decode_prepack_bytes(int64_t N, int64_t K, mxp_mode b_mode)
+{
+    return mxp::decode_prepack_bytes(N, K, b_mode);
+}
+
+size_t mxp_gemm_decode_workspace_bytes(int64_t M, int64_t K)
+{
+    return mxp::decode_workspace_bytes(M, K);
+}
+
+mxp_status mxp_gemm_decode_prepack(const mxp_packed* B_packed, void* out, size_t out_bytes,
+                                   void* cuda_stream)
+{
+    if (!valid_packed(B_packed, false)) return MXP_ERR_INVALID_ARG;
+    if (B_packed->rows == 0 || B_packed->cols == 0) return MXP_ERR_UNSUPPORTED;
+    if (B_packed->mode != MXP_MODE_MXFP4 && B_packed->mode != MXP_MODE_MXFP4_PLUS)
+        return MXP_ERR_UNSUPPORTED;
+    return mxp::decode_prepack(*B_packed, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+mxp_status mxp_gemm_decode_prepacked(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16,
+                                     int64_t lda, mxp_mode b_mode, const void* B_prepacked,
+                                     size_t B_prepacked_bytes, void* D, mxp_dtype d_dt, int64_t ldd,
+                                     void* workspace, size_t workspace_bytes, int chained,
+                                     void* cuda_stream)
+{
+    if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
+    if (!valid_dtype(d_dt) || !valid_mode(b_mode)) return MXP_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return MXP_OK;
+    if (A_dense_bf16 == nullptr || B_prepacked == nullptr || D == nullptr) return MXP_ERR_INVALID_ARG;
+    if (lda < K || lda % 8 != 0 || !aligned(A_dense_bf16, 16) || ldd < N) return MXP_ERR_INVALID_ARG;
+    if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4) || !aligned(B_prepacked, 256)) return MXP_ERR_INVALID_ARG;
+    if (workspace != nullptr && !aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;
+    return mxp::launch_gemm_decode_tc(M, N, K, A_dense_bf16, lda, b_mode, B_prepacked,
+                                      B_prepacked_bytes, D, d_dt, ldd, workspace, workspace_bytes,
+                                      chained != 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide)

@@ -53,21 +53,14 @@ cudaError_t launch_quantize_wide(const void* src, mxp_dtype dt, int64_t rows, in
 cudaError_t launch_dequantize_wide(const mxp_packed& p, void* dst, mxp_dtype dt, int64_t ld_dst,
                                    cudaStream_t stream);
 
-// Tensor-core variant for decode shapes whose weights no thread touches (TMA unpacks the 4-bit
-// codes into the layout kind::mxf8f6f4 reads; MXFP4 and MXFP4+ weights, K % 512 == 0, M <= 64).
-bool wo_tma_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                      const mxp_packed& B);
-cudaError_t launch_gemm_wo_tma(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                               const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                               void* status, cudaStream_t stream);
-
-// Tensor-core variant on the FP4 path (kind::mxf4 on the nibble plane as stored; activations as
-// base-4 digit planes; MXFP4 and MXFP4+ weights, K % 512 == 0, M <= 4).
-bool wo_fp4_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                      const mxp_packed& B);
-cudaError_t launch_gemm_wo_fp4(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
-                               const mxp_packed& B, void* D, mxp_dtype d_dt, int64_t ldd,
-                               void* status, cudaStream_t stream);
+// Decode shapes (M <= 16) on the FP4 tensor path with weights re-tiled once (gemm_decode_tc.cu).
+size_t decode_prepack_bytes(int64_t N, int64_t K, mxp_mode mode);  // 0: not supported
+size_t decode_workspace_bytes(int64_t M, int64_t K);               // 0: not supported
+mxp_status decode_prepack(const mxp_packed& B, void* out, size_t out_bytes, cudaStream_t stream);
+mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                 mxp_mode b_mode, const void* b_prepacked, size_t b_prepacked_bytes,
+                                 void* D, mxp_dtype d_dt, int64_t ldd, void* workspace,
+                                 size_t workspace_bytes, bool chained, cudaStream_t stream);
 
 // Block-scaled tensor-core form: both operands packed.
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);
@@ -101,6 +94,10 @@ cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, m
 size_t stream_prepack_bytes(int64_t rows, int64_t K, bool wide);
 mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_bytes,
                           cudaStream_t stream);
+
+// Kernel choices a test or a measurement may force (mxp_debug_override): process-wide, 0 = the
+// library decides.
+int override_get(int knob);
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no libcuda link).
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,

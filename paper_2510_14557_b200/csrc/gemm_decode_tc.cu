@@ -1,0 +1,726 @@
+// Weight-only GEMM for decode shapes (1 <= M <= 16) on the FP4 tensor path:
+//
+//   D[M,N] = A(bf16)[M,K] * dec(W)[N,K]^T          (Sec. 7.1 setting; decode per Eq. 3)
+//
+// The operation is bound by streaming the weights once (0.5625 bytes per element), so the
+// design removes everything else from the path of the bytes:
+//   * tcgen05.mma kind::mxf4 reads packed E2M1 codes with one E8M0 scale per 32 elements, which
+//     is how the weights are stored: no thread ever touches a weight.
+//   * The weights are re-tiled ONCE (decode_prepack_kernel; a re-ordering of the 4-bit codes,
+//     not a dequantization): every CTA owns a fixed range of weight rows, and what it needs for
+//     256 elements of K -- its rows' codes in the 128-byte-swizzled order the MMA reads, their
+//     scales in the 32-lane atoms tcgen05.cp copies, the BM records -- is one contiguous piece
+//     of about 11 KB that a single cp.async.bulk brings in.  148 CTAs read 148 sequential
+//     streams.
+//   * MX+ (Eq. 4): the re-tiled codes hold BM_H (4 or 6, an E2M1 value) in the BM's place; the
+//     rest, BM_L in {0, 0.5, 1, 1.5}, also E2M1, goes into a second operand tile that is zero
+//     elsewhere, built per stage from one record byte per block (position, BM_L, sign) by four
+//     warps, and multiplied by a second MMA into the same accumulator with the same scales.
+//   * The bf16 activations become FP4 as well: per block of 32 the magnitudes, 13 bits below
+//     the block's largest exponent, are written in balanced base 8 (five digits -4..3), each
+//     digit plane an operand row of E2M1 values 0..4 with its own block scale 2^(E - 3 j); the
+//     epilogue adds the planes' accumulator columns.  An element within 2^5 of its block's
+//     maximum is exact, a smaller one is rounded at 2^-13 of that maximum's binade.
+//     A small kernel does this once per call (decode_act_kernel) and leaves the operand images
+//     of all stages in the workspace; the GEMM is launched as its programmatic dependent, so
+//     its CTAs stream weights meanwhile, and fetches the images stage by stage next to the
+//     weights.  (Converting inside the GEMM, every CTA for itself, was built and measured: the
+//     conversion is ~500 instructions per eight elements and costs a CTA 4 us per activation
+//     row, more than the second launch.)
+//   * warp 0 issues the weight copies (the first ring-full before the CTA's set-up barrier),
+//     warp 1 the activation copies, warps 2-5 the MMAs (each every fourth stage, with an
+//     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 build the BM_L
+//     tiles (three groups of four, a stage each in turn: one group needs ~0.8 us per stage,
+//     the stream delivers one every 0.26 us).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <cstring>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace mxp {
+namespace {
+
+constexpr int kIssueWarp0 = 2, kIssuers = 4;
+constexpr int kRowWarp0 = 6;
+constexpr int kResWarp0 = 10, kResWarps = 4, kResGroups = 3;  // three groups of four warps take turns
+constexpr int kWarps = kResWarp0 + kResWarps * kResGroups;
+constexpr int kThreads = 32 * kWarps;
+constexpr int kStageK = 256;   // elements of K per stage: 128 bytes of codes per row
+constexpr int kPlanes = 5;     // balanced base-8 digit planes of an activation
+constexpr int kMaxM = 16;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemSf = 384;  // scale-factor columns: 16 per issuer
+constexpr int kAtom = 512;
+constexpr int kMaxStages = 16;
+constexpr long long kWaitLimit = 4000000000ll;
+constexpr size_t kSmemMax = 227 * 1024;
+constexpr uint32_t kMagic = 0x4D58D0C1u;
+constexpr size_t kHeaderBytes = 256;
+
+// Rows of the activation operand: five planes per activation row, padded to the MMA's N.
+__host__ __device__ constexpr int act_rows(int M) { return (kPlanes * M + 15) / 16 * 16; }
+__host__ __device__ constexpr int sfb_bytes(int nact) { return (nact < 32 ? nact : 32) * 16; }
+__host__ __device__ constexpr size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// How the weight rows are dealt out: a function of the shape and of the SM count only, so the
+// one-off re-tiling and every later call agree.
+struct DecodePlan {
+    int rows;      // weight rows per tile (<= 128)
+    int tiles;     // tiles per CTA
+    int ctas;
+    int nst;       // stages of kStageK per tile
+    uint32_t wimg;  // bytes of one (CTA, tile, stage) weight image
+};
+__host__ inline bool decode_plan(int64_t N, int64_t K, bool plus, int sms, DecodePlan* p)
+{
+    if (N < 1 || K < kStageK || K % kStageK != 0 || K > 32768 || sms < 1 || N > (1ll << 30)) return false;
+    p->tiles = (int)((N + (int64_t)sms * 128 - 1) / ((int64_t)sms * 128));
+    int64_t r = (N + (int64_t)sms * p->tiles - 1) / ((int64_t)sms * p->tiles);
+    if (r < 8) r = 8;
+    p->rows = (int)r;
+    p->ctas = (int)((N + r * p->tiles - 1) / (r * p->tiles));
+    p->nst = (int)(K / kStageK);
+    p->wimg = (uint32_t)up((size_t)p->rows * 128 + 2 * kAtom + (plus ? (size_t)p->rows * 8 : 0), 16);
+    return true;
+}
+
+struct PrepackHeader {
+    uint32_t magic, mode, rows, tiles, ctas, nst, wimg, pad;
+    int64_t N, K;
+};
+
+// Shared memory of the GEMM kernel (bytes from the 1024-byte aligned base).
+// A slot holds a stage's weight image, its activation image (codes at act_off, scale atoms
+// behind) and, for MX+, the BM_L tile built from the image's records (at res_off).
+struct DecodeLayout {
+    size_t act_off, res_off, slot, bars, total;
+    int stages;
+};
+__host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages)
+{
+    DecodeLayout l;
+    l.act_off = up(wimg, 1024);
+    l.res_off = up(l.act_off + (size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact), 1024);
+    l.slot = l.res_off + (plus ? up((size_t)rows * 128, 1024) : 0);
+    l.stages = stages;
+    // an MMA reads 128 rows of 128 bytes from the start of a tile that holds fewer: what follows
+    // the last tile must exist (any bytes are finite E2M1 codes; the rows are never read back)
+    size_t off = up((size_t)stages * l.slot + 16384, 16);
+    l.bars = off;
+    l.total = off + 1024 + 1024;  // barriers; slack for aligning the base
+    return l;
+}
+
+struct DecodeParams {
+    int M, N;
+    const uint8_t* wimg;   // weight images [cta][tile][stage]
+    const uint8_t* aimg;   // activation images [stage]
+    void* D;
+    int64_t ldd;
+    StatusBlock* status;   // may be nullptr
+    int rows, tiles, nst, stages;
+    uint32_t wimg_bytes;
+};
+
+__device__ __forceinline__ void report(StatusBlock* st, volatile uint32_t* abort, uint32_t where)
+{
+    *abort = 1u;
+    if (st != nullptr && atomicCAS(&st->code, 0u, (uint32_t)MXP_ERR_TIMEOUT) == 0u) st->where = where;
+}
+
+// Offset of 16-byte chunk c (0..7) of row r inside a 128B-swizzled tile.
+__host__ __device__ __forceinline__ uint32_t swz_chunk(uint32_t r, uint32_t c)
+{
+    return r * 128u + ((c ^ (r & 7u)) << 4);
+}
+
+__device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(ptx::smem_u32(smem_dst)),
+        "l"(gmem_src), "r"(bytes), "r"(ptx::smem_u32(bar))
+        : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// One-off re-tiling of the weights.  grid (ctas * tiles, nst), 128 threads: thread r = row r
+// of the tile.  Image of one (CTA, tile, stage):
+//   [rows x 128 bytes of codes, 16-byte chunk c of row r at chunk c ^ (r & 7)]
+//   [2 scale atoms of 512 bytes: byte of row r, block b at (r % 32) * 16 + (r / 32) * 4 + b % 4]
+//   [MX+: rows x 8 record bytes: BM position | BM_L code << 5 | sign << 7; 0 = nothing to add]
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+decode_prepack_kernel(const uint8_t* __restrict__ nibbles, const uint8_t* __restrict__ scales,
+                      const uint8_t* __restrict__ bm_index, int64_t N, int64_t K, int plus, int rows,
+                      uint32_t wimg, uint8_t* __restrict__ out, PrepackHeader hdr)
+{
+    const int r = threadIdx.x;
+    const int64_t tile = blockIdx.x;
+    const int st = blockIdx.y;
+    if (tile == 0 && st == 0 && r == 0) *reinterpret_cast<PrepackHeader*>(out) = hdr;
+    uint8_t* img = out + kHeaderBytes + ((size_t)tile * gridDim.y + st) * wimg;
+    const int64_t n = tile * rows + r;
+    const bool live = r < rows && n < N;
+    uint4 code[8];
+    uint8_t sc[8], rec[8];
+#pragma unroll
+    for (int kb = 0; kb < 8; ++kb) {
+        code[kb] = make_uint4(0u, 0u, 0u, 0u);
+        sc[kb] = 0x7F;
+        rec[kb] = 0;
+    }
+    if (live) {
+        const int64_t b0 = n * (K / 32) + (int64_t)st * 8;
+#pragma unroll
+        for (int kb = 0; kb < 8; ++kb) {
+            code[kb] = __ldg(reinterpret_cast<const uint4*>(nibbles + (b0 + kb) * 16));
+            sc[kb] = scales[b0 + kb];
+            if (sc[kb] == 0) code[kb] = make_uint4(0u, 0u, 0u, 0u);  // flushed block: zeros
+            if (plus && sc[kb] != 0 && sc[kb] != 0xFF) {
+                const uint32_t pos = bm_index[b0 + kb] & 31u;
+                uint32_t* w = &code[kb].x + (pos >> 3);  // (x, y, z, w are consecutive words)
+                const uint32_t sh = (pos & 7u) * 4u;
+                const uint32_t nib = (*w >> sh) & 15u;   // sign, m2 m1 m0
+                const uint32_t hi = (nib & 8u) | 6u | ((nib >> 2) & 1u);  // BM_H: E2M1 code 11 m2
+                *w = (*w & ~(15u << sh)) | (hi << sh);
+                rec[kb] = (uint8_t)(pos | ((nib & 3u) << 5) | ((nib & 8u) << 4));
+                if ((nib & 3u) == 0u) rec[kb] = 0;       // BM_L = 0
+            }
+        }
+    }
+    if (r < rows) {
+#pragma unroll
+        for (int kb = 0; kb < 8; ++kb)
+            *reinterpret_cast<uint4*>(img + swz_chunk((uint32_t)r, (uint32_t)kb)) = code[kb];
+        if (plus) {
+            uint2 v;
+            v.x = (uint32_t)rec[0] | ((uint32_t)rec[1] << 8) | ((uint32_t)rec[2] << 16) | ((uint32_t)rec[3] << 24);
+            v.y = (uint32_t)rec[4] | ((uint32_t)rec[5] << 8) | ((uint32_t)rec[6] << 16) | ((uint32_t)rec[7] << 24);
+            *reinterpret_cast<uint2*>(img + (size_t)rows * 128 + 2 * kAtom + (size_t)r * 8) = v;
+        }
+    }
+    // every row of the atoms gets a finite scale, also those past the tile
+    uint8_t* atoms = img + (size_t)rows * 128;
+    const uint32_t so = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;
+    const bool use = r < rows;
+    *reinterpret_cast<uint32_t*>(atoms + so) =
+        use ? (uint32_t)sc[0] | ((uint32_t)sc[1] << 8) | ((uint32_t)sc[2] << 16) | ((uint32_t)sc[3] << 24) : 0x7F7F7F7Fu;
+    *reinterpret_cast<uint32_t*>(atoms + kAtom + so) =
+        use ? (uint32_t)sc[4] | ((uint32_t)sc[5] << 8) | ((uint32_t)sc[6] << 16) | ((uint32_t)sc[7] << 24) : 0x7F7F7F7Fu;
+}
+
+// Eight activations (quarter `qd` of block `kb` of a stage, activation row m; the four lanes of
+// a quad hold the four quarters of one block) -> their five digit planes: one word of codes per
+// plane into the stage's tile `codes`, and the planes' scale bytes into its atoms `sf`.
+__device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, int qd, uint8_t* codes, uint8_t* sf,
+                                                int sfb)
+{
+    const uint32_t x[4] = {v.x, v.y, v.z, v.w};
+    // largest exponent field of the block (zero and subnormals count as field 1)
+    uint32_t eb = 1;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        eb = max(eb, (x[q] >> 7) & 255u);
+        eb = max(eb, (x[q] >> 23) & 255u);
+    }
+    eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 1));
+    eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 2));
+    const bool nonfinite = eb == 255u;
+    // t = |a| / 2^(E - 12), rounded to an integer below 2^13, plus 4 in each of five octal
+    // places: octal digit j of t, minus 4, is the balanced digit d_j in -4..3 with
+    // |a| = sum_j d_j 2^(E - 3 j)
+    uint32_t t[8], neg = 0u;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const uint32_t h = (e & 1) ? x[e >> 1] >> 16 : x[e >> 1] & 0xFFFFu;
+        const uint32_t ef = (h >> 7) & 255u;
+        const uint32_t m13 = ((ef ? 128u : 0u) | (h & 127u)) << 5;  // at the block's largest exponent
+        const uint32_t down = min(eb - max(ef, 1u), 31u);           // binades below it
+        t[e] = ((m13 + ((1u << down) >> 1)) >> down) + 0x4924u;     // rounded to nearest
+        neg |= (h >> 15) << e;
+    }
+#pragma unroll
+    for (int j = 0; j < kPlanes; ++j) {
+        const int sbyte = (int)eb - 3 * j;  // E8M0 byte of 2^(E - 3 j)
+        uint32_t w = 0u;
+        if (sbyte >= 0 && !nonfinite) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int d = (int)((t[e] >> (3 * (4 - j))) & 7u) - 4;
+                const uint32_t ad = (uint32_t)(d < 0 ? -d : d);
+                const uint32_t code = (0x65420u >> (4u * ad)) & 7u;  // E2M1 codes of 0 1 2 3 4
+                const uint32_t sg = ((neg >> e) & 1u) ^ (d < 0 ? 1u : 0u);
+                w |= (code | (sg << 3)) << (4 * e);
+            }
+        }
+        const int row = kPlanes * m + j;
+        *reinterpret_cast<uint32_t*>(codes + swz_chunk((uint32_t)row, (uint32_t)kb) + 4 * qd) = w;
+        if (qd == 0)
+            sf[(kb >> 2) * sfb + (row & 31) * 16 + (row >> 5) * 4 + (kb & 3)] =
+                (uint8_t)(nonfinite ? 255 : max(sbyte, 0));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Activations -> FP4 digit planes, once per call.  grid nst, 32 * M threads (four per block of
+// 32 elements, eight elements each).  Image of one stage:
+//   [nact rows x 128 bytes of codes, swizzled as above; row 5 m + j = plane j of activation m]
+//   [2 scale atoms of sfb_bytes(nact): byte of row n, block b at (n % 32) * 16 + (n / 32) * 4 + b % 4]
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32 * kMaxM)
+decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int nact, uint8_t* __restrict__ aimg,
+                  StatusBlock* status, int clear_status)
+{
+    ptx::grid_launch_dependents();  // the GEMM's CTAs may start streaming weights now
+    extern __shared__ uint8_t img[];  // nact * 128 + 2 * sfb
+    const int st = blockIdx.x;
+    const int sfb = sfb_bytes(nact);
+    const int bytes = nact * 128 + 2 * sfb;
+    for (int i = threadIdx.x; i < nact * 128 / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(img)[i] = make_uint4(0u, 0u, 0u, 0u);   // absent rows: zero codes ...
+    for (int i = threadIdx.x; i < 2 * sfb / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(img + nact * 128)[i] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+    __syncthreads();  // ... with a finite scale; the rows in use land on top
+    ptx::grid_dependency_wait();  // A may come from the kernel before
+    if (clear_status && st == 0 && threadIdx.x == 0 && status != nullptr) {
+        status->code = 0u;
+        status->where = 0u;
+    }
+    const int i = threadIdx.x, blk = i >> 2, qd = i & 3;
+    const int m = blk >> 3, kb = blk & 7;
+    if (m < M) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(A + (int64_t)m * lda + (int64_t)st * kStageK + kb * 32) + qd);
+        convert_quarter(v, m, kb, qd, img, img + nact * 128, sfb);
+    }
+    __syncthreads();
+    uint4* dst = reinterpret_cast<uint4*>(aimg + (size_t)st * bytes);
+    for (int k = threadIdx.x; k < bytes / 16; k += blockDim.x) dst[k] = reinterpret_cast<const uint4*>(img)[k];
+}
+
+// ------------------------------------------------------------------------------------------
+// The GEMM.  kNact: rows of the activation operand (16 .. 80); kPlus: MXFP4+ weights.
+// ------------------------------------------------------------------------------------------
+template <int kNact, bool kPlus, typename OutT>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_decode_tc_kernel(const DecodeParams prm)
+{
+    constexpr int kSfb = sfb_bytes(kNact);
+    constexpr int kMt = kNact / kPlanes;  // activation rows the operand can hold
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int S = prm.stages;
+    const int nst = prm.nst;
+    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // the slot's copies landed
+    uint64_t* empty = full + kMaxStages;       // the slot's MMAs are done
+    uint64_t* res_full = empty + kMaxStages;   // the slot's BM_L tile is written
+    uint64_t* acc_full = res_full + kMaxStages;
+    uint64_t* acc_empty = acc_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+    volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    auto slot = [&](int s) { return smem + (size_t)s * L.slot; };
+    const int64_t row0 = (int64_t)blockIdx.x * prm.tiles * prm.rows;  // first weight row of this CTA
+    // tiles of this CTA that hold rows, and its stages in all
+    const int ntl = (int)min((int64_t)prm.tiles, (prm.N - row0 + prm.rows - 1) / prm.rows);
+    const uint32_t total = (uint32_t)(ntl * nst);
+    const uint8_t* wsrc = prm.wimg + (size_t)blockIdx.x * prm.tiles * nst * prm.wimg_bytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            ptx::mbar_init(&full[s], 2);
+            ptx::mbar_init(&empty[s], 1);
+            ptx::mbar_init(&res_full[s], kResWarps);
+        }
+        ptx::mbar_init(acc_full, kIssuers);
+        ptx::mbar_init(acc_empty, 4);
+        *abort = 0u;
+        ptx::fence_mbar_init();
+        // The first ring-full of weight copies goes out before anything else: the weights do not
+        // depend on the kernel before, and every later step of the set-up overlaps their latency.
+        for (uint32_t c = 0; c < total && c < (uint32_t)S; ++c) {
+            ptx::mbar_arrive_expect_tx(&full[c], prm.wimg_bytes);
+            bulk_g2s(slot((int)c), wsrc + (size_t)c * prm.wimg_bytes, prm.wimg_bytes, &full[c]);
+        }
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(tmem_slot, kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    ptx::grid_launch_dependents();  // whatever follows on the stream may be scheduled
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- weight copies (the rest)
+        if (lane == 0) {
+            for (uint32_t c = (uint32_t)S; c < total; ++c) {
+                const int s = c % S;
+                if (!ptx::mbar_wait(&empty[s], (c / S - 1) & 1, abort, kWaitLimit)) {
+                    report(prm.status, abort, 0x7100 + s);
+                    break;
+                }
+                ptx::mbar_arrive_expect_tx(&full[s], prm.wimg_bytes);
+                bulk_g2s(slot(s), wsrc + (size_t)c * prm.wimg_bytes, prm.wimg_bytes, &full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- activation copies
+        if (lane == 0) {
+            ptx::grid_dependency_wait();  // the activation images are the preceding kernel's output
+            constexpr uint32_t kBytes = kNact * 128 + 2 * kSfb;
+            for (uint32_t c = 0; c < total; ++c) {
+                const int s = c % S;
+                if (c >= (uint32_t)S && !ptx::mbar_wait(&empty[s], (c / S - 1) & 1, abort, kWaitLimit)) {
+                    report(prm.status, abort, 0x7200 + s);
+                    break;
+                }
+                ptx::mbar_arrive_expect_tx(&full[s], kBytes);
+                bulk_g2s(slot(s) + L.act_off, prm.aimg + (size_t)(c % (uint32_t)nst) * kBytes, kBytes, &full[s]);
+            }
+        }
+    } else if (warp >= kIssueWarp0 && warp < kIssueWarp0 + kIssuers) {
+        // ---------------------------------------------------------------- MMA issuers
+        // Issuer i takes the stages whose running number is i (mod 4): the number of slots is a
+        // multiple of four, so a slot always belongs to the same issuer, which sees every fill
+        // of it in turn (the parity it waits for is never ambiguous).
+        const int iss = warp - kIssueWarp0;
+        const uint32_t tmem_acc = tmem_base + (uint32_t)(iss * kNact);
+        uint32_t c = 0;
+        bool ok = true;
+        for (int t = 0; t < ntl && ok; ++t) {
+            if (t > 0 && !ptx::mbar_wait(acc_empty, (uint32_t)(t - 1) & 1, abort, kWaitLimit)) {
+                if (lane == 0) report(prm.status, abort, 0x7300);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int first = (iss - (int)(c % kIssuers) + kIssuers) % kIssuers;
+            for (int st = first; st < nst; st += kIssuers) {
+                const uint32_t cc = c + (uint32_t)st;
+                const int s = cc % S;
+                const uint32_t ph = (cc / S) & 1;
+                if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit)) {
+                    if (lane == 0) report(prm.status, abort, 0x7400 + s);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint8_t* sl = slot(s);
+                const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(sl));
+                const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(sl + L.act_off));
+                const uint32_t sfa = ptx::smem_u32(sl + (size_t)prm.rows * 128);
+                const uint32_t sfb = ptx::smem_u32(sl + L.act_off + kNact * 128);
+                const uint32_t t_sf = tmem_base + kTmemSf + 16u * (uint32_t)iss;
+                if (ptx::elect_one()) {
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {  // 128 elements: one scale atom per operand
+                        const uint32_t t_sfa = t_sf + 8u * (uint32_t)g, t_sfb = t_sfa + 4u;
+                        ptx::tc_cp_sf(t_sfa, ptx::smem_desc_sf(sfa + (uint32_t)(g * kAtom)));
+                        ptx::tc_cp_sf(t_sfb, ptx::smem_desc_sf(sfb + (uint32_t)(g * kSfb)));
+#pragma unroll
+                        for (int kk = 0; kk < 2; ++kk) {  // 64 elements = 32 bytes per MMA
+                            const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
+                            ptx::mma_mxf4(tmem_acc, da + adv, db + adv,
+                                          ptx::idesc_block_scaled(1, 1, 128, kNact, 2 * kk, 2 * kk), t_sfa, t_sfb,
+                                          (st == first && g == 0 && kk == 0) ? 0u : 1u);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (kPlus) {
+                    // the BM_L tile of the stage, same scales, same accumulator (Eq. 4)
+                    if (!ptx::mbar_wait(&res_full[s], ph, abort, kWaitLimit)) {
+                        if (lane == 0) report(prm.status, abort, 0x7500 + s);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint64_t dr = ptx::smem_desc_sw128(ptx::smem_u32(sl + L.res_off));
+                    if (ptx::elect_one()) {
+#pragma unroll
+                        for (int g = 0; g < 2; ++g) {
+                            const uint32_t t_sfa = t_sf + 8u * (uint32_t)g, t_sfb = t_sfa + 4u;
+#pragma unroll
+                            for (int kk = 0; kk < 2; ++kk) {
+                                const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);
+                                ptx::mma_mxf4(tmem_acc, dr + adv, db + adv,
+                                              ptx::idesc_block_scaled(1, 1, 128, kNact, 2 * kk, 2 * kk), t_sfa,
+                                              t_sfb, 1u);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (ptx::elect_one()) ptx::tc_commit(&empty[s]);
+                __syncwarp();
+            }
+            c += (uint32_t)nst;
+            if (!ok) break;
+            if (ptx::elect_one()) ptx::tc_commit(acc_full);
+            __syncwarp();
+        }
+    } else if (warp < kRowWarp0 + 4) {
+        // ---------------------------------------------------------------- row warps (epilogue)
+        // Thread = weight row of the tile = TMEM lane.  An output is the sum of its five planes'
+        // columns over the four issuers' accumulators.
+        const int q = warp & 3;  // the TMEM lane quarter this warp may read
+        const int row = 32 * q + lane;
+        ptx::grid_dependency_wait();  // D may still be in use by the kernel before
+        for (int t = 0; t < ntl; ++t) {
+            const int64_t n0 = row0 + (int64_t)t * prm.rows;
+            const int rows_here = (int)min((int64_t)prm.rows, (int64_t)prm.N - n0);
+            if (!ptx::mbar_wait_relaxed(acc_full, (uint32_t)t & 1, abort, kWaitLimit, 200u)) {
+                if (lane == 0) report(prm.status, abort, 0x7600);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            float o[kMt];
+#pragma unroll
+            for (int m = 0; m < kMt; ++m) o[m] = 0.f;
+            const uint32_t c0 = (uint32_t)t * (uint32_t)nst;
+#pragma unroll
+            for (int ch = 0; ch < kNact / 16; ++ch) {
+                float part[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) part[j] = 0.f;
+#pragma unroll
+                for (int a = 0; a < kIssuers; ++a) {
+                    // issuer a wrote its accumulator only if it had a stage of this tile
+                    if ((a - (int)(c0 % kIssuers) + kIssuers) % kIssuers >= nst) continue;
+                    uint32_t r2[16];
+                    ptx::tmem_ld_32x16(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(a * kNact + 16 * ch), r2);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) part[j] += __uint_as_float(r2[j]);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if ((16 * ch + j) / kPlanes < kMt) o[(16 * ch + j) / kPlanes] += part[j];
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(acc_empty);
+            if (row < rows_here) {
+#pragma unroll
+                for (int m = 0; m < kMt; ++m) {
+                    if (m < prm.M) {
+                        const int64_t off = (int64_t)m * prm.ldd + n0 + row;
+                        if (sizeof(OutT) == 4)
+                            static_cast<float*>(prm.D)[off] = o[m];
+                        else
+                            static_cast<__nv_bfloat16*>(prm.D)[off] = __float2bfloat16_rn(o[m]);
+                    }
+                }
+            }
+        }
+    } else if (kPlus) {
+        // ---------------------------------------------------------------- BM_L tiles
+        // Group g of four warps takes the stages whose running number is g (mod 3).  The tile
+        // lives in the stage's slot, so once the slot's copies have landed nothing else can be
+        // using it.  The four warps clear it together (consecutive threads, consecutive 16
+        // bytes), then thread = weight row drops in, per block, the code its record byte names.
+        const int grp = (warp - kResWarp0) / kResWarps;
+        const int r = (int)threadIdx.x - 32 * (kResWarp0 + grp * kResWarps);
+        for (uint32_t c = (uint32_t)grp; c < total; c += kResGroups) {
+            const int s = c % S;
+            if (!ptx::mbar_wait(&full[s], (c / S) & 1, abort, kWaitLimit)) {
+                if (lane == 0) report(prm.status, abort, 0x7700 + s);
+                break;
+            }
+            uint8_t* tile = slot(s) + L.res_off;
+            for (int k = r; k < prm.rows * 8; k += 32 * kResWarps)
+                reinterpret_cast<uint4*>(tile)[k] = make_uint4(0u, 0u, 0u, 0u);
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(32 * kResWarps) : "memory");
+            if (r < prm.rows) {
+                uint8_t* mine = tile + (size_t)r * 128;
+                const uint2 rec = *reinterpret_cast<const uint2*>(slot(s) + (size_t)prm.rows * 128 + 2 * kAtom + (size_t)r * 8);
+#pragma unroll
+                for (int kb = 0; kb < 8; ++kb) {
+                    const uint32_t b = ((kb < 4 ? rec.x : rec.y) >> (8 * (kb & 3))) & 255u;
+                    if (b & 0x60u) {
+                        const uint32_t pos = b & 31u;
+                        const uint32_t nib = ((b >> 5) & 3u) | ((b >> 4) & 8u);
+                        mine[(((uint32_t)kb ^ ((uint32_t)r & 7u)) << 4) + (pos >> 1)] = (uint8_t)(nib << (4u * (pos & 1u)));
+                    }
+                }
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&res_full[s]);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncthreads();
+    if (*abort != 0u && threadIdx.x == 0) {
+        // after a timeout, copies may still be in flight into this CTA's shared memory: give
+        // them (bounded) time to land before the CTA leaves
+        const long long t0 = clock64();
+        for (int s = 0; s < S; ++s)
+            while (!ptx::mbar_try_wait(&full[s], 0) && !ptx::mbar_try_wait(&full[s], 1) &&
+                   clock64() - t0 < kWaitLimit) {
+            }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// Ring slots that fit: a multiple of four (see the issuers), at most sixteen.
+int pick_stages(const DecodePlan& p, int nact, bool plus)
+{
+    for (int s = kMaxStages; s >= 4; s -= 4)
+        if (decode_layout(p.rows, p.wimg, nact, plus, s).total <= kSmemMax) return s;
+    return 0;
+}
+
+template <int kNact, bool kPlus, typename OutT>
+cudaError_t launch(const DecodeParams& prm, int ctas, size_t smem, cudaStream_t stream)
+{
+    auto kern = gemm_decode_tc_kernel<kNact, kPlus, OutT>;
+    static SmemAttrOnce once;
+    cudaError_t e = ensure_dynamic_smem(kern, (int)kSmemMax, once);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, prm);
+}
+
+template <int kNact>
+cudaError_t launch_n(bool plus, bool f32, const DecodeParams& prm, int ctas, size_t smem, cudaStream_t stream)
+{
+    if (plus)
+        return f32 ? launch<kNact, true, float>(prm, ctas, smem, stream)
+                   : launch<kNact, true, __nv_bfloat16>(prm, ctas, smem, stream);
+    return f32 ? launch<kNact, false, float>(prm, ctas, smem, stream)
+               : launch<kNact, false, __nv_bfloat16>(prm, ctas, smem, stream);
+}
+
+}  // namespace
+
+size_t decode_prepack_bytes(int64_t N, int64_t K, mxp_mode mode)
+{
+    if (mode != MXP_MODE_MXFP4 && mode != MXP_MODE_MXFP4_PLUS) return 0;
+    DecodePlan p;
+    if (!decode_plan(N, K, mode == MXP_MODE_MXFP4_PLUS, sm_count(), &p)) return 0;
+    return kHeaderBytes + (size_t)p.ctas * p.tiles * p.nst * p.wimg;
+}
+
+size_t decode_workspace_bytes(int64_t M, int64_t K)
+{
+    if (M < 1 || M > kMaxM || K < kStageK || K % kStageK != 0 || K > 32768) return 0;
+    const int nact = act_rows((int)M);
+    return kStatusBytes + (size_t)(K / kStageK) * ((size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact));
+}
+
+mxp_status decode_prepack(const mxp_packed& B, void* out, size_t out_bytes, cudaStream_t stream)
+{
+    const bool plus = B.mode == MXP_MODE_MXFP4_PLUS;
+    DecodePlan p;
+    if (!decode_plan(B.rows, B.cols, plus, sm_count(), &p)) return MXP_ERR_UNSUPPORTED;
+    const size_t need = decode_prepack_bytes(B.rows, B.cols, B.mode);
+    if (need == 0) return MXP_ERR_UNSUPPORTED;
+    if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(out) & 255) return MXP_ERR_INVALID_ARG;
+    PrepackHeader h = {};
+    h.magic = kMagic;
+    h.mode = (uint32_t)B.mode;
+    h.rows = (uint32_t)p.rows;
+    h.tiles = (uint32_t)p.tiles;
+    h.ctas = (uint32_t)p.ctas;
+    h.nst = (uint32_t)p.nst;
+    h.wimg = p.wimg;
+    h.N = B.rows;
+    h.K = B.cols;
+    decode_prepack_kernel<<<dim3((unsigned)(p.ctas * p.tiles), (unsigned)p.nst), 128, 0, stream>>>(
+        B.nibbles, B.scales, B.bm_index, B.rows, B.cols, plus ? 1 : 0, p.rows, p.wimg,
+        static_cast<uint8_t*>(out), h);
+    return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, mxp_mode b_mode,
+                                 const void* b_prepacked, size_t b_prepacked_bytes, void* D, mxp_dtype d_dt,
+                                 int64_t ldd, void* workspace, size_t workspace_bytes, bool chained,
+                                 cudaStream_t stream)
+{
+    const bool plus = b_mode == MXP_MODE_MXFP4_PLUS;
+    DecodePlan p;
+    if (M < 1 || M > kMaxM || !decode_plan(N, K, plus, sm_count(), &p)) return MXP_ERR_UNSUPPORTED;
+    if (b_mode != MXP_MODE_MXFP4 && b_mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
+    // the re-tiled weights must be those of this shape, mode and device: their size says so
+    if (b_prepacked_bytes != decode_prepack_bytes(N, K, b_mode)) return MXP_ERR_INVALID_ARG;
+    const size_t need = decode_workspace_bytes(M, K);
+    if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
+    const int nact = act_rows((int)M);
+    const int stages = pick_stages(p, nact, plus);
+    if (stages == 0) return MXP_ERR_UNSUPPORTED;
+    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    DecodeParams prm = {};
+    prm.M = (int)M;
+    prm.N = (int)N;
+    prm.wimg = static_cast<const uint8_t*>(b_prepacked) + kHeaderBytes;
+    prm.aimg = ws + kStatusBytes;
+    prm.D = D;
+    prm.ldd = ldd;
+    prm.status = reinterpret_cast<StatusBlock*>(ws);
+    prm.rows = p.rows;
+    prm.tiles = p.tiles;
+    prm.nst = p.nst;
+    prm.stages = stages;
+    prm.wimg_bytes = p.wimg;
+    {   // activations -> digit planes; in a chain it may start while the kernel before drains
+        // (same shared-memory carve-out as the GEMM, so that the SMs are not reconfigured
+        // between the two kernels of every call: that alone cost 1.6 us per call)
+        static SmemAttrOnce carve;
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !carve.done[dev]) {
+            cudaFuncSetAttribute(decode_act_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+            carve.done[dev] = true;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)p.nst);
+        cfg.blockDim = dim3((unsigned)(32 * M < 64 ? 64 : 32 * M));
+        cfg.dynamicSmemBytes = (size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = chained ? 1 : 0;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, decode_act_kernel, static_cast<const __nv_bfloat16*>(A), lda,
+                                           (int)M, nact, ws + kStatusBytes, prm.status, chained ? 0 : 1);
+        if (e != cudaSuccess) return MXP_ERR_CUDA;
+    }
+    const bool f32 = d_dt == MXP_F32;
+    cudaError_t e;
+    switch (nact) {
+        case 16: e = launch_n<16>(plus, f32, prm, p.ctas, L.total, stream); break;
+        case 32: e = launch_n<32>(plus, f32, prm, p.ctas, L.total, stream); break;
+        case 48: e = launch_n<48>(plus, f32, prm, p.ctas, L.total, stream); break;
+        case 64: e = launch_n<64>(plus, f32, prm, p.ctas, L.total, stream); break;
+        default: e = launch_n<80>(plus, f32, prm, p.ctas, L.total, stream); break;
+    }
+    return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+}
+
+}  // namespace mxp

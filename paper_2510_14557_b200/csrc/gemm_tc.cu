@@ -1229,14 +1229,14 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     if (prm.num_sms <= 0) return MXP_ERR_CUDA;
     // Kernel choice by measurement on the prefill shapes: the pair kernel wins whenever an
     // operand is MX+ (a third less residual-tile memory and patch work per CTA buys pipeline
-    // depth); the single-CTA kernel wins for plain MXFP4.  MXP_GEMM_KERNEL=single|pair
-    // overrides the choice (measurement aid).
-    const char* force = getenv("MXP_GEMM_KERNEL");
+    // depth); the single-CTA kernel wins for plain MXFP4.  mxp_debug_override can force
+    // either (tests and measurements).
+    const int force = override_get(MXP_KNOB_INPLACE_KERNEL);  // 1: single CTA, 2: CTA pair
     // Default: the streamed pair kernel on prepacked operands, when the shape allows it and
     // the caller's workspace has room for the prepacked copies; otherwise the kernels below,
     // which work in place and need only the status block.
     const size_t fast = stream_workspace_bytes(M, N, K, A.mode, B.mode);
-    const bool forced_other = force != nullptr && (force[0] == 's' || force[0] == 'p');
+    const bool forced_other = force != 0;
     if (fast != 0 && workspace_bytes >= fast && !forced_other)
         return launch_gemm_tc_stream(M, N, K, A, B, nullptr, D, d_dt, ldd, workspace, workspace_bytes,
                                      stream);
@@ -1245,8 +1245,8 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     // status block and clock stamp (these kernels leave no stamp)
     if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return MXP_ERR_CUDA;
     bool use_pair = M > 128 && N > 128 && (ap || bp);
-    if (force != nullptr && force[0] == 's') use_pair = false;
-    if (force != nullptr && force[0] == 'p') use_pair = M > 128 && N > 128;
+    if (force == 1) use_pair = false;
+    if (force == 2) use_pair = M > 128 && N > 128;
     if (use_pair) {
         if (d_dt == MXP_F32) return launch_pair_modes<float>(ap, bp, ta, tb, prm, stream);
         return launch_pair_modes<__nv_bfloat16>(ap, bp, ta, tb, prm, stream);

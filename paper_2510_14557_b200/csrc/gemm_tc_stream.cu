@@ -770,8 +770,8 @@ Layout layout(int64_t M, int64_t N, int64_t K, bool wide, int parts_a = 1, int p
 // halves would: compare the columns each CTA pair walks through either way.
 int choose_halves(int64_t M, int64_t N, bool wide, int num_sms)
 {
-    const char* env = std::getenv("MXP_S_HALVES");  // "1" / "2": tests and experiments
-    if (env != nullptr && (env[0] == '1' || env[0] == '2')) return env[0] - '0';
+    const int forced = override_get(MXP_KNOB_STREAM_HALVES);  // tests and measurements
+    if (forced == 1 || forced == 2) return forced;
     const int64_t clusters = num_sms / 2, tiles_m = (M + kTileM - 1) / kTileM;
     auto cost = [&](int h) {  // columns a CTA pair walks through
         const int64_t tile_n = (int64_t)h * sub_n(wide, h);

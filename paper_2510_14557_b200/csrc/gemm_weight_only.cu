@@ -249,30 +249,9 @@ cudaError_t launch_gemm_weight_only(int64_t M, int64_t N, int64_t K, const void*
                                     void* workspace, size_t workspace_bytes, cudaStream_t stream)
 {
     if (M > (1 << 20) || N > (1ll << 30) || K > (1ll << 30)) return cudaErrorNotSupported;
-    // Decode shapes go to the streamed kernel; MXP_WO_KERNEL=old|stream overrides (measurement
-    // and test aid).  A workspace, if given, receives the status of its bounded waits.
-    const char* force = getenv("MXP_WO_KERNEL");
-    const bool want_old = force != nullptr && force[0] == 'o';
-    const bool want_tma = force != nullptr && force[0] == 't';
-    const bool want_fp4 = force != nullptr && force[0] == 'f';
-    if (want_fp4 && wo_fp4_supported(M, N, K, A, lda, B)) {
-        void* status = nullptr;
-        if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {
-            status = workspace;
-            if (cudaMemsetAsync(status, 0, sizeof(StatusBlock), stream) != cudaSuccess)
-                return cudaErrorUnknown;
-        }
-        return launch_gemm_wo_fp4(M, N, K, A, lda, B, D, d_dt, ldd, status, stream);
-    }
-    if (want_tma && wo_tma_supported(M, N, K, A, lda, B)) {
-        void* status = nullptr;
-        if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {
-            status = workspace;
-            if (cudaMemsetAsync(status, 0, sizeof(StatusBlock), stream) != cudaSuccess)
-                return cudaErrorUnknown;
-        }
-        return launch_gemm_wo_tma(M, N, K, A, lda, B, D, d_dt, ldd, status, stream);
-    }
+    // Decode shapes go to the streamed kernel (mxp_debug_override can force the general one).
+    // A workspace, if given, receives the status of its bounded waits.
+    const bool want_old = override_get(MXP_KNOB_WEIGHT_ONLY_KERNEL) == 1;
     if (!want_old && M <= 64 && wo_stream_supported(M, N, K, A, lda, B)) {
         void* status = nullptr;
         if (workspace != nullptr && workspace_bytes >= sizeof(StatusBlock)) {

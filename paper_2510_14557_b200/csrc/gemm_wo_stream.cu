@@ -763,15 +763,8 @@ cudaError_t launch(WoParams prm, int num_sms, bool chained, cudaStream_t stream)
 
 // Largest M for which the correction warps beat patching (measured on config 3, CUDA graph:
 // 14.1 vs 15.2 us at M = 1, 14.8 vs 15.5 at M = 2, 15.7 vs 15.6 at M = 3, 21.3 vs 17.4 at
-// M = 8).  MXP_WO_CORR_MAXM=<0..8> moves the switch-over for measurements.
-int corr_max_m()
-{
-    if (const char* e = getenv("MXP_WO_CORR_MAXM")) {
-        const int v = atoi(e);
-        return v < 0 ? 0 : (v > 8 ? 8 : v);
-    }
-    return 2;
-}
+// M = 8).
+constexpr int kCorrMaxM = 2;
 
 }  // namespace
 
@@ -787,7 +780,7 @@ bool wo_stream_supported(int64_t M, int64_t N, int64_t K, const void* A, int64_t
     const bool plus = B.mode != MXP_MODE_MXFP4;
     if (plus && (reinterpret_cast<uintptr_t>(B.bm_index) & 15)) return false;
     int st, rb, mb;
-    return wo_plan((int)K, M <= 8 ? 8 : 16, plus, plus && M <= corr_max_m(), &st, &rb, &mb);
+    return wo_plan((int)K, M <= 8 ? 8 : 16, plus, plus && M <= kCorrMaxM, &st, &rb, &mb);
 }
 
 cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
@@ -824,7 +817,7 @@ cudaError_t launch_gemm_wo_stream(int64_t M, int64_t N, int64_t K, const void* A
                        : launch<MT, 0, false, __nv_bfloat16>(prm, sms, chained, stream);   \
     }
     // one or two activation rows: the BM goes to the correction warps (see the kernel)
-    if (M <= corr_max_m()) {
+    if (M <= kCorrMaxM) {
         MXP_WO_LAUNCH(1, true)
     }
     if (M <= 8) {

@@ -12,12 +12,12 @@
 // code = the E2M1 value nearest to |x| / d (ties to the even code, saturating at 6, sign of the
 // input kept);  BM: m = nearest integer to (clamp(amax / d, 4, 8) - 4) * 2, ties to even, at
 // most 7.  Decode: +-E * d rounded once to the output type.
-// How: every quotient is first taken in binary32 through a reciprocal, twice -- scaled down and
-// up by 2^-20, which brackets the exact quotient (the binary32 steps err by < 2^-22) -- and
-// both go through the hardware cast.  Where the two casts agree no rounding boundary lies in
-// between and the code is the definition's.  Where they differ, exactly one boundary t lies in
-// between, and the side is decided by comparing |x| with t * d (resp. amax with 6 t ts) in
-// binary64, where those products (at most 33 significant bits) are exact; equality is the tie.
+// How: every quotient is first taken in binary32 through a reciprocal (error below 2^-22) and
+// cast by the hardware; that is the definition's code unless a rounding boundary t of the cast
+// lies within that error of the product.  Those cases are found cheaply (elements: by the
+// product's bit pattern; scale byte and BM: by casting the product scaled down and up by
+// 2^-20) and settled by comparing |x| with t * d (resp. amax with 6 t ts) in binary64, where
+// those products (at most 33 significant bits) are exact; equality is the tie.
 //
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -58,40 +58,41 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float* f)
 constexpr float kDown = 1.f - 9.5367431640625e-07f;  // 1 - 2^-20
 constexpr float kUp = 1.f + 9.5367431640625e-07f;    // 1 + 2^-20
 
-// Value of an E2M1 magnitude code (0..7) times four: 0 2 4 6 8 12 16 24, five bits each.
-__device__ __forceinline__ uint32_t e2m1_times4(uint32_t c)
-{
-    return (uint32_t)((0xC418831040ull >> (5u * c)) & 31ull);
-}
-
 // One block of 16: two words of codes, the scale byte and the BM index (0 when not extended).
-// `src` points at the block's 16 source elements (read again only for the rare element whose
-// two bracketing casts differ).
 // kKey: the values came from bf16, so their low 16 bits are zero and (magnitude bits | 15 -
 // position) is a key whose unsigned maximum gives the largest magnitude and, among equal
 // ones, the first position in one pass.
+// The block's source words stay as loaded (bf16: two elements per word), which halves the
+// registers a lane holds while it works on the other block; an element is widened where used.
+template <bool kHalf>
+__device__ __forceinline__ float elem(const uint32_t* raw, int i)
+{
+    if (!kHalf) return __uint_as_float(raw[i]);
+    return __uint_as_float((i & 1) ? raw[i >> 1] & 0xFFFF0000u : raw[i >> 1] << 16);
+}
+
 template <typename T, bool kPlus>
-__device__ __forceinline__ void nvfp4_block(const float* x, const T* __restrict__ src, float ts,
-                                            float six_ts, uint32_t& w0, uint32_t& w1,
+__device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float six_ts, uint32_t& w0, uint32_t& w1,
                                             uint32_t& scale_byte, uint32_t& index)
 {
     constexpr bool kKey = sizeof(T) == 2;
+#define X(i) elem<kKey>(raw, (i))
     float amax = 0.f;
     int bm = 0;
     if (kPlus && kKey) {
         uint32_t key = 0;
 #pragma unroll
         for (int i = 0; i < 16; ++i)
-            key = max(key, (__float_as_uint(x[i]) & 0x7FFFFFFFu) | (uint32_t)(15 - i));
+            key = max(key, (__float_as_uint(X(i)) & 0x7FFFFFFFu) | (uint32_t)(15 - i));
         amax = __uint_as_float(key & 0x7FFF0000u);
         bm = 15 - (int)(key & 15u);
     } else {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(x[i]));
+        for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(X(i)));
         if (kPlus) {
 #pragma unroll
             for (int i = 15; i >= 0; --i)
-                if (fabsf(x[i]) == amax) bm = i;  // the first of equal maxima
+                if (fabsf(X(i)) == amax) bm = i;  // the first of equal maxima
         }
     }
     // scale byte: E4M3 nearest to amax / (6 ts)
@@ -106,37 +107,44 @@ __device__ __forceinline__ void nvfp4_block(const float* x, const T* __restrict_
     }
     const float e = e4m3_byte_to_f32(sb);
     const float r = __frcp_rn(__fmul_rn(e, ts));
-    const float r_dn = __fmul_rn(r, kDown), r_up = __fmul_rn(r, kUp);
     // r > 0, so x * r has the sign of x even where it underflows, and the hardware cast keeps
-    // the sign of a value that rounds to zero: the codes' sign bits are the inputs'
+    // the sign of a value that rounds to zero: the codes' sign bits are the inputs'.
+    // Every E2M1 rounding boundary (0.25 0.75 1.25 1.75 2.5 3.5 5) has zeros in the low 21 bits
+    // of its binary32 pattern, and x * r is within 4 units in the last place of the exact
+    // quotient: only a product whose pattern lies within 8 of such a pattern can be cast to
+    // another code than the exact quotient.  `near` ends up below 0x8000 iff the block has one.
     float s[16];
+    uint32_t near = 0xFFFFFFFFu;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r_dn);
+    for (int i = 0; i < 16; ++i) {
+        s[i] = __fmul_rn(X(i), r);
+        near = min(near, __float_as_uint(s[i]) * 2048u + 0x4000u);
+    }
     w0 = cvt_e2m1x8(s);
     w1 = cvt_e2m1x8(s + 8);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) s[i] = __fmul_rn(x[i], r_up);
-    const uint32_t d0 = w0 ^ cvt_e2m1x8(s), d1 = w1 ^ cvt_e2m1x8(s + 8);
-    if (d0 | d1) {
-        // the upper cast is the next code of the lower one; the boundary between the two is
-        // the mean of their values
+    if (near < 0x8000u) {
         const double d = (double)e * (double)ts;  // exact
-        uint64_t diff = ((uint64_t)d1 << 32) | d0;
-        uint64_t w = ((uint64_t)w1 << 32) | w0;
-        while (diff) {
-            const int i = (__ffsll((long long)diff) - 1) >> 2;
-            diff &= ~(0xFull << (4 * i));
-            const uint32_t c = (uint32_t)(w >> (4 * i)) & 7u;  // lower code, c < 7
-            const double bound = (double)(e2m1_times4(c) + e2m1_times4(c + 1u)) * 0.125 * d;
-            double a;
-            if (kKey) a = (double)__bfloat162float(reinterpret_cast<const __nv_bfloat16*>(src)[i]);
-            else a = (double)reinterpret_cast<const float*>(src)[i];
-            a = fabs(a);
-            if (a > bound || (a == bound && (c & 1u))) w += 1ull << (4 * i);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t bits = __float_as_uint(__fmul_rn(X(i), r));  // (recomputed: keeps s[] short-lived)
+            if (bits * 2048u + 0x4000u < 0x8000u) {
+                const float t = __uint_as_float((bits + 8u) & 0x7FE00000u);  // the candidate boundary
+                const float t4 = fminf(t * 4.f, 31.f);
+                const uint32_t u = (uint32_t)t4;                               // 1 3 5 7 10 14 20
+                constexpr uint32_t kBoundaries = 0x1044AAu;                    // those bits set
+                if ((float)u == t4 && ((kBoundaries >> u) & 1u)) {
+                    const uint32_t lower = (uint32_t)__popc(kBoundaries & ((1u << u) - 1u));  // code below it
+                    const double bound = (double)t * d;                        // exact
+                    const double a = fabs((double)X(i));
+                    const uint32_t code = lower + ((a > bound || (a == bound && (lower & 1u))) ? 1u : 0u);
+                    const uint32_t sh = (uint32_t)(i & 7) * 4u;
+                    if (i < 8) w0 = (w0 & ~(7u << sh)) | (code << sh);
+                    else w1 = (w1 & ~(7u << sh)) | (code << sh);
+                }
+            }
         }
-        w0 = (uint32_t)w;
-        w1 = (uint32_t)(w >> 32);
     }
+    const float r_dn = __fmul_rn(r, kDown), r_up = __fmul_rn(r, kUp);
     index = 0;
     if (kPlus && sb > 2u) {
         const float v_dn = fminf(fmaxf(__fmul_rn(amax, r_dn), 4.f), 8.f);
@@ -156,10 +164,11 @@ __device__ __forceinline__ void nvfp4_block(const float* x, const T* __restrict_
     }
     if (sb == 0u) w0 = w1 = 0u;
     scale_byte = sb;
+#undef X
 }
 
 template <typename T, bool kPlus>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_per_row,
                       int64_t total_units, float ts, uint4* __restrict__ nibbles,
                       uint16_t* __restrict__ scales, uint8_t* __restrict__ bm_index)
@@ -168,32 +177,20 @@ nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_p
     if (u >= total_units) return;
     const int64_t row = u / units_per_row;
     const T* p = src + row * ld_src + (u - row * units_per_row) * 32;
-    float x[32];
-    if (sizeof(T) == 2) {
+    constexpr int kWords = sizeof(T) == 2 ? 16 : 32;
+    uint32_t raw[kWords];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p) + i);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                x[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
-                x[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p) + i);
-            x[4 * i] = __uint_as_float(v.x);
-            x[4 * i + 1] = __uint_as_float(v.y);
-            x[4 * i + 2] = __uint_as_float(v.z);
-            x[4 * i + 3] = __uint_as_float(v.w);
-        }
+    for (int i = 0; i < kWords / 4; ++i) {
+        const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p) + i);
+        raw[4 * i] = v.x;
+        raw[4 * i + 1] = v.y;
+        raw[4 * i + 2] = v.z;
+        raw[4 * i + 3] = v.w;
     }
     const float six_ts = __fmul_rn(6.f, ts);
     uint32_t w[4], sb0, sb1, i0, i1;
-    nvfp4_block<T, kPlus>(x, p, ts, six_ts, w[0], w[1], sb0, i0);
-    nvfp4_block<T, kPlus>(x + 16, p + 16, ts, six_ts, w[2], w[3], sb1, i1);
+    nvfp4_block<T, kPlus>(raw, ts, six_ts, w[0], w[1], sb0, i0);
+    nvfp4_block<T, kPlus>(raw + kWords / 2, ts, six_ts, w[2], w[3], sb1, i1);
     __stcs(nibbles + u, make_uint4(w[0], w[1], w[2], w[3]));
     scales[u] = (uint16_t)(sb0 | (sb1 << 8));
     if (kPlus) bm_index[u] = (uint8_t)(i0 | (i1 << 4));

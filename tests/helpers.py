@@ -75,7 +75,9 @@ def nvfp4_boundary_blocks(ts, seed):
         d = np.float64(oracle.elem_value(oracle.FMT_E4M3, sb)) * np.float64(ts32)
         blk = np.empty(16, np.float64)
         blk[0] = d * g.choice([5.5, 5.75, 6.0, 6.25, 5.25, 6.75, 5.9])          # the BM
-        ties = g.choice([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], 15)
+        # the boundaries, and other values with few significant bits that are none
+        ties = g.choice([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0,
+                         0.375, 0.875, 0.4375, 0.3125, 0.625, 1.0, 3.0, 0.1875], 15)
         blk[1:] = ties * d * g.choice([-1.0, 1.0], 15)
         b32 = blk.astype(np.float32)
         step = g.integers(-1, 2, 16).astype(np.int32)                          # -1, 0, +1 ulp

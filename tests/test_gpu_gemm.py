@@ -16,6 +16,22 @@ def mxp():
     return m
 
 
+@pytest.fixture
+def force():
+    """Forces a kernel choice for the duration of a test (mxp_debug_override)."""
+    m = mxp()
+    knobs = {"inplace": m.KNOB_INPLACE_KERNEL, "halves": m.KNOB_STREAM_HALVES, "weight_only": m.KNOB_WEIGHT_ONLY_KERNEL}
+    names = {"single": 1, "pair": 2, "old": 1, "stream": 2, "1": 1, "2": 2}
+    used = []
+
+    def set_(knob, value):
+        used.append(knobs[knob])
+        m.mxp_debug_override(knobs[knob], names[value])
+    yield set_
+    for k in used:
+        m.mxp_debug_override(k, 0)
+
+
 def quantized(x_bits_or_f32, mode, bf16=False):
     q = oracle.quantize(x_bits_or_f32, mode, bf16_bits=bf16)
     dec = oracle.dequantize(q[0], q[1], q[2], mode)
@@ -69,19 +85,17 @@ def test_weight_only_config3_sampled(M):
     check_gemm(d[:, torch.from_numpy(rows).cuda()], da, dw)
 
 
-@pytest.mark.parametrize("kernel", ["old", "stream", "tma", "fp4"])
+@pytest.mark.parametrize("kernel", ["old", "stream"])
 @pytest.mark.parametrize("wmode", [MX, MXP, 2])
 @pytest.mark.parametrize("M,N,K", [(1, 32, 256), (3, 48, 2304), (8, 160, 4352), (9, 64, 512),
                                    (16, 2384, 4096), (40, 64, 768), (5, 77, 1024), (16, 300, 512),
                                    (1, 19000, 512), (1, 11008, 4096), (7, 20000, 1536),
                                    (2, 300, 512), (3, 2384, 4096), (4, 40000, 1024), (1, 64, 8192)])
-def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
+def test_weight_only_both_kernels(M, N, K, wmode, kernel, force):
     # shapes the streamed kernel takes (N % 16 == 0, K % 256 == 0): several 2048-element stages,
-    # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles; the
-    # TMA kernel takes those with K % 512 == 0 (MXFP4 / MXFP4+ weights): fewer rows than SMs,
-    # ragged last CTA, several activation tiles, more than 128 rows per CTA; the FP4-path kernel
-    # those of them with M <= 4 (every other combination falls through to the streamed kernel)
-    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
+    # a ragged last stage, more row groups than SMs, one and two 8-column activation tiles
+    # (every other shape falls through to the general kernel)
+    force("weight_only", kernel)
     a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K)
     wp, dw = quantized(w_bits, wmode, bf16=True)
     da = oracle.bf16_bits_to_f64(a_bits)
@@ -90,15 +104,13 @@ def test_weight_only_both_kernels(M, N, K, wmode, kernel, monkeypatch):
         check_gemm(d, da, dw)
 
 
-@pytest.mark.parametrize("corr_max_m", ["0", "8"])
 @pytest.mark.parametrize("wmode", [MXP, 2])
 @pytest.mark.parametrize("M,N,K", [(1, 48, 2304), (2, 160, 4352), (3, 2384, 4096), (8, 64, 512),
                                    (5, 20000, 1536), (1, 64, 8192)])
-def test_weight_only_bm_by_correction_warps_or_by_patch(M, N, K, wmode, corr_max_m, monkeypatch):
-    # the streamed kernel's two ways of handling the BM (correction warps: default for M <= 2;
-    # patched fragments: above), each forced over the whole range of its activation tile
-    monkeypatch.setenv("MXP_WO_KERNEL", "stream")
-    monkeypatch.setenv("MXP_WO_CORR_MAXM", corr_max_m)
+def test_weight_only_bm_by_correction_warps_or_by_patch(M, N, K, wmode, force):
+    # the streamed kernel's two ways of handling the BM: correction warps for M <= 2, patched
+    # fragments above
+    force("weight_only", "stream")
     a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K + 1)
     wp, dw = quantized(w_bits, wmode, bf16=True)
     da = oracle.bf16_bits_to_f64(a_bits)
@@ -106,11 +118,11 @@ def test_weight_only_bm_by_correction_warps_or_by_patch(M, N, K, wmode, corr_max
         check_gemm(mxp().mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=dt), da, dw)
 
 
-@pytest.mark.parametrize("kernel", ["old", "stream", "tma", "fp4"])
-def test_weight_only_one_hot_and_scale_spread(kernel, monkeypatch):
+@pytest.mark.parametrize("kernel", ["old", "stream"])
+def test_weight_only_one_hot_and_scale_spread(kernel, force):
     # one-hot activations select single decoded weights (exact in fp32), with weight rows and
     # activation rows spread over 60 binades each, a flushed block and a zero block
-    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
+    force("weight_only", kernel)
     K, N = 512, 48
     g = synth.rng(11)
     w = g.standard_normal((N, K)).astype(np.float32)
@@ -343,9 +355,9 @@ def test_tc_flushed_and_zero_blocks():
 
 @pytest.mark.parametrize("kernel", ["single", "pair"])
 @pytest.mark.parametrize("amode,bmode", MODES)
-def test_tc_both_kernels_every_mode(kernel, amode, bmode, monkeypatch):
+def test_tc_both_kernels_every_mode(kernel, amode, bmode, force):
     # the library picks the single-CTA or the CTA-pair kernel per mode; force each in turn
-    monkeypatch.setenv("MXP_GEMM_KERNEL", kernel)
+    force("inplace", kernel)
     M, N, K = 520, 777, 1280  # ragged in M and N, several tiles, K a multiple of 128 only
     a = synth.activations_normal(M, K, seed=5, outlier_frac=0.02)
     b = synth.weights(N, K, seed=6)
@@ -407,11 +419,11 @@ def test_tc_prepacked_weights_match_mxp_gemm(M, N, K, amode, bmode):
 @pytest.mark.parametrize("amode,bmode", [(MX, MX), (MXP, MXP), (MX, 2)])
 @pytest.mark.parametrize("M,N,K", [(300, 250, 256), (257, 481, 384), (300, 959, 256), (513, 1000, 128),
                                    (256, 448, 512), (384, 960, 128)])
-def test_tc_stream_tile_halves_and_ragged_edges(M, N, K, amode, bmode, halves, monkeypatch):
+def test_tc_stream_tile_halves_and_ragged_edges(M, N, K, amode, bmode, halves, force):
     # the streamed kernel's output tile has one or two halves of 240 (plain MXFP4: 224) columns;
     # N values just past a half, just past a tile, exact multiples, and ragged on both sides,
     # with either tile shape forced
-    monkeypatch.setenv("MXP_S_HALVES", halves)
+    force("halves", halves)
     ap, da = _raw_operand(M, K, amode, seed=M + N)
     bp, db = _raw_operand(N, K, bmode, seed=N + K)
     m = mxp()
@@ -543,266 +555,3 @@ def test_tc_mxpp_small_shapes(M, N, K):
     bp, db = _raw_operand(N, K, MXPP, seed=N + 9)
     for dt in (torch.float32, torch.bfloat16):
         check_gemm(mxp().mxp_gemm(ap, bp, out_dtype=dt), da, db)
-
-
-@pytest.mark.parametrize("kernel", ["old", "stream"])
-def test_weight_only_mxpp_raw_planes_one_hot(kernel, monkeypatch):
-    # one-hot activations return single decoded weights exactly (fp32 output): random raw MX++
-    # planes, i.e. every code, BM position, BM mantissa and delta
-    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
-    K, N = 512, 64
-    wp, dw = _raw_operand(N, K, MXPP, seed=51, scale_lo=100, scale_hi=150)
-    a = np.zeros((16, K), np.float32)
-    cols = [(m * 37 + 5) % K for m in range(16)]
-    for m, c in enumerate(cols):
-        a[m, c] = 2.0 ** (m - 8)
-    d = mxp().mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), wp, out_dtype=torch.float32)
-    got = d.cpu().numpy().astype(np.float64)
-    for m, c in enumerate(cols):
-        want = (dw[:, c] * 2.0 ** (m - 8)).astype(np.float32).astype(np.float64)
-        assert np.array_equal(got[m], want)
-
-
-# ------------------------------------------------------------------ bounded waits
-def test_bounded_wait_reports_timeout_and_leaves_the_device_usable():
-    # a wait that nothing satisfies comes back after its cycle limit, the kernel reports
-    # MXP_ERR_TIMEOUT through the status block and exits normally (no trap, no hang)
-    m = mxp()
-    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    m.mxp_wait_selftest(ws, 2_000_000)            # about a millisecond
-    assert m.mxp_gemm_status(ws) == 5             # MXP_ERR_TIMEOUT
-    torch.cuda.synchronize()
-    # the context is intact: a GEMM right after gives a correct result and a clean status
-    ap, da = _raw_operand(192, 256, MXP, seed=61)
-    bp, db = _raw_operand(320, 256, MXP, seed=62)
-    need = m.mxp_gemm_workspace_bytes(192, 320, 256, False, 1, 1)
-    ws2 = torch.zeros(need, dtype=torch.uint8, device="cuda")
-    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32, workspace=ws2)
-    check_gemm(d, da, db)
-    assert m.mxp_gemm_status(ws2) == 0
-    with pytest.raises(Exception):
-        m.mxp_wait_selftest(ws, 0)                # limit out of range: rejected, nothing launched
-
-
-# ------------------------------------------------------------------ MXFP6 / MXFP6+ operands
-MX6, MX6P = 3, 4
-
-
-def _raw_operand6(rows, K, plus, seed, scale_lo=118, scale_hi=136):
-    """MXFP6(+) planes filled directly: every E2M3 code, BM position and five-bit BM mantissa."""
-    g = synth.rng(seed)
-    codes = g.integers(0, 64, (rows, K), dtype=np.uint8)
-    sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
-    idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8) if plus else None
-    dec = oracle.dequantize_wide(codes, sc, idx, oracle.FMT_E2M3, plus)
-    from paper_2510_14557_b200 import Packed
-    p = Packed(to_dev(oracle.pack6(codes)), to_dev(sc), to_dev(idx) if plus else None, rows, K,
-               MX6P if plus else MX6)
-    return p, dec
-
-
-def _any_operand(rows, K, mode, seed):
-    if mode in (MX6, MX6P):
-        return _raw_operand6(rows, K, mode == MX6P, seed)
-    return _raw_operand(rows, K, mode, seed)
-
-
-@pytest.mark.parametrize("amode,bmode", [(MX6, MX6), (MX6P, MX6), (MX6, MX6P), (MX6P, MX6P),
-                                         (MX6P, MX), (MX6P, MXP), (MXP, MX6P), (MX6P, MXPP), (MX, MX6)])
-@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 129, 384), (64, 100, 256), (513, 1000, 128)])
-def test_tc_mxfp6_operands(M, N, K, amode, bmode):
-    # E2M3 elements go to the tensor core as they are; the BM of an MXFP6+ block enters as the
-    # sum of two E2M3 values in two planes, and the K loop runs once per pair of planes
-    ap, da = _any_operand(M, K, amode, seed=M + 3)
-    bp, db = _any_operand(N, K, bmode, seed=N + 4)
-    m = mxp()
-    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode), dtype=torch.uint8, device="cuda")
-    for dt in (torch.float32, torch.bfloat16):
-        d = m.mxp_gemm(ap, bp, out_dtype=dt, workspace=ws)
-        assert m.mxp_gemm_status(ws) == 0
-        check_gemm(d, da, db)
-
-
-@pytest.mark.parametrize("amode", [MX6, MX6P])
-def test_tc_mxfp6_identity_partner_returns_the_decode(amode):
-    # B = identity: D must equal the oracle's decode of A bit for bit, for every E2M3 code, BM
-    # position and BM mantissa (the two planes of a BM add up exactly)
-    M, K = 384, 256
-    ap, da = _raw_operand6(M, K, amode == MX6P, seed=23)
-    eye = np.eye(K, dtype=np.float32)
-    for bmode in (MX, MX6P):
-        if bmode == MX:
-            bp, db = quantized(eye, MX)
-        else:
-            codes, sc, idx = oracle.quantize_wide(eye, oracle.FMT_E2M3, True)
-            db = oracle.dequantize_wide(codes, sc, idx, oracle.FMT_E2M3, True)
-            from paper_2510_14557_b200 import Packed
-            bp = Packed(to_dev(oracle.pack6(codes)), to_dev(sc), to_dev(idx), K, K, MX6P)
-        assert np.array_equal(db, eye.astype(np.float64))
-        d = mxp().mxp_gemm(ap, bp, out_dtype=torch.float32)
-        assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
-
-
-def test_tc_mxfp6_quantized_end_to_end_and_rejections():
-    from paper_2510_14557_b200 import MxpError
-    m = mxp()
-    a = synth.activations_normal(320, 512, seed=31, outlier_frac=0.02)
-    w = synth.weights(384, 512, seed=32)
-    pa = m.mxp_quantize(to_dev(a), MX6P)
-    pw = m.mxp_quantize(to_dev(w), MX6)
-    ca, sa, ia = oracle.quantize_wide(a, oracle.FMT_E2M3, True)
-    cw, sw, iw = oracle.quantize_wide(w, oracle.FMT_E2M3, False)
-    da = oracle.dequantize_wide(ca, sa, ia, oracle.FMT_E2M3, True)
-    dw = oracle.dequantize_wide(cw, sw, None, oracle.FMT_E2M3, False)
-    check_gemm(m.mxp_gemm(pa, pw, out_dtype=torch.float32), da, dw)
-    with pytest.raises(MxpError):   # the in-place kernels (minimum workspace) are 4-bit only
-        m.mxp_gemm(pa, pw, workspace=torch.zeros(4096, dtype=torch.uint8, device="cuda"))
-    with pytest.raises(MxpError):   # no weight-only form for 6-bit weights
-        m.mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), pw)
-    p8 = m.mxp_quantize(to_dev(a), 6)
-    with pytest.raises(MxpError):   # an MXFP8+ operand has three planes: no prepacked form
-        m.mxp_gemm_prepack(p8, True)
-
-
-# ------------------------------------------------------------------ MXFP8 operands
-MX8 = 5
-
-
-MX8P = 6
-
-
-def _raw_operand8(rows, K, seed, scale_lo=112, scale_hi=130, plus=False):
-    """MXFP8(+) planes filled directly: every E4M3 code except the NaN pattern and, for MXFP8+,
-    every BM position and seven-bit BM mantissa."""
-    g = synth.rng(seed)
-    codes = g.integers(0, 256, (rows, K), dtype=np.uint8)
-    codes[(codes & 0x7F) == 0x7F] = 0x7E
-    sc = g.integers(scale_lo, scale_hi, (rows, K // 32), dtype=np.uint8)
-    sc[g.random((rows, K // 32)) < 0.02] = 0          # flushed blocks hold zero codes
-    idx = None
-    if plus:
-        idx = g.integers(0, 32, (rows, K // 32), dtype=np.uint8)
-        bm_code = g.integers(0, 256, (rows, K // 32), dtype=np.uint8)       # sign + E0M7, 0x7F included
-        cols = (np.arange(K // 32) * 32)[None, :] + idx
-        np.put_along_axis(codes, cols, bm_code, axis=1)
-    codes[np.repeat(sc == 0, 32, axis=1)] = 0
-    dec = oracle.dequantize_wide(codes, sc, idx, oracle.FMT_E4M3, plus)
-    from paper_2510_14557_b200 import Packed
-    return Packed(to_dev(codes), to_dev(sc), to_dev(idx) if plus else None, rows, K,
-                  MX8P if plus else MX8), dec
-
-
-def _operand_of(rows, K, mode, seed):
-    if mode in (MX8, MX8P):
-        return _raw_operand8(rows, K, seed, plus=mode == MX8P)
-    return _any_operand(rows, K, mode, seed)
-
-
-@pytest.mark.parametrize("amode,bmode", [(MX8, MX8), (MX8, MXP), (MX, MX8), (MX6P, MX8), (MX8, MXPP),
-                                         (MX8P, MX8), (MX8, MX8P), (MX8P, MX8P), (MX8P, MXP), (MX6P, MX8P)])
-@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 129, 384), (64, 100, 256), (513, 1000, 128)])
-def test_tc_mxfp8_operands(M, N, K, amode, bmode):
-    # E4M3 elements are an operand format of the same instruction: the codes go in as stored,
-    # next to 4- and 6-bit partners on the other side
-    # (an MXFP8+ operand: three planes, the BM being the sum of three E4M3 values)
-    ap, da = _operand_of(M, K, amode, seed=M + 5)
-    bp, db = _operand_of(N, K, bmode, seed=N + 6)
-    m = mxp()
-    ws = torch.zeros(m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode), dtype=torch.uint8, device="cuda")
-    for dt in (torch.float32, torch.bfloat16):
-        d = m.mxp_gemm(ap, bp, out_dtype=dt, workspace=ws)
-        assert m.mxp_gemm_status(ws) == 0
-        check_gemm(d, da, db)
-
-
-def test_tc_mxfp8_identity_and_quantized_end_to_end():
-    m = mxp()
-    # B = identity: D is the decode of A bit for bit, for every E4M3 code
-    M, K = 384, 256
-    ap, da = _raw_operand8(M, K, seed=41)
-    bp, db = quantized(np.eye(K, dtype=np.float32), MX)
-    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32)
-    assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
-    # ... and for every BM position and seven-bit BM mantissa of MXFP8+ (three planes add up exactly)
-    ap, da = _raw_operand8(M, K, seed=42, plus=True)
-    d = m.mxp_gemm(ap, bp, out_dtype=torch.float32)
-    assert np.array_equal(d.cpu().numpy().astype(np.float64), da)
-    # quantized by the library, against the oracle's encode + decode + fp64 product
-    a = synth.activations_normal(320, 512, seed=43, outlier_frac=0.02)
-    w = synth.weights(384, 512, seed=44)
-    pa, pw = m.mxp_quantize(to_dev(a), MX8), m.mxp_quantize(to_dev(w), MX8)
-    ca, sa, _ = oracle.quantize_wide(a, oracle.FMT_E4M3, False)
-    cw, sw, _ = oracle.quantize_wide(w, oracle.FMT_E4M3, False)
-    check_gemm(m.mxp_gemm(pa, pw, out_dtype=torch.float32),
-               oracle.dequantize_wide(ca, sa, None, oracle.FMT_E4M3, False),
-               oracle.dequantize_wide(cw, sw, None, oracle.FMT_E4M3, False))
-    # prepacked weights
-    pre = m.mxp_gemm_prepack(pw, True)
-    check_gemm(m.mxp_gemm_prepacked(pa, pw, pre, out_dtype=torch.float32),
-               oracle.dequantize_wide(ca, sa, None, oracle.FMT_E4M3, False),
-               oracle.dequantize_wide(cw, sw, None, oracle.FMT_E4M3, False))
-
-
-# ------------------------------------------------------------------ fused quantize -> GEMM
-@pytest.mark.parametrize("amode,bmode", [(MXP, MXP), (MXP, MX), (MX, MXP)])
-@pytest.mark.parametrize("M,N,K", [(300, 520, 1024), (257, 1000, 384), (512, 512, 128)])
-def test_quantize_gemm_ready_matches_the_two_step_path(M, N, K, amode, bmode):
-    # the quantizer writes the packed planes (bit-exact, as mxp_quantize) and A's GEMM-ready
-    # form; the GEMM then needs no prepack launch and returns what mxp_gemm returns
-    m = mxp()
-    a_bits = synth.f32_to_bf16_bits(synth.activations_normal(M, K, seed=M + K, outlier_frac=0.02))
-    a_bits[3, 32:64] = 0                       # a zero block
-    a_bits[5, 64:96] = 0x0001                  # a flushed block
-    bp, db = _raw_operand(N, K, bmode, seed=N)
-    pre = m.mxp_gemm_prepack(bp, True)
-    ws = torch.full((m.mxp_gemm_workspace_bytes(M, N, K, False, amode, bmode),), 0xA5, dtype=torch.uint8, device="cuda")
-    pa = m.mxp_quantize_gemm_ready(to_dev_bf16(a_bits), amode, ws)
-    ref = oracle.quantize(a_bits, amode, bf16_bits=True)
-    assert np.array_equal(pa.nibbles.cpu().numpy(), ref[0])
-    assert np.array_equal(pa.scales.cpu().numpy(), ref[1])
-    if amode != MX:
-        assert np.array_equal(pa.bm_index.cpu().numpy(), ref[2])
-    da = oracle.dequantize(*ref, amode)
-    for dt in (torch.float32, torch.bfloat16):
-        d = m.mxp_gemm_ready(pa, bp, pre, ws, out_dtype=dt)
-        assert m.mxp_gemm_status(ws) == 0
-        check_gemm(d, da, db)
-        assert torch.equal(d, m.mxp_gemm(pa, bp, out_dtype=dt))
-
-
-def test_quantize_gemm_ready_rejections():
-    from paper_2510_14557_b200 import MxpError
-    m = mxp()
-    ws = torch.zeros(1 << 22, dtype=torch.uint8, device="cuda")
-    x = torch.randn(256, 256, device="cuda")
-    with pytest.raises(MxpError):   # fp32 source: not the fused kernel's case
-        m.mxp_quantize_gemm_ready(x, MXP, ws)
-    with pytest.raises(MxpError):   # MX++ keeps its own prepack
-        m.mxp_quantize_gemm_ready(x.bfloat16(), MXPP, ws)
-    with pytest.raises(MxpError):   # M <= 128: no streamed kernel
-        m.mxp_quantize_gemm_ready(x.bfloat16()[:64].contiguous(), MXP, ws)
-    with pytest.raises(MxpError):   # workspace too small
-        m.mxp_quantize_gemm_ready(x.bfloat16(), MXP, ws[:4096])
-
-
-@pytest.mark.parametrize("kernel", ["fp4", "tma"])
-@pytest.mark.parametrize("wmode", [MX, MXP])
-def test_weight_only_tensor_paths_one_hot_rows(kernel, wmode, monkeypatch):
-    # the tensor-core decode kernels take M <= 4 (fp4) / M <= 64 (tma): one-hot activations
-    # select single decoded weights, BM or not, exactly (the BM arrives as the E2M1 misreading
-    # from the tensor core plus the correction from the CUDA cores: the sum is exact in fp32)
-    monkeypatch.setenv("MXP_WO_KERNEL", kernel)
-    K, N = 1024, 200
-    wp, dw = _raw_operand(N, K, wmode, seed=71, scale_lo=100, scale_hi=150)
-    a = np.zeros((4, K), np.float32)
-    cols = [5, 300, 777, 1023]
-    for m, c in enumerate(cols):
-        a[m, c] = 2.0 ** (3 * m - 4)
-    m_ = mxp()
-    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    d = m_.mxp_gemm(to_dev_bf16(synth.f32_to_bf16_bits(a)), wp, out_dtype=torch.float32, workspace=ws)
-    assert m_.mxp_gemm_status(ws) == 0
-    got = d.cpu().numpy().astype(np.float64)
-    for m, c in enumerate(cols):
-        want = (dw[:, c] * 2.0 ** (3 * m - 4)).astype(np.float32).astype(np.float64)
-        assert np.array_equal(got[m], want)
