@@ -187,7 +187,12 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  *     maximum are rounded at 2^-17 of that maximum; with less workspace a slower
  *     general kernel answers);
  *   - A_packed (host pointer to a descriptor): both operands are consumed by the
- *     block-scaled tensor-core path; any combination of MXFP4 / MXFP4+ modes.
+ *     block-scaled tensor-core path; any combination of MXFP4 / MXFP4+ modes.  With the full
+ *     workspace: MXFP4 x MXFP4 runs FP4 instructions on the stored planes; one MXFP4+ operand
+ *     against an MXFP4 one runs the same main pass with every BM replaced by its upper part
+ *     BM_H plus Eq. 4's residual (BM_L) as a sparse tensor-core instruction (Sec. 5.2,
+ *     Algorithm 1: "sparse MMA"), 1.5 times the plain MXFP4 tensor work; two MXFP4+ operands
+ *     run one pass on 6-bit codes that hold the decoded values of Eq. 3 exactly, 2 times.
  *   B_packed   host pointer to the descriptor of the N x K weight operand
  *   D          M x N of `d_dt` (bf16 rounded to nearest even, or fp32), row stride ldd
  *              elements (ldd >= N; 16-byte aligned rows let the epilogue use wide stores)
@@ -219,22 +224,31 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
 
 /*
  * Weights prepared once.  mxp_gemm with the full workspace re-tiles the scales of both
- * operands and, when either is MXFP4+, widens both to E2M3 / E4M3 codes on every call (see
- * `workspace` above).  For an operand that does not change between calls (the N x K
- * weights) that work can be done once:
- *   mxp_gemm_prepack_bytes  bytes of the prepacked form of a rows x K operand; `wide` != 0
- *                           if the GEMMs it will be used in have an MXFP4+ operand on
- *                           either side (then it holds 16 bytes per 16 elements: E2M3 codes
- *                           or, for MX++, E4M3 bytes, exact for every E2M1 value and for
- *                           the BM values of Eq. 3), 0 for
- *                           MXFP4 x MXFP4 (scale atoms only).  0: shape not supported
- *                           (K % 128 != 0).
+ * operands and prepares the MX+ ones (split per Eq. 4, or widened to E2M3 / E4M3 codes) on
+ * every call (see `workspace` above).  For an operand that does not change between calls (the
+ * N x K weights) that work can be done once.  Which form a GEMM reads depends on both
+ * operands' modes; mxp_gemm_prepack_form tells:
+ *   MXP_PREPACK_PLAIN  scale atoms only: B is MXFP4 and A is MXFP4 or MXFP4+
+ *   MXP_PREPACK_WIDE   16 bytes per 16 elements (E2M3 codes or, for MX++ and MXFP8, E4M3
+ *                      bytes: exact for every E2M1 value and for the BM values of Eq. 3):
+ *                      both operands MX+, the wider modes, and the weight-only tensor-core path
+ *   MXP_PREPACK_SPLIT  B is MXFP4+ and A is MXFP4: Eq. 4's split for the sparse residual
+ *                      instruction -- B's nibble plane with BM_H in every BM's place, BM_L
+ *                      compressed 2:1, and the metadata that says where each BM_L sits
+ *   mxp_gemm_prepack_form   the form (an mxp_prepack_form) of B's copy that mxp_gemm_prepacked
+ *                           reads for these two modes
+ *   mxp_gemm_prepack_bytes  bytes of that form of a rows x K operand.  0: shape or form not
+ *                           supported (K % 128 != 0).
  *   mxp_gemm_prepack        writes that form of `P` into `out` (device, 256-byte aligned,
  *                           `out_bytes` >= the size above).  Asynchronous on `cuda_stream`.
  *   mxp_gemm_prepacked      mxp_gemm's packed-operand form with B's prepacked copy:
- *                           `B_prepacked` must come from mxp_gemm_prepack(B_packed, wide)
- *                           with wide == (A is MXFP4+ or B is MXFP4+); B_packed still
- *                           describes the operand (planes, shape, mode).  Needs M > 128 and
+ *                           `B_prepacked` must come from mxp_gemm_prepack(B_packed, form) with
+ *                           form == mxp_gemm_prepack_form(A's mode, B's mode), and
+ *                           `B_prepacked_bytes` must be mxp_gemm_prepack_bytes(N, K, form): the
+ *                           call checks that before any launch (MXP_ERR_INVALID_ARG), so a copy
+ *                           made for another shape or another pairing of modes is refused
+ *                           instead of being read past its end.  B_packed still describes the
+ *                           operand (planes, shape, mode).  Needs M > 128 and
  *                           N > 128 and mxp_gemm_workspace_bytes(...) of workspace
  *                           (MXP_ERR_UNSUPPORTED / MXP_ERR_WORKSPACE otherwise; fall back
  *                           to mxp_gemm).  Same result as mxp_gemm.
@@ -242,26 +256,28 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
  * an implementation device of this library.
  *   mxp_gemm_dense_prepacked  the weight-only form (bf16 activations, more than one tile's
  *                           worth of rows is where it pays: see mxp_gemm) with B's prepacked
- *                           copy, which must have been made with wide != 0.  Workspace
+ *                           copy in the form MXP_PREPACK_WIDE (size checked as above).  Workspace
  *                           (device, 256-byte aligned): at least
  *                           mxp_gemm_dense_prepacked_workspace_bytes(M, K) bytes (0: shape
  *                           not supported), which hold the activations' two planes and
  *                           scales.  Any M >= 1; 4-bit weight modes; K % 128 == 0.  Same
  *                           result as mxp_gemm's tensor-core weight-only path.
  */
-size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide);
-mxp_status mxp_gemm_prepack(const mxp_packed *P, int wide, void *out, size_t out_bytes,
+typedef enum { MXP_PREPACK_PLAIN = 0, MXP_PREPACK_WIDE = 1, MXP_PREPACK_SPLIT = 2 } mxp_prepack_form;
+int mxp_gemm_prepack_form(mxp_mode a_mode, mxp_mode b_mode);
+size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int form);
+mxp_status mxp_gemm_prepack(const mxp_packed *P, int form, void *out, size_t out_bytes,
                             void *cuda_stream);
 mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
-                              const mxp_packed *B_packed, const void *B_prepacked, void *D,
-                              mxp_dtype d_dt, int64_t ldd, void *workspace,
-                              size_t workspace_bytes, void *cuda_stream);
+                              const mxp_packed *B_packed, const void *B_prepacked,
+                              size_t B_prepacked_bytes, void *D, mxp_dtype d_dt, int64_t ldd,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 size_t mxp_gemm_dense_prepacked_workspace_bytes(int64_t M, int64_t K);
 mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void *A_dense_bf16,
                                     int64_t lda, const mxp_packed *B_packed,
-                                    const void *B_prepacked, void *D, mxp_dtype d_dt,
-                                    int64_t ldd, void *workspace, size_t workspace_bytes,
-                                    void *cuda_stream);
+                                    const void *B_prepacked, size_t B_prepacked_bytes, void *D,
+                                    mxp_dtype d_dt, int64_t ldd, void *workspace,
+                                    size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Quantization fused with the preparation of the GEMM operand (Sec. 5, software integration:
@@ -277,16 +293,17 @@ mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void 
  *                            K % 128 == 0.
  *   mxp_gemm_ready           mxp_gemm_prepacked for an A prepared that way in the same
  *                            `workspace` (nothing may have written to it in between) and a B
- *                            prepacked with wide != 0: one launch.  Same result as mxp_gemm.
+ *                            prepacked in the form MXP_PREPACK_WIDE (size checked as for
+ *                            mxp_gemm_prepacked): one launch.  Same result as mxp_gemm.
  */
 mxp_status mxp_quantize_gemm_ready(const void *src, mxp_dtype src_dt, int64_t M, int64_t K,
                                    int64_t ld_src, mxp_mode mode, uint8_t *nibbles,
                                    uint8_t *scales, uint8_t *bm_index, void *workspace,
                                    size_t workspace_bytes, void *cuda_stream);
 mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
-                          const mxp_packed *B_packed, const void *B_prepacked, void *D,
-                          mxp_dtype d_dt, int64_t ldd, void *workspace, size_t workspace_bytes,
-                          void *cuda_stream);
+                          const mxp_packed *B_packed, const void *B_prepacked,
+                          size_t B_prepacked_bytes, void *D, mxp_dtype d_dt, int64_t ldd,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * The weight-only form of mxp_gemm for a chain of decode GEMMs on one stream (Sec. 7.1:
@@ -398,8 +415,13 @@ mxp_status mxp_wait_selftest(void *workspace, size_t workspace_bytes, int64_t li
  *   kind 2: as kind 0 plus the three scale-factor copies (tcgen05.cp) a 128 x 256 tile needs
  *           per 128 elements of K, into one TMEM buffer
  *   kind 3: as kind 2 with the copies alternating between two TMEM buffers
- * `iters` counts groups of two instructions.
- * *flops receives the multiply-add work done (2 * M * N * K summed over CTAs).
+ *   kind 4: the sparse form (Sec. 5.2, "sparse MMA"): one tcgen05.mma.sp of 128 x 256 x 128
+ *           per group, A stored 2:1 compressed
+ *   kind 5: two dense instructions of kind 0 and one sparse one per group: the instruction mix
+ *           of a main pass plus a sparse residual pass over the same 128 elements of K
+ * `iters` counts groups (128 elements of K for the FP4 kinds, 64 for kind 1).
+ * *flops receives 2 * M * N * K of the groups summed over CTAs (for kind 5 the K of the main
+ * pass only: the residual instruction is overhead).
  * The paper has no counterpart; it exists so that fractions of peak have a measured
  * denominator on the device the library runs on.
  */
@@ -445,13 +467,17 @@ mxp_status mxp_gemm_noalloc(int64_t M, int64_t N, int64_t K, const mxp_packed *A
  *   MXP_KNOB_WEIGHT_ONLY_KERNEL  weight-only mxp_gemm: 1 = the general kernel, 2 = the streamed
  *                                decode kernel where it applies (either keeps M > 64 calls
  *                                away from the tensor-core path)
+ *   MXP_KNOB_ONE_SIDED           one MXFP4+ operand against an MXFP4 one: 1 = the single pass on
+ *                                widened codes instead of the sparse residual instruction (the
+ *                                prepacked form of B such calls read is then MXP_PREPACK_WIDE)
  * Returns MXP_ERR_INVALID_ARG for an unknown knob or a value outside 0..2.
  */
 typedef enum {
     MXP_KNOB_INPLACE_KERNEL = 0,
     MXP_KNOB_STREAM_HALVES = 1,
     MXP_KNOB_WEIGHT_ONLY_KERNEL = 2,
-    MXP_KNOB_COUNT_ = 3
+    MXP_KNOB_ONE_SIDED = 3,
+    MXP_KNOB_COUNT_ = 4
 } mxp_knob;
 mxp_status mxp_debug_override(int knob, int value);
 

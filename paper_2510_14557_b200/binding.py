@@ -26,7 +26,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
 EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_decode_prepack_bytes", "mxp_gemm_decode_workspace_bytes", "mxp_gemm_decode_prepack", "mxp_gemm_decode_prepacked", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
-           "mxp_gemm_prepack_bytes", "mxp_gemm_prepack", "mxp_gemm_prepacked",
+           "mxp_gemm_prepack_bytes", "mxp_gemm_prepack_form", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_gemm_dense_prepacked", "mxp_gemm_dense_prepacked_workspace_bytes",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
            "mxp_debug_override", "mxp_gemm_status", "mxp_gemm_clock_stamp", "mxp_wait_selftest", "mxp_tensor_peak_probe", "mxp_status_string", "mxp_version"]
@@ -67,7 +67,7 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_noalloc.restype = ci
         l.mxp_gemm_dense_prepacked_workspace_bytes.argtypes = [i64, i64]
         l.mxp_gemm_dense_prepacked_workspace_bytes.restype = sz
-        l.mxp_gemm_dense_prepacked.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, vp, ci,
+        l.mxp_gemm_dense_prepacked.argtypes = [i64, i64, i64, vp, i64, ctypes.POINTER(_Packed), vp, sz, vp, ci,
                                                i64, vp, sz, vp]
         l.mxp_gemm_dense_prepacked.restype = ci
         l.mxp_quantize_reordered.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp, vp, vp, vp]
@@ -97,8 +97,10 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_prepack_bytes.restype = sz
         l.mxp_gemm_prepack.argtypes = [ctypes.POINTER(_Packed), ci, vp, sz, vp]
         l.mxp_gemm_prepack.restype = ci
+        l.mxp_gemm_prepack_form.argtypes = [ci, ci]
+        l.mxp_gemm_prepack_form.restype = ci
         l.mxp_gemm_prepacked.argtypes = [i64, i64, i64, ctypes.POINTER(_Packed), ctypes.POINTER(_Packed),
-                                         vp, vp, ci, i64, vp, sz, vp]
+                                         vp, sz, vp, ci, i64, vp, sz, vp]
         l.mxp_gemm_prepacked.restype = ci
         l.mxp_gemm_ready.argtypes = l.mxp_gemm_prepacked.argtypes
         l.mxp_gemm_ready.restype = ci
@@ -290,9 +292,18 @@ def mxp_gemm(a, b: Packed, out_dtype=torch.bfloat16, out: Optional[torch.Tensor]
     return out
 
 
-def mxp_gemm_prepack(p: Packed, wide: bool, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """Prepacked copy of an operand (normally the weights) for mxp_gemm_prepacked.  `wide` must
-    be True when either operand of the later GEMMs is MXFP4+."""
+PREPACK_PLAIN, PREPACK_WIDE, PREPACK_SPLIT = 0, 1, 2
+
+
+def mxp_gemm_prepack_form(a_mode: int, b_mode: int) -> int:
+    """The form of B's prepacked copy that mxp_gemm_prepacked reads for these modes."""
+    return int(lib().mxp_gemm_prepack_form(a_mode, b_mode))
+
+
+def mxp_gemm_prepack(p: Packed, wide, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Prepacked copy of an operand (normally the weights) for mxp_gemm_prepacked.  `wide`: a
+    PREPACK_* form (True / False mean PREPACK_WIDE / PREPACK_PLAIN); take it from
+    mxp_gemm_prepack_form(a_mode, b_mode) of the GEMMs the copy is for."""
     need = int(lib().mxp_gemm_prepack_bytes(p.rows, p.cols, int(wide)))
     if need == 0:
         raise MxpError("mxp_gemm_prepack_bytes", 2)
@@ -316,7 +327,7 @@ def mxp_gemm_prepacked(a: Packed, b: Packed, b_prepacked: torch.Tensor, out_dtyp
                                 dtype=torch.uint8, device=b.nibbles.device)
     as_, bs = a.c_struct(), b.c_struct()
     st = lib().mxp_gemm_prepacked(M, N, K, ctypes.byref(as_), ctypes.byref(bs), b_prepacked.data_ptr(),
-                                  out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
+                                  b_prepacked.numel(), out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
                                   workspace.numel(), _stream())
     _check("mxp_gemm_prepacked", st)
     return out
@@ -345,7 +356,7 @@ def mxp_gemm_ready(a: Packed, b: Packed, b_prepacked: torch.Tensor, workspace: t
         out = torch.empty((M, N), dtype=out_dtype, device=b.nibbles.device)
     as_, bs = a.c_struct(), b.c_struct()
     st = lib().mxp_gemm_ready(M, N, K, ctypes.byref(as_), ctypes.byref(bs), b_prepacked.data_ptr(),
-                              out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
+                              b_prepacked.numel(), out.data_ptr(), _dt(out), out.stride(0), workspace.data_ptr(),
                               workspace.numel(), _stream())
     _check("mxp_gemm_ready", st)
     return out
@@ -436,14 +447,14 @@ def mxp_gemm_dense_prepacked(a: torch.Tensor, b: Packed, b_prepacked: torch.Tens
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=a.device)
     bs = b.c_struct()
     st = lib().mxp_gemm_dense_prepacked(M, N, K, a.data_ptr(), a.stride(0), ctypes.byref(bs),
-                                        b_prepacked.data_ptr(), out.data_ptr(), _dt(out),
+                                        b_prepacked.data_ptr(), b_prepacked.numel(), out.data_ptr(), _dt(out),
                                         out.stride(0), workspace.data_ptr(), workspace.numel(),
                                         _stream())
     _check("mxp_gemm_dense_prepacked", st)
     return out
 
 
-KNOB_INPLACE_KERNEL, KNOB_STREAM_HALVES, KNOB_WEIGHT_ONLY_KERNEL = 0, 1, 2
+KNOB_INPLACE_KERNEL, KNOB_STREAM_HALVES, KNOB_WEIGHT_ONLY_KERNEL, KNOB_ONE_SIDED = 0, 1, 2, 3
 
 
 def mxp_debug_override(knob: int, value: int) -> None:

@@ -347,24 +347,28 @@ mxp_status mxp_gemm_decode_prepacked(int64_t M, int64_t N, int64_t K, const void
                                       chained != 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
-size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int wide)
+size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int form)
 {
-    return mxp::stream_prepack_bytes(rows, K, wide != 0);
+    return mxp::stream_prepack_bytes(rows, K, form);
 }
 
-mxp_status mxp_gemm_prepack(const mxp_packed* P, int wide, void* out, size_t out_bytes,
+int mxp_gemm_prepack_form(mxp_mode a_mode, mxp_mode b_mode) { return mxp::stream_b_form(a_mode, b_mode); }
+
+mxp_status mxp_gemm_prepack(const mxp_packed* P, int form, void* out, size_t out_bytes,
                             void* cuda_stream)
 {
     if (!valid_packed(P, true)) return MXP_ERR_INVALID_ARG;
+    if (form < MXP_PREPACK_PLAIN || form > MXP_PREPACK_SPLIT) return MXP_ERR_INVALID_ARG;
     if (P->rows == 0 || P->cols == 0) return MXP_OK;
-    if (P->mode != MXP_MODE_MXFP4 && !wide) return MXP_ERR_INVALID_ARG;
-    return mxp::stream_prepack(*P, wide != 0, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
+    if (P->mode != MXP_MODE_MXFP4 && form == MXP_PREPACK_PLAIN) return MXP_ERR_INVALID_ARG;
+    if (P->mode != MXP_MODE_MXFP4_PLUS && form == MXP_PREPACK_SPLIT) return MXP_ERR_INVALID_ARG;
+    return mxp::stream_prepack(*P, form, out, out_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed* A_packed,
-                              const mxp_packed* B_packed, const void* B_prepacked, void* D,
-                              mxp_dtype d_dt, int64_t ldd, void* workspace,
-                              size_t workspace_bytes, void* cuda_stream)
+                              const mxp_packed* B_packed, const void* B_prepacked,
+                              size_t B_prepacked_bytes, void* D, mxp_dtype d_dt, int64_t ldd,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
@@ -378,6 +382,16 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
     if (!aligned(A_packed->scales, 4) || !aligned(B_packed->scales, 4)) return MXP_ERR_INVALID_ARG;
     if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)
         return MXP_ERR_UNSUPPORTED;
+    // the copy must be the one this pairing of modes reads, made for this shape: its size says so
+    const int form = mxp::stream_b_form(A_packed->mode, B_packed->mode);
+    const size_t want = mxp::stream_prepack_bytes(N, K, form);
+    if (want == 0) return MXP_ERR_UNSUPPORTED;
+    if (B_prepacked_bytes != want || !aligned(B_prepacked, 256)) return MXP_ERR_INVALID_ARG;
+    if (form != MXP_PREPACK_WIDE &&
+        mxp::stream_sparse_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode, true) != 0)
+        return mxp::launch_gemm_tc_sparse(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
+                                          workspace, workspace_bytes,
+                                          static_cast<cudaStream_t>(cuda_stream));
     return mxp::launch_gemm_tc_stream(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
                                       workspace, workspace_bytes,
                                       static_cast<cudaStream_t>(cuda_stream));
@@ -390,8 +404,9 @@ size_t mxp_gemm_dense_prepacked_workspace_bytes(int64_t M, int64_t K)
 
 mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16,
                                     int64_t lda, const mxp_packed* B_packed,
-                                    const void* B_prepacked, void* D, mxp_dtype d_dt, int64_t ldd,
-                                    void* workspace, size_t workspace_bytes, void* cuda_stream)
+                                    const void* B_prepacked, size_t B_prepacked_bytes, void* D,
+                                    mxp_dtype d_dt, int64_t ldd, void* workspace,
+                                    size_t workspace_bytes, void* cuda_stream)
 {
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt) || A_dense_bf16 == nullptr) return MXP_ERR_INVALID_ARG;
@@ -402,7 +417,9 @@ mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void*
     if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     const size_t need = mxp::stream_dense_prepacked_workspace_bytes(M, K);
-    if (need == 0 || mxp::stream_prepack_bytes(N, K, true) == 0) return MXP_ERR_UNSUPPORTED;
+    if (need == 0 || mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) == 0) return MXP_ERR_UNSUPPORTED;
+    if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) || !aligned(B_prepacked, 256))
+        return MXP_ERR_INVALID_ARG;
     if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
     mxp_packed none = {};
     none.mode = MXP_MODE_MXFP4;
@@ -434,9 +451,9 @@ mxp_status mxp_quantize_gemm_ready(const void* src, mxp_dtype src_dt, int64_t M,
 }
 
 mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed* A_packed,
-                          const mxp_packed* B_packed, const void* B_prepacked, void* D,
-                          mxp_dtype d_dt, int64_t ldd, void* workspace, size_t workspace_bytes,
-                          void* cuda_stream)
+                          const mxp_packed* B_packed, const void* B_prepacked,
+                          size_t B_prepacked_bytes, void* D, mxp_dtype d_dt, int64_t ldd,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
@@ -453,6 +470,8 @@ mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed* A_p
         return MXP_ERR_UNSUPPORTED;
     if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)
         return MXP_ERR_UNSUPPORTED;
+    if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) || !aligned(B_prepacked, 256))
+        return MXP_ERR_INVALID_ARG;
     return mxp::launch_gemm_tc_stream(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
                                       workspace, workspace_bytes,
                                       static_cast<cudaStream_t>(cuda_stream), true);
@@ -497,7 +516,7 @@ mxp_status mxp_gemm_clock_stamp(const void* workspace, void* cuda_stream, uint64
 
 mxp_status mxp_tensor_peak_probe(int kind, int iters, double* ms, double* flops)
 {
-    if (ms == nullptr || flops == nullptr || iters <= 0 || kind < 0 || kind > 3)
+    if (ms == nullptr || flops == nullptr || iters <= 0 || kind < 0 || kind > 5)
         return MXP_ERR_INVALID_ARG;
     return mxp::tensor_peak_probe(kind, iters, ms, flops);
 }

@@ -89,11 +89,22 @@ bool stream_a_ready_layout(int64_t M, int64_t K, size_t* atoms, size_t* slots, s
 cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, mxp_mode mode,
                                   uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
                                   uint8_t* atoms, uint8_t* slots, void* status, cudaStream_t stream);
-// One operand in the form that kernel reads (scale atoms; E4M3 bytes when `wide`), written
-// once, e.g. for weights.  stream_prepack_bytes() == 0: shape not supported.
-size_t stream_prepack_bytes(int64_t rows, int64_t K, bool wide);
-mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_bytes,
+// One operand in the form that kernel reads, written once, e.g. for weights.  `form` is an
+// mxp_prepack_form: scale atoms only, atoms + widened codes, or atoms + the Eq. 4 split of an
+// MXFP4+ operand.  stream_prepack_bytes() == 0: shape or form not supported.
+size_t stream_prepack_bytes(int64_t rows, int64_t K, int form);
+mxp_status stream_prepack(const mxp_packed& P, int form, void* out, size_t out_bytes,
                           cudaStream_t stream);
+// One MXFP4+ operand against one MXFP4 operand: FP4 main pass plus sparse residual MMA (Eq. 4,
+// Algorithm 1).  Workspace it needs (0: not this case, or shape not supported); `b_prepacked`:
+// B comes prepacked (form MXP_PREPACK_SPLIT if B is the MXFP4+ side, MXP_PREPACK_PLAIN if not).
+size_t stream_sparse_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode,
+                                     bool b_prepacked);
+mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_packed& A, const mxp_packed& B,
+                                 const void* b_prepacked, void* D, mxp_dtype d_dt, int64_t ldd,
+                                 void* workspace, size_t workspace_bytes, cudaStream_t stream);
+// The form of B's prepacked copy that a packed x packed GEMM with these modes reads.
+int stream_b_form(mxp_mode a_mode, mxp_mode b_mode);
 
 // Kernel choices a test or a measurement may force (mxp_debug_override): process-wide, 0 = the
 // library decides.

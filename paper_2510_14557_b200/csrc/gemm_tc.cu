@@ -1080,7 +1080,9 @@ mxp_status launch_pair_modes(bool ap, bool bp, const CUtensorMap& ta, const CUte
 // Issue-only loop: operands and scale atoms sit in shared memory (contents irrelevant), one
 // thread per CTA issues `iters` groups of two MMAs (K = 128 of FP4, or K = 64 of 8-bit
 // containers) into the same accumulator, optionally with the three scale-factor copies a
-// 128x256 tile needs per group, then commits and waits.
+// 128x256 tile needs per group, then commits and waits.  Kind 4: one sparse FP4 MMA (K = 128)
+// per group; kind 5: two dense FP4 MMAs and one sparse one per group, the instruction mix of a
+// main pass plus a sparse residual pass over the same 128 elements of K.
 template <int kKind>
 __global__ void __launch_bounds__(128, 1) peak_probe_kernel(int iters, uint32_t* status)
 {
@@ -1089,12 +1091,14 @@ __global__ void __launch_bounds__(128, 1) peak_probe_kernel(int iters, uint32_t*
                                                ~(uintptr_t)1023);
     uint8_t* a_tile = smem;                 // 128 rows x 128 B
     uint8_t* b_tile = smem + 16384;         // 256 rows x 128 B
-    uint8_t* sf = smem + 16384 + 32768;     // 3 atoms of 512 B
-    uint64_t* bar = reinterpret_cast<uint64_t*>(sf + 2048);
+    uint8_t* sf = smem + 16384 + 32768;     // 3 atoms of 512 B; behind them 128 x 16 B of sparsity metadata
+    uint64_t* bar = reinterpret_cast<uint64_t*>(sf + 4096);
     uint32_t* slot = reinterpret_cast<uint32_t*>(bar + 1);
     __shared__ uint32_t abort_flag;
     for (int i = threadIdx.x; i < (16384 + 32768 + 2048) / 16; i += blockDim.x)
         reinterpret_cast<uint4*>(smem)[i] = make_uint4(0x22222222u, 0x22222222u, 0x22222222u, 0x22222222u);
+    for (int i = threadIdx.x; i < 2048 / 16; i += blockDim.x)  // metadata: pairs 0 and 1 of every group
+        reinterpret_cast<uint4*>(sf + 2048)[i] = make_uint4(0x44444444u, 0x44444444u, 0x44444444u, 0x44444444u);
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar, 1);
         abort_flag = 0;
@@ -1114,7 +1118,11 @@ __global__ void __launch_bounds__(128, 1) peak_probe_kernel(int iters, uint32_t*
         const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(b_tile));
         const uint32_t t_sfa = tm + 256, t_sfb = tm + 264;
         constexpr bool kF8 = (kKind == 1);
-        constexpr bool kCopies = (kKind >= 2);
+        constexpr bool kCopies = (kKind == 2 || kKind == 3);
+        constexpr bool kDense = (kKind != 4);
+        constexpr bool kSparse = (kKind >= 4);
+        const uint32_t t_meta = tm + 288;
+        if (kSparse) ptx::tc_cp_128x128b(t_meta, ptx::smem_desc_sf(ptx::smem_u32(sf + 2048)));
         for (int it = 0; it < iters; ++it) {
             const uint32_t buf = (kKind == 3) ? (uint32_t)(it & 1) * 16u : 0u;
             if (kCopies) {
@@ -1123,7 +1131,7 @@ __global__ void __launch_bounds__(128, 1) peak_probe_kernel(int iters, uint32_t*
                 ptx::tc_cp_sf(t_sfb + buf + 4, ptx::smem_desc_sf(ptx::smem_u32(sf + 1024)));
             }
 #pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {
+            for (int kk = 0; kk < (kDense ? 2 : 0); ++kk) {
                 if (kF8)
                     ptx::mma_mxf8f6f4(tm, da + 2 * kk, db + 2 * kk,
                                       ptx::idesc_block_scaled(3, 3, 128, 256, kk, kk), t_sfa, t_sfb,
@@ -1133,6 +1141,10 @@ __global__ void __launch_bounds__(128, 1) peak_probe_kernel(int iters, uint32_t*
                                   ptx::idesc_block_scaled(1, 1, 128, 256, 2 * kk, 2 * kk),
                                   t_sfa + buf, t_sfb + buf, (it | kk) ? 1u : 0u);
             }
+            if (kSparse)
+                ptx::mma_sp_mxf4(tm, da + 4, db, t_meta,
+                                 ptx::idesc_block_scaled(1, 1, 128, 256, 0, 0) | ptx::kIdescSparse, t_sfa, t_sfb,
+                                 (kDense || it) ? 1u : 0u);
         }
         ptx::tc_commit(bar);
         if (!ptx::mbar_wait(bar, 0, &abort_flag, kWaitLimit) && status != nullptr)
@@ -1151,7 +1163,7 @@ mxp_status run_probe(int iters, double* ms, double* flops)
 {
     const int sms = sm_count();
     if (sms <= 0) return MXP_ERR_CUDA;
-    constexpr int kSmem = 16384 + 32768 + 2048 + 64 + 1024;
+    constexpr int kSmem = 16384 + 32768 + 4096 + 64 + 1024;
     auto kern = peak_probe_kernel<kKind>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
         return MXP_ERR_CUDA;
@@ -1186,7 +1198,9 @@ size_t tc_compact_workspace_bytes()
 
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode)
 {
-    const size_t fast = stream_workspace_bytes(M, N, K, a_mode, b_mode);
+    size_t fast = stream_workspace_bytes(M, N, K, a_mode, b_mode);
+    const size_t sparse = stream_sparse_workspace_bytes(M, N, K, a_mode, b_mode, false);
+    if (sparse > fast) fast = sparse;
     const size_t compact = tc_compact_workspace_bytes();
     return fast > compact ? fast : compact;
 }
@@ -1237,6 +1251,11 @@ mxp_status launch_gemm_tc(int64_t M, int64_t N, int64_t K, const mxp_packed& A,
     // which work in place and need only the status block.
     const size_t fast = stream_workspace_bytes(M, N, K, A.mode, B.mode);
     const bool forced_other = force != 0;
+    // one MXFP4+ operand against a plain one: FP4 main pass + sparse residual (1.5 instead of 2
+    // times the plain MXFP4 tensor work)
+    const size_t sparse = stream_sparse_workspace_bytes(M, N, K, A.mode, B.mode, false);
+    if (sparse != 0 && workspace_bytes >= sparse && !forced_other && override_get(MXP_KNOB_ONE_SIDED) != 1)
+        return launch_gemm_tc_sparse(M, N, K, A, B, nullptr, D, d_dt, ldd, workspace, workspace_bytes, stream);
     if (fast != 0 && workspace_bytes >= fast && !forced_other)
         return launch_gemm_tc_stream(M, N, K, A, B, nullptr, D, d_dt, ldd, workspace, workspace_bytes,
                                      stream);
@@ -1265,6 +1284,8 @@ mxp_status tensor_peak_probe(int kind, int iters, double* ms, double* flops)
         case 1: return run_probe<1>(iters, ms, flops);
         case 2: return run_probe<2>(iters, ms, flops);
         case 3: return run_probe<3>(iters, ms, flops);
+        case 4: return run_probe<4>(iters, ms, flops);
+        case 5: return run_probe<5>(iters, ms, flops);
     }
     return MXP_ERR_INVALID_ARG;
 }

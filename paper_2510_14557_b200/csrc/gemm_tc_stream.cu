@@ -19,6 +19,18 @@
 //
 // Plain MXFP4 x MXFP4 needs only the scale pass and runs kind::mxf4 on the nibble planes.
 //
+// One MXFP4+ operand against a plain MXFP4 one (the paper's main software scenario, Sec. 5:
+// MXFP4+ activations, MXFP4 weights) keeps the FP4 rate for the main pass and adds Eq. 4's
+// residual as a SPARSE MMA (Sec. 5.2, Algorithm 1): the MX+ operand is split once into
+//   * its nibble plane with every BM's code replaced by BM_H (4 or 6, an E2M1 value), and
+//   * BM_L (0, 0.5, 1 or 1.5 with the BM's sign; one value per block of 32, so the operand is
+//     almost all zeros) stored 2:1 compressed with the metadata saying where each value sits.
+// Per 128 elements of K the tensor core runs two dense kind::mxf4 instructions on the first
+// and one sparse instruction (K = 128) on the second, into the same accumulator with the same
+// scales: measured 1.5 times the plain MXFP4 issue time, against 2 times for the widened pass.
+// The sparse operand has to be the instruction's A operand, so when the weights are the MX+
+// side the kernel computes D^T = W A^T and its epilogue stores the tile transposed.
+//
 // Kernel: clusters of two CTAs, persistent, one 256 x 480 (kind::mxf4: 256 x 448) output tile
 // per cluster and step, held in two accumulators that share the A tile: per flop that is 23 %
 // fewer bytes through TMA than a 256 x 256 tile (kept for shapes whose larger tiles would fill
@@ -88,8 +100,12 @@ constexpr uint32_t kFmtE4M3 = 0, kFmtE2M3 = 3;  // instruction-descriptor codes,
 // kWide = true : rows are 128 E2M3 / E4M3 code slots (one scale atom per stage), kind::mxf8f6f4.
 // kHalves = 2: the tile has two halves (accumulators); 1: a single 256 x 256 accumulator, for
 // shapes whose larger tiles would not fill the GPU evenly.
-template <bool kWide, int kHalves>
+// kSparse (with kWide = false): A is an MXFP4+ operand split per Eq. 4; a stage also brings its
+// compressed BM_L tile (64 bytes per row: 64-byte swizzle) and the sparsity metadata (16 bytes
+// per row).
+template <bool kWide, int kHalves, bool kSparse = false>
 struct SCfg {
+    static_assert(!(kWide && kSparse), "the sparse residual belongs to the FP4 path");
     static constexpr int kGroups = kWide ? 1 : 2;           // K groups of 128 elements per stage
     static constexpr int kSfA = kGroups * kAtom;            // own 128 rows of A
     static constexpr int kSubN = sub_n(kWide, kHalves);     // columns of one accumulator
@@ -97,9 +113,12 @@ struct SCfg {
     static constexpr int kBRows = kSubN / 2;                // rows of a B half each CTA supplies
     static constexpr int kBTile = kBRows * kRowBytes;       // 15 (14) KB
     static constexpr int kSfB = 2 * kHalves * kGroups * kAtom;  // all rows of the B halves
-    static constexpr int kStageRaw = kHalfTile + kHalves * kBTile + kSfA + kSfB;
+    static constexpr int kRes = kSparse ? 128 * 64 : 0;     // compressed BM_L rows of this CTA
+    static constexpr int kMeta = kSparse ? 128 * 16 : 0;    // their sparsity metadata
+    static constexpr int kResOff = kHalfTile + kHalves * kBTile + kSfA + kSfB;  // multiple of 1024
+    static constexpr int kStageRaw = kResOff + kRes + kMeta;
     static constexpr int kStage = (kStageRaw + 1023) / 1024 * 1024;  // swizzled tiles: 1024-aligned
-    static constexpr int kStages = kHalves == 2 ? 4 : 6;
+    static constexpr int kStages = kSparse ? (kHalves == 2 ? 3 : 5) : (kHalves == 2 ? 4 : 6);
     static constexpr int kSmem = kStages * kStage + 1024 /*barriers*/ + 1024 /*align*/;
     static constexpr int kElemsPerStage = kWide ? 128 : 256;
 };
@@ -114,6 +133,7 @@ struct SParams {
     void* D;
     int64_t ldd;
     int d_vec_ok;
+    int transposed;  // the tile is D^T: accumulator row r, column c belong at D[c][r]
     StatusBlock* status;
 };
 
@@ -144,14 +164,16 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
     tm = band * kBand + (r - tn * h);
 }
 
-template <bool kWide, int kHalves, typename OutT>
+template <bool kWide, int kHalves, bool kSparse, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                       const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_sfa,
-                      const __grid_constant__ CUtensorMap tmap_sfb, const SParams prm)
+                      const __grid_constant__ CUtensorMap tmap_sfb,
+                      const __grid_constant__ CUtensorMap tmap_res,
+                      const __grid_constant__ CUtensorMap tmap_meta, const SParams prm)
 {
-    using C = SCfg<kWide, kHalves>;
+    using C = SCfg<kWide, kHalves, kSparse>;
     constexpr int S = C::kStages;
     constexpr int G = C::kGroups;
 
@@ -170,6 +192,8 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
     auto b_tile = [&](int s, int j) { return smem + s * C::kStage + kHalfTile + j * C::kBTile; };
     auto sfa = [&](int s) { return smem + s * C::kStage + kHalfTile + kHalves * C::kBTile; };
     auto sfb = [&](int s) { return smem + s * C::kStage + kHalfTile + kHalves * C::kBTile + C::kSfA; };
+    auto res_tile = [&](int s) { return smem + s * C::kStage + C::kResOff; };
+    auto meta_tile = [&](int s) { return smem + s * C::kStage + C::kResOff + C::kRes; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0: issues the MMAs
@@ -193,6 +217,10 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
         ptx::prefetch_tmap(&tmap_b);
         ptx::prefetch_tmap(&tmap_sfa);
         ptx::prefetch_tmap(&tmap_sfb);
+        if (kSparse) {
+            ptx::prefetch_tmap(&tmap_res);
+            ptx::prefetch_tmap(&tmap_meta);
+        }
     }
     if (warp == 1) {
         ptx::tmem_alloc_2cta(tmem_slot, kTmemCols);
@@ -205,10 +233,6 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const uint32_t tmem_base = *tmem_slot;
     ClockStamp* stamp = reinterpret_cast<ClockStamp*>(reinterpret_cast<uint8_t*>(prm.status) +
                                                       kClockStampOffset);
-    if (blockIdx.x == 0 && threadIdx.x == 64) {  // an epilogue warp: the last to finish
-        stamp->clk_begin = (unsigned long long)clock64();
-        stamp->ns_begin = ptx::globaltimer_ns();
-    }
 #ifdef MXP_S_GRIDSTAMP  // measurement builds: earliest begin, latest and earliest end over all CTAs
     if (threadIdx.x == 64) atomicMin(reinterpret_cast<unsigned long long*>(stamp) + 4, ptx::globaltimer_ns());
 #endif
@@ -225,6 +249,9 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                             : kWide      ? (j == 0 ? 248u : 496u)
                                          : 232u + 256u * g + 8u * j);
     };
+    // Sparsity metadata of a stage: four columns (two per K group) behind the scale factors
+    // (two halves: group 0's occupy columns 224..247; one half: 256..279).
+    const uint32_t tmem_meta = tmem_base + (kHalves == 1 ? 288u : 248u);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -233,6 +260,11 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             // the launch may overlap the tail of the prepack kernel: its output is first
             // touched here
             ptx::grid_dependency_wait();
+            if (blockIdx.x == 0) {  // the kernel's own work starts here: what came before is the
+                                    // tail of the grid it depends on
+                stamp->clk_begin = (unsigned long long)clock64();
+                stamp->ns_begin = ptx::globaltimer_ns();
+            }
             uint32_t c = 0;
             bool ok = true;
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
@@ -257,10 +289,6 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                         ok = false;
                         break;
                     }
-#ifdef MXP_EXP_NOTMA
-                    if (rank == 0) ptx::mbar_arrive(&full[s]);
-                    continue;
-#endif
                     if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * C::kStageRaw);
                     ptx::tma_load_2d_pair(a_tile(s), &tmap_a, full0 + 8u * (uint32_t)s, ka * kRowBytes, ya + m0);
 #pragma unroll
@@ -270,6 +298,11 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     ptx::tma_load_3d_pair(sfa(s), &tmap_sfa, full0 + 8u * (uint32_t)s, 0, ka * G, 2 * tm + (int)rank);
                     ptx::tma_load_3d_pair(sfb(s), &tmap_sfb, full0 + 8u * (uint32_t)s, 0, ka * G,
                                           2 * kHalves * tn);
+                    if (kSparse) {
+                        ptx::tma_load_2d_pair(res_tile(s), &tmap_res, full0 + 8u * (uint32_t)s, ka * 64, m0);
+                        ptx::tma_load_3d_pair(meta_tile(s), &tmap_meta, full0 + 8u * (uint32_t)s, 0, ka * 4,
+                                              2 * tm + (int)rank);
+                    }
                 }
             }
         }
@@ -306,17 +339,15 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     const int groups =
                         kWide ? 1 : ((prm.K - (kt % kbase) * C::kElemsPerStage) >= C::kElemsPerStage ? 2 : 1);
                     if (ptx::elect_one()) {
-#ifdef MXP_EXP_NOMMA
-                        for (int g = 0; g < 0; ++g) {
-#else
                         for (int g = 0; g < groups; ++g) {
-#endif
                             ptx::tc_cp_sf_2cta(tmem_sfa(g), d_sfa + (uint64_t)(kAtom * g >> 4));
                             // B's atoms in shared memory: [half j][128-row part h][K group g]
 #pragma unroll
                             for (int jh = 0; jh < 2 * kHalves; ++jh)
                                 ptx::tc_cp_sf_2cta(tmem_sfb(g, jh >> 1) + 4 * (jh & 1),
                                                    d_sfb + (uint64_t)((G * kAtom * jh + kAtom * g) >> 4));
+                            if (kSparse && g == 0)
+                                ptx::tc_cp_128x128b_2cta(tmem_meta, ptx::smem_desc_sf(ptx::smem_u32(meta_tile(s))));
                             for (int j = 0; j < halves; ++j) {
                                 const uint32_t tmem_acc = tmem_base + 256u * j;
                                 const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(b_tile(s, j)));
@@ -339,6 +370,18 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                         ptx::mma_mxf4_2cta(tmem_acc, da + adv, db + adv, idesc,
                                                            tmem_sfa(g), tmem_sfb(g, j),
                                                            accumulate | (uint32_t)(g | kk));
+                                    }
+                                    if (kSparse) {
+                                        // Eq. 4's BM_L term over the same 128 elements of K: 32
+                                        // bytes of compressed A per row, 64 bytes of B, all four
+                                        // scale bytes of either operand's column
+                                        const uint64_t dr =
+                                            ptx::smem_desc_sw64(ptx::smem_u32(res_tile(s))) + (uint64_t)(2 * g);
+                                        const uint32_t idesc =
+                                            ptx::idesc_block_scaled(1, 1, kTileM, C::kSubN, 0, 0) | ptx::kIdescSparse;
+                                        ptx::mma_sp_mxf4_2cta(tmem_acc, dr, db + (uint64_t)(4 * g),
+                                                              tmem_meta + 2u * (uint32_t)g, idesc, tmem_sfa(g),
+                                                              tmem_sfb(g, j), 1u);
                                     }
                                 }
                             }
@@ -398,6 +441,22 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 }
                 const int col0 = n0 + ch * kCols;
                 if (row >= prm.M || col0 >= prm.N) continue;
+                if (kSparse && prm.transposed) {
+                    // D[col][row]: a register holds one column of the tile, the warp's lanes
+                    // hold 32 consecutive rows, i.e. 32 consecutive elements of a row of D
+                    OutT* dcol = static_cast<OutT*>(prm.D) + (int64_t)col0 * prm.ldd + row;
+#pragma unroll
+                    for (int i = 0; i < kCols; ++i) {
+                        if (col0 + i < prm.N) {
+                            if (sizeof(OutT) == 4)
+                                reinterpret_cast<float*>(dcol)[(int64_t)i * prm.ldd] = __uint_as_float(rr[i]);
+                            else
+                                reinterpret_cast<__nv_bfloat16*>(dcol)[(int64_t)i * prm.ldd] =
+                                    __float2bfloat16_rn(__uint_as_float(rr[i]));
+                        }
+                    }
+                    continue;
+                }
                 OutT* drow = static_cast<OutT*>(prm.D) + (int64_t)row * prm.ldd + col0;
                 if (col0 + kCols <= prm.N && prm.d_vec_ok) {
                     uint4* p = reinterpret_cast<uint4*>(drow);
@@ -497,6 +556,13 @@ struct PrepackOperand {
     size_t plane_bytes;       // MXFP6+: distance to the second plane of the widened copy, else 0
     unsigned scale_ctas;      // row groups * ceil(nbk/128)
     unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
+    // Eq. 4 split of an MXFP4+ operand for the sparse residual MMA (nullptr / 0: not wanted)
+    uint8_t* sp_main;         // [rows][K/2]: the nibble plane with BM_H in every BM's place
+    uint8_t* sp_res;          // [rows][K/4]: BM_L, 2:1 compressed
+    uint8_t* sp_meta;         // [row group of 128][stage of 256 elements][128 rows x 16 bytes]
+    int sp_stages;            // ceil(K / 256)
+    int sp_row_groups;        // row groups of 128 the metadata covers (two per output tile)
+    unsigned split_ctas;      // ceil(row groups * 128 * (nbk / 4) / 256)
 };
 
 __device__ __forceinline__ void prepack_scales(const PrepackOperand& op, unsigned id, uint32_t* tile)
@@ -671,23 +737,83 @@ __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned i
         dst[e] = (uint8_t)(((nib & 8u) << 4) | (0x48u + (shift << 3)) | (nib & 7u));
 }
 
+// Eq. 4 / Algorithm 1 (ReplaceBM, MakeFragment) done once per operand instead of once per tile:
+// one thread per 128 elements of a row (four blocks: one K group of the sparse instruction).
+//   main plane: the block's codes with the BM's code s m2 m1 m0 replaced by BM_H = s 1 1 m2
+//     (4 or 6);
+//   residual: BM_L = s 0 m1 m0 (0, 0.5, 1, 1.5) as the only non-zero of the block, compressed
+//     2:1 the way tcgen05.mma.sp reads it: of each 8 consecutive elements two aligned pairs are
+//     kept (4 codes), and a nibble of metadata names the pairs -- low two bits the first, high
+//     two bits the second, ascending.  The group of 8 that holds the BM keeps the BM's pair and
+//     pair 3 (pairs 0 and 3 if the BM sits in pair 3); every other group keeps pairs 0 and 1.
+//   Blocks with scale byte 0 become zeros in both.  Rows past the operand's end (the row groups
+//   are whole) get metadata only, so that every nibble the tensor core reads is a valid one.
+__device__ __forceinline__ void split_codes(const PrepackOperand& op, unsigned id)
+{
+    const uint32_t t = id * 256u + threadIdx.x;
+    const uint32_t kgroups = (uint32_t)op.nbk >> 2;
+    if (t >= (uint32_t)op.sp_row_groups * 128u * kgroups) return;
+    const uint32_t row = t / kgroups, g = t - row * kgroups;
+    uint8_t* meta_dst = op.sp_meta + ((size_t)(row >> 7) * (size_t)op.sp_stages + (g >> 1)) * 2048u +
+                        (row & 127u) * 16u + (g & 1u) * 8u;
+    unsigned long long meta = 0x4444444444444444ull;
+    if (row < (uint32_t)op.rows) {
+        const size_t b0 = (size_t)row * (size_t)op.nbk + 4u * g;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const uint4 c = __ldg(reinterpret_cast<const uint4*>(op.nibbles) + b0 + b);
+            uint32_t w[4] = {c.x, c.y, c.z, c.w};
+            const uint32_t sc = op.scales[b0 + b];
+            unsigned long long res = 0ull;
+            if (sc == 0u) {
+                w[0] = w[1] = w[2] = w[3] = 0u;
+            } else {
+                const uint32_t pos = op.bm_index[b0 + b] & 31u;
+                const uint32_t sh = (pos & 7u) * 4u;
+                uint32_t word = pos < 8u ? w[0] : pos < 16u ? w[1] : pos < 24u ? w[2] : w[3];
+                const uint32_t nib = (word >> sh) & 15u;
+                word = (word & ~(15u << sh)) | (((nib & 8u) | 6u | ((nib >> 2) & 1u)) << sh);
+                if (pos < 8u) w[0] = word; else if (pos < 16u) w[1] = word; else if (pos < 24u) w[2] = word; else w[3] = word;
+                const uint32_t gi = pos >> 3, pair = (pos & 7u) >> 1, slot = pair == 3u ? 1u : 0u;
+                const uint32_t mnib = pair == 3u ? 0xCu : (pair | 0xCu);
+                meta = (meta & ~(15ull << (16 * b + 4 * gi))) | ((unsigned long long)mnib << (16 * b + 4 * gi));
+                if (nib & 3u)
+                    res = (unsigned long long)((nib & 8u) | (nib & 3u)) << (4u * (4u * gi + 2u * slot + (pos & 1u)));
+            }
+            reinterpret_cast<uint4*>(op.sp_main)[b0 + b] = make_uint4(w[0], w[1], w[2], w[3]);
+            reinterpret_cast<unsigned long long*>(op.sp_res)[b0 + b] = res;
+        }
+    }
+    *reinterpret_cast<unsigned long long*>(meta_dst) = meta;
+    // an odd number of K groups: the last stage's second group does not exist, its metadata must
+    if (g == kgroups - 1u && (kgroups & 1u))
+        *reinterpret_cast<unsigned long long*>(meta_dst + 8) = 0x4444444444444444ull;
+}
+
 __global__ void __launch_bounds__(256) prepack_kernel(const PrepackOperand a, const PrepackOperand b,
                                                       StatusBlock* status)
 {
     __shared__ uint32_t tile[32 * 129];
-    ptx::grid_launch_dependents();  // the GEMM's prologue may start while this grid drains
     unsigned id = blockIdx.x;
     if (id == 0 && threadIdx.x == 0 && status != nullptr) {
         status->code = 0u;  // the GEMM that follows on the stream reports into this block
         status->where = 0u;
+        __threadfence();
     }
+    // the GEMM's prologue may start while this grid drains (its first CTA has cleared the status
+    // block by then: a dependent grid is released only when every CTA has passed this point)
+    ptx::grid_launch_dependents();
     if (id < a.scale_ctas) return prepack_scales(a, id, tile);
     id -= a.scale_ctas;
     if (id < b.scale_ctas) return prepack_scales(b, id, tile);
     id -= b.scale_ctas;
     if (id < a.widen_ctas) return widen_codes(a, id);
     id -= a.widen_ctas;
-    widen_codes(b, id);
+    if (id < b.widen_ctas) return widen_codes(b, id);
+    id -= b.widen_ctas;
+    if (id < a.split_ctas) return split_codes(a, id);
+    id -= a.split_ctas;
+    split_codes(b, id);
 }
 
 #ifndef MXP_S_L2PROMO
@@ -781,13 +907,13 @@ int choose_halves(int64_t M, int64_t N, bool wide, int num_sms)
     return cost(1) < cost(2) ? 1 : 2;
 }
 
-template <bool kWide, int kHalves, typename OutT>
+template <bool kWide, int kHalves, bool kSparse, typename OutT>
 mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tsa,
-                         const CUtensorMap& tsb, const SParams& prm, int num_sms,
-                         cudaStream_t stream)
+                         const CUtensorMap& tsb, const CUtensorMap& tres, const CUtensorMap& tmeta,
+                         const SParams& prm, int num_sms, cudaStream_t stream)
 {
-    using C = SCfg<kWide, kHalves>;
-    auto kern = gemm_tc_stream_kernel<kWide, kHalves, OutT>;
+    using C = SCfg<kWide, kHalves, kSparse>;
+    auto kern = gemm_tc_stream_kernel<kWide, kHalves, kSparse, OutT>;
     static SmemAttrOnce once;
     if (ensure_dynamic_smem(kern, C::kSmem, once) != cudaSuccess) return MXP_ERR_CUDA;
     const int64_t tiles =
@@ -808,8 +934,8 @@ mxp_status launch_stream(const CUtensorMap& ta, const CUtensorMap& tb, const CUt
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, ta, tb, tsa, tsb, prm) == cudaSuccess ? MXP_OK
-                                                                               : MXP_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, kern, ta, tb, tsa, tsb, tres, tmeta, prm) == cudaSuccess ? MXP_OK
+                                                                                             : MXP_ERR_CUDA;
 }
 
 // Weight-only form at prefill sizes (Sec. 7.1, "conversion before computation"; the paper's
@@ -826,12 +952,13 @@ prepack_dense_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, in
                      uint8_t* __restrict__ atoms, uint4* __restrict__ slots, size_t plane_slots,
                      StatusBlock* status)
 {
-    ptx::grid_launch_dependents();  // the GEMM's prologue may start while this grid drains
     const int64_t blk = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (blk == 0 && status != nullptr) {
         status->code = 0u;
         status->where = 0u;
+        __threadfence();
     }
+    ptx::grid_launch_dependents();  // the GEMM's prologue may start while this grid drains
     const int64_t row = blk / nbk;
     const int kb = (int)(blk - row * nbk);
     if (row >= rows_pad) return;
@@ -953,7 +1080,85 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     op.tile_rows = tile_rows;
     op.scale_ctas = (unsigned)(row_groups(rows, tile_rows) * ((kgroups + 31) / 32));
     op.widen_ctas = wide ? (unsigned)((rows * nbk * 2 + 255) / 256) : 0u;
+    op.sp_main = op.sp_res = op.sp_meta = nullptr;
+    op.sp_stages = op.sp_row_groups = 0;
+    op.split_ctas = 0u;
     return op;
+}
+
+// Prepacked form of an MXFP4+ operand that takes the A slot of the sparse-residual kernel: scale
+// atoms tiled for 256-row output tiles, then the three planes split_codes() writes.
+struct SplitLayout {
+    size_t atoms, main, res, meta, total;
+};
+SplitLayout split_layout(int64_t rows, int64_t K)
+{
+    SplitLayout l;
+    const size_t rgs = (size_t)row_groups(rows, kTileM), kgroups = (size_t)(K / 128);
+    l.atoms = 0;
+    l.main = round_up(rgs * kgroups * kAtom, 1024);
+    l.res = l.main + round_up((size_t)rows * (size_t)K / 2, 1024);
+    l.meta = l.res + round_up((size_t)rows * (size_t)K / 4, 1024);
+    l.total = l.meta + round_up(rgs * (size_t)((K + 255) / 256) * 2048, 1024);
+    return l;
+}
+PrepackOperand split_operand(const mxp_packed& P, uint8_t* base)
+{
+    const SplitLayout l = split_layout(P.rows, P.cols);
+    PrepackOperand op = prepack_operand(P, P.rows, P.cols, false, kTileM, base + l.atoms, nullptr);
+    op.sp_main = base + l.main;
+    op.sp_res = base + l.res;
+    op.sp_meta = base + l.meta;
+    op.sp_stages = (int)((P.cols + 255) / 256);
+    op.sp_row_groups = (int)row_groups(P.rows, kTileM);
+    op.split_ctas = (unsigned)(((int64_t)op.sp_row_groups * 128 * (P.cols / 128) + 255) / 256);
+    return op;
+}
+// 2-D byte tensor [rows][row_bytes], boxes of 64 bytes x 128 rows, 64-byte swizzle (the
+// compressed residual tile of the sparse instruction).
+bool make_tmap_rows64(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t row_bytes)
+{
+    EncodeFn fn = tensormap_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {64u, 128u};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+              MXP_S_L2PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Sparsity metadata [row groups][stages][2048 bytes] as 32-bit words, one box = one stage's
+// 128 rows x 16 bytes.
+bool make_tmap_meta(CUtensorMap* m, const uint8_t* base, int64_t row_groups_total, int64_t stages)
+{
+    EncodeFn fn = tensormap_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {128u, (cuuint64_t)(4 * stages), (cuuint64_t)row_groups_total};
+    const cuuint64_t strides[2] = {512u, (cuuint64_t)2048 * (cuuint64_t)stages};
+    const cuuint32_t box[3] = {128u, 4u, 1u};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Workspace of a sparse-residual call: status block, then what is not prepacked -- the MX+
+// operand's split form, the plain operand's scale atoms (sized for either tiling).
+struct SparseLayout {
+    size_t x, y, total;
+};
+SparseLayout sparse_layout(int64_t rows_x, int64_t rows_y, int64_t K, bool x_prepacked, bool y_prepacked)
+{
+    SparseLayout l;
+    size_t off = round_up(kStatusBytes, 1024);
+    l.x = off;
+    if (!x_prepacked) off += split_layout(rows_x, K).total;
+    l.y = off;
+    if (!y_prepacked)
+        off += round_up((size_t)std::max(row_groups(rows_y, sub_n(false, 1)), row_groups(rows_y, sub_n(false, 2))) *
+                            (size_t)(K / 128) * kAtom, 1024);
+    l.total = off;
+    return l;
 }
 PrepackOperand no_operand()
 {
@@ -962,18 +1167,32 @@ PrepackOperand no_operand()
 }
 }  // namespace
 
-size_t stream_prepack_bytes(int64_t rows, int64_t K, bool wide)
+size_t stream_prepack_bytes(int64_t rows, int64_t K, int form)
 {
-    if (rows <= 0 || K <= 0 || K % 128 != 0) return 0;
+    if (rows <= 0 || K <= 0 || K % 128 != 0 || form < 0 || form > 2) return 0;
     if ((uint64_t)rows * (uint64_t)K / 16 >= (1ull << 32)) return 0;
-    return packed_layout(rows, K, wide).total;
+    if (form == 2) return split_layout(rows, K).total;
+    return packed_layout(rows, K, form == 1).total;
 }
 
-mxp_status stream_prepack(const mxp_packed& P, bool wide, void* out, size_t out_bytes,
+mxp_status stream_prepack(const mxp_packed& P, int form, void* out, size_t out_bytes,
                           cudaStream_t stream)
 {
-    const size_t need = stream_prepack_bytes(P.rows, P.cols, wide);
+    const bool wide = form == 1;
+    const size_t need = stream_prepack_bytes(P.rows, P.cols, form);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
+    if (form == 2) {
+        if (P.mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
+        if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
+            (reinterpret_cast<uintptr_t>(P.scales) & 3))
+            return MXP_ERR_INVALID_ARG;
+        const PrepackOperand px = split_operand(P, static_cast<uint8_t*>(out));
+        const uint64_t ctas = (uint64_t)px.scale_ctas + px.split_ctas;
+        if (ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
+        prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(px, no_operand(), nullptr);
+        return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+    }
     // an MXFP6+ operand needs two planes, which this form has no room for: mxp_gemm takes it
     if ((P.mode > MXP_MODE_MXFP6 && P.mode != MXP_MODE_MXFP8) ||
         ((mode_six(P.mode) || mode_eight(P.mode)) && !wide))
@@ -1101,14 +1320,105 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     prm.ldd = ldd;
     prm.d_vec_ok = ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
                    ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
+    prm.transposed = 0;
     prm.status = static_cast<StatusBlock*>(workspace);
     const bool f32 = d_dt == MXP_F32;
 #define MXP_S_LAUNCH(W, H)                                                                    \
-    (f32 ? launch_stream<W, H, float>(ta, tb, tsa, tsb, prm, num_sms, stream)                 \
-         : launch_stream<W, H, __nv_bfloat16>(ta, tb, tsa, tsb, prm, num_sms, stream))
+    (f32 ? launch_stream<W, H, false, float>(ta, tb, tsa, tsb, ta, ta, prm, num_sms, stream)  \
+         : launch_stream<W, H, false, __nv_bfloat16>(ta, tb, tsa, tsb, ta, ta, prm, num_sms, stream))
     if (wide) return halves == 2 ? MXP_S_LAUNCH(true, 2) : MXP_S_LAUNCH(true, 1);
     return halves == 2 ? MXP_S_LAUNCH(false, 2) : MXP_S_LAUNCH(false, 1);
 #undef MXP_S_LAUNCH
+}
+
+// ------------------------------------------------------------------------------ sparse residual
+int stream_b_form(mxp_mode a_mode, mxp_mode b_mode)
+{
+    const bool one_sided = (a_mode == MXP_MODE_MXFP4_PLUS && b_mode == MXP_MODE_MXFP4) ||
+                           (a_mode == MXP_MODE_MXFP4 && b_mode == MXP_MODE_MXFP4_PLUS);
+    if (one_sided && override_get(MXP_KNOB_ONE_SIDED) != 1)
+        return b_mode == MXP_MODE_MXFP4_PLUS ? MXP_PREPACK_SPLIT : MXP_PREPACK_PLAIN;
+    return (a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4) ? MXP_PREPACK_WIDE : MXP_PREPACK_PLAIN;
+}
+
+// One operand MXFP4+, the other MXFP4 (see the head of this file).  0: not supported.
+size_t stream_sparse_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode,
+                                     bool b_prepacked)
+{
+    const bool ap = a_mode == MXP_MODE_MXFP4_PLUS, bp = b_mode == MXP_MODE_MXFP4_PLUS;
+    if (ap == bp || (ap ? b_mode : a_mode) != MXP_MODE_MXFP4) return 0;
+    if (M <= 128 || N <= 128 || K < 128 || K % 128 != 0) return 0;
+    if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 32) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
+        return 0;
+    const int64_t rows_x = ap ? M : N, rows_y = ap ? N : M;
+    return sparse_layout(rows_x, rows_y, K, b_prepacked && bp, b_prepacked && ap).total;
+}
+
+mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_packed& A, const mxp_packed& B,
+                                 const void* b_prepacked, void* D, mxp_dtype d_dt, int64_t ldd,
+                                 void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    const size_t need = stream_sparse_workspace_bytes(M, N, K, A.mode, B.mode, b_prepacked != nullptr);
+    if (need == 0) return MXP_ERR_UNSUPPORTED;
+    if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(b_prepacked) & 255))
+        return MXP_ERR_INVALID_ARG;
+    // X: the MX+ operand, in the instruction's A slot; Y: the plain one.  X = B: D^T = B A^T.
+    const bool swap = B.mode == MXP_MODE_MXFP4_PLUS;
+    const mxp_packed& X = swap ? B : A;
+    const mxp_packed& Y = swap ? A : B;
+    const int64_t rows_x = X.rows, rows_y = Y.rows;
+    if (((reinterpret_cast<uintptr_t>(X.nibbles) | reinterpret_cast<uintptr_t>(Y.nibbles)) & 15) ||
+        ((reinterpret_cast<uintptr_t>(X.scales) | reinterpret_cast<uintptr_t>(Y.scales)) & 3))
+        return MXP_ERR_INVALID_ARG;
+    const int num_sms = sm_count();
+    if (num_sms <= 0) return MXP_ERR_CUDA;
+    const bool x_pre = swap && b_prepacked != nullptr, y_pre = !swap && b_prepacked != nullptr;
+    const SparseLayout l = sparse_layout(rows_x, rows_y, K, x_pre, y_pre);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const int kgroups = (int)(K / 128);
+    const int halves = choose_halves(rows_x, rows_y, false, num_sms);
+    const int sub = sub_n(false, halves);
+    const int rgx = (int)row_groups(rows_x, kTileM), rgy = (int)row_groups(rows_y, sub);
+    const uint8_t* x_base = x_pre ? static_cast<const uint8_t*>(b_prepacked) : ws + l.x;
+    const SplitLayout lx = split_layout(rows_x, K);
+    const uint8_t* y_atoms =
+        y_pre ? static_cast<const uint8_t*>(b_prepacked) + packed_layout(rows_y, K, false).atoms[halves - 1]
+              : ws + l.y;
+    const PrepackOperand px = x_pre ? no_operand() : split_operand(X, ws + l.x);
+    const PrepackOperand py =
+        y_pre ? no_operand() : prepack_operand(Y, rows_y, K, false, sub, ws + l.y, nullptr);
+    const uint64_t ctas = (uint64_t)px.scale_ctas + py.scale_ctas + px.split_ctas;
+    if (ctas == 0 || ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
+    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(px, py, static_cast<StatusBlock*>(workspace));
+    if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+
+    CUtensorMap ta, tb, tsa, tsb, tres, tmeta;
+    const bool maps_ok = make_tmap_rows(&ta, x_base + lx.main, rows_x, K / 2, 128) &&
+                         make_tmap_rows(&tb, Y.nibbles, rows_y, K / 2, sub / 2) &&
+                         make_tmap_atoms(&tsa, x_base + lx.atoms, rgx, kgroups, 2, 1) &&
+                         make_tmap_atoms(&tsb, y_atoms, rgy, kgroups, 2, 2 * halves) &&
+                         make_tmap_rows64(&tres, x_base + lx.res, rows_x, K / 4) &&
+                         make_tmap_meta(&tmeta, x_base + lx.meta, rgx, (K + 255) / 256);
+    if (!maps_ok) return MXP_ERR_CUDA;
+    SParams prm;
+    prm.M = (int)rows_x;
+    prm.N = (int)rows_y;
+    prm.K = (int)K;
+    prm.a_fmt = prm.b_fmt = 0;
+    prm.parts_a = prm.parts_b = 1;
+    prm.D = D;
+    prm.ldd = ldd;
+    prm.d_vec_ok = !swap && ((reinterpret_cast<uintptr_t>(D) & 15) == 0) &&
+                   ((ldd * (d_dt == MXP_BF16 ? 2 : 4)) % 16 == 0);
+    prm.transposed = swap ? 1 : 0;
+    prm.status = static_cast<StatusBlock*>(workspace);
+    const bool f32 = d_dt == MXP_F32;
+    if (halves == 2)
+        return f32 ? launch_stream<false, 2, true, float>(ta, tb, tsa, tsb, tres, tmeta, prm, num_sms, stream)
+                   : launch_stream<false, 2, true, __nv_bfloat16>(ta, tb, tsa, tsb, tres, tmeta, prm, num_sms, stream);
+    return f32 ? launch_stream<false, 1, true, float>(ta, tb, tsa, tsb, tres, tmeta, prm, num_sms, stream)
+               : launch_stream<false, 1, true, __nv_bfloat16>(ta, tb, tsa, tsb, tres, tmeta, prm, num_sms, stream);
 }
 
 }  // namespace mxp

@@ -18,9 +18,18 @@
 // product's bit pattern; scale byte and BM: by casting the product scaled down and up by
 // 2^-20) and settled by comparing |x| with t * d (resp. amax with 6 t ts) in binary64, where
 // those products (at most 33 significant bits) are exact; equality is the tie.
+// Short operands (kShort: bf16 source, tensor scale with at most 12 significant bits, which
+// covers every power of two): |x| has at most 8 significant bits and t * d at most 19, so a
+// quotient that is not exactly on a boundary is at least 2^-20 of it away, and ties themselves
+// are common (with a power-of-two d every 128th bf16 value of a binade is one).  There the
+// quotient is taken with one Newton step on the reciprocal product, which returns it exactly
+// whenever it is representable; the hardware cast then sees the tie as a tie, and nothing is
+// left to settle per element.
 //
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+
+#include <cstring>
 
 #include "common.cuh"
 
@@ -71,7 +80,7 @@ __device__ __forceinline__ float elem(const uint32_t* raw, int i)
     return __uint_as_float((i & 1) ? raw[i >> 1] & 0xFFFF0000u : raw[i >> 1] << 16);
 }
 
-template <typename T, bool kPlus>
+template <typename T, bool kPlus, bool kShort>
 __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float six_ts, uint32_t& w0, uint32_t& w1,
                                             uint32_t& scale_byte, uint32_t& index)
 {
@@ -114,32 +123,46 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
     // quotient: only a product whose pattern lies within 8 of such a pattern can be cast to
     // another code than the exact quotient.  `near` ends up below 0x8000 iff the block has one.
     float s[16];
-    uint32_t near = 0xFFFFFFFFu;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        s[i] = __fmul_rn(X(i), r);
-        near = min(near, __float_as_uint(s[i]) * 2048u + 0x4000u);
-    }
-    w0 = cvt_e2m1x8(s);
-    w1 = cvt_e2m1x8(s + 8);
-    if (near < 0x8000u) {
-        const double d = (double)e * (double)ts;  // exact
+    if (kShort) {
+        // d is exact in binary32 here.  rho = x - s0 d (rounded down, so that an exact zero is
+        // -0 and the sum below keeps the sign of a zero input), s = s0 + rho r.
+        const float d32 = __fmul_rn(e, ts);
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const uint32_t bits = __float_as_uint(__fmul_rn(X(i), r));  // (recomputed: keeps s[] short-lived)
-            if (bits * 2048u + 0x4000u < 0x8000u) {
-                const float t = __uint_as_float((bits + 8u) & 0x7FE00000u);  // the candidate boundary
-                const float t4 = fminf(t * 4.f, 31.f);
-                const uint32_t u = (uint32_t)t4;                               // 1 3 5 7 10 14 20
-                constexpr uint32_t kBoundaries = 0x1044AAu;                    // those bits set
-                if ((float)u == t4 && ((kBoundaries >> u) & 1u)) {
-                    const uint32_t lower = (uint32_t)__popc(kBoundaries & ((1u << u) - 1u));  // code below it
-                    const double bound = (double)t * d;                        // exact
-                    const double a = fabs((double)X(i));
-                    const uint32_t code = lower + ((a > bound || (a == bound && (lower & 1u))) ? 1u : 0u);
-                    const uint32_t sh = (uint32_t)(i & 7) * 4u;
-                    if (i < 8) w0 = (w0 & ~(7u << sh)) | (code << sh);
-                    else w1 = (w1 & ~(7u << sh)) | (code << sh);
+            const float x = X(i);
+            const float s0 = __fmul_rn(x, r);
+            s[i] = __fmaf_rn(__fmaf_rd(-s0, d32, x), r, s0);
+        }
+        w0 = cvt_e2m1x8(s);
+        w1 = cvt_e2m1x8(s + 8);
+    } else {
+        uint32_t near = 0xFFFFFFFFu;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            s[i] = __fmul_rn(X(i), r);
+            near = min(near, __float_as_uint(s[i]) * 2048u + 0x4000u);
+        }
+        w0 = cvt_e2m1x8(s);
+        w1 = cvt_e2m1x8(s + 8);
+        if (near < 0x8000u) {
+            const double d = (double)e * (double)ts;  // exact
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint32_t bits = __float_as_uint(__fmul_rn(X(i), r));  // (recomputed: keeps s[] short-lived)
+                if (bits * 2048u + 0x4000u < 0x8000u) {
+                    const float t = __uint_as_float((bits + 8u) & 0x7FE00000u);  // the candidate boundary
+                    const float t4 = fminf(t * 4.f, 31.f);
+                    const uint32_t u = (uint32_t)t4;                               // 1 3 5 7 10 14 20
+                    constexpr uint32_t kBoundaries = 0x1044AAu;                    // those bits set
+                    if ((float)u == t4 && ((kBoundaries >> u) & 1u)) {
+                        const uint32_t lower = (uint32_t)__popc(kBoundaries & ((1u << u) - 1u));  // code below it
+                        const double bound = (double)t * d;                        // exact
+                        const double a = fabs((double)X(i));
+                        const uint32_t code = lower + ((a > bound || (a == bound && (lower & 1u))) ? 1u : 0u);
+                        const uint32_t sh = (uint32_t)(i & 7) * 4u;
+                        if (i < 8) w0 = (w0 & ~(7u << sh)) | (code << sh);
+                        else w1 = (w1 & ~(7u << sh)) | (code << sh);
+                    }
                 }
             }
         }
@@ -167,7 +190,7 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
 #undef X
 }
 
-template <typename T, bool kPlus>
+template <typename T, bool kPlus, bool kShort>
 __global__ void __launch_bounds__(kThreads, 4)
 nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_per_row,
                       int64_t total_units, float ts, uint4* __restrict__ nibbles,
@@ -189,8 +212,8 @@ nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_p
     }
     const float six_ts = __fmul_rn(6.f, ts);
     uint32_t w[4], sb0, sb1, i0, i1;
-    nvfp4_block<T, kPlus>(raw, ts, six_ts, w[0], w[1], sb0, i0);
-    nvfp4_block<T, kPlus>(raw + kWords / 2, ts, six_ts, w[2], w[3], sb1, i1);
+    nvfp4_block<T, kPlus, kShort>(raw, ts, six_ts, w[0], w[1], sb0, i0);
+    nvfp4_block<T, kPlus, kShort>(raw + kWords / 2, ts, six_ts, w[2], w[3], sb1, i1);
     __stcs(nibbles + u, make_uint4(w[0], w[1], w[2], w[3]));
     scales[u] = (uint16_t)(sb0 | (sb1 << 8));
     if (kPlus) bm_index[u] = (uint8_t)(i0 | (i1 << 4));
@@ -260,16 +283,26 @@ cudaError_t launch_nvfp4_quantize(const void* src, mxp_dtype dt, int64_t rows, i
 {
     const int64_t units = rows * (cols / 32);
     const unsigned grid = (unsigned)((units + kThreads - 1) / kThreads);
-#define MXP_NVQ(T, P)                                                                         \
-    nvfp4_quantize_kernel<T, P><<<grid, kThreads, 0, stream>>>(                               \
+#define MXP_NVQ(T, P, S)                                                                      \
+    nvfp4_quantize_kernel<T, P, S><<<grid, kThreads, 0, stream>>>(                            \
         static_cast<const T*>(src), ld_src, cols / 32, units, ts, reinterpret_cast<uint4*>(nibbles), \
         reinterpret_cast<uint16_t*>(scales), bm_index)
+    // short operands: bf16 source, at most 12 significant bits in the tensor scale, and a
+    // scale large enough for value(byte) * ts to stay a normal number (bytes reach down to 2^-9)
+    uint32_t ts_bits;
+    memcpy(&ts_bits, &ts, 4);
+    const bool shortop = dt == MXP_BF16 && (ts_bits & 0xFFFu) == 0u && ts >= 0x1p-100f && ts <= 0x1p100f;
     if (dt == MXP_BF16) {
-        if (plus) MXP_NVQ(__nv_bfloat16, true);
-        else MXP_NVQ(__nv_bfloat16, false);
+        if (shortop) {
+            if (plus) MXP_NVQ(__nv_bfloat16, true, true);
+            else MXP_NVQ(__nv_bfloat16, false, true);
+        } else {
+            if (plus) MXP_NVQ(__nv_bfloat16, true, false);
+            else MXP_NVQ(__nv_bfloat16, false, false);
+        }
     } else {
-        if (plus) MXP_NVQ(float, true);
-        else MXP_NVQ(float, false);
+        if (plus) MXP_NVQ(float, true, false);
+        else MXP_NVQ(float, false, false);
     }
 #undef MXP_NVQ
     return cudaGetLastError();

@@ -176,6 +176,18 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
     d |= (uint64_t)2 << 61;                    // SWIZZLE_128B
     return d;
 }
+// The same for operand rows of 64 bytes with the 64-byte swizzle (16-byte chunk c of row r at
+// chunk c ^ ((r >> 1) & 3)): 8-row groups 512 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(512u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;                    // SWIZZLE_64B
+    return d;
+}
 // Descriptor of a scale-factor atom: 32 rows of 16 bytes, contiguous, no swizzle.
 __device__ __forceinline__ uint64_t smem_desc_sf(uint32_t saddr)
 {
@@ -195,6 +207,7 @@ __host__ __device__ constexpr uint32_t idesc_block_scaled(uint32_t a_fmt, uint32
     return (b_sf_id << 4) | (a_fmt << 7) | (b_fmt << 10) | ((uint32_t)(N >> 3) << 17) |
            (1u << 23) | ((uint32_t)(M >> 4) << 24) | (a_sf_id << 29);
 }
+constexpr uint32_t kIdescSparse = 1u << 2;  // A is stored 2:1 compressed, metadata in TMEM
 
 // D[tmem] (+)= A[smem] * B[smem]^T with per-32 E8M0 scales in TMEM; FP4 operands, K = 64.
 __device__ __forceinline__ void mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
@@ -221,6 +234,31 @@ __device__ __forceinline__ void mma_mxf8f6f4(uint32_t d_tmem, uint64_t a_desc, u
         "[%5], [%6], p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
         : "memory");
+}
+// Sparse form (Sec. 5.2: the residual operand of an MX+ block is almost all zeros): A is stored
+// compressed, 64 of every 128 elements along K -- of each 8 consecutive elements two aligned
+// pairs are kept -- and [meta_tmem] says which: per operand row 64 bits in two TMEM columns,
+// one nibble per group of 8 elements in K order, low two bits = index (0..3) of the first kept
+// pair, high two bits = index of the second, which must be the larger one.  K = 128 per
+// instruction at the cost of the dense K = 64.  kind::mxf4nvf4 with scale_vec::4X is the form
+// whose scales cover 32 elements of the uncompressed K (four E8M0 bytes per row and
+// instruction: a whole TMEM column, scale-factor id 0).  idesc: sparsity flag = bit 2.
+__device__ __forceinline__ void mma_sp_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t meta_tmem, uint32_t idesc, uint32_t sfa_tmem,
+                                            uint32_t sfb_tmem, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, [%7], %3, "
+        "[%5], [%6], p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(meta_tmem)
+        : "memory");
+}
+// 128 rows x 16 bytes of shared memory (row r at 16 r) -> 4 TMEM columns of lanes 0..127.
+__device__ __forceinline__ void tc_cp_128x128b(uint32_t taddr, uint64_t sdesc)
+{
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 // mbarrier arrives once all tcgen05 operations issued so far by this thread are complete.
 __device__ __forceinline__ void tc_commit(uint64_t* bar)
@@ -395,6 +433,22 @@ __device__ __forceinline__ void mma_mxf8f6f4_2cta(uint32_t d_tmem, uint64_t a_de
         "[%5], [%6], p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
         : "memory");
+}
+__device__ __forceinline__ void mma_sp_mxf4_2cta(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                 uint32_t meta_tmem, uint32_t idesc, uint32_t sfa_tmem,
+                                                 uint32_t sfb_tmem, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, [%7], %3, "
+        "[%5], [%6], p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(meta_tmem)
+        : "memory");
+}
+__device__ __forceinline__ void tc_cp_128x128b_2cta(uint32_t taddr, uint64_t sdesc)
+{
+    asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 __device__ __forceinline__ void tc_cp_sf_2cta(uint32_t taddr, uint64_t sdesc)
 {

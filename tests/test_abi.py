@@ -100,10 +100,12 @@ def test_argument_validation_of_the_later_entry_points(lib):
     b6 = _Packed(4096, 4096, None, 32, 256, 3)
     assert ch(1, 32, 256, fake, 256, ctypes.byref(b6), fake, 1, 32, null, null) == 1  # 6-bit weights
     dp = lib.mxp_gemm_dense_prepacked
-    assert dp(70, 32, 256, null, 256, ctypes.byref(b), fake, fake, 1, 32, fake, 1 << 20, null) == 1  # no activations
-    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), null, fake, 1, 32, fake, 1 << 20, null) == 1  # no prepacked copy
-    assert dp(70, 32, 256, fake, 256, ctypes.byref(b6), fake, fake, 1, 32, fake, 1 << 20, null) == 1  # 6-bit weights
-    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), fake, fake, 1, 32, fake, 16, null) == 3       # workspace
+    wide32 = lib.mxp_gemm_prepack_bytes(32, 256, 1)
+    assert dp(70, 32, 256, null, 256, ctypes.byref(b), fake, wide32, fake, 1, 32, fake, 1 << 20, null) == 1  # no activations
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), null, wide32, fake, 1, 32, fake, 1 << 20, null) == 1  # no prepacked copy
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b6), fake, wide32, fake, 1, 32, fake, 1 << 20, null) == 1  # 6-bit weights
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), fake, wide32, fake, 1, 32, fake, 16, null) == 3       # workspace
+    assert dp(70, 32, 256, fake, 256, ctypes.byref(b), fake, wide32 - 1024, fake, 1, 32, fake, 1 << 20, null) == 1  # copy of another size
     assert lib.mxp_gemm_dense_prepacked_workspace_bytes(70, 256) > 70 * 256 * 2
     assert lib.mxp_gemm_dense_prepacked_workspace_bytes(70, 96) == 0
     # the ordering rule runs on the host
@@ -114,3 +116,44 @@ def test_argument_validation_of_the_later_entry_points(lib):
     assert sorted(out.tolist()) == list(range(64)) and out[0] == 63 and out[32] == 62
     assert co(cnt.ctypes.data, 48, out.ctypes.data) == 1
     assert co(null, 64, out.ctypes.data) == 1
+
+
+def test_prepacked_copies_are_checked_against_the_call(lib):
+    # A prepacked weight copy is a bare device pointer: the calls that read one take its size and
+    # refuse, before any launch, a copy made for another shape or for another pairing of operand
+    # modes (a plain copy under an MXFP4+ partner would otherwise be read far past its end).
+    from paper_2510_14557_b200.binding import _Packed
+    null = None
+    fake = ctypes.c_void_p(4096)
+    M, N, K = 512, 384, 256
+    MX, MXP = 0, 1
+    PLAIN, WIDE, SPLIT = 0, 1, 2
+    form = lib.mxp_gemm_prepack_form
+    assert (form(MX, MX), form(MXP, MX), form(MX, MXP), form(MXP, MXP)) == (PLAIN, PLAIN, SPLIT, WIDE)
+    assert form(2, MX) == WIDE and form(MX, 2) == WIDE          # MX++ is read widened
+    size = {f: lib.mxp_gemm_prepack_bytes(N, K, f) for f in (PLAIN, WIDE, SPLIT)}
+    assert 0 < size[PLAIN] < size[SPLIT] < size[WIDE]
+    assert lib.mxp_gemm_prepack_bytes(N, K, 3) == 0 and lib.mxp_gemm_prepack_bytes(N, 96, WIDE) == 0
+    ws = 1 << 30
+    gp = lib.mxp_gemm_prepacked
+
+    def call(amode, bmode, nbytes, n=N):
+        a = _Packed(4096, 4096, 4096, M, K, amode)
+        b = _Packed(4096, 4096, 4096, n, K, bmode)
+        return gp(M, n, K, ctypes.byref(a), ctypes.byref(b), fake, nbytes, fake, 1, n, fake, ws, null)
+
+    for amode, bmode in ((MX, MX), (MXP, MX), (MX, MXP), (MXP, MXP)):
+        right = form(amode, bmode)
+        for f in (PLAIN, WIDE, SPLIT):
+            if f != right:
+                assert call(amode, bmode, size[f]) == 1, (amode, bmode, f)
+        assert call(amode, bmode, lib.mxp_gemm_prepack_bytes(N + 128, K, right)) == 1  # another shape's copy
+    gr = lib.mxp_gemm_ready
+    a = _Packed(4096, 4096, 4096, M, K, MXP)
+    b = _Packed(4096, 4096, 4096, N, K, MX)
+    assert gr(M, N, K, ctypes.byref(a), ctypes.byref(b), fake, size[PLAIN], fake, 1, N, fake, ws, null) == 1
+    # mxp_gemm_prepack: the form must fit the operand's mode
+    pk = lib.mxp_gemm_prepack
+    assert pk(ctypes.byref(a), PLAIN, fake, ws, null) == 1      # an MXFP4+ operand has no plain form
+    assert pk(ctypes.byref(b), SPLIT, fake, ws, null) == 1      # a plain operand has nothing to split
+    assert pk(ctypes.byref(a), 7, fake, ws, null) == 1

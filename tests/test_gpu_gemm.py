@@ -20,8 +20,9 @@ def mxp():
 def force():
     """Forces a kernel choice for the duration of a test (mxp_debug_override)."""
     m = mxp()
-    knobs = {"inplace": m.KNOB_INPLACE_KERNEL, "halves": m.KNOB_STREAM_HALVES, "weight_only": m.KNOB_WEIGHT_ONLY_KERNEL}
-    names = {"single": 1, "pair": 2, "old": 1, "stream": 2, "1": 1, "2": 2}
+    knobs = {"inplace": m.KNOB_INPLACE_KERNEL, "halves": m.KNOB_STREAM_HALVES, "weight_only": m.KNOB_WEIGHT_ONLY_KERNEL,
+             "one_sided": m.KNOB_ONE_SIDED}
+    names = {"single": 1, "pair": 2, "old": 1, "stream": 2, "1": 1, "2": 2, "wide": 1}
     used = []
 
     def set_(knob, value):
@@ -406,8 +407,7 @@ def test_tc_prepacked_weights_match_mxp_gemm(M, N, K, amode, bmode):
     ap, da = _raw_operand(M, K, amode, seed=M + 1)
     bp, db = _raw_operand(N, K, bmode, seed=N + 2)
     m = mxp()
-    wide = amode == MXP or bmode == MXP
-    pre = m.mxp_gemm_prepack(bp, wide)
+    pre = m.mxp_gemm_prepack(bp, m.mxp_gemm_prepack_form(amode, bmode))
     for dt in (torch.float32, torch.bfloat16):
         d0 = m.mxp_gemm(ap, bp, out_dtype=dt)
         d1 = m.mxp_gemm_prepacked(ap, bp, pre, out_dtype=dt)

@@ -130,12 +130,18 @@ def test_rounding_boundaries_bit_exact(plus):
         ref = oracle.nvfp4_quantize(x, ts, plus)
         got = mxp().mxp_nvfp4_quantize(to_dev(x), ts, plus)
         check_planes(got, ref, plus)
-    # bf16 sources: boundaries t * d that bf16 holds (power-of-two tensor scale)
-    x = nvfp4_boundary_blocks(2.0 ** -3, 9)
-    bits = synth.f32_to_bf16_bits(x)
-    ref = oracle.nvfp4_quantize(bits, 2.0 ** -3, plus, bf16_bits=True)
-    got = mxp().mxp_nvfp4_quantize(to_dev_bf16(bits), 2.0 ** -3, plus)
-    check_planes(got, ref, plus)
+    # bf16 sources: boundaries t * d that bf16 holds.  Tensor scales of up to 12 significant bits
+    # take the kernel's short-operand form (quotient by a Newton step, no per-element settling),
+    # longer ones the general form; signed zeros and tiny elements keep their sign in both.
+    for ts, seed in ((2.0 ** -3, 9), (0.75, 10), (2867.0 / 4096.0, 11), (1.0 + 2.0 ** -11, 12),
+                     (1.0 + 2.0 ** -12, 13), (3.0 * 2.0 ** -40, 14)):
+        x = nvfp4_boundary_blocks(ts, seed)
+        x[::7, 3] = -0.0
+        x[::5, 11] = np.float32(-2.0 ** -120)
+        bits = synth.f32_to_bf16_bits(x)
+        ref = oracle.nvfp4_quantize(bits, ts, plus, bf16_bits=True)
+        got = mxp().mxp_nvfp4_quantize(to_dev_bf16(bits), ts, plus)
+        check_planes(got, ref, plus)
 
 
 def test_config2_whole_matrix_and_argument_checks():
