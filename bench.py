@@ -538,7 +538,8 @@ def targets(mxp, synth, peaks):
     del x
     # ---- config 3: decode GEMM, eight rotating weight copies (> L2), graphs of eight launches.
     # "tc": weights re-tiled once, FP4 tensor path (mxp_gemm_decode_prepacked); "reg": the
-    # streamed register-decode kernel behind mxp_gemm, launches chained.
+    # streamed register-decode kernel behind mxp_gemm; both as chains of programmatic dependents
+    # (constant weights), which is what a captured decode loop can use.
     a16, w_bits = synth.config3(16)
     w = dev_bf16(w_bits)
     N, K = w.shape
@@ -556,7 +557,7 @@ def targets(mxp, synth, peaks):
             tot = wbytes + M * K * 2 + M * N * 2
 
             def run_tc():
-                mxp.mxp_gemm_decode_prepacked(a, tiled[st["i"] % 8], out=d, workspace=ws)
+                mxp.mxp_gemm_decode_prepacked(a, tiled[st["i"] % 8], out=d, workspace=ws, chained=True)
                 st["i"] += 1
 
             def run_reg():

@@ -27,6 +27,15 @@
 //     weights.  (Converting inside the GEMM, every CTA for itself, was built and measured: the
 //     conversion is ~500 instructions per eight elements and costs a CTA 4 us per activation
 //     row, more than the second launch.)
+//   * One or two activation rows (kSelf): the dependent chain "kernel before -> conversion
+//     kernel -> this kernel's copies of the images" costs ~4 us of a ~10 us call, more than
+//     the conversion itself.  There every CTA converts the rows for itself, straight into
+//     shared memory where the images of all stages stay (40 KB at K = 4096), while its weights
+//     are already streaming: one launch per call, and no image travels through global memory.
+//     (The BM's lower part stays on the tensor cores there too: adding (BM_L 2^shared_exp)
+//     a[k_BM] per block on the CUDA cores from the record byte, the scale byte and the raw
+//     activation was built and measured -- twelve warps need ~0.45 us per stage for it, three
+//     dependent shared-memory loads per record, against ~0.15 us for the four extra MMAs.)
 //   * warp 0 issues the weight copies (the first ring-full before the CTA's set-up barrier),
 //     warp 1 the activation copies, warps 2-5 the MMAs (each every fourth stage, with an
 //     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 build the BM_L
@@ -58,7 +67,9 @@ constexpr int kMaxStages = 16;
 constexpr long long kWaitLimit = 4000000000ll;
 constexpr size_t kSmemMax = 227 * 1024;
 constexpr uint32_t kMagic = 0x4D58D0C1u;
+}  // namespace
 constexpr size_t kHeaderBytes = 256;
+namespace {
 
 // Rows of the activation operand: five planes per activation row, padded to the MMA's N.
 __host__ __device__ constexpr int act_rows(int M) { return (kPlanes * M + 15) / 16 * 16; }
@@ -95,17 +106,38 @@ struct PrepackHeader {
 // Shared memory of the GEMM kernel (bytes from the 1024-byte aligned base).
 // A slot holds a stage's weight image, its activation image (codes at act_off, scale atoms
 // behind) and, for MX+, the BM_L tile built from the image's records (at res_off).
+// kSelf form (self_nst > 0: number of stages whose activation images stay resident): a slot
+// holds the weight image and, for MX+, the BM_L tile; behind the ring come the images' code
+// tiles (2 KB a stage) and their scale atoms (512 bytes a stage).
 struct DecodeLayout {
     size_t act_off, res_off, slot, bars, total;
+    size_t img_codes, img_sf;  // kSelf only
     int stages;
 };
-__host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages)
+constexpr int kSelfMaxM = 2;
+__host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages,
+                                                      int self_nst = 0)
 {
     DecodeLayout l;
+    l.stages = stages;
+    l.img_codes = l.img_sf = 0;
+    if (self_nst > 0) {
+        l.act_off = 0;
+        l.res_off = up(wimg, 1024);
+        l.slot = l.res_off + (plus ? up((size_t)rows * 128, 1024) : 0);
+        const size_t last = (size_t)(stages - 1) * l.slot + (plus ? l.res_off : 0) + 128 * 128;  // (see below)
+        size_t o = up(last > (size_t)stages * l.slot ? last : (size_t)stages * l.slot, 1024);
+        l.img_codes = o;
+        o += (size_t)self_nst * 2048;
+        l.img_sf = o;
+        o += (size_t)self_nst * 512;
+        l.bars = up(o, 16);
+        l.total = l.bars + 1024 + 1024;
+        return l;
+    }
     l.act_off = up(wimg, 1024);
     l.res_off = up(l.act_off + (size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact), 1024);
     l.slot = l.res_off + (plus ? up((size_t)rows * 128, 1024) : 0);
-    l.stages = stages;
     // an MMA reads 128 rows of 128 bytes from the start of a tile that holds fewer: what follows
     // the last tile must exist (any bytes are finite E2M1 codes; the rows are never read back)
     size_t off = up((size_t)stages * l.slot + 16384, 16);
@@ -114,10 +146,29 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
     return l;
 }
 
+#ifdef MXP_DECODE_TIMELINE  // measurement build: per-CTA stamps of the phases, read back by a probe
+__device__ unsigned long long g_decode_tl[8 * 256 * 8];   // [launch key][CTA][phase]
+__device__ const void* g_decode_tl_keys[8];                // weight buffers of the launches to tell apart
+__device__ unsigned long long g_decode_tl2[256 * 64];      // [CTA][event]: per-stage stamps of one role
+#define MXP_TL(slot)                                                                              \
+    do {                                                                                          \
+        int key_ = 0;                                                                             \
+        for (int k_ = 0; k_ < 8; ++k_)                                                            \
+            if (g_decode_tl_keys[k_] == (const void*)prm.wimg) key_ = k_;                         \
+        g_decode_tl[(key_ * 256 + blockIdx.x) * 8 + (slot)] = ptx::globaltimer_ns();              \
+    } while (0)
+#else
+#define MXP_TL(slot) do { } while (0)
+#endif
+
+
 struct DecodeParams {
     int M, N;
+    const __nv_bfloat16* A;  // kSelf: the activations, row stride lda
+    int64_t lda;
+    int clear_status;      // kSelf: this launch clears the status block (no kernel ahead of it does)
     const uint8_t* wimg;   // weight images [cta][tile][stage]
-    const uint8_t* aimg;   // activation images [stage]
+    const uint8_t* aimg;   // activation images [stage] (not kSelf)
     void* D;
     int64_t ldd;
     StatusBlock* status;   // may be nullptr
@@ -233,7 +284,9 @@ __device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, in
     // t = |a| / 2^(E - 12), rounded to an integer below 2^13, plus 4 in each of five octal
     // places: octal digit j of t, minus 4, is the balanced digit d_j in -4..3 with
     // |a| = sum_j d_j 2^(E - 3 j)
-    uint32_t t[8], neg = 0u;
+    // The digit's code comes from a table of eight nibbles indexed by the octal digit (sign bit =
+    // the element's sign, flipped for the negative digits 0..3): E2M1 codes of 4 3 2 1 0 1 2 3.
+    uint32_t t[8], lut[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         const uint32_t h = (e & 1) ? x[e >> 1] >> 16 : x[e >> 1] & 0xFFFFu;
@@ -241,7 +294,7 @@ __device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, in
         const uint32_t m13 = ((ef ? 128u : 0u) | (h & 127u)) << 5;  // at the block's largest exponent
         const uint32_t down = min(eb - max(ef, 1u), 31u);           // binades below it
         t[e] = ((m13 + ((1u << down) >> 1)) >> down) + 0x4924u;     // rounded to nearest
-        neg |= (h >> 15) << e;
+        lut[e] = (h & 0x8000u) ? 0xDCA82456u : 0x5420ACDEu;
     }
 #pragma unroll
     for (int j = 0; j < kPlanes; ++j) {
@@ -250,11 +303,8 @@ __device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, in
         if (sbyte >= 0 && !nonfinite) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const int d = (int)((t[e] >> (3 * (4 - j))) & 7u) - 4;
-                const uint32_t ad = (uint32_t)(d < 0 ? -d : d);
-                const uint32_t code = (0x65420u >> (4u * ad)) & 7u;  // E2M1 codes of 0 1 2 3 4
-                const uint32_t sg = ((neg >> e) & 1u) ^ (d < 0 ? 1u : 0u);
-                w |= (code | (sg << 3)) << (4 * e);
+                const uint32_t sh4 = (j < 4 ? t[e] >> (3 * (4 - j) - 2) : t[e] << 2) & 28u;  // 4 x octal digit j
+                w |= ((lut[e] >> sh4) & 15u) << (4 * e);
             }
         }
         const int row = kPlanes * m + j;
@@ -304,17 +354,18 @@ decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int n
 // ------------------------------------------------------------------------------------------
 // The GEMM.  kNact: rows of the activation operand (16 .. 80); kPlus: MXFP4+ weights.
 // ------------------------------------------------------------------------------------------
-template <int kNact, bool kPlus, typename OutT>
+template <int kNact, bool kPlus, bool kSelf, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_decode_tc_kernel(const DecodeParams prm)
 {
+    static_assert(!kSelf || kNact == 16, "self-converted activations: at most two rows");
     constexpr int kSfb = sfb_bytes(kNact);
-    constexpr int kMt = kNact / kPlanes;  // activation rows the operand can hold
+    constexpr int kMt = kSelf ? kSelfMaxM : kNact / kPlanes;  // activation rows the operand can hold
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int S = prm.stages;
     const int nst = prm.nst;
-    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S);
+    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S, kSelf ? nst : 0);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // the slot's copies landed
     uint64_t* empty = full + kMaxStages;       // the slot's MMAs are done
     uint64_t* res_full = empty + kMaxStages;   // the slot's BM_L tile is written
@@ -332,8 +383,9 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     const uint8_t* wsrc = prm.wimg + (size_t)blockIdx.x * prm.tiles * nst * prm.wimg_bytes;
 
     if (threadIdx.x == 0) {
+        MXP_TL(0);  // kernel entry
         for (int s = 0; s < kMaxStages; ++s) {
-            ptx::mbar_init(&full[s], 2);
+            ptx::mbar_init(&full[s], kSelf ? 1 : 2);
             ptx::mbar_init(&empty[s], 1);
             ptx::mbar_init(&res_full[s], kResWarps);
         }
@@ -341,9 +393,14 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         ptx::mbar_init(acc_empty, 4);
         *abort = 0u;
         ptx::fence_mbar_init();
-        // The first ring-full of weight copies goes out before anything else: the weights do not
-        // depend on the kernel before, and every later step of the set-up overlaps their latency.
-        for (uint32_t c = 0; c < total && c < (uint32_t)S; ++c) {
+    }
+    if (warp == 0) {
+        // The first ring-full of weight copies goes out before anything else, a lane each: the
+        // weights do not depend on the kernel before, and every later step of the set-up
+        // overlaps their latency.
+        __syncwarp();
+        const uint32_t c = (uint32_t)lane;
+        if (c < total && c < (uint32_t)S) {
             ptx::mbar_arrive_expect_tx(&full[c], prm.wimg_bytes);
             bulk_g2s(slot((int)c), wsrc + (size_t)c * prm.wimg_bytes, prm.wimg_bytes, &full[c]);
         }
@@ -352,11 +409,41 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         ptx::tmem_alloc(tmem_slot, kTmemCols);
         ptx::tmem_relinquish();
     }
+    if (kSelf) {
+        // the images' unused rows: zero codes under a finite scale (the rows in use land on top)
+        for (int i = threadIdx.x; i < nst * 128; i += kThreads)
+            reinterpret_cast<uint4*>(smem + L.img_codes)[i] = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = threadIdx.x; i < nst * 32; i += kThreads)
+            reinterpret_cast<uint4*>(smem + L.img_sf)[i] =
+                make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     ptx::grid_launch_dependents();  // whatever follows on the stream may be scheduled
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) MXP_TL(1);  // set-up done
+    if (kSelf) {
+        // Activations -> digit planes, by this CTA for itself: a quad of lanes per block of 32,
+        // eight elements per lane, straight into the resident images.  A, D and the status block
+        // are in stream order from here on.
+        ptx::grid_dependency_wait();
+        if (prm.clear_status && blockIdx.x == 0 && threadIdx.x == 0 && prm.status != nullptr) {
+            prm.status->code = 0u;
+            prm.status->where = 0u;
+        }
+        for (int i = threadIdx.x; i < prm.M * nst * 32; i += kThreads) {
+            const int m = i / (nst * 32), rem = i - m * nst * 32;
+            const int st = rem >> 5, kb = (rem >> 2) & 7, qd = rem & 3;
+            const int64_t k0 = (int64_t)st * kStageK + kb * 32 + qd * 8;
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + k0));
+            convert_quarter(v, m, kb, qd, smem + L.img_codes + (size_t)st * 2048, smem + L.img_sf + (size_t)st * 512,
+                            kSfb);
+        }
+        ptx::fence_proxy_async_smem();  // the MMAs read the images through the async proxy
+        __syncthreads();
+        if (threadIdx.x == 0) MXP_TL(2);  // activations available
+    }
 
     if (warp == 0) {
         // ---------------------------------------------------------------- weight copies (the rest)
@@ -373,8 +460,9 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- activation copies
-        if (lane == 0) {
+        if (!kSelf && lane == 0) {
             ptx::grid_dependency_wait();  // the activation images are the preceding kernel's output
+            MXP_TL(2);  // activations available
             constexpr uint32_t kBytes = kNact * 128 + 2 * kSfb;
             for (uint32_t c = 0; c < total; ++c) {
                 const int s = c % S;
@@ -412,11 +500,18 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     break;
                 }
                 ptx::tc_fence_after_sync();
+#ifdef MXP_DECODE_TIMELINE
+                if (lane == 0 && st < 32) g_decode_tl2[blockIdx.x * 64 + 32 + st] = ptx::globaltimer_ns();
+#endif
+                if (lane == 0 && cc == 0) MXP_TL(3);          // first stage landed
+                if (lane == 0 && cc == total - 1) MXP_TL(4);  // last stage landed
                 const uint8_t* sl = slot(s);
                 const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(sl));
-                const uint64_t db = ptx::smem_desc_sw128(ptx::smem_u32(sl + L.act_off));
+                const uint64_t db = ptx::smem_desc_sw128(
+                    ptx::smem_u32(kSelf ? smem + L.img_codes + (size_t)st * 2048 : sl + L.act_off));
                 const uint32_t sfa = ptx::smem_u32(sl + (size_t)prm.rows * 128);
-                const uint32_t sfb = ptx::smem_u32(sl + L.act_off + kNact * 128);
+                const uint32_t sfb =
+                    ptx::smem_u32(kSelf ? smem + L.img_sf + (size_t)st * 512 : sl + L.act_off + kNact * 128);
                 const uint32_t t_sf = tmem_base + kTmemSf + 16u * (uint32_t)iss;
                 if (ptx::elect_one()) {
 #pragma unroll
@@ -481,6 +576,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 break;
             }
             ptx::tc_fence_after_sync();
+            if (warp == kRowWarp0 && lane == 0 && t == ntl - 1) MXP_TL(5);  // all MMAs done
             float o[kMt];
 #pragma unroll
             for (int m = 0; m < kMt; ++m) o[m] = 0.f;
@@ -559,6 +655,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
 
     // ---------------------------------------------------------------------- teardown
     __syncthreads();
+    if (threadIdx.x == 0) MXP_TL(6);  // output stored
     if (*abort != 0u && threadIdx.x == 0) {
         // after a timeout, copies may still be in flight into this CTA's shared memory: give
         // them (bounded) time to land before the CTA leaves
@@ -576,18 +673,19 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     }
 }
 
-// Ring slots that fit: a multiple of four (see the issuers), at most sixteen.
-int pick_stages(const DecodePlan& p, int nact, bool plus)
+// Ring slots that fit: a multiple of four (see the issuers), at most sixteen.  self_nst > 0: the
+// form with resident activation images.
+int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0)
 {
     for (int s = kMaxStages; s >= 4; s -= 4)
-        if (decode_layout(p.rows, p.wimg, nact, plus, s).total <= kSmemMax) return s;
+        if (decode_layout(p.rows, p.wimg, nact, plus, s, self_nst).total <= kSmemMax) return s;
     return 0;
 }
 
-template <int kNact, bool kPlus, typename OutT>
-cudaError_t launch(const DecodeParams& prm, int ctas, size_t smem, cudaStream_t stream)
+template <int kNact, bool kPlus, bool kSelf, typename OutT>
+cudaError_t launch(const DecodeParams& prm, int ctas, size_t smem, bool dependent, cudaStream_t stream)
 {
-    auto kern = gemm_decode_tc_kernel<kNact, kPlus, OutT>;
+    auto kern = gemm_decode_tc_kernel<kNact, kPlus, kSelf, OutT>;
     static SmemAttrOnce once;
     cudaError_t e = ensure_dynamic_smem(kern, (int)kSmemMax, once);
     if (e != cudaSuccess) return e;
@@ -600,21 +698,41 @@ cudaError_t launch(const DecodeParams& prm, int ctas, size_t smem, cudaStream_t 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    // A grid that may start before the kernel ahead of it has finished: always behind this
+    // library's own conversion kernel; behind a caller's kernel only on the caller's promise.
+    cfg.numAttrs = dependent ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kern, prm);
 }
 
-template <int kNact>
-cudaError_t launch_n(bool plus, bool f32, const DecodeParams& prm, int ctas, size_t smem, cudaStream_t stream)
+template <int kNact, bool kSelf>
+cudaError_t launch_n(bool plus, bool f32, const DecodeParams& prm, int ctas, size_t smem, bool dependent,
+                     cudaStream_t stream)
 {
     if (plus)
-        return f32 ? launch<kNact, true, float>(prm, ctas, smem, stream)
-                   : launch<kNact, true, __nv_bfloat16>(prm, ctas, smem, stream);
-    return f32 ? launch<kNact, false, float>(prm, ctas, smem, stream)
-               : launch<kNact, false, __nv_bfloat16>(prm, ctas, smem, stream);
+        return f32 ? launch<kNact, true, kSelf, float>(prm, ctas, smem, dependent, stream)
+                   : launch<kNact, true, kSelf, __nv_bfloat16>(prm, ctas, smem, dependent, stream);
+    return f32 ? launch<kNact, false, kSelf, float>(prm, ctas, smem, dependent, stream)
+               : launch<kNact, false, kSelf, __nv_bfloat16>(prm, ctas, smem, dependent, stream);
 }
 
 }  // namespace
+
+#ifdef MXP_DECODE_TIMELINE
+extern "C" int mxp_decode_timeline_read(unsigned long long* host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_decode_tl, sizeof(unsigned long long) * (size_t)n);
+}
+extern "C" int mxp_decode_timeline_read2(unsigned long long* host, int n)
+{
+    return (int)cudaMemcpyFromSymbol(host, g_decode_tl2, sizeof(unsigned long long) * (size_t)n);
+}
+extern "C" int mxp_decode_timeline_keys(const void* const* prepacked8)
+{
+    const void* keys[8];
+    for (int i = 0; i < 8; ++i) keys[i] = static_cast<const char*>(prepacked8[i]) + mxp::kHeaderBytes;
+    return (int)cudaMemcpyToSymbol(g_decode_tl_keys, keys, sizeof(keys));
+}
+#endif
 
 size_t decode_prepack_bytes(int64_t N, int64_t K, mxp_mode mode)
 {
@@ -670,13 +788,19 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     const size_t need = decode_workspace_bytes(M, K);
     if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
     const int nact = act_rows((int)M);
-    const int stages = pick_stages(p, nact, plus);
+    // one or two rows: every CTA converts them for itself, if their images fit beside a ring
+    const int self_stages = M <= kSelfMaxM ? pick_stages(p, nact, plus, p.nst) : 0;
+    const bool self = self_stages != 0;
+    const int stages = self ? self_stages : pick_stages(p, nact, plus);
     if (stages == 0) return MXP_ERR_UNSUPPORTED;
-    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages);
+    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages, self ? p.nst : 0);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     DecodeParams prm = {};
     prm.M = (int)M;
     prm.N = (int)N;
+    prm.A = static_cast<const __nv_bfloat16*>(A);
+    prm.lda = lda;
+    prm.clear_status = chained ? 0 : 1;
     prm.wimg = static_cast<const uint8_t*>(b_prepacked) + kHeaderBytes;
     prm.aimg = ws + kStatusBytes;
     prm.D = D;
@@ -687,6 +811,11 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     prm.nst = p.nst;
     prm.stages = stages;
     prm.wimg_bytes = p.wimg;
+    const bool f32 = d_dt == MXP_F32;
+    if (self) {  // one launch; a programmatic dependent only on the caller's promise
+        const cudaError_t e = launch_n<16, true>(plus, f32, prm, p.ctas, L.total, chained, stream);
+        return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+    }
     {   // activations -> digit planes; in a chain it may start while the kernel before drains
         // (same shared-memory carve-out as the GEMM, so that the SMs are not reconfigured
         // between the two kernels of every call: that alone cost 1.6 us per call)
@@ -711,14 +840,13 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
                                            (int)M, nact, ws + kStatusBytes, prm.status, chained ? 0 : 1);
         if (e != cudaSuccess) return MXP_ERR_CUDA;
     }
-    const bool f32 = d_dt == MXP_F32;
     cudaError_t e;
     switch (nact) {
-        case 16: e = launch_n<16>(plus, f32, prm, p.ctas, L.total, stream); break;
-        case 32: e = launch_n<32>(plus, f32, prm, p.ctas, L.total, stream); break;
-        case 48: e = launch_n<48>(plus, f32, prm, p.ctas, L.total, stream); break;
-        case 64: e = launch_n<64>(plus, f32, prm, p.ctas, L.total, stream); break;
-        default: e = launch_n<80>(plus, f32, prm, p.ctas, L.total, stream); break;
+        case 16: e = launch_n<16, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 32: e = launch_n<32, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 48: e = launch_n<48, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 64: e = launch_n<64, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        default: e = launch_n<80, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
     }
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }
