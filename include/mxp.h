@@ -180,7 +180,9 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  * Exactly one of A_dense_bf16 / A_packed is non-NULL:
  *   - A_dense_bf16 (device, bf16, row stride lda elements): weight-only form, the
  *     weights B are decoded inside the kernel and multiplied with bf16 activations
- *     (up to 64 rows: streamed decode kernels, no workspace needed; more rows, given
+ *     (up to 64 rows: streamed decode kernels, no workspace needed -- they bring each chunk of
+ *     256 activations into half-precision range by a power of two, so an activation more than
+ *     2^28 below the largest of its chunk is rounded at 2^-39 of that largest one; more rows, given
  *     mxp_gemm_workspace_bytes(..., a_dense = 1, ...) bytes of workspace: the tensor-core
  *     kernel, the activations entering as the exact sum of two E4M3 planes with a
  *     power-of-two scale per block of 32 -- elements more than 2^9 below their block's
@@ -441,8 +443,17 @@ mxp_status mxp_tensor_peak_probe(int kind, int iters, double *ms, double *flops)
  * mxp_gemm.  A problem whose workspace need exceeds those 4096 bytes is rejected with
  * MXP_ERR_WORKSPACE before anything is launched.
  *
+ * With so little scratch the call always runs the kernels that work on the packed planes in
+ * place (Eq. 4 / Algorithm 1 with dense residual passes), never the faster ones that first
+ * prepare the operands in a workspace: on the 8192 x 28672 x 8192 prefill shape about 0.89 ms
+ * for MXFP4 x MXFP4 against 0.68 ms, 1.8 ms for one MXFP4+ operand against 0.95 ms, and
+ * 2.6 ms for two against 1.3 ms.  MX++ and the 6- and 8-bit modes need the workspace forms:
+ * MXP_ERR_UNSUPPORTED here.
+ *
  * The first call on a device looks up the array's device address (with that device
- * current) and remembers it; make that first call outside any stream capture.
+ * current) and remembers it; make that first call outside any stream capture.  The
+ * remembered address belongs to the device's context: after cudaDeviceReset the library
+ * must be reloaded before this entry point is used again.
  * All calls on a device share the one array and it keeps what the previous call left:
  * the status block is cleared on `cuda_stream` at the start of every call, but two calls
  * whose kernels overlap on the GPU (different streams) race on it; serialise them.

@@ -50,18 +50,27 @@ extern "C" mxp_status mxp_gemm_noalloc(int64_t M, int64_t N, int64_t K, const mx
     if (d_dt != MXP_F32 && d_dt != MXP_BF16) return MXP_ERR_INVALID_ARG;
     if (A_packed == nullptr || B_packed == nullptr) return MXP_ERR_INVALID_ARG;
     for (const mxp_packed* p : {A_packed, B_packed}) {
-        if (p->mode == MXP_MODE_MXFP4_PP) return MXP_ERR_UNSUPPORTED;  // needs the prepacked path
-        if (p->mode != MXP_MODE_MXFP4 && p->mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_INVALID_ARG;
-        if (p->cols != K || p->nibbles == nullptr || p->scales == nullptr) return MXP_ERR_INVALID_ARG;
-        if (reinterpret_cast<uintptr_t>(p->nibbles) % 16 != 0) return MXP_ERR_INVALID_ARG;
-        if (p->mode == MXP_MODE_MXFP4_PLUS && p->bm_index == nullptr) return MXP_ERR_INVALID_ARG;
+        if (p->mode < MXP_MODE_MXFP4 || p->mode > MXP_MODE_MXFP8_PLUS) return MXP_ERR_INVALID_ARG;
+        if (p->rows < 0 || p->cols != K) return MXP_ERR_INVALID_ARG;
+        if (p->rows > 0 && p->cols > 0) {  // an empty operand needs no planes (as for mxp_gemm)
+            if (p->nibbles == nullptr || p->scales == nullptr) return MXP_ERR_INVALID_ARG;
+            if (reinterpret_cast<uintptr_t>(p->nibbles) % 16 != 0) return MXP_ERR_INVALID_ARG;
+            if (p->mode != MXP_MODE_MXFP4 && p->mode != MXP_MODE_MXFP6 && p->mode != MXP_MODE_MXFP8 &&
+                p->bm_index == nullptr)
+                return MXP_ERR_INVALID_ARG;
+        }
     }
     if (A_packed->rows != M || B_packed->rows != N) return MXP_ERR_INVALID_ARG;
+    if (M > 0 && N > 0) {
+        if (K == 0) return MXP_ERR_UNSUPPORTED;
+        if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(D) % (d_dt == MXP_BF16 ? 2 : 4) != 0) return MXP_ERR_INVALID_ARG;
+        // MX++ and the 6- and 8-bit modes run only on operands prepared in a workspace
+        if (A_packed->mode > MXP_MODE_MXFP4_PLUS || B_packed->mode > MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
+    }
+    // every argument is acceptable from here on: only now is the out-parameter touched
     if (kernel_status != nullptr) *kernel_status = MXP_OK;
     if (M == 0 || N == 0) return MXP_OK;
-    if (K == 0) return MXP_ERR_UNSUPPORTED;
-    if (D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(D) % (d_dt == MXP_BF16 ? 2 : 4) != 0) return MXP_ERR_INVALID_ARG;
 
     // the scratch this problem needs must fit the array the library carries
     const size_t need = mxp::tc_compact_workspace_bytes();

@@ -106,8 +106,10 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
     }
     // scale byte: E4M3 nearest to amax / (6 ts)
     const float q = __fdiv_rn(amax, six_ts);
-    uint32_t sb = f32_to_e4m3_byte(__fmul_rn(q, kDown));
-    const uint32_t sb_up = f32_to_e4m3_byte(__fmul_rn(q, kUp));
+    // (short operands: 6 ts is exact, the division is correctly rounded, and a quotient that is
+    // not exactly on a boundary between two bytes is at least 2^-21 of it away: one cast decides)
+    uint32_t sb = f32_to_e4m3_byte(kShort ? q : __fmul_rn(q, kDown));
+    const uint32_t sb_up = kShort ? sb : f32_to_e4m3_byte(__fmul_rn(q, kUp));
     if (sb != sb_up) {  // a boundary between the bytes sb and sb + 1 (never at saturation)
         const float t = 0.5f * (e4m3_byte_to_f32(sb) + e4m3_byte_to_f32(sb_up));  // exact
         const double bound = (double)t * 6.0 * (double)ts;                        // exact
@@ -167,13 +169,23 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
             }
         }
     }
-    const float r_dn = __fmul_rn(r, kDown), r_up = __fmul_rn(r, kUp);
     index = 0;
     if (kPlus && sb > 2u) {
-        const float v_dn = fminf(fmaxf(__fmul_rn(amax, r_dn), 4.f), 8.f);
-        const float v_up = fminf(fmaxf(__fmul_rn(amax, r_up), 4.f), 8.f);
-        uint32_t m = (uint32_t)__float2int_rn((v_dn - 4.f) * 2.f);  // 0..8
-        const uint32_t m_up = (uint32_t)__float2int_rn((v_up - 4.f) * 2.f);
+        uint32_t m, m_up;
+        if (kShort) {
+            // amax / d by the same Newton step as the elements: exact whenever it is representable,
+            // and otherwise at least 2^-20 of a boundary 4.25 + m / 2 away from it
+            const float d32 = __fmul_rn(e, ts);
+            const float v0 = __fmul_rn(amax, r);
+            const float v = fminf(fmaxf(__fmaf_rn(__fmaf_rn(-v0, d32, amax), r, v0), 4.f), 8.f);
+            m = m_up = (uint32_t)__float2int_rn((v - 4.f) * 2.f);  // 0..8, ties to even
+        } else {
+            const float r_dn = __fmul_rn(r, kDown), r_up = __fmul_rn(r, kUp);
+            const float v_dn = fminf(fmaxf(__fmul_rn(amax, r_dn), 4.f), 8.f);
+            const float v_up = fminf(fmaxf(__fmul_rn(amax, r_up), 4.f), 8.f);
+            m = (uint32_t)__float2int_rn((v_dn - 4.f) * 2.f);  // 0..8
+            m_up = (uint32_t)__float2int_rn((v_up - 4.f) * 2.f);
+        }
         if (m != m_up) {  // boundary 4.25 + m / 2 between m and m + 1
             const double bound = (double)(17u + 2u * m) * 0.25 * ((double)e * (double)ts);
             const double a = (double)amax;

@@ -6,7 +6,8 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import to_dev
+import oracle
+from helpers import check_gemm, packed_to_host, to_dev
 from paper_2510_14557_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -30,6 +31,10 @@ def test_noalloc_matches_mxp_gemm_twice_in_a_row():
         tol = 1e-3 * da.norm(dim=1)[:, None] * dw.norm(dim=1)[None, :]
         err = (out.double() - ref.double()).abs()
         assert bool((err <= tol).all()), "call %d: max err/tol %g" % (call, float((err / tol).max()))
+        # and against the oracle: the fp64 product of its own decode of the same planes
+        na, sa, ia = packed_to_host(pa)
+        nw, sw, iw = packed_to_host(pw)
+        check_gemm(out, oracle.dequantize(na, sa, ia, amode), oracle.dequantize(nw, sw, iw, bmode))
         results.append(out)
     # asynchronous form (no status read) on a bf16 output, after the two calls above
     out16 = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
@@ -47,3 +52,8 @@ def test_noalloc_rejects_bad_arguments():
     with pytest.raises(m.MxpError) as e:
         m.mxp_gemm_noalloc(pa, pb, out)
     assert e.value.status == 1
+    # modes that need operands prepared in a workspace are "unsupported", as for mxp_gemm
+    pp = m.mxp_quantize(to_dev(synth.weights(16, 128, seed=3)), m.MODE_MXFP4_PP)
+    with pytest.raises(m.MxpError) as e:
+        m.mxp_gemm_noalloc(pa, pp, out)
+    assert e.value.status == 2
