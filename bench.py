@@ -230,6 +230,54 @@ def parts(mxp, synth, peaks, only=None, iters_scale=1.0):
         out.update(part_decode(mxp, synth, peaks, max(2, int(40 * iters_scale))))
     if only in (None, "prefill"):
         out.update(part_prefill(mxp, synth, peaks, max(1, int(10 * iters_scale))))
+    if only == "prefill_cfg4":
+        out.update(part_small_prefill(mxp, synth, max(1, int(4 * iters_scale))))
+    if only == "decode_tc":
+        out.update(part_decode_tc(mxp, synth, max(1, int(4 * iters_scale))))
+    return out
+
+
+def part_small_prefill(mxp, synth, iters):
+    """Config 4 through mxp_gemm_prepacked for the four mode pairs, a few launches each: a
+    case small enough for multi-pass profiler captures of the streamed GEMM kernel."""
+    import torch
+    out = {}
+    a_bits, w_bits = synth.config4()
+    a, w = dev_bf16(a_bits), dev_bf16(w_bits)
+    M, K = a.shape
+    N = w.shape[0]
+    d = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(mxp.mxp_gemm_workspace_bytes(M, N, K, False, 1, 1), dtype=torch.uint8, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for name, am, bm in (("plain", 0, 0), ("A+", 1, 0), ("W+", 0, 1), ("both", 1, 1)):
+        pa, pw = mxp.mxp_quantize(a, am), mxp.mxp_quantize(w, bm)
+        pre = mxp.mxp_gemm_prepack(pw, mxp.mxp_gemm_prepack_form(am, bm))
+        ms = timed_flushed(lambda: mxp.mxp_gemm_prepacked(pa, pw, pre, out=d, workspace=ws), iters, flush, pre=1)
+        out["prefill_cfg4_" + name] = {"us": ms * 1e3}
+    return out
+
+
+def part_decode_tc(mxp, synth, iters):
+    """Config 3 at M = 1 on the FP4 tensor-path decode kernel, eight weight copies, a few eager
+    launches per mode: the case for profiler captures of that kernel."""
+    import torch
+    out = {}
+    a16, w_bits = synth.config3(1)
+    w = dev_bf16(w_bits)
+    a = dev_bf16(a16)
+    N, K = w.shape
+    d = torch.empty((1, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(max(256, mxp.mxp_gemm_decode_workspace_bytes(1, K)), dtype=torch.uint8, device="cuda")
+    for name, mode in (("mxfp4+", mxp.MODE_MXFP4_PLUS), ("mxfp4", mxp.MODE_MXFP4)):
+        tiled = [mxp.mxp_gemm_decode_prepack(mxp.mxp_quantize(w, mode)) for _ in range(8)]
+        st = {"i": 0}
+
+        def run():
+            mxp.mxp_gemm_decode_prepacked(a, tiled[st["i"] % 8], out=d, workspace=ws)
+            st["i"] += 1
+        ms = time_loop(run, 8 * iters, warmup=8)
+        out["decode_tc_cfg3_M1_" + name] = {"us": ms * 1e3}
+        del tiled
     return out
 
 
@@ -928,7 +976,8 @@ def main():
     ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
     ap.add_argument("--no-targets", action="store_true", help="skip the per-configuration scorecard")
     ap.add_argument("--parts", action="store_true", help="add the long per-kernel list")
-    ap.add_argument("--only", default=None, choices=["quantize", "decode", "prefill"],
+    ap.add_argument("--only", default=None,
+                    choices=["quantize", "decode", "prefill", "prefill_cfg4", "decode_tc"],
                     help="run one per-config part only and print its numbers (profiler captures)")
     ap.add_argument("--iters-scale", type=float, default=1.0)
     args = ap.parse_args()
