@@ -3,7 +3,7 @@
 the block-scaled GEMM against pre-quantized MXFP4+ weights.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg5|cfg4|small] [--no-targets] [--parts]
+                    [--workload cfg5|cfg4|small] [--no-targets] [--parts] [--only PART]
 
 One "step" = mxp_quantize(A) + mxp_gemm(A_q, W_q) on one batch of synthetic activations.
 Prints ONE JSON line (rank 0).  Besides the timed steps the line carries `sustained` (the same
@@ -692,6 +692,16 @@ def targets(mxp, synth, peaks):
             mxp.mxp_gemm_ready(pa, qw[MXP], pre, ws, out=d)
         ms = timed_queued(step, n_it, flush)
         pf["step_both"] = {"us": _r(ms * 1e3), "TFLOPs": _r(fl / ms / 1e9), "frac_fp4": _r(fl / ms / 1e9 / fp4, 3)}
+        # the paper's main scenario as a step: activations to MXFP4+, split per Eq. 4 by the
+        # quantizer itself, against MXFP4 weights prepared once (sparse residual GEMM): 2 launches
+        pre_plain = mxp.mxp_gemm_prepack(qw[MX], mxp.PREPACK_PLAIN)
+
+        def step_a_plus():
+            mxp.mxp_quantize_gemm_ready(a, MXP, ws, out=pa, b_mode=MX)
+            mxp.mxp_gemm_ready(pa, qw[MX], pre_plain, ws, out=d)
+        ms = timed_queued(step_a_plus, n_it, flush)
+        pf["step_A+"] = {"us": _r(ms * 1e3), "TFLOPs": _r(fl / ms / 1e9), "frac_fp4": _r(fl / ms / 1e9 / fp4, 3)}
+        del pre_plain
         out["prefill_" + cfg] = pf
         del a, w, d, ws, qa, qw, pre, pa
         torch.cuda.empty_cache()
@@ -976,12 +986,16 @@ def main():
     ap.add_argument("--workload", default="cfg5", choices=sorted(WORKLOADS))
     ap.add_argument("--no-targets", action="store_true", help="skip the per-configuration scorecard")
     ap.add_argument("--parts", action="store_true", help="add the long per-kernel list")
+    ap.add_argument("--no-parts", action="store_true",
+                    help="the step only: same as --no-targets (the flag's older name)")
     ap.add_argument("--only", default=None,
                     choices=["quantize", "decode", "prefill", "prefill_cfg4", "decode_tc"],
                     help="run one per-config part only and print its numbers (profiler captures)")
     ap.add_argument("--iters-scale", type=float, default=1.0)
     args = ap.parse_args()
     M, N, K, label = WORKLOADS[args.workload]
+    if args.no_parts:
+        args.no_targets = True
     if args.only is not None:
         from paper_2510_14557_b200 import build, synth
         build.build()

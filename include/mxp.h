@@ -289,19 +289,24 @@ mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void 
  *                            that also writes, into `workspace`, the operand in the form the
  *                            streamed tensor-core kernel reads (what mxp_gemm_prepacked would
  *                            otherwise derive from the packed planes in a launch of its own)
- *                            and clears the workspace's status block.  `workspace`: device,
- *                            256-byte aligned, at least mxp_gemm_workspace_bytes(M, N, K, 0,
- *                            mode, b_mode) bytes for the GEMM it will serve; M > 128,
- *                            K % 128 == 0.
+ *                            and clears the workspace's status block.  `b_mode`: the mode of
+ *                            the operand the result will be multiplied with; it decides the
+ *                            form, as for mxp_gemm: an MXFP4+ A against an MXFP4 B is split per
+ *                            Eq. 4 for the sparse residual instruction (needs K % 256 == 0),
+ *                            every other pairing is widened.  `workspace`: device, 256-byte
+ *                            aligned, at least mxp_gemm_workspace_bytes(M, N, K, 0, mode,
+ *                            b_mode) bytes for the GEMM it will serve; M > 128, K % 128 == 0.
  *   mxp_gemm_ready           mxp_gemm_prepacked for an A prepared that way in the same
  *                            `workspace` (nothing may have written to it in between) and a B
- *                            prepacked in the form MXP_PREPACK_WIDE (size checked as for
- *                            mxp_gemm_prepacked): one launch.  Same result as mxp_gemm.
+ *                            prepacked in the form mxp_gemm_prepack_form(A's mode, B's mode)
+ *                            says, except that an MXFP4 A against an MXFP4+ B reads the widened
+ *                            forms here (size checked as for mxp_gemm_prepacked): one launch.
+ *                            Same result as mxp_gemm.
  */
 mxp_status mxp_quantize_gemm_ready(const void *src, mxp_dtype src_dt, int64_t M, int64_t K,
-                                   int64_t ld_src, mxp_mode mode, uint8_t *nibbles,
-                                   uint8_t *scales, uint8_t *bm_index, void *workspace,
-                                   size_t workspace_bytes, void *cuda_stream);
+                                   int64_t ld_src, mxp_mode mode, mxp_mode b_mode,
+                                   uint8_t *nibbles, uint8_t *scales, uint8_t *bm_index,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
 mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed *A_packed,
                           const mxp_packed *B_packed, const void *B_prepacked,
                           size_t B_prepacked_bytes, void *D, mxp_dtype d_dt, int64_t ldd,

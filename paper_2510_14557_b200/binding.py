@@ -104,7 +104,7 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_prepacked.restype = ci
         l.mxp_gemm_ready.argtypes = l.mxp_gemm_prepacked.argtypes
         l.mxp_gemm_ready.restype = ci
-        l.mxp_quantize_gemm_ready.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, vp, sz, vp]
+        l.mxp_quantize_gemm_ready.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, vp, vp, vp, sz, vp]
         l.mxp_quantize_gemm_ready.restype = ci
         l.mxp_debug_override.argtypes = [ci, ci]
         l.mxp_debug_override.restype = ci
@@ -334,13 +334,15 @@ def mxp_gemm_prepacked(a: Packed, b: Packed, b_prepacked: torch.Tensor, out_dtyp
 
 
 def mxp_quantize_gemm_ready(src: torch.Tensor, mode: int, workspace: torch.Tensor,
-                            out: Optional[Packed] = None) -> Packed:
-    """mxp_quantize that also writes A's GEMM-ready form into `workspace` (see include/mxp.h)."""
+                            out: Optional[Packed] = None, b_mode: Optional[int] = None) -> Packed:
+    """mxp_quantize that also writes A's GEMM-ready form into `workspace` (see include/mxp.h).
+    `b_mode`: the mode of the operand it will be multiplied with (default: the same mode)."""
     assert src.is_cuda and src.dim() == 2 and src.stride(1) == 1
     rows, cols = src.shape
     if out is None:
         out = alloc_packed(rows, cols, mode, src.device)
     st = lib().mxp_quantize_gemm_ready(src.data_ptr(), _dt(src), rows, cols, src.stride(0), mode,
+                                       mode if b_mode is None else b_mode,
                                        out.nibbles.data_ptr(), out.scales.data_ptr(),
                                        out.bm_index.data_ptr() if out.bm_index is not None else None,
                                        workspace.data_ptr(), workspace.numel(), _stream())

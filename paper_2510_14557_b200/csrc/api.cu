@@ -429,9 +429,9 @@ mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void*
 }
 
 mxp_status mxp_quantize_gemm_ready(const void* src, mxp_dtype src_dt, int64_t M, int64_t K,
-                                   int64_t ld_src, mxp_mode mode, uint8_t* nibbles, uint8_t* scales,
-                                   uint8_t* bm_index, void* workspace, size_t workspace_bytes,
-                                   void* cuda_stream)
+                                   int64_t ld_src, mxp_mode mode, mxp_mode b_mode, uint8_t* nibbles,
+                                   uint8_t* scales, uint8_t* bm_index, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream)
 {
     if (mode != MXP_MODE_MXFP4 && mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
     if (!valid_dtype(src_dt) || M <= 0 || K <= 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
@@ -439,13 +439,27 @@ mxp_status mxp_quantize_gemm_ready(const void* src, mxp_dtype src_dt, int64_t M,
     if (mode != MXP_MODE_MXFP4 && bm_index == nullptr) return MXP_ERR_INVALID_ARG;
     if (!aligned(src, 16) || !aligned(nibbles, 16)) return MXP_ERR_INVALID_ARG;
     if (src_dt != MXP_BF16 || ld_src != K) return MXP_ERR_UNSUPPORTED;  // the fused kernel's case
+    if (b_mode < MXP_MODE_MXFP4 || b_mode > MXP_MODE_MXFP8_PLUS) return MXP_ERR_INVALID_ARG;
+    if (mode == MXP_MODE_MXFP4_PLUS && mxp::stream_b_form(mode, b_mode) == MXP_PREPACK_PLAIN) {
+        // MXFP4+ against plain MXFP4: Eq. 4's split for the sparse residual instruction
+        size_t at = 0, mn = 0, rs = 0, mt = 0, po = 0, pb = 0, tot = 0;
+        if (!mxp::stream_a_split_layout(M, K, &at, &mn, &rs, &mt, &po, &pb, &tot)) return MXP_ERR_UNSUPPORTED;
+        if (workspace == nullptr || workspace_bytes < tot) return MXP_ERR_WORKSPACE;
+        if (!aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;
+        uint8_t* w8 = static_cast<uint8_t*>(workspace);
+        const mxp::QuantizeSplitOut sp = {w8 + mn, w8 + rs, w8 + mt, po, pb};
+        cudaError_t e = mxp::launch_quantize_ready(src, M, K, mode, nibbles, scales, bm_index, w8 + at, nullptr,
+                                                   &sp, workspace, static_cast<cudaStream_t>(cuda_stream));
+        if (e == cudaErrorNotSupported) return MXP_ERR_UNSUPPORTED;
+        return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
+    }
     size_t atoms = 0, slots = 0, total = 0;
     if (!mxp::stream_a_ready_layout(M, K, &atoms, &slots, &total)) return MXP_ERR_UNSUPPORTED;
     if (workspace == nullptr || workspace_bytes < total) return MXP_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaError_t e = mxp::launch_quantize_ready(src, M, K, mode, nibbles, scales, bm_index, ws + atoms,
-                                               ws + slots, workspace,
+                                               ws + slots, nullptr, workspace,
                                                static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }
@@ -470,6 +484,14 @@ mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed* A_p
         return MXP_ERR_UNSUPPORTED;
     if (mxp::stream_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode) == 0)
         return MXP_ERR_UNSUPPORTED;
+    if (A_packed->mode == MXP_MODE_MXFP4_PLUS &&
+        mxp::stream_b_form(A_packed->mode, B_packed->mode) == MXP_PREPACK_PLAIN) {
+        // A was split by the quantizer (Eq. 4), B comes with plain scale atoms: sparse residual path
+        if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, MXP_PREPACK_PLAIN) || !aligned(B_prepacked, 256))
+            return MXP_ERR_INVALID_ARG;
+        return mxp::launch_gemm_tc_sparse(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd, workspace,
+                                          workspace_bytes, static_cast<cudaStream_t>(cuda_stream), true);
+    }
     if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) || !aligned(B_prepacked, 256))
         return MXP_ERR_INVALID_ARG;
     return mxp::launch_gemm_tc_stream(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,

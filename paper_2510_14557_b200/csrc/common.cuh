@@ -86,9 +86,19 @@ size_t stream_dense_prepacked_workspace_bytes(int64_t M, int64_t K);  // with B 
 // launch is left): offsets inside the GEMM's workspace, and the launch (bf16, contiguous rows,
 // MXFP4 / MXFP4+).
 bool stream_a_ready_layout(int64_t M, int64_t K, size_t* atoms, size_t* slots, size_t* total);
+// The same for the sparse-residual form (A is MXFP4+, its partner plain MXFP4): where inside the
+// workspace the quantizer writes Eq. 4's split of A, and which of the metadata's bytes belong to
+// rows past A's end (they are filled with valid nibbles before the quantizer runs).
+struct QuantizeSplitOut {
+    uint8_t *main, *res, *meta;
+    size_t meta_pad_offset, meta_pad_bytes;
+};
+bool stream_a_split_layout(int64_t M, int64_t K, size_t* atoms, size_t* main, size_t* res, size_t* meta,
+                           size_t* meta_pad_offset, size_t* meta_pad_bytes, size_t* total);
 cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, mxp_mode mode,
                                   uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
-                                  uint8_t* atoms, uint8_t* slots, void* status, cudaStream_t stream);
+                                  uint8_t* atoms, uint8_t* slots, const QuantizeSplitOut* split, void* status,
+                                  cudaStream_t stream);
 // One operand in the form that kernel reads, written once, e.g. for weights.  `form` is an
 // mxp_prepack_form: scale atoms only, atoms + widened codes, or atoms + the Eq. 4 split of an
 // MXFP4+ operand.  stream_prepack_bytes() == 0: shape or form not supported.
@@ -102,7 +112,8 @@ size_t stream_sparse_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a
                                      bool b_prepacked);
 mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_packed& A, const mxp_packed& B,
                                  const void* b_prepacked, void* D, mxp_dtype d_dt, int64_t ldd,
-                                 void* workspace, size_t workspace_bytes, cudaStream_t stream);
+                                 void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                                 bool a_ready = false);
 // The form of B's prepacked copy that a packed x packed GEMM with these modes reads.
 int stream_b_form(mxp_mode a_mode, mxp_mode b_mode);
 

@@ -1354,10 +1354,33 @@ size_t stream_sparse_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a
     return sparse_layout(rows_x, rows_y, K, b_prepacked && bp, b_prepacked && ap).total;
 }
 
+// Where a quantizer that prepares an MXFP4+ A for the sparse-residual GEMM itself has to write
+// inside the workspace of a call with a prepacked (plain MXFP4) B.
+bool stream_a_split_layout(int64_t M, int64_t K, size_t* atoms, size_t* main, size_t* res, size_t* meta,
+                           size_t* meta_pad_offset, size_t* meta_pad_bytes, size_t* total)
+{
+    if (M <= 128 || K < 256 || K % 256 != 0 || (uint64_t)M * (uint64_t)K / 16 >= (1ull << 32)) return false;
+    const SparseLayout l = sparse_layout(M, 0, K, false, true);
+    const SplitLayout lx = split_layout(M, K);
+    *atoms = l.x + lx.atoms;
+    *main = l.x + lx.main;
+    *res = l.x + lx.res;
+    *meta = l.x + lx.meta;
+    // row groups (of 128 rows) that reach past row M: their blocks are contiguous at the end
+    const size_t rgs = (size_t)row_groups(M, kTileM), full = (size_t)(M / 128), stages = (size_t)(K / 256);
+    *meta_pad_offset = full * stages * 2048;
+    *meta_pad_bytes = (rgs - full) * stages * 2048;
+    *total = l.total;
+    return true;
+}
+
+// `a_ready`: A (the MXFP4+ side) has been split into the workspace by the quantizer, which also
+// cleared the status block; needs a prepacked B, so that nothing is left to prepare.
 mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_packed& A, const mxp_packed& B,
                                  const void* b_prepacked, void* D, mxp_dtype d_dt, int64_t ldd,
-                                 void* workspace, size_t workspace_bytes, cudaStream_t stream)
+                                 void* workspace, size_t workspace_bytes, cudaStream_t stream, bool a_ready)
 {
+    if (a_ready && (b_prepacked == nullptr || A.mode != MXP_MODE_MXFP4_PLUS || K % 256 != 0)) return MXP_ERR_UNSUPPORTED;
     const size_t need = stream_sparse_workspace_bytes(M, N, K, A.mode, B.mode, b_prepacked != nullptr);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
     if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
@@ -1385,13 +1408,15 @@ mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_pack
     const uint8_t* y_atoms =
         y_pre ? static_cast<const uint8_t*>(b_prepacked) + packed_layout(rows_y, K, false).atoms[halves - 1]
               : ws + l.y;
-    const PrepackOperand px = x_pre ? no_operand() : split_operand(X, ws + l.x);
+    const PrepackOperand px = (x_pre || a_ready) ? no_operand() : split_operand(X, ws + l.x);
     const PrepackOperand py =
         y_pre ? no_operand() : prepack_operand(Y, rows_y, K, false, sub, ws + l.y, nullptr);
     const uint64_t ctas = (uint64_t)px.scale_ctas + py.scale_ctas + px.split_ctas;
-    if (ctas == 0 || ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
-    prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(px, py, static_cast<StatusBlock*>(workspace));
-    if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+    if ((ctas == 0 && !a_ready) || ctas > 0x7FFFFFFFull) return MXP_ERR_UNSUPPORTED;
+    if (ctas != 0) {
+        prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(px, py, static_cast<StatusBlock*>(workspace));
+        if (cudaGetLastError() != cudaSuccess) return MXP_ERR_CUDA;
+    }
 
     CUtensorMap ta, tb, tsa, tsb, tres, tmeta;
     const bool maps_ok = make_tmap_rows(&ta, x_base + lx.main, rows_x, K / 2, 128) &&

@@ -417,17 +417,24 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8_bf16(uint32_t p0, uint32_t p1, ui
 // What the kReady variant also writes: the operand in the form the streamed tensor-core GEMM
 // reads (Sec. 5: quantization fused with the preparation of the matrix-multiply operand), i.e.
 // what prepack_kernel would make of the packed planes: the scale byte inside its 32-row x
-// 16-byte atom and the block's 32 codes as two 16-byte slots of E2M3 codes, BM included.
+// 16-byte atom and either (kReady = 1) the block's 32 codes as two 16-byte slots of E2M3 codes,
+// BM included, or (kReady = 2, MXFP4+ against a plain MXFP4 partner) Eq. 4's split for the
+// sparse residual instruction: the codes with BM_H in the BM's place, BM_L 2:1 compressed,
+// and the metadata nibbles that say where it sits.
 struct GemmReady {
     uint8_t* atoms;      // [ceil(rows/128)][nbk/4][512]
-    uint4* slots;        // [rows][nbk][2]
+    uint4* slots;        // kReady = 1: [rows][nbk][2]
+    uint4* sp_main;      // kReady = 2: [rows][nbk] codes with BM_H
+    uint2* sp_res;       //             [rows][nbk] compressed BM_L
+    uint8_t* sp_meta;    //             [row group of 128][stage of 8 blocks][128 rows x 16 bytes]
+    int sp_stages;       //             stages per row (nbk / 8)
     int nbk;             // blocks per row
     StatusBlock* status; // zeroed here for the GEMM that follows
 };
 
 // One block of 32 bf16 values (x: sixteen pairs, element 0 in the low half of x[0]) -> its
 // codes, scale byte and index byte, stored as block number `blk`.
-template <int kMode, bool kReady>
+template <int kMode, int kReady>
 __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t blk,
                                                     uint4* __restrict__ nibbles,
                                                     uint8_t* __restrict__ scales,
@@ -503,8 +510,38 @@ __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t b
     __stcs(nibbles + blk, outv);
     scales[blk] = (uint8_t)sb;
     if (bm_index != nullptr) bm_index[blk] = (uint8_t)(dead ? 0u : (bm | (delta << 5)));
-    if (kReady) {
-        static_assert(!kReady || kMode <= 1, "GEMM-ready output: MXFP4 and MXFP4+ only");
+    if (kReady == 2) {
+        static_assert(kReady != 2 || kMode == 1, "split output: MXFP4+ only");
+        // Eq. 4: BM = BM_H + BM_L.  The BM's code in w[] is s m2 m1 m0.
+        uint32_t mw[4] = {outv.x, outv.y, outv.z, outv.w};
+        unsigned long long res = 0ull;
+        uint32_t meta = 0x4444u;  // pairs 0 and 1 of every group of eight: all zeros
+        if (!dead) {
+            const uint32_t sh = (bm & 7u) * 4u, gi = bm >> 3, pair = (bm & 7u) >> 1;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (gi == (uint32_t)i) {
+                    const uint32_t sign = (mw[i] >> sh) & 8u;
+                    mw[i] = (mw[i] & ~(7u << sh)) | ((6u | (m >> 2)) << sh);  // BM_H: E2M1 code 11 m2
+                    if (m & 3u)  // BM_L: E2M1 code 0 m1 m0 in the kept pair's slot
+                        res = (unsigned long long)(sign | (m & 3u))
+                              << (4u * (4u * gi + (pair == 3u ? 2u : 0u) + (bm & 1u)));
+                }
+            // the BM's group keeps the BM's pair and pair 3 (pairs 0 and 3 if the BM is in pair 3)
+            meta = (meta & ~(15u << (4u * gi))) | ((pair == 3u ? 0xCu : (pair | 0xCu)) << (4u * gi));
+        }
+        __stcs(ready.sp_main + blk, make_uint4(mw[0], mw[1], mw[2], mw[3]));
+        __stcs(ready.sp_res + blk, make_uint2((uint32_t)res, (uint32_t)(res >> 32)));
+        const int64_t row = blk / ready.nbk;
+        const int kb = (int)(blk - row * ready.nbk);
+        const int r = (int)(row & 127);
+        *reinterpret_cast<uint16_t*>(ready.sp_meta + ((size_t)(row >> 7) * ready.sp_stages + (kb >> 3)) * 2048 + r * 16 +
+                                     (kb & 7) * 2) = (uint16_t)meta;
+        ready.atoms[((row >> 7) * (ready.nbk >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)] =
+            (uint8_t)sb;
+    }
+    if (kReady == 1) {
+        static_assert(kReady != 1 || kMode <= 1, "GEMM-ready output: MXFP4 and MXFP4+ only");
         const uint32_t p = (kPlus && !dead) ? bm : 32u;  // BM position, none in a dead block
         uint4 s0 = e2m1x16_to_e2m3_slot(outv.x, outv.y, p < 16u ? p : 16u);
         uint4 s1 = e2m1x16_to_e2m3_slot(outv.z, outv.w, (p >= 16u && p < 32u) ? p - 16u : 16u);
@@ -518,7 +555,7 @@ __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t b
     }
 }
 
-template <int kMode, bool kReady>
+template <int kMode, int kReady>
 __global__ void __launch_bounds__(kThreads)
 quantize_bf16_lane_kernel(const uint4* __restrict__ src, int64_t total_blocks,
                           uint4* __restrict__ nibbles, uint8_t* __restrict__ scales,
@@ -602,7 +639,7 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
                     x[4 * k + i] = (uint32_t)row_s[ow[i] & 0xFFFFu] |
                                    ((uint32_t)row_s[ow[i] >> 16] << 16);
             }
-            quantize_block_bf16<kMode, false>(x, row * cols_blocks + b, nibbles, scales, bm_index, none);
+            quantize_block_bf16<kMode, 0>(x, row * cols_blocks + b, nibbles, scales, bm_index, none);
         }
         __syncthreads();  // all reads of this buffer are done before the next pass refills it
     }
@@ -678,7 +715,7 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
     const int aligned4 = ((reinterpret_cast<uintptr_t>(scales) & 3) == 0) &&
                          ((reinterpret_cast<uintptr_t>(bm_index) & 3) == 0);
     if (ld_src == cols && sizeof(T) == 2)
-        quantize_bf16_lane_kernel<kMode, false>
+        quantize_bf16_lane_kernel<kMode, 0>
             <<<(unsigned)((total_blocks + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
                 static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles),
                 scales, bm_index, GemmReady{});
@@ -765,24 +802,39 @@ cudaError_t launch_quantize_reordered(const void* src, mxp_dtype dt, int64_t row
 #undef MXP_QR
 }
 
-// bf16, contiguous rows, MXFP4 / MXFP4+: quantize and write the GEMM-ready form as well.
+// bf16, contiguous rows, MXFP4 / MXFP4+: quantize and write the GEMM-ready form as well
+// (`slots`: widened codes; or, with `split` given instead, Eq. 4's split of an MXFP4+ operand).
 cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, mxp_mode mode,
                                   uint8_t* nibbles, uint8_t* scales, uint8_t* bm_index,
-                                  uint8_t* atoms, uint8_t* slots, void* status, cudaStream_t stream)
+                                  uint8_t* atoms, uint8_t* slots, const QuantizeSplitOut* split, void* status,
+                                  cudaStream_t stream)
 {
     const int64_t total_blocks = rows * (cols / 32);
-    GemmReady ready;
+    GemmReady ready = {};
     ready.atoms = atoms;
     ready.slots = reinterpret_cast<uint4*>(slots);
     ready.nbk = (int)(cols / 32);
     ready.status = static_cast<StatusBlock*>(status);
     const unsigned grid = (unsigned)((total_blocks + kThreads - 1) / kThreads);
-    if (mode == MXP_MODE_MXFP4_PLUS)
-        quantize_bf16_lane_kernel<1, true><<<grid, kThreads, 0, stream>>>(
+    if (split != nullptr) {
+        if (mode != MXP_MODE_MXFP4_PLUS || cols % 256 != 0) return cudaErrorNotSupported;
+        ready.sp_main = reinterpret_cast<uint4*>(split->main);
+        ready.sp_res = reinterpret_cast<uint2*>(split->res);
+        ready.sp_meta = split->meta;
+        ready.sp_stages = (int)(cols / 256);
+        // rows past the operand's end inside its last row groups: metadata only, every nibble valid
+        if (split->meta_pad_bytes != 0 &&
+            cudaMemsetAsync(split->meta + split->meta_pad_offset, 0x44, split->meta_pad_bytes, stream) != cudaSuccess)
+            return cudaErrorUnknown;
+        quantize_bf16_lane_kernel<1, 2><<<grid, kThreads, 0, stream>>>(
+            static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles), scales,
+            bm_index, ready);
+    } else if (mode == MXP_MODE_MXFP4_PLUS)
+        quantize_bf16_lane_kernel<1, 1><<<grid, kThreads, 0, stream>>>(
             static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles), scales,
             bm_index, ready);
     else
-        quantize_bf16_lane_kernel<0, true><<<grid, kThreads, 0, stream>>>(
+        quantize_bf16_lane_kernel<0, 1><<<grid, kThreads, 0, stream>>>(
             static_cast<const uint4*>(src), total_blocks, reinterpret_cast<uint4*>(nibbles), scales,
             bm_index, ready);
     return cudaGetLastError();

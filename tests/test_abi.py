@@ -151,7 +151,11 @@ def test_prepacked_copies_are_checked_against_the_call(lib):
     gr = lib.mxp_gemm_ready
     a = _Packed(4096, 4096, 4096, M, K, MXP)
     b = _Packed(4096, 4096, 4096, N, K, MX)
-    assert gr(M, N, K, ctypes.byref(a), ctypes.byref(b), fake, size[PLAIN], fake, 1, N, fake, ws, null) == 1
+    # an MXFP4+ A prepared by the quantizer against a plain B reads B's plain copy, nothing else
+    assert gr(M, N, K, ctypes.byref(a), ctypes.byref(b), fake, size[WIDE], fake, 1, N, fake, ws, null) == 1
+    assert gr(M, N, K, ctypes.byref(a), ctypes.byref(b), fake, size[SPLIT], fake, 1, N, fake, ws, null) == 1
+    both = _Packed(4096, 4096, 4096, N, K, MXP)
+    assert gr(M, N, K, ctypes.byref(a), ctypes.byref(both), fake, size[PLAIN], fake, 1, N, fake, ws, null) == 1
     # mxp_gemm_prepack: the form must fit the operand's mode
     pk = lib.mxp_gemm_prepack
     assert pk(ctypes.byref(a), PLAIN, fake, ws, null) == 1      # an MXFP4+ operand has no plain form

@@ -161,3 +161,35 @@ def test_integer_valued_operands_are_exact():
         wp = host_to_packed(qw[0], qw[1], qw[2] if bmode == MXP else None, bmode)
         d = m.mxp_gemm(ap, wp, out_dtype=torch.float32)
         assert np.array_equal(d.cpu().numpy().astype(np.float64), oracle.gemm_fp64(da, dw))
+
+
+@pytest.mark.parametrize("M,N,K", [(512, 640, 512), (300, 481, 1024), (129, 200, 256), (1000, 300, 768)])
+def test_quantizer_emits_the_split_form_for_the_gemm(M, N, K):
+    # the paper's main scenario as two launches: activations quantized to MXFP4+ and split per
+    # Eq. 4 by the same kernel, straight into the GEMM's workspace, then the sparse-residual GEMM
+    # against MXFP4 weights prepared once.  Same packed planes as mxp_quantize (bit-exact against
+    # the oracle), same product as mxp_gemm on those planes (bit-identical: same kernel, same
+    # operands).  M not a multiple of 256: the last row groups' metadata is filled for rows the
+    # activations do not have.
+    from helpers import packed_to_host, to_dev_bf16
+    m = mxp()
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + K)
+    a = to_dev_bf16(a_bits)
+    pw = m.mxp_quantize(to_dev_bf16(w_bits), MX)
+    pre = m.mxp_gemm_prepack(pw, m.mxp_gemm_prepack_form(MXP, MX))
+    ws = torch.full((m.mxp_gemm_workspace_bytes(M, N, K, False, MXP, MX),), 0xEE, dtype=torch.uint8, device="cuda")
+    pa = m.mxp_quantize_gemm_ready(a, MXP, ws, b_mode=MX)
+    qa = oracle.quantize(a_bits, MXP, bf16_bits=True)
+    for got, want in zip(packed_to_host(pa), qa):
+        assert np.array_equal(got, want)
+    ws2 = torch.zeros_like(ws)
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm_ready(pa, pw, pre, ws, out_dtype=dt)
+        assert m.mxp_gemm_status(ws) == 0
+        assert torch.equal(d, m.mxp_gemm(pa, pw, out_dtype=dt, workspace=ws2))
+    qw = oracle.quantize(w_bits, MX, bf16_bits=True)
+    check_gemm(d, oracle.dequantize(qa[0], qa[1], qa[2], MXP), oracle.dequantize(qw[0], qw[1], qw[2], MX))
+    # K with half a stage at its end is not taken by the fused form
+    if K == 768:
+        with pytest.raises(m.MxpError):
+            m.mxp_quantize_gemm_ready(a[:, :640].contiguous(), MXP, ws, b_mode=MX)
