@@ -72,6 +72,10 @@ double oracle_e2m1_value(int code)
  * the largest magnitude saturates to it (Sec. 4.3 example: 7.92 -> 6.0). */
 static int e2m1_nearest(double r)
 {
+    /* saturation first: beyond 2^53 the distances to 4 and to 6 round to the same double and
+     * the search below could no longer tell them apart */
+    if (r >= 6.0)
+        return 7;
     int best = 0;
     double best_d = fabs(r - oracle_e2m1_value(0));
     for (int c = 1; c < 8; ++c) {

@@ -88,7 +88,30 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
 #define X(i) elem<kKey>(raw, (i))
     float amax = 0.f;
     int bm = 0;
-    if (kPlus && kKey) {
+    if (kKey && kShort) {
+        // bf16 pairs as loaded: the largest magnitude with a packed maximum, its first position
+        // from a packed compare (one bit per element, even elements in bits 0,2,.., odd ones in
+        // bits 16,18,..)
+        uint32_t t[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t[i] = raw[i] & 0x7FFF7FFFu;
+        uint32_t m2 = t[0];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) asm("max.NaN.bf16x2 %0, %0, %1;" : "+r"(m2) : "r"(t[i]));
+        asm("max.NaN.bf16x2 %0, %0, %1;" : "+r"(m2) : "r"(__byte_perm(m2, m2, 0x1032)));
+        amax = __uint_as_float(m2 << 16);
+        if (kPlus) {
+            uint32_t r1 = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                uint32_t eq;
+                asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(eq) : "r"(t[i]), "r"(m2));
+                r1 |= eq & ((1u << (2 * i)) | (1u << (16 + 2 * i)));
+            }
+            const uint32_t map = (r1 & 0xFFFFu) | ((r1 >> 15) & 0xAAAAu);
+            bm = __ffs((int)map) - 1;
+        }
+    } else if (kPlus && kKey) {
         uint32_t key = 0;
 #pragma unroll
         for (int i = 0; i < 16; ++i)
@@ -105,7 +128,16 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
         }
     }
     // scale byte: E4M3 nearest to amax / (6 ts)
-    const float q = __fdiv_rn(amax, six_ts);
+    float q;
+    if (kShort) {
+        // the quotient by one Newton step on amax * (1 / 6 ts): exact whenever it is representable
+        const float r6 = __frcp_rn(six_ts);  // (uniform over the grid: hoisted by the compiler)
+        const float q0 = __fmul_rn(amax, r6);
+        // (an enormous quotient needs no step: it saturates the cast; an infinite one would not)
+        q = q0 < 1e30f ? __fmaf_rn(__fmaf_rn(-q0, six_ts, amax), r6, q0) : 1e30f;
+    } else {
+        q = fminf(__fdiv_rn(amax, six_ts), 1e30f);  // (the cast saturates finite values only)
+    }
     // (short operands: 6 ts is exact, the division is correctly rounded, and a quotient that is
     // not exactly on a boundary between two bytes is at least 2^-21 of it away: one cast decides)
     uint32_t sb = f32_to_e4m3_byte(kShort ? q : __fmul_rn(q, kDown));
@@ -117,7 +149,11 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
         if (a > bound || (a == bound && (sb & 1u))) sb = sb_up;
     }
     const float e = e4m3_byte_to_f32(sb);
-    const float r = __frcp_rn(__fmul_rn(e, ts));
+    // (short operands: the Newton step below squares the reciprocal's error, so the fast
+    // approximate reciprocal serves)
+    float r;
+    if (kShort) asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fmul_rn(e, ts)));
+    else r = __frcp_rn(__fmul_rn(e, ts));
     // r > 0, so x * r has the sign of x even where it underflows, and the hardware cast keeps
     // the sign of a value that rounds to zero: the codes' sign bits are the inputs'.
     // Every E2M1 rounding boundary (0.25 0.75 1.25 1.75 2.5 3.5 5) has zeros in the low 21 bits
@@ -129,11 +165,22 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
         // d is exact in binary32 here.  rho = x - s0 d (rounded down, so that an exact zero is
         // -0 and the sum below keeps the sign of a zero input), s = s0 + rho r.
         const float d32 = __fmul_rn(e, ts);
+        if (__fmul_rn(amax, r) < 1e30f) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const float x = X(i);
-            const float s0 = __fmul_rn(x, r);
-            s[i] = __fmaf_rn(__fmaf_rd(-s0, d32, x), r, s0);
+            for (int i = 0; i < 16; ++i) {
+                const float x = X(i);
+                const float s0 = __fmul_rn(x, r);
+                s[i] = __fmaf_rn(__fmaf_rd(-s0, d32, x), r, s0);
+            }
+        } else {
+            // a saturated scale under an enormous block: products may overflow; clamped first,
+            // the step still returns the quotient (or an infinity that saturates the cast)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float x = X(i);
+                const float s0 = fminf(fmaxf(__fmul_rn(x, r), -16.f), 16.f);
+                s[i] = __fmaf_rn(__fmaf_rd(-s0, d32, x), r, s0);
+            }
         }
         w0 = cvt_e2m1x8(s);
         w1 = cvt_e2m1x8(s + 8);
@@ -177,7 +224,8 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
             // and otherwise at least 2^-20 of a boundary 4.25 + m / 2 away from it
             const float d32 = __fmul_rn(e, ts);
             const float v0 = __fmul_rn(amax, r);
-            const float v = fminf(fmaxf(__fmaf_rn(__fmaf_rn(-v0, d32, amax), r, v0), 4.f), 8.f);
+            // (an overflowed product clamps to 8 like any quotient of 8 or more)
+            const float v = v0 < 1e30f ? fminf(fmaxf(__fmaf_rn(__fmaf_rn(-v0, d32, amax), r, v0), 4.f), 8.f) : 8.f;
             m = m_up = (uint32_t)__float2int_rn((v - 4.f) * 2.f);  // 0..8, ties to even
         } else {
             const float r_dn = __fmul_rn(r, kDown), r_up = __fmul_rn(r, kUp);

@@ -138,6 +138,8 @@ def test_rounding_boundaries_bit_exact(plus):
         x = nvfp4_boundary_blocks(ts, seed)
         x[::7, 3] = -0.0
         x[::5, 11] = np.float32(-2.0 ** -120)
+        x[::9, 17] = np.float32(3.0e38)       # the scale saturates and quotients overflow binary32
+        x[1::9, 5] = np.float32(-2.0e30)
         bits = synth.f32_to_bf16_bits(x)
         ref = oracle.nvfp4_quantize(bits, ts, plus, bf16_bits=True)
         got = mxp().mxp_nvfp4_quantize(to_dev_bf16(bits), ts, plus)

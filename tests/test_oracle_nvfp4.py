@@ -246,3 +246,24 @@ def test_how_often_a_binary32_recipe_departs_from_the_definition():
     assert counts["2^-8"] > 0
     # and the two agree on the overwhelming majority, so the recipe above is a faithful restatement
     assert max(counts.values()) < 262144 // 20
+
+
+def test_enormous_quotients_saturate():
+    # a block whose scale saturates at 448 leaves quotients |x| / d far beyond the E2M1 range,
+    # up to ~1e36 for binary32 inputs (beyond 2^53, where a nearest-value search in binary64 can
+    # no longer tell the distances to 4 and to 6 apart): they saturate to 6, code 7, sign kept
+    # (Sec. 4.3's 7.92 -> 6.0 at any magnitude), and the scale byte is the largest finite one
+    x = np.zeros((1, 32), np.float32)
+    x[0, 3] = 3.0e38
+    x[0, 5] = -2.0e30
+    x[0, 6] = 1.0e20
+    x[0, 7] = 5.9 * 448.0          # below 6 d: the ordinary search
+    x[0, 20] = -1.0e25
+    for plus in (False, True):
+        nib, sc, idx = oracle.nvfp4_quantize(x, 1.0, plus)
+        codes = nib_codes(nib)[0]
+        assert sc[0, 0] == 0x7E and sc[0, 1] == 0x7E
+        assert codes[5] == 0xF and codes[6] == 0x7 and codes[7] == 0x7
+        assert codes[3] == 0x7                      # (the BM: m = 7 and saturation are the same code)
+        assert codes[20] == 0xF
+        assert not codes[[0, 1, 2, 4, 8, 16, 31]].any()
