@@ -32,15 +32,20 @@
 //     the conversion itself.  There every CTA converts the rows for itself, straight into
 //     shared memory where the images of all stages stay (40 KB at K = 4096), while its weights
 //     are already streaming: one launch per call, and no image travels through global memory.
-//     (The BM's lower part stays on the tensor cores there too: adding (BM_L 2^shared_exp)
-//     a[k_BM] per block on the CUDA cores from the record byte, the scale byte and the raw
-//     activation was built and measured -- twelve warps need ~0.45 us per stage for it, three
-//     dependent shared-memory loads per record, against ~0.15 us for the four extra MMAs.)
+//     MX+ there takes Eq. 4's BM_L term off the tensor cores: sum over blocks of
+//     (+-BM_L 2^shared_exp) a[k_BM] is eight products per weight row and stage, so warps 10-21
+//     add it on the CUDA cores in fp32 from the record bytes, the scale bytes and a raw bf16
+//     copy of the activations in shared memory -- one thread per weight row, the eight weights
+//     built without a branch and the eight activations fetched by independent loads (a form
+//     with a thread per (row, block) and the loads behind one another was ~3x slower and lost
+//     to the extra MMAs).  No BM_L tile is built and the MMA count per stage is that of plain
+//     MXFP4; the epilogue adds the three groups' partial sums in a fixed order.
 //   * warp 0 issues the weight copies (the first ring-full before the CTA's set-up barrier),
 //     warp 1 the activation copies, warps 2-5 the MMAs (each every fourth stage, with an
-//     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 build the BM_L
-//     tiles (three groups of four, a stage each in turn: one group needs ~0.8 us per stage,
-//     the stream delivers one every 0.26 us).
+//     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 handle BM_L
+//     (three groups of four, a stage each in turn): for M >= 3 they build the BM_L operand
+//     tiles (one group needs ~0.8 us per stage, the stream delivers one every 0.26 us), for
+//     M <= 2 they sum the term themselves.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -107,11 +112,11 @@ struct PrepackHeader {
 // A slot holds a stage's weight image, its activation image (codes at act_off, scale atoms
 // behind) and, for MX+, the BM_L tile built from the image's records (at res_off).
 // kSelf form (self_nst > 0: number of stages whose activation images stay resident): a slot
-// holds the weight image and, for MX+, the BM_L tile; behind the ring come the images' code
-// tiles (2 KB a stage) and their scale atoms (512 bytes a stage).
+// holds the weight image only; behind the ring come the images' code tiles (2 KB a stage), their
+// scale atoms (512 bytes a stage) and, for MX+, the raw activations and the BM_L term's sums.
 struct DecodeLayout {
     size_t act_off, res_off, slot, bars, total;
-    size_t img_codes, img_sf;  // kSelf only
+    size_t img_codes, img_sf, raw, corr;  // kSelf only (raw, corr: MX+)
     int stages;
 };
 constexpr int kSelfMaxM = 2;
@@ -120,17 +125,22 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
 {
     DecodeLayout l;
     l.stages = stages;
-    l.img_codes = l.img_sf = 0;
+    l.img_codes = l.img_sf = l.raw = l.corr = 0;
     if (self_nst > 0) {
-        l.act_off = 0;
-        l.res_off = up(wimg, 1024);
-        l.slot = l.res_off + (plus ? up((size_t)rows * 128, 1024) : 0);
-        const size_t last = (size_t)(stages - 1) * l.slot + (plus ? l.res_off : 0) + 128 * 128;  // (see below)
+        l.act_off = l.res_off = 0;
+        l.slot = up(wimg, 1024);
+        const size_t last = (size_t)(stages - 1) * l.slot + 128 * 128;  // (see below)
         size_t o = up(last > (size_t)stages * l.slot ? last : (size_t)stages * l.slot, 1024);
         l.img_codes = o;
         o += (size_t)self_nst * 2048;
         l.img_sf = o;
         o += (size_t)self_nst * 512;
+        if (plus) {
+            l.raw = o;   // the activation rows as given (bf16), for the BM_L term
+            o += (size_t)kSelfMaxM * (size_t)self_nst * kStageK * 2;
+            l.corr = o;  // its sums [tile parity][group][row m][weight row]
+            o += 2 * kResGroups * kSelfMaxM * 128 * sizeof(float);
+        }
         l.bars = up(o, 16);
         l.total = l.bars + 1024 + 1024;
         return l;
@@ -371,7 +381,9 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     uint64_t* res_full = empty + kMaxStages;   // the slot's BM_L tile is written
     uint64_t* acc_full = res_full + kMaxStages;
     uint64_t* acc_empty = acc_full + 1;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+    uint64_t* corr_full = acc_empty + 1;       // [2] kSelf MX+: a tile's BM_L sums are complete
+    uint64_t* corr_empty = corr_full + 2;      // [2] ... and have been taken
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(corr_empty + 2);
     volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -386,11 +398,15 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         MXP_TL(0);  // kernel entry
         for (int s = 0; s < kMaxStages; ++s) {
             ptx::mbar_init(&full[s], kSelf ? 1 : 2);
-            ptx::mbar_init(&empty[s], 1);
+            ptx::mbar_init(&empty[s], (kSelf && kPlus) ? 1 + kResWarps : 1);  // + the warps that read its records
             ptx::mbar_init(&res_full[s], kResWarps);
         }
         ptx::mbar_init(acc_full, kIssuers);
         ptx::mbar_init(acc_empty, 4);
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&corr_full[b], kResWarps * kResGroups);
+            ptx::mbar_init(&corr_empty[b], 4);
+        }
         *abort = 0u;
         ptx::fence_mbar_init();
     }
@@ -437,6 +453,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             const int st = rem >> 5, kb = (rem >> 2) & 7, qd = rem & 3;
             const int64_t k0 = (int64_t)st * kStageK + kb * 32 + qd * 8;
             const uint4 v = __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + k0));
+            if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)k0) * 2) = v;
             convert_quarter(v, m, kb, qd, smem + L.img_codes + (size_t)st * 2048, smem + L.img_sf + (size_t)st * 512,
                             kSfb);
         }
@@ -529,7 +546,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     }
                 }
                 __syncwarp();
-                if (kPlus) {
+                if (kPlus && !kSelf) {
                     // the BM_L tile of the stage, same scales, same accumulator (Eq. 4)
                     if (!ptx::mbar_wait(&res_full[s], ph, abort, kWaitLimit)) {
                         if (lane == 0) report(prm.status, abort, 0x7500 + s);
@@ -603,6 +620,24 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(acc_empty);
+            if (kSelf && kPlus) {
+                // Eq. 4's BM_L term of this tile, summed on the CUDA cores by the warps below
+                if (!ptx::mbar_wait_relaxed(&corr_full[t & 1], (uint32_t)(t >> 1) & 1, abort, kWaitLimit, 100u)) {
+                    if (lane == 0) report(prm.status, abort, 0x7900);
+                    break;
+                }
+                const float* corr =
+                    reinterpret_cast<const float*>(smem + L.corr) + (size_t)(t & 1) * kResGroups * kSelfMaxM * 128;
+#pragma unroll
+                for (int m = 0; m < kSelfMaxM; ++m) {
+                    float c = 0.f;
+#pragma unroll
+                    for (int g = 0; g < kResGroups; ++g) c += corr[(g * kSelfMaxM + m) * 128 + row];  // fixed order
+                    o[m] += c;
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&corr_empty[t & 1]);
+            }
             if (row < rows_here) {
 #pragma unroll
                 for (int m = 0; m < kMt; ++m) {
@@ -615,6 +650,72 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     }
                 }
             }
+        }
+    } else if (kPlus && kSelf) {
+        // ---------------------------------------------------------------- BM_L on the CUDA cores
+        // Group g of four warps takes the stages whose running number is g (mod 3); thread = weight
+        // row.  A stage gives a row eight record bytes (BM position | BM_L code << 5 | sign << 7)
+        // and eight scale bytes: eight weights (BM_L 2^shared_exp), eight activations fetched
+        // independently of one another, eight FMAs per activation row.  No branch: an absent
+        // BM_L is a zero weight.
+        const int grp = (warp - kResWarp0) / kResWarps;
+        const int r = (int)threadIdx.x - 32 * (kResWarp0 + grp * kResWarps);
+        const __nv_bfloat16* raw = reinterpret_cast<const __nv_bfloat16*>(smem + L.raw);
+        const uint32_t so = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;
+        bool ok = true;
+        for (int t = 0; t < ntl && ok; ++t) {
+            float acc[kSelfMaxM] = {};
+            const int first = (grp + 3 * kResGroups - (int)(((uint32_t)t * (uint32_t)nst) % kResGroups)) % kResGroups;
+            for (int st = first; st < nst; st += kResGroups) {
+                const uint32_t c = (uint32_t)t * (uint32_t)nst + (uint32_t)st;
+                const int s = c % S;
+                if (!ptx::mbar_wait(&full[s], (c / S) & 1, abort, kWaitLimit)) {
+                    if (lane == 0) report(prm.status, abort, 0x7700 + s);
+                    ok = false;
+                    break;
+                }
+                if (r < prm.rows) {
+                    const uint8_t* atoms = slot(s) + (size_t)prm.rows * 128;
+                    const uint2 rec = *reinterpret_cast<const uint2*>(atoms + 2 * kAtom + (size_t)r * 8);
+                    const uint32_t sc_lo = *reinterpret_cast<const uint32_t*>(atoms + so);
+                    const uint32_t sc_hi = *reinterpret_cast<const uint32_t*>(atoms + kAtom + so);
+                    float w[8];
+                    uint32_t k[8];
+#pragma unroll
+                    for (int kb = 0; kb < 8; ++kb) {
+                        const uint32_t b = ((kb < 4 ? rec.x : rec.y) >> (8 * (kb & 3))) & 255u;
+                        const uint32_t sc = ((kb < 4 ? sc_lo : sc_hi) >> (8 * (kb & 3))) & 255u;
+                        // BM_L 2^(sc - 127) = (code / 2) 2^(sc - 127), the sign from the record
+                        const float mag = (float)((b >> 5) & 3u) * 0.5f * __uint_as_float(sc << 23);
+                        w[kb] = __uint_as_float(__float_as_uint(mag) | ((b & 0x80u) << 24));
+                        k[kb] = (uint32_t)st * kStageK + (uint32_t)kb * 32u + (b & 31u);
+                    }
+#pragma unroll
+                    for (int m = 0; m < kSelfMaxM; ++m) {
+                        if (m < prm.M) {
+                            float a[8];
+#pragma unroll
+                            for (int kb = 0; kb < 8; ++kb) a[kb] = __bfloat162float(raw[(size_t)m * nst * kStageK + k[kb]]);
+#pragma unroll
+                            for (int kb = 0; kb < 8; ++kb) acc[m] = fmaf(w[kb], a[kb], acc[m]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&empty[s]);  // the slot's records have been read
+            }
+            if (!ok) break;
+            // the sums of tile t - 2 must have been taken before this tile's are written
+            if (t >= 2 && !ptx::mbar_wait(&corr_empty[t & 1], (uint32_t)((t - 2) >> 1) & 1, abort, kWaitLimit)) {
+                if (lane == 0) report(prm.status, abort, 0x7A00);
+                break;
+            }
+            float* corr = reinterpret_cast<float*>(smem + L.corr) +
+                          ((size_t)(t & 1) * kResGroups + grp) * kSelfMaxM * 128;
+#pragma unroll
+            for (int m = 0; m < kSelfMaxM; ++m) corr[m * 128 + r] = acc[m];  // this group's share, zeros included
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&corr_full[t & 1]);
         }
     } else if (kPlus) {
         // ---------------------------------------------------------------- BM_L tiles
