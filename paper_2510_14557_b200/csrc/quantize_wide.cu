@@ -157,6 +157,131 @@ quantize_wide_kernel(const T* __restrict__ src, int64_t ld_src, int nbk, int64_t
     if (bm_index != nullptr) bm_index[blk] = (uint8_t)((kPlus && !dead) ? bm : 0);
 }
 
+// bf16 sources with contiguous rows: the block stays packed two elements per register from the
+// load to the cast.  Magnitudes, the maximum and the compare that finds its first position run
+// on pairs (max.bf16x2, set.eq.bf16x2: 16 instead of 32 of each), the scaling is one packed
+// multiply by 2^-shared_exp (exact: a result below the bf16 normal range is far below half the
+// format's smallest subnormal and casts to a zero of its sign either way), and the 6-bit
+// codes are packed with two selects per four codes and byte permutes.
+__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_max_nan(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+template <int kFmt, bool kPlus>
+__global__ void __launch_bounds__(kThreads)
+quantize_wide_bf16_kernel(const uint4* __restrict__ src, int64_t total_blocks,
+                          uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                          uint8_t* __restrict__ bm_index)
+{
+    constexpr uint32_t kEmax = kFmt == 8 ? 8u : 2u;
+    constexpr int kMb = kFmt - 1;
+    const int64_t blk = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (blk >= total_blocks) return;
+    uint32_t x[16], t[16];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 v = __ldg(src + blk * 4 + i);
+        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t[i] = x[i] & 0x7FFF7FFFu;
+    uint32_t q[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        q[i] = bf16x2_max_nan(bf16x2_max_nan(t[4 * i], t[4 * i + 1]), bf16x2_max_nan(t[4 * i + 2], t[4 * i + 3]));
+    uint32_t m2 = bf16x2_max_nan(bf16x2_max_nan(q[0], q[1]), bf16x2_max_nan(q[2], q[3]));
+    m2 = bf16x2_max_nan(m2, __byte_perm(m2, m2, 0x1032));  // both halves = block maximum
+    const uint32_t amax16 = m2 & 0xFFFFu;
+    const uint32_t E = amax16 >> 7;
+    const bool flush = E <= kEmax, nonfinite = E == 255u;
+    const bool dead = flush || nonfinite;
+    const uint32_t sb = flush ? 0u : (nonfinite ? 255u : E - kEmax);
+    uint32_t bm = 0;
+    if (kPlus) {
+        // one bit per element where |x| equals the maximum; lowest set bit = first BM (Sec. 3.2)
+        uint32_t r1 = 0, r2 = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t e1, e2;
+            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e1) : "r"(t[i]), "r"(m2));
+            asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e2) : "r"(t[8 + i]), "r"(m2));
+            const uint32_t sel = (1u << (2 * i)) | (1u << (16 + 2 * i));
+            r1 |= e1 & sel;
+            r2 |= e2 & sel;
+        }
+        // even elements sit in bits 0,2,..14, odd ones in bits 16,18,..30: interleave
+        const uint32_t lo = (r1 & 0xFFFFu) | ((r1 >> 15) & 0xAAAAu);
+        const uint32_t hi = (r2 & 0xFFFFu) | ((r2 >> 15) & 0xAAAAu);
+        bm = (uint32_t)(__ffs((int)(lo | (hi << 16))) - 1) & 31u;
+    }
+    scales[blk] = (uint8_t)sb;
+    if (bm_index != nullptr) bm_index[blk] = (uint8_t)((kPlus && !dead) ? bm : 0u);
+    if (dead) {  // flushed or non-finite block: all codes zero (rare; the branch costs the others nothing)
+        if (kFmt == 8) {
+            uint4* out = reinterpret_cast<uint4*>(codes + blk * 32);
+            out[0] = make_uint4(0, 0, 0, 0);
+            out[1] = make_uint4(0, 0, 0, 0);
+        } else {
+            uint2* out = reinterpret_cast<uint2*>(codes + blk * 24);
+            out[0] = out[1] = out[2] = make_uint2(0, 0);
+        }
+        return;
+    }
+    const uint32_t inv2 = ((254u - sb) << 7) * 0x00010001u;  // 2^-shared_exp, twice
+    uint32_t w[8];  // four codes each, one per byte
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t y0 = bf16x2_mul(x[2 * i], inv2), y1 = bf16x2_mul(x[2 * i + 1], inv2);
+        w[i] = cvt_pair<kFmt>(__uint_as_float(y0 << 16), __uint_as_float(y0 & 0xFFFF0000u)) |
+               (cvt_pair<kFmt>(__uint_as_float(y1 << 16), __uint_as_float(y1 & 0xFFFF0000u)) << 16);
+    }
+    if (kPlus) {
+        // Sec. 4.1: the BM's stored mantissa is its fraction rounded to kMb bits (nearest, ties
+        // to even; bf16 has seven), clamped below the next binade; the cast's sign bit stays.
+        // Every word is patched under a mask (no branch on the BM's position).
+        const uint32_t frac = amax16 & 0x7Fu;
+        constexpr int sh = 7 - kMb;
+        uint32_t m = frac >> sh;
+        if (sh > 0) {
+            const uint32_t rem = frac & ((1u << sh) - 1u), half = 1u << (sh > 0 ? sh - 1 : 0);
+            m = min(m + ((rem > half || (rem == half && (m & 1u))) ? 1u : 0u), (1u << kMb) - 1u);
+        }
+        const uint32_t pos = 8u * (bm & 3u);
+        const uint32_t field = ((1u << kMb) - 1u) << pos, value = m << pos;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)  // w[i] = (w[i] & ~field) | value in the BM's word, predicated
+            asm("{ .reg .pred p;\n  setp.eq.u32 p, %1, %2;\n  @p lop3.b32 %0, %0, %3, %4, 0xBA; }"
+                : "+r"(w[i]) : "r"(bm >> 2), "r"((uint32_t)i), "r"(field), "r"(value));
+    }
+    if (kFmt == 8) {
+        uint4* out = reinterpret_cast<uint4*>(codes + blk * 32);
+        out[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        out[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    } else {
+        // bytes a b c d (six bits each) -> a | b << 6 | c << 12 | d << 18: pairs first (bits 14
+        // and 15 of the intermediate hold stray bits the second select drops), then the halves
+        uint32_t g[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t p = (w[i] & 0x003F003Fu) | ((w[i] >> 2) & ~0x003F003Fu);
+            g[i] = (p & 0xFFFu) | ((p >> 4) & ~0xFFFu);
+        }
+        uint2* out = reinterpret_cast<uint2*>(codes + blk * 24);
+        out[0] = make_uint2(__byte_perm(g[0], g[1], 0x4210), __byte_perm(g[1], g[2], 0x5421));
+        out[1] = make_uint2(__byte_perm(g[2], g[3], 0x6542), __byte_perm(g[4], g[5], 0x4210));
+        out[2] = make_uint2(__byte_perm(g[5], g[6], 0x5421), __byte_perm(g[6], g[7], 0x6542));
+    }
+}
+
 // Eq. 3 at the wider formats; exact in fp32 and bf16 (at most 8 significant bits).
 template <typename T, int kFmt, bool kPlus>
 __global__ void __launch_bounds__(kThreads)
@@ -249,6 +374,11 @@ cudaError_t launch_q(const void* src, int64_t rows, int64_t cols, int64_t ld_src
                      uint8_t* scales, uint8_t* bm_index, cudaStream_t stream)
 {
     const int64_t total = rows * (cols / 32);
+    if (sizeof(T) == 2 && ld_src == cols) {
+        quantize_wide_bf16_kernel<kFmt, kPlus><<<(unsigned)((total + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
+            static_cast<const uint4*>(src), total, codes, scales, bm_index);
+        return cudaGetLastError();
+    }
     quantize_wide_kernel<T, kFmt, kPlus><<<(unsigned)((total + kThreads - 1) / kThreads), kThreads, 0, stream>>>(
         static_cast<const T*>(src), ld_src, (int)(cols / 32), total, codes, scales, bm_index);
     return cudaGetLastError();
