@@ -500,11 +500,14 @@ __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t b
         w[i] = cvt_e2m1x8_bf16(bf16x2_mul(x[4 * i], inv2), bf16x2_mul(x[4 * i + 1], inv2),
                                bf16x2_mul(x[4 * i + 2], inv2), bf16x2_mul(x[4 * i + 3], inv2));
     if (kPlus) {
+        // the BM's three mantissa bits over the exponent and mantissa bits of its code, in the
+        // BM's word only: w[i] = (w[i] & ~field) | value under a predicate (no branch)
         const uint32_t sh = (bm & 7u) * 4u;
+        const uint32_t field = 7u << sh, value = m << sh;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if ((bm >> 3) == (uint32_t)i)
-                asm("bfi.b32 %0, %1, %0, %2, 3;" : "+r"(w[i]) : "r"(m), "r"(sh));
+            asm("{ .reg .pred p;\n  setp.eq.u32 p, %1, %2;\n  @p lop3.b32 %0, %0, %3, %4, 0xBA; }"
+                : "+r"(w[i]) : "r"(bm >> 3), "r"((uint32_t)i), "r"(field), "r"(value));
     }
     const uint4 outv = dead ? make_uint4(0, 0, 0, 0) : make_uint4(w[0], w[1], w[2], w[3]);
     __stcs(nibbles + blk, outv);
