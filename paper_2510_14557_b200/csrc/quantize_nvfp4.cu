@@ -250,8 +250,10 @@ __device__ __forceinline__ void nvfp4_block(const uint32_t* raw, float ts, float
 #undef X
 }
 
+// (bf16 rows in the short-operand form fit 32 registers: eight CTAs per SM hide the load latency
+// this HBM-bound kernel is exposed to -- 40.0 -> 36.2 us on 8192 x 8192 against four CTAs)
 template <typename T, bool kPlus, bool kShort>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, (sizeof(T) == 2 && kShort) ? 8 : 4)
 nvfp4_quantize_kernel(const T* __restrict__ src, int64_t ld_src, int64_t units_per_row,
                       int64_t total_units, float ts, uint4* __restrict__ nibbles,
                       uint16_t* __restrict__ scales, uint8_t* __restrict__ bm_index)
