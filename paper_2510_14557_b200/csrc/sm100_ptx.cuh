@@ -103,29 +103,6 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
     }
 }
 
-// The same for a whole warp (all 32 lanes must call it): lane 0 polls, the outcome is shared.
-// The lanes' own polls of one barrier are handled one after the other, so a warp-wide wait
-// costs 32 barrier operations per poll; a dozen warps waiting that way on every stage of a
-// pipeline spend more time on the barrier than on their work.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
-                                               long long limit_cycles)
-{
-    uint32_t ok = 0;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort, limit_cycles) ? 1u : 0u;
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    __syncwarp();  // what lane 0 may see after its wait, the other lanes may see too
-    return ok != 0u;
-}
-__device__ __forceinline__ bool mbar_wait_relaxed_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
-                                                       long long limit_cycles, unsigned pause_ns)
-{
-    uint32_t ok = 0;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait_relaxed(bar, parity, abort, limit_cycles, pause_ns) ? 1u : 0u;
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    __syncwarp();
-    return ok != 0u;
-}
-
 // ---------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
