@@ -41,7 +41,7 @@ NOMINAL_FP4_OVER_BF16 = 4.0  # 9 PF dense FP4 vs 2.25 PF dense bf16
 NOMINAL_FP8_OVER_BF16 = 2.0  # 4.5 PF dense for 8-bit containers (kind::mxf8f6f4)
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemm_tc_stream_kernel<wide> launch, from
 # single-pass ncu captures of this program (summaries under profiles/); bytes per launch.
-NCU_DRAM_TRAFFIC = {"cfg5": 922.96e6 + 450.60e6, "cfg4": 26.11e6 + 72.7e3}
+NCU_DRAM_TRAFFIC = {"cfg5": 531.75e6 + 441.83e6, "cfg4": 19.82e6 + 64.8e3}
 
 
 def measured_peaks():

@@ -231,9 +231,12 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
  * N x K weights) that work can be done once.  Which form a GEMM reads depends on both
  * operands' modes; mxp_gemm_prepack_form tells:
  *   MXP_PREPACK_PLAIN  scale atoms only: B is MXFP4 and A is MXFP4 or MXFP4+
- *   MXP_PREPACK_WIDE   16 bytes per 16 elements (E2M3 codes or, for MX++ and MXFP8, E4M3
- *                      bytes: exact for every E2M1 value and for the BM values of Eq. 3):
- *                      both operands MX+, the wider modes, and the weight-only tensor-core path
+ *   MXP_PREPACK_WIDE   12 bytes per 16 elements: E2M3 codes (exact for every E2M1 value and
+ *                      for the BM values of Eq. 3), packed; the tensor map spreads them into
+ *                      the 16-byte slots the tensor core reads.  B is MXFP4, MXFP4+ or MXFP6
+ *                      and the pairing is not one of the two above or below: both operands
+ *                      MX+, the wider modes, and the weight-only tensor-core path
+ *   MXP_PREPACK_WIDE8  16 bytes per 16 elements: E4M3 bytes, where B is MX++ or MXFP8
  *   MXP_PREPACK_SPLIT  B is MXFP4+ and A is MXFP4: Eq. 4's split for the sparse residual
  *                      instruction -- B's nibble plane with BM_H in every BM's place, BM_L
  *                      compressed 2:1, and the metadata that says where each BM_L sits
@@ -258,14 +261,15 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
  * an implementation device of this library.
  *   mxp_gemm_dense_prepacked  the weight-only form (bf16 activations, more than one tile's
  *                           worth of rows is where it pays: see mxp_gemm) with B's prepacked
- *                           copy in the form MXP_PREPACK_WIDE (size checked as above).  Workspace
+ *                           copy in its widened form, MXP_PREPACK_WIDE or, for MX++ weights,
+ *                           MXP_PREPACK_WIDE8 (size checked as above).  Workspace
  *                           (device, 256-byte aligned): at least
  *                           mxp_gemm_dense_prepacked_workspace_bytes(M, K) bytes (0: shape
  *                           not supported), which hold the activations' two planes and
  *                           scales.  Any M >= 1; 4-bit weight modes; K % 128 == 0.  Same
  *                           result as mxp_gemm's tensor-core weight-only path.
  */
-typedef enum { MXP_PREPACK_PLAIN = 0, MXP_PREPACK_WIDE = 1, MXP_PREPACK_SPLIT = 2 } mxp_prepack_form;
+typedef enum { MXP_PREPACK_PLAIN = 0, MXP_PREPACK_WIDE = 1, MXP_PREPACK_SPLIT = 2, MXP_PREPACK_WIDE8 = 3 } mxp_prepack_form;
 int mxp_gemm_prepack_form(mxp_mode a_mode, mxp_mode b_mode);
 size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int form);
 mxp_status mxp_gemm_prepack(const mxp_packed *P, int form, void *out, size_t out_bytes,

@@ -358,7 +358,7 @@ mxp_status mxp_gemm_prepack(const mxp_packed* P, int form, void* out, size_t out
                             void* cuda_stream)
 {
     if (!valid_packed(P, true)) return MXP_ERR_INVALID_ARG;
-    if (form < MXP_PREPACK_PLAIN || form > MXP_PREPACK_SPLIT) return MXP_ERR_INVALID_ARG;
+    if (form < MXP_PREPACK_PLAIN || form > MXP_PREPACK_WIDE8) return MXP_ERR_INVALID_ARG;
     if (P->rows == 0 || P->cols == 0) return MXP_OK;
     if (P->mode != MXP_MODE_MXFP4 && form == MXP_PREPACK_PLAIN) return MXP_ERR_INVALID_ARG;
     if (P->mode != MXP_MODE_MXFP4_PLUS && form == MXP_PREPACK_SPLIT) return MXP_ERR_INVALID_ARG;
@@ -387,7 +387,7 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
     const size_t want = mxp::stream_prepack_bytes(N, K, form);
     if (want == 0) return MXP_ERR_UNSUPPORTED;
     if (B_prepacked_bytes != want || !aligned(B_prepacked, 256)) return MXP_ERR_INVALID_ARG;
-    if (form != MXP_PREPACK_WIDE &&
+    if (form != MXP_PREPACK_WIDE && form != MXP_PREPACK_WIDE8 &&
         mxp::stream_sparse_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode, true) != 0)
         return mxp::launch_gemm_tc_sparse(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
                                           workspace, workspace_bytes,
@@ -417,8 +417,9 @@ mxp_status mxp_gemm_dense_prepacked(int64_t M, int64_t N, int64_t K, const void*
     if (B_prepacked == nullptr || D == nullptr || ldd < N) return MXP_ERR_INVALID_ARG;
     if (!aligned(D, d_dt == MXP_BF16 ? 2 : 4)) return MXP_ERR_INVALID_ARG;
     const size_t need = mxp::stream_dense_prepacked_workspace_bytes(M, K);
-    if (need == 0 || mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) == 0) return MXP_ERR_UNSUPPORTED;
-    if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) || !aligned(B_prepacked, 256))
+    const int wform = mxp::stream_wide_form(B_packed->mode);
+    if (need == 0 || mxp::stream_prepack_bytes(N, K, wform) == 0) return MXP_ERR_UNSUPPORTED;
+    if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, wform) || !aligned(B_prepacked, 256))
         return MXP_ERR_INVALID_ARG;
     if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
     mxp_packed none = {};
@@ -492,7 +493,8 @@ mxp_status mxp_gemm_ready(int64_t M, int64_t N, int64_t K, const mxp_packed* A_p
         return mxp::launch_gemm_tc_sparse(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd, workspace,
                                           workspace_bytes, static_cast<cudaStream_t>(cuda_stream), true);
     }
-    if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, MXP_PREPACK_WIDE) || !aligned(B_prepacked, 256))
+    if (B_prepacked_bytes != mxp::stream_prepack_bytes(N, K, mxp::stream_wide_form(B_packed->mode)) ||
+        !aligned(B_prepacked, 256))
         return MXP_ERR_INVALID_ARG;
     return mxp::launch_gemm_tc_stream(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
                                       workspace, workspace_bytes,

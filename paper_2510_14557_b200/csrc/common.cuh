@@ -116,6 +116,8 @@ mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_pack
                                  bool a_ready = false);
 // The form of B's prepacked copy that a packed x packed GEMM with these modes reads.
 int stream_b_form(mxp_mode a_mode, mxp_mode b_mode);
+// The widened form of an operand of this mode: MXP_PREPACK_WIDE (E2M3 codes) or MXP_PREPACK_WIDE8 (E4M3 bytes).
+int stream_wide_form(mxp_mode b_mode);
 
 // Kernel choices a test or a measurement may force (mxp_debug_override): process-wide, 0 = the
 // library decides.

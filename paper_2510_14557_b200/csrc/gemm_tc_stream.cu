@@ -267,6 +267,12 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
             uint32_t c = 0;
             bool ok = true;
+            // Bytes the barrier of a stage sees from both CTAs' copies.  E2M3 operands lie packed in
+            // global memory, 12 bytes per 16 codes, and the copy spreads them into 16-byte slots:
+            // the barrier counts the 12.
+            const uint32_t stage_tx =
+                2u * (uint32_t)(C::kStageRaw - ((kWide && prm.a_fmt == kFmtE2M3) ? kHalfTile / 4 : 0) -
+                                ((kWide && prm.b_fmt == kFmtE2M3) ? kHalves * C::kBTile / 4 : 0));
             for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
                 int tm, tn;
                 tile_coords(tile, tiles_m, tiles_n, tm, tn);
@@ -289,7 +295,7 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap tmap_a,
                         ok = false;
                         break;
                     }
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], 2 * C::kStageRaw);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full[s], stage_tx);
                     ptx::tma_load_2d_pair(a_tile(s), &tmap_a, full0 + 8u * (uint32_t)s, ka * kRowBytes, ya + m0);
 #pragma unroll
                     for (int j = 0; j < kHalves; ++j)
@@ -555,7 +561,7 @@ struct PrepackOperand {
     int eight_plus;           // MXFP8+: E4M3 bytes whose BM is an E0M7 code, entered as three planes
     size_t plane_bytes;       // MXFP6+: distance to the second plane of the widened copy, else 0
     unsigned scale_ctas;      // row groups * ceil(nbk/128)
-    unsigned widen_ctas;      // ceil(rows * nbk * 2 / 256), 0 when not widened
+    unsigned widen_ctas;      // CTAs of 256 widening threads (a block or half a block each), 0 when not widened
     // Eq. 4 split of an MXFP4+ operand for the sparse residual MMA (nullptr / 0: not wanted)
     uint8_t* sp_main;         // [rows][K/2]: the nibble plane with BM_H in every BM's place
     uint8_t* sp_res;          // [rows][K/4]: BM_L, 2:1 compressed
@@ -619,36 +625,57 @@ __device__ __forceinline__ void set_code6(uint4& v, uint32_t bit, uint32_t code)
 // of two that are, 4 + (m >> 2)/2 in the first plane (code s 11 hhh) and (m & 3)/8 in a second
 // plane that is zero everywhere else (subnormal code s 00 0ll); the GEMM adds the products of
 // both planes (Eq. 4's split at this width, with dense residual passes).
-__device__ __forceinline__ void widen_six(const PrepackOperand& op, uint32_t t, uint32_t b)
+// Sixteen 6-bit codes (x, y, z of `o`) to their 12 bytes: the operand lies packed in global
+// memory and the tensor map (16 codes to a 16-byte slot) adds the padding on the way in.
+// Threads t (even) and t + 1 are neighbouring lanes and hold the two halves of one block: its 24
+// bytes leave as three 8-byte stores, the middle one put together with one shuffle.  All lanes
+// of the warp must call it (`live`: this lane has something to store; a block's two halves are
+// live or not together).
+__device__ __forceinline__ void store_codes6(uint8_t* half0, const uint4 o, bool odd, bool live)
 {
-    const uint32_t* in = reinterpret_cast<const uint32_t*>(op.nibbles) + (size_t)t * 3u;
-    uint4 o = make_uint4(in[0], in[1], in[2], 0u), lo = make_uint4(0u, 0u, 0u, 0u);
-    const uint32_t sc = op.scales[b];
-    if (op.bm_index != nullptr) {
-        const uint32_t p = op.bm_index[b] & 31u;
-        if ((p >> 4) == (t & 1u)) {
-            const uint32_t bit = 6u * (p & 15u);
-            const uint32_t x[4] = {o.x, o.y, o.z, o.w};
-            const uint32_t wi = bit >> 5;
-            const unsigned long long win =
-                (unsigned long long)(wi == 0 ? x[0] : wi == 1 ? x[1] : x[2]) |
-                ((unsigned long long)(wi == 0 ? x[1] : wi == 1 ? x[2] : x[3]) << 32);
-            const uint32_t code = (uint32_t)(win >> (bit & 31u)) & 63u;
-            const uint32_t sign = code & 32u, m = code & 31u;
-            set_code6(o, bit, sign | 0x18u | (m >> 2));
-            set_code6(lo, bit, sign | (m & 3u));
-        }
+    const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, odd ? o.x : o.z, 1);  // even lane: partner's x
+    if (!live) return;
+    uint2* w = reinterpret_cast<uint2*>(half0);  // the block's first byte: 8-byte aligned
+    if (!odd) {
+        w[0] = make_uint2(o.x, o.y);
+        w[1] = make_uint2(o.z, other);
+    } else {
+        w[2] = make_uint2(o.y, o.z);
     }
-    if (sc == 0u) o = lo = make_uint4(0u, 0u, 0u, 0u);
-    uint8_t* dst = op.wide + (size_t)t * 16u;
-    *reinterpret_cast<uint4*>(dst) = o;
-    if (op.plane_bytes != 0) *reinterpret_cast<uint4*>(dst + op.plane_bytes) = lo;
+}
+__device__ __forceinline__ void widen_six(const PrepackOperand& op, uint32_t t, uint32_t b, bool live)
+{
+    uint4 o = make_uint4(0u, 0u, 0u, 0u), lo = o;
+    if (live) {
+        const uint32_t* in = reinterpret_cast<const uint32_t*>(op.nibbles) + (size_t)t * 3u;
+        o = make_uint4(in[0], in[1], in[2], 0u);
+        const uint32_t sc = op.scales[b];
+        if (op.bm_index != nullptr) {
+            const uint32_t p = op.bm_index[b] & 31u;
+            if ((p >> 4) == (t & 1u)) {
+                const uint32_t bit = 6u * (p & 15u);
+                const uint32_t x[4] = {o.x, o.y, o.z, o.w};
+                const uint32_t wi = bit >> 5;
+                const unsigned long long win =
+                    (unsigned long long)(wi == 0 ? x[0] : wi == 1 ? x[1] : x[2]) |
+                    ((unsigned long long)(wi == 0 ? x[1] : wi == 1 ? x[2] : x[3]) << 32);
+                const uint32_t code = (uint32_t)(win >> (bit & 31u)) & 63u;
+                const uint32_t sign = code & 32u, m = code & 31u;
+                set_code6(o, bit, sign | 0x18u | (m >> 2));
+                set_code6(lo, bit, sign | (m & 3u));
+            }
+        }
+        if (sc == 0u) o = lo = make_uint4(0u, 0u, 0u, 0u);
+    }
+    store_codes6(op.wide + (size_t)b * 24u, o, (t & 1u) != 0u, live);
+    if (op.plane_bytes != 0) store_codes6(op.wide + op.plane_bytes + (size_t)b * 24u, lo, (t & 1u) != 0u, live);
 }
 
-// One thread per 16 elements (half a block): 8 bytes of codes in, 16 bytes out.
-//  * E2M3 (MXFP4 and MXFP4+ operands): the 16 six-bit codes packed into 12 bytes, then 4 bytes
-//    of padding, which is how kind::mxf8f6f4 reads 6-bit operands from shared memory.  The BM of
-//    an MX+ block, 4 + m/2 (Eq. 3), is the E2M3 code s 11 mmm.
+// One thread per 32 (MXFP4, MXFP4+) or 16 elements (the other modes): 12 or 16 bytes out per 16 codes.
+//  * E2M3 (MXFP4 and MXFP4+ operands): the 16 six-bit codes packed into 12 bytes; kind::mxf8f6f4
+//    reads 6-bit operands from shared memory as 12 bytes and 4 bytes of padding, which the
+//    tensor map's packed 6-bit type adds on the way in, so that global memory and L2 hold 12.
+//    The BM of an MX+ block, 4 + m/2 (Eq. 3), is the E2M3 code s 11 mmm.
 //  * E4M3 (MX++ operands, whose rescaled values need the exponent range): one byte per code.
 // E4M3 code (sign 0) of a positive integer with at most four significant bits.
 __device__ __forceinline__ uint32_t e4m3_of_small_int(uint32_t x)
@@ -695,10 +722,27 @@ __device__ __forceinline__ void widen_eight_plus(const PrepackOperand& op, uint3
 
 __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned id)
 {
+    if (!op.pp && !op.eight_plus && !op.eight && !op.six) {
+        // MXFP4 / MXFP4+ -> E2M3: a thread per block, 16 bytes in, 24 bytes out
+        const uint32_t blk = id * 256u + threadIdx.x;
+        if (blk >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
+        const uint4 w = __ldg(reinterpret_cast<const uint4*>(op.nibbles) + blk);
+        const uint32_t p = op.bm_index != nullptr ? op.bm_index[blk] & 31u : 32u;
+        // Eq. 3, BM branch included, in the half that holds the BM
+        uint4 s0 = e2m1x16_to_e2m3_slot(w.x, w.y, p < 16u ? p : 16u);
+        uint4 s1 = e2m1x16_to_e2m3_slot(w.z, w.w, (p >= 16u && p < 32u) ? p - 16u : 16u);
+        if (op.scales[blk] == 0u) s0 = s1 = make_uint4(0u, 0u, 0u, 0u);
+        uint2* out = reinterpret_cast<uint2*>(op.wide + (size_t)blk * 24u);
+        out[0] = make_uint2(s0.x, s0.y);
+        out[1] = make_uint2(s0.z, s1.x);
+        out[2] = make_uint2(s1.y, s1.z);
+        return;
+    }
     const uint32_t t = id * 256u + threadIdx.x;  // half block: 16 elements
     const uint32_t b = t >> 1;
-    if (b >= (uint32_t)op.rows * (uint32_t)op.nbk) return;
-    if (op.six) return widen_six(op, t, b);
+    const bool live = b < (uint32_t)op.rows * (uint32_t)op.nbk;
+    if (op.six) return widen_six(op, t, b, live);  // (every lane takes part in its stores)
+    if (!live) return;
     if (op.eight_plus) return widen_eight_plus(op, t, b);
     if (op.eight) {
         // MXFP8: one byte per element already; a flushed block's codes are zero by construction
@@ -714,12 +758,6 @@ __device__ __forceinline__ void widen_codes(const PrepackOperand& op, unsigned i
     const uint32_t nib = (((e & 8u) ? w.y : w.x) >> ((e & 7u) * 4u)) & 15u;
     const bool has_bm = op.bm_index != nullptr && (p >> 4) == (t & 1u);
     uint8_t* dst = op.wide + (size_t)t * 16u;
-    if (!op.pp) {
-        uint4 o = e2m1x16_to_e2m3_slot(w.x, w.y, has_bm ? e : 16u);  // Eq. 3, BM branch included
-        if (sc == 0u) o = make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(dst) = o;
-        return;
-    }
     // MX++: BM scaled up by 2^shift, NBMs down by 2^-(delta - shift) (see mxpp_shift)
     const uint32_t delta = ib >> 5;
     const uint32_t shift = mxpp_shift(sc, delta);
@@ -833,6 +871,23 @@ bool make_tmap_rows(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t r
               MXP_S_L2PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D tensor of 6-bit codes [rows][K], 16 codes packed into 12 bytes in global memory and spread
+// into 16-byte slots in shared memory (the form kind::mxf8f6f4 reads): boxes of 128 codes (a
+// 128-byte swizzle span in shared memory) x box_rows rows.  The base must be 32-byte aligned and
+// K a multiple of 128; the innermost coordinate of a copy is in codes, a multiple of 128.
+bool make_tmap_rows6(CUtensorMap* m, const uint8_t* base, int64_t rows, int64_t K, int box_rows)
+{
+    EncodeFn fn = tensormap_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 3 / 4};
+    const cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_16U6_ALIGN16B, 2, const_cast<uint8_t*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              MXP_S_L2PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Scale atoms as a 3-D tensor of 32-bit words [row groups][K groups][128], boxes of
 // 128 x kgroups_per_stage x rgs.
 bool make_tmap_atoms(CUtensorMap* m, const uint8_t* base, int64_t rgs_total, int64_t kgroups,
@@ -864,6 +919,9 @@ inline int mode_parts(mxp_mode m)
 }
 inline bool mode_six(mxp_mode m) { return m == MXP_MODE_MXFP6 || m == MXP_MODE_MXFP6_PLUS; }
 inline bool mode_eight(mxp_mode m) { return m == MXP_MODE_MXFP8 || m == MXP_MODE_MXFP8_PLUS; }
+// Bits per code of an operand's widened form: E4M3 bytes for MX++ and MXFP8(+), E2M3 codes
+// packed 16 to 12 bytes for the rest.
+inline int wide_bits(mxp_mode m) { return (m == MXP_MODE_MXFP4_PP || mode_eight(m)) ? 8 : 6; }
 inline bool mode_plus(mxp_mode m)
 {
     return m == MXP_MODE_MXFP4_PLUS || m == MXP_MODE_MXFP4_PP || m == MXP_MODE_MXFP6_PLUS ||
@@ -1048,14 +1106,16 @@ struct PackedLayout {
     size_t atoms[2];  // scale atoms tiled for one-half tiles, for two-half tiles
     size_t wide, total;
 };
-PackedLayout packed_layout(int64_t rows, int64_t K, bool wide)
+// bits: 0 (scale atoms only), 6 or 8 (widened codes behind them)
+PackedLayout packed_layout(int64_t rows, int64_t K, int bits)
 {
+    const bool wide = bits != 0;
     PackedLayout l;
     l.atoms[0] = 0;
     l.atoms[1] = round_up((size_t)row_groups(rows, sub_n(wide, 1)) * (size_t)(K / 128) * kAtom, 1024);
     l.wide = l.atoms[1] +
              round_up((size_t)row_groups(rows, sub_n(wide, 2)) * (size_t)(K / 128) * kAtom, 1024);
-    l.total = l.wide + (wide ? round_up((size_t)rows * (size_t)K, 1024) : 0);
+    l.total = l.wide + round_up((size_t)rows * (size_t)K * (size_t)bits / 8, 1024);
     return l;
 }
 
@@ -1072,14 +1132,16 @@ PrepackOperand prepack_operand(const mxp_packed& P, int64_t rows, int64_t K, boo
     op.six = mode_six(P.mode);
     op.eight = P.mode == MXP_MODE_MXFP8;
     op.eight_plus = P.mode == MXP_MODE_MXFP8_PLUS;
-    op.plane_bytes = mode_parts(P.mode) > 1 ? (size_t)rows * (size_t)K : 0;
+    op.plane_bytes = mode_parts(P.mode) > 1 ? (size_t)rows * (size_t)K * (size_t)wide_bits(P.mode) / 8 : 0;
     op.atoms = atoms;
     op.wide = wide ? wide_bytes : nullptr;
     op.rows = (int)rows;
     op.nbk = nbk;
     op.tile_rows = tile_rows;
     op.scale_ctas = (unsigned)(row_groups(rows, tile_rows) * ((kgroups + 31) / 32));
-    op.widen_ctas = wide ? (unsigned)((rows * nbk * 2 + 255) / 256) : 0u;
+    // a thread per block for the 4-bit modes that widen to E2M3, per half block otherwise
+    const bool per_block = !op.pp && !op.six && !op.eight && !op.eight_plus;
+    op.widen_ctas = wide ? (unsigned)((rows * nbk * (per_block ? 1 : 2) + 255) / 256) : 0u;
     op.sp_main = op.sp_res = op.sp_meta = nullptr;
     op.sp_stages = op.sp_row_groups = 0;
     op.split_ctas = 0u;
@@ -1169,19 +1231,22 @@ PrepackOperand no_operand()
 
 size_t stream_prepack_bytes(int64_t rows, int64_t K, int form)
 {
-    if (rows <= 0 || K <= 0 || K % 128 != 0 || form < 0 || form > 2) return 0;
+    if (rows <= 0 || K <= 0 || K % 128 != 0 || form < 0 || form > MXP_PREPACK_WIDE8) return 0;
     if ((uint64_t)rows * (uint64_t)K / 16 >= (1ull << 32)) return 0;
-    if (form == 2) return split_layout(rows, K).total;
-    return packed_layout(rows, K, form == 1).total;
+    if (form == MXP_PREPACK_SPLIT) return split_layout(rows, K).total;
+    return packed_layout(rows, K, form == MXP_PREPACK_WIDE ? 6 : form == MXP_PREPACK_WIDE8 ? 8 : 0).total;
 }
+
+int stream_wide_form(mxp_mode b_mode) { return wide_bits(b_mode) == 8 ? MXP_PREPACK_WIDE8 : MXP_PREPACK_WIDE; }
 
 mxp_status stream_prepack(const mxp_packed& P, int form, void* out, size_t out_bytes,
                           cudaStream_t stream)
 {
-    const bool wide = form == 1;
+    const bool wide = form == MXP_PREPACK_WIDE || form == MXP_PREPACK_WIDE8;
     const size_t need = stream_prepack_bytes(P.rows, P.cols, form);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
-    if (form == 2) {
+    if (wide && form != stream_wide_form(P.mode)) return MXP_ERR_INVALID_ARG;  // 6-bit codes or bytes: the mode's
+    if (form == MXP_PREPACK_SPLIT) {
         if (P.mode != MXP_MODE_MXFP4_PLUS) return MXP_ERR_UNSUPPORTED;
         if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
         if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
@@ -1202,7 +1267,7 @@ mxp_status stream_prepack(const mxp_packed& P, int form, void* out, size_t out_b
         (reinterpret_cast<uintptr_t>(P.scales) & 3) ||
         (P.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(P.bm_index) & 3)))
         return MXP_ERR_INVALID_ARG;
-    const PackedLayout l = packed_layout(P.rows, P.cols, wide);
+    const PackedLayout l = packed_layout(P.rows, P.cols, wide ? wide_bits(P.mode) : 0);
     uint8_t* o = static_cast<uint8_t*>(out);
     // both tilings of the scales (the GEMM picks its tile shape per call); widened bytes once
     const PrepackOperand p1 =
@@ -1272,7 +1337,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
         (B.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(B.bm_index) & 3)))
         return MXP_ERR_INVALID_ARG;
 
-    const PackedLayout lb = packed_layout(N, K, wide);
+    const PackedLayout lb = packed_layout(N, K, wide ? wide_bits(B.mode) : 0);
     const uint8_t* b_atoms =
         b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms[halves - 1] : ws + l.sfb;
     const uint8_t* b_wide = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.wide : ws + l.wb;
@@ -1300,8 +1365,10 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     CUtensorMap ta, tb, tsa, tsb;
     const int box_kg = wide ? 1 : 2;
     const bool maps_ok =
-        (wide ? make_tmap_rows(&ta, ws + l.wa, M * parts_a, K, 128) &&
-                    make_tmap_rows(&tb, b_wide, N * parts_b, K, sub / 2)
+        (wide ? ((dense || wide_bits(A.mode) == 8) ? make_tmap_rows(&ta, ws + l.wa, M * parts_a, K, 128)
+                                                     : make_tmap_rows6(&ta, ws + l.wa, M * parts_a, K, 128)) &&
+                    (wide_bits(B.mode) == 8 ? make_tmap_rows(&tb, b_wide, N * parts_b, K, sub / 2)
+                                            : make_tmap_rows6(&tb, b_wide, N * parts_b, K, sub / 2))
               : make_tmap_rows(&ta, A.nibbles, M, K / 2, 128) &&
                     make_tmap_rows(&tb, B.nibbles, N, K / 2, sub / 2)) &&
         make_tmap_atoms(&tsa, ws + l.sfa, rga, kgroups, box_kg, 1) &&
@@ -1338,7 +1405,7 @@ int stream_b_form(mxp_mode a_mode, mxp_mode b_mode)
                            (a_mode == MXP_MODE_MXFP4 && b_mode == MXP_MODE_MXFP4_PLUS);
     if (one_sided && override_get(MXP_KNOB_ONE_SIDED) != 1)
         return b_mode == MXP_MODE_MXFP4_PLUS ? MXP_PREPACK_SPLIT : MXP_PREPACK_PLAIN;
-    return (a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4) ? MXP_PREPACK_WIDE : MXP_PREPACK_PLAIN;
+    return (a_mode != MXP_MODE_MXFP4 || b_mode != MXP_MODE_MXFP4) ? stream_wide_form(b_mode) : MXP_PREPACK_PLAIN;
 }
 
 // One operand MXFP4+, the other MXFP4 (see the head of this file).  0: not supported.
@@ -1406,7 +1473,7 @@ mxp_status launch_gemm_tc_sparse(int64_t M, int64_t N, int64_t K, const mxp_pack
     const uint8_t* x_base = x_pre ? static_cast<const uint8_t*>(b_prepacked) : ws + l.x;
     const SplitLayout lx = split_layout(rows_x, K);
     const uint8_t* y_atoms =
-        y_pre ? static_cast<const uint8_t*>(b_prepacked) + packed_layout(rows_y, K, false).atoms[halves - 1]
+        y_pre ? static_cast<const uint8_t*>(b_prepacked) + packed_layout(rows_y, K, 0).atoms[halves - 1]
               : ws + l.y;
     const PrepackOperand px = (x_pre || a_ready) ? no_operand() : split_operand(X, ws + l.x);
     const PrepackOperand py =

@@ -417,13 +417,13 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8_bf16(uint32_t p0, uint32_t p1, ui
 // What the kReady variant also writes: the operand in the form the streamed tensor-core GEMM
 // reads (Sec. 5: quantization fused with the preparation of the matrix-multiply operand), i.e.
 // what prepack_kernel would make of the packed planes: the scale byte inside its 32-row x
-// 16-byte atom and either (kReady = 1) the block's 32 codes as two 16-byte slots of E2M3 codes,
+// 16-byte atom and either (kReady = 1) the block's 32 codes as E2M3 codes packed into 24 bytes,
 // BM included, or (kReady = 2, MXFP4+ against a plain MXFP4 partner) Eq. 4's split for the
 // sparse residual instruction: the codes with BM_H in the BM's place, BM_L 2:1 compressed,
 // and the metadata nibbles that say where it sits.
 struct GemmReady {
     uint8_t* atoms;      // [ceil(rows/128)][nbk/4][512]
-    uint4* slots;        // kReady = 1: [rows][nbk][2]
+    uint4* slots;        // kReady = 1: [rows][nbk] records of 24 bytes (32 E2M3 codes)
     uint4* sp_main;      // kReady = 2: [rows][nbk] codes with BM_H
     uint2* sp_res;       //             [rows][nbk] compressed BM_L
     uint8_t* sp_meta;    //             [row group of 128][stage of 8 blocks][128 rows x 16 bytes]
@@ -548,8 +548,11 @@ __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t b
         const uint32_t p = (kPlus && !dead) ? bm : 32u;  // BM position, none in a dead block
         uint4 s0 = e2m1x16_to_e2m3_slot(outv.x, outv.y, p < 16u ? p : 16u);
         uint4 s1 = e2m1x16_to_e2m3_slot(outv.z, outv.w, (p >= 16u && p < 32u) ? p - 16u : 16u);
-        __stcs(ready.slots + 2 * blk, s0);
-        __stcs(ready.slots + 2 * blk + 1, s1);
+        // 32 six-bit codes = 24 bytes (the GEMM's tensor map spreads every 12 into a 16-byte slot)
+        uint2* out6 = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(ready.slots) + blk * 24);
+        __stcs(out6, make_uint2(s0.x, s0.y));
+        __stcs(out6 + 1, make_uint2(s0.z, s1.x));
+        __stcs(out6 + 2, make_uint2(s1.y, s1.z));
         const int64_t row = blk / ready.nbk;
         const int kb = (int)(blk - row * ready.nbk);
         const int r = (int)(row & 127);

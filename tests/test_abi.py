@@ -127,13 +127,15 @@ def test_prepacked_copies_are_checked_against_the_call(lib):
     fake = ctypes.c_void_p(4096)
     M, N, K = 512, 384, 256
     MX, MXP = 0, 1
-    PLAIN, WIDE, SPLIT = 0, 1, 2
+    PLAIN, WIDE, SPLIT, WIDE8 = 0, 1, 2, 3
     form = lib.mxp_gemm_prepack_form
     assert (form(MX, MX), form(MXP, MX), form(MX, MXP), form(MXP, MXP)) == (PLAIN, PLAIN, SPLIT, WIDE)
-    assert form(2, MX) == WIDE and form(MX, 2) == WIDE          # MX++ is read widened
-    size = {f: lib.mxp_gemm_prepack_bytes(N, K, f) for f in (PLAIN, WIDE, SPLIT)}
-    assert 0 < size[PLAIN] < size[SPLIT] < size[WIDE]
-    assert lib.mxp_gemm_prepack_bytes(N, K, 3) == 0 and lib.mxp_gemm_prepack_bytes(N, 96, WIDE) == 0
+    # MX++ is read widened: the partner as 6-bit E2M3 codes, the MX++ operand itself as E4M3 bytes
+    assert form(2, MX) == WIDE and form(MX, 2) == WIDE8 and form(MXP, 5) == WIDE8 and form(MXP, 3) == WIDE
+    size = {f: lib.mxp_gemm_prepack_bytes(N, K, f) for f in (PLAIN, WIDE, SPLIT, WIDE8)}
+    assert 0 < size[PLAIN] < min(size[SPLIT], size[WIDE]) and size[WIDE] < size[WIDE8] and len(set(size.values())) == 4
+    assert size[WIDE] - size[PLAIN] == N * K * 3 // 4 and size[WIDE8] - size[PLAIN] == N * K
+    assert lib.mxp_gemm_prepack_bytes(N, K, 4) == 0 and lib.mxp_gemm_prepack_bytes(N, 96, WIDE) == 0
     ws = 1 << 30
     gp = lib.mxp_gemm_prepacked
 
@@ -144,7 +146,7 @@ def test_prepacked_copies_are_checked_against_the_call(lib):
 
     for amode, bmode in ((MX, MX), (MXP, MX), (MX, MXP), (MXP, MXP)):
         right = form(amode, bmode)
-        for f in (PLAIN, WIDE, SPLIT):
+        for f in (PLAIN, WIDE, SPLIT, WIDE8):
             if f != right:
                 assert call(amode, bmode, size[f]) == 1, (amode, bmode, f)
         assert call(amode, bmode, lib.mxp_gemm_prepack_bytes(N + 128, K, right)) == 1  # another shape's copy
@@ -161,3 +163,6 @@ def test_prepacked_copies_are_checked_against_the_call(lib):
     assert pk(ctypes.byref(a), PLAIN, fake, ws, null) == 1      # an MXFP4+ operand has no plain form
     assert pk(ctypes.byref(b), SPLIT, fake, ws, null) == 1      # a plain operand has nothing to split
     assert pk(ctypes.byref(a), 7, fake, ws, null) == 1
+    assert pk(ctypes.byref(a), WIDE8, fake, ws, null) == 1      # E2M3 codes are this operand's widened form
+    pp = _Packed(4096, 4096, 4096, N, K, 2)
+    assert pk(ctypes.byref(pp), WIDE, fake, ws, null) == 1      # ... and E4M3 bytes an MX++ operand's
