@@ -291,31 +291,43 @@ __device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, in
     eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 1));
     eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 2));
     const bool nonfinite = eb == 255u;
-    // t = |a| / 2^(E - 12), rounded to an integer below 2^13, plus 4 in each of five octal
-    // places: octal digit j of t, minus 4, is the balanced digit d_j in -4..3 with
-    // |a| = sum_j d_j 2^(E - 3 j)
-    // The digit's code comes from a table of eight nibbles indexed by the octal digit (sign bit =
-    // the element's sign, flipped for the negative digits 0..3): E2M1 codes of 4 3 2 1 0 1 2 3.
-    uint32_t t[8], lut[8];
+    // t = |a| / 2^(E - 12), rounded to an integer below 2^13 (half up), plus 4 in each of five
+    // octal places: octal digit j of t, minus 4, is the balanced digit d_j in -4..3 with
+    // |a| = sum_j d_j 2^(E - 3 j).  The scaling is a multiply by a power of two (exact), the
+    // rounding an add of one half and a truncating conversion (the sum is exact wherever the
+    // truncation could depend on it).  2^(12 - E) has exponent field 266 - eb: beyond 254 (blocks
+    // below 2^-115) it is applied in two steps.
+    const uint32_t fld = 266u - eb, f1 = min(fld, 254u);
+    const float s1 = __uint_as_float(f1 << 23), s2 = __uint_as_float((127u + fld - f1) << 23);
+    uint32_t t[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-        const uint32_t h = (e & 1) ? x[e >> 1] >> 16 : x[e >> 1] & 0xFFFFu;
-        const uint32_t ef = (h >> 7) & 255u;
-        const uint32_t m13 = ((ef ? 128u : 0u) | (h & 127u)) << 5;  // at the block's largest exponent
-        const uint32_t down = min(eb - max(ef, 1u), 31u);           // binades below it
-        t[e] = ((m13 + ((1u << down) >> 1)) >> down) + 0x4924u;     // rounded to nearest
-        lut[e] = (h & 0x8000u) ? 0xDCA82456u : 0x5420ACDEu;
+        float f = __uint_as_float((e & 1) ? x[e >> 1] & 0x7FFF0000u : (x[e >> 1] << 16) & 0x7FFF0000u);
+        if (fld > 254u) f *= s2;
+        t[e] = (nonfinite ? 0u : __float2uint_rz(fmaf(f, s1, 0.5f))) + 0x4924u;
     }
+    // two elements per register, then per plane: the octal digits of four elements as the four
+    // selector nibbles of one byte permute, which looks the digits' E2M1 codes up in an
+    // eight-byte table (codes of 4 3 2 1 0 1 2 3, the sign bit set for the negative digits 0..3);
+    // an element's own sign is exclusive-ored on top
+    const uint32_t p01 = t[0] | (t[1] << 16), p23 = t[2] | (t[3] << 16);
+    const uint32_t p45 = t[4] | (t[5] << 16), p67 = t[6] | (t[7] << 16);
+    const uint32_t sg0 = __byte_perm((x[0] >> 12) & 0x00080008u, (x[1] >> 12) & 0x00080008u, 0x6420);
+    const uint32_t sg1 = __byte_perm((x[2] >> 12) & 0x00080008u, (x[3] >> 12) & 0x00080008u, 0x6420);
+    constexpr uint32_t kLutLo = 0x0A0C0D0Eu, kLutHi = 0x05040200u;
 #pragma unroll
     for (int j = 0; j < kPlanes; ++j) {
         const int sbyte = (int)eb - 3 * j;  // E8M0 byte of 2^(E - 3 j)
         uint32_t w = 0u;
         if (sbyte >= 0 && !nonfinite) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const uint32_t sh4 = (j < 4 ? t[e] >> (3 * (4 - j) - 2) : t[e] << 2) & 28u;  // 4 x octal digit j
-                w |= ((lut[e] >> sh4) & 15u) << (4 * e);
-            }
+            const int sh = 3 * (4 - j);
+            const uint32_t d0 = __byte_perm((p01 >> sh) & 0x00070007u, (p23 >> sh) & 0x00070007u, 0x6420);
+            const uint32_t d1 = __byte_perm((p45 >> sh) & 0x00070007u, (p67 >> sh) & 0x00070007u, 0x6420);
+            const uint32_t n0 = d0 | (d0 >> 4), n1 = d1 | (d1 >> 4);  // bytes 0 and 2: two digits each
+            const uint32_t c0 = __byte_perm(kLutLo, kLutHi, __byte_perm(n0, 0u, 0x4420)) ^ sg0;
+            const uint32_t c1 = __byte_perm(kLutLo, kLutHi, __byte_perm(n1, 0u, 0x4420)) ^ sg1;
+            const uint32_t y0 = c0 | (c0 >> 4), y1 = c1 | (c1 >> 4);  // bytes 0 and 2: two codes each
+            w = __byte_perm(y0, y1, 0x6420);
         }
         const int row = kPlanes * m + j;
         *reinterpret_cast<uint32_t*>(codes + swz_chunk((uint32_t)row, (uint32_t)kb) + 4 * qd) = w;
