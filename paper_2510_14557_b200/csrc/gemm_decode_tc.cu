@@ -24,14 +24,15 @@
 //     A small kernel does this once per call (decode_act_kernel) and leaves the operand images
 //     of all stages in the workspace; the GEMM is launched as its programmatic dependent, so
 //     its CTAs stream weights meanwhile, and fetches the images stage by stage next to the
-//     weights.  (Converting inside the GEMM, every CTA for itself, was built and measured: the
-//     conversion is ~500 instructions per eight elements and costs a CTA 4 us per activation
-//     row, more than the second launch.)
-//   * One or two activation rows (kSelf): the dependent chain "kernel before -> conversion
-//     kernel -> this kernel's copies of the images" costs ~4 us of a ~10 us call, more than
-//     the conversion itself.  There every CTA converts the rows for itself, straight into
-//     shared memory where the images of all stages stay (40 KB at K = 4096), while its weights
-//     are already streaming: one launch per call, and no image travels through global memory.
+//     weights.  (Converting inside the GEMM, every CTA for itself, costs a CTA ~1.6 us per
+//     activation row -- ~400 instructions per eight elements, sixteen warps' worth per row --
+//     which from the second row on is more than the second launch costs in a chain.)
+//   * A single activation row (kSelf): the dependent chain "kernel before -> conversion
+//     kernel -> this kernel's copies of the images" costs more than the conversion itself.
+//     There every CTA converts the row for itself, straight into shared memory where the
+//     images of all stages stay (40 KB at K = 4096), while its weights are already
+//     streaming: one launch per call, and no image travels through global memory.  (Two rows
+//     that way: 9.6 us against 8.75 us with the conversion kernel, calls chained in a graph.)
 //     MX+ there takes Eq. 4's BM_L term off the tensor cores: sum over blocks of
 //     (+-BM_L 2^shared_exp) a[k_BM] is eight products per weight row and stage, so warps 10-21
 //     add it on the CUDA cores in fp32 from the record bytes, the scale bytes and a raw bf16
@@ -43,9 +44,9 @@
 //   * warp 0 issues the weight copies (the first ring-full before the CTA's set-up barrier),
 //     warp 1 the activation copies, warps 2-5 the MMAs (each every fourth stage, with an
 //     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 handle BM_L
-//     (three groups of four, a stage each in turn): for M >= 3 they build the BM_L operand
+//     (three groups of four, a stage each in turn): for M >= 2 they build the BM_L operand
 //     tiles (one group needs ~0.8 us per stage, the stream delivers one every 0.26 us), for
-//     M <= 2 they sum the term themselves.
+//     M = 1 they sum the term themselves.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -119,7 +120,7 @@ struct DecodeLayout {
     size_t img_codes, img_sf, raw, corr;  // kSelf only (raw, corr: MX+)
     int stages;
 };
-constexpr int kSelfMaxM = 2;
+constexpr int kSelfMaxM = 1;
 __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages,
                                                       int self_nst = 0)
 {
@@ -277,17 +278,18 @@ decode_prepack_kernel(const uint8_t* __restrict__ nibbles, const uint8_t* __rest
 // Eight activations (quarter `qd` of block `kb` of a stage, activation row m; the four lanes of
 // a quad hold the four quarters of one block) -> their five digit planes: one word of codes per
 // plane into the stage's tile `codes`, and the planes' scale bytes into its atoms `sf`.
-__device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, int qd, uint8_t* codes, uint8_t* sf,
+// (`codes`, `sf`: shared-memory addresses; the stores name the shared window, which saves the
+// 64-bit address arithmetic of generic stores.)
+__device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, int qd, uint32_t codes, uint32_t sf,
                                                 int sfb)
 {
     const uint32_t x[4] = {v.x, v.y, v.z, v.w};
-    // largest exponent field of the block (zero and subnormals count as field 1)
-    uint32_t eb = 1;
+    // largest exponent field of the block (zero and subnormals count as field 1): both halves of
+    // a register at once
+    uint32_t e2 = 0x00010001u;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        eb = max(eb, (x[q] >> 7) & 255u);
-        eb = max(eb, (x[q] >> 23) & 255u);
-    }
+    for (int q = 0; q < 4; ++q) e2 = __vmaxu2(e2, (x[q] >> 7) & 0x00FF00FFu);
+    uint32_t eb = max(e2 & 0xFFFFu, e2 >> 16);
     eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 1));
     eb = max(eb, __shfl_xor_sync(0xFFFFFFFFu, eb, 2));
     const bool nonfinite = eb == 255u;
@@ -299,41 +301,41 @@ __device__ __forceinline__ void convert_quarter(const uint4 v, int m, int kb, in
     // below 2^-115) it is applied in two steps.
     const uint32_t fld = 266u - eb, f1 = min(fld, 254u);
     const float s1 = __uint_as_float(f1 << 23), s2 = __uint_as_float((127u + fld - f1) << 23);
-    uint32_t t[8];
+    uint32_t p[4];  // two elements per register
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        float f = __uint_as_float((e & 1) ? x[e >> 1] & 0x7FFF0000u : (x[e >> 1] << 16) & 0x7FFF0000u);
-        if (fld > 254u) f *= s2;
-        t[e] = (nonfinite ? 0u : __float2uint_rz(fmaf(f, s1, 0.5f))) + 0x4924u;
+    for (int q = 0; q < 4; ++q) {
+        const float lo = __uint_as_float((x[q] << 16) & 0x7FFF0000u) * s2;
+        const float hi = __uint_as_float(x[q] & 0x7FFF0000u) * s2;
+        p[q] = (__float2uint_rz(fmaf(lo, s1, 0.5f)) | (__float2uint_rz(fmaf(hi, s1, 0.5f)) << 16)) + 0x49244924u;
     }
-    // two elements per register, then per plane: the octal digits of four elements as the four
-    // selector nibbles of one byte permute, which looks the digits' E2M1 codes up in an
-    // eight-byte table (codes of 4 3 2 1 0 1 2 3, the sign bit set for the negative digits 0..3);
-    // an element's own sign is exclusive-ored on top
-    const uint32_t p01 = t[0] | (t[1] << 16), p23 = t[2] | (t[3] << 16);
-    const uint32_t p45 = t[4] | (t[5] << 16), p67 = t[6] | (t[7] << 16);
+    // per plane: the octal digits of four elements as the four selector nibbles of one byte
+    // permute, which looks the digits' E2M1 codes up in an eight-byte table (codes of 4 3 2 1 0 1
+    // 2 3, the sign bit set for the negative digits 0..3); an element's own sign is
+    // exclusive-ored on top
     const uint32_t sg0 = __byte_perm((x[0] >> 12) & 0x00080008u, (x[1] >> 12) & 0x00080008u, 0x6420);
     const uint32_t sg1 = __byte_perm((x[2] >> 12) & 0x00080008u, (x[3] >> 12) & 0x00080008u, 0x6420);
     constexpr uint32_t kLutLo = 0x0A0C0D0Eu, kLutHi = 0x05040200u;
+    const uint32_t row0 = (uint32_t)(kPlanes * m);
+    const uint32_t sf0 = sf + (uint32_t)((kb >> 2) * sfb + (kb & 3));
 #pragma unroll
     for (int j = 0; j < kPlanes; ++j) {
         const int sbyte = (int)eb - 3 * j;  // E8M0 byte of 2^(E - 3 j)
-        uint32_t w = 0u;
-        if (sbyte >= 0 && !nonfinite) {
-            const int sh = 3 * (4 - j);
-            const uint32_t d0 = __byte_perm((p01 >> sh) & 0x00070007u, (p23 >> sh) & 0x00070007u, 0x6420);
-            const uint32_t d1 = __byte_perm((p45 >> sh) & 0x00070007u, (p67 >> sh) & 0x00070007u, 0x6420);
-            const uint32_t n0 = d0 | (d0 >> 4), n1 = d1 | (d1 >> 4);  // bytes 0 and 2: two digits each
-            const uint32_t c0 = __byte_perm(kLutLo, kLutHi, __byte_perm(n0, 0u, 0x4420)) ^ sg0;
-            const uint32_t c1 = __byte_perm(kLutLo, kLutHi, __byte_perm(n1, 0u, 0x4420)) ^ sg1;
-            const uint32_t y0 = c0 | (c0 >> 4), y1 = c1 | (c1 >> 4);  // bytes 0 and 2: two codes each
-            w = __byte_perm(y0, y1, 0x6420);
-        }
-        const int row = kPlanes * m + j;
-        *reinterpret_cast<uint32_t*>(codes + swz_chunk((uint32_t)row, (uint32_t)kb) + 4 * qd) = w;
+        const int sh = 3 * (4 - j);
+        const uint32_t d0 = __byte_perm((p[0] >> sh) & 0x00070007u, (p[1] >> sh) & 0x00070007u, 0x6420);
+        const uint32_t d1 = __byte_perm((p[2] >> sh) & 0x00070007u, (p[3] >> sh) & 0x00070007u, 0x6420);
+        const uint32_t n0 = d0 | (d0 >> 4), n1 = d1 | (d1 >> 4);  // bytes 0 and 2: two digits each
+        const uint32_t c0 = __byte_perm(kLutLo, kLutHi, __byte_perm(n0, 0u, 0x4420)) ^ sg0;
+        const uint32_t c1 = __byte_perm(kLutLo, kLutHi, __byte_perm(n1, 0u, 0x4420)) ^ sg1;
+        const uint32_t y0 = c0 | (c0 >> 4), y1 = c1 | (c1 >> 4);  // bytes 0 and 2: two codes each
+        // a plane whose scale would lie below the format's range, or a block with an Inf or NaN: zeros
+        const uint32_t w = (sbyte >= 0 && !nonfinite) ? __byte_perm(y0, y1, 0x6420) : 0u;
+        const uint32_t row = row0 + (uint32_t)j;
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(codes + swz_chunk(row, (uint32_t)kb) + 4u * (uint32_t)qd), "r"(w)
+                     : "memory");
         if (qd == 0)
-            sf[(kb >> 2) * sfb + (row & 31) * 16 + (row >> 5) * 4 + (kb & 3)] =
-                (uint8_t)(nonfinite ? 255 : max(sbyte, 0));
+            asm volatile("st.shared.u8 [%0], %1;" ::"r"(sf0 + (row & 31u) * 16u + (row >> 5) * 4u),
+                         "r"(nonfinite ? 255u : (uint32_t)max(sbyte, 0))
+                         : "memory");
     }
 }
 
@@ -366,7 +368,7 @@ decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int n
     const int m = blk >> 3, kb = blk & 7;
     if (m < M) {
         const uint4 v = __ldg(reinterpret_cast<const uint4*>(A + (int64_t)m * lda + (int64_t)st * kStageK + kb * 32) + qd);
-        convert_quarter(v, m, kb, qd, img, img + nact * 128, sfb);
+        convert_quarter(v, m, kb, qd, ptx::smem_u32(img), ptx::smem_u32(img + nact * 128), sfb);
     }
     __syncthreads();
     uint4* dst = reinterpret_cast<uint4*>(aimg + (size_t)st * bytes);
@@ -380,7 +382,7 @@ template <int kNact, bool kPlus, bool kSelf, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_decode_tc_kernel(const DecodeParams prm)
 {
-    static_assert(!kSelf || kNact == 16, "self-converted activations: at most two rows");
+    static_assert(!kSelf || kNact == 16, "self-converted activations: one operand tile of 16 rows");
     constexpr int kSfb = sfb_bytes(kNact);
     constexpr int kMt = kSelf ? kSelfMaxM : kNact / kPlanes;  // activation rows the operand can hold
     extern __shared__ uint8_t smem_raw[];
@@ -460,14 +462,26 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             prm.status->code = 0u;
             prm.status->where = 0u;
         }
-        for (int i = threadIdx.x; i < prm.M * nst * 32; i += kThreads) {
-            const int m = i / (nst * 32), rem = i - m * nst * 32;
+        // (a thread's next eight elements are on their way from L2 while it converts these)
+        const int per_row = nst * 32, tasks = prm.M * per_row;
+        const uint32_t img_codes0 = ptx::smem_u32(smem + L.img_codes), img_sf0 = ptx::smem_u32(smem + L.img_sf);
+        auto fetch = [&](int i) {
+            const int m = i / per_row, rem = i - m * per_row;
+            return __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + (int64_t)rem * 8));
+        };
+        int i = (int)threadIdx.x;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i < tasks) v = fetch(i);
+        while (i < tasks) {
+            const int nxt = i + kThreads;
+            uint4 vn = make_uint4(0u, 0u, 0u, 0u);
+            if (nxt < tasks) vn = fetch(nxt);
+            const int m = i / per_row, rem = i - m * per_row;
             const int st = rem >> 5, kb = (rem >> 2) & 7, qd = rem & 3;
-            const int64_t k0 = (int64_t)st * kStageK + kb * 32 + qd * 8;
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + k0));
-            if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)k0) * 2) = v;
-            convert_quarter(v, m, kb, qd, smem + L.img_codes + (size_t)st * 2048, smem + L.img_sf + (size_t)st * 512,
-                            kSfb);
+            if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)rem * 8) * 2) = v;
+            convert_quarter(v, m, kb, qd, img_codes0 + (uint32_t)st * 2048u, img_sf0 + (uint32_t)st * 512u, kSfb);
+            v = vn;
+            i = nxt;
         }
         ptx::fence_proxy_async_smem();  // the MMAs read the images through the async proxy
         __syncthreads();
@@ -901,7 +915,7 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     const size_t need = decode_workspace_bytes(M, K);
     if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
     const int nact = act_rows((int)M);
-    // one or two rows: every CTA converts them for itself, if their images fit beside a ring
+    // a single row: every CTA converts it for itself, if its images fit beside a ring
     const int self_stages = M <= kSelfMaxM ? pick_stages(p, nact, plus, p.nst) : 0;
     const bool self = self_stages != 0;
     const int stages = self ? self_stages : pick_stages(p, nact, plus);

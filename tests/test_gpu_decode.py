@@ -33,11 +33,12 @@ def raw_weights(N, K, mode, seed, lo=118, hi=136):
 @pytest.mark.parametrize("M,N,K", [(1, 64, 256), (1, 11008, 4096), (2, 300, 512), (3, 2384, 4096), (4, 77, 1024),
                                    (5, 1000, 768), (7, 19000, 512), (8, 11008, 4096), (9, 160, 4352),
                                    (12, 40000, 256), (13, 333, 1280), (16, 11008, 4096), (16, 8, 256), (1, 1, 256),
-                                   (2, 40000, 256), (1, 19000, 8192), (2, 700, 16384), (2, 11008, 4096)])
+                                   (2, 40000, 256), (1, 40000, 256), (1, 19000, 8192), (1, 700, 16384), (2, 700, 16384),
+                                   (2, 11008, 4096)])
 def test_decode_prepacked_parity(M, N, K, wmode):
     # ragged N (last CTA short, rows not a multiple of 8), more than 128 rows per CTA (several
     # tiles), every activation-operand width (16 .. 80 rows), K from one stage to seventeen.
-    # One and two rows take the form in which every CTA converts the activations for itself and
+    # A single row takes the form in which every CTA converts the activations for itself and
     # adds the BM's lower part on the CUDA cores: also with several tiles per CTA, with images
     # that leave room for few ring slots (K = 8192) and with images that do not fit at all
     # (K = 16384: back to the conversion kernel)
