@@ -43,10 +43,11 @@
 //     MXFP4; the epilogue adds the three groups' partial sums in a fixed order.
 //   * warp 0 issues the weight copies (the first ring-full before the CTA's set-up barrier),
 //     warp 1 the activation copies, warps 2-5 the MMAs (each every fourth stage, with an
-//     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 handle BM_L
-//     (three groups of four, a stage each in turn): for M >= 2 they build the BM_L operand
-//     tiles (one group needs ~0.8 us per stage, the stream delivers one every 0.26 us), for
-//     M = 1 they sum the term themselves.
+//     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 handle BM_L:
+//     for M >= 2 they build the BM_L operand tiles (four groups of three, group g owning slot g
+//     of the tile ring: one group needs ~1 us per stage, the stream delivers one every
+//     0.26 us), for M = 1 they sum the term themselves (three groups of four, a stage each in
+//     turn).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -60,7 +61,8 @@ namespace {
 
 constexpr int kIssueWarp0 = 2, kIssuers = 4;
 constexpr int kRowWarp0 = 6;
-constexpr int kResWarp0 = 10, kResWarps = 4, kResGroups = 3;  // three groups of four warps take turns
+constexpr int kResWarp0 = 10, kResWarps = 4, kResGroups = 3;  // BM_L sums: three groups of four warps take turns
+constexpr int kTileWarps = 3, kTileGroups = 4;  // BM_L tiles: the same twelve warps as four groups of three
 constexpr int kWarps = kResWarp0 + kResWarps * kResGroups;
 constexpr int kThreads = 32 * kWarps;
 constexpr int kStageK = 256;   // elements of K per stage: 128 bytes of codes per row
@@ -110,26 +112,32 @@ struct PrepackHeader {
 };
 
 // Shared memory of the GEMM kernel (bytes from the 1024-byte aligned base).
-// A slot holds a stage's weight image, its activation image (codes at act_off, scale atoms
-// behind) and, for MX+, the BM_L tile built from the image's records (at res_off).
-// kSelf form (self_nst > 0: number of stages whose activation images stay resident): a slot
-// holds the weight image only; behind the ring come the images' code tiles (2 KB a stage), their
-// scale atoms (512 bytes a stage) and, for MX+, the raw activations and the BM_L term's sums.
+// Three rings.  The weight ring (`stages` slots of `slot` bytes) is as deep as the rest allows:
+// the weights do not depend on the kernel before, so whatever fits streams in while the
+// activations are still being waited for.  The activation images (from L2, available late,
+// needed only just before their MMAs) and, for MX+, the BM_L tiles built from the weight
+// images' records have rings of their own (`astages` slots of `aslot` bytes, kSideSlots slots of
+// `rslot` bytes).
+// kSelf form (self_nst > 0: number of stages whose activation images stay resident): no side
+// rings; behind the weight ring come the images' code tiles (2 KB a stage), their scale atoms
+// (512 bytes a stage) and, for MX+, the raw activations and the BM_L term's sums.
 struct DecodeLayout {
-    size_t act_off, res_off, slot, bars, total;
+    size_t slot, act0, aslot, res0, rslot, bars, total;
     size_t img_codes, img_sf, raw, corr;  // kSelf only (raw, corr: MX+)
-    int stages;
+    int stages, astages;
 };
 constexpr int kSelfMaxM = 1;
+constexpr int kSideSlots = 4;
 __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages,
-                                                      int self_nst = 0)
+                                                      int self_nst = 0, int astages = kSideSlots)
 {
     DecodeLayout l;
     l.stages = stages;
+    l.astages = astages;
     l.img_codes = l.img_sf = l.raw = l.corr = 0;
+    l.act0 = l.aslot = l.res0 = l.rslot = 0;
+    l.slot = up(wimg, 1024);
     if (self_nst > 0) {
-        l.act_off = l.res_off = 0;
-        l.slot = up(wimg, 1024);
         const size_t last = (size_t)(stages - 1) * l.slot + 128 * 128;  // (see below)
         size_t o = up(last > (size_t)stages * l.slot ? last : (size_t)stages * l.slot, 1024);
         l.img_codes = o;
@@ -146,12 +154,13 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
         l.total = l.bars + 1024 + 1024;
         return l;
     }
-    l.act_off = up(wimg, 1024);
-    l.res_off = up(l.act_off + (size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact), 1024);
-    l.slot = l.res_off + (plus ? up((size_t)rows * 128, 1024) : 0);
+    l.act0 = (size_t)stages * l.slot;
+    l.aslot = up((size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact), 1024);
+    l.res0 = l.act0 + (size_t)astages * l.aslot;
+    l.rslot = plus ? up((size_t)rows * 128, 1024) : 0;
     // an MMA reads 128 rows of 128 bytes from the start of a tile that holds fewer: what follows
     // the last tile must exist (any bytes are finite E2M1 codes; the rows are never read back)
-    size_t off = up((size_t)stages * l.slot + 16384, 16);
+    size_t off = up(l.res0 + kSideSlots * l.rslot + 16384, 16);
     l.bars = off;
     l.total = off + 1024 + 1024;  // barriers; slack for aligning the base
     return l;
@@ -183,7 +192,7 @@ struct DecodeParams {
     void* D;
     int64_t ldd;
     StatusBlock* status;   // may be nullptr
-    int rows, tiles, nst, stages;
+    int rows, tiles, nst, stages, astages;
     uint32_t wimg_bytes;
 };
 
@@ -389,11 +398,15 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int S = prm.stages;
     const int nst = prm.nst;
-    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S, kSelf ? nst : 0);
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // the slot's copies landed
-    uint64_t* empty = full + kMaxStages;       // the slot's MMAs are done
-    uint64_t* res_full = empty + kMaxStages;   // the slot's BM_L tile is written
-    uint64_t* acc_full = res_full + kMaxStages;
+    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S, kSelf ? nst : 0, prm.astages);
+    const int SA = prm.astages;  // slots of the activation ring
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // the slot's weight image landed
+    uint64_t* empty = full + kMaxStages;       // the slot's MMAs are done (and its records read)
+    uint64_t* afull = empty + kMaxStages;      // the slot's activation image landed
+    uint64_t* aempty = afull + kMaxStages;     // its MMAs are done
+    uint64_t* res_full = aempty + kMaxStages;  // [kSideSlots] the slot's BM_L tile is written
+    uint64_t* res_empty = res_full + kSideSlots;  //           its MMAs are done
+    uint64_t* acc_full = res_empty + kSideSlots;
     uint64_t* acc_empty = acc_full + 1;
     uint64_t* corr_full = acc_empty + 1;       // [2] kSelf MX+: a tile's BM_L sums are complete
     uint64_t* corr_empty = corr_full + 2;      // [2] ... and have been taken
@@ -402,6 +415,8 @@ gemm_decode_tc_kernel(const DecodeParams prm)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     auto slot = [&](int s) { return smem + (size_t)s * L.slot; };
+    auto act_slot = [&](int sa) { return smem + L.act0 + (size_t)sa * L.aslot; };
+    auto res_slot = [&](int sr) { return smem + L.res0 + (size_t)sr * L.rslot; };
     const int64_t row0 = (int64_t)blockIdx.x * prm.tiles * prm.rows;  // first weight row of this CTA
     // tiles of this CTA that hold rows, and its stages in all
     const int ntl = (int)min((int64_t)prm.tiles, (prm.N - row0 + prm.rows - 1) / prm.rows);
@@ -411,9 +426,14 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     if (threadIdx.x == 0) {
         MXP_TL(0);  // kernel entry
         for (int s = 0; s < kMaxStages; ++s) {
-            ptx::mbar_init(&full[s], kSelf ? 1 : 2);
-            ptx::mbar_init(&empty[s], (kSelf && kPlus) ? 1 + kResWarps : 1);  // + the warps that read its records
-            ptx::mbar_init(&res_full[s], kResWarps);
+            ptx::mbar_init(&afull[s], 1);
+            ptx::mbar_init(&aempty[s], 1);
+            ptx::mbar_init(&full[s], 1);
+            ptx::mbar_init(&empty[s], !kPlus ? 1 : kSelf ? 1 + kResWarps : 1 + kTileWarps);  // + the warps that read its records
+        }
+        for (int s = 0; s < kSideSlots; ++s) {
+            ptx::mbar_init(&res_full[s], kTileWarps);
+            ptx::mbar_init(&res_empty[s], 1);
         }
         ptx::mbar_init(acc_full, kIssuers);
         ptx::mbar_init(acc_empty, 4);
@@ -508,13 +528,13 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             MXP_TL(2);  // activations available
             constexpr uint32_t kBytes = kNact * 128 + 2 * kSfb;
             for (uint32_t c = 0; c < total; ++c) {
-                const int s = c % S;
-                if (c >= (uint32_t)S && !ptx::mbar_wait(&empty[s], (c / S - 1) & 1, abort, kWaitLimit)) {
-                    report(prm.status, abort, 0x7200 + s);
+                const int sa = c % SA;
+                if (c >= (uint32_t)SA && !ptx::mbar_wait(&aempty[sa], (c / SA - 1) & 1, abort, kWaitLimit)) {
+                    report(prm.status, abort, 0x7200 + sa);
                     break;
                 }
-                ptx::mbar_arrive_expect_tx(&full[s], kBytes);
-                bulk_g2s(slot(s) + L.act_off, prm.aimg + (size_t)(c % (uint32_t)nst) * kBytes, kBytes, &full[s]);
+                ptx::mbar_arrive_expect_tx(&afull[sa], kBytes);
+                bulk_g2s(act_slot(sa), prm.aimg + (size_t)(c % (uint32_t)nst) * kBytes, kBytes, &afull[sa]);
             }
         }
     } else if (warp >= kIssueWarp0 && warp < kIssueWarp0 + kIssuers) {
@@ -537,7 +557,11 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 const uint32_t cc = c + (uint32_t)st;
                 const int s = cc % S;
                 const uint32_t ph = (cc / S) & 1;
-                if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit)) {
+                const int sa = kSelf ? 0 : cc % SA;                 // slot of the activation ring
+                const int sd = cc % kSideSlots;                     // slot of the tile ring
+                const uint32_t phd = (cc / kSideSlots) & 1;
+                if (!ptx::mbar_wait(&full[s], ph, abort, kWaitLimit) ||
+                    (!kSelf && !ptx::mbar_wait(&afull[sa], (cc / SA) & 1, abort, kWaitLimit))) {
                     if (lane == 0) report(prm.status, abort, 0x7400 + s);
                     ok = false;
                     break;
@@ -551,10 +575,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 const uint8_t* sl = slot(s);
                 const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(sl));
                 const uint64_t db = ptx::smem_desc_sw128(
-                    ptx::smem_u32(kSelf ? smem + L.img_codes + (size_t)st * 2048 : sl + L.act_off));
+                    ptx::smem_u32(kSelf ? smem + L.img_codes + (size_t)st * 2048 : act_slot(sa)));
                 const uint32_t sfa = ptx::smem_u32(sl + (size_t)prm.rows * 128);
                 const uint32_t sfb =
-                    ptx::smem_u32(kSelf ? smem + L.img_sf + (size_t)st * 512 : sl + L.act_off + kNact * 128);
+                    ptx::smem_u32(kSelf ? smem + L.img_sf + (size_t)st * 512 : act_slot(sa) + kNact * 128);
                 const uint32_t t_sf = tmem_base + kTmemSf + 16u * (uint32_t)iss;
                 if (ptx::elect_one()) {
 #pragma unroll
@@ -574,13 +598,13 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 __syncwarp();
                 if (kPlus && !kSelf) {
                     // the BM_L tile of the stage, same scales, same accumulator (Eq. 4)
-                    if (!ptx::mbar_wait(&res_full[s], ph, abort, kWaitLimit)) {
-                        if (lane == 0) report(prm.status, abort, 0x7500 + s);
+                    if (!ptx::mbar_wait(&res_full[sd], phd, abort, kWaitLimit)) {
+                        if (lane == 0) report(prm.status, abort, 0x7500 + sd);
                         ok = false;
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint64_t dr = ptx::smem_desc_sw128(ptx::smem_u32(sl + L.res_off));
+                    const uint64_t dr = ptx::smem_desc_sw128(ptx::smem_u32(res_slot(sd)));
                     if (ptx::elect_one()) {
 #pragma unroll
                         for (int g = 0; g < 2; ++g) {
@@ -596,7 +620,11 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     }
                     __syncwarp();
                 }
-                if (ptx::elect_one()) ptx::tc_commit(&empty[s]);
+                if (ptx::elect_one()) {  // the stage's slots are free once these MMAs have read them
+                    ptx::tc_commit(&empty[s]);
+                    if (!kSelf) ptx::tc_commit(&aempty[sa]);
+                    if (kPlus && !kSelf) ptx::tc_commit(&res_empty[sd]);
+                }
                 __syncwarp();
             }
             c += (uint32_t)nst;
@@ -745,23 +773,28 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         }
     } else if (kPlus) {
         // ---------------------------------------------------------------- BM_L tiles
-        // Group g of four warps takes the stages whose running number is g (mod 3).  The tile
-        // lives in the stage's slot, so once the slot's copies have landed nothing else can be
-        // using it.  The four warps clear it together (consecutive threads, consecutive 16
-        // bytes), then thread = weight row drops in, per block, the code its record byte names.
-        const int grp = (warp - kResWarp0) / kResWarps;
-        const int r = (int)threadIdx.x - 32 * (kResWarp0 + grp * kResWarps);
-        for (uint32_t c = (uint32_t)grp; c < total; c += kResGroups) {
-            const int s = c % S;
-            if (!ptx::mbar_wait(&full[s], (c / S) & 1, abort, kWaitLimit)) {
+        // Group g of three warps owns slot g of the tile ring and takes the stages whose running
+        // number is g (mod 4), like issuer g: every barrier of the slot is waited on by one party
+        // only, stage after stage, so a parity never stands for the wrong phase.  The three warps
+        // clear the tile together (consecutive threads, consecutive 16 bytes), then a thread drops
+        // in, for its weight rows and per block, the code the record byte names.
+        static_assert(kTileGroups == kSideSlots && kTileGroups == kIssuers, "one owner per slot");
+        const int grp = (warp - kResWarp0) / kTileWarps;
+        const int r0 = (int)threadIdx.x - 32 * (kResWarp0 + grp * kTileWarps);
+        for (uint32_t c = (uint32_t)grp; c < total; c += kTileGroups) {
+            const int s = c % S, sr = grp;
+            // the stage's records have landed, and the MMAs that read the tile's last contents are done
+            if (!ptx::mbar_wait(&full[s], (c / S) & 1, abort, kWaitLimit) ||
+                (c >= (uint32_t)kSideSlots &&
+                 !ptx::mbar_wait(&res_empty[sr], (c / kSideSlots - 1) & 1, abort, kWaitLimit))) {
                 if (lane == 0) report(prm.status, abort, 0x7700 + s);
                 break;
             }
-            uint8_t* tile = slot(s) + L.res_off;
-            for (int k = r; k < prm.rows * 8; k += 32 * kResWarps)
+            uint8_t* tile = res_slot(sr);
+            for (int k = r0; k < prm.rows * 8; k += 32 * kTileWarps)
                 reinterpret_cast<uint4*>(tile)[k] = make_uint4(0u, 0u, 0u, 0u);
-            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(32 * kResWarps) : "memory");
-            if (r < prm.rows) {
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(32 * kTileWarps) : "memory");
+            for (int r = r0; r < prm.rows; r += 32 * kTileWarps) {
                 uint8_t* mine = tile + (size_t)r * 128;
                 const uint2 rec = *reinterpret_cast<const uint2*>(slot(s) + (size_t)prm.rows * 128 + 2 * kAtom + (size_t)r * 8);
 #pragma unroll
@@ -776,7 +809,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             }
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&res_full[s]);
+            if (lane == 0) {
+                ptx::mbar_arrive(&res_full[sr]);
+                ptx::mbar_arrive(&empty[s]);  // the slot's records have been read
+            }
         }
     }
 
@@ -791,6 +827,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             while (!ptx::mbar_try_wait(&full[s], 0) && !ptx::mbar_try_wait(&full[s], 1) &&
                    clock64() - t0 < kWaitLimit) {
             }
+        for (int s = 0; s < SA && !kSelf; ++s)
+            while (!ptx::mbar_try_wait(&afull[s], 0) && !ptx::mbar_try_wait(&afull[s], 1) &&
+                   clock64() - t0 < kWaitLimit) {
+            }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -802,10 +842,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
 
 // Ring slots that fit: a multiple of four (see the issuers), at most sixteen.  self_nst > 0: the
 // form with resident activation images.
-int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0)
+int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0, int astages = kSideSlots)
 {
     for (int s = kMaxStages; s >= 4; s -= 4)
-        if (decode_layout(p.rows, p.wimg, nact, plus, s, self_nst).total <= kSmemMax) return s;
+        if (decode_layout(p.rows, p.wimg, nact, plus, s, self_nst, astages).total <= kSmemMax) return s;
     return 0;
 }
 
@@ -918,9 +958,13 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     // a single row: every CTA converts it for itself, if its images fit beside a ring
     const int self_stages = M <= kSelfMaxM ? pick_stages(p, nact, plus, p.nst) : 0;
     const bool self = self_stages != 0;
-    const int stages = self ? self_stages : pick_stages(p, nact, plus);
+    // The activation ring: eight slots (the images come from L2 with ~1 us of latency: with four,
+    // every fourth stage waits for its image) unless that leaves the weight ring fewer than eight.
+    int astages = 2 * kSideSlots;
+    if (self || pick_stages(p, nact, plus, 0, astages) < 8) astages = kSideSlots;
+    const int stages = self ? self_stages : pick_stages(p, nact, plus, 0, astages);
     if (stages == 0) return MXP_ERR_UNSUPPORTED;
-    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages, self ? p.nst : 0);
+    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages, self ? p.nst : 0, astages);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     DecodeParams prm = {};
     prm.M = (int)M;
@@ -937,6 +981,7 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     prm.tiles = p.tiles;
     prm.nst = p.nst;
     prm.stages = stages;
+    prm.astages = astages;
     prm.wimg_bytes = p.wimg;
     const bool f32 = d_dt == MXP_F32;
     if (self) {  // one launch; a programmatic dependent only on the caller's promise
