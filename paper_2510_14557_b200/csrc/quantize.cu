@@ -600,9 +600,11 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
 {
     extern __shared__ uint4 dyn_smem[];
     const int cols = cols_blocks * 32;
-    unsigned short* row_buf[2] = {reinterpret_cast<unsigned short*>(dyn_smem),
-                                  reinterpret_cast<unsigned short*>(dyn_smem) + cols};
-    unsigned short* ord_s = row_buf[1] + cols;
+    // (no array of row pointers: a pointer picked from an array at run time makes the gather's
+    // loads generic ones, with 64-bit address arithmetic for each)
+    const uint32_t row_sa[2] = {(uint32_t)__cvta_generic_to_shared(dyn_smem),
+                                (uint32_t)__cvta_generic_to_shared(dyn_smem) + 2u * (uint32_t)cols};
+    unsigned short* ord_s = reinterpret_cast<unsigned short*>(dyn_smem) + 2 * cols;
     constexpr int kPerVec = 8;  // ordering entries per 16-byte vector
     constexpr int kVecs = 4;    // vectors per block
     // ordering entry e of block b sits in vector (e / kPerVec) * cols_blocks + b
@@ -619,7 +621,7 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
     auto fetch = [&](int64_t row, int buf) {
         if (row < rows) {
             const uint4* src_row = reinterpret_cast<const uint4*>(src + row * ld_src);
-            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(row_buf[buf]);
+            const uint32_t dst = buf ? row_sa[1] : row_sa[0];
             for (int i = threadIdx.x; i < vecs; i += kThreads)
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i),
                              "l"(src_row + i)
@@ -633,7 +635,7 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
         fetch(row + gridDim.x, (it + 1) & 1);
         asm volatile("cp.async.wait_group 1;" ::: "memory");
         __syncthreads();  // this row has landed for every thread (first pass: the ordering too)
-        const unsigned short* row_s = row_buf[it & 1];
+        const unsigned short* row_s = reinterpret_cast<const unsigned short*>(dyn_smem) + ((it & 1) ? cols : 0);
         for (int b = threadIdx.x; b < cols_blocks; b += kThreads) {
             uint32_t x[16];
 #pragma unroll
@@ -642,8 +644,7 @@ quantize_bf16_reordered_kernel(const __nv_bfloat16* __restrict__ src, int64_t ld
                 const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
-                    x[4 * k + i] = (uint32_t)row_s[ow[i] & 0xFFFFu] |
-                                   ((uint32_t)row_s[ow[i] >> 16] << 16);
+                    x[4 * k + i] = __byte_perm((uint32_t)row_s[ow[i] & 0xFFFFu], (uint32_t)row_s[ow[i] >> 16], 0x5410);
             }
             quantize_block_bf16<kMode, 0>(x, row * cols_blocks + b, nibbles, scales, bm_index, none);
         }
