@@ -535,8 +535,9 @@ __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t b
         }
         __stcs(ready.sp_main + blk, make_uint4(mw[0], mw[1], mw[2], mw[3]));
         __stcs(ready.sp_res + blk, make_uint2((uint32_t)res, (uint32_t)(res >> 32)));
-        const int64_t row = blk / ready.nbk;
-        const int kb = (int)(blk - row * ready.nbk);
+        // (block numbers fit 32 bits here: the launcher checks; a 64-bit division costs ~80 instructions)
+        const uint32_t row = (uint32_t)blk / (uint32_t)ready.nbk;
+        const int kb = (int)((uint32_t)blk - row * (uint32_t)ready.nbk);
         const int r = (int)(row & 127);
         *reinterpret_cast<uint16_t*>(ready.sp_meta + ((size_t)(row >> 7) * ready.sp_stages + (kb >> 3)) * 2048 + r * 16 +
                                      (kb & 7) * 2) = (uint16_t)meta;
@@ -545,18 +546,42 @@ __device__ __forceinline__ void quantize_block_bf16(uint32_t (&x)[16], int64_t b
     }
     if (kReady == 1) {
         static_assert(kReady != 1 || kMode <= 1, "GEMM-ready output: MXFP4 and MXFP4+ only");
-        const uint32_t p = (kPlus && !dead) ? bm : 32u;  // BM position, none in a dead block
-        uint4 s0 = e2m1x16_to_e2m3_slot(outv.x, outv.y, p < 16u ? p : 16u);
-        uint4 s1 = e2m1x16_to_e2m3_slot(outv.z, outv.w, (p >= 16u && p < 32u) ? p - 16u : 16u);
-        // 32 six-bit codes = 24 bytes (the GEMM's tensor map spreads every 12 into a 16-byte slot)
+        // E2M1 code s e e m -> E2M3 code s e e m 0 0 (same exponent bias): a nibble times four,
+        // one code per byte first (even and odd nibbles by two masks, interleaved by byte permutes)
+        const uint32_t ov[4] = {outv.x, outv.y, outv.z, outv.w};
+        uint32_t c[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t ev = (ov[i] << 2) & 0x3C3C3C3Cu, od = (ov[i] >> 2) & 0x3C3C3C3Cu;
+            c[2 * i] = __byte_perm(ev, od, 0x5140);
+            c[2 * i + 1] = __byte_perm(ev, od, 0x7362);
+        }
+        if (kPlus) {
+            // Eq. 3's BM branch: 4 + m/2 is the E2M3 code s 11 mmm; the sign bit the cast wrote stays
+            const uint32_t pos = 8u * (bm & 3u);
+            const uint32_t field = 0x1Fu << pos, value = (0x18u | m) << pos;
+            const uint32_t word = dead ? 8u : bm >> 2;  // (a dead block's codes are zero already)
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                asm("{ .reg .pred p;\n  setp.eq.u32 p, %1, %2;\n  @p lop3.b32 %0, %0, %3, %4, 0xBA; }"
+                    : "+r"(c[i]) : "r"(word), "r"((uint32_t)i), "r"(field), "r"(value));
+        }
+        // 32 six-bit codes = 24 bytes (the GEMM's tensor map spreads every 12 into a 16-byte slot):
+        // bytes a b c d -> a | b << 6 | c << 12 | d << 18 by two bit-selects, then byte permutes
+        uint32_t g[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t q = (c[i] & 0x003F003Fu) | ((c[i] >> 2) & ~0x003F003Fu);
+            g[i] = (q & 0xFFFu) | ((q >> 4) & ~0xFFFu);
+        }
         uint2* out6 = reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(ready.slots) + blk * 24);
-        __stcs(out6, make_uint2(s0.x, s0.y));
-        __stcs(out6 + 1, make_uint2(s0.z, s1.x));
-        __stcs(out6 + 2, make_uint2(s1.y, s1.z));
-        const int64_t row = blk / ready.nbk;
-        const int kb = (int)(blk - row * ready.nbk);
+        __stcs(out6, make_uint2(__byte_perm(g[0], g[1], 0x4210), __byte_perm(g[1], g[2], 0x5421)));
+        __stcs(out6 + 1, make_uint2(__byte_perm(g[2], g[3], 0x6542), __byte_perm(g[4], g[5], 0x4210)));
+        __stcs(out6 + 2, make_uint2(__byte_perm(g[5], g[6], 0x5421), __byte_perm(g[6], g[7], 0x6542)));
+        const uint32_t row = (uint32_t)blk / (uint32_t)ready.nbk;
+        const int kb = (int)((uint32_t)blk - row * (uint32_t)ready.nbk);
         const int r = (int)(row & 127);
-        ready.atoms[((row >> 7) * (ready.nbk >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)] =
+        ready.atoms[((size_t)(row >> 7) * (ready.nbk >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (kb & 3)] =
             (uint8_t)sb;
     }
 }
@@ -817,6 +842,7 @@ cudaError_t launch_quantize_ready(const void* src, int64_t rows, int64_t cols, m
                                   cudaStream_t stream)
 {
     const int64_t total_blocks = rows * (cols / 32);
+    if (total_blocks >= (1ll << 32)) return cudaErrorNotSupported;  // the kernel's block numbers are 32-bit
     GemmReady ready = {};
     ready.atoms = atoms;
     ready.slots = reinterpret_cast<uint4*>(slots);
