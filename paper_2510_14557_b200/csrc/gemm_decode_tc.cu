@@ -147,11 +147,11 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
         if (plus) {
             l.raw = o;   // the activation rows as given (bf16), for the BM_L term
             o += (size_t)kSelfMaxM * (size_t)self_nst * kStageK * 2;
-            l.corr = o;  // its sums [tile parity][group][row m][weight row]
-            o += 2 * kResGroups * kSelfMaxM * 128 * sizeof(float);
+            l.corr = o;  // its sums [group][row m][weight row]
+            o += kResGroups * kSelfMaxM * 128 * sizeof(float);
         }
         l.bars = up(o, 16);
-        l.total = l.bars + 1024 + 1024;
+        l.total = l.bars + 512 + 1024;  // barriers (under 512 bytes); slack for aligning the base
         return l;
     }
     l.act0 = (size_t)stages * l.slot;
@@ -400,18 +400,21 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     const int nst = prm.nst;
     const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S, kSelf ? nst : 0, prm.astages);
     const int SA = prm.astages;  // slots of the activation ring
+    // (what the kSelf form uses comes first and stays under the 512 bytes its layout reserves)
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // the slot's weight image landed
     uint64_t* empty = full + kMaxStages;       // the slot's MMAs are done (and its records read)
-    uint64_t* afull = empty + kMaxStages;      // the slot's activation image landed
+    uint64_t* acc_full = empty + kMaxStages;
+    uint64_t* acc_empty = acc_full + 1;
+    uint64_t* corr_full = acc_empty + 1;       // kSelf MX+: a tile's BM_L sums are complete
+    uint64_t* corr_empty = corr_full + 1;      // ... and have been taken
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(corr_empty + 1);
+    volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
+    static_assert((2 * kMaxStages + 4) * 8 + 8 <= 384, "barriers of the kSelf form");
+    uint64_t* afull = reinterpret_cast<uint64_t*>(smem + L.bars + 384);  // the slot's activation image landed
     uint64_t* aempty = afull + kMaxStages;     // its MMAs are done
     uint64_t* res_full = aempty + kMaxStages;  // [kSideSlots] the slot's BM_L tile is written
     uint64_t* res_empty = res_full + kSideSlots;  //           its MMAs are done
-    uint64_t* acc_full = res_empty + kSideSlots;
-    uint64_t* acc_empty = acc_full + 1;
-    uint64_t* corr_full = acc_empty + 1;       // [2] kSelf MX+: a tile's BM_L sums are complete
-    uint64_t* corr_empty = corr_full + 2;      // [2] ... and have been taken
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(corr_empty + 2);
-    volatile uint32_t* abort = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
+    static_assert(384 + (2 * kMaxStages + 2 * kSideSlots) * 8 <= 1024, "barriers of the three-ring form");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     auto slot = [&](int s) { return smem + (size_t)s * L.slot; };
@@ -426,21 +429,21 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     if (threadIdx.x == 0) {
         MXP_TL(0);  // kernel entry
         for (int s = 0; s < kMaxStages; ++s) {
-            ptx::mbar_init(&afull[s], 1);
-            ptx::mbar_init(&aempty[s], 1);
+            if (!kSelf) {
+                ptx::mbar_init(&afull[s], 1);
+                ptx::mbar_init(&aempty[s], 1);
+            }
             ptx::mbar_init(&full[s], 1);
             ptx::mbar_init(&empty[s], !kPlus ? 1 : kSelf ? 1 + kResWarps : 1 + kTileWarps);  // + the warps that read its records
         }
-        for (int s = 0; s < kSideSlots; ++s) {
+        for (int s = 0; s < kSideSlots && !kSelf; ++s) {
             ptx::mbar_init(&res_full[s], kTileWarps);
             ptx::mbar_init(&res_empty[s], 1);
         }
         ptx::mbar_init(acc_full, kIssuers);
         ptx::mbar_init(acc_empty, 4);
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(&corr_full[b], kResWarps * kResGroups);
-            ptx::mbar_init(&corr_empty[b], 4);
-        }
+        ptx::mbar_init(corr_full, kResWarps * kResGroups);
+        ptx::mbar_init(corr_empty, 4);
         *abort = 0u;
         ptx::fence_mbar_init();
     }
@@ -676,12 +679,12 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             if (lane == 0) ptx::mbar_arrive(acc_empty);
             if (kSelf && kPlus) {
                 // Eq. 4's BM_L term of this tile, summed on the CUDA cores by the warps below
-                if (!ptx::mbar_wait_relaxed(&corr_full[t & 1], (uint32_t)(t >> 1) & 1, abort, kWaitLimit, 100u)) {
+                if (!ptx::mbar_wait_relaxed(&corr_full[0], (uint32_t)t & 1, abort, kWaitLimit, 100u)) {
                     if (lane == 0) report(prm.status, abort, 0x7900);
                     break;
                 }
                 const float* corr =
-                    reinterpret_cast<const float*>(smem + L.corr) + (size_t)(t & 1) * kResGroups * kSelfMaxM * 128;
+                    reinterpret_cast<const float*>(smem + L.corr);
 #pragma unroll
                 for (int m = 0; m < kSelfMaxM; ++m) {
                     float c = 0.f;
@@ -690,7 +693,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     o[m] += c;
                 }
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&corr_empty[t & 1]);
+                if (lane == 0) ptx::mbar_arrive(&corr_empty[0]);
             }
             if (row < rows_here) {
 #pragma unroll
@@ -759,17 +762,17 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 if (lane == 0) ptx::mbar_arrive(&empty[s]);  // the slot's records have been read
             }
             if (!ok) break;
-            // the sums of tile t - 2 must have been taken before this tile's are written
-            if (t >= 2 && !ptx::mbar_wait(&corr_empty[t & 1], (uint32_t)((t - 2) >> 1) & 1, abort, kWaitLimit)) {
+            // the sums of the tile before must have been taken before this tile's are written
+            if (t >= 1 && !ptx::mbar_wait(&corr_empty[0], (uint32_t)(t - 1) & 1, abort, kWaitLimit)) {
                 if (lane == 0) report(prm.status, abort, 0x7A00);
                 break;
             }
             float* corr = reinterpret_cast<float*>(smem + L.corr) +
-                          ((size_t)(t & 1) * kResGroups + grp) * kSelfMaxM * 128;
+                          (size_t)grp * kSelfMaxM * 128;
 #pragma unroll
             for (int m = 0; m < kSelfMaxM; ++m) corr[m * 128 + r] = acc[m];  // this group's share, zeros included
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&corr_full[t & 1]);
+            if (lane == 0) ptx::mbar_arrive(&corr_full[0]);
         }
     } else if (kPlus) {
         // ---------------------------------------------------------------- BM_L tiles
