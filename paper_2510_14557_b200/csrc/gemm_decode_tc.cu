@@ -489,7 +489,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         const int per_row = nst * 32, tasks = prm.M * per_row;
         const uint32_t img_codes0 = ptx::smem_u32(smem + L.img_codes), img_sf0 = ptx::smem_u32(smem + L.img_sf);
         auto fetch = [&](int i) {
-            const int m = i / per_row, rem = i - m * per_row;
+            const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;
             return __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + (int64_t)rem * 8));
         };
         int i = (int)threadIdx.x;
@@ -499,7 +499,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             const int nxt = i + kThreads;
             uint4 vn = make_uint4(0u, 0u, 0u, 0u);
             if (nxt < tasks) vn = fetch(nxt);
-            const int m = i / per_row, rem = i - m * per_row;
+            const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;  // (a literal row: the planes' addresses fold)
             const int st = rem >> 5, kb = (rem >> 2) & 7, qd = rem & 3;
             if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)rem * 8) * 2) = v;
             convert_quarter(v, m, kb, qd, img_codes0 + (uint32_t)st * 2048u, img_sf0 + (uint32_t)st * 512u, kSfb);
