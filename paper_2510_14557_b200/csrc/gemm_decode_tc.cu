@@ -717,7 +717,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         // BM_L is a zero weight.
         const int grp = (warp - kResWarp0) / kResWarps;
         const int r = (int)threadIdx.x - 32 * (kResWarp0 + grp * kResWarps);
-        const __nv_bfloat16* raw = reinterpret_cast<const __nv_bfloat16*>(smem + L.raw);
+        const uint32_t raw_sa = ptx::smem_u32(smem + L.raw), slot0_sa = ptx::smem_u32(smem), slot_bytes = (uint32_t)L.slot;
         const uint32_t so = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;
         bool ok = true;
         for (int t = 0; t < ntl && ok; ++t) {
@@ -732,10 +732,14 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     break;
                 }
                 if (r < prm.rows) {
-                    const uint8_t* atoms = slot(s) + (size_t)prm.rows * 128;
-                    const uint2 rec = *reinterpret_cast<const uint2*>(atoms + 2 * kAtom + (size_t)r * 8);
-                    const uint32_t sc_lo = *reinterpret_cast<const uint32_t*>(atoms + so);
-                    const uint32_t sc_hi = *reinterpret_cast<const uint32_t*>(atoms + kAtom + so);
+                    // (loads that name the shared window: as generic loads through pointers the
+                    // compiler cannot place, each costs 64-bit address arithmetic and more latency)
+                    const uint32_t atoms = slot0_sa + (uint32_t)s * slot_bytes + (uint32_t)prm.rows * 128u;
+                    uint2 rec;
+                    uint32_t sc_lo, sc_hi;
+                    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(rec.x), "=r"(rec.y) : "r"(atoms + 2u * kAtom + (uint32_t)r * 8u) : "memory");
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc_lo) : "r"(atoms + so) : "memory");
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc_hi) : "r"(atoms + kAtom + so) : "memory");
                     float w[8];
                     uint32_t k[8];
 #pragma unroll
@@ -745,14 +749,18 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                         // BM_L 2^(sc - 127) = (code / 2) 2^(sc - 127), the sign from the record
                         const float mag = (float)((b >> 5) & 3u) * 0.5f * __uint_as_float(sc << 23);
                         w[kb] = __uint_as_float(__float_as_uint(mag) | ((b & 0x80u) << 24));
-                        k[kb] = (uint32_t)st * kStageK + (uint32_t)kb * 32u + (b & 31u);
+                        k[kb] = raw_sa + 2u * ((uint32_t)st * kStageK + (uint32_t)kb * 32u + (b & 31u));
                     }
 #pragma unroll
                     for (int m = 0; m < kSelfMaxM; ++m) {
                         if (m < prm.M) {
                             float a[8];
 #pragma unroll
-                            for (int kb = 0; kb < 8; ++kb) a[kb] = __bfloat162float(raw[(size_t)m * nst * kStageK + k[kb]]);
+                            for (int kb = 0; kb < 8; ++kb) {
+                                uint32_t h;
+                                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(h) : "r"(k[kb] + 2u * (uint32_t)(m * nst * kStageK)) : "memory");
+                                a[kb] = __uint_as_float(h << 16);
+                            }
 #pragma unroll
                             for (int kb = 0; kb < 8; ++kb) acc[m] = fmaf(w[kb], a[kb], acc[m]);
                         }
