@@ -786,9 +786,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         // ---------------------------------------------------------------- BM_L tiles
         // Group g of three warps owns slot g of the tile ring and takes the stages whose running
         // number is g (mod 4), like issuer g: every barrier of the slot is waited on by one party
-        // only, stage after stage, so a parity never stands for the wrong phase.  The three warps
-        // clear the tile together (consecutive threads, consecutive 16 bytes), then a thread drops
-        // in, for its weight rows and per block, the code the record byte names.
+        // only, stage after stage, so a parity never stands for the wrong phase.
         static_assert(kTileGroups == kSideSlots && kTileGroups == kIssuers, "one owner per slot");
         const int grp = (warp - kResWarp0) / kTileWarps;
         const int r0 = (int)threadIdx.x - 32 * (kResWarp0 + grp * kTileWarps);
@@ -801,21 +799,25 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 if (lane == 0) report(prm.status, abort, 0x7700 + s);
                 break;
             }
-            uint8_t* tile = res_slot(sr);
-            for (int k = r0; k < prm.rows * 8; k += 32 * kTileWarps)
-                reinterpret_cast<uint4*>(tile)[k] = make_uint4(0u, 0u, 0u, 0u);
-            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(32 * kTileWarps) : "memory");
+            // A thread writes whole rows: per block one 16-byte chunk, zero but for the nibble its
+            // record byte names (stores and loads name the shared window).
+            const uint32_t tile = ptx::smem_u32(res_slot(sr));
+            const uint32_t recs = ptx::smem_u32(slot(s)) + (uint32_t)prm.rows * 128u + 2u * kAtom;
             for (int r = r0; r < prm.rows; r += 32 * kTileWarps) {
-                uint8_t* mine = tile + (size_t)r * 128;
-                const uint2 rec = *reinterpret_cast<const uint2*>(slot(s) + (size_t)prm.rows * 128 + 2 * kAtom + (size_t)r * 8);
+                uint2 rec;
+                asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(rec.x), "=r"(rec.y) : "r"(recs + (uint32_t)r * 8u) : "memory");
 #pragma unroll
                 for (int kb = 0; kb < 8; ++kb) {
                     const uint32_t b = ((kb < 4 ? rec.x : rec.y) >> (8 * (kb & 3))) & 255u;
-                    if (b & 0x60u) {
-                        const uint32_t pos = b & 31u;
-                        const uint32_t nib = ((b >> 5) & 3u) | ((b >> 4) & 8u);
-                        mine[(((uint32_t)kb ^ ((uint32_t)r & 7u)) << 4) + (pos >> 1)] = (uint8_t)(nib << (4u * (pos & 1u)));
-                    }
+                    // code 0 m1 m0 with the sign on top (0 when the record is empty), at nibble `pos` of the chunk
+                    const uint32_t pos = b & 31u;
+                    const uint32_t nib = (b & 0x60u) ? (((b >> 5) & 3u) | ((b >> 4) & 8u)) : 0u;
+                    const uint32_t v = nib << (4u * (pos & 7u));
+                    const uint32_t wi = pos >> 3;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(
+                                     tile + (uint32_t)r * 128u + ((((uint32_t)kb) ^ ((uint32_t)r & 7u)) << 4)),
+                                 "r"(wi == 0u ? v : 0u), "r"(wi == 1u ? v : 0u), "r"(wi == 2u ? v : 0u), "r"(wi == 3u ? v : 0u)
+                                 : "memory");
                 }
             }
             ptx::fence_proxy_async_smem();
