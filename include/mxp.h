@@ -59,8 +59,10 @@ typedef enum {
      * mxp_quantize and mxp_dequantize, and operands of the packed x packed mxp_gemm with its
      * full workspace (MXFP8 codes are read as stored; an MXFP6+ operand costs one more pass
      * over K, its BM being entered as the sum of two E2M3 values, an MXFP8+ operand two more,
-     * its BM being the sum of three E4M3 values); plain MXFP6 / MXFP8 also of mxp_gemm_prepack /
-     * mxp_gemm_prepacked; the other GEMM forms reject them. */
+     * its BM being the sum of three E4M3 values); as weights of the weight-only mxp_gemm (bf16
+     * activations) with the workspace mxp_gemm_workspace_bytes(..., a_dense = 1, ...) gives, at
+     * any M, K % 128 == 0; plain MXFP6 / MXFP8 also of mxp_gemm_prepack / mxp_gemm_prepacked;
+     * the other GEMM forms (decode kernels, chained and re-tiled forms) reject them. */
     MXP_MODE_MXFP6 = 3,      /* E2M3 elements, emax 2 */
     MXP_MODE_MXFP6_PLUS = 4, /* ... with the BM as sign + 5 mantissa bits: 4 + m/8, index byte */
     MXP_MODE_MXFP8 = 5,      /* E4M3 elements, emax 8 */
@@ -187,7 +189,8 @@ mxp_status mxp_dequantize(const mxp_packed *p, void *dst, mxp_dtype dst_dt, int6
  *     kernel, the activations entering as the exact sum of two E4M3 planes with a
  *     power-of-two scale per block of 32 -- elements more than 2^9 below their block's
  *     maximum are rounded at 2^-17 of that maximum; with less workspace a slower
- *     general kernel answers);
+ *     general kernel answers; MXFP6(+) / MXFP8(+) weights take the tensor-core kernel at every
+ *     M and return MXP_ERR_WORKSPACE without its workspace);
  *   - A_packed (host pointer to a descriptor): both operands are consumed by the
  *     block-scaled tensor-core path; any combination of MXFP4 / MXFP4+ modes.  With the full
  *     workspace: MXFP4 x MXFP4 runs FP4 instructions on the stored planes; one MXFP4+ operand

@@ -219,9 +219,9 @@ size_t mxp_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense, mx
     if (a_dense) {
         // more than 64 activation rows: the tensor-core kernel, which needs room for both
         // operands' prepared forms; decode shapes need none
-        if (M > 64 && N >= 128) {
+        if ((M > 64 && N >= 128) || wide_mode(b_mode)) {
             const size_t fast = mxp::stream_dense_workspace_bytes(M, N, K, b_mode);
-            if (fast != 0) return fast;
+            if (fast != 0 || wide_mode(b_mode)) return fast;
         }
         return mxp::skinny_workspace_bytes(M, N, K);
     }
@@ -244,7 +244,7 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt)) return MXP_ERR_INVALID_ARG;
     if ((A_dense_bf16 == nullptr) == (A_packed == nullptr)) return MXP_ERR_INVALID_ARG;
-    if (!valid_packed(B_packed, A_packed != nullptr)) return MXP_ERR_INVALID_ARG;
+    if (!valid_packed(B_packed, true)) return MXP_ERR_INVALID_ARG;
     if (B_packed->rows != N || B_packed->cols != K) return MXP_ERR_INVALID_ARG;
     if (A_packed != nullptr) {
         if (!valid_packed(A_packed, true)) return MXP_ERR_INVALID_ARG;
@@ -265,7 +265,10 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (A_dense_bf16 != nullptr) {
-        if (M > 64 && N >= 128 && workspace != nullptr && aligned(workspace, 256) &&
+        // the wider weight formats have the tensor-core kernel only, at any M and N
+        const bool wide_b = wide_mode(B_packed->mode);
+        if (wide_b && K % 128 != 0) return MXP_ERR_UNSUPPORTED;
+        if ((wide_b || (M > 64 && N >= 128)) && workspace != nullptr && aligned(workspace, 256) &&
             aligned(B_packed->scales, 4) && mxp::override_get(MXP_KNOB_WEIGHT_ONLY_KERNEL) == 0 &&
             (B_packed->mode != MXP_MODE_MXFP4_PP || aligned(B_packed->bm_index, 4))) {
             const size_t fast = mxp::stream_dense_workspace_bytes(M, N, K, B_packed->mode);
@@ -277,6 +280,7 @@ mxp_status mxp_gemm(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16, i
                                                   A_dense_bf16, lda);
             }
         }
+        if (wide_b) return MXP_ERR_WORKSPACE;  // needs mxp_gemm_workspace_bytes(..., a_dense = 1, ...)
         cudaError_t e = mxp::launch_gemm_weight_only(M, N, K, A_dense_bf16, lda, *B_packed, D,
                                                      d_dt, ldd, workspace, workspace_bytes, stream);
         if (e == cudaErrorNotSupported) return MXP_ERR_UNSUPPORTED;

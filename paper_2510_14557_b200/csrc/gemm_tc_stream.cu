@@ -1070,10 +1070,10 @@ prepack_dense_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, in
 
 size_t stream_dense_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode b_mode)
 {
-    if (M < 1 || N < 1 || K % 128 != 0 || b_mode > MXP_MODE_MXFP4_PP) return 0;
+    if (M < 1 || N < 1 || K % 128 != 0 || b_mode > MXP_MODE_MXFP8_PLUS) return 0;
     if ((uint64_t)M * (uint64_t)K / 16 >= (1ull << 31) || (uint64_t)N * (uint64_t)K / 16 >= (1ull << 32))
         return 0;
-    return layout(M, N, K, true, 2, 1).total;
+    return layout(M, N, K, true, 2, mode_parts(b_mode)).total;
 }
 
 size_t stream_dense_prepacked_workspace_bytes(int64_t M, int64_t K)
@@ -1303,7 +1303,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
 {
     // `a_dense`: bf16 activations (weight-only form); `A` is then a placeholder of mode MXFP4
     const bool dense = a_dense != nullptr;
-    if (dense && (a_ready || B.mode > MXP_MODE_MXFP4_PP)) return MXP_ERR_UNSUPPORTED;
+    if (dense && a_ready) return MXP_ERR_UNSUPPORTED;
     const bool ap = A.mode != MXP_MODE_MXFP4, bp = B.mode != MXP_MODE_MXFP4;
     const bool wide = ap || bp || a_ready || dense;
     // `a_ready`: A's atoms and code slots are in the workspace already (and the status block is

@@ -147,11 +147,37 @@ def test_unsupported_uses_of_the_wide_modes_are_rejected():
     a = torch.randn(256, 256, device="cuda", dtype=torch.bfloat16)
     p6 = m.mxp_quantize(a, 4)
     p8 = m.mxp_quantize(a, 6)
-    with pytest.raises(MxpError):  # weight-only form: 4-bit weights only
-        m.mxp_gemm(a, p6)
-    with pytest.raises(MxpError):  # weight-only form: 4-bit weights only
-        m.mxp_gemm(a, p8)
+    tiny = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(MxpError):  # weight-only form at these widths: the tensor-core kernel and its workspace only
+        m.mxp_gemm(a, p6, workspace=tiny)
+    with pytest.raises(MxpError):
+        m.mxp_gemm(a, p8, workspace=tiny)
     with pytest.raises(MxpError):  # an MXFP8+ operand has three planes: no prepacked form
         m.mxp_gemm_prepack(p8, True)
     with pytest.raises(MxpError):  # the + modes need the index plane
         m.mxp_quantize(a, 6, out=m.Packed(p8.nibbles, p8.scales, None, 256, 256, 6))
+
+
+@pytest.mark.parametrize("mode", [3, 4, 5, 6])
+@pytest.mark.parametrize("M,N,K", [(1, 300, 256), (16, 129, 512), (70, 520, 384), (300, 1000, 1024)])
+def test_weight_only_with_the_wider_weight_formats(M, N, K, mode):
+    # bf16 activations x MXFP6 / MXFP6+ / MXFP8 / MXFP8+ weights (Sec. 4.2 lists these widths beside
+    # MXFP4+): the block-scaled tensor-core kernel at any M, the activations as two E4M3 planes,
+    # the weights' BM as the sum of two (MXFP6+) or three (MXFP8+) planes; against the oracle's
+    # fp64 product of the decoded operands
+    from helpers import check_gemm
+    m = mxp()
+    a_bits, w_bits = synth.config3(M, N, K, seed=M + N + K + mode)
+    fmt, plus = MODES[mode]
+    codes, sc, idx = oracle.quantize_wide(w_bits, fmt, plus, bf16_bits=True)
+    dw = oracle.dequantize_wide(codes, sc, idx, fmt, plus)
+    da = oracle.bf16_bits_to_f64(a_bits)
+    wp = m.mxp_quantize(to_dev_bf16(w_bits), mode)
+    assert_equal(wp, reference_planes(w_bits, mode, bf16_bits=True), mode)
+    need = m.mxp_gemm_workspace_bytes(M, N, K, True, 0, mode)
+    assert need > 4096
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    for dt in (torch.float32, torch.bfloat16):
+        d = m.mxp_gemm(to_dev_bf16(a_bits), wp, out_dtype=dt, workspace=ws)
+        assert m.mxp_gemm_status(ws) == 0
+        check_gemm(d, da, dw)
