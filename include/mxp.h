@@ -61,7 +61,7 @@ typedef enum {
      * over K, its BM being entered as the sum of two E2M3 values, an MXFP8+ operand two more,
      * its BM being the sum of three E4M3 values); as weights of the weight-only mxp_gemm (bf16
      * activations) with the workspace mxp_gemm_workspace_bytes(..., a_dense = 1, ...) gives, at
-     * any M, K % 128 == 0; plain MXFP6 / MXFP8 also of mxp_gemm_prepack / mxp_gemm_prepacked;
+     * any M, K % 128 == 0; also of mxp_gemm_prepack / mxp_gemm_prepacked;
      * the other GEMM forms (decode kernels, chained and re-tiled forms) reject them. */
     MXP_MODE_MXFP6 = 3,      /* E2M3 elements, emax 2 */
     MXP_MODE_MXFP6_PLUS = 4, /* ... with the BM as sign + 5 mantissa bits: 4 + m/8, index byte */
@@ -240,6 +240,8 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
  *                      and the pairing is not one of the two above or below: both operands
  *                      MX+, the wider modes, and the weight-only tensor-core path
  *   MXP_PREPACK_WIDE8  16 bytes per 16 elements: E4M3 bytes, where B is MX++ or MXFP8
+ *   MXP_PREPACK_WIDE_X2   B is MXFP6+: two planes of E2M3 codes (its BM is the sum of two)
+ *   MXP_PREPACK_WIDE8_X3  B is MXFP8+: three planes of E4M3 bytes (its BM is the sum of three)
  *   MXP_PREPACK_SPLIT  B is MXFP4+ and A is MXFP4: Eq. 4's split for the sparse residual
  *                      instruction -- B's nibble plane with BM_H in every BM's place, BM_L
  *                      compressed 2:1, and the metadata that says where each BM_L sits
@@ -272,7 +274,14 @@ size_t mxp_gemm_min_workspace_bytes(int64_t M, int64_t N, int64_t K, int a_dense
  *                           scales.  Any M >= 1; 4-bit weight modes; K % 128 == 0.  Same
  *                           result as mxp_gemm's tensor-core weight-only path.
  */
-typedef enum { MXP_PREPACK_PLAIN = 0, MXP_PREPACK_WIDE = 1, MXP_PREPACK_SPLIT = 2, MXP_PREPACK_WIDE8 = 3 } mxp_prepack_form;
+typedef enum {
+    MXP_PREPACK_PLAIN = 0,
+    MXP_PREPACK_WIDE = 1,
+    MXP_PREPACK_SPLIT = 2,
+    MXP_PREPACK_WIDE8 = 3,
+    MXP_PREPACK_WIDE_X2 = 4,
+    MXP_PREPACK_WIDE8_X3 = 5
+} mxp_prepack_form;
 int mxp_gemm_prepack_form(mxp_mode a_mode, mxp_mode b_mode);
 size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int form);
 mxp_status mxp_gemm_prepack(const mxp_packed *P, int form, void *out, size_t out_bytes,

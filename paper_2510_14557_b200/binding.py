@@ -292,7 +292,7 @@ def mxp_gemm(a, b: Packed, out_dtype=torch.bfloat16, out: Optional[torch.Tensor]
     return out
 
 
-PREPACK_PLAIN, PREPACK_WIDE, PREPACK_SPLIT, PREPACK_WIDE8 = 0, 1, 2, 3
+PREPACK_PLAIN, PREPACK_WIDE, PREPACK_SPLIT, PREPACK_WIDE8, PREPACK_WIDE_X2, PREPACK_WIDE8_X3 = 0, 1, 2, 3, 4, 5
 
 
 def mxp_gemm_prepack_form(a_mode: int, b_mode: int) -> int:
@@ -305,7 +305,7 @@ def mxp_gemm_prepack(p: Packed, wide, out: Optional[torch.Tensor] = None) -> tor
     PREPACK_* form (True: the operand's widened form, False: PREPACK_PLAIN); take it from
     mxp_gemm_prepack_form(a_mode, b_mode) of the GEMMs the copy is for."""
     if wide is True:  # the operand's own widened form: E4M3 bytes for MX++ and MXFP8, E2M3 codes otherwise
-        wide = PREPACK_WIDE8 if p.mode in (2, 5, 6) else PREPACK_WIDE
+        wide = {2: PREPACK_WIDE8, 5: PREPACK_WIDE8, 4: PREPACK_WIDE_X2, 6: PREPACK_WIDE8_X3}.get(p.mode, PREPACK_WIDE)
     need = int(lib().mxp_gemm_prepack_bytes(p.rows, p.cols, int(wide)))
     if need == 0:
         raise MxpError("mxp_gemm_prepack_bytes", 2)

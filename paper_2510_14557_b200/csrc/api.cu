@@ -362,7 +362,7 @@ mxp_status mxp_gemm_prepack(const mxp_packed* P, int form, void* out, size_t out
                             void* cuda_stream)
 {
     if (!valid_packed(P, true)) return MXP_ERR_INVALID_ARG;
-    if (form < MXP_PREPACK_PLAIN || form > MXP_PREPACK_WIDE8) return MXP_ERR_INVALID_ARG;
+    if (form < MXP_PREPACK_PLAIN || form > MXP_PREPACK_WIDE8_X3) return MXP_ERR_INVALID_ARG;
     if (P->rows == 0 || P->cols == 0) return MXP_OK;
     if (P->mode != MXP_MODE_MXFP4 && form == MXP_PREPACK_PLAIN) return MXP_ERR_INVALID_ARG;
     if (P->mode != MXP_MODE_MXFP4_PLUS && form == MXP_PREPACK_SPLIT) return MXP_ERR_INVALID_ARG;
@@ -391,7 +391,7 @@ mxp_status mxp_gemm_prepacked(int64_t M, int64_t N, int64_t K, const mxp_packed*
     const size_t want = mxp::stream_prepack_bytes(N, K, form);
     if (want == 0) return MXP_ERR_UNSUPPORTED;
     if (B_prepacked_bytes != want || !aligned(B_prepacked, 256)) return MXP_ERR_INVALID_ARG;
-    if (form != MXP_PREPACK_WIDE && form != MXP_PREPACK_WIDE8 &&
+    if ((form == MXP_PREPACK_PLAIN || form == MXP_PREPACK_SPLIT) &&
         mxp::stream_sparse_workspace_bytes(M, N, K, A_packed->mode, B_packed->mode, true) != 0)
         return mxp::launch_gemm_tc_sparse(M, N, K, *A_packed, *B_packed, B_prepacked, D, d_dt, ldd,
                                           workspace, workspace_bytes,

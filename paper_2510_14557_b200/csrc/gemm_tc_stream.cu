@@ -1106,8 +1106,8 @@ struct PackedLayout {
     size_t atoms[2];  // scale atoms tiled for one-half tiles, for two-half tiles
     size_t wide, total;
 };
-// bits: 0 (scale atoms only), 6 or 8 (widened codes behind them)
-PackedLayout packed_layout(int64_t rows, int64_t K, int bits)
+// bits: 0 (scale atoms only), 6 or 8 (widened codes behind them, `parts` planes of them)
+PackedLayout packed_layout(int64_t rows, int64_t K, int bits, int parts = 1)
 {
     const bool wide = bits != 0;
     PackedLayout l;
@@ -1115,7 +1115,7 @@ PackedLayout packed_layout(int64_t rows, int64_t K, int bits)
     l.atoms[1] = round_up((size_t)row_groups(rows, sub_n(wide, 1)) * (size_t)(K / 128) * kAtom, 1024);
     l.wide = l.atoms[1] +
              round_up((size_t)row_groups(rows, sub_n(wide, 2)) * (size_t)(K / 128) * kAtom, 1024);
-    l.total = l.wide + round_up((size_t)rows * (size_t)K * (size_t)bits / 8, 1024);
+    l.total = l.wide + round_up((size_t)parts * (size_t)rows * (size_t)K * (size_t)bits / 8, 1024);
     return l;
 }
 
@@ -1231,18 +1231,25 @@ PrepackOperand no_operand()
 
 size_t stream_prepack_bytes(int64_t rows, int64_t K, int form)
 {
-    if (rows <= 0 || K <= 0 || K % 128 != 0 || form < 0 || form > MXP_PREPACK_WIDE8) return 0;
+    if (rows <= 0 || K <= 0 || K % 128 != 0 || form < 0 || form > MXP_PREPACK_WIDE8_X3) return 0;
     if ((uint64_t)rows * (uint64_t)K / 16 >= (1ull << 32)) return 0;
     if (form == MXP_PREPACK_SPLIT) return split_layout(rows, K).total;
+    if (form == MXP_PREPACK_WIDE_X2) return packed_layout(rows, K, 6, 2).total;
+    if (form == MXP_PREPACK_WIDE8_X3) return packed_layout(rows, K, 8, 3).total;
     return packed_layout(rows, K, form == MXP_PREPACK_WIDE ? 6 : form == MXP_PREPACK_WIDE8 ? 8 : 0).total;
 }
 
-int stream_wide_form(mxp_mode b_mode) { return wide_bits(b_mode) == 8 ? MXP_PREPACK_WIDE8 : MXP_PREPACK_WIDE; }
+int stream_wide_form(mxp_mode b_mode)
+{
+    if (b_mode == MXP_MODE_MXFP6_PLUS) return MXP_PREPACK_WIDE_X2;   // its BM is the sum of two E2M3 planes
+    if (b_mode == MXP_MODE_MXFP8_PLUS) return MXP_PREPACK_WIDE8_X3;  // ... of three E4M3 planes
+    return wide_bits(b_mode) == 8 ? MXP_PREPACK_WIDE8 : MXP_PREPACK_WIDE;
+}
 
 mxp_status stream_prepack(const mxp_packed& P, int form, void* out, size_t out_bytes,
                           cudaStream_t stream)
 {
-    const bool wide = form == MXP_PREPACK_WIDE || form == MXP_PREPACK_WIDE8;
+    const bool wide = form != MXP_PREPACK_PLAIN && form != MXP_PREPACK_SPLIT;
     const size_t need = stream_prepack_bytes(P.rows, P.cols, form);
     if (need == 0) return MXP_ERR_UNSUPPORTED;
     if (wide && form != stream_wide_form(P.mode)) return MXP_ERR_INVALID_ARG;  // 6-bit codes or bytes: the mode's
@@ -1258,16 +1265,13 @@ mxp_status stream_prepack(const mxp_packed& P, int form, void* out, size_t out_b
         prepack_kernel<<<(unsigned)ctas, 256, 0, stream>>>(px, no_operand(), nullptr);
         return cudaGetLastError() == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
     }
-    // an MXFP6+ operand needs two planes, which this form has no room for: mxp_gemm takes it
-    if ((P.mode > MXP_MODE_MXFP6 && P.mode != MXP_MODE_MXFP8) ||
-        ((mode_six(P.mode) || mode_eight(P.mode)) && !wide))
-        return MXP_ERR_UNSUPPORTED;
+    if ((mode_six(P.mode) || mode_eight(P.mode)) && !wide) return MXP_ERR_UNSUPPORTED;
     if (out == nullptr || out_bytes < need) return MXP_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(out) & 255) || (reinterpret_cast<uintptr_t>(P.nibbles) & 15) ||
         (reinterpret_cast<uintptr_t>(P.scales) & 3) ||
         (P.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(P.bm_index) & 3)))
         return MXP_ERR_INVALID_ARG;
-    const PackedLayout l = packed_layout(P.rows, P.cols, wide ? wide_bits(P.mode) : 0);
+    const PackedLayout l = packed_layout(P.rows, P.cols, wide ? wide_bits(P.mode) : 0, mode_parts(P.mode));
     uint8_t* o = static_cast<uint8_t*>(out);
     // both tilings of the scales (the GEMM picks its tile shape per call); widened bytes once
     const PrepackOperand p1 =
@@ -1311,7 +1315,6 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
     if (a_ready && (b_prepacked == nullptr || A.mode > MXP_MODE_MXFP4_PLUS)) return MXP_ERR_UNSUPPORTED;
     if (A.mode > MXP_MODE_MXFP8_PLUS || B.mode > MXP_MODE_MXFP8_PLUS) return MXP_ERR_UNSUPPORTED;
     const int parts_a = dense ? 2 : mode_parts(A.mode), parts_b = mode_parts(B.mode);
-    if (b_prepacked != nullptr && parts_b != 1) return MXP_ERR_UNSUPPORTED;
     const Layout l = layout(M, b_prepacked ? 0 : N, K, wide, parts_a, parts_b);
     if (workspace == nullptr || workspace_bytes < l.total) return MXP_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return MXP_ERR_INVALID_ARG;
@@ -1337,7 +1340,7 @@ mxp_status launch_gemm_tc_stream(int64_t M, int64_t N, int64_t K, const mxp_pack
         (B.mode == MXP_MODE_MXFP4_PP && (reinterpret_cast<uintptr_t>(B.bm_index) & 3)))
         return MXP_ERR_INVALID_ARG;
 
-    const PackedLayout lb = packed_layout(N, K, wide ? wide_bits(B.mode) : 0);
+    const PackedLayout lb = packed_layout(N, K, wide ? wide_bits(B.mode) : 0, parts_b);
     const uint8_t* b_atoms =
         b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.atoms[halves - 1] : ws + l.sfb;
     const uint8_t* b_wide = b_prepacked ? static_cast<const uint8_t*>(b_prepacked) + lb.wide : ws + l.wb;

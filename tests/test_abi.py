@@ -135,7 +135,11 @@ def test_prepacked_copies_are_checked_against_the_call(lib):
     size = {f: lib.mxp_gemm_prepack_bytes(N, K, f) for f in (PLAIN, WIDE, SPLIT, WIDE8)}
     assert 0 < size[PLAIN] < min(size[SPLIT], size[WIDE]) and size[WIDE] < size[WIDE8] and len(set(size.values())) == 4
     assert size[WIDE] - size[PLAIN] == N * K * 3 // 4 and size[WIDE8] - size[PLAIN] == N * K
-    assert lib.mxp_gemm_prepack_bytes(N, K, 4) == 0 and lib.mxp_gemm_prepack_bytes(N, 96, WIDE) == 0
+    assert lib.mxp_gemm_prepack_bytes(N, K, 6) == 0 and lib.mxp_gemm_prepack_bytes(N, 96, WIDE) == 0
+    # MXFP6+ / MXFP8+ weights: two planes of E2M3 codes, three planes of E4M3 bytes
+    assert form(MX, 4) == 4 and form(MXP, 6) == 5
+    assert lib.mxp_gemm_prepack_bytes(N, K, 4) - size[PLAIN] == 2 * N * K * 3 // 4
+    assert lib.mxp_gemm_prepack_bytes(N, K, 5) - size[PLAIN] == 3 * N * K
     ws = 1 << 30
     gp = lib.mxp_gemm_prepacked
 

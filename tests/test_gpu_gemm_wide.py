@@ -169,9 +169,8 @@ def test_tc_mxfp6_quantized_end_to_end_and_rejections():
     # weight-only with 6-bit weights: the same kernel, bf16 activations as two E4M3 planes
     a_bits = synth.f32_to_bf16_bits(a)
     check_gemm(m.mxp_gemm(to_dev_bf16(a_bits), pw, out_dtype=torch.float32), oracle.bf16_bits_to_f64(a_bits), dw)
-    p8 = m.mxp_quantize(to_dev(a), 6)
-    with pytest.raises(MxpError):   # an MXFP8+ operand has three planes: no prepacked form
-        m.mxp_gemm_prepack(p8, True)
+    with pytest.raises(MxpError):   # the copy's form is the operand's own: one plane is not an MXFP6+ operand's
+        m.mxp_gemm_prepack(pa, m.PREPACK_WIDE)
 
 
 # ------------------------------------------------------------------ MXFP8 operands
@@ -297,3 +296,22 @@ def test_quantize_gemm_ready_rejections():
     with pytest.raises(MxpError):   # workspace too small
         m.mxp_quantize_gemm_ready(x.bfloat16(), MXP, ws[:4096])
 
+
+@pytest.mark.parametrize("bmode", [3, 4, 5, 6])
+@pytest.mark.parametrize("amode", [MXP, 4])
+def test_tc_prepacked_weights_at_the_wider_formats(amode, bmode):
+    # weights prepared once, all planes of an MXFP6+ (two) or MXFP8+ (three) operand included:
+    # the same result as mxp_gemm on the same operands, to the bit
+    m = mxp()
+    M, N, K = 300, 520, 512
+    ap, da = _operand_of(M, K, amode, seed=81)
+    bp, db = _operand_of(N, K, bmode, seed=82)
+    form = m.mxp_gemm_prepack_form(amode, bmode)
+    assert form == {3: m.PREPACK_WIDE, 4: m.PREPACK_WIDE_X2, 5: m.PREPACK_WIDE8, 6: m.PREPACK_WIDE8_X3}[bmode]
+    pre = m.mxp_gemm_prepack(bp, form)
+    assert pre.numel() == m.mxp_gemm_prepack(bp, True).numel()
+    for dt in (torch.float32, torch.bfloat16):
+        d0 = m.mxp_gemm(ap, bp, out_dtype=dt)
+        d1 = m.mxp_gemm_prepacked(ap, bp, pre, out_dtype=dt)
+        check_gemm(d1, da, db)
+        assert torch.equal(d0, d1)

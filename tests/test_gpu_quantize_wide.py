@@ -152,8 +152,8 @@ def test_unsupported_uses_of_the_wide_modes_are_rejected():
         m.mxp_gemm(a, p6, workspace=tiny)
     with pytest.raises(MxpError):
         m.mxp_gemm(a, p8, workspace=tiny)
-    with pytest.raises(MxpError):  # an MXFP8+ operand has three planes: no prepacked form
-        m.mxp_gemm_prepack(p8, True)
+    with pytest.raises(MxpError):  # an MXFP8+ operand's prepacked copy has three planes, not one
+        m.mxp_gemm_prepack(p8, m.PREPACK_WIDE8)
     with pytest.raises(MxpError):  # the + modes need the index plane
         m.mxp_quantize(a, 6, out=m.Packed(p8.nibbles, p8.scales, None, 256, 256, 6))
 
