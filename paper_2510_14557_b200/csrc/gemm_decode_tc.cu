@@ -426,31 +426,31 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     const uint32_t total = (uint32_t)(ntl * nst);
     const uint8_t* wsrc = prm.wimg + (size_t)blockIdx.x * prm.tiles * nst * prm.wimg_bytes;
 
-    if (threadIdx.x == 0) {
-        MXP_TL(0);  // kernel entry
-        for (int s = 0; s < kMaxStages; ++s) {
-            if (!kSelf) {
-                ptx::mbar_init(&afull[s], 1);
-                ptx::mbar_init(&aempty[s], 1);
-            }
-            ptx::mbar_init(&full[s], 1);
-            ptx::mbar_init(&empty[s], !kPlus ? 1 : kSelf ? 1 + kResWarps : 1 + kTileWarps);  // + the warps that read its records
-        }
-        for (int s = 0; s < kSideSlots && !kSelf; ++s) {
-            ptx::mbar_init(&res_full[s], kTileWarps);
-            ptx::mbar_init(&res_empty[s], 1);
-        }
-        ptx::mbar_init(acc_full, kIssuers);
-        ptx::mbar_init(acc_empty, 4);
-        ptx::mbar_init(corr_full, kResWarps * kResGroups);
-        ptx::mbar_init(corr_empty, 4);
-        *abort = 0u;
-        ptx::fence_mbar_init();
-    }
     if (warp == 0) {
-        // The first ring-full of weight copies goes out before anything else, a lane each: the
-        // weights do not depend on the kernel before, and every later step of the set-up
-        // overlaps their latency.
+        // Barriers: a lane per ring slot.  Then the first ring-full of weight copies, a lane each,
+        // before anything else: the weights do not depend on the kernel before, and every later
+        // step of the set-up overlaps their latency.
+        if (lane == 0) MXP_TL(0);  // kernel entry
+        if (lane < kMaxStages) {
+            if (!kSelf) {
+                ptx::mbar_init(&afull[lane], 1);
+                ptx::mbar_init(&aempty[lane], 1);
+            }
+            ptx::mbar_init(&full[lane], 1);
+            ptx::mbar_init(&empty[lane], !kPlus ? 1 : kSelf ? 1 + kResWarps : 1 + kTileWarps);  // + the warps that read its records
+        } else if (lane < kMaxStages + kSideSlots) {
+            if (!kSelf) {
+                ptx::mbar_init(&res_full[lane - kMaxStages], kTileWarps);
+                ptx::mbar_init(&res_empty[lane - kMaxStages], 1);
+            }
+        } else if (lane == kMaxStages + kSideSlots) {
+            ptx::mbar_init(acc_full, kIssuers);
+            ptx::mbar_init(acc_empty, 4);
+            ptx::mbar_init(corr_full, kResWarps * kResGroups);
+            ptx::mbar_init(corr_empty, 4);
+            *abort = 0u;
+        }
+        ptx::fence_mbar_init();
         __syncwarp();
         const uint32_t c = (uint32_t)lane;
         if (c < total && c < (uint32_t)S) {
