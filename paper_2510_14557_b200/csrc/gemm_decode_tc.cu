@@ -170,15 +170,11 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
 __device__ unsigned long long g_decode_tl[8 * 256 * 8];   // [launch key][CTA][phase]
 __device__ const void* g_decode_tl_keys[8];                // weight buffers of the launches to tell apart
 __device__ unsigned long long g_decode_tl2[256 * 64];      // [CTA][event]: per-stage stamps of one role
-#define MXP_TL(slot)                                                                              \
-    do {                                                                                          \
-        int key_ = 0;                                                                             \
-        for (int k_ = 0; k_ < 8; ++k_)                                                            \
-            if (g_decode_tl_keys[k_] == (const void*)prm.wimg) key_ = k_;                         \
-        g_decode_tl[(key_ * 256 + blockIdx.x) * 8 + (slot)] = ptx::globaltimer_ns();              \
-    } while (0)
+#define MXP_TL(slot) do { g_decode_tl2[blockIdx.x * 64 + 56 + (slot)] = ptx::globaltimer_ns(); } while (0)
+#define MXP_TL2(ev) do { g_decode_tl2[blockIdx.x * 64 + (ev)] = ptx::globaltimer_ns(); } while (0)
 #else
 #define MXP_TL(slot) do { } while (0)
+#define MXP_TL2(ev) do { } while (0)
 #endif
 
 
@@ -426,10 +422,22 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     const uint32_t total = (uint32_t)(ntl * nst);
     const uint8_t* wsrc = prm.wimg + (size_t)blockIdx.x * prm.tiles * nst * prm.wimg_bytes;
 
+    // ---------------------------------------------------------------------- set-up
+    // Warp 0: barriers (a lane per ring slot), then the first ring-full of weight copies, a lane
+    // each: the weights do not depend on the kernel before, and everything else overlaps their
+    // latency.  Issuing sixteen bulk copies takes the warp ~0.5 us, so it only ARRIVES at the
+    // set-up barrier (before the copies) and the other warps do not wait for it.
+    // kSelf, warps 2 and up: the activations are asked for first of all (A is in stream order
+    // after the wait; once the weight stream is running, a load from L2 queues behind it).
+    constexpr int kConv0 = 64, kConv = kThreads - kConv0;  // threads that convert activations
+    const int cid = (int)threadIdx.x - kConv0;
+    const int per_row = nst * 32, tasks = kSelf ? prm.M * per_row : 0;
+    auto fetch = [&](int i) {
+        const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;
+        return __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + (int64_t)rem * 8));
+    };
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (warp == 0) {
-        // Barriers: a lane per ring slot.  Then the first ring-full of weight copies, a lane each,
-        // before anything else: the weights do not depend on the kernel before, and every later
-        // step of the set-up overlaps their latency.
         if (lane == 0) MXP_TL(0);  // kernel entry
         if (lane < kMaxStages) {
             if (!kSelf) {
@@ -451,52 +459,47 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             *abort = 0u;
         }
         ptx::fence_mbar_init();
+        __threadfence_block();
+        ptx::named_bar_arrive(1, kThreads);
         __syncwarp();
         const uint32_t c = (uint32_t)lane;
         if (c < total && c < (uint32_t)S) {
             ptx::mbar_arrive_expect_tx(&full[c], prm.wimg_bytes);
             bulk_g2s(slot((int)c), wsrc + (size_t)c * prm.wimg_bytes, prm.wimg_bytes, &full[c]);
         }
+        if (lane == 0) MXP_TL2(55);
+    } else {
+        if (warp == 1) {
+            ptx::tmem_alloc(tmem_slot, kTmemCols);
+            ptx::tmem_relinquish();
+        } else if (kSelf) {
+            ptx::grid_dependency_wait();
+            if (cid < tasks) v = fetch(cid);
+            // the images' unused rows: zero codes under a finite scale (the rows in use land on top)
+            for (int i = cid; i < nst * 128; i += kConv)
+                reinterpret_cast<uint4*>(smem + L.img_codes)[i] = make_uint4(0u, 0u, 0u, 0u);
+            for (int i = cid; i < nst * 32; i += kConv)
+                reinterpret_cast<uint4*>(smem + L.img_sf)[i] =
+                    make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+        }
+        ptx::tc_fence_before_sync();
+        ptx::named_bar_sync(1, kThreads);
+        ptx::tc_fence_after_sync();
     }
-    if (warp == 1) {
-        ptx::tmem_alloc(tmem_slot, kTmemCols);
-        ptx::tmem_relinquish();
-    }
-    if (kSelf) {
-        // the images' unused rows: zero codes under a finite scale (the rows in use land on top)
-        for (int i = threadIdx.x; i < nst * 128; i += kThreads)
-            reinterpret_cast<uint4*>(smem + L.img_codes)[i] = make_uint4(0u, 0u, 0u, 0u);
-        for (int i = threadIdx.x; i < nst * 32; i += kThreads)
-            reinterpret_cast<uint4*>(smem + L.img_sf)[i] =
-                make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::tc_fence_after_sync();
     ptx::grid_launch_dependents();  // whatever follows on the stream may be scheduled
-    const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 0) MXP_TL(1);  // set-up done
+    if (cid == 0) MXP_TL(1);  // set-up done
     if (kSelf) {
         // Activations -> digit planes, by this CTA for itself: a quad of lanes per block of 32,
-        // eight elements per lane, straight into the resident images.  A, D and the status block
-        // are in stream order from here on.
-        ptx::grid_dependency_wait();
-        if (prm.clear_status && blockIdx.x == 0 && threadIdx.x == 0 && prm.status != nullptr) {
+        // eight elements per lane, straight into the resident images.
+        if (prm.clear_status && blockIdx.x == 0 && cid == 0 && prm.status != nullptr) {
             prm.status->code = 0u;
             prm.status->where = 0u;
         }
         // (a thread's next eight elements are on their way from L2 while it converts these)
-        const int per_row = nst * 32, tasks = prm.M * per_row;
         const uint32_t img_codes0 = ptx::smem_u32(smem + L.img_codes), img_sf0 = ptx::smem_u32(smem + L.img_sf);
-        auto fetch = [&](int i) {
-            const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;
-            return __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + (int64_t)rem * 8));
-        };
-        int i = (int)threadIdx.x;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (i < tasks) v = fetch(i);
+        int i = cid >= 0 ? cid : tasks;
         while (i < tasks) {
-            const int nxt = i + kThreads;
+            const int nxt = i + kConv;
             uint4 vn = make_uint4(0u, 0u, 0u, 0u);
             if (nxt < tasks) vn = fetch(nxt);
             const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;  // (a literal row: the planes' addresses fold)
@@ -506,10 +509,14 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             v = vn;
             i = nxt;
         }
+        if (cid == 0) MXP_TL2(54);
         ptx::fence_proxy_async_smem();  // the MMAs read the images through the async proxy
+        ptx::tc_fence_before_sync();
         __syncthreads();
-        if (threadIdx.x == 0) MXP_TL(2);  // activations available
+        ptx::tc_fence_after_sync();
+        if (cid == 0) MXP_TL(2);  // activations available
     }
+    const uint32_t tmem_base = *tmem_slot;  // (warp 0 of the form without this barrier does not use it)
 
     if (warp == 0) {
         // ---------------------------------------------------------------- weight copies (the rest)
@@ -589,6 +596,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                         const uint32_t t_sfa = t_sf + 8u * (uint32_t)g, t_sfb = t_sfa + 4u;
                         ptx::tc_cp_sf(t_sfa, ptx::smem_desc_sf(sfa + (uint32_t)(g * kAtom)));
                         ptx::tc_cp_sf(t_sfb, ptx::smem_desc_sf(sfb + (uint32_t)(g * kSfb)));
+                    }
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const uint32_t t_sfa = t_sf + 8u * (uint32_t)g, t_sfb = t_sfa + 4u;
 #pragma unroll
                         for (int kk = 0; kk < 2; ++kk) {  // 64 elements = 32 bytes per MMA
                             const uint64_t adv = (uint64_t)((g * 2 + kk) * 32 >> 4);

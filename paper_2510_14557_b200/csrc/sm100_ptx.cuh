@@ -103,6 +103,18 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
     }
 }
 
+// ---------------------------------------------------------------------------- named barriers
+// Barrier `id` (1..15; 0 is __syncthreads) over `threads` threads of the CTA: a warp either
+// waits at it or only announces itself (its earlier writes are then visible to those who wait).
+__device__ __forceinline__ void named_bar_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_bar_arrive(int id, int threads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // ---------------------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
