@@ -11,7 +11,7 @@
 //     256 elements of K -- its rows' codes in the 128-byte-swizzled order the MMA reads, their
 //     scales in the 32-lane atoms tcgen05.cp copies, the BM records -- is one contiguous piece
 //     of about 11 KB that a single cp.async.bulk brings in.  148 CTAs read 148 sequential
-//     streams.
+//     streams.  The rows are dealt out evenly, a CTA on every SM (decode_plan says why).
 //   * MX+ (Eq. 4): the re-tiled codes hold BM_H (4 or 6, an E2M1 value) in the BM's place; the
 //     rest, BM_L in {0, 0.5, 1, 1.5}, also E2M1, goes into a second operand tile that is zero
 //     elsewhere, built per stage from one record byte per block (position, BM_L, sign) by four
@@ -41,7 +41,13 @@
 //     with a thread per (row, block) and the loads behind one another was ~3x slower and lost
 //     to the extra MMAs).  No BM_L tile is built and the MMA count per stage is that of plain
 //     MXFP4; the epilogue adds the three groups' partial sums in a fixed order.
-//   * warp 0 issues the weight copies (the first ring-full before the CTA's set-up barrier),
+//   * Set-up order (each step measured with per-phase time stamps): warp 0 initialises the
+//     barriers, a lane per ring slot, and issues the first ring-full of weight copies; sixteen
+//     bulk-copy instructions take that warp ~0.5 us, so it only arrives at the set-up barrier
+//     and nobody waits for it.  With kSelf the other warps ask for the activations before
+//     anything else: a load from L2 issued once the weight stream is running queues behind it
+//     (~1 us instead of ~0.3).  A stage's four scale copies go out ahead of its four MMAs.
+//   * warp 0 issues the weight copies,
 //     warp 1 the activation copies, warps 2-5 the MMAs (each every fourth stage, with an
 //     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 handle BM_L:
 //     for M >= 2 they build the BM_L operand tiles (four groups of three, group g owning slot g
