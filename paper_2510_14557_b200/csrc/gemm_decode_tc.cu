@@ -196,10 +196,14 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
     return l;
 }
 
-#ifdef MXP_DECODE_TIMELINE  // measurement build: per-CTA stamps of the phases, read back by a probe
-__device__ unsigned long long g_decode_tl[8 * 256 * 8];   // [launch key][CTA][phase]
-__device__ const void* g_decode_tl_keys[8];                // weight buffers of the launches to tell apart
-__device__ unsigned long long g_decode_tl2[256 * 64];      // [CTA][event]: per-stage stamps of one role
+#ifdef MXP_DECODE_TIMELINE  // measurement build: per-CTA time stamps of the last launch, read back by a probe
+// [CTA][event]: 32 + st = an issuer starts stage st; 54 = thread 64 has converted its share,
+// 55 = warp 0 has issued its copies; 56 + p = phase p (MXP_TL: 0 entry, 1 set-up done,
+// 2 activations available, 3 / 4 first / last stage seen by its issuer, 5 all MMAs done,
+// 6 output stored).  A stamp is one store and nothing else: a form that first looked up
+// which launch of a graph it belonged to (eight loads) held the stamping warp up by ~0.6 us
+// and moved every phase behind it.
+__device__ unsigned long long g_decode_tl2[256 * 64];
 #define MXP_TL(slot) do { g_decode_tl2[blockIdx.x * 64 + 56 + (slot)] = ptx::globaltimer_ns(); } while (0)
 #define MXP_TL2(ev) do { g_decode_tl2[blockIdx.x * 64 + (ev)] = ptx::globaltimer_ns(); } while (0)
 #else
@@ -941,19 +945,9 @@ cudaError_t launch_n(bool plus, bool f32, const DecodeParams& prm, int ctas, siz
 }  // namespace
 
 #ifdef MXP_DECODE_TIMELINE
-extern "C" int mxp_decode_timeline_read(unsigned long long* host, int n)
-{
-    return (int)cudaMemcpyFromSymbol(host, g_decode_tl, sizeof(unsigned long long) * (size_t)n);
-}
 extern "C" int mxp_decode_timeline_read2(unsigned long long* host, int n)
 {
     return (int)cudaMemcpyFromSymbol(host, g_decode_tl2, sizeof(unsigned long long) * (size_t)n);
-}
-extern "C" int mxp_decode_timeline_keys(const void* const* prepacked8)
-{
-    const void* keys[8];
-    for (int i = 0; i < 8; ++i) keys[i] = static_cast<const char*>(prepacked8[i]) + mxp::kHeaderBytes;
-    return (int)cudaMemcpyToSymbol(g_decode_tl_keys, keys, sizeof(keys));
 }
 #endif
 
