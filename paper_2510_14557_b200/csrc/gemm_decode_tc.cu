@@ -80,6 +80,7 @@ constexpr int kAtom = 512;
 constexpr int kMaxStages = 16;
 constexpr long long kWaitLimit = 4000000000ll;
 constexpr size_t kSmemMax = 227 * 1024;
+constexpr size_t kActSpread = 116 * 1024;  // shared memory that only one CTA per SM can have
 constexpr uint32_t kMagic = 0x4D58D0C2u;
 }  // namespace
 constexpr size_t kHeaderBytes = 256;
@@ -206,9 +207,13 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
 __device__ unsigned long long g_decode_tl2[256 * 64];
 #define MXP_TL(slot) do { g_decode_tl2[blockIdx.x * 64 + 56 + (slot)] = ptx::globaltimer_ns(); } while (0)
 #define MXP_TL2(ev) do { g_decode_tl2[blockIdx.x * 64 + (ev)] = ptx::globaltimer_ns(); } while (0)
+// the conversion kernel's CTA c uses row 200 + c: 0 entry, 1 images cleared, 2 dependency wait over,
+// 3 converted, 4 stored, 8 = the SM it ran on
+#define MXP_TLA(ev) do { if (threadIdx.x == 0) g_decode_tl2[(200 + blockIdx.x) * 64 + (ev)] = ptx::globaltimer_ns(); } while (0)
 #else
 #define MXP_TL(slot) do { } while (0)
 #define MXP_TL2(ev) do { } while (0)
+#define MXP_TLA(ev) do { } while (0)
 #endif
 
 
@@ -389,6 +394,14 @@ __global__ void __launch_bounds__(32 * kMaxM)
 decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int nact, uint8_t* __restrict__ aimg,
                   StatusBlock* status, int clear_status)
 {
+    MXP_TLA(0);
+#ifdef MXP_DECODE_TIMELINE
+    if (threadIdx.x == 0) {
+        unsigned sm;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+        g_decode_tl2[(200 + blockIdx.x) * 64 + 8] = sm;
+    }
+#endif
     ptx::grid_launch_dependents();  // the GEMM's CTAs may start streaming weights now
     extern __shared__ uint8_t img[];  // nact * 128 + 2 * sfb
     const int st = blockIdx.x;
@@ -399,7 +412,9 @@ decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int n
     for (int i = threadIdx.x; i < 2 * sfb / 16; i += blockDim.x)
         reinterpret_cast<uint4*>(img + nact * 128)[i] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
     __syncthreads();  // ... with a finite scale; the rows in use land on top
+    MXP_TLA(1);
     ptx::grid_dependency_wait();  // A may come from the kernel before
+    MXP_TLA(2);
     if (clear_status && st == 0 && threadIdx.x == 0 && status != nullptr) {
         status->code = 0u;
         status->where = 0u;
@@ -411,8 +426,10 @@ decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int n
         convert_quarter(v, m, kb, qd, ptx::smem_u32(img), ptx::smem_u32(img + nact * 128), sfb);
     }
     __syncthreads();
+    MXP_TLA(3);
     uint4* dst = reinterpret_cast<uint4*>(aimg + (size_t)st * bytes);
     for (int k = threadIdx.x; k < bytes / 16; k += blockDim.x) dst[k] = reinterpret_cast<const uint4*>(img)[k];
+    MXP_TLA(4);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1048,12 +1065,21 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
         if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !carve.done[dev]) {
             cudaFuncSetAttribute(decode_act_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
+            if (cudaFuncSetAttribute(decode_act_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kActSpread) != cudaSuccess)
+                return MXP_ERR_CUDA;
             carve.done[dev] = true;
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)p.nst);
         cfg.blockDim = dim3((unsigned)(32 * M < 64 ? 64 : 32 * M));
         cfg.dynamicSmemBytes = (size_t)nact * 128 + 2 * (size_t)sfb_bytes(nact);
+        // Up to eight rows its CTAs (8 KB, 256 threads) find room beside the GEMM's CTAs of the
+        // call before and wait there.  With more rows they do not (registers): they start when
+        // the first SMs become free, and four of them would share one of those SMs and take
+        // turns on its issue slots (measured: 5.6 us for the conversion instead of ~1).  Asking
+        // for more than half an SM's shared memory puts each on an SM of its own.
+        if (M > 8) cfg.dynamicSmemBytes = kActSpread;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
