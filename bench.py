@@ -589,7 +589,7 @@ def targets(mxp, synth, peaks):
     MXFP4, in a form short enough to survive at the end of the JSON line.
       quantize (config 2) and decode (config 3): fraction of the measured HBM copy bandwidth;
       prefill (configs 4 and 5): fraction of the dense FP4 peak = 4 x measured bf16 burst rate.
-    One launch (or one graph of eight) at a time with cold L2, i.e. the burst power state."""
+    One launch (or one graph of 32 chained calls) at a time with cold L2, i.e. the burst power state."""
     import torch
     hbm = peaks["hbm_gbs"]
     fp4 = peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16
@@ -607,7 +607,11 @@ def targets(mxp, synth, peaks):
     q["mx+/mxfp4"] = _r(q["mx+"]["us"] / q["mxfp4"]["us"], 3)
     out["quantize_cfg2"] = q
     del x
-    # ---- config 3: decode GEMM, eight rotating weight copies (> L2), graphs of eight launches.
+    # ---- config 3: decode GEMM, eight rotating weight copies (> L2), graphs of 32 launches (a
+    # token's pass over a model's layers is hundreds of such calls in one graph; the first call of
+    # a graph cannot overlap the graph before it, and with eight calls per graph that boundary
+    # alone adds ~0.5 us to every call's average).
+    kChain = 32
     # "tc": weights re-tiled once, FP4 tensor path (mxp_gemm_decode_prepacked); "reg": the
     # streamed register-decode kernel behind mxp_gemm; both as chains of programmatic dependents
     # (constant weights), which is what a captured decode loop can use.
@@ -634,8 +638,8 @@ def targets(mxp, synth, peaks):
             def run_reg():
                 mxp.mxp_gemm_decode_chained(a, packed[st["i"] % 8], d)
                 st["i"] += 1
-            us_tc = time_loop(graph_of(run_tc).replay, 6, warmup=2) / 8 * 1e3
-            us_reg = time_loop(graph_of(run_reg).replay, 6, warmup=2) / 8 * 1e3
+            us_tc = time_loop(graph_of(run_tc, kChain).replay, 6, warmup=2) / kChain * 1e3
+            us_reg = time_loop(graph_of(run_reg, kChain).replay, 6, warmup=2) / kChain * 1e3
             row["M%d" % M] = {"tc_us": _r(us_tc), "reg_us": _r(us_reg),
                               "frac": _r(tot / min(us_tc, us_reg) / 1e3 / hbm, 3)}
         dec[name] = row
@@ -644,6 +648,28 @@ def targets(mxp, synth, peaks):
                              min(dec["mxfp4"]["M1"]["tc_us"], dec["mxfp4"]["M1"]["reg_us"]), 3)
     out["decode_cfg3"] = dec
     del w
+    # ---- the same at M = 1 on a larger weight matrix (14336 x 4096, an 8B model's MLP width):
+    # the part of a call that carries no weight traffic weighs less.  Not one of the configs:
+    # beside them for context, the goal below is judged on config 3.
+    big = {}
+    N2, K2 = 14336, 4096
+    a2_bits, w2_bits = synth.config3(1, N2, K2, seed=11)
+    a2, w2 = dev_bf16(a2_bits), dev_bf16(w2_bits)
+    for name, mode in (("mx+", MXP), ("mxfp4", MX)):
+        tiled = [mxp.mxp_gemm_decode_prepack(mxp.mxp_quantize(w2, mode)) for _ in range(8)]
+        d = torch.empty((1, N2), dtype=torch.bfloat16, device="cuda")
+        ws = torch.zeros(max(256, mxp.mxp_gemm_decode_workspace_bytes(1, K2)), dtype=torch.uint8, device="cuda")
+        st = {"i": 0}
+
+        def run_big():
+            mxp.mxp_gemm_decode_prepacked(a2, tiled[st["i"] % 8], out=d, workspace=ws, chained=True)
+            st["i"] += 1
+        us = time_loop(graph_of(run_big, kChain).replay, 6, warmup=2) / kChain * 1e3
+        tot = N2 * K2 * (0.5 + 1 / 32 + (1 / 32 if mode == MXP else 0)) + K2 * 2 + N2 * 2
+        big[name] = {"tc_us": _r(us), "frac": _r(tot / us / 1e3 / hbm, 3)}
+        del tiled
+    out["decode_14336x4096_M1"] = big
+    del w2, a2
     # ---- configs 4 and 5: prefill.  Per mode pair the mxp_gemm_prepacked call (weights prepared
     # once; the activations' preparation is inside the timed call), queued behind an L2 eviction
     # (timed_queued: device time, not the host's launch latency).  One-sided pairs three ways:
