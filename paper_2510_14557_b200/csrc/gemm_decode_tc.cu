@@ -24,15 +24,15 @@
 //     A small kernel does this once per call (decode_act_kernel) and leaves the operand images
 //     of all stages in the workspace; the GEMM is launched as its programmatic dependent, so
 //     its CTAs stream weights meanwhile, and fetches the images stage by stage next to the
-//     weights.  (Converting inside the GEMM, every CTA for itself, costs a CTA ~1.6 us per
-//     activation row -- ~400 instructions per eight elements, sixteen warps' worth per row --
-//     which from the second row on is more than the second launch costs in a chain.)
-//   * A single activation row (kSelf): the dependent chain "kernel before -> conversion
-//     kernel -> this kernel's copies of the images" costs more than the conversion itself.
-//     There every CTA converts the row for itself, straight into shared memory where the
-//     images of all stages stay (40 KB at K = 4096), while its weights are already
-//     streaming: one launch per call, and no image travels through global memory.  (Two rows
-//     that way: 9.6 us against 8.75 us with the conversion kernel, calls chained in a graph.)
+//     weights.  (Converting inside the GEMM, every CTA for itself, costs a CTA 0.5-0.9 us per
+//     activation row -- ~280 instructions per eight elements, sixteen warps' worth per row --
+//     which from the fourth row on is more than the second launch costs in a chain.)
+//   * Up to three activation rows (kSelf; two with MX+ weights): the dependent chain "kernel
+//     before -> conversion kernel -> this kernel's copies of the images" costs more than the
+//     conversion itself.  There every CTA converts the rows for itself, straight into shared
+//     memory where the images of all stages stay (40 KB at K = 4096: three rows' planes fill
+//     one 16-row operand tile), while its weights are already streaming: one launch per call,
+//     and no image travels through global memory.  The number of rows is a template argument.
 //     MX+ there takes Eq. 4's BM_L term off the tensor cores: sum over blocks of
 //     (+-BM_L 2^shared_exp) a[k_BM] is eight products per weight row and stage, so warps 10-21
 //     add it on the CUDA cores in fp32 from the record bytes, the scale bytes and a raw bf16
@@ -157,10 +157,10 @@ struct DecodeLayout {
     size_t img_codes, img_sf, raw, corr;  // kSelf only (raw, corr: MX+)
     int stages, astages;
 };
-constexpr int kSelfMaxM = 1;
+constexpr int kSelfMaxM = 3;  // rows the self-converting form takes: three rows' planes fill one 16-row operand tile
 constexpr int kSideSlots = 4;
 __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages,
-                                                      int self_nst = 0, int astages = kSideSlots)
+                                                      int self_nst = 0, int astages = kSideSlots, int self_m = 1)
 {
     DecodeLayout l;
     l.stages = stages;
@@ -177,9 +177,9 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
         o += (size_t)self_nst * 512;
         if (plus) {
             l.raw = o;   // the activation rows as given (bf16), for the BM_L term
-            o += (size_t)kSelfMaxM * (size_t)self_nst * kStageK * 2;
+            o += (size_t)self_m * (size_t)self_nst * kStageK * 2;
             l.corr = o;  // its sums [group][row m][weight row]
-            o += kResGroups * kSelfMaxM * 128 * sizeof(float);
+            o += (size_t)kResGroups * self_m * 128 * sizeof(float);
         }
         l.bars = up(o, 16);
         l.total = l.bars + 512 + 1024;  // barriers (under 512 bytes); slack for aligning the base
@@ -435,18 +435,23 @@ decode_act_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, int M, int n
 // ------------------------------------------------------------------------------------------
 // The GEMM.  kNact: rows of the activation operand (16 .. 80); kPlus: MXFP4+ weights.
 // ------------------------------------------------------------------------------------------
-template <int kNact, bool kPlus, bool kSelf, typename OutT>
+// kSelfM: 0 = the activation images come from the conversion kernel; 1..3 = that many
+// activation rows, converted by every CTA for itself (a literal, so that the planes' addresses fold).
+template <int kNact, bool kPlus, int kSelfM, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_decode_tc_kernel(const DecodeParams prm)
 {
+    constexpr bool kSelf = kSelfM > 0;
+    constexpr int kSelfRows = kSelf ? kSelfM : 1;
+    static_assert(kSelfM <= kSelfMaxM && kPlanes * kSelfMaxM <= 16, "self-converted rows share one 16-row tile");
     static_assert(!kSelf || kNact == 16, "self-converted activations: one operand tile of 16 rows");
     constexpr int kSfb = sfb_bytes(kNact);
-    constexpr int kMt = kSelf ? kSelfMaxM : kNact / kPlanes;  // activation rows the operand can hold
+    constexpr int kMt = kSelf ? kSelfRows : kNact / kPlanes;  // activation rows the operand can hold
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int S = prm.stages;
     const int nst = prm.nst;
-    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S, kSelf ? nst : 0, prm.astages);
+    const DecodeLayout L = decode_layout(prm.rows, prm.wimg_bytes, kNact, kPlus, S, kSelf ? nst : 0, prm.astages, kSelfRows);
     const int SA = prm.astages;  // slots of the activation ring
     // (what the kSelf form uses comes first and stays under the 512 bytes its layout reserves)
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);  // the slot's weight image landed
@@ -484,12 +489,13 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     // after the wait; once the weight stream is running, a load from L2 queues behind it).
     constexpr int kConv0 = 64, kConv = kThreads - kConv0;  // threads that convert activations
     const int cid = (int)threadIdx.x - kConv0;
-    const int per_row = nst * 32, tasks = kSelf ? prm.M * per_row : 0;
-    auto fetch = [&](int i) {
-        const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;
-        return __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + (int64_t)rem * 8));
+    const int per_row = kSelf ? nst * 32 : 0;  // eight-element pieces of a row: a thread takes piece i of every row
+    auto fetch = [&](int m, int i) {
+        return __ldg(reinterpret_cast<const uint4*>(prm.A + (int64_t)m * prm.lda + (int64_t)i * 8));
     };
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    uint4 v[kSelfRows];
+#pragma unroll
+    for (int m = 0; m < kSelfRows; ++m) v[m] = make_uint4(0u, 0u, 0u, 0u);
     if (warp == 0) {
         if (lane == 0) MXP_TL(0);  // kernel entry
         if (lane < kMaxStages) {
@@ -527,7 +533,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
             ptx::tmem_relinquish();
         } else if (kSelf) {
             ptx::grid_dependency_wait();
-            if (cid < tasks) v = fetch(cid);
+            if (cid < per_row) {
+#pragma unroll
+                for (int m = 0; m < kSelfRows; ++m) v[m] = fetch(m, cid);
+            }
             // the images' unused rows: zero codes under a finite scale (the rows in use land on top)
             for (int i = cid; i < nst * 128; i += kConv)
                 reinterpret_cast<uint4*>(smem + L.img_codes)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -550,16 +559,19 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         }
         // (a thread's next eight elements are on their way from L2 while it converts these)
         const uint32_t img_codes0 = ptx::smem_u32(smem + L.img_codes), img_sf0 = ptx::smem_u32(smem + L.img_sf);
-        int i = cid >= 0 ? cid : tasks;
-        while (i < tasks) {
+        int i = cid >= 0 ? cid : per_row;
+        while (i < per_row) {
             const int nxt = i + kConv;
-            uint4 vn = make_uint4(0u, 0u, 0u, 0u);
-            if (nxt < tasks) vn = fetch(nxt);
-            const int m = kSelfMaxM == 1 ? 0 : i / per_row, rem = i - m * per_row;  // (a literal row: the planes' addresses fold)
-            const int st = rem >> 5, kb = (rem >> 2) & 7, qd = rem & 3;
-            if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)rem * 8) * 2) = v;
-            convert_quarter(v, m, kb, qd, img_codes0 + (uint32_t)st * 2048u, img_sf0 + (uint32_t)st * 512u, kSfb);
-            v = vn;
+            uint4 vn[kSelfRows];
+#pragma unroll
+            for (int m = 0; m < kSelfRows; ++m) vn[m] = nxt < per_row ? fetch(m, nxt) : make_uint4(0u, 0u, 0u, 0u);
+            const int st = i >> 5, kb = (i >> 2) & 7, qd = i & 3;
+#pragma unroll
+            for (int m = 0; m < kSelfRows; ++m) {
+                if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)i * 8) * 2) = v[m];
+                convert_quarter(v[m], m, kb, qd, img_codes0 + (uint32_t)st * 2048u, img_sf0 + (uint32_t)st * 512u, kSfb);
+                v[m] = vn[m];
+            }
             i = nxt;
         }
         if (cid == 0) MXP_TL2(54);
@@ -750,10 +762,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 const float* corr =
                     reinterpret_cast<const float*>(smem + L.corr);
 #pragma unroll
-                for (int m = 0; m < kSelfMaxM; ++m) {
+                for (int m = 0; m < kSelfRows; ++m) {
                     float c = 0.f;
 #pragma unroll
-                    for (int g = 0; g < kResGroups; ++g) c += corr[(g * kSelfMaxM + m) * 128 + row];  // fixed order
+                    for (int g = 0; g < kResGroups; ++g) c += corr[(g * kSelfRows + m) * 128 + row];  // fixed order
                     o[m] += c;
                 }
                 __syncwarp();
@@ -785,7 +797,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         const uint32_t so = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;
         bool ok = true;
         for (int t = 0; t < ntl && ok; ++t) {
-            float acc[kSelfMaxM] = {};
+            float acc[kSelfRows] = {};
             const int first = (grp + 3 * kResGroups - (int)(((uint32_t)t * (uint32_t)nst) % kResGroups)) % kResGroups;
             for (int st = first; st < nst; st += kResGroups) {
                 const uint32_t c = (uint32_t)t * (uint32_t)nst + (uint32_t)st;
@@ -816,7 +828,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                         k[kb] = raw_sa + 2u * ((uint32_t)st * kStageK + (uint32_t)kb * 32u + (b & 31u));
                     }
 #pragma unroll
-                    for (int m = 0; m < kSelfMaxM; ++m) {
+                    for (int m = 0; m < kSelfRows; ++m) {
                         if (m < prm.M) {
                             float a[8];
 #pragma unroll
@@ -840,9 +852,9 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 break;
             }
             float* corr = reinterpret_cast<float*>(smem + L.corr) +
-                          (size_t)grp * kSelfMaxM * 128;
+                          (size_t)grp * kSelfRows * 128;
 #pragma unroll
-            for (int m = 0; m < kSelfMaxM; ++m) corr[m * 128 + r] = acc[m];  // this group's share, zeros included
+            for (int m = 0; m < kSelfRows; ++m) corr[m * 128 + r] = acc[m];  // this group's share, zeros included
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&corr_full[0]);
         }
@@ -919,17 +931,17 @@ gemm_decode_tc_kernel(const DecodeParams prm)
 
 // Ring slots that fit: a multiple of four (see the issuers), at most sixteen.  self_nst > 0: the
 // form with resident activation images.
-int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0, int astages = kSideSlots)
+int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0, int astages = kSideSlots, int self_m = 1)
 {
     for (int s = kMaxStages; s >= 4; s -= 4)
-        if (decode_layout(p.rows, p.wimg, nact, plus, s, self_nst, astages).total <= kSmemMax) return s;
+        if (decode_layout(p.rows, p.wimg, nact, plus, s, self_nst, astages, self_m).total <= kSmemMax) return s;
     return 0;
 }
 
-template <int kNact, bool kPlus, bool kSelf, typename OutT>
+template <int kNact, bool kPlus, int kSelfM, typename OutT>
 cudaError_t launch(const DecodeParams& prm, int ctas, size_t smem, bool dependent, cudaStream_t stream)
 {
-    auto kern = gemm_decode_tc_kernel<kNact, kPlus, kSelf, OutT>;
+    auto kern = gemm_decode_tc_kernel<kNact, kPlus, kSelfM, OutT>;
     static SmemAttrOnce once;
     cudaError_t e = ensure_dynamic_smem(kern, (int)kSmemMax, once);
     if (e != cudaSuccess) return e;
@@ -948,15 +960,15 @@ cudaError_t launch(const DecodeParams& prm, int ctas, size_t smem, bool dependen
     return cudaLaunchKernelEx(&cfg, kern, prm);
 }
 
-template <int kNact, bool kSelf>
+template <int kNact, int kSelfM>
 cudaError_t launch_n(bool plus, bool f32, const DecodeParams& prm, int ctas, size_t smem, bool dependent,
                      cudaStream_t stream)
 {
     if (plus)
-        return f32 ? launch<kNact, true, kSelf, float>(prm, ctas, smem, dependent, stream)
-                   : launch<kNact, true, kSelf, __nv_bfloat16>(prm, ctas, smem, dependent, stream);
-    return f32 ? launch<kNact, false, kSelf, float>(prm, ctas, smem, dependent, stream)
-               : launch<kNact, false, kSelf, __nv_bfloat16>(prm, ctas, smem, dependent, stream);
+        return f32 ? launch<kNact, true, kSelfM, float>(prm, ctas, smem, dependent, stream)
+                   : launch<kNact, true, kSelfM, __nv_bfloat16>(prm, ctas, smem, dependent, stream);
+    return f32 ? launch<kNact, false, kSelfM, float>(prm, ctas, smem, dependent, stream)
+               : launch<kNact, false, kSelfM, __nv_bfloat16>(prm, ctas, smem, dependent, stream);
 }
 
 }  // namespace
@@ -1022,8 +1034,13 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     const size_t need = decode_workspace_bytes(M, K);
     if (workspace == nullptr || workspace_bytes < need) return MXP_ERR_WORKSPACE;
     const int nact = act_rows((int)M);
-    // a single row: every CTA converts it for itself, if its images fit beside a ring
-    const int self_stages = M <= kSelfMaxM ? pick_stages(p, nact, plus, p.nst) : 0;
+    // up to three rows (one 16-row operand tile): every CTA converts them for itself, if the
+    // images of all stages fit beside a ring.  (Measured at 11008 x 4096, chained: 7.7 / 8.1 us
+    // for two / three rows against 8.6 / 8.8 us with the conversion kernel; with MX+ weights
+    // 8.9 against 9.7 us for two rows, but 10.3 against 9.9 us for three: three rows as given
+    // take 24 KB from the ring and triple the BM_L sums' gathers.)
+    const bool try_self = M <= (plus ? 2 : kSelfMaxM);
+    const int self_stages = try_self ? pick_stages(p, nact, plus, p.nst, kSideSlots, (int)M) : 0;
     const bool self = self_stages != 0;
     // The activation ring: eight slots (the images come from L2 with ~1 us of latency: with four,
     // every fourth stage waits for its image) unless that leaves the weight ring fewer than eight.
@@ -1031,7 +1048,7 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     if (self || pick_stages(p, nact, plus, 0, astages) < 8) astages = kSideSlots;
     const int stages = self ? self_stages : pick_stages(p, nact, plus, 0, astages);
     if (stages == 0) return MXP_ERR_UNSUPPORTED;
-    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages, self ? p.nst : 0, astages);
+    const DecodeLayout L = decode_layout(p.rows, p.wimg, nact, plus, stages, self ? p.nst : 0, astages, self ? (int)M : 1);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     DecodeParams prm = {};
     prm.M = (int)M;
@@ -1054,7 +1071,9 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     prm.wimg_bytes = p.wimg;
     const bool f32 = d_dt == MXP_F32;
     if (self) {  // one launch; a programmatic dependent only on the caller's promise
-        const cudaError_t e = launch_n<16, true>(plus, f32, prm, p.ctas, L.total, chained, stream);
+        const cudaError_t e = M == 1   ? launch_n<16, 1>(plus, f32, prm, p.ctas, L.total, chained, stream)
+                              : M == 2 ? launch_n<16, 2>(plus, f32, prm, p.ctas, L.total, chained, stream)
+                                       : launch_n<16, 3>(plus, f32, prm, p.ctas, L.total, chained, stream);
         return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
     }
     {   // activations -> digit planes; in a chain it may start while the kernel before drains
@@ -1092,11 +1111,11 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     }
     cudaError_t e;
     switch (nact) {
-        case 16: e = launch_n<16, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
-        case 32: e = launch_n<32, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
-        case 48: e = launch_n<48, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
-        case 64: e = launch_n<64, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
-        default: e = launch_n<80, false>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 16: e = launch_n<16, 0>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 32: e = launch_n<32, 0>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 48: e = launch_n<48, 0>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        case 64: e = launch_n<64, 0>(plus, f32, prm, p.ctas, L.total, true, stream); break;
+        default: e = launch_n<80, 0>(plus, f32, prm, p.ctas, L.total, true, stream); break;
     }
     return e == cudaSuccess ? MXP_OK : MXP_ERR_CUDA;
 }

@@ -34,7 +34,7 @@ def raw_weights(N, K, mode, seed, lo=118, hi=136):
                                    (5, 1000, 768), (7, 19000, 512), (8, 11008, 4096), (9, 160, 4352),
                                    (12, 40000, 256), (13, 333, 1280), (16, 11008, 4096), (16, 8, 256), (1, 1, 256),
                                    (2, 40000, 256), (1, 40000, 256), (1, 19000, 8192), (1, 700, 16384), (2, 700, 16384),
-                                   (2, 11008, 4096)])
+                                   (2, 11008, 4096), (3, 11008, 4096), (3, 40000, 256), (3, 700, 16384)])
 def test_decode_prepacked_parity(M, N, K, wmode):
     # ragged N (last CTA short, rows not a multiple of 8), more than 128 rows per CTA (several
     # tiles), every activation-operand width (16 .. 80 rows), K from one stage to seventeen.
