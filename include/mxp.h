@@ -373,13 +373,16 @@ mxp_status mxp_gemm_decode_chained(int64_t M, int64_t N, int64_t K, const void *
  *   mxp_gemm_decode_prepacked  D[M,N] = A(bf16)[M,K] * dec(B)[N,K]^T.  `b_mode`, N, K must be
  *                            those B_prepacked was made with, and B_prepacked_bytes the size
  *                            mxp_gemm_decode_prepack_bytes gives for them (checked before any
- *                            launch: MXP_ERR_INVALID_ARG).  Two launches: a small kernel turns
- *                            the activations into five FP4 digit planes per row (balanced base
- *                            8, a block scale per plane: an element within 2^5 of the largest
- *                            magnitude of its block of 32 is exact, a smaller one is rounded at
- *                            2^-13 of that magnitude's binade -- far inside the GEMM's error
- *                            bound, which is relative to the row norm); the GEMM is launched as
- *                            its programmatic dependent and starts streaming weights at once.
+ *                            launch: MXP_ERR_INVALID_ARG).  The activations become five FP4
+ *                            digit planes per row (balanced base 8, a block scale per plane: an
+ *                            element within 2^5 of the largest magnitude of its block of 32 is
+ *                            exact, a smaller one is rounded at 2^-13 of that magnitude's
+ *                            binade -- far inside the GEMM's error bound, which is relative to
+ *                            the row norm).  Up to three rows (two with MXFP4+ weights), when
+ *                            the planes of all of K fit shared memory: one launch, every CTA
+ *                            converts the rows for itself.  Otherwise two launches: a small
+ *                            kernel writes the planes to the workspace and the GEMM is launched
+ *                            as its programmatic dependent and starts streaming weights at once.
  *                            chained != 0: the first kernel is itself launched as a
  *                            programmatic dependent of whatever precedes it on the stream, with
  *                            the promise and the status-block rule of mxp_gemm_decode_chained
