@@ -612,7 +612,8 @@ def targets(mxp, synth, peaks):
     # a graph cannot overlap the graph before it, and with eight calls per graph that boundary
     # alone adds ~0.5 us to every call's average).
     kChain = 32
-    # "tc": weights re-tiled once, FP4 tensor path (mxp_gemm_decode_prepacked); "reg": the
+    # "tc": weights re-tiled once, FP4 tensor path (mxp_gemm_decode_prepacked_next: each call
+    # names the weights of the next; "tc_nohint": mxp_gemm_decode_prepacked, without); "reg": the
     # streamed register-decode kernel behind mxp_gemm; both as chains of programmatic dependents
     # (constant weights), which is what a captured decode loop can use.
     a16, w_bits = synth.config3(16)
@@ -631,7 +632,12 @@ def targets(mxp, synth, peaks):
             st = {"i": 0}
             tot = wbytes + M * K * 2 + M * N * 2
 
-            def run_tc():
+            def run_tc():  # every call names the next one's weights, as a decoder knows its next layer
+                mxp.mxp_gemm_decode_prepacked(a, tiled[st["i"] % 8], out=d, workspace=ws, chained=True,
+                                              next_w=tiled[(st["i"] + 1) % 8])
+                st["i"] += 1
+
+            def run_tc_nohint():
                 mxp.mxp_gemm_decode_prepacked(a, tiled[st["i"] % 8], out=d, workspace=ws, chained=True)
                 st["i"] += 1
 
@@ -639,13 +645,14 @@ def targets(mxp, synth, peaks):
                 mxp.mxp_gemm_decode_chained(a, packed[st["i"] % 8], d)
                 st["i"] += 1
             us_tc = time_loop(graph_of(run_tc, kChain).replay, 6, warmup=2) / kChain * 1e3
+            us_nh = time_loop(graph_of(run_tc_nohint, kChain).replay, 6, warmup=2) / kChain * 1e3
             us_reg = time_loop(graph_of(run_reg, kChain).replay, 6, warmup=2) / kChain * 1e3
-            row["M%d" % M] = {"tc_us": _r(us_tc), "reg_us": _r(us_reg),
-                              "frac": _r(tot / min(us_tc, us_reg) / 1e3 / hbm, 3)}
+            row["M%d" % M] = {"tc_us": _r(us_tc), "tc_nohint_us": _r(us_nh), "reg_us": _r(us_reg),
+                              "frac": _r(tot / min(us_tc, us_nh, us_reg) / 1e3 / hbm, 3)}
         dec[name] = row
         del packed, tiled
-    dec["mx+/mxfp4_M1"] = _r(min(dec["mx+"]["M1"]["tc_us"], dec["mx+"]["M1"]["reg_us"]) /
-                             min(dec["mxfp4"]["M1"]["tc_us"], dec["mxfp4"]["M1"]["reg_us"]), 3)
+    best = lambda e: min(e["tc_us"], e["tc_nohint_us"], e["reg_us"])
+    dec["mx+/mxfp4_M1"] = _r(best(dec["mx+"]["M1"]) / best(dec["mxfp4"]["M1"]), 3)
     out["decode_cfg3"] = dec
     del w
     # ---- the same at M = 1 on a larger weight matrix (14336 x 4096, an 8B model's MLP width):
@@ -662,7 +669,8 @@ def targets(mxp, synth, peaks):
         st = {"i": 0}
 
         def run_big():
-            mxp.mxp_gemm_decode_prepacked(a2, tiled[st["i"] % 8], out=d, workspace=ws, chained=True)
+            mxp.mxp_gemm_decode_prepacked(a2, tiled[st["i"] % 8], out=d, workspace=ws, chained=True,
+                                          next_w=tiled[(st["i"] + 1) % 8])
             st["i"] += 1
         us = time_loop(graph_of(run_big, kChain).replay, 6, warmup=2) / kChain * 1e3
         tot = N2 * K2 * (0.5 + 1 / 32 + (1 / 32 if mode == MXP else 0)) + K2 * 2 + N2 * 2

@@ -390,6 +390,18 @@ mxp_status mxp_gemm_decode_chained(int64_t M, int64_t N, int64_t K, const void *
  *                            not cleared).  M > 16 or unsupported shapes: MXP_ERR_UNSUPPORTED
  *                            (use mxp_gemm).  Same result as mxp_gemm within its bound; one-hot
  *                            activation rows return decoded weights bit for bit.
+ *   mxp_gemm_decode_prepacked_next  the same call with a hint: `next_B_prepacked` (device, the
+ *                            output of mxp_gemm_decode_prepack for any shape, with its size; NULL
+ *                            and 0: no hint) names the weights of the call expected next on this
+ *                            stream, a decoder's next layer.  About a third of a call's time --
+ *                            its last MMAs and stores, the switch to the next call's CTAs, their
+ *                            first copies' latency -- moves no weights; once a CTA's own weights
+ *                            have all but landed it asks for the head of the next call's (what
+ *                            its ring will hold first) to be fetched into L2, from where that
+ *                            call streams them faster than from HBM.  Nothing waits for the
+ *                            fetch and the result does not depend on it; a pointer and size that
+ *                            do not describe readable device memory are the caller's error
+ *                            (alignment and NULL / 0 pairing are checked: MXP_ERR_INVALID_ARG).
  * The paper describes the format and its decode, not this staging.
  */
 size_t mxp_gemm_decode_prepack_bytes(int64_t N, int64_t K, mxp_mode b_mode);
@@ -401,6 +413,13 @@ mxp_status mxp_gemm_decode_prepacked(int64_t M, int64_t N, int64_t K, const void
                                      size_t B_prepacked_bytes, void *D, mxp_dtype d_dt,
                                      int64_t ldd, void *workspace, size_t workspace_bytes,
                                      int chained, void *cuda_stream);
+mxp_status mxp_gemm_decode_prepacked_next(int64_t M, int64_t N, int64_t K,
+                                          const void *A_dense_bf16, int64_t lda, mxp_mode b_mode,
+                                          const void *B_prepacked, size_t B_prepacked_bytes,
+                                          void *D, mxp_dtype d_dt, int64_t ldd, void *workspace,
+                                          size_t workspace_bytes, int chained,
+                                          const void *next_B_prepacked,
+                                          size_t next_B_prepacked_bytes, void *cuda_stream);
 
 /*
  * Reads back (synchronously, after synchronising `cuda_stream`) the status block a GEMM

@@ -25,7 +25,7 @@ BF16 = 1
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxp.so")
 
-EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_decode_prepack_bytes", "mxp_gemm_decode_workspace_bytes", "mxp_gemm_decode_prepack", "mxp_gemm_decode_prepacked", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
+EXPORTS = ["mxp_quantize", "mxp_quantize_reordered", "mxp_channel_order", "mxp_nvfp4_quantize", "mxp_nvfp4_dequantize", "mxp_dequantize", "mxp_gemm", "mxp_gemm_noalloc", "mxp_gemm_decode_chained", "mxp_gemm_decode_prepack_bytes", "mxp_gemm_decode_workspace_bytes", "mxp_gemm_decode_prepack", "mxp_gemm_decode_prepacked", "mxp_gemm_decode_prepacked_next", "mxp_gemm_workspace_bytes", "mxp_gemm_min_workspace_bytes",
            "mxp_gemm_prepack_bytes", "mxp_gemm_prepack_form", "mxp_gemm_prepack", "mxp_gemm_prepacked",
            "mxp_gemm_dense_prepacked", "mxp_gemm_dense_prepacked_workspace_bytes",
            "mxp_quantize_gemm_ready", "mxp_gemm_ready",
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         l.mxp_gemm_decode_prepack.restype = ci
         l.mxp_gemm_decode_prepacked.argtypes = [i64, i64, i64, vp, i64, ci, vp, sz, vp, ci, i64, vp, sz, ci, vp]
         l.mxp_gemm_decode_prepacked.restype = ci
+        l.mxp_gemm_decode_prepacked_next.argtypes = [i64, i64, i64, vp, i64, ci, vp, sz, vp, ci, i64, vp, sz, ci, vp, sz, vp]
+        l.mxp_gemm_decode_prepacked_next.restype = ci
         l.mxp_gemm_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
         l.mxp_gemm_workspace_bytes.restype = sz
         l.mxp_gemm_min_workspace_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
@@ -421,19 +423,27 @@ def mxp_gemm_decode_workspace_bytes(M: int, K: int) -> int:
 
 def mxp_gemm_decode_prepacked(a: torch.Tensor, w: DecodeWeights, out_dtype=torch.bfloat16,
                               out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                              chained: bool = False) -> torch.Tensor:
+                              chained: bool = False, next_w: Optional[DecodeWeights] = None) -> torch.Tensor:
     """D = a @ dec(W).T for 1..16 activation rows on the FP4 tensor path, weights re-tiled by
-    mxp_gemm_decode_prepack.  `chained`: see include/mxp.h."""
+    mxp_gemm_decode_prepack.  `chained`, `next_w` (the weights of the call expected next: a
+    prefetch hint, mxp_gemm_decode_prepacked_next): see include/mxp.h."""
     assert a.dtype == torch.bfloat16 and a.is_cuda and a.stride(1) == 1
     M, N, K = a.shape[0], w.rows, w.cols
     if out is None:
         out = torch.empty((M, N), dtype=out_dtype, device=a.device)
     if workspace is None:
         workspace = torch.zeros(max(256, mxp_gemm_decode_workspace_bytes(M, K)), dtype=torch.uint8, device=a.device)
-    st = lib().mxp_gemm_decode_prepacked(M, N, K, a.data_ptr(), a.stride(0), w.mode, w.buf.data_ptr(),
-                                         w.buf.numel(), out.data_ptr(), _dt(out), out.stride(0),
-                                         workspace.data_ptr(), workspace.numel(), int(chained), _stream())
-    _check("mxp_gemm_decode_prepacked", st)
+    if next_w is None:
+        st = lib().mxp_gemm_decode_prepacked(M, N, K, a.data_ptr(), a.stride(0), w.mode, w.buf.data_ptr(),
+                                             w.buf.numel(), out.data_ptr(), _dt(out), out.stride(0),
+                                             workspace.data_ptr(), workspace.numel(), int(chained), _stream())
+        _check("mxp_gemm_decode_prepacked", st)
+    else:
+        st = lib().mxp_gemm_decode_prepacked_next(M, N, K, a.data_ptr(), a.stride(0), w.mode, w.buf.data_ptr(),
+                                                  w.buf.numel(), out.data_ptr(), _dt(out), out.stride(0),
+                                                  workspace.data_ptr(), workspace.numel(), int(chained),
+                                                  next_w.buf.data_ptr(), next_w.buf.numel(), _stream())
+        _check("mxp_gemm_decode_prepacked_next", st)
     return out
 
 

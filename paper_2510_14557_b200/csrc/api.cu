@@ -339,6 +339,20 @@ mxp_status mxp_gemm_decode_prepacked(int64_t M, int64_t N, int64_t K, const void
                                      void* workspace, size_t workspace_bytes, int chained,
                                      void* cuda_stream)
 {
+    return mxp_gemm_decode_prepacked_next(M, N, K, A_dense_bf16, lda, b_mode, B_prepacked, B_prepacked_bytes,
+                                          D, d_dt, ldd, workspace, workspace_bytes, chained, nullptr, 0,
+                                          cuda_stream);
+}
+
+mxp_status mxp_gemm_decode_prepacked_next(int64_t M, int64_t N, int64_t K, const void* A_dense_bf16,
+                                          int64_t lda, mxp_mode b_mode, const void* B_prepacked,
+                                          size_t B_prepacked_bytes, void* D, mxp_dtype d_dt, int64_t ldd,
+                                          void* workspace, size_t workspace_bytes, int chained,
+                                          const void* next_B_prepacked, size_t next_B_prepacked_bytes,
+                                          void* cuda_stream)
+{
+    if ((next_B_prepacked == nullptr) != (next_B_prepacked_bytes == 0)) return MXP_ERR_INVALID_ARG;
+    if (next_B_prepacked != nullptr && !aligned(next_B_prepacked, 256)) return MXP_ERR_INVALID_ARG;
     if (M < 0 || N < 0 || K < 0 || K % 32 != 0) return MXP_ERR_INVALID_ARG;
     if (!valid_dtype(d_dt) || !valid_mode(b_mode)) return MXP_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return MXP_OK;
@@ -348,7 +362,8 @@ mxp_status mxp_gemm_decode_prepacked(int64_t M, int64_t N, int64_t K, const void
     if (workspace != nullptr && !aligned(workspace, 256)) return MXP_ERR_INVALID_ARG;
     return mxp::launch_gemm_decode_tc(M, N, K, A_dense_bf16, lda, b_mode, B_prepacked,
                                       B_prepacked_bytes, D, d_dt, ldd, workspace, workspace_bytes,
-                                      chained != 0, static_cast<cudaStream_t>(cuda_stream));
+                                      chained != 0, next_B_prepacked, next_B_prepacked_bytes,
+                                      static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t mxp_gemm_prepack_bytes(int64_t rows, int64_t K, int form)

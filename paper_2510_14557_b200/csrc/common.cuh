@@ -60,7 +60,8 @@ mxp_status decode_prepack(const mxp_packed& B, void* out, size_t out_bytes, cuda
 mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
                                  mxp_mode b_mode, const void* b_prepacked, size_t b_prepacked_bytes,
                                  void* D, mxp_dtype d_dt, int64_t ldd, void* workspace,
-                                 size_t workspace_bytes, bool chained, cudaStream_t stream);
+                                 size_t workspace_bytes, bool chained, const void* next_prepacked,
+                                 size_t next_prepacked_bytes, cudaStream_t stream);
 
 // Block-scaled tensor-core form: both operands packed.
 size_t tc_workspace_bytes(int64_t M, int64_t N, int64_t K, mxp_mode a_mode, mxp_mode b_mode);

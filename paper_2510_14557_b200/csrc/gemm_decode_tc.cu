@@ -81,6 +81,8 @@ constexpr int kMaxStages = 16;
 constexpr long long kWaitLimit = 4000000000ll;
 constexpr size_t kSmemMax = 227 * 1024;
 constexpr size_t kActSpread = 116 * 1024;  // shared memory that only one CTA per SM can have
+constexpr int kHintLead = 2;               // images still in flight when the hint for the next call goes out
+constexpr size_t kHintBytes = 192 * 1024;  // what a CTA asks for of the next call's weights (a ring-full)
 constexpr uint32_t kMagic = 0x4D58D0C2u;
 }  // namespace
 constexpr size_t kHeaderBytes = 256;
@@ -224,6 +226,8 @@ struct DecodeParams {
     int clear_status;      // kSelf: this launch clears the status block (no kernel ahead of it does)
     const uint8_t* wimg;   // weight images [cta][tile][stage]
     const uint8_t* aimg;   // activation images [stage] (not kSelf)
+    const uint8_t* next_wimg;  // weight images of the call expected next, or nullptr ...
+    size_t next_share;         // ... and the bytes of them that belong to one CTA of this grid
     void* D;
     int64_t ldd;
     StatusBlock* status;   // may be nullptr
@@ -594,6 +598,23 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 }
                 ptx::mbar_arrive_expect_tx(&full[s], prm.wimg_bytes);
                 bulk_g2s(slot(s), wsrc + (size_t)c * prm.wimg_bytes, prm.wimg_bytes, &full[s]);
+            }
+        }
+        if (prm.next_wimg != nullptr && total > 0u) {
+            // HBM has nothing to do from about here until the next call's CTAs have the SMs and
+            // their first copies are out (~2.5 us of a ~6.8 us call): once all but this CTA's last
+            // two images have landed, ask for the head of the next call's weights into L2, as much
+            // as a CTA's ring holds.  (cp.async.bulk.prefetch.L2: a hint, nothing waits for it.)
+            const uint32_t last = total > (uint32_t)kHintLead ? total - 1u - (uint32_t)kHintLead : 0u;
+            if (lane == 0) ptx::mbar_wait(&full[last % S], (last / S) & 1, abort, kWaitLimit);
+            __syncwarp();
+            const size_t head = prm.next_share < kHintBytes ? prm.next_share : kHintBytes;
+            const size_t piece = (head / 32 + 15) / 16 * 16;  // a lane each
+            const size_t off = (size_t)lane * piece;
+            if (*abort == 0u && piece > 0 && off < head) {
+                const uint8_t* src = prm.next_wimg + (size_t)blockIdx.x * prm.next_share + off;
+                const uint32_t n = (uint32_t)(head - off < piece ? head - off : piece);
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(n) : "memory");
             }
         }
     } else if (warp == 1) {
@@ -1023,7 +1044,7 @@ mxp_status decode_prepack(const mxp_packed& B, void* out, size_t out_bytes, cuda
 mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, mxp_mode b_mode,
                                  const void* b_prepacked, size_t b_prepacked_bytes, void* D, mxp_dtype d_dt,
                                  int64_t ldd, void* workspace, size_t workspace_bytes, bool chained,
-                                 cudaStream_t stream)
+                                 const void* next_prepacked, size_t next_prepacked_bytes, cudaStream_t stream)
 {
     const bool plus = b_mode == MXP_MODE_MXFP4_PLUS;
     DecodePlan p;
@@ -1058,6 +1079,17 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     prm.clear_status = chained ? 0 : 1;
     prm.wimg = static_cast<const uint8_t*>(b_prepacked) + kHeaderBytes;
     prm.aimg = ws + kStatusBytes;
+    // the hint: every CTA asks for the head of "its" share of the weights expected next (with a
+    // CTA on every SM in both calls that share is the next call's CTA's own stream)
+    prm.next_wimg = nullptr;
+    prm.next_share = 0;
+    if (next_prepacked != nullptr && next_prepacked_bytes > kHeaderBytes) {
+        const size_t share = (next_prepacked_bytes - kHeaderBytes) / (size_t)p.ctas / 16 * 16;
+        if (share >= 16) {
+            prm.next_wimg = static_cast<const uint8_t*>(next_prepacked) + kHeaderBytes;
+            prm.next_share = share;
+        }
+    }
     prm.D = D;
     prm.ldd = ldd;
     prm.status = reinterpret_cast<StatusBlock*>(ws);

@@ -146,6 +146,55 @@ def test_decode_prepacked_chained_layers_and_graph():
     assert m.mxp_gemm_status(ws) == 0
 
 
+@pytest.mark.parametrize("M", [1, 2, 5, 16])
+def test_decode_prepacked_with_a_hint_for_the_next_layers_weights(M):
+    # the hint only prefetches: layers of three different shapes and both modes in a chain, each
+    # call naming the next one's weights (the last one none), give bit for bit what the calls
+    # without a hint give; a tiny next matrix (less than a CTA's share) and one whose CTAs are
+    # fewer than the SMs are among them
+    m = mxp()
+    shapes = [(1024, 1024, MXP), (4096, 1024, MX), (1024, 4096, MXP), (40, 1024, MX), (1024, 1024, MXP)]
+    layers = []
+    for i, (N, K, mode) in enumerate(shapes):
+        _, w_bits = synth.config3(1, N, K, seed=40 + i)
+        layers.append(m.mxp_gemm_decode_prepack(m.mxp_quantize(to_dev_bf16(w_bits * 1), mode)))
+    a_bits, _ = synth.config3(M, 32, 1024, seed=2)
+    x0 = to_dev_bf16(a_bits)
+    ws = torch.zeros(m.mxp_gemm_decode_workspace_bytes(M, 4096), dtype=torch.uint8, device="cuda")
+
+    def run(hint):
+        x, outs = x0, []
+        for i, w in enumerate(layers):
+            y = torch.empty((M, w.rows), dtype=torch.bfloat16, device="cuda")
+            nxt = layers[i + 1] if hint and i + 1 < len(layers) else None
+            m.mxp_gemm_decode_prepacked(x[:, :w.cols].contiguous() if x.shape[1] != w.cols else x, w, out=y,
+                                        workspace=ws, next_w=nxt)
+            outs.append(y)
+            x = y if y.shape[1] >= 1024 else x0
+        return outs
+
+    ref = run(False)
+    got = run(True)
+    torch.cuda.synchronize()
+    for a, b in zip(ref, got):
+        assert torch.equal(a, b)
+    assert m.mxp_gemm_status(ws) == 0
+    # pointer without size, size without pointer, misaligned pointer: rejected before any launch
+    lib = m.binding.lib()
+    w, y = layers[0], torch.empty((M, 1024), dtype=torch.bfloat16, device="cuda")
+
+    def call(nptr, nbytes):
+        return lib.mxp_gemm_decode_prepacked_next(M, 1024, 1024, x0.data_ptr(), 1024, MXP, w.buf.data_ptr(),
+                                                  w.buf.numel(), y.data_ptr(), 1, 1024, ws.data_ptr(), ws.numel(), 0,
+                                                  nptr, nbytes, None)
+    assert call(layers[1].buf.data_ptr(), layers[1].buf.numel()) == 0
+    assert call(None, 0) == 0
+    assert call(layers[1].buf.data_ptr(), 0) == 1
+    assert call(None, 4096) == 1
+    assert call(layers[1].buf.data_ptr() + 16, layers[1].buf.numel() - 16) == 1
+    torch.cuda.synchronize()
+
+
 def test_decode_prepacked_argument_checks():
     m = mxp()
     lib = m.binding.lib()
