@@ -161,6 +161,12 @@ struct DecodeLayout {
 };
 constexpr int kSelfMaxM = 3;  // rows the self-converting form takes: three rows' planes fill one 16-row operand tile
 constexpr int kSideSlots = 4;
+// kSelf: bytes between the code tiles of two stages.  The MMA's second group of eight operand
+// rows lies 1024 bytes behind the first (the descriptor's stride).  A single activation row has
+// five planes, so its second group holds nothing the epilogue looks at and may as well be the
+// next stage's first group: a tile then costs 1 KB instead of 2 (plus one tile of room at the
+// end), which lets the MXFP4+ form keep all sixteen stages of K = 4096 in its ring.
+__host__ __device__ constexpr int self_img_bytes(int self_m) { return kPlanes * self_m <= 8 ? 1024 : 2048; }
 __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, int nact, bool plus, int stages,
                                                       int self_nst = 0, int astages = kSideSlots, int self_m = 1)
 {
@@ -174,7 +180,7 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
         const size_t last = (size_t)(stages - 1) * l.slot + 128 * 128;  // (see below)
         size_t o = up(last > (size_t)stages * l.slot ? last : (size_t)stages * l.slot, 1024);
         l.img_codes = o;
-        o += (size_t)self_nst * 2048;
+        o += (size_t)(self_nst + 1) * self_img_bytes(self_m);
         l.img_sf = o;
         o += (size_t)self_nst * 512;
         if (plus) {
@@ -542,7 +548,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 for (int m = 0; m < kSelfRows; ++m) v[m] = fetch(m, cid);
             }
             // the images' unused rows: zero codes under a finite scale (the rows in use land on top)
-            for (int i = cid; i < nst * 128; i += kConv)
+            for (int i = cid; i < (nst + 1) * (self_img_bytes(kSelfRows) / 16); i += kConv)
                 reinterpret_cast<uint4*>(smem + L.img_codes)[i] = make_uint4(0u, 0u, 0u, 0u);
             for (int i = cid; i < nst * 32; i += kConv)
                 reinterpret_cast<uint4*>(smem + L.img_sf)[i] =
@@ -573,7 +579,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
 #pragma unroll
             for (int m = 0; m < kSelfRows; ++m) {
                 if (kPlus) *reinterpret_cast<uint4*>(smem + L.raw + ((size_t)m * nst * kStageK + (size_t)i * 8) * 2) = v[m];
-                convert_quarter(v[m], m, kb, qd, img_codes0 + (uint32_t)st * 2048u, img_sf0 + (uint32_t)st * 512u, kSfb);
+                convert_quarter(v[m], m, kb, qd, img_codes0 + (uint32_t)st * (uint32_t)self_img_bytes(kSelfRows), img_sf0 + (uint32_t)st * 512u, kSfb);
                 v[m] = vn[m];
             }
             i = nxt;
@@ -671,7 +677,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 const uint8_t* sl = slot(s);
                 const uint64_t da = ptx::smem_desc_sw128(ptx::smem_u32(sl));
                 const uint64_t db = ptx::smem_desc_sw128(
-                    ptx::smem_u32(kSelf ? smem + L.img_codes + (size_t)st * 2048 : act_slot(sa)));
+                    ptx::smem_u32(kSelf ? smem + L.img_codes + (size_t)st * self_img_bytes(kSelfRows) : act_slot(sa)));
                 const uint32_t sfa = ptx::smem_u32(sl + (size_t)prm.rows * 128);
                 const uint32_t sfb =
                     ptx::smem_u32(kSelf ? smem + L.img_sf + (size_t)st * 512 : act_slot(sa) + kNact * 128);
@@ -952,9 +958,10 @@ gemm_decode_tc_kernel(const DecodeParams prm)
 
 // Ring slots that fit: a multiple of four (see the issuers), at most sixteen.  self_nst > 0: the
 // form with resident activation images.
-int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0, int astages = kSideSlots, int self_m = 1)
+int pick_stages(const DecodePlan& p, int nact, bool plus, int self_nst = 0, int astages = kSideSlots, int self_m = 1,
+                int most = kMaxStages)
 {
-    for (int s = kMaxStages; s >= 4; s -= 4)
+    for (int s = most; s >= 4; s -= 4)
         if (decode_layout(p.rows, p.wimg, nact, plus, s, self_nst, astages, self_m).total <= kSmemMax) return s;
     return 0;
 }
@@ -1061,7 +1068,13 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     // 8.9 against 9.7 us for two rows, but 10.3 against 9.9 us for three: three rows as given
     // take 24 KB from the ring and triple the BM_L sums' gathers.)
     const bool try_self = M <= (plus ? 2 : kSelfMaxM);
-    const int self_stages = try_self ? pick_stages(p, nact, plus, p.nst, kSideSlots, (int)M) : 0;
+    // (MX+, one row: with all sixteen stages of K = 4096 in the ring a call takes 8.1 us, with
+    // twelve 7.6 us -- the CTAs of a call then finish closer together; why is not understood.
+    // With the next call's weights on their way into L2 it is the other way round, 7.2 against
+    // 7.6 us.  So: twelve unless there is a hint; a CTA with more than sixteen stages needs the
+    // deeper ring either way.)
+    const int most = (plus && M == 1 && next_prepacked == nullptr && p.tiles * p.nst <= kMaxStages) ? 12 : kMaxStages;
+    const int self_stages = try_self ? pick_stages(p, nact, plus, p.nst, kSideSlots, (int)M, most) : 0;
     const bool self = self_stages != 0;
     // The activation ring: eight slots (the images come from L2 with ~1 us of latency: with four,
     // every fourth stage waits for its image) unless that leaves the weight ring fewer than eight.
