@@ -67,9 +67,9 @@ namespace {
 
 constexpr int kIssueWarp0 = 2, kIssuers = 4;
 constexpr int kRowWarp0 = 6;
-constexpr int kResWarp0 = 10, kResWarps = 4, kResGroups = 3;  // BM_L sums: three groups of four warps take turns
-constexpr int kTileWarps = 3, kTileGroups = 4;  // BM_L tiles: the same twelve warps as four groups of three
-constexpr int kWarps = kResWarp0 + kResWarps * kResGroups;
+constexpr int kResWarp0 = 10;  // the first of the twelve warps that handle BM_L
+constexpr int kTileWarps = 3, kTileGroups = 4;  // ... as four groups of three (tiles for M >= 4, sums below)
+constexpr int kWarps = kResWarp0 + kTileWarps * kTileGroups;
 constexpr int kThreads = 32 * kWarps;
 constexpr int kStageK = 256;   // elements of K per stage: 128 bytes of codes per row
 constexpr int kPlanes = 5;     // balanced base-8 digit planes of an activation
@@ -187,7 +187,7 @@ __host__ __device__ inline DecodeLayout decode_layout(int rows, uint32_t wimg, i
             l.raw = o;   // the activation rows as given (bf16), for the BM_L term
             o += (size_t)self_m * (size_t)self_nst * kStageK * 2;
             l.corr = o;  // its sums [group][row m][weight row]
-            o += (size_t)kResGroups * self_m * 128 * sizeof(float);
+            o += (size_t)kTileGroups * self_m * 128 * sizeof(float);
         }
         l.bars = up(o, 16);
         l.total = l.bars + 512 + 1024;  // barriers (under 512 bytes); slack for aligning the base
@@ -480,6 +480,9 @@ gemm_decode_tc_kernel(const DecodeParams prm)
     static_assert(384 + (2 * kMaxStages + 2 * kSideSlots) * 8 <= 1024, "barriers of the three-ring form");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // kSelf, MX+: the twelve BM_L warps as four groups of three (a thread per weight row, up to 96)
+    // or, for taller tiles, three groups of four
+    const int sum_warps = prm.rows <= 32 * kTileWarps ? kTileWarps : 4, sum_groups = 12 / sum_warps;
     auto slot = [&](int s) { return smem + (size_t)s * L.slot; };
     auto act_slot = [&](int sa) { return smem + L.act0 + (size_t)sa * L.aslot; };
     auto res_slot = [&](int sr) { return smem + L.res0 + (size_t)sr * L.rslot; };
@@ -514,7 +517,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 ptx::mbar_init(&aempty[lane], 1);
             }
             ptx::mbar_init(&full[lane], 1);
-            ptx::mbar_init(&empty[lane], !kPlus ? 1 : kSelf ? 1 + kResWarps : 1 + kTileWarps);  // + the warps that read its records
+            ptx::mbar_init(&empty[lane], !kPlus ? 1 : kSelf ? 1 + sum_warps : 1 + kTileWarps);  // + the warps that read its records
         } else if (lane < kMaxStages + kSideSlots) {
             if (!kSelf) {
                 ptx::mbar_init(&res_full[lane - kMaxStages], kTileWarps);
@@ -523,7 +526,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         } else if (lane == kMaxStages + kSideSlots) {
             ptx::mbar_init(acc_full, kIssuers);
             ptx::mbar_init(acc_empty, 4);
-            ptx::mbar_init(corr_full, kResWarps * kResGroups);
+            ptx::mbar_init(corr_full, kTileWarps * kTileGroups);
             ptx::mbar_init(corr_empty, 4);
             *abort = 0u;
         }
@@ -792,7 +795,7 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 for (int m = 0; m < kSelfRows; ++m) {
                     float c = 0.f;
 #pragma unroll
-                    for (int g = 0; g < kResGroups; ++g) c += corr[(g * kSelfRows + m) * 128 + row];  // fixed order
+                    for (int g = 0; g < sum_groups; ++g) c += corr[(g * kSelfRows + m) * 128 + row];  // fixed order
                     o[m] += c;
                 }
                 __syncwarp();
@@ -813,20 +816,24 @@ gemm_decode_tc_kernel(const DecodeParams prm)
         }
     } else if (kPlus && kSelf) {
         // ---------------------------------------------------------------- BM_L on the CUDA cores
-        // Group g of four warps takes the stages whose running number is g (mod 3); thread = weight
-        // row.  A stage gives a row eight record bytes (BM position | BM_L code << 5 | sign << 7)
-        // and eight scale bytes: eight weights (BM_L 2^shared_exp), eight activations fetched
-        // independently of one another, eight FMAs per activation row.  No branch: an absent
-        // BM_L is a zero weight.
-        const int grp = (warp - kResWarp0) / kResWarps;
-        const int r = (int)threadIdx.x - 32 * (kResWarp0 + grp * kResWarps);
+        // Group g of three warps takes the stages whose running number is g (mod 4); thread =
+        // weight row (tiles of more than 96 rows: three groups of four warps).  A stage gives a row eight
+        // record bytes (BM position | BM_L code << 5 | sign << 7) and eight scale bytes: eight
+        // weights (BM_L 2^shared_exp), eight activations fetched independently of one another,
+        // eight FMAs per activation row.  No branch: an absent BM_L is a zero weight.
+        // (The sums are bound by instruction issue, ~160 per row and stage.  Three groups of four
+        // warps, a thread per row of up to 128, left the fourth warp of every group without rows
+        // at config 3's 75 and one of the SM's four schedulers without work: 0.65 us per stage
+        // and group, the last group done 1.3 us after the MMAs.)
+        const int grp = (warp - kResWarp0) / sum_warps;
+        const int r = (int)threadIdx.x - 32 * (kResWarp0 + grp * sum_warps);
         const uint32_t raw_sa = ptx::smem_u32(smem + L.raw), slot0_sa = ptx::smem_u32(smem), slot_bytes = (uint32_t)L.slot;
         const uint32_t so = (uint32_t)(r & 31) * 16u + (uint32_t)(r >> 5) * 4u;
         bool ok = true;
         for (int t = 0; t < ntl && ok; ++t) {
             float acc[kSelfRows] = {};
-            const int first = (grp + 3 * kResGroups - (int)(((uint32_t)t * (uint32_t)nst) % kResGroups)) % kResGroups;
-            for (int st = first; st < nst; st += kResGroups) {
+            const int first = (grp + 12 - (int)(((uint32_t)t * (uint32_t)nst) % (uint32_t)sum_groups)) % sum_groups;
+            for (int st = first; st < nst; st += sum_groups) {
                 const uint32_t c = (uint32_t)t * (uint32_t)nst + (uint32_t)st;
                 const int s = c % S;
                 if (!ptx::mbar_wait(&full[s], (c / S) & 1, abort, kWaitLimit)) {
@@ -834,38 +841,40 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                     ok = false;
                     break;
                 }
-                if (r < prm.rows) {
-                    // (loads that name the shared window: as generic loads through pointers the
-                    // compiler cannot place, each costs 64-bit address arithmetic and more latency)
-                    const uint32_t atoms = slot0_sa + (uint32_t)s * slot_bytes + (uint32_t)prm.rows * 128u;
-                    uint2 rec;
-                    uint32_t sc_lo, sc_hi;
-                    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(rec.x), "=r"(rec.y) : "r"(atoms + 2u * kAtom + (uint32_t)r * 8u) : "memory");
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc_lo) : "r"(atoms + so) : "memory");
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc_hi) : "r"(atoms + kAtom + so) : "memory");
-                    float w[8];
-                    uint32_t k[8];
+                {
+                    if (r < prm.rows) {
+                        // (loads that name the shared window: as generic loads through pointers the
+                        // compiler cannot place, each costs 64-bit address arithmetic and more latency)
+                        const uint32_t atoms = slot0_sa + (uint32_t)s * slot_bytes + (uint32_t)prm.rows * 128u;
+                        uint2 rec;
+                        uint32_t sc_lo, sc_hi;
+                        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(rec.x), "=r"(rec.y) : "r"(atoms + 2u * kAtom + (uint32_t)r * 8u) : "memory");
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc_lo) : "r"(atoms + so) : "memory");
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(sc_hi) : "r"(atoms + kAtom + so) : "memory");
+                        float w[8];
+                        uint32_t k[8];
 #pragma unroll
-                    for (int kb = 0; kb < 8; ++kb) {
-                        const uint32_t b = ((kb < 4 ? rec.x : rec.y) >> (8 * (kb & 3))) & 255u;
-                        const uint32_t sc = ((kb < 4 ? sc_lo : sc_hi) >> (8 * (kb & 3))) & 255u;
-                        // BM_L 2^(sc - 127) = (code / 2) 2^(sc - 127), the sign from the record
-                        const float mag = (float)((b >> 5) & 3u) * 0.5f * __uint_as_float(sc << 23);
-                        w[kb] = __uint_as_float(__float_as_uint(mag) | ((b & 0x80u) << 24));
-                        k[kb] = raw_sa + 2u * ((uint32_t)st * kStageK + (uint32_t)kb * 32u + (b & 31u));
-                    }
+                        for (int kb = 0; kb < 8; ++kb) {
+                            const uint32_t b = ((kb < 4 ? rec.x : rec.y) >> (8 * (kb & 3))) & 255u;
+                            const uint32_t sc = ((kb < 4 ? sc_lo : sc_hi) >> (8 * (kb & 3))) & 255u;
+                            // BM_L 2^(sc - 127) = (code / 2) 2^(sc - 127), the sign from the record
+                            const float mag = (float)((b >> 5) & 3u) * 0.5f * __uint_as_float(sc << 23);
+                            w[kb] = __uint_as_float(__float_as_uint(mag) | ((b & 0x80u) << 24));
+                            k[kb] = raw_sa + 2u * ((uint32_t)st * kStageK + (uint32_t)kb * 32u + (b & 31u));
+                        }
 #pragma unroll
-                    for (int m = 0; m < kSelfRows; ++m) {
-                        if (m < prm.M) {
-                            float a[8];
+                        for (int m = 0; m < kSelfRows; ++m) {
+                            if (m < prm.M) {
+                                float a[8];
 #pragma unroll
-                            for (int kb = 0; kb < 8; ++kb) {
-                                uint32_t h;
-                                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(h) : "r"(k[kb] + 2u * (uint32_t)(m * nst * kStageK)) : "memory");
-                                a[kb] = __uint_as_float(h << 16);
+                                for (int kb = 0; kb < 8; ++kb) {
+                                    uint32_t hw;
+                                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hw) : "r"(k[kb] + 2u * (uint32_t)(m * nst * kStageK)) : "memory");
+                                    a[kb] = __uint_as_float(hw << 16);
+                                }
+#pragma unroll
+                                for (int kb = 0; kb < 8; ++kb) acc[m] = fmaf(w[kb], a[kb], acc[m]);
                             }
-#pragma unroll
-                            for (int kb = 0; kb < 8; ++kb) acc[m] = fmaf(w[kb], a[kb], acc[m]);
                         }
                     }
                 }
@@ -878,10 +887,13 @@ gemm_decode_tc_kernel(const DecodeParams prm)
                 if (lane == 0) report(prm.status, abort, 0x7A00);
                 break;
             }
-            float* corr = reinterpret_cast<float*>(smem + L.corr) +
-                          (size_t)grp * kSelfRows * 128;
+            float* corr = reinterpret_cast<float*>(smem + L.corr) + (size_t)grp * kSelfRows * 128;
+            // this group's share, zeros included; with three warps the rows from 96 on hold no weights
 #pragma unroll
-            for (int m = 0; m < kSelfRows; ++m) corr[m * 128 + r] = acc[m];  // this group's share, zeros included
+            for (int m = 0; m < kSelfRows; ++m) {
+                corr[m * 128 + r] = acc[m];
+                if (sum_warps == kTileWarps && r < 32) corr[m * 128 + 96 + r] = 0.f;
+            }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&corr_full[0]);
         }
@@ -1096,7 +1108,9 @@ mxp_status launch_gemm_decode_tc(int64_t M, int64_t N, int64_t K, const void* A,
     // CTA on every SM in both calls that share is the next call's CTA's own stream)
     prm.next_wimg = nullptr;
     prm.next_share = 0;
-    if (next_prepacked != nullptr && next_prepacked_bytes > kHeaderBytes) {
+    // (two self-converted rows against MX+ weights are the one case measured slower with it: 8.85
+    // against 8.47 us)
+    if (next_prepacked != nullptr && next_prepacked_bytes > kHeaderBytes && !(self && plus && M > 1)) {
         const size_t share = (next_prepacked_bytes - kHeaderBytes) / (size_t)p.ctas / 16 * 16;
         if (share >= 16) {
             prm.next_wimg = static_cast<const uint8_t*>(next_prepacked) + kHeaderBytes;
