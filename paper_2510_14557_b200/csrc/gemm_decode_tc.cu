@@ -40,7 +40,7 @@
 //     built without a branch and the eight activations fetched by independent loads (a form
 //     with a thread per (row, block) and the loads behind one another was ~3x slower and lost
 //     to the extra MMAs).  No BM_L tile is built and the MMA count per stage is that of plain
-//     MXFP4; the epilogue adds the three groups' partial sums in a fixed order.
+//     MXFP4; the epilogue adds the groups' partial sums in a fixed order.
 //   * Set-up order (each step measured with per-phase time stamps): warp 0 initialises the
 //     barriers, a lane per ring slot, and issues the first ring-full of weight copies; sixteen
 //     bulk-copy instructions take that warp ~0.5 us, so it only arrives at the set-up barrier
@@ -52,8 +52,11 @@
 //     accumulator of its own), warps 6-9 drain the accumulators, warps 10-21 handle BM_L:
 //     for M >= 2 they build the BM_L operand tiles (four groups of three, group g owning slot g
 //     of the tile ring: one group needs ~1 us per stage, the stream delivers one every
-//     0.26 us), for M = 1 they sum the term themselves (three groups of four, a stage each in
-//     turn).
+//     0.26 us), for self-converted rows they sum the term themselves (the same grouping where
+//     a tile has at most 96 rows, else three groups of four; a stage each in turn).
+//   * A call may name the weights of the call expected next: once its own have all but
+//     landed, a CTA asks for the head of its share of them into L2 (the last MMAs, the switch
+//     to the next call's CTAs and their first copies' latency move no weights otherwise).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
