@@ -742,7 +742,8 @@ def targets(mxp, synth, peaks):
     del flush
     best_dec = min(out["decode_cfg3"][m]["M%d" % M_]["frac"] for m in ("mx+", "mxfp4") for M_ in (1, 8, 16))
     out["goals"] = {"quantize>=0.70_hbm": out["quantize_cfg2"]["mx+"]["frac"] >= 0.70,
-                    "decode>=0.60_hbm": best_dec >= 0.60,
+                    "decode>=0.60_hbm": best_dec >= 0.60,   # every M of config 3, both formats
+                    "decode_M1>=0.60_hbm": {m: out["decode_cfg3"][m]["M1"]["frac"] >= 0.60 for m in ("mxfp4", "mx+")},
                     "prefill_mx+>=0.50_fp4": out["prefill_cfg5"]["A+"]["frac_fp4"] >= 0.50,
                     "prefill_both>=0.50_fp4": out["prefill_cfg5"]["both"]["frac_fp4"] >= 0.50,
                     "mx+_within_1.15x_plain": {"quantize": out["quantize_cfg2"]["mx+/mxfp4"] <= 1.15,
